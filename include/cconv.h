@@ -1,0 +1,142 @@
+/*
+ * cconv -- communication-optimal direct convolution for NVIDIA B200 (sm_100a).
+ *
+ * C ABI of the library built from paper_1802_06905_b200/csrc (libcconv.so).
+ *
+ * The operation is the seven-nested-loop CNN of Demmel & Dinh, "Communication-Optimal
+ * Convolutional Neural Nets" (Eq. 1, Section 2):
+ *
+ *     for b<B, c<C, k<K, w<W, h<H, r<R, s<S:
+ *         Out(k,h,w,b) += Image(r + sw*w, s + sh*h, c, b) * Filter(k,r,s,c)
+ *
+ * with Out starting from zero (the library overwrites Out).  It is a cross-correlation (the filter
+ * is not flipped), without padding, dilation, groups or bias.
+ *
+ * Array layout (the paper gives subscripts only; this ABI fixes dense row-major storage with the
+ * LAST subscript fastest):
+ *     Image  [Wi][Hi][C][B]   bf16,  Wi = sw*(W-1)+R,  Hi = sh*(H-1)+S  (valid-window extent)
+ *     Filter [K][R][S][C]     bf16
+ *     Out    [K][H][W][B]     bf16 or fp32 (h before w; Image is indexed w-direction first)
+ * r runs along the first Image subscript (w-direction), s along the second (h-direction).
+ * Products are accumulated in fp32.  Out is either that fp32 sum (CCONV_OUT_F32) or the sum
+ * rounded once to bf16, nearest even (CCONV_OUT_BF16: one word size for all three arrays, as in
+ * the paper's cost model).
+ *
+ * Ownership: the caller owns Image, Filter and Out.  Unless a function says "host", they are
+ * DEVICE pointers on the plan's device, 16-byte aligned, and Out must not overlap the inputs.
+ * The library keeps no caller pointer after a call returns.  Device calls are asynchronous on the
+ * given stream and never synchronise it.
+ *
+ * Errors: every function returns CCONV_OK (0) or a negative code; nothing throws, aborts or traps.
+ * All positive loop bounds are accepted, also those outside the paper's assumptions
+ * (sw <= R, sh <= S, R <= sw*W, S <= sh*H); the result is still Eq. 1.
+ */
+#ifndef CCONV_H_
+#define CCONV_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define CCONV_OK 0
+#define CCONV_EINVAL (-1)          /* null pointer, non-positive bound, misaligned pointer      */
+#define CCONV_EUNSUPPORTED (-2)    /* requested variant cannot run this shape / this device     */
+#define CCONV_ECUDA (-3)           /* a CUDA call failed; see cconv_last_cuda_error()           */
+#define CCONV_EDEVICE_TIMEOUT (-4) /* a bounded device-side wait expired (kernel bug guard)     */
+#define CCONV_ENOMEM (-5)
+
+/* Kernel variants (cconv_plan_create's `variant`). */
+#define CCONV_VARIANT_AUTO 0
+#define CCONV_VARIANT_SIMT 1 /* CUDA-core kernel: any shape, any alignment                      */
+#define CCONV_VARIANT_HALO 2 /* TMA halo tiles -> tcgen05.mma -> TMEM; needs B%32==0, C%8==0    */
+
+/* Element type of Out (cconv_plan_create's `out_dtype`). */
+#define CCONV_OUT_BF16 0
+#define CCONV_OUT_F32 1
+
+typedef struct cconv_plan cconv_plan; /* opaque; created and destroyed by the library */
+
+typedef struct {
+  /* Theorem 1 at M_words: the five terms in the paper's order, their maximum and its index 1..5 */
+  double term[5];
+  double bound_words;
+  int bound_argmax;
+  double M_words;
+  /* Continuous optimum of the Section-5 tiling LP at M_words: block sizes in the order
+   * b_b, b_c, b_k, b_w, b_h, b_r', b_r'', b_s', b_s''; G = their product; lp_words = F*M/G. */
+  double lp_tile[9];
+  double lp_G;
+  double lp_words;
+  /* The integer tile the kernel runs (0 where a variant has no such notion). */
+  int variant;
+  int out_dtype;
+  int bb, bc, bk, bw, bh; /* batch, channel (per pipeline stage), out-channel, w, h block sizes */
+  int halo_w, halo_h;     /* Image block extent: sw*(bw-1)+R, sh*(bh-1)+S                       */
+  int stages;             /* shared-memory ring depth                                           */
+  int grid;               /* CTAs launched (persistent kernel: <= SM count)                     */
+  int tiles;              /* output tiles in total                                              */
+  int smem_bytes;         /* dynamic shared memory per CTA                                      */
+  int tmem_cols;          /* tensor-memory columns allocated per CTA                            */
+  /* Exact traffic the integer tiling implies, in words (bf16 elements):
+   * fast-memory level = shared memory of one CTA; slow side = L2/HBM. */
+  double tile_words_smem; /* words staged into shared memory over the whole problem + Out words */
+  double compulsory_words; /* |Image| + |Filter| + |Out| with the real Image extent             */
+} cconv_plan_info;
+
+/* Theorem 1 (Section 4.1): the five lower-bound terms, in words, for a fast memory of M_words.
+ * Pure host arithmetic.  terms_out[0..4] = BKWH, sw*sh*BCWH, CKRS, BCKWHRS/M, BCKWH*sqrt(RS*sw*sh/M).
+ * Returns CCONV_EINVAL for non-positive arguments. */
+int cconv_lower_bound(int B, int C, int K, int W, int H, int R, int S, int sw, int sh,
+                      double M_words, double terms_out[5]);
+
+/* Section 5 tiling LP (maximise the sum of log_M block sizes subject to the block-fits-in-M
+ * constraints), solved at the concrete parameters with a dense simplex.  Pure host.
+ * tiles_out: b_b,b_c,b_k,b_w,b_h,b_r',b_r'',b_s',b_s'' (real numbers >= 1); *G_out their product;
+ * *words_out = B*C*K*W*H*R*S * M / G.  pooling != 0 drops the Filter constraint (Section 6). */
+int cconv_tiling_lp(int B, int C, int K, int W, int H, int R, int S, int sw, int sh,
+                    double M_words, int pooling, double tiles_out[9], double* G_out,
+                    double* words_out);
+
+/* Plan: evaluate the bound, solve the LP, pick a hardware-legal tile and kernel variant for
+ * `device`, and build the TMA descriptors' shape data.  M_words <= 0 means "the shared memory one
+ * CTA can use, in bf16 words".  variant: CCONV_VARIANT_*; out_dtype: CCONV_OUT_*.  device >= 0 is a
+ * CUDA ordinal (a small device status word is allocated there); device = -1 plans for a nominal
+ * B200 without any CUDA call, for inspection only (forward calls on such a plan return EINVAL).
+ * The plan is immutable afterwards and may be used from any stream of that device, one launch at a
+ * time per plan (launches of one plan share its status word). */
+int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, int R, int S,
+                      int sw, int sh, int device, double M_words, int variant, int out_dtype);
+int cconv_plan_info_get(const cconv_plan* plan, cconv_plan_info* info_out);
+void cconv_plan_destroy(cconv_plan* plan);
+
+/* Eq. 1 on device buffers (layouts above), asynchronous on `cuda_stream` (a cudaStream_t, may be
+ * NULL for the default stream).  Launch errors are returned; device-side guards are read back by
+ * cconv_plan_status. */
+int cconv_forward_planned(const cconv_plan* plan, const void* Image, const void* Filter, void* Out,
+                          void* cuda_stream);
+
+/* Convenience: plan (cached per shape, device and out_dtype; variant AUTO) and launch on the
+ * current device. */
+int cconv_forward(const void* Image, const void* Filter, void* Out, int B, int C, int K, int W,
+                  int H, int R, int S, int sw, int sh, int out_dtype, void* cuda_stream);
+
+/* Eq. 1 on HOST buffers (same layouts; pinned memory gives true asynchronous copies): copies Image
+ * and Filter to device staging buffers owned by the plan (allocated on first use), launches, copies
+ * Out back, all on `cuda_stream`, then synchronises that stream.  Returns the device status too. */
+int cconv_forward_host(cconv_plan* plan, const void* hImage, const void* hFilter, void* hOut,
+                       void* cuda_stream);
+
+/* Synchronises `cuda_stream`, reads the plan's device status word and clears it.  Returns CCONV_OK,
+ * CCONV_EDEVICE_TIMEOUT (and *detail_out = bit mask of the waits that expired) or CCONV_ECUDA. */
+int cconv_plan_status(const cconv_plan* plan, void* cuda_stream, int* detail_out);
+
+const char* cconv_strerror(int code);
+const char* cconv_last_cuda_error(void); /* message of the last failed CUDA call on this thread */
+int cconv_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CCONV_H_ */

@@ -9,8 +9,8 @@ from .synth import CONFIGS, ConvShape, make_inputs  # noqa: F401
 
 def __getattr__(name):
     # Lazy so that the seeded input generators can be imported without the native library.
-    if name in ("binding", "conv_forward", "lower_bound", "Plan", "library_path", "load_library",
-                "CconvError"):
-        from . import binding
-        return binding if name == "binding" else getattr(binding, name)
+    if name in ("conv_forward", "lower_bound", "tiling_lp", "Plan", "library_path",
+                "load_library", "CconvError"):
+        import importlib
+        return getattr(importlib.import_module(__name__ + ".binding"), name)
     raise AttributeError(name)

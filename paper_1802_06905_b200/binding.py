@@ -1,0 +1,214 @@
+"""ctypes binding of ``libcconv.so`` -- argument marshalling only; every step runs in the library.
+
+Function names mirror the C ABI (``include/cconv.h``).  Tensors are torch CUDA tensors of dtype
+``bfloat16`` in the layouts of Eq. 1 / Section 2:
+    Image  [Wi][Hi][C][B], Filter [K][R][S][C], Out [K][H][W][B]   (last subscript fastest).
+PyTorch supplies device memory and streams; nothing is computed with it.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libcconv.so")
+_lib = None
+
+OK = 0
+EINVAL, EUNSUPPORTED, ECUDA, EDEVICE_TIMEOUT, ENOMEM = -1, -2, -3, -4, -5
+VARIANT_AUTO, VARIANT_SIMT, VARIANT_HALO = 0, 1, 2
+OUT_BF16, OUT_F32 = 0, 1
+
+EXPORTS = (
+    "cconv_lower_bound", "cconv_tiling_lp", "cconv_plan_create", "cconv_plan_info_get",
+    "cconv_plan_destroy", "cconv_forward_planned", "cconv_forward", "cconv_forward_host",
+    "cconv_plan_status", "cconv_strerror", "cconv_last_cuda_error", "cconv_version",
+)
+
+
+class CconvError(RuntimeError):
+    def __init__(self, code, where):
+        lib = load_library()
+        msg = lib.cconv_strerror(code).decode()
+        if code == ECUDA:
+            msg += ": " + lib.cconv_last_cuda_error().decode()
+        super().__init__(f"{where}: {msg} ({code})")
+        self.code = code
+
+
+class PlanInfo(ctypes.Structure):
+    _fields_ = [
+        ("term", ctypes.c_double * 5), ("bound_words", ctypes.c_double),
+        ("bound_argmax", ctypes.c_int), ("M_words", ctypes.c_double),
+        ("lp_tile", ctypes.c_double * 9), ("lp_G", ctypes.c_double), ("lp_words", ctypes.c_double),
+        ("variant", ctypes.c_int), ("out_dtype", ctypes.c_int),
+        ("bb", ctypes.c_int), ("bc", ctypes.c_int), ("bk", ctypes.c_int), ("bw", ctypes.c_int),
+        ("bh", ctypes.c_int), ("halo_w", ctypes.c_int), ("halo_h", ctypes.c_int),
+        ("stages", ctypes.c_int), ("grid", ctypes.c_int), ("tiles", ctypes.c_int),
+        ("smem_bytes", ctypes.c_int), ("tmem_cols", ctypes.c_int),
+        ("tile_words_smem", ctypes.c_double), ("compulsory_words", ctypes.c_double),
+    ]
+
+    def asdict(self):
+        out = {}
+        for name, _ in self._fields_:
+            v = getattr(self, name)
+            out[name] = list(v) if hasattr(v, "__len__") else v
+        return out
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def load_library():
+    """Load libcconv.so; raises loudly when it has not been built (there is no fallback)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise RuntimeError(
+            f"{_LIB_PATH} is missing: build it with `python -m paper_1802_06905_b200.build` "
+            "(nvcc, sm_100a).  There is no CPU fallback.")
+    lib = ctypes.CDLL(_LIB_PATH)
+    i, d, vp = ctypes.c_int, ctypes.c_double, ctypes.c_void_p
+    dp = ctypes.POINTER(ctypes.c_double)
+    nine = [i] * 9
+    lib.cconv_lower_bound.restype = i
+    lib.cconv_lower_bound.argtypes = nine + [d, dp]
+    lib.cconv_tiling_lp.restype = i
+    lib.cconv_tiling_lp.argtypes = nine + [d, i, dp, dp, dp]
+    lib.cconv_plan_create.restype = i
+    lib.cconv_plan_create.argtypes = [ctypes.POINTER(vp)] + nine + [i, d, i, i]
+    lib.cconv_plan_info_get.restype = i
+    lib.cconv_plan_info_get.argtypes = [vp, ctypes.POINTER(PlanInfo)]
+    lib.cconv_plan_destroy.restype = None
+    lib.cconv_plan_destroy.argtypes = [vp]
+    lib.cconv_forward_planned.restype = i
+    lib.cconv_forward_planned.argtypes = [vp, vp, vp, vp, vp]
+    lib.cconv_forward.restype = i
+    lib.cconv_forward.argtypes = [vp, vp, vp] + nine + [i, vp]
+    lib.cconv_forward_host.restype = i
+    lib.cconv_forward_host.argtypes = [vp, vp, vp, vp, vp]
+    lib.cconv_plan_status.restype = i
+    lib.cconv_plan_status.argtypes = [vp, vp, ctypes.POINTER(i)]
+    lib.cconv_strerror.restype = ctypes.c_char_p
+    lib.cconv_strerror.argtypes = [i]
+    lib.cconv_last_cuda_error.restype = ctypes.c_char_p
+    lib.cconv_version.restype = i
+    _lib = lib
+    return lib
+
+
+def _check(code, where):
+    if code != OK:
+        raise CconvError(code, where)
+
+
+def lower_bound(B, C, K, W, H, R, S, sw, sh, M_words):
+    """cconv_lower_bound: the five terms of Theorem 1 (host arithmetic inside the library)."""
+    t = (ctypes.c_double * 5)()
+    _check(load_library().cconv_lower_bound(B, C, K, W, H, R, S, sw, sh, float(M_words), t),
+           "cconv_lower_bound")
+    return list(t)
+
+
+def tiling_lp(B, C, K, W, H, R, S, sw, sh, M_words, pooling=False):
+    """cconv_tiling_lp: (tiles[9], G, words) of the Section-5 LP."""
+    t = (ctypes.c_double * 9)()
+    G, wd = ctypes.c_double(), ctypes.c_double()
+    _check(load_library().cconv_tiling_lp(B, C, K, W, H, R, S, sw, sh, float(M_words),
+                                          int(bool(pooling)), t, ctypes.byref(G), ctypes.byref(wd)),
+           "cconv_tiling_lp")
+    return list(t), G.value, wd.value
+
+
+def _stream_ptr(stream):
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def _tensor_args(image, filt, out, dims, out_dtype=OUT_BF16):
+    import torch
+    B, C, K, W, H, R, S, sw, sh = dims
+    exp = ((sw * (W - 1) + R, sh * (H - 1) + S, C, B), (K, R, S, C), (K, H, W, B))
+    dts = (torch.bfloat16, torch.bfloat16, torch.float32 if out_dtype == OUT_F32 else torch.bfloat16)
+    for name, t, shp, dt in zip(("Image", "Filter", "Out"), (image, filt, out), exp, dts):
+        if not (t.is_cuda and t.dtype == dt and t.is_contiguous()):
+            raise ValueError(f"{name} must be a contiguous CUDA {dt} tensor")
+        if tuple(t.shape) != shp:
+            raise ValueError(f"{name} shape {tuple(t.shape)} != {shp}")
+    return (ctypes.c_void_p(image.data_ptr()), ctypes.c_void_p(filt.data_ptr()),
+            ctypes.c_void_p(out.data_ptr()))
+
+
+class Plan:
+    """Owner of a ``cconv_plan`` handle."""
+
+    def __init__(self, B, C, K, W, H, R, S, sw=1, sh=1, device=0, M_words=0.0,
+                 variant=VARIANT_AUTO, out_dtype=OUT_BF16):
+        self._lib = load_library()
+        self.dims = (B, C, K, W, H, R, S, sw, sh)
+        self.out_dtype = int(out_dtype)
+        self._h = ctypes.c_void_p()
+        _check(self._lib.cconv_plan_create(ctypes.byref(self._h), *self.dims, int(device),
+                                           float(M_words), int(variant), self.out_dtype),
+               "cconv_plan_create")
+
+    def info(self) -> dict:
+        pi = PlanInfo()
+        _check(self._lib.cconv_plan_info_get(self._h, ctypes.byref(pi)), "cconv_plan_info_get")
+        return pi.asdict()
+
+    def forward(self, image, filt, out, stream=None):
+        """cconv_forward_planned on torch CUDA tensors; asynchronous on ``stream``."""
+        pi, pf, po = _tensor_args(image, filt, out, self.dims, self.out_dtype)
+        _check(self._lib.cconv_forward_planned(self._h, pi, pf, po, _stream_ptr(stream)),
+               "cconv_forward_planned")
+        return out
+
+    def forward_ptrs(self, image_ptr, filt_ptr, out_ptr, stream_ptr):
+        """cconv_forward_planned on raw device addresses (the benchmark's inner loop)."""
+        return self._lib.cconv_forward_planned(self._h, image_ptr, filt_ptr, out_ptr, stream_ptr)
+
+    def forward_host(self, h_image, h_filt, h_out, stream=None):
+        """cconv_forward_host on CPU tensors (pinned for asynchronous copies); synchronises."""
+        _check(self._lib.cconv_forward_host(self._h, ctypes.c_void_p(h_image.data_ptr()),
+                                            ctypes.c_void_p(h_filt.data_ptr()),
+                                            ctypes.c_void_p(h_out.data_ptr()), _stream_ptr(stream)),
+               "cconv_forward_host")
+        return h_out
+
+    def status(self, stream=None):
+        """cconv_plan_status: synchronises and returns (code, detail bit mask)."""
+        detail = ctypes.c_int(0)
+        code = self._lib.cconv_plan_status(self._h, _stream_ptr(stream), ctypes.byref(detail))
+        return code, detail.value
+
+    def check(self, stream=None):
+        code, detail = self.status(stream)
+        if code != OK:
+            raise CconvError(code, f"cconv_plan_status (detail={detail:#x})")
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h:
+            self._lib.cconv_plan_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def conv_forward(image, filt, out, B, C, K, W, H, R, S, sw=1, sh=1, out_dtype=OUT_BF16,
+                 stream=None):
+    """cconv_forward: plan (cached per shape) and launch; asynchronous on ``stream``."""
+    dims = (B, C, K, W, H, R, S, sw, sh)
+    pi, pf, po = _tensor_args(image, filt, out, dims, out_dtype)
+    _check(load_library().cconv_forward(pi, pf, po, *dims, int(out_dtype), _stream_ptr(stream)),
+           "cconv_forward")
+    return out

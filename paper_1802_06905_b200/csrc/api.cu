@@ -1,0 +1,437 @@
+// C ABI of libcconv (declared in include/cconv.h): argument checking, plans, TMA descriptors,
+// launches.  No compute happens on the host; there is no CPU fallback.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <map>
+#include <mutex>
+#include <string>
+#include <tuple>
+
+#include "../../include/cconv.h"
+#include "kernels.h"
+#include "planner.h"
+
+using namespace cconv;
+
+namespace {
+
+thread_local std::string g_last_cuda_error;
+
+int cuda_fail(cudaError_t e, const char* what) {
+  g_last_cuda_error = std::string(what) + ": " + cudaGetErrorString(e);
+  return CCONV_ECUDA;
+}
+#define CCONV_CUDA(call)                                  \
+  do {                                                    \
+    cudaError_t e_ = (call);                              \
+    if (e_ != cudaSuccess) return cuda_fail(e_, #call);   \
+  } while (0)
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver is reached through the runtime so that the library loads on machines without one.
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) !=
+            cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
+int env_int(const char* name, int dflt) {
+  const char* v = std::getenv(name);
+  return (v && *v) ? std::atoi(v) : dflt;
+}
+
+}  // namespace
+
+struct cconv_plan {
+  Dims d{};
+  int device = -1;
+  int variant = CCONV_VARIANT_SIMT;
+  int out_dtype = CCONV_OUT_BF16;
+  Machine m{};
+  double M_words = 0;
+  double terms[5] = {0, 0, 0, 0, 0};
+  double lp_tile[9] = {0};
+  double lp_G = 0, lp_words = 0;
+  HaloTile tile{};
+  HaloKernelParams kp{};
+  int* d_status = nullptr;
+  // host-buffer entry point: device staging owned by the plan
+  void* st_image = nullptr;
+  void* st_filter = nullptr;
+  void* st_out = nullptr;
+  // tensor maps are rebuilt only when the base pointers change
+  mutable std::mutex mu;
+  mutable const void* tm_image_ptr = nullptr;
+  mutable const void* tm_filter_ptr = nullptr;
+  mutable CUtensorMap tm_image{};
+  mutable CUtensorMap tm_filter{};
+};
+
+namespace {
+
+uint64_t make_smem_desc(uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout_type) {
+  // tcgen05 shared-memory matrix descriptor: start address [0,14) (set on the device),
+  // leading byte offset [16,30), stride byte offset [32,46), version=1 [46,48),
+  // base offset [49,52)=0, layout type [61,64).  Offsets are stored >> 4.
+  uint64_t d = 0;
+  d |= uint64_t((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= uint64_t((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= uint64_t(1) << 46;
+  d |= uint64_t(layout_type & 7u) << 61;
+  return d;
+}
+
+void fill_kernel_params(cconv_plan* pl) {
+  const Dims& d = pl->d;
+  const HaloTile& t = pl->tile;
+  HaloKernelParams& p = pl->kp;
+  p.K = d.K; p.H = d.H; p.W = d.W; p.B = d.B; p.C = d.C;
+  p.R = d.R; p.S = d.S; p.sw = d.sw; p.sh = d.sh;
+  p.bb = t.bb; p.bw = t.bw; p.bh = t.bh; p.bc = t.bc;
+  p.halo_w = t.halo_w;
+  p.cchunks = t.cchunks; p.stages = t.stages;
+  p.tiles_k = t.tiles_k; p.tiles_b = t.tiles_b; p.tiles_w = t.tiles_w; p.tiles_h = t.tiles_h;
+  p.total_tiles = int(t.tiles);
+  p.n_mma = t.bb * t.bw;
+  p.acc_cols = p.n_mma * t.bh;
+  p.acc_bufs = t.acc_bufs;
+  p.tmem_cols = t.tmem_cols;
+  p.filt_stage_bytes = t.filt_stage_bytes;
+  p.img_stage_bytes = t.img_stage_bytes;
+  p.tap_bytes = uint32_t(t.bk) * t.bc * 2;
+  p.slab_bytes = uint32_t(t.bc) * t.bb * 2;
+  p.b_kstep_bytes = 16u * t.bb * 2;
+  // instruction descriptor: D=f32 [4,6)=1, A=bf16 [7,10)=1, B=bf16 [10,13)=1, A K-major [15]=0,
+  // B MN-major [16]=1, N>>3 [17,23), M>>4 [24,29)
+  p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
+            (uint32_t(p.n_mma >> 3) << 17) | (uint32_t(128 >> 4) << 24);
+  // A = Filter slab [bk rows][bc channels], K-major; row = bc*2 bytes = the swizzle span.
+  // layout types: 2 = 128B swizzle, 4 = 64B, 6 = 32B.  SBO = 8 rows.
+  const uint32_t a_row = uint32_t(t.bc) * 2;
+  const uint32_t a_layout = a_row == 128 ? 2u : a_row == 64 ? 4u : 6u;
+  p.a_desc = make_smem_desc(16, 8 * a_row, a_layout);
+  // B = Image halo view [channels][n = (w, b)], MN-major; row = bb*2 bytes = the swizzle span.
+  // SBO: from one group of 8 channels to the next; LBO: from one pixel's bb images to the next
+  // pixel along w, sw halo pixels further.
+  const uint32_t b_row = uint32_t(t.bb) * 2;
+  const uint32_t b_layout = b_row == 128 ? 2u : 4u;
+  uint32_t lbo = uint32_t(d.sw) * p.slab_bytes, sbo = 8 * b_row;
+  if (env_int("CCONV_DEBUG_FLAGS", 0) & 1) std::swap(lbo, sbo);
+  p.b_desc = make_smem_desc(lbo, sbo, b_layout);
+  p.wait_limit_ns = uint64_t(env_int("CCONV_WAIT_LIMIT_MS", 1000)) * 1000000ull;
+}
+
+int encode_maps(const cconv_plan* pl, const void* image, const void* filter) {
+  std::lock_guard<std::mutex> lk(pl->mu);
+  if (pl->tm_image_ptr == image && pl->tm_filter_ptr == filter) return CCONV_OK;
+  EncodeTiledFn enc = encode_tiled_fn();
+  if (!enc) {
+    g_last_cuda_error = "cuTensorMapEncodeTiled is not available from this driver";
+    return CCONV_ECUDA;
+  }
+  const Dims& d = pl->d;
+  const HaloTile& t = pl->tile;
+  {
+    // Image viewed as (b, c, x, y): b fastest; x is the w-direction subscript (slowest in memory).
+    const cuuint64_t dims[4] = {cuuint64_t(d.B), cuuint64_t(d.C), cuuint64_t(d.Wi()),
+                                cuuint64_t(d.Hi())};
+    const cuuint64_t strides[3] = {cuuint64_t(d.B) * 2, cuuint64_t(d.Hi()) * d.C * d.B * 2,
+                                   cuuint64_t(d.C) * d.B * 2};
+    const cuuint32_t box[4] = {cuuint32_t(t.bb), cuuint32_t(t.bc), cuuint32_t(t.halo_w),
+                               cuuint32_t(t.halo_h)};
+    const cuuint32_t es[4] = {1, 1, 1, 1};
+    const CUtensorMapSwizzle sw = t.bb == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
+    CUresult r = enc(&pl->tm_image, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(image),
+                     dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+      g_last_cuda_error = "cuTensorMapEncodeTiled(Image) failed with CUresult " + std::to_string(int(r));
+      return CCONV_ECUDA;
+    }
+  }
+  {
+    // Filter viewed as (c, k, rs): one box brings all R*S taps of b_k channels x b_c channels and
+    // lands as [rs][k][c], i.e. one K-major MMA operand per tap.
+    const cuuint64_t dims[3] = {cuuint64_t(d.C), cuuint64_t(d.K), cuuint64_t(d.R) * d.S};
+    const cuuint64_t strides[2] = {cuuint64_t(d.R) * d.S * d.C * 2, cuuint64_t(d.C) * 2};
+    const cuuint32_t box[3] = {cuuint32_t(t.bc), cuuint32_t(t.bk), cuuint32_t(d.R * d.S)};
+    const cuuint32_t es[3] = {1, 1, 1};
+    const CUtensorMapSwizzle sw = t.bc == 64   ? CU_TENSOR_MAP_SWIZZLE_128B
+                                  : t.bc == 32 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                               : CU_TENSOR_MAP_SWIZZLE_32B;
+    CUresult r = enc(&pl->tm_filter, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(filter),
+                     dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+      g_last_cuda_error = "cuTensorMapEncodeTiled(Filter) failed with CUresult " + std::to_string(int(r));
+      return CCONV_ECUDA;
+    }
+  }
+  pl->tm_image_ptr = image;
+  pl->tm_filter_ptr = filter;
+  return CCONV_OK;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+std::mutex g_cache_mu;
+std::map<std::tuple<int, int, int, int, int, int, int, int, int, int, int>, cconv_plan*> g_cache;
+
+}  // namespace
+
+extern "C" {
+
+int cconv_version(void) { return 100; }
+
+const char* cconv_strerror(int code) {
+  switch (code) {
+    case CCONV_OK: return "ok";
+    case CCONV_EINVAL: return "invalid argument";
+    case CCONV_EUNSUPPORTED: return "unsupported shape or device for the requested variant";
+    case CCONV_ECUDA: return "CUDA error";
+    case CCONV_EDEVICE_TIMEOUT: return "a bounded device-side wait expired";
+    case CCONV_ENOMEM: return "out of memory";
+    default: return "unknown error";
+  }
+}
+
+const char* cconv_last_cuda_error(void) { return g_last_cuda_error.c_str(); }
+
+int cconv_lower_bound(int B, int C, int K, int W, int H, int R, int S, int sw, int sh,
+                      double M_words, double terms_out[5]) {
+  const Dims d{B, C, K, W, H, R, S, sw, sh};
+  if (!d.positive() || !(M_words > 0) || !terms_out) return CCONV_EINVAL;
+  theorem1_terms(d, M_words, terms_out);
+  return CCONV_OK;
+}
+
+int cconv_tiling_lp(int B, int C, int K, int W, int H, int R, int S, int sw, int sh,
+                    double M_words, int pooling, double tiles_out[9], double* G_out,
+                    double* words_out) {
+  const Dims d{B, C, K, W, H, R, S, sw, sh};
+  if (!d.positive() || !(M_words > 1.0) || !tiles_out || !G_out || !words_out) return CCONV_EINVAL;
+  return tiling_lp(d, M_words, pooling != 0, tiles_out, G_out, words_out) ? CCONV_OK : CCONV_EINVAL;
+}
+
+int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, int R, int S,
+                      int sw, int sh, int device, double M_words, int variant, int out_dtype) {
+  if (!plan_out) return CCONV_EINVAL;
+  *plan_out = nullptr;
+  const Dims d{B, C, K, W, H, R, S, sw, sh};
+  if (!d.positive()) return CCONV_EINVAL;
+  if (variant < CCONV_VARIANT_AUTO || variant > CCONV_VARIANT_HALO) return CCONV_EINVAL;
+  if (out_dtype != CCONV_OUT_BF16 && out_dtype != CCONV_OUT_F32) return CCONV_EINVAL;
+  // element counts must fit the kernels' index arithmetic
+  const double lim = 9.0e18;
+  if (double(d.Wi()) * d.Hi() * C * B > lim || double(K) * H * W * B > lim ||
+      double(K) * R * S * C > lim)
+    return CCONV_EINVAL;
+  cconv_plan* pl = new (std::nothrow) cconv_plan();
+  if (!pl) return CCONV_ENOMEM;
+  pl->d = d;
+  pl->device = device;
+  pl->out_dtype = out_dtype;
+  if (device >= 0) {
+    // device < 0: a plan for a nominal B200, for inspection only (no CUDA call is made)
+    cudaDeviceProp prop;
+    cudaError_t e = cudaGetDeviceProperties(&prop, device);
+    if (e != cudaSuccess) {
+      delete pl;
+      return cuda_fail(e, "cudaGetDeviceProperties");
+    }
+    pl->m.sm_count = prop.multiProcessorCount;
+    pl->m.smem_optin_bytes = int(prop.sharedMemPerBlockOptin);
+    pl->m.l2_bytes = prop.l2CacheSize;
+    if (prop.major != 10 && variant == CCONV_VARIANT_HALO) {
+      delete pl;
+      return CCONV_EUNSUPPORTED;
+    }
+  }
+  pl->M_words = M_words > 0 ? M_words : pl->m.smem_optin_bytes / 2.0;
+  theorem1_terms(d, pl->M_words, pl->terms);
+  if (pl->M_words > 1.0) tiling_lp(d, pl->M_words, false, pl->lp_tile, &pl->lp_G, &pl->lp_words);
+
+  int force[5] = {0, 0, 0, 0, 0};
+  if (const char* f = std::getenv("CCONV_FORCE_TILE"))
+    std::sscanf(f, "%d,%d,%d,%d,%d", &force[0], &force[1], &force[2], &force[3], &force[4]);
+  const int env_variant = env_int("CCONV_VARIANT", 0);
+  if (variant == CCONV_VARIANT_AUTO && env_variant >= 1 && env_variant <= 2) variant = env_variant;
+
+  const bool halo_ok = halo_supported(d, nullptr) && choose_halo_tile(d, pl->m, force, &pl->tile);
+  if (variant == CCONV_VARIANT_HALO && !halo_ok) {
+    delete pl;
+    return CCONV_EUNSUPPORTED;
+  }
+  if (variant == CCONV_VARIANT_AUTO) variant = halo_ok ? CCONV_VARIANT_HALO : CCONV_VARIANT_SIMT;
+  pl->variant = variant;
+  if (variant == CCONV_VARIANT_HALO) fill_kernel_params(pl);
+
+  if (device >= 0) {
+    int prev = 0;
+    cudaGetDevice(&prev);
+    cudaError_t e = cudaSetDevice(device);
+    if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&pl->d_status), 256);
+    if (e == cudaSuccess) e = cudaMemset(pl->d_status, 0, 256);
+    if (e == cudaSuccess && variant == CCONV_VARIANT_HALO)
+      e = halo_kernel_prepare(pl->tile.smem_bytes);
+    cudaSetDevice(prev);
+    if (e != cudaSuccess) {
+      if (pl->d_status) cudaFree(pl->d_status);
+      delete pl;
+      return cuda_fail(e, "plan device setup");
+    }
+  }
+  if (env_int("CCONV_LOG", 0)) {
+    const HaloTile& t = pl->tile;
+    std::fprintf(stderr,
+                 "[cconv] B%d C%d K%d W%d H%d R%d S%d s%dx%d variant=%d tile bb=%d bw=%d bh=%d "
+                 "bc=%d stages=%d acc_bufs=%d tmem=%d tiles=%lld grid=%d smem=%d est_cyc=%.0f\n",
+                 B, C, K, W, H, R, S, sw, sh, variant, t.bb, t.bw, t.bh, t.bc, t.stages,
+                 t.acc_bufs, t.tmem_cols, t.tiles, t.grid, t.smem_bytes, t.est_cycles);
+  }
+  *plan_out = pl;
+  return CCONV_OK;
+}
+
+int cconv_plan_info_get(const cconv_plan* pl, cconv_plan_info* o) {
+  if (!pl || !o) return CCONV_EINVAL;
+  std::memset(o, 0, sizeof(*o));
+  int arg = 0;
+  for (int i = 0; i < 5; ++i) {
+    o->term[i] = pl->terms[i];
+    if (pl->terms[i] > pl->terms[arg]) arg = i;
+  }
+  o->bound_words = pl->terms[arg];
+  o->bound_argmax = arg + 1;
+  o->M_words = pl->M_words;
+  for (int i = 0; i < 9; ++i) o->lp_tile[i] = pl->lp_tile[i];
+  o->lp_G = pl->lp_G;
+  o->lp_words = pl->lp_words;
+  o->variant = pl->variant;
+  o->out_dtype = pl->out_dtype;
+  const Dims& d = pl->d;
+  o->compulsory_words =
+      double(d.Wi()) * d.Hi() * d.C * d.B + double(d.K) * d.R * d.S * d.C + double(d.K) * d.H * d.W * d.B;
+  if (pl->variant == CCONV_VARIANT_HALO) {
+    const HaloTile& t = pl->tile;
+    o->bb = t.bb; o->bc = t.bc; o->bk = t.bk; o->bw = t.bw; o->bh = t.bh;
+    o->halo_w = t.halo_w; o->halo_h = t.halo_h;
+    o->stages = t.stages; o->grid = t.grid; o->tiles = int(t.tiles);
+    o->smem_bytes = t.smem_bytes; o->tmem_cols = t.tmem_cols;
+    o->tile_words_smem = t.words_smem;
+  }
+  return CCONV_OK;
+}
+
+void cconv_plan_destroy(cconv_plan* pl) {
+  if (!pl) return;
+  if (pl->device >= 0) {
+    int prev = 0;
+    cudaGetDevice(&prev);
+    cudaSetDevice(pl->device);
+    if (pl->d_status) cudaFree(pl->d_status);
+    if (pl->st_image) cudaFree(pl->st_image);
+    if (pl->st_filter) cudaFree(pl->st_filter);
+    if (pl->st_out) cudaFree(pl->st_out);
+    cudaSetDevice(prev);
+  }
+  delete pl;
+}
+
+int cconv_forward_planned(const cconv_plan* pl, const void* Image, const void* Filter, void* Out,
+                          void* cuda_stream) {
+  if (!pl || !Image || !Filter || !Out) return CCONV_EINVAL;
+  if (pl->device < 0) return CCONV_EINVAL;  // inspection-only plan
+  if (!aligned16(Image) || !aligned16(Filter) || !aligned16(Out)) return CCONV_EINVAL;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (pl->variant == CCONV_VARIANT_SIMT) {
+    cudaError_t e = launch_simt(Image, Filter, Out, pl->out_dtype == CCONV_OUT_F32, pl->d, stream);
+    return e == cudaSuccess ? CCONV_OK : cuda_fail(e, "launch_simt");
+  }
+  int rc = encode_maps(pl, Image, Filter);
+  if (rc != CCONV_OK) return rc;
+  CUtensorMap tmi, tmf;
+  {
+    std::lock_guard<std::mutex> lk(pl->mu);
+    tmi = pl->tm_image;
+    tmf = pl->tm_filter;
+  }
+  cudaError_t e = launch_halo(tmi, tmf, Out, pl->out_dtype == CCONV_OUT_F32, pl->kp, pl->tile.grid,
+                              pl->tile.smem_bytes, pl->d_status, stream);
+  return e == cudaSuccess ? CCONV_OK : cuda_fail(e, "launch_halo");
+}
+
+int cconv_forward(const void* Image, const void* Filter, void* Out, int B, int C, int K, int W,
+                  int H, int R, int S, int sw, int sh, int out_dtype, void* cuda_stream) {
+  int dev = 0;
+  CCONV_CUDA(cudaGetDevice(&dev));
+  cconv_plan* pl = nullptr;
+  {
+    std::lock_guard<std::mutex> lk(g_cache_mu);
+    auto key = std::make_tuple(dev, B, C, K, W, H, R, S, sw, sh, out_dtype);
+    auto it = g_cache.find(key);
+    if (it == g_cache.end()) {
+      int rc = cconv_plan_create(&pl, B, C, K, W, H, R, S, sw, sh, dev, 0.0, CCONV_VARIANT_AUTO,
+                                 out_dtype);
+      if (rc != CCONV_OK) return rc;
+      g_cache[key] = pl;
+    } else {
+      pl = it->second;
+    }
+  }
+  return cconv_forward_planned(pl, Image, Filter, Out, cuda_stream);
+}
+
+int cconv_forward_host(cconv_plan* pl, const void* hImage, const void* hFilter, void* hOut,
+                       void* cuda_stream) {
+  if (!pl || !hImage || !hFilter || !hOut || pl->device < 0) return CCONV_EINVAL;
+  const Dims& d = pl->d;
+  const size_t ni = size_t(d.Wi()) * d.Hi() * d.C * d.B * 2;
+  const size_t nf = size_t(d.K) * d.R * d.S * d.C * 2;
+  const size_t no = size_t(d.K) * d.H * d.W * d.B * (pl->out_dtype == CCONV_OUT_F32 ? 4 : 2);
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (!pl->st_image) {
+    CCONV_CUDA(cudaMalloc(&pl->st_image, ni));
+    CCONV_CUDA(cudaMalloc(&pl->st_filter, nf));
+    CCONV_CUDA(cudaMalloc(&pl->st_out, no));
+  }
+  CCONV_CUDA(cudaMemcpyAsync(pl->st_image, hImage, ni, cudaMemcpyHostToDevice, stream));
+  CCONV_CUDA(cudaMemcpyAsync(pl->st_filter, hFilter, nf, cudaMemcpyHostToDevice, stream));
+  int rc = cconv_forward_planned(pl, pl->st_image, pl->st_filter, pl->st_out, cuda_stream);
+  if (rc != CCONV_OK) return rc;
+  CCONV_CUDA(cudaMemcpyAsync(hOut, pl->st_out, no, cudaMemcpyDeviceToHost, stream));
+  int detail = 0;
+  return cconv_plan_status(pl, cuda_stream, &detail);
+}
+
+int cconv_plan_status(const cconv_plan* pl, void* cuda_stream, int* detail_out) {
+  if (!pl || pl->device < 0 || !pl->d_status) return CCONV_EINVAL;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  int st = 0;
+  CCONV_CUDA(cudaMemcpyAsync(&st, pl->d_status, sizeof(int), cudaMemcpyDeviceToHost, stream));
+  CCONV_CUDA(cudaStreamSynchronize(stream));
+  if (detail_out) *detail_out = st;
+  if (st != 0) {
+    CCONV_CUDA(cudaMemsetAsync(pl->d_status, 0, sizeof(int), stream));
+    CCONV_CUDA(cudaStreamSynchronize(stream));
+    return CCONV_EDEVICE_TIMEOUT;
+  }
+  return CCONV_OK;
+}
+
+}  // extern "C"

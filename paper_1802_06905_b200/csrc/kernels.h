@@ -1,0 +1,48 @@
+// Device kernels of the seven-nested-loop CNN (Eq. 1) and their launchers.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "planner.h"
+
+namespace cconv {
+
+// Bits of the device status word (also returned through cconv_plan_status's detail).
+enum : int {
+  kStatProducerWait = 1,   // TMA producer: a stage never became free
+  kStatMmaWaitFull = 2,    // MMA issuer: a stage never filled
+  kStatMmaWaitTmem = 4,    // MMA issuer: an accumulator buffer never drained
+  kStatEpilogueWait = 8,   // epilogue: an accumulator never completed
+  kStatDrainWait = 16,     // teardown: outstanding MMAs / copies did not retire in time
+};
+
+// Everything the halo/tcgen05 kernel needs besides the two tensor maps and the Out pointer.
+struct HaloKernelParams {
+  int K, H, W, B, C, R, S, sw, sh;
+  int bb, bw, bh, bc;           // block sizes b_b, b_w, b_h, b_c (per stage)
+  int halo_w;                   // Image block extent along w: sw*(bw-1)+R
+  int cchunks, stages;
+  int tiles_k, tiles_b, tiles_w, tiles_h;
+  int total_tiles;
+  int n_mma;                    // N of one MMA = bb*bw
+  int acc_cols, acc_bufs, tmem_cols;
+  uint32_t filt_stage_bytes, img_stage_bytes;
+  uint32_t tap_bytes;           // one (r,s) Filter slab: bk*bc*2
+  uint32_t slab_bytes;          // one Image pixel slab: bc*bb*2
+  uint32_t b_kstep_bytes;       // 16 channels of an Image slab: 16*bb*2
+  uint32_t idesc;               // tcgen05 instruction descriptor
+  uint64_t a_desc, b_desc;      // shared-memory descriptors with a zero start address
+  uint64_t wait_limit_ns;       // bound of every device-side wait
+};
+
+cudaError_t launch_simt(const void* image, const void* filter, void* out, bool out_f32,
+                        const Dims& d, cudaStream_t stream);
+
+cudaError_t halo_kernel_prepare(int smem_bytes);
+cudaError_t launch_halo(const CUtensorMap& tm_image, const CUtensorMap& tm_filter, void* out,
+                        bool out_f32, const HaloKernelParams& p, int grid, int smem_bytes,
+                        int* status, cudaStream_t stream);
+
+}  // namespace cconv

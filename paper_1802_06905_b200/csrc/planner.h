@@ -1,0 +1,61 @@
+// Host-side tile planner: Theorem 1 evaluation, the Section-5 tiling LP, and the hardware legaliser
+// that turns the LP's continuous block sizes into a tile the sm_100a kernels can run.
+#pragma once
+#include <cstdint>
+
+namespace cconv {
+
+struct Dims {
+  int B, C, K, W, H, R, S, sw, sh;
+  int Wi() const { return sw * (W - 1) + R; }
+  int Hi() const { return sh * (H - 1) + S; }
+  double macs() const { return double(B) * C * K * W * H * R * S; }
+  bool positive() const {
+    return B > 0 && C > 0 && K > 0 && W > 0 && H > 0 && R > 0 && S > 0 && sw > 0 && sh > 0;
+  }
+};
+
+// What the device offers; filled from cudaGetDeviceProperties (or defaults for a B200 when a plan
+// is only inspected on a machine without a GPU).
+struct Machine {
+  int sm_count = 148;
+  int smem_optin_bytes = 232448;  // 227 KB
+  int tmem_cols = 512;
+  int l2_bytes = 126 * 1024 * 1024;
+};
+
+// Integer tile of the halo/tcgen05 kernel.  Names follow the paper's block sizes b_x.
+struct HaloTile {
+  int bb = 0;      // b_b: images per tile (32 or 64; one swizzle row of the Image operand)
+  int bw = 0;      // b_w: output pixels along w, the N extent of one MMA is bb*bw
+  int bh = 0;      // b_h: output pixels along h, one MMA per row
+  int bk = 128;    // b_k: output channels per tile = MMA M
+  int bc = 0;      // b_c: channels per shared-memory stage (16, 32 or 64)
+  int halo_w = 0, halo_h = 0;
+  int stages = 0;
+  int acc_bufs = 1;  // TMEM accumulator buffers (2 when two fit in 512 columns)
+  int tmem_cols = 0;
+  int cchunks = 0;
+  int tiles_k = 0, tiles_b = 0, tiles_w = 0, tiles_h = 0;
+  long long tiles = 0;
+  int grid = 0;
+  uint32_t filt_stage_bytes = 0, img_stage_bytes = 0, stage_bytes = 0;
+  int smem_bytes = 0;
+  double est_cycles = 0;   // cost-model estimate for the whole problem, SM cycles
+  double words_smem = 0;   // words staged into shared memory over the whole problem + |Out|
+};
+
+void theorem1_terms(const Dims& d, double M, double t[5]);
+
+// Dense primal simplex on the LP of Section 5 in log_M space.  tiles[9] in the order
+// b_b,b_c,b_k,b_w,b_h,b_r',b_r'',b_s',b_s''.  Returns false on non-positive arguments.
+bool tiling_lp(const Dims& d, double M, bool pooling, double tiles[9], double* G, double* words);
+
+// True when the halo/tcgen05 kernel can run this shape at all.
+bool halo_supported(const Dims& d, const char** why);
+
+// Enumerate legal tiles and keep the one with the least estimated time (ties: fewer staged words).
+// `force` may carry "bw,bh,bc,stages,bb" (0 = free) from the CCONV_FORCE_TILE environment variable.
+bool choose_halo_tile(const Dims& d, const Machine& m, const int force[5], HaloTile* out);
+
+}  // namespace cconv

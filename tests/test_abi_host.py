@@ -1,0 +1,151 @@
+"""Host-side checks of the C-ABI library: it loads without a GPU, exports every declared symbol,
+rejects bad arguments, and its planner agrees with the planner oracle.  No compute calls."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import bounds as ob
+from paper_1802_06905_b200 import binding
+from paper_1802_06905_b200.synth import CONFIGS
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_1802_06905_b200 import build
+    build.build()
+    return binding.load_library()
+
+
+def test_every_declared_symbol_is_exported(lib):
+    hdr = open(os.path.join(ROOT, "include", "cconv.h")).read()
+    hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
+    declared = set(re.findall(r"\b(cconv_[a-z_0-9]+)\s*\(", hdr))
+    assert declared, "no declarations found"
+    assert declared == set(binding.EXPORTS)
+    for name in declared:
+        assert hasattr(lib, name), name
+
+
+def test_strerror_and_version(lib):
+    assert lib.cconv_version() >= 100
+    assert lib.cconv_strerror(0) == b"ok"
+    assert b"invalid" in lib.cconv_strerror(binding.EINVAL)
+
+
+def test_lower_bound_matches_oracle_terms():
+    rng = np.random.default_rng(5)
+    for _ in range(100):
+        B, C, K, W, H = (int(v) for v in rng.integers(1, 500, size=5))
+        R, S = (int(v) for v in rng.integers(1, 12, size=2))
+        sw, sh = (int(v) for v in rng.integers(1, 5, size=2))
+        M = float(rng.integers(2, 10 ** 6))
+        got = binding.lower_bound(B, C, K, W, H, R, S, sw, sh, M)
+        exp = ob.theorem1_terms(B, C, K, W, H, R, S, sw, sh, M)
+        np.testing.assert_allclose(got, exp, rtol=1e-13)
+
+
+def test_lower_bound_rejects_bad_arguments(lib):
+    t = (ctypes.c_double * 5)()
+    assert lib.cconv_lower_bound(0, 1, 1, 1, 1, 1, 1, 1, 1, 10.0, t) == binding.EINVAL
+    assert lib.cconv_lower_bound(1, 1, 1, 1, 1, 1, 1, 1, 1, 0.0, t) == binding.EINVAL
+    assert lib.cconv_lower_bound(1, 1, 1, 1, 1, 1, 1, 1, 1, 10.0, None) == binding.EINVAL
+
+
+def lp_shapes():
+    shapes = [c.dims() for c in CONFIGS] + [(1000, 3, 96, 55, 55, 11, 11, 4, 4)]
+    rng = np.random.default_rng(17)
+    for _ in range(60):
+        B, C, K = (int(v) for v in rng.integers(1, 400, size=3))
+        sw, sh = (int(v) for v in rng.integers(1, 4, size=2))
+        R, S = int(rng.integers(1, 4 * sw + 1)), int(rng.integers(1, 4 * sh + 1))
+        W, H = int(rng.integers(1, 80)), int(rng.integers(1, 80))
+        shapes.append((B, C, K, W, H, R, S, sw, sh))
+    return shapes
+
+
+@pytest.mark.parametrize("dims", lp_shapes(), ids=lambda d: "-".join(map(str, d)))
+def test_tiling_lp_objective_matches_oracle(dims):
+    """The optimiser is not unique; its objective G (hence the words moved) is."""
+    for M in (64.0, 1024.0, 116224.0, 6.0e7):
+        tiles, G, words = binding.tiling_lp(*dims, M)
+        _, G_o, words_o = ob.tiling_lp(*dims, M)
+        assert G == pytest.approx(G_o, rel=1e-7)
+        assert words == pytest.approx(words_o, rel=1e-7)
+        # feasibility of the library's own point in the block constraints
+        bb, bc, bk, bw, bh, r1, r2, s1, s2 = tiles
+        B, C, K, W, H, R, S, sw, sh = dims
+        tol = 1 + 1e-9
+        assert all(t >= 1 / tol for t in tiles)
+        assert bb <= B * tol and bc <= C * tol and bk <= K * tol and bw <= W * tol and bh <= H * tol
+        assert r2 <= sw * tol and s2 <= sh * tol
+        assert r1 <= max(1.0, R / sw) * tol and s1 <= max(1.0, S / sh) * tol
+        assert bb * bk * bw * bh <= M * tol
+        assert bc * bk * r1 * r2 * s1 * s2 <= M * tol
+        for x in (bw, r1):
+            for y in (bh, s1):
+                assert bb * bc * x * y * r2 * s2 <= M * tol
+        assert np.prod(tiles) == pytest.approx(G, rel=1e-9)
+
+
+def test_pooling_lp_matches_oracle():
+    d = CONFIGS[4].dims()
+    for M in (512.0, 8192.0):
+        _, G, _ = binding.tiling_lp(*d, M, pooling=True)
+        assert G == pytest.approx(ob.tiling_lp(*d, M, pooling=True)[1], rel=1e-7)
+
+
+def test_inspection_plans_are_hardware_legal():
+    """device=-1: a plan for a nominal B200, no CUDA call; the chosen tile must fit the SM."""
+    for cfg in CONFIGS:
+        p = binding.Plan(*cfg.dims(), device=-1)
+        info = p.info()
+        exp_terms = ob.theorem1_terms(*cfg.dims(), info["M_words"])
+        np.testing.assert_allclose(info["term"], exp_terms, rtol=1e-13)
+        assert info["bound_argmax"] == int(np.argmax(exp_terms)) + 1
+        assert info["lp_words"] == pytest.approx(ob.tiling_lp(*cfg.dims(), info["M_words"])[2], rel=1e-7)
+        assert info["compulsory_words"] == cfg.image_words + cfg.filter_words + cfg.out_words
+        if info["variant"] == binding.VARIANT_HALO:
+            assert cfg.B % 32 == 0 and cfg.C % 8 == 0
+            n = info["bb"] * info["bw"]
+            assert n % 16 == 0 and 16 <= n <= 256                      # tcgen05 N rule at M=128
+            assert n * info["bh"] <= 512 and info["tmem_cols"] <= 512   # tensor memory
+            assert info["smem_bytes"] <= 232448                        # 227 KB
+            assert info["stages"] >= 2
+            assert info["halo_w"] == cfg.sw * (info["bw"] - 1) + cfg.R
+            assert info["halo_h"] == cfg.sh * (info["bh"] - 1) + cfg.S
+            stage = (cfg.R * cfg.S * info["bk"] * info["bc"]
+                     + info["halo_w"] * info["halo_h"] * info["bc"] * info["bb"]) * 2
+            assert info["stages"] * stage <= info["smem_bytes"]
+            # the staged words can never undercut the bound at the shared-memory size
+            assert info["tile_words_smem"] >= max(exp_terms) * 0.999 or max(exp_terms) < info["M_words"]
+        else:
+            assert info["variant"] == binding.VARIANT_SIMT
+        # forward on an inspection plan is refused on the host, before any launch
+        assert p._lib.cconv_forward_planned(p._h, 16, 16, 16, None) == binding.EINVAL
+        p.close()
+
+
+def test_plan_create_rejects_bad_arguments(lib):
+    h = ctypes.c_void_p()
+    assert lib.cconv_plan_create(ctypes.byref(h), 0, 8, 8, 4, 4, 3, 3, 1, 1, -1, 0.0, 0, 0) == binding.EINVAL
+    assert lib.cconv_plan_create(ctypes.byref(h), 2, 8, 8, 4, 4, 3, 3, 1, 1, -1, 0.0, 7, 0) == binding.EINVAL
+    assert lib.cconv_plan_create(None, 2, 8, 8, 4, 4, 3, 3, 1, 1, -1, 0.0, 0, 0) == binding.EINVAL
+    assert lib.cconv_plan_create(ctypes.byref(h), 2, 8, 8, 4, 4, 3, 3, 1, 1, -1, 0.0, 0, 5) == binding.EINVAL
+    # the tensor-core variant refuses shapes it cannot tile (B not a multiple of 32)
+    assert lib.cconv_plan_create(ctypes.byref(h), 2, 8, 16, 14, 14, 3, 3, 1, 1, -1, 0.0,
+                                 binding.VARIANT_HALO, 0) == binding.EUNSUPPORTED
+    # ... and C not a multiple of 8
+    assert lib.cconv_plan_create(ctypes.byref(h), 64, 3, 64, 112, 112, 7, 7, 2, 2, -1, 0.0,
+                                 binding.VARIANT_HALO, 0) == binding.EUNSUPPORTED
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "_LIB_PATH", str(tmp_path / "nope.so"))
+    with pytest.raises(RuntimeError, match="no CPU fallback"):
+        binding.load_library()

@@ -1,0 +1,194 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 CPU oracle of Eq. 1,
+element by element on the same seeded bf16 inputs.  Tolerance: 2e-3 * sum|Image*Filter|."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import cnn as ocnn
+from paper_1802_06905_b200 import binding, synth
+from paper_1802_06905_b200.synth import CONFIGS, ConvShape
+
+from gpu_util import assert_close, check_full, oshape, run_gpu, to_bits, to_dev
+
+pytestmark = pytest.mark.gpu
+
+BY = {c.name: c for c in CONFIGS}
+
+
+def cs(name, B, C, K, W, H, R, S, sw=1, sh=1, seed=1234):
+    return ConvShape(name, B, C, K, W, H, R, S, sw, sh, seed=seed)
+
+
+# ---- the benchmark configurations ----------------------------------------------------------------
+
+DTYPES = [binding.OUT_F32, binding.OUT_BF16]
+DT_IDS = ["f32out", "bf16out"]
+
+
+@pytest.mark.parametrize("out_dtype", DTYPES, ids=DT_IDS)
+@pytest.mark.parametrize("name", ["cfg1_tiny_3x3", "cfg2_resnet_3x3", "cfg3_stem_7x7_s2",
+                                  "cfg4_pointwise_1x1"])
+def test_config_full_parity(name, out_dtype):
+    info = check_full(BY[name], out_dtype=out_dtype)
+    if name in ("cfg2_resnet_3x3", "cfg4_pointwise_1x1"):
+        assert info["variant"] == binding.VARIANT_HALO     # the tensor-core path is the one that ran
+
+
+@pytest.mark.parametrize("out_dtype", DTYPES, ids=DT_IDS)
+def test_config5_sampled_parity(out_dtype):
+    """Full size, launch configuration of the benchmark; the oracle evaluates sampled elements one by
+    one: 60 000 random (k,h,w,b), plus every element of two (k,h) rows and of the last pixel."""
+    c = BY["cfg5_large_3x3"]
+    ib, fb = synth.make_inputs(c)
+    got, info = run_gpu(c, ib, fb, out_dtype=out_dtype)
+    assert info["variant"] == binding.VARIANT_HALO
+    rng = np.random.default_rng(55)
+    idx = np.stack([rng.integers(0, n, size=60000) for n in c.out_shape], axis=1).astype(np.int32)
+    rows = []
+    for (k, h) in [(0, 0), (c.K - 1, c.H - 1), (257, 13)]:
+        for w in range(c.W):
+            for b in range(c.B):
+                rows.append((k, h, w, b))
+    for k in range(c.K):
+        rows.append((k, c.H - 1, c.W - 1, c.B - 1))
+    idx = np.concatenate([idx, np.array(rows, dtype=np.int32)])
+    exp, ab = ocnn.cnn_bf16_at(ib, fb, idx, oshape(c))
+    g = got[idx[:, 0], idx[:, 1], idx[:, 2], idx[:, 3]]
+    assert not np.isnan(got).any()
+    assert_close(g, exp, ab, "cfg5 sampled", bf16_out=out_dtype == binding.OUT_BF16)
+
+
+# ---- CUDA-core kernel: odd shapes ------------------------------------------------------------------
+
+SIMT_SHAPES = [
+    cs("s1", 1, 1, 1, 1, 1, 1, 1),
+    cs("s2", 3, 5, 7, 6, 5, 3, 2, 2, 1),
+    cs("s3", 2, 3, 5, 9, 4, 2, 5, 3, 2),          # sw > R: skipped Image columns
+    cs("s4", 5, 4, 9, 3, 7, 4, 1, 1, 3),
+    cs("s5", 33, 9, 17, 5, 6, 3, 3, 2, 2),
+    cs("s6", 2, 8, 16, 14, 14, 3, 3),
+    cs("s7", 7, 13, 6, 1, 1, 5, 4),
+]
+
+
+@pytest.mark.parametrize("out_dtype", DTYPES, ids=DT_IDS)
+@pytest.mark.parametrize("c", SIMT_SHAPES, ids=lambda c: c.name)
+def test_simt_odd_shapes(c, out_dtype):
+    check_full(c, variant=binding.VARIANT_SIMT, out_dtype=out_dtype)
+
+
+# ---- tensor-core kernel: shapes that span several tiles, ragged tails, padded K and C ----------------
+
+HALO_SHAPES = [
+    cs("h_1x1", 64, 64, 128, 4, 4, 1, 1),
+    cs("h_3x3", 32, 32, 128, 6, 5, 3, 3),
+    cs("h_ragged_w", 32, 16, 64, 9, 7, 3, 3),              # K < 128: zero-filled Filter rows
+    cs("h_c_tail", 64, 24, 200, 7, 5, 3, 2),               # C, K not multiples of the blocks
+    cs("h_stride2", 32, 16, 96, 10, 9, 3, 3, 2, 2),
+    cs("h_stride_mixed", 64, 8, 136, 11, 6, 5, 2, 2, 1),
+    cs("h_5x5_s2", 32, 8, 64, 12, 12, 5, 5, 2, 2),
+    cs("h_asym", 96, 40, 130, 5, 13, 2, 4, 1, 3),          # B = 3 batch blocks of 32; sh > 1
+    cs("h_big_c", 32, 520, 128, 3, 3, 3, 3),               # many channel chunks: ring wraps often
+    cs("h_many_tiles", 128, 64, 384, 20, 18, 3, 3),        # more tiles than SMs: persistent loop
+]
+
+
+@pytest.mark.parametrize("out_dtype", DTYPES, ids=DT_IDS)
+@pytest.mark.parametrize("c", HALO_SHAPES, ids=lambda c: c.name)
+def test_halo_shapes(c, out_dtype):
+    info = check_full(c, variant=binding.VARIANT_HALO, out_dtype=out_dtype)
+    assert info["variant"] == binding.VARIANT_HALO
+
+
+def test_halo_matches_simt_kernel_on_device():
+    c = cs("cross", 64, 48, 160, 9, 8, 3, 3)
+    ib, fb = synth.make_inputs(c)
+    a, _ = run_gpu(c, ib, fb, binding.VARIANT_HALO)
+    b, _ = run_gpu(c, ib, fb, binding.VARIANT_SIMT)
+    _, ab = ocnn.cnn_bf16(ib, fb, oshape(c))
+    # two fp32 accumulations of the same C*R*S products in different orders
+    assert np.all(np.abs(a - b) <= c.C * c.R * c.S * 2.0 ** -23 * ab)
+
+
+# ---- index pins on the device ---------------------------------------------------------------------------
+
+@pytest.mark.parametrize("variant", [binding.VARIANT_SIMT, binding.VARIANT_HALO])
+def test_delta_filter_on_device(variant):
+    c = cs("delta", 32, 16, 40, 6, 5, 3, 2, 2, 1)
+    ib, _ = synth.make_inputs(c)
+    fb = np.zeros(c.filter_shape, dtype=np.uint16)
+    k0, r0, s0, c0 = 33, 2, 1, 9
+    fb[k0, r0, s0, c0] = 0x3F80                  # 1.0
+    got, _ = run_gpu(c, ib, fb, variant, binding.OUT_BF16)
+    img = ocnn.bf16_bits_to_f64(ib)
+    for h in range(c.H):
+        for w in range(c.W):
+            np.testing.assert_array_equal(got[k0, h, w, :], img[r0 + c.sw * w, s0 + c.sh * h, c0, :])
+    got[k0] = 0
+    assert not got.any()
+
+
+@pytest.mark.parametrize("variant", [binding.VARIANT_SIMT, binding.VARIANT_HALO])
+def test_constant_inputs_on_device(variant):
+    c = cs("const", 32, 16, 24, 5, 4, 3, 3)
+    ib = np.full(c.image_shape, 0x3F00, dtype=np.uint16)     # 0.5
+    fb = np.full(c.filter_shape, 0xBE80, dtype=np.uint16)    # -0.25
+    for dt in DTYPES:
+        got, _ = run_gpu(c, ib, fb, variant, dt)
+        np.testing.assert_array_equal(got, np.full(c.out_shape, c.C * c.R * c.S * 0.5 * -0.25))
+
+
+# ---- the other entry points --------------------------------------------------------------------------------
+
+def test_cconv_forward_cached_plan_and_guard_bands():
+    c = BY["cfg1_tiny_3x3"]
+    ib, fb = synth.make_inputs(c)
+    img, flt = to_dev(ib), to_dev(fb)
+    n = int(np.prod(c.out_shape))
+    buf = torch.full((n + 256,), -7.0, dtype=torch.bfloat16, device="cuda")
+    out = buf[128:128 + n].view(c.out_shape)
+    for _ in range(2):                                         # second call hits the plan cache
+        binding.conv_forward(img, flt, out, *c.dims())
+    torch.cuda.synchronize()
+    exp, ab = ocnn.cnn_bf16(ib, fb, oshape(c))
+    assert_close(ocnn.bf16_bits_to_f64(to_bits(out)), exp, ab, "cconv_forward", bf16_out=True)
+    assert (buf[:128] == -7.0).all() and (buf[128 + n:] == -7.0).all()   # nothing written outside Out
+
+
+def test_forward_host_entry_point():
+    c = cs("host", 32, 16, 128, 6, 6, 3, 3)
+    ib, fb = synth.make_inputs(c)
+    hi = torch.from_numpy(ib.view(np.int16)).view(torch.bfloat16).pin_memory()
+    hf = torch.from_numpy(fb.view(np.int16)).view(torch.bfloat16).pin_memory()
+    ho = torch.empty(c.out_shape, dtype=torch.bfloat16).pin_memory()
+    plan = binding.Plan(*c.dims(), device=0)
+    plan.forward_host(hi, hf, ho)
+    exp, ab = ocnn.cnn_bf16(ib, fb, oshape(c))
+    assert_close(ocnn.bf16_bits_to_f64(to_bits(ho)), exp, ab, "cconv_forward_host", bf16_out=True)
+    plan.close()
+
+
+def test_misaligned_and_null_pointers_are_rejected_on_the_host():
+    c = BY["cfg1_tiny_3x3"]
+    plan = binding.Plan(*c.dims(), device=0)
+    buf = torch.zeros(1 << 16, dtype=torch.bfloat16, device="cuda")
+    p = buf.data_ptr()
+    assert plan.forward_ptrs(p + 2, p + 4096, p + 8192, None) == binding.EINVAL
+    assert plan.forward_ptrs(None, p + 4096, p + 8192, None) == binding.EINVAL
+    plan.close()
+
+
+def test_repeated_launches_are_deterministic():
+    c = BY["cfg2_resnet_3x3"]
+    ib, fb = synth.make_inputs(c)
+    img, flt = to_dev(ib), to_dev(fb)
+    plan = binding.Plan(*c.dims(), device=0)
+    outs = []
+    for _ in range(3):
+        out = torch.empty(c.out_shape, dtype=torch.bfloat16, device="cuda")
+        plan.forward(img, flt, out)
+        outs.append(to_bits(out))
+    plan.check()
+    np.testing.assert_array_equal(outs[0], outs[1])
+    np.testing.assert_array_equal(outs[0], outs[2])
+    plan.close()
