@@ -50,7 +50,7 @@ extern "C" {
 /* Kernel variants (cconv_plan_create's `variant`). */
 #define CCONV_VARIANT_AUTO 0
 #define CCONV_VARIANT_SIMT 1 /* CUDA-core kernel: any shape, any alignment                      */
-#define CCONV_VARIANT_HALO 2 /* TMA halo tiles -> tcgen05.mma -> TMEM; needs B%32==0, C%8==0    */
+#define CCONV_VARIANT_HALO 2 /* TMA halo tiles -> tcgen05.mma -> TMEM; needs B % 32 == 0         */
 
 /* Element type of Out (cconv_plan_create's `out_dtype`). */
 #define CCONV_OUT_BF16 0
@@ -74,7 +74,8 @@ typedef struct {
   int out_dtype;
   int bb, bc, bk, bw, bh; /* batch, channel (per pipeline stage), out-channel, w, h block sizes */
   int halo_w, halo_h;     /* Image block extent: sw*(bw-1)+R, sh*(bh-1)+S                       */
-  int stages;             /* shared-memory ring depth                                           */
+  int stages;             /* Image shared-memory ring depth                                     */
+  int filter_stages;      /* Filter shared-memory ring depth                                    */
   int grid;               /* CTAs launched (persistent kernel: <= SM count)                     */
   int tiles;              /* output tiles in total                                              */
   int smem_bytes;         /* dynamic shared memory per CTA                                      */
@@ -83,6 +84,7 @@ typedef struct {
    * fast-memory level = shared memory of one CTA; slow side = L2/HBM. */
   double tile_words_smem; /* words staged into shared memory over the whole problem + Out words */
   double compulsory_words; /* |Image| + |Filter| + |Out| with the real Image extent             */
+  double scratch_bytes;   /* device scratch the plan owns (the packed Filter)                   */
 } cconv_plan_info;
 
 /* Theorem 1 (Section 4.1): the five lower-bound terms, in words, for a fast memory of M_words.
@@ -102,7 +104,8 @@ int cconv_tiling_lp(int B, int C, int K, int W, int H, int R, int S, int sw, int
 /* Plan: evaluate the bound, solve the LP, pick a hardware-legal tile and kernel variant for
  * `device`, and build the TMA descriptors' shape data.  M_words <= 0 means "the shared memory one
  * CTA can use, in bf16 words".  variant: CCONV_VARIANT_*; out_dtype: CCONV_OUT_*.  device >= 0 is a
- * CUDA ordinal (a small device status word is allocated there); device = -1 plans for a nominal
+ * CUDA ordinal (a status word and, for the HALO variant, scratch for the repacked Filter are
+ * allocated there; every forward call rewrites that scratch); device = -1 plans for a nominal
  * B200 without any CUDA call, for inspection only (forward calls on such a plan return EINVAL).
  * The plan is immutable afterwards and may be used from any stream of that device, one launch at a
  * time per plan (launches of one plan share its status word). */
@@ -131,6 +134,14 @@ int cconv_forward_host(cconv_plan* plan, const void* hImage, const void* hFilter
 /* Synchronises `cuda_stream`, reads the plan's device status word and clears it.  Returns CCONV_OK,
  * CCONV_EDEVICE_TIMEOUT (and *detail_out = bit mask of the waits that expired) or CCONV_ECUDA. */
 int cconv_plan_status(const cconv_plan* plan, void* cuda_stream, int* detail_out);
+
+/* Diagnostics.  When the environment variable CCONV_TRACE=1 is set at plan creation, the HALO
+ * kernel stamps %globaltimer (ns) at fixed points of each CTA's roles into a [grid][16] table:
+ * 0 entry, 1 set-up done, 2 first Image copy issued, 3 Image producer done, 4 Filter producer done,
+ * 5 first MMA issued, 6 first tile's MMAs issued, 7 all MMAs issued, 8 first accumulator ready,
+ * 9 first tile stored, 10 all tiles stored, 11 exit.  Synchronous copy to host_out (at most
+ * max_u64 values); returns the number of values copied, 0 when tracing is off, or a negative code. */
+int cconv_plan_trace_read(const cconv_plan* plan, unsigned long long* host_out, int max_u64);
 
 const char* cconv_strerror(int code);
 const char* cconv_last_cuda_error(void); /* message of the last failed CUDA call on this thread */

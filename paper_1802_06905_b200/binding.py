@@ -22,7 +22,7 @@ OUT_BF16, OUT_F32 = 0, 1
 EXPORTS = (
     "cconv_lower_bound", "cconv_tiling_lp", "cconv_plan_create", "cconv_plan_info_get",
     "cconv_plan_destroy", "cconv_forward_planned", "cconv_forward", "cconv_forward_host",
-    "cconv_plan_status", "cconv_strerror", "cconv_last_cuda_error", "cconv_version",
+    "cconv_plan_status", "cconv_plan_trace_read", "cconv_strerror", "cconv_last_cuda_error", "cconv_version",
 )
 
 
@@ -44,9 +44,11 @@ class PlanInfo(ctypes.Structure):
         ("variant", ctypes.c_int), ("out_dtype", ctypes.c_int),
         ("bb", ctypes.c_int), ("bc", ctypes.c_int), ("bk", ctypes.c_int), ("bw", ctypes.c_int),
         ("bh", ctypes.c_int), ("halo_w", ctypes.c_int), ("halo_h", ctypes.c_int),
-        ("stages", ctypes.c_int), ("grid", ctypes.c_int), ("tiles", ctypes.c_int),
+        ("stages", ctypes.c_int), ("filter_stages", ctypes.c_int), ("grid", ctypes.c_int),
+        ("tiles", ctypes.c_int),
         ("smem_bytes", ctypes.c_int), ("tmem_cols", ctypes.c_int),
         ("tile_words_smem", ctypes.c_double), ("compulsory_words", ctypes.c_double),
+        ("scratch_bytes", ctypes.c_double),
     ]
 
     def asdict(self):
@@ -92,6 +94,8 @@ def load_library():
     lib.cconv_forward_host.argtypes = [vp, vp, vp, vp, vp]
     lib.cconv_plan_status.restype = i
     lib.cconv_plan_status.argtypes = [vp, vp, ctypes.POINTER(i)]
+    lib.cconv_plan_trace_read.restype = i
+    lib.cconv_plan_trace_read.argtypes = [vp, ctypes.POINTER(ctypes.c_ulonglong), i]
     lib.cconv_strerror.restype = ctypes.c_char_p
     lib.cconv_strerror.argtypes = [i]
     lib.cconv_last_cuda_error.restype = ctypes.c_char_p
@@ -186,6 +190,16 @@ class Plan:
         detail = ctypes.c_int(0)
         code = self._lib.cconv_plan_status(self._h, _stream_ptr(stream), ctypes.byref(detail))
         return code, detail.value
+
+    def trace(self):
+        """cconv_plan_trace_read: (grid, 16) array of device time stamps in ns (empty if off)."""
+        import numpy as np
+        n = (148 + 16) * 16
+        buf = (ctypes.c_ulonglong * n)()
+        got = self._lib.cconv_plan_trace_read(self._h, buf, n)
+        if got < 0:
+            raise CconvError(got, "cconv_plan_trace_read")
+        return np.array(buf[:got], dtype=np.uint64).reshape(-1, 16)
 
     def check(self, stream=None):
         code, detail = self.status(stream)

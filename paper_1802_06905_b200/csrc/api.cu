@@ -3,6 +3,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -70,16 +71,16 @@ struct cconv_plan {
   HaloTile tile{};
   HaloKernelParams kp{};
   int* d_status = nullptr;
+  void* d_packed = nullptr;  // scratch: the packed Filter (rewritten by every forward call)
+  unsigned long long* d_trace = nullptr;  // diagnostics: [grid][16] device time stamps
   // host-buffer entry point: device staging owned by the plan
   void* st_image = nullptr;
   void* st_filter = nullptr;
   void* st_out = nullptr;
-  // tensor maps are rebuilt only when the base pointers change
+  // the tensor map is rebuilt only when the base pointer changes
   mutable std::mutex mu;
   mutable const void* tm_image_ptr = nullptr;
-  mutable const void* tm_filter_ptr = nullptr;
   mutable CUtensorMap tm_image{};
-  mutable CUtensorMap tm_filter{};
 };
 
 namespace {
@@ -104,41 +105,42 @@ void fill_kernel_params(cconv_plan* pl) {
   p.R = d.R; p.S = d.S; p.sw = d.sw; p.sh = d.sh;
   p.bb = t.bb; p.bw = t.bw; p.bh = t.bh; p.bc = t.bc;
   p.halo_w = t.halo_w;
-  p.cchunks = t.cchunks; p.stages = t.stages;
+  p.c16 = t.c16;
+  p.units = t.c16 * d.R * d.S;
+  p.units_per_img = (t.bc / 16) * d.R * d.S;
+  p.uf = t.uf;
+  p.i_stages = t.i_stages; p.f_stages = t.f_stages;
   p.tiles_k = t.tiles_k; p.tiles_b = t.tiles_b; p.tiles_w = t.tiles_w; p.tiles_h = t.tiles_h;
   p.total_tiles = int(t.tiles);
   p.n_mma = t.bb * t.bw;
   p.acc_cols = p.n_mma * t.bh;
   p.acc_bufs = t.acc_bufs;
   p.tmem_cols = t.tmem_cols;
-  p.filt_stage_bytes = t.filt_stage_bytes;
   p.img_stage_bytes = t.img_stage_bytes;
-  p.tap_bytes = uint32_t(t.bk) * t.bc * 2;
+  p.filt_stage_bytes = t.filt_stage_bytes;
   p.slab_bytes = uint32_t(t.bc) * t.bb * 2;
   p.b_kstep_bytes = 16u * t.bb * 2;
   // instruction descriptor: D=f32 [4,6)=1, A=bf16 [7,10)=1, B=bf16 [10,13)=1, A K-major [15]=0,
   // B MN-major [16]=1, N>>3 [17,23), M>>4 [24,29)
   p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
             (uint32_t(p.n_mma >> 3) << 17) | (uint32_t(128 >> 4) << 24);
-  // A = Filter slab [bk rows][bc channels], K-major; row = bc*2 bytes = the swizzle span.
-  // layout types: 2 = 128B swizzle, 4 = 64B, 6 = 32B.  SBO = 8 rows.
-  const uint32_t a_row = uint32_t(t.bc) * 2;
-  const uint32_t a_layout = a_row == 128 ? 2u : a_row == 64 ? 4u : 6u;
-  p.a_desc = make_smem_desc(16, 8 * a_row, a_layout);
-  // B = Image halo view [channels][n = (w, b)], MN-major; row = bb*2 bytes = the swizzle span.
-  // SBO: from one group of 8 channels to the next; LBO: from one pixel's bb images to the next
-  // pixel along w, sw halo pixels further.
+  // A = one packed Filter block [128 rows][16 channels], K-major, no swizzle (layout type 0):
+  // 8x8 core matrices of 128 B; LBO = 128 B between the two channel halves, SBO = 256 B between
+  // groups of 8 rows.
+  p.a_desc = make_smem_desc(128, 256, 0);
+  // B = Image halo view [channels][n = (w, b)], MN-major; row = bb*2 bytes = the swizzle span
+  // (layout type 2 = 128B swizzle, 4 = 64B).  SBO: from one group of 8 channels to the next;
+  // LBO: from one pixel's bb images to the next pixel along w, sw halo pixels further.
   const uint32_t b_row = uint32_t(t.bb) * 2;
   const uint32_t b_layout = b_row == 128 ? 2u : 4u;
-  uint32_t lbo = uint32_t(d.sw) * p.slab_bytes, sbo = 8 * b_row;
-  if (env_int("CCONV_DEBUG_FLAGS", 0) & 1) std::swap(lbo, sbo);
-  p.b_desc = make_smem_desc(lbo, sbo, b_layout);
+  p.b_desc = make_smem_desc(uint32_t(d.sw) * p.slab_bytes, 8 * b_row, b_layout);
   p.wait_limit_ns = uint64_t(env_int("CCONV_WAIT_LIMIT_MS", 1000)) * 1000000ull;
+  p.trace = nullptr;
 }
 
-int encode_maps(const cconv_plan* pl, const void* image, const void* filter) {
+int encode_maps(const cconv_plan* pl, const void* image) {
   std::lock_guard<std::mutex> lk(pl->mu);
-  if (pl->tm_image_ptr == image && pl->tm_filter_ptr == filter) return CCONV_OK;
+  if (pl->tm_image_ptr == image) return CCONV_OK;
   EncodeTiledFn enc = encode_tiled_fn();
   if (!enc) {
     g_last_cuda_error = "cuTensorMapEncodeTiled is not available from this driver";
@@ -146,44 +148,24 @@ int encode_maps(const cconv_plan* pl, const void* image, const void* filter) {
   }
   const Dims& d = pl->d;
   const HaloTile& t = pl->tile;
-  {
-    // Image viewed as (b, c, x, y): b fastest; x is the w-direction subscript (slowest in memory).
-    const cuuint64_t dims[4] = {cuuint64_t(d.B), cuuint64_t(d.C), cuuint64_t(d.Wi()),
-                                cuuint64_t(d.Hi())};
-    const cuuint64_t strides[3] = {cuuint64_t(d.B) * 2, cuuint64_t(d.Hi()) * d.C * d.B * 2,
-                                   cuuint64_t(d.C) * d.B * 2};
-    const cuuint32_t box[4] = {cuuint32_t(t.bb), cuuint32_t(t.bc), cuuint32_t(t.halo_w),
-                               cuuint32_t(t.halo_h)};
-    const cuuint32_t es[4] = {1, 1, 1, 1};
-    const CUtensorMapSwizzle sw = t.bb == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
-    CUresult r = enc(&pl->tm_image, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(image),
-                     dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
-                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) {
-      g_last_cuda_error = "cuTensorMapEncodeTiled(Image) failed with CUresult " + std::to_string(int(r));
-      return CCONV_ECUDA;
-    }
-  }
-  {
-    // Filter viewed as (c, k, rs): one box brings all R*S taps of b_k channels x b_c channels and
-    // lands as [rs][k][c], i.e. one K-major MMA operand per tap.
-    const cuuint64_t dims[3] = {cuuint64_t(d.C), cuuint64_t(d.K), cuuint64_t(d.R) * d.S};
-    const cuuint64_t strides[2] = {cuuint64_t(d.R) * d.S * d.C * 2, cuuint64_t(d.C) * 2};
-    const cuuint32_t box[3] = {cuuint32_t(t.bc), cuuint32_t(t.bk), cuuint32_t(d.R * d.S)};
-    const cuuint32_t es[3] = {1, 1, 1};
-    const CUtensorMapSwizzle sw = t.bc == 64   ? CU_TENSOR_MAP_SWIZZLE_128B
-                                  : t.bc == 32 ? CU_TENSOR_MAP_SWIZZLE_64B
-                                               : CU_TENSOR_MAP_SWIZZLE_32B;
-    CUresult r = enc(&pl->tm_filter, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(filter),
-                     dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
-                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) {
-      g_last_cuda_error = "cuTensorMapEncodeTiled(Filter) failed with CUresult " + std::to_string(int(r));
-      return CCONV_ECUDA;
-    }
+  // Image viewed as (b, c, x, y): b fastest; x is the w-direction subscript (slowest in memory).
+  // A box lands in shared memory as [y][x][c][b]: one slab of b_c x b_b per halo pixel.
+  const cuuint64_t dims[4] = {cuuint64_t(d.B), cuuint64_t(d.C), cuuint64_t(d.Wi()),
+                              cuuint64_t(d.Hi())};
+  const cuuint64_t strides[3] = {cuuint64_t(d.B) * 2, cuuint64_t(d.Hi()) * d.C * d.B * 2,
+                                 cuuint64_t(d.C) * d.B * 2};
+  const cuuint32_t box[4] = {cuuint32_t(t.bb), cuuint32_t(t.bc), cuuint32_t(t.halo_w),
+                             cuuint32_t(t.halo_h)};
+  const cuuint32_t es[4] = {1, 1, 1, 1};
+  const CUtensorMapSwizzle sw = t.bb == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
+  CUresult r = enc(&pl->tm_image, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(image),
+                   dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    g_last_cuda_error = "cuTensorMapEncodeTiled(Image) failed with CUresult " + std::to_string(int(r));
+    return CCONV_ECUDA;
   }
   pl->tm_image_ptr = image;
-  pl->tm_filter_ptr = filter;
   return CCONV_OK;
 }
 
@@ -289,9 +271,17 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
     if (e == cudaSuccess) e = cudaMemset(pl->d_status, 0, 256);
     if (e == cudaSuccess && variant == CCONV_VARIANT_HALO)
       e = halo_kernel_prepare(pl->tile.smem_bytes);
+    if (e == cudaSuccess && variant == CCONV_VARIANT_HALO)
+      e = cudaMalloc(&pl->d_packed, size_t(pl->tile.packed_filter_bytes));
+    if (e == cudaSuccess && variant == CCONV_VARIANT_HALO && env_int("CCONV_TRACE", 0)) {
+      e = cudaMalloc(reinterpret_cast<void**>(&pl->d_trace), size_t(pl->tile.grid + 16) * 16 * 8);
+      if (e == cudaSuccess) e = cudaMemset(pl->d_trace, 0, size_t(pl->tile.grid + 16) * 16 * 8);
+      pl->kp.trace = pl->d_trace;
+    }
     cudaSetDevice(prev);
     if (e != cudaSuccess) {
       if (pl->d_status) cudaFree(pl->d_status);
+      if (pl->d_packed) cudaFree(pl->d_packed);
       delete pl;
       return cuda_fail(e, "plan device setup");
     }
@@ -300,9 +290,11 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
     const HaloTile& t = pl->tile;
     std::fprintf(stderr,
                  "[cconv] B%d C%d K%d W%d H%d R%d S%d s%dx%d variant=%d tile bb=%d bw=%d bh=%d "
-                 "bc=%d stages=%d acc_bufs=%d tmem=%d tiles=%lld grid=%d smem=%d est_cyc=%.0f\n",
-                 B, C, K, W, H, R, S, sw, sh, variant, t.bb, t.bw, t.bh, t.bc, t.stages,
-                 t.acc_bufs, t.tmem_cols, t.tiles, t.grid, t.smem_bytes, t.est_cycles);
+                 "bc=%d i_stages=%d f_stages=%d uf=%d acc_bufs=%d tmem=%d tiles=%lld grid=%d smem=%d "
+                 "est_cyc=%.0f\n",
+                 B, C, K, W, H, R, S, sw, sh, variant, t.bb, t.bw, t.bh, t.bc, t.i_stages,
+                 t.f_stages, t.uf, t.acc_bufs, t.tmem_cols, t.tiles, t.grid, t.smem_bytes,
+                 t.est_cycles);
   }
   *plan_out = pl;
   return CCONV_OK;
@@ -331,9 +323,10 @@ int cconv_plan_info_get(const cconv_plan* pl, cconv_plan_info* o) {
     const HaloTile& t = pl->tile;
     o->bb = t.bb; o->bc = t.bc; o->bk = t.bk; o->bw = t.bw; o->bh = t.bh;
     o->halo_w = t.halo_w; o->halo_h = t.halo_h;
-    o->stages = t.stages; o->grid = t.grid; o->tiles = int(t.tiles);
+    o->stages = t.i_stages; o->filter_stages = t.f_stages; o->grid = t.grid; o->tiles = int(t.tiles);
     o->smem_bytes = t.smem_bytes; o->tmem_cols = t.tmem_cols;
     o->tile_words_smem = t.words_smem;
+    o->scratch_bytes = double(t.packed_filter_bytes);
   }
   return CCONV_OK;
 }
@@ -345,6 +338,8 @@ void cconv_plan_destroy(cconv_plan* pl) {
     cudaGetDevice(&prev);
     cudaSetDevice(pl->device);
     if (pl->d_status) cudaFree(pl->d_status);
+    if (pl->d_packed) cudaFree(pl->d_packed);
+    if (pl->d_trace) cudaFree(pl->d_trace);
     if (pl->st_image) cudaFree(pl->st_image);
     if (pl->st_filter) cudaFree(pl->st_filter);
     if (pl->st_out) cudaFree(pl->st_out);
@@ -363,16 +358,18 @@ int cconv_forward_planned(const cconv_plan* pl, const void* Image, const void* F
     cudaError_t e = launch_simt(Image, Filter, Out, pl->out_dtype == CCONV_OUT_F32, pl->d, stream);
     return e == cudaSuccess ? CCONV_OK : cuda_fail(e, "launch_simt");
   }
-  int rc = encode_maps(pl, Image, Filter);
+  int rc = encode_maps(pl, Image);
   if (rc != CCONV_OK) return rc;
-  CUtensorMap tmi, tmf;
+  CUtensorMap tmi;
   {
     std::lock_guard<std::mutex> lk(pl->mu);
     tmi = pl->tm_image;
-    tmf = pl->tm_filter;
   }
-  cudaError_t e = launch_halo(tmi, tmf, Out, pl->out_dtype == CCONV_OUT_F32, pl->kp, pl->tile.grid,
-                              pl->tile.smem_bytes, pl->d_status, stream);
+  cudaError_t e = launch_pack_filter(Filter, pl->d_packed, pl->d, pl->tile.c16, pl->tile.tiles_k,
+                                     stream);
+  if (e != cudaSuccess) return cuda_fail(e, "launch_pack_filter");
+  e = launch_halo(tmi, pl->d_packed, Out, pl->out_dtype == CCONV_OUT_F32, pl->kp, pl->tile.grid,
+                  pl->tile.smem_bytes, pl->d_status, stream);
   return e == cudaSuccess ? CCONV_OK : cuda_fail(e, "launch_halo");
 }
 
@@ -417,6 +414,14 @@ int cconv_forward_host(cconv_plan* pl, const void* hImage, const void* hFilter, 
   CCONV_CUDA(cudaMemcpyAsync(hOut, pl->st_out, no, cudaMemcpyDeviceToHost, stream));
   int detail = 0;
   return cconv_plan_status(pl, cuda_stream, &detail);
+}
+
+int cconv_plan_trace_read(const cconv_plan* pl, unsigned long long* host_out, int max_u64) {
+  if (!pl || !host_out || max_u64 <= 0) return CCONV_EINVAL;
+  if (!pl->d_trace) return 0;
+  const int n = std::min(max_u64, (pl->tile.grid + 16) * 16);
+  CCONV_CUDA(cudaMemcpy(host_out, pl->d_trace, size_t(n) * 8, cudaMemcpyDeviceToHost));
+  return n;
 }
 
 int cconv_plan_status(const cconv_plan* pl, void* cuda_stream, int* detail_out) {

@@ -119,8 +119,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 // Bounded wait: gives up when another role raised the CTA's abort flag or when the time limit
 // passes; on expiry it records `code` in the global status word and raises the abort flag.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          int* status, int code, uint64_t limit_ns) {
+// The polling loop is kept out of line so that the callers' loop bodies stay small.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                            int* status, int code, uint64_t limit_ns) {
   uint64_t t0 = 0;
   for (uint32_t i = 0;; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -137,19 +138,37 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
   }
 }
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          int* status, int code, uint64_t limit_ns) {
+  if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, abort_flag, status, code, limit_ns);
+}
+// Wait used by warps whose 32 lanes walk a loop together (the MMA issuer, the epilogue).
+// Two measured rules shape it (each cost almost 2x in tcgen05 issue rate when broken):
+//  * EVERY lane polls the barrier itself -- no "lane 0 polls, then warp sync";
+//  * nothing is called: a function call anywhere in the issuing loop, even on a path that never
+//    runs, slows the whole loop, so the time-limit check is inline and rare.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity,
+                                               volatile int* abort_flag, int* status, int code,
+                                               uint64_t limit_ns) {
+  uint64_t t0 = 0;
+  for (uint32_t i = 1;; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 0x3FFFu) == 0u) {
+      if (*abort_flag) return false;
+      const uint64_t t = globaltimer_ns();
+      if (t0 == 0) {
+        t0 = t;
+      } else if (t - t0 > limit_ns) {
+        *abort_flag = 1;
+        atomicOr(status, code);
+        return false;
+      }
+    }
+  }
+}
 __device__ __forceinline__ void fence_barrier_init() {
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-}
-__device__ __forceinline__ void fence_proxy_async() {
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-}
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, int c0, int c1,
-                                            int c2, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
-      " [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
-      "l"(reinterpret_cast<uint64_t>(tm)), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
-      : "memory");
 }
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tm, int c0, int c1,
                                             int c2, int c3, uint32_t bar) {
@@ -180,13 +199,15 @@ __device__ __forceinline__ void tc_fence_before() {
 __device__ __forceinline__ void tc_fence_after() {
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 }
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
-                                          uint32_t idesc, uint32_t accumulate) {
+// D[tmem] (+)= A[smem] * B[smem], executed only where `issue` is true (the warp stays converged).
+__device__ __forceinline__ void umma_bf16_if(bool issue, uint32_t d_tmem, uint64_t a_desc,
+                                             uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
+      "{\n\t.reg .pred p, q;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
-      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      "setp.ne.b32 q, %5, 0;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(uint32_t(issue))
       : "memory");
 }
 // Arrives on the mbarrier once every tcgen05.mma issued so far by this thread has completed.
@@ -208,6 +229,16 @@ __device__ __forceinline__ void tmem_ld_32x32b_x32(uint32_t taddr, uint32_t (&v)
       : "r"(taddr)
       : "memory");
 }
+// True in exactly one (always the same) lane of a fully active warp.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile(
+      "{\n\t.reg .pred P;\n\t"
+      "elect.sync _|P, 0xffffffff;\n\t"
+      "selp.u32 %0, 1, 0, P;\n\t}"
+      : "=r"(pred));
+  return pred != 0;
+}
 __device__ __forceinline__ void tmem_ld_wait() {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
@@ -216,14 +247,88 @@ __device__ __forceinline__ uint32_t pack_bf16x2(uint32_t lo_f32_bits, uint32_t h
       __floats2bfloat162_rn(__uint_as_float(lo_f32_bits), __uint_as_float(hi_f32_bits));
   return *reinterpret_cast<const uint32_t*>(&v);
 }
-// Start-address field of a shared-memory matrix descriptor: bits [0,14) hold (address >> 4).
-__device__ __forceinline__ uint64_t desc_at(uint64_t desc0, uint32_t smem_addr) {
-  return desc0 | uint64_t((smem_addr >> 4) & 0x3FFFu);
+
+constexpr int kThreads = 224;
+// warp 0: Image TMA producer, warp 1: MMA issuer, warps 2-5: epilogue, warp 6: Filter producer
+
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes,
+                                          uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::
+          "r"(dst),
+      "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar)
+      : "memory");
 }
 
-constexpr int kThreads = 192;  // warp 0: TMA producer, warp 1: MMA issuer, warps 2-5: epilogue
+// After the main loop a producer must not leave while its copies may still be landing.
+__device__ __forceinline__ void drain_ring(uint32_t bar_full0, uint32_t it, uint32_t stages,
+                                           int* status, uint64_t limit) {
+  const uint32_t back = it < stages ? it : stages;
+  for (uint32_t j = 0; j < back; ++j) {
+    const uint32_t i2 = it - 1 - j;
+    const uint32_t s = i2 % stages;
+    const uint32_t ph = (i2 / stages) & 1u;
+    const uint64_t t0 = globaltimer_ns();
+    while (!mbar_try_wait(bar_full0 + 8u * s, ph)) {
+      if (globaltimer_ns() - t0 > limit) {
+        atomicOr(status, kStatDrainWait);
+        break;
+      }
+    }
+  }
+}
 
 }  // namespace
+
+// ------------------------------------------------------------------------------------------------
+// Filter packing: [K][R][S][C] -> [k-tile][16-channel chunk][tap][128 x 16 block].
+// Inside a block element (k, c) sits at ((k/8)*2 + c/8)*128 + (k%8)*16 + (c%8)*2 bytes: 8x8 "core
+// matrices" of 128 contiguous bytes, K-major, so a block is a ready tcgen05 A operand
+// (no swizzle, LBO = 128 B between the two channel halves, SBO = 256 B between 8-row groups).
+// Rows k >= K and channels c >= C are zero.  One thread writes 16 bytes.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+    cconv_pack_filter_kernel(const __nv_bfloat16* __restrict__ filter, uint4* __restrict__ packed,
+                             Dims d, int c16, long long slots) {
+  const long long slot = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+  if (slot >= slots) return;
+  const int RS = d.R * d.S;
+  const int j = int(slot & 255);
+  long long unit = slot >> 8;
+  const int tap = int(unit % RS);
+  unit /= RS;
+  const int cc = int(unit % c16);
+  const int kt = int(unit / c16);
+  const int core = j >> 3, row = j & 7;
+  const int k = kt * 128 + (core >> 1) * 8 + row;
+  const int c0 = cc * 16 + (core & 1) * 8;
+  uint4 v = make_uint4(0u, 0u, 0u, 0u);
+  if (k < d.K && c0 < d.C) {
+    const __nv_bfloat16* src = filter + ((long long)k * RS + tap) * d.C + c0;
+    if ((d.C & 7) == 0) {
+      v = *reinterpret_cast<const uint4*>(src);
+    } else {
+      unsigned short e[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        e[i] = (c0 + i < d.C) ? *reinterpret_cast<const unsigned short*>(src + i) : (unsigned short)0;
+      v.x = e[0] | (uint32_t(e[1]) << 16);
+      v.y = e[2] | (uint32_t(e[3]) << 16);
+      v.z = e[4] | (uint32_t(e[5]) << 16);
+      v.w = e[6] | (uint32_t(e[7]) << 16);
+    }
+  }
+  packed[slot] = v;
+}
+
+cudaError_t launch_pack_filter(const void* filter, void* packed, const Dims& d, int c16,
+                               int tiles_k, cudaStream_t stream) {
+  const long long slots = 1ll * tiles_k * c16 * d.R * d.S * (kPackedBlockBytes / 16);
+  const long long blocks = (slots + 255) / 256;
+  cconv_pack_filter_kernel<<<(unsigned)blocks, 256, 0, stream>>>(
+      static_cast<const __nv_bfloat16*>(filter), static_cast<uint4*>(packed), d, c16, slots);
+  return cudaGetLastError();
+}
 
 // ------------------------------------------------------------------------------------------------
 // Halo-tile tcgen05 kernel
@@ -231,16 +336,18 @@ constexpr int kThreads = 192;  // warp 0: TMA producer, warp 1: MMA issuer, warp
 template <typename OutT>
 __global__ void __launch_bounds__(kThreads, 1)
     cconv_halo_kernel(const __grid_constant__ CUtensorMap tm_image,
-                      const __grid_constant__ CUtensorMap tm_filter, OutT* __restrict__ out,
+                      const uint8_t* __restrict__ packed_filter, OutT* __restrict__ out,
                       const HaloKernelParams p, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;  // swizzle atoms need 1024 B
-  const uint32_t stage_bytes = p.filt_stage_bytes + p.img_stage_bytes;
-  const uint32_t bars = smem0 + uint32_t(p.stages) * stage_bytes;
-  // barrier block: full[stages], empty[stages], tfull[2], tempty[2], drain, then two 32-bit slots
-  const uint32_t bar_full = bars;
-  const uint32_t bar_empty = bars + 8u * p.stages;
-  const uint32_t bar_tfull = bars + 16u * p.stages;
+  const uint32_t img_ring = smem0;
+  const uint32_t filt_ring = img_ring + uint32_t(p.i_stages) * p.img_stage_bytes;
+  const uint32_t bars = filt_ring + uint32_t(p.f_stages) * p.filt_stage_bytes;
+  const uint32_t bar_ifull = bars;
+  const uint32_t bar_iempty = bar_ifull + 8u * p.i_stages;
+  const uint32_t bar_ffull = bar_iempty + 8u * p.i_stages;
+  const uint32_t bar_fempty = bar_ffull + 8u * p.f_stages;
+  const uint32_t bar_tfull = bar_fempty + 8u * p.f_stages;
   const uint32_t bar_tempty = bar_tfull + 16u;
   const uint32_t bar_drain = bar_tempty + 16u;
   const uint32_t slot_addr = bar_drain + 8u;
@@ -251,11 +358,20 @@ __global__ void __launch_bounds__(kThreads, 1)
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+#define CCONV_TRACE(slot)                                                        \
+  do {                                                                           \
+    if (p.trace) p.trace[blockIdx.x * 16 + (slot)] = globaltimer_ns();           \
+  } while (0)
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < p.stages; ++s) {
-      mbar_init(bar_full + 8u * s, 1);
-      mbar_init(bar_empty + 8u * s, 1);
+    CCONV_TRACE(0);
+    for (int s = 0; s < p.i_stages; ++s) {
+      mbar_init(bar_ifull + 8u * s, 1);
+      mbar_init(bar_iempty + 8u * s, 1);
+    }
+    for (int s = 0; s < p.f_stages; ++s) {
+      mbar_init(bar_ffull + 8u * s, 1);
+      mbar_init(bar_fempty + 8u * s, 1);
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(bar_tfull + 8u * a, 1);
@@ -265,7 +381,6 @@ __global__ void __launch_bounds__(kThreads, 1)
     *abort_flag = 0;
     fence_barrier_init();
     prefetch_tensormap(&tm_image);
-    prefetch_tensormap(&tm_filter);
   }
   if (warp == 1) {
     tmem_alloc(slot_addr, uint32_t(p.tmem_cols));
@@ -275,102 +390,177 @@ __global__ void __launch_bounds__(kThreads, 1)
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-
   const uint64_t limit = p.wait_limit_ns;
+  if (threadIdx.x == 0) CCONV_TRACE(1);
 
+  // Ring positions advance by increment-and-wrap; a runtime division per stage would cost more
+  // single-thread issue time than the stage's tensor-core work.
   if (warp == 0) {
-    // ===================== TMA producer =====================
+    // ===================== Image halo producer (TMA) =====================
     if (lane == 0) {
-      uint32_t it = 0;
+      uint32_t it = 0, s = 0, ph = 0;
       bool ok = true;
+      const int cchunks = (p.C + p.bc - 1) / p.bc;
+      const uint32_t n_st = uint32_t(p.i_stages);
       for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
-        int t = tile;
-        const int kt = t % p.tiles_k; t /= p.tiles_k;
+        int t = tile / p.tiles_k;
         const int bt = t % p.tiles_b; t /= p.tiles_b;
         const int wt = t % p.tiles_w; t /= p.tiles_w;
         const int ht = t;
-        const int k0 = kt * 128, b0 = bt * p.bb;
+        const int b0 = bt * p.bb;
         const int x0 = wt * p.bw * p.sw, y0 = ht * p.bh * p.sh;
-        for (int cc = 0; cc < p.cchunks; ++cc, ++it) {
-          const uint32_t s = it % uint32_t(p.stages);
-          const uint32_t ph = (it / uint32_t(p.stages)) & 1u;
-          if (!mbar_wait(bar_empty + 8u * s, ph ^ 1u, abort_flag, status, kStatProducerWait,
+        for (int cc = 0, c0 = 0; cc < cchunks; ++cc, c0 += p.bc, ++it) {
+          if (!mbar_wait(bar_iempty + 8u * s, ph ^ 1u, abort_flag, status, kStatProducerWait,
                          limit)) {
             ok = false;
             break;
           }
-          const uint32_t full = bar_full + 8u * s;
-          mbar_arrive_expect_tx(full, stage_bytes);
-          const uint32_t dst = smem0 + s * stage_bytes;
-          tma_load_3d(dst, &tm_filter, cc * p.bc, k0, 0, full);
-          tma_load_4d(dst + p.filt_stage_bytes, &tm_image, b0, cc * p.bc, x0, y0, full);
-        }
-      }
-      // Do not leave while copies may still be landing in this CTA's shared memory.
-      const uint32_t back = it < uint32_t(p.stages) ? it : uint32_t(p.stages);
-      for (uint32_t j = 0; j < back; ++j) {
-        const uint32_t i2 = it - 1 - j;
-        const uint32_t s = i2 % uint32_t(p.stages);
-        const uint32_t ph = (i2 / uint32_t(p.stages)) & 1u;
-        uint64_t t0 = globaltimer_ns();
-        while (!mbar_try_wait(bar_full + 8u * s, ph)) {
-          if (globaltimer_ns() - t0 > limit) {
-            atomicOr(status, kStatDrainWait);
-            break;
+          const uint32_t full = bar_ifull + 8u * s;
+          mbar_arrive_expect_tx(full, p.img_stage_bytes);
+          tma_load_4d(img_ring + s * p.img_stage_bytes, &tm_image, b0, c0, x0, y0, full);
+          if (it == 0) CCONV_TRACE(2);
+          if (++s == n_st) {
+            s = 0;
+            ph ^= 1u;
           }
         }
       }
+      CCONV_TRACE(3);
+      drain_ring(bar_ifull, it, n_st, status, limit);
     }
-  } else if (warp == 1) {
-    // ===================== MMA issuer =====================
+  } else if (warp == 6) {
+    // ===================== Filter producer (bulk copies of packed blocks) =====================
     if (lane == 0) {
-      uint32_t it = 0, tcount = 0;
+      uint32_t it = 0, s = 0, ph = 0;
       bool ok = true;
-      const uint32_t taps = uint32_t(p.R * p.S);
-      const uint32_t ksteps = uint32_t(p.bc / 16);
-      for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x, ++tcount) {
-        const uint32_t abuf = tcount % uint32_t(p.acc_bufs);
-        const uint32_t aph = (tcount / uint32_t(p.acc_bufs)) & 1u;
-        if (!mbar_wait(bar_tempty + 8u * abuf, aph ^ 1u, abort_flag, status, kStatMmaWaitTmem,
-                       limit)) {
-          ok = false;
-          break;
-        }
-        tc_fence_after();
-        const uint32_t d_base = tmem_base + abuf * uint32_t(p.acc_cols);
-        for (int cc = 0; cc < p.cchunks; ++cc, ++it) {
-          const uint32_t s = it % uint32_t(p.stages);
-          const uint32_t ph = (it / uint32_t(p.stages)) & 1u;
-          if (!mbar_wait(bar_full + 8u * s, ph, abort_flag, status, kStatMmaWaitFull, limit)) {
+      const uint32_t n_st = uint32_t(p.f_stages);
+      for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
+        const int kt = tile % p.tiles_k;
+        const uint8_t* src = packed_filter + (size_t)kt * p.units * kPackedBlockBytes;
+        for (int left = p.units; left > 0; left -= p.uf, ++it) {
+          const uint32_t bytes = uint32_t(left < p.uf ? left : p.uf) * kPackedBlockBytes;
+          if (!mbar_wait(bar_fempty + 8u * s, ph ^ 1u, abort_flag, status, kStatFilterWait,
+                         limit)) {
             ok = false;
             break;
           }
-          tc_fence_after();
-          const uint32_t filt = smem0 + s * stage_bytes;
-          const uint32_t img = filt + p.filt_stage_bytes;
-          for (uint32_t kk = 0; kk < ksteps; ++kk) {
-            for (int r = 0; r < p.R; ++r) {
-              for (int sx = 0; sx < p.S; ++sx) {
-                const uint32_t tap = uint32_t(r * p.S + sx);
-                const uint64_t a_desc = desc_at(p.a_desc, filt + tap * p.tap_bytes + kk * 32u);
-                const uint32_t acc = (cc | int(kk) | int(tap)) != 0 ? 1u : 0u;
-                for (int hh = 0; hh < p.bh; ++hh) {
-                  const uint32_t pix = uint32_t((hh * p.sh + sx) * p.halo_w + r);
-                  const uint64_t b_desc =
-                      desc_at(p.b_desc, img + pix * p.slab_bytes + kk * p.b_kstep_bytes);
-                  umma_bf16(d_base + uint32_t(hh * p.n_mma), a_desc, b_desc, p.idesc, acc);
-                }
-              }
+          const uint32_t full = bar_ffull + 8u * s;
+          mbar_arrive_expect_tx(full, bytes);
+          bulk_load(filt_ring + s * p.filt_stage_bytes, src, bytes, full);
+          src += bytes;
+          if (++s == n_st) {
+            s = 0;
+            ph ^= 1u;
+          }
+        }
+      }
+      CCONV_TRACE(4);
+      drain_ring(bar_ffull, it, n_st, status, limit);
+    }
+  } else if (warp == 1) {
+    // ===================== MMA issuer =====================
+    // The whole warp walks the loops (descriptor arithmetic stays warp-uniform) and one fixed lane
+    // issues the tcgen05 instructions.  Per unit the loop does one table read (the tap's halo
+    // offset), b_h MMAs and a few counter updates.
+    {
+      const bool leader = elect_one();
+      uint32_t is = 0, iph = 0, fs = 0, fph = 0, abuf = 0, aph = 0;
+      bool ok = true, first_tile = true;
+      const int R = p.R, S = p.S, units = p.units, units_per_img = p.units_per_img;
+      const uint32_t slab16 = p.slab_bytes >> 4, row16 = uint32_t(p.halo_w) * slab16;
+      // Descriptors differ only in their low word (start address >> 4, bits [0,14)); all
+      // per-instruction arithmetic below is on 32-bit "address >> 4" quantities.
+      const uint32_t a_lo0 = uint32_t(p.a_desc), a_hi = uint32_t(p.a_desc >> 32);
+      const uint32_t b_lo0 = uint32_t(p.b_desc), b_hi = uint32_t(p.b_desc >> 32);
+      const uint32_t hstep16 = uint32_t(p.sh * p.halo_w) * (p.slab_bytes >> 4);  // next output row
+      const uint32_t kstep16 = p.b_kstep_bytes >> 4;
+      const uint32_t img16 = p.img_stage_bytes >> 4, filt16 = p.filt_stage_bytes >> 4;
+      const uint32_t img_ring16 = img_ring >> 4, filt_ring16 = filt_ring >> 4;
+      const uint32_t idesc = p.idesc, n_mma = uint32_t(p.n_mma);
+      const uint32_t n_ist = uint32_t(p.i_stages), n_fst = uint32_t(p.f_stages);
+      const int bh = p.bh, uf = p.uf;
+      for (int tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
+        if (!mbar_wait_warp(bar_tempty + 8u * abuf, aph ^ 1u, abort_flag, status, kStatMmaWaitTmem,
+                            limit))
+          break;
+        tc_fence_after();
+        const uint32_t d_base = tmem_base + abuf * uint32_t(p.acc_cols);
+        uint32_t acc = 0;
+        int f_left = 0, i_left = 0;   // units left in the current Filter / Image stage
+        int sx = 0, tap_r = 0;
+        uint32_t tap_off = 0, col_off = 0;  // halo offset of the current tap, in 16 B units
+        uint32_t a16 = 0, img_kk16 = 0;
+        for (int units_left = units; units_left > 0; --units_left) {
+          if (i_left == 0) {
+            if (!mbar_wait_warp(bar_ifull + 8u * is, iph, abort_flag, status, kStatMmaWaitFull,
+                                limit)) {
+              ok = false;
+              break;
+            }
+            tc_fence_after();
+            img_kk16 = img_ring16 + is * img16;
+            i_left = units_left < units_per_img ? units_left : units_per_img;
+          }
+          if (f_left == 0) {
+            if (!mbar_wait_warp(bar_ffull + 8u * fs, fph, abort_flag, status, kStatMmaWaitFull,
+                                limit)) {
+              ok = false;
+              break;
+            }
+            tc_fence_after();
+            a16 = filt_ring16 + fs * filt16;
+            f_left = units_left < uf ? units_left : uf;
+          }
+          // descriptors are built by the whole warp (uniform values); only the issue is elected
+          const uint64_t a_desc = (uint64_t(a_hi) << 32) | (a_lo0 | a16);
+          uint32_t b16 = img_kk16 + tap_off, d = d_base;
+          for (int hh = 0; hh < bh; ++hh, b16 += hstep16, d += n_mma)
+            umma_bf16_if(leader, d, a_desc, (uint64_t(b_hi) << 32) | (b_lo0 | b16), idesc, acc);
+          acc = 1;
+          a16 += kPackedBlockBytes >> 4;
+          // next tap: one halo row down; after S rows, one pixel to the right; after R*S taps,
+          // the next 16 channels of the same Image stage
+          tap_off += row16;
+          if (++sx == S) {
+            sx = 0;
+            col_off += slab16;
+            tap_off = col_off;
+            if (++tap_r == R) {
+              tap_r = 0;
+              col_off = 0;
+              tap_off = 0;
+              img_kk16 += kstep16;
             }
           }
-          (void)taps;
-          umma_commit(bar_empty + 8u * s);  // stage reusable once these MMAs have read it
+          if (--f_left == 0) {
+            // the Filter stage is free once the MMAs issued so far have read it
+            if (leader) umma_commit(bar_fempty + 8u * fs);
+            if (++fs == n_fst) {
+              fs = 0;
+              fph ^= 1u;
+            }
+          }
+          if (--i_left == 0) {
+            if (leader) umma_commit(bar_iempty + 8u * is);
+            if (++is == n_ist) {
+              is = 0;
+              iph ^= 1u;
+            }
+          }
         }
-        if (ok) umma_commit(bar_tfull + 8u * abuf);  // accumulator complete
+        if (!ok) break;
+        if (leader) umma_commit(bar_tfull + 8u * abuf);  // accumulator complete
+        if (first_tile && lane == 0) CCONV_TRACE(6);
+        first_tile = false;
+        if (++abuf == uint32_t(p.acc_bufs)) {
+          abuf = 0;
+          aph ^= 1u;
+        }
       }
       // All MMAs must have retired before TMEM is released.
-      umma_commit(bar_drain);
-      uint64_t t0 = globaltimer_ns();
+      if (lane == 0) CCONV_TRACE(7);
+      if (leader) umma_commit(bar_drain);
+      const uint64_t t0 = globaltimer_ns();
       while (!mbar_try_wait(bar_drain, 0)) {
         if (globaltimer_ns() - t0 > limit) {
           atomicOr(status, kStatDrainWait);
@@ -379,12 +569,12 @@ __global__ void __launch_bounds__(kThreads, 1)
       }
     }
   } else {
-    // ===================== epilogue: TMEM -> registers -> bf16 -> global =====================
+    // ===================== epilogue: TMEM -> registers -> Out =====================
     const int q = warp & 3;  // this warp may touch TMEM lanes [32q, 32q+32)
-    uint32_t tcount = 0;
-    bool ok = true;
+    uint32_t abuf = 0, aph = 0;
+    bool first_tile = true;
     const int chunks = p.bb / 32;
-    for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x, ++tcount) {
+    for (int tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
       int t = tile;
       const int kt = t % p.tiles_k; t /= p.tiles_k;
       const int bt = t % p.tiles_b; t /= p.tiles_b;
@@ -392,13 +582,10 @@ __global__ void __launch_bounds__(kThreads, 1)
       const int ht = t;
       const int k = kt * 128 + q * 32 + lane;
       const int b0 = bt * p.bb;
-      const uint32_t abuf = tcount % uint32_t(p.acc_bufs);
-      const uint32_t aph = (tcount / uint32_t(p.acc_bufs)) & 1u;
-      if (!mbar_wait(bar_tfull + 8u * abuf, aph, abort_flag, status, kStatEpilogueWait, limit)) {
-        ok = false;
+      if (!mbar_wait_warp(bar_tfull + 8u * abuf, aph, abort_flag, status, kStatEpilogueWait, limit))
         break;
-      }
       tc_fence_after();
+      if (first_tile && threadIdx.x == 64) CCONV_TRACE(8);
       const uint32_t t_base = tmem_base + (uint32_t(q * 32) << 16) + abuf * uint32_t(p.acc_cols);
       for (int hh = 0; hh < p.bh; ++hh) {
         const int h = ht * p.bh + hh;
@@ -434,7 +621,14 @@ __global__ void __launch_bounds__(kThreads, 1)
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_tempty + 8u * abuf);
+      if (first_tile && threadIdx.x == 64) CCONV_TRACE(9);
+      first_tile = false;
+      if (++abuf == uint32_t(p.acc_bufs)) {
+        abuf = 0;
+        aph ^= 1u;
+      }
     }
+    if (threadIdx.x == 64) CCONV_TRACE(10);
   }
 
   // ===================== teardown =====================
@@ -444,6 +638,8 @@ __global__ void __launch_bounds__(kThreads, 1)
     tc_fence_after();
     tmem_dealloc(tmem_base, uint32_t(p.tmem_cols));
   }
+  if (threadIdx.x == 0) CCONV_TRACE(11);
+#undef CCONV_TRACE
 }
 
 cudaError_t halo_kernel_prepare(int smem_bytes) {
@@ -454,15 +650,16 @@ cudaError_t halo_kernel_prepare(int smem_bytes) {
                               cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
 }
 
-cudaError_t launch_halo(const CUtensorMap& tm_image, const CUtensorMap& tm_filter, void* out,
+cudaError_t launch_halo(const CUtensorMap& tm_image, const void* packed_filter, void* out,
                         bool out_f32, const HaloKernelParams& p, int grid, int smem_bytes,
                         int* status, cudaStream_t stream) {
+  const uint8_t* pf = static_cast<const uint8_t*>(packed_filter);
   if (out_f32)
     cconv_halo_kernel<float><<<grid, kThreads, smem_bytes, stream>>>(
-        tm_image, tm_filter, static_cast<float*>(out), p, status);
+        tm_image, pf, static_cast<float*>(out), p, status);
   else
     cconv_halo_kernel<__nv_bfloat16><<<grid, kThreads, smem_bytes, stream>>>(
-        tm_image, tm_filter, static_cast<__nv_bfloat16*>(out), p, status);
+        tm_image, pf, static_cast<__nv_bfloat16*>(out), p, status);
   return cudaGetLastError();
 }
 

@@ -11,37 +11,52 @@ namespace cconv {
 
 // Bits of the device status word (also returned through cconv_plan_status's detail).
 enum : int {
-  kStatProducerWait = 1,   // TMA producer: a stage never became free
+  kStatProducerWait = 1,   // Image producer: a stage never became free
+  kStatFilterWait = 32,    // Filter producer: a stage never became free
   kStatMmaWaitFull = 2,    // MMA issuer: a stage never filled
   kStatMmaWaitTmem = 4,    // MMA issuer: an accumulator buffer never drained
   kStatEpilogueWait = 8,   // epilogue: an accumulator never completed
   kStatDrainWait = 16,     // teardown: outstanding MMAs / copies did not retire in time
 };
 
-// Everything the halo/tcgen05 kernel needs besides the two tensor maps and the Out pointer.
+// Everything the halo/tcgen05 kernel needs besides the Image tensor map and the pointers.
+// A "unit" is one K=16 step of the contraction: 16 channels x one (r,s) tap; units run
+// channel-chunk major, tap minor (u = c16_index * R*S + r*S + s).
 struct HaloKernelParams {
   int K, H, W, B, C, R, S, sw, sh;
-  int bb, bw, bh, bc;           // block sizes b_b, b_w, b_h, b_c (per stage)
+  int bb, bw, bh, bc;           // block sizes b_b, b_w, b_h, b_c (channels per Image stage)
   int halo_w;                   // Image block extent along w: sw*(bw-1)+R
-  int cchunks, stages;
+  int c16;                      // 16-channel chunks of C
+  int units;                    // c16 * R*S
+  int units_per_img;            // (bc/16) * R*S: units served by one Image stage
+  int uf;                       // units per Filter stage
+  int i_stages, f_stages;       // ring depths
   int tiles_k, tiles_b, tiles_w, tiles_h;
   int total_tiles;
   int n_mma;                    // N of one MMA = bb*bw
   int acc_cols, acc_bufs, tmem_cols;
-  uint32_t filt_stage_bytes, img_stage_bytes;
-  uint32_t tap_bytes;           // one (r,s) Filter slab: bk*bc*2
+  uint32_t img_stage_bytes, filt_stage_bytes;
   uint32_t slab_bytes;          // one Image pixel slab: bc*bb*2
   uint32_t b_kstep_bytes;       // 16 channels of an Image slab: 16*bb*2
   uint32_t idesc;               // tcgen05 instruction descriptor
   uint64_t a_desc, b_desc;      // shared-memory descriptors with a zero start address
   uint64_t wait_limit_ns;       // bound of every device-side wait
+  unsigned long long* trace;    // optional [grid][16] globaltimer stamps (diagnostics), or null
 };
+
+// One packed Filter block: 128 output channels x 16 input channels of one tap, 4 KB, stored in the
+// tensor core's K-major no-swizzle core-matrix order.
+constexpr int kPackedBlockBytes = 4096;
 
 cudaError_t launch_simt(const void* image, const void* filter, void* out, bool out_f32,
                         const Dims& d, cudaStream_t stream);
 
+// Filter [K][R][S][C] -> packed [k-tile][16-channel chunk][tap][4 KB block], zero padded.
+cudaError_t launch_pack_filter(const void* filter, void* packed, const Dims& d, int c16,
+                               int tiles_k, cudaStream_t stream);
+
 cudaError_t halo_kernel_prepare(int smem_bytes);
-cudaError_t launch_halo(const CUtensorMap& tm_image, const CUtensorMap& tm_filter, void* out,
+cudaError_t launch_halo(const CUtensorMap& tm_image, const void* packed_filter, void* out,
                         bool out_f32, const HaloKernelParams& p, int grid, int smem_bytes,
                         int* status, cudaStream_t stream);
 

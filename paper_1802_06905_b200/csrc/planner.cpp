@@ -120,12 +120,6 @@ bool halo_supported(const Dims& d, const char** why) {
   const char* w = nullptr;
   if (d.B % 32 != 0)
     w = "B must be a multiple of 32 (one swizzled shared-memory row of images)";
-  else if (d.C % 8 != 0)
-    w = "C must be a multiple of 8 (16-byte TMA strides of Filter)";
-  else if (d.R * d.S > 256)
-    w = "R*S must be <= 256 (TMA box extent)";
-  else if (d.K < 8)
-    w = "K must be >= 8";
   if (why) *why = w;
   return w == nullptr;
 }
@@ -134,15 +128,23 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[5], HaloT
   if (!halo_supported(d, nullptr)) return false;
   const int reserve = 2048;  // barriers, TMEM slot, 1024-byte alignment slack
   const int cap = m.smem_optin_bytes - reserve;
-  const double l2_bytes_per_clk = 48.0;  // per SM, sustained; calibrated on B200
+  // Cost-model constants, measured on B200 with this kernel (SM cycles):
+  //  * words staged into shared memory are served by L2 at about 30 B/clk per SM when all SMs pull
+  //    (8 TB/s in aggregate), at most ~60 B/clk for one SM -- this, the paper's "words moved into
+  //    fast memory", is what binds the large 3x3 shapes;
+  //  * one elected thread issues a unit (b_h MMAs) in about 130 + 60*b_h cycles at best;
+  //  * the epilogue drains an accumulator at about 24 cycles per TMEM column.
+  const double l2_total_bytes_per_clk = 30.0 * m.sm_count, l2_sm_max_bytes_per_clk = 60.0;
+  const int RS = d.R * d.S;
+  const int c16 = (d.C + 15) / 16;
+  const long long units = 1ll * c16 * RS;
   bool found = false;
   HaloTile best;
-  const int c16 = (d.C + 15) / 16 * 16;
   for (int bb : {64, 32}) {
     if (d.B % bb) continue;
     if (force[4] && bb != force[4]) continue;
     for (int bc : {64, 32, 16}) {
-      if (bc > c16 && bc != 16) continue;
+      if (bc > c16 * 16 && bc != 16) continue;
       if (force[2] && bc != force[2]) continue;
       for (int bw = 1; bw <= std::min(d.W, 256 / bb); ++bw) {
         if (force[0] && bw != force[0]) continue;
@@ -153,17 +155,23 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[5], HaloT
           t.bb = bb; t.bw = bw; t.bh = bh; t.bc = bc; t.bk = 128;
           t.halo_w = d.sw * (bw - 1) + d.R;
           t.halo_h = d.sh * (bh - 1) + d.S;
-          if (t.halo_w > 256 || t.halo_h > 256) continue;
-          t.filt_stage_bytes = uint32_t(d.R) * d.S * t.bk * bc * 2;
-          t.img_stage_bytes = uint32_t(t.halo_w) * t.halo_h * bc * bb * 2;
-          t.stage_bytes = t.filt_stage_bytes + t.img_stage_bytes;
-          if (2ll * t.stage_bytes > cap) continue;
+          if (t.halo_w > 256 || t.halo_h > 256) continue;  // TMA box extents
+          t.c16 = c16;
           t.cchunks = (d.C + bc - 1) / bc;
-          t.stages = std::min({8, int(cap / t.stage_bytes), std::max(2, 2 * t.cchunks)});
+          t.uf = int(std::min<long long>(units, 9));
+          t.filt_stage_bytes = uint32_t(t.uf) * 4096u;
+          t.f_stages = (t.filt_stage_bytes <= 24576u) ? 3 : 2;
+          const long long img = 1ll * t.halo_w * t.halo_h * bc * bb * 2;
+          if (img > cap) continue;
+          t.img_stage_bytes = uint32_t(img);
+          const long long left = cap - 1ll * t.f_stages * t.filt_stage_bytes;
+          int is = int(std::min<long long>(6, left / img));
           if (force[3]) {
-            if (int(cap / t.stage_bytes) < force[3]) continue;
-            t.stages = force[3];
+            if (is < force[3]) continue;
+            is = force[3];
           }
+          if (is < 1) continue;
+          t.i_stages = is;  // a single Image stage (huge filters only) runs without overlap
           const int acc_cols = N * bh;
           t.acc_bufs = (2 * acc_cols <= m.tmem_cols) ? 2 : 1;
           int cols = 32;
@@ -174,20 +182,27 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[5], HaloT
           t.tiles_w = (d.W + bw - 1) / bw;
           t.tiles_h = (d.H + bh - 1) / bh;
           t.tiles = 1ll * t.tiles_k * t.tiles_b * t.tiles_w * t.tiles_h;
+          if (t.tiles > 0x7fffffffll) continue;
           t.grid = int(std::min<long long>(t.tiles, m.sm_count));
+          t.packed_filter_bytes = 1ll * t.tiles_k * units * 4096;
           // at least ~115 KB so that two CTAs never share an SM (each would want the tensor memory)
-          t.smem_bytes = std::max(int(t.stages * t.stage_bytes) + reserve, 117760);
+          t.smem_bytes = std::max(int(t.i_stages * t.img_stage_bytes +
+                                      t.f_stages * t.filt_stage_bytes) + reserve, 117760);
           // ---- cycle model (per SM) ------------------------------------------------------
-          const double per_mma = std::max(N / 2.0, 32.0 + N / 4.0);  // math vs operand reads
-          const double n_mma = double(t.cchunks) * (bc / 16) * d.R * d.S * bh;
-          const double cyc_mma = n_mma * per_mma;
-          const double cyc_l2 = double(t.cchunks) * t.stage_bytes / l2_bytes_per_clk;
-          const double cyc_epi = acc_cols * 6.0 + 600.0;  // TMEM loads, convert, 128 rows of stores
-          const double tile_cyc = (t.acc_bufs == 2) ? std::max({cyc_mma, cyc_l2, cyc_epi})
-                                                    : std::max(cyc_mma, cyc_l2) + cyc_epi;
+          const double exec = std::max(N / 2.0, (4096.0 + 32.0 * N) / 128.0);  // math vs operand reads
+          const double unit_clk = std::max(bh * exec, 130.0 + 60.0 * bh);      // issue-rate floor
+          const double cyc_mma = double(units) * unit_clk;
+          const double tile_bytes = double(t.cchunks) * double(img) + double(units) * 4096.0;
+          const double l2_rate = std::min(l2_sm_max_bytes_per_clk, l2_total_bytes_per_clk / t.grid);
+          // 64-byte rows (bb = 32) use the copy engine and the swizzle half as well as 128-byte rows
+          const double cyc_copy = tile_bytes / l2_rate * (bb == 32 ? 1.08 : 1.0);
+          const double cyc_epi = 24.0 * acc_cols;
+          double tile_cyc = (t.acc_bufs == 2) ? std::max({cyc_mma, cyc_copy, cyc_epi})
+                                              : std::max(cyc_mma, cyc_copy) + cyc_epi;
+          if (t.i_stages == 1) tile_cyc = cyc_mma + cyc_copy + cyc_epi;
           const double waves = std::ceil(double(t.tiles) / t.grid);
-          t.est_cycles = waves * tile_cyc + 4000.0;
-          t.words_smem = double(t.tiles) * t.cchunks * (t.stage_bytes / 2) +
+          t.est_cycles = waves * tile_cyc + cyc_epi + 4000.0;
+          t.words_smem = double(t.tiles) * (double(t.cchunks) * (img / 2) + double(units) * 2048.0) +
                          double(d.K) * d.H * d.W * d.B;
           if (!found || t.est_cycles < best.est_cycles * (1 - 1e-9) ||
               (std::fabs(t.est_cycles - best.est_cycles) <= 1e-9 * best.est_cycles &&

@@ -25,21 +25,32 @@ struct Machine {
 };
 
 // Integer tile of the halo/tcgen05 kernel.  Names follow the paper's block sizes b_x.
+//
+// The contraction over (c, r, s) is cut into "units": one unit = 16 channels x one (r,s) tap, i.e.
+// one K=16 step of the tensor core.  Units are ordered channel-chunk major, tap minor.  Two
+// shared-memory rings feed them:
+//   * the Image ring: one stage = the halo block b_b x b_c x (sw(b_w-1)+R) x (sh(b_h-1)+S),
+//     shared by all R*S taps of its b_c channels;
+//   * the Filter ring: one stage = `uf` consecutive units of the packed Filter (b_k x 16 each).
 struct HaloTile {
-  int bb = 0;      // b_b: images per tile (32 or 64; one swizzle row of the Image operand)
-  int bw = 0;      // b_w: output pixels along w, the N extent of one MMA is bb*bw
+  int bb = 0;      // b_b: images per tile (32 or 64; one swizzled shared-memory row)
+  int bw = 0;      // b_w: output pixels along w; the N extent of one MMA is bb*bw
   int bh = 0;      // b_h: output pixels along h, one MMA per row
   int bk = 128;    // b_k: output channels per tile = MMA M
-  int bc = 0;      // b_c: channels per shared-memory stage (16, 32 or 64)
+  int bc = 0;      // b_c: channels per Image stage (16, 32 or 64)
   int halo_w = 0, halo_h = 0;
-  int stages = 0;
-  int acc_bufs = 1;  // TMEM accumulator buffers (2 when two fit in 512 columns)
+  int i_stages = 0;   // Image ring depth
+  int f_stages = 0;   // Filter ring depth
+  int uf = 0;         // units per Filter stage
+  int acc_bufs = 1;   // TMEM accumulator buffers (2 when two fit in 512 columns)
   int tmem_cols = 0;
-  int cchunks = 0;
+  int c16 = 0;        // 16-channel chunks: ceil(C/16)
+  int cchunks = 0;    // Image stages per tile: ceil(C/bc)
   int tiles_k = 0, tiles_b = 0, tiles_w = 0, tiles_h = 0;
   long long tiles = 0;
   int grid = 0;
-  uint32_t filt_stage_bytes = 0, img_stage_bytes = 0, stage_bytes = 0;
+  uint32_t img_stage_bytes = 0, filt_stage_bytes = 0;
+  long long packed_filter_bytes = 0;  // scratch: tiles_k * c16 * R*S blocks of 4 KB
   int smem_bytes = 0;
   double est_cycles = 0;   // cost-model estimate for the whole problem, SM cycles
   double words_smem = 0;   // words staged into shared memory over the whole problem + |Out|

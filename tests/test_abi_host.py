@@ -110,17 +110,19 @@ def test_inspection_plans_are_hardware_legal():
         assert info["lp_words"] == pytest.approx(ob.tiling_lp(*cfg.dims(), info["M_words"])[2], rel=1e-7)
         assert info["compulsory_words"] == cfg.image_words + cfg.filter_words + cfg.out_words
         if info["variant"] == binding.VARIANT_HALO:
-            assert cfg.B % 32 == 0 and cfg.C % 8 == 0
+            assert cfg.B % 32 == 0
             n = info["bb"] * info["bw"]
             assert n % 16 == 0 and 16 <= n <= 256                      # tcgen05 N rule at M=128
             assert n * info["bh"] <= 512 and info["tmem_cols"] <= 512   # tensor memory
             assert info["smem_bytes"] <= 232448                        # 227 KB
-            assert info["stages"] >= 2
+            assert info["stages"] >= 1                                     # Image ring
             assert info["halo_w"] == cfg.sw * (info["bw"] - 1) + cfg.R
             assert info["halo_h"] == cfg.sh * (info["bh"] - 1) + cfg.S
-            stage = (cfg.R * cfg.S * info["bk"] * info["bc"]
-                     + info["halo_w"] * info["halo_h"] * info["bc"] * info["bb"]) * 2
-            assert info["stages"] * stage <= info["smem_bytes"]
+            img_stage = info["halo_w"] * info["halo_h"] * info["bc"] * info["bb"] * 2
+            assert info["filter_stages"] >= 2
+            assert info["stages"] * img_stage + info["filter_stages"] * 4096 <= info["smem_bytes"]
+            units = -(-cfg.C // 16) * cfg.R * cfg.S
+            assert info["scratch_bytes"] == -(-cfg.K // 128) * units * 4096
             # the staged words can never undercut the bound at the shared-memory size
             assert info["tile_words_smem"] >= max(exp_terms) * 0.999 or max(exp_terms) < info["M_words"]
         else:
@@ -139,8 +141,7 @@ def test_plan_create_rejects_bad_arguments(lib):
     # the tensor-core variant refuses shapes it cannot tile (B not a multiple of 32)
     assert lib.cconv_plan_create(ctypes.byref(h), 2, 8, 16, 14, 14, 3, 3, 1, 1, -1, 0.0,
                                  binding.VARIANT_HALO, 0) == binding.EUNSUPPORTED
-    # ... and C not a multiple of 8
-    assert lib.cconv_plan_create(ctypes.byref(h), 64, 3, 64, 112, 112, 7, 7, 2, 2, -1, 0.0,
+    assert lib.cconv_plan_create(ctypes.byref(h), 48, 8, 64, 12, 12, 3, 3, 1, 1, -1, 0.0,
                                  binding.VARIANT_HALO, 0) == binding.EUNSUPPORTED
 
 

@@ -87,6 +87,9 @@ HALO_SHAPES = [
     cs("h_stride2", 32, 16, 96, 10, 9, 3, 3, 2, 2),
     cs("h_stride_mixed", 64, 8, 136, 11, 6, 5, 2, 2, 1),
     cs("h_5x5_s2", 32, 8, 64, 12, 12, 5, 5, 2, 2),
+    cs("h_7x7_s2_c3", 64, 3, 64, 20, 18, 7, 7, 2, 2),      # C = 3: zero-padded channel chunk
+    cs("h_c_odd", 32, 21, 72, 6, 6, 3, 3),                 # C % 8 != 0: element-wise packing
+    cs("h_11x11_s4", 32, 3, 96, 5, 5, 11, 11, 4, 4),       # the worked example's filter: 121 taps
     cs("h_asym", 96, 40, 130, 5, 13, 2, 4, 1, 3),          # B = 3 batch blocks of 32; sh > 1
     cs("h_big_c", 32, 520, 128, 3, 3, 3, 3),               # many channel chunks: ring wraps often
     cs("h_many_tiles", 128, 64, 384, 20, 18, 3, 3),        # more tiles than SMs: persistent loop
