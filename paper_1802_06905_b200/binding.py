@@ -226,3 +226,4 @@ def conv_forward(image, filt, out, B, C, K, W, H, R, S, sw=1, sh=1, out_dtype=OU
     _check(load_library().cconv_forward(pi, pf, po, *dims, int(out_dtype), _stream_ptr(stream)),
            "cconv_forward")
     return out
+

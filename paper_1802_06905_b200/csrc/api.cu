@@ -13,6 +13,7 @@
 #include <tuple>
 
 #include "../../include/cconv.h"
+#include "host_setup.h"
 #include "kernels.h"
 #include "planner.h"
 
@@ -20,10 +21,8 @@ using namespace cconv;
 
 namespace {
 
-thread_local std::string g_last_cuda_error;
-
 int cuda_fail(cudaError_t e, const char* what) {
-  g_last_cuda_error = std::string(what) + ": " + cudaGetErrorString(e);
+  set_last_cuda_error(std::string(what) + ": " + cudaGetErrorString(e));
   return CCONV_ECUDA;
 }
 #define CCONV_CUDA(call)                                  \
@@ -31,25 +30,6 @@ int cuda_fail(cudaError_t e, const char* what) {
     cudaError_t e_ = (call);                              \
     if (e_ != cudaSuccess) return cuda_fail(e_, #call);   \
   } while (0)
-
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
-                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
-                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-// The driver is reached through the runtime so that the library loads on machines without one.
-EncodeTiledFn encode_tiled_fn() {
-  static EncodeTiledFn fn = [] {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) !=
-            cudaSuccess ||
-        q != cudaDriverEntryPointSuccess)
-      p = nullptr;
-    return reinterpret_cast<EncodeTiledFn>(p);
-  }();
-  return fn;
-}
 
 int env_int(const char* name, int dflt) {
   const char* v = std::getenv(name);
@@ -85,90 +65,6 @@ struct cconv_plan {
 
 namespace {
 
-uint64_t make_smem_desc(uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout_type) {
-  // tcgen05 shared-memory matrix descriptor: start address [0,14) (set on the device),
-  // leading byte offset [16,30), stride byte offset [32,46), version=1 [46,48),
-  // base offset [49,52)=0, layout type [61,64).  Offsets are stored >> 4.
-  uint64_t d = 0;
-  d |= uint64_t((lbo_bytes >> 4) & 0x3FFFu) << 16;
-  d |= uint64_t((sbo_bytes >> 4) & 0x3FFFu) << 32;
-  d |= uint64_t(1) << 46;
-  d |= uint64_t(layout_type & 7u) << 61;
-  return d;
-}
-
-void fill_kernel_params(cconv_plan* pl) {
-  const Dims& d = pl->d;
-  const HaloTile& t = pl->tile;
-  HaloKernelParams& p = pl->kp;
-  p.K = d.K; p.H = d.H; p.W = d.W; p.B = d.B; p.C = d.C;
-  p.R = d.R; p.S = d.S; p.sw = d.sw; p.sh = d.sh;
-  p.bb = t.bb; p.bw = t.bw; p.bh = t.bh; p.bc = t.bc;
-  p.halo_w = t.halo_w;
-  p.c16 = t.c16;
-  p.units = t.c16 * d.R * d.S;
-  p.units_per_img = (t.bc / 16) * d.R * d.S;
-  p.uf = t.uf;
-  p.i_stages = t.i_stages; p.f_stages = t.f_stages;
-  p.tiles_k = t.tiles_k; p.tiles_b = t.tiles_b; p.tiles_w = t.tiles_w; p.tiles_h = t.tiles_h;
-  p.total_tiles = int(t.tiles);
-  p.n_mma = t.bb * t.bw;
-  p.acc_cols = p.n_mma * t.bh;
-  p.acc_bufs = t.acc_bufs;
-  p.tmem_cols = t.tmem_cols;
-  p.img_stage_bytes = t.img_stage_bytes;
-  p.filt_stage_bytes = t.filt_stage_bytes;
-  p.slab_bytes = uint32_t(t.bc) * t.bb * 2;
-  p.b_kstep_bytes = 16u * t.bb * 2;
-  // instruction descriptor: D=f32 [4,6)=1, A=bf16 [7,10)=1, B=bf16 [10,13)=1, A K-major [15]=0,
-  // B MN-major [16]=1, N>>3 [17,23), M>>4 [24,29)
-  p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
-            (uint32_t(p.n_mma >> 3) << 17) | (uint32_t(128 >> 4) << 24);
-  // A = one packed Filter block [128 rows][16 channels], K-major, no swizzle (layout type 0):
-  // 8x8 core matrices of 128 B; LBO = 128 B between the two channel halves, SBO = 256 B between
-  // groups of 8 rows.
-  p.a_desc = make_smem_desc(128, 256, 0);
-  // B = Image halo view [channels][n = (w, b)], MN-major; row = bb*2 bytes = the swizzle span
-  // (layout type 2 = 128B swizzle, 4 = 64B).  SBO: from one group of 8 channels to the next;
-  // LBO: from one pixel's bb images to the next pixel along w, sw halo pixels further.
-  const uint32_t b_row = uint32_t(t.bb) * 2;
-  const uint32_t b_layout = b_row == 128 ? 2u : 4u;
-  p.b_desc = make_smem_desc(uint32_t(d.sw) * p.slab_bytes, 8 * b_row, b_layout);
-  p.wait_limit_ns = uint64_t(env_int("CCONV_WAIT_LIMIT_MS", 1000)) * 1000000ull;
-  p.trace = nullptr;
-}
-
-int encode_maps(const cconv_plan* pl, const void* image) {
-  std::lock_guard<std::mutex> lk(pl->mu);
-  if (pl->tm_image_ptr == image) return CCONV_OK;
-  EncodeTiledFn enc = encode_tiled_fn();
-  if (!enc) {
-    g_last_cuda_error = "cuTensorMapEncodeTiled is not available from this driver";
-    return CCONV_ECUDA;
-  }
-  const Dims& d = pl->d;
-  const HaloTile& t = pl->tile;
-  // Image viewed as (b, c, x, y): b fastest; x is the w-direction subscript (slowest in memory).
-  // A box lands in shared memory as [y][x][c][b]: one slab of b_c x b_b per halo pixel.
-  const cuuint64_t dims[4] = {cuuint64_t(d.B), cuuint64_t(d.C), cuuint64_t(d.Wi()),
-                              cuuint64_t(d.Hi())};
-  const cuuint64_t strides[3] = {cuuint64_t(d.B) * 2, cuuint64_t(d.Hi()) * d.C * d.B * 2,
-                                 cuuint64_t(d.C) * d.B * 2};
-  const cuuint32_t box[4] = {cuuint32_t(t.bb), cuuint32_t(t.bc), cuuint32_t(t.halo_w),
-                             cuuint32_t(t.halo_h)};
-  const cuuint32_t es[4] = {1, 1, 1, 1};
-  const CUtensorMapSwizzle sw = t.bb == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
-  CUresult r = enc(&pl->tm_image, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(image),
-                   dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
-                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) {
-    g_last_cuda_error = "cuTensorMapEncodeTiled(Image) failed with CUresult " + std::to_string(int(r));
-    return CCONV_ECUDA;
-  }
-  pl->tm_image_ptr = image;
-  return CCONV_OK;
-}
-
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 std::mutex g_cache_mu;
@@ -192,7 +88,7 @@ const char* cconv_strerror(int code) {
   }
 }
 
-const char* cconv_last_cuda_error(void) { return g_last_cuda_error.c_str(); }
+const char* cconv_last_cuda_error(void) { return last_cuda_error(); }
 
 int cconv_lower_bound(int B, int C, int K, int W, int H, int R, int S, int sw, int sh,
                       double M_words, double terms_out[5]) {
@@ -261,7 +157,7 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
   }
   if (variant == CCONV_VARIANT_AUTO) variant = halo_ok ? CCONV_VARIANT_HALO : CCONV_VARIANT_SIMT;
   pl->variant = variant;
-  if (variant == CCONV_VARIANT_HALO) fill_kernel_params(pl);
+  if (variant == CCONV_VARIANT_HALO) build_halo_params(pl->d, pl->tile, &pl->kp);
 
   if (device >= 0) {
     int prev = 0;
@@ -358,11 +254,15 @@ int cconv_forward_planned(const cconv_plan* pl, const void* Image, const void* F
     cudaError_t e = launch_simt(Image, Filter, Out, pl->out_dtype == CCONV_OUT_F32, pl->d, stream);
     return e == cudaSuccess ? CCONV_OK : cuda_fail(e, "launch_simt");
   }
-  int rc = encode_maps(pl, Image);
-  if (rc != CCONV_OK) return rc;
   CUtensorMap tmi;
   {
+    // the tensor map is rebuilt only when the Image pointer changes
     std::lock_guard<std::mutex> lk(pl->mu);
+    if (pl->tm_image_ptr != Image) {
+      int rc = encode_image_map(pl->d, pl->tile, Image, &pl->tm_image);
+      if (rc != CCONV_OK) return rc;
+      pl->tm_image_ptr = Image;
+    }
     tmi = pl->tm_image;
   }
   cudaError_t e = launch_pack_filter(Filter, pl->d_packed, pl->d, pl->tile.c16, pl->tile.tiles_k,

@@ -1,0 +1,123 @@
+// Host-side helpers shared by the entry points (see host_setup.h).
+#include "host_setup.h"
+
+#include <cuda_runtime.h>
+
+#include <cstdlib>
+
+#include "../../include/cconv.h"
+
+namespace cconv {
+
+namespace {
+
+thread_local std::string g_last_cuda_error;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver is reached through the runtime so that the library loads on machines without one.
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) !=
+            cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
+int env_int(const char* name, int dflt) {
+  const char* v = std::getenv(name);
+  return (v && *v) ? std::atoi(v) : dflt;
+}
+
+uint64_t make_smem_desc(uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout_type) {
+  // tcgen05 shared-memory matrix descriptor: start address [0,14) (set on the device),
+  // leading byte offset [16,30), stride byte offset [32,46), version=1 [46,48),
+  // base offset [49,52)=0, layout type [61,64).  Offsets are stored >> 4.
+  uint64_t d = 0;
+  d |= uint64_t((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= uint64_t((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= uint64_t(1) << 46;
+  d |= uint64_t(layout_type & 7u) << 61;
+  return d;
+}
+
+}  // namespace
+
+void build_halo_params(const Dims& d, const HaloTile& t, HaloKernelParams* out) {
+  HaloKernelParams& p = *out;
+  p.K = d.K; p.H = d.H; p.W = d.W; p.B = d.B; p.C = d.C;
+  p.R = d.R; p.S = d.S; p.sw = d.sw; p.sh = d.sh;
+  p.bb = t.bb; p.bw = t.bw; p.bh = t.bh; p.bc = t.bc;
+  p.halo_w = t.halo_w;
+  p.c16 = t.c16;
+  p.units = t.c16 * d.R * d.S;
+  p.units_per_img = (t.bc / 16) * d.R * d.S;
+  p.uf = t.uf;
+  p.i_stages = t.i_stages; p.f_stages = t.f_stages;
+  p.tiles_k = t.tiles_k; p.tiles_b = t.tiles_b; p.tiles_w = t.tiles_w; p.tiles_h = t.tiles_h;
+  p.total_tiles = int(t.tiles);
+  p.n_mma = t.bb * t.bw;
+  p.acc_cols = p.n_mma * t.bh;
+  p.acc_bufs = t.acc_bufs;
+  p.tmem_cols = t.tmem_cols;
+  p.img_stage_bytes = t.img_stage_bytes;
+  p.filt_stage_bytes = t.filt_stage_bytes;
+  p.slab_bytes = uint32_t(t.bc) * t.bb * 2;
+  p.b_kstep_bytes = 16u * t.bb * 2;
+  // instruction descriptor: D=f32 [4,6)=1, A=bf16 [7,10)=1, B=bf16 [10,13)=1, A K-major [15]=0,
+  // B MN-major [16]=1, N>>3 [17,23), M>>4 [24,29)
+  p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
+            (uint32_t(p.n_mma >> 3) << 17) | (uint32_t(128 >> 4) << 24);
+  // A = one packed Filter block [128 rows][16 channels], K-major, no swizzle (layout type 0):
+  // 8x8 core matrices of 128 B; LBO = 128 B between the two channel halves, SBO = 256 B between
+  // groups of 8 rows.
+  p.a_desc = make_smem_desc(128, 256, 0);
+  // B = Image halo view [channels][n = (w, b)], MN-major; row = bb*2 bytes = the swizzle span
+  // (layout type 2 = 128B swizzle, 4 = 64B).  SBO: from one group of 8 channels to the next;
+  // LBO: from one pixel's bb images to the next pixel along w, sw halo pixels further.
+  const uint32_t b_row = uint32_t(t.bb) * 2;
+  const uint32_t b_layout = b_row == 128 ? 2u : 4u;
+  p.b_desc = make_smem_desc(uint32_t(d.sw) * p.slab_bytes, 8 * b_row, b_layout);
+  p.wait_limit_ns = uint64_t(env_int("CCONV_WAIT_LIMIT_MS", 1000)) * 1000000ull;
+  p.trace = nullptr;
+}
+
+int encode_image_map(const Dims& d, const HaloTile& t, const void* image, CUtensorMap* tm) {
+  EncodeTiledFn enc = encode_tiled_fn();
+  if (!enc) {
+    set_last_cuda_error("cuTensorMapEncodeTiled is not available from this driver");
+    return CCONV_ECUDA;
+  }
+  // Image viewed as (b, c, x, y): b fastest; x is the w-direction subscript (slowest in memory).
+  // A box lands in shared memory as [y][x][c][b]: one slab of b_c x b_b per halo pixel.
+  const cuuint64_t dims[4] = {cuuint64_t(d.B), cuuint64_t(d.C), cuuint64_t(d.Wi()),
+                              cuuint64_t(d.Hi())};
+  const cuuint64_t strides[3] = {cuuint64_t(d.B) * 2, cuuint64_t(d.Hi()) * d.C * d.B * 2,
+                                 cuuint64_t(d.C) * d.B * 2};
+  const cuuint32_t box[4] = {cuuint32_t(t.bb), cuuint32_t(t.bc), cuuint32_t(t.halo_w),
+                             cuuint32_t(t.halo_h)};
+  const cuuint32_t es[4] = {1, 1, 1, 1};
+  const CUtensorMapSwizzle sw = t.bb == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
+  CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(image),
+                   dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    set_last_cuda_error("cuTensorMapEncodeTiled(Image) failed with CUresult " +
+                        std::to_string(int(r)));
+    return CCONV_ECUDA;
+  }
+  return CCONV_OK;
+}
+
+void set_last_cuda_error(const std::string& msg) { g_last_cuda_error = msg; }
+const char* last_cuda_error() { return g_last_cuda_error.c_str(); }
+
+}  // namespace cconv
