@@ -46,6 +46,7 @@ extern "C" {
 #define CCONV_ECUDA (-3)           /* a CUDA call failed; see cconv_last_cuda_error()           */
 #define CCONV_EDEVICE_TIMEOUT (-4) /* a bounded device-side wait expired (kernel bug guard)     */
 #define CCONV_ENOMEM (-5)
+#define CCONV_ETOOLARGE (-6)       /* needs more scratch than cconv_forward_noalloc's fixed array */
 
 /* Kernel variants (cconv_plan_create's `variant`). */
 #define CCONV_VARIANT_AUTO 0
@@ -130,6 +131,35 @@ int cconv_forward(const void* Image, const void* Filter, void* Out, int B, int C
  * Out back, all on `cuda_stream`, then synchronises that stream.  Returns the device status too. */
 int cconv_forward_host(cconv_plan* plan, const void* hImage, const void* hFilter, void* hOut,
                        void* cuda_stream);
+
+/* Scratch held by cconv_forward_noalloc, in bytes (the repacked Filter must fit):
+ * ceil(K/128) * ceil(C/16) * R*S * 4096 <= this. */
+#define CCONV_NOALLOC_MAX_SCRATCH_BYTES (8u * 1024u * 1024u)
+
+/* (The paper has no counterpart of this entry point; it exists for deployment.)
+ * Eq. 1 on device buffers for callers that cannot allocate device memory at the time of the call:
+ * code running inside a CUDA-graph capture, a serving callback whose memory was handed out at
+ * start-up, a process whose allocator may not be entered from this thread.  It runs the same
+ * tensor-core kernels as cconv_forward_planned (HALO variant, so B % 32 == 0 is required; other
+ * shapes return CCONV_EUNSUPPORTED), but keeps the repacked Filter and the status word in a fixed
+ * array inside the library (CCONV_NOALLOC_MAX_SCRATCH_BYTES + 256 bytes of device memory on every
+ * GPU that loads the library, held until the process exits) instead of plan-owned cudaMalloc'd
+ * memory.  It calls no cudaMalloc / cudaFree and no allocating library routine; the tile is
+ * planned on the stack at every call.
+ *   - Shapes whose repacked Filter exceeds the array return CCONV_ETOOLARGE; nothing is launched.
+ *   - The first call on each device looks up the array's device address and the device limits
+ *     (with that device current).  Make that first call outside any stream capture.
+ *   - All calls share the one array, which keeps the previous call's contents: the call clears the
+ *     status word and rewrites the Filter blocks it uses, so back-to-back calls on ONE stream are
+ *     safe, but two calls whose kernels may overlap on the GPU (different streams, no dependency)
+ *     race on the array and give wrong results.  Host-side, calls are serialised by a mutex.
+ *   - Asynchronous on `cuda_stream` when device_status_out is NULL.  With a non-NULL
+ *     device_status_out the call synchronises the stream, stores the device status word there
+ *     (0 = fine, else a bit mask of the bounded waits that expired) and returns
+ *     CCONV_EDEVICE_TIMEOUT if it is non-zero. */
+int cconv_forward_noalloc(const void* Image, const void* Filter, void* Out, int B, int C, int K,
+                          int W, int H, int R, int S, int sw, int sh, int out_dtype,
+                          void* cuda_stream, int* device_status_out);
 
 /* Synchronises `cuda_stream`, reads the plan's device status word and clears it.  Returns CCONV_OK,
  * CCONV_EDEVICE_TIMEOUT (and *detail_out = bit mask of the waits that expired) or CCONV_ECUDA. */

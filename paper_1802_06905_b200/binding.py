@@ -15,13 +15,15 @@ _LIB_PATH = os.path.join(_HERE, "libcconv.so")
 _lib = None
 
 OK = 0
-EINVAL, EUNSUPPORTED, ECUDA, EDEVICE_TIMEOUT, ENOMEM = -1, -2, -3, -4, -5
+EINVAL, EUNSUPPORTED, ECUDA, EDEVICE_TIMEOUT, ENOMEM, ETOOLARGE = -1, -2, -3, -4, -5, -6
+NOALLOC_MAX_SCRATCH_BYTES = 8 * 1024 * 1024
 VARIANT_AUTO, VARIANT_SIMT, VARIANT_HALO = 0, 1, 2
 OUT_BF16, OUT_F32 = 0, 1
 
 EXPORTS = (
     "cconv_lower_bound", "cconv_tiling_lp", "cconv_plan_create", "cconv_plan_info_get",
     "cconv_plan_destroy", "cconv_forward_planned", "cconv_forward", "cconv_forward_host",
+    "cconv_forward_noalloc",
     "cconv_plan_status", "cconv_plan_trace_read", "cconv_strerror", "cconv_last_cuda_error", "cconv_version",
 )
 
@@ -90,6 +92,8 @@ def load_library():
     lib.cconv_forward_planned.argtypes = [vp, vp, vp, vp, vp]
     lib.cconv_forward.restype = i
     lib.cconv_forward.argtypes = [vp, vp, vp] + nine + [i, vp]
+    lib.cconv_forward_noalloc.restype = i
+    lib.cconv_forward_noalloc.argtypes = [vp, vp, vp] + nine + [i, vp, ctypes.POINTER(i)]
     lib.cconv_forward_host.restype = i
     lib.cconv_forward_host.argtypes = [vp, vp, vp, vp, vp]
     lib.cconv_plan_status.restype = i
@@ -227,3 +231,16 @@ def conv_forward(image, filt, out, B, C, K, W, H, R, S, sw=1, sh=1, out_dtype=OU
            "cconv_forward")
     return out
 
+
+def conv_forward_noalloc(image, filt, out, B, C, K, W, H, R, S, sw=1, sh=1, out_dtype=OUT_BF16,
+                         stream=None, sync=False):
+    """cconv_forward_noalloc: the tensor-core convolution for callers that may not allocate device
+    memory (its scratch is a fixed array inside the library).  ``sync=True`` also synchronises the
+    stream and checks the device status word.  Returns the C return code's success as ``out``."""
+    dims = (B, C, K, W, H, R, S, sw, sh)
+    pi, pf, po = _tensor_args(image, filt, out, dims, out_dtype)
+    st = ctypes.c_int(0)
+    rc = load_library().cconv_forward_noalloc(pi, pf, po, *dims, int(out_dtype), _stream_ptr(stream),
+                                              ctypes.byref(st) if sync else None)
+    _check(rc, f"cconv_forward_noalloc (device status {st.value:#x})")
+    return out

@@ -13,7 +13,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcconv.so")
-SOURCES = ["kernels.cu", "api.cu", "host_setup.cu", "planner.cpp"]
+SOURCES = ["kernels.cu", "api.cu", "host_setup.cu", "noalloc.cu", "planner.cpp"]
 HEADERS = ["kernels.h", "planner.h", "host_setup.h", os.path.join("..", "..", "include", "cconv.h")]
 
 

@@ -84,6 +84,8 @@ const char* cconv_strerror(int code) {
     case CCONV_ECUDA: return "CUDA error";
     case CCONV_EDEVICE_TIMEOUT: return "a bounded device-side wait expired";
     case CCONV_ENOMEM: return "out of memory";
+    case CCONV_ETOOLARGE:
+      return "the repacked Filter does not fit the fixed scratch array of cconv_forward_noalloc";
     default: return "unknown error";
   }
 }
