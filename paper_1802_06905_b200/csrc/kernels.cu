@@ -468,6 +468,10 @@ __global__ void __launch_bounds__(kThreads, 1)
       bool ok = true, first_tile = true;
       const int R = p.R, S = p.S, units = p.units, units_per_img = p.units_per_img;
       const uint32_t slab16 = p.slab_bytes >> 4, row16 = uint32_t(p.halo_w) * slab16;
+      const bool taps9 = (R == 3 && S == 3);
+      uint32_t off9[9];  // halo offset of tap (r, s) = r*3 + s, in 16 B units
+#pragma unroll
+      for (int t = 0; t < 9; ++t) off9[t] = uint32_t(t % 3) * row16 + uint32_t(t / 3) * slab16;
       // Descriptors differ only in their low word (start address >> 4, bits [0,14)); all
       // per-instruction arithmetic below is on 32-bit "address >> 4" quantities.
       const uint32_t a_lo0 = uint32_t(p.a_desc), a_hi = uint32_t(p.a_desc >> 32);
@@ -490,7 +494,8 @@ __global__ void __launch_bounds__(kThreads, 1)
         int sx = 0, tap_r = 0;
         uint32_t tap_off = 0, col_off = 0;  // halo offset of the current tap, in 16 B units
         uint32_t a16 = 0, img_kk16 = 0;
-        for (int units_left = units; units_left > 0; --units_left) {
+        int units_left = units;
+        while (units_left > 0) {
           if (i_left == 0) {
             if (!mbar_wait_warp(bar_ifull + 8u * is, iph, abort_flag, status, kStatMmaWaitFull,
                                 limit)) {
@@ -511,28 +516,55 @@ __global__ void __launch_bounds__(kThreads, 1)
             a16 = filt_ring16 + fs * filt16;
             f_left = units_left < uf ? units_left : uf;
           }
-          // descriptors are built by the whole warp (uniform values); only the issue is elected
-          const uint64_t a_desc = (uint64_t(a_hi) << 32) | (a_lo0 | a16);
-          uint32_t b16 = img_kk16 + tap_off, d = d_base;
-          for (int hh = 0; hh < bh; ++hh, b16 += hstep16, d += n_mma)
-            umma_bf16_if(leader, d, a_desc, (uint64_t(b_hi) << 32) | (b_lo0 | b16), idesc, acc);
-          acc = 1;
-          a16 += kPackedBlockBytes >> 4;
-          // next tap: one halo row down; after S rows, one pixel to the right; after R*S taps,
-          // the next 16 channels of the same Image stage
-          tap_off += row16;
-          if (++sx == S) {
-            sx = 0;
-            col_off += slab16;
-            tap_off = col_off;
-            if (++tap_r == R) {
-              tap_r = 0;
-              col_off = 0;
-              tap_off = 0;
+          // Issue every unit both resident stages cover, with no barrier work in between.
+          // Descriptors are built by the whole warp (uniform values); only the issue is elected.
+          const int n = i_left < f_left ? i_left : f_left;
+          if (taps9 && sx == 0 && tap_r == 0 && n >= 9) {
+            // 3x3 filters: whole 16-channel steps, the nine tap offsets held in registers
+            for (int done = 0; done + 9 <= n; done += 9) {
+#pragma unroll
+              for (int t = 0; t < 9; ++t) {
+                const uint64_t a_desc = (uint64_t(a_hi) << 32) | (a_lo0 | (a16 + uint32_t(t) * 256u));
+                uint32_t b16 = img_kk16 + off9[t], d = d_base;
+                for (int hh = 0; hh < bh; ++hh, b16 += hstep16, d += n_mma)
+                  umma_bf16_if(leader, d, a_desc, (uint64_t(b_hi) << 32) | (b_lo0 | b16), idesc, acc);
+                acc = 1;
+              }
+              a16 += 9u * 256u;
               img_kk16 += kstep16;
             }
+            const int issued = n - n % 9;
+            i_left -= issued;
+            f_left -= issued;
+            units_left -= issued;
+          } else {
+            for (int j = 0; j < n; ++j) {
+              const uint64_t a_desc = (uint64_t(a_hi) << 32) | (a_lo0 | a16);
+              uint32_t b16 = img_kk16 + tap_off, d = d_base;
+              for (int hh = 0; hh < bh; ++hh, b16 += hstep16, d += n_mma)
+                umma_bf16_if(leader, d, a_desc, (uint64_t(b_hi) << 32) | (b_lo0 | b16), idesc, acc);
+              acc = 1;
+              a16 += kPackedBlockBytes >> 4;
+              // next tap: one halo row down; after S rows, one pixel to the right; after R*S taps,
+              // the next 16 channels of the same Image stage
+              tap_off += row16;
+              if (++sx == S) {
+                sx = 0;
+                col_off += slab16;
+                tap_off = col_off;
+                if (++tap_r == R) {
+                  tap_r = 0;
+                  col_off = 0;
+                  tap_off = 0;
+                  img_kk16 += kstep16;
+                }
+              }
+            }
+            i_left -= n;
+            f_left -= n;
+            units_left -= n;
           }
-          if (--f_left == 0) {
+          if (f_left == 0) {
             // the Filter stage is free once the MMAs issued so far have read it
             if (leader) umma_commit(bar_fempty + 8u * fs);
             if (++fs == n_fst) {
@@ -540,7 +572,7 @@ __global__ void __launch_bounds__(kThreads, 1)
               fph ^= 1u;
             }
           }
-          if (--i_left == 0) {
+          if (i_left == 0) {
             if (leader) umma_commit(bar_iempty + 8u * is);
             if (++is == n_ist) {
               is = 0;
