@@ -23,7 +23,8 @@
  * the paper's cost model).
  *
  * Ownership: the caller owns Image, Filter and Out.  Unless a function says "host", they are
- * DEVICE pointers on the plan's device, 16-byte aligned, and Out must not overlap the inputs.
+ * DEVICE pointers on the plan's device, 16-byte aligned (Out: 32-byte aligned), and Out must not
+ * overlap the inputs.
  * The library keeps no caller pointer after a call returns.  Device calls are asynchronous on the
  * given stream and never synchronise it.
  *

@@ -250,7 +250,8 @@ int cconv_forward_planned(const cconv_plan* pl, const void* Image, const void* F
                           void* cuda_stream) {
   if (!pl || !Image || !Filter || !Out) return CCONV_EINVAL;
   if (pl->device < 0) return CCONV_EINVAL;  // inspection-only plan
-  if (!aligned16(Image) || !aligned16(Filter) || !aligned16(Out)) return CCONV_EINVAL;
+  if (!aligned16(Image) || !aligned16(Filter) || (reinterpret_cast<uintptr_t>(Out) & 31u))
+    return CCONV_EINVAL;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   if (pl->variant == CCONV_VARIANT_SIMT) {
     cudaError_t e = launch_simt(Image, Filter, Out, pl->out_dtype == CCONV_OUT_F32, pl->d, stream);

@@ -242,14 +242,26 @@ __device__ __forceinline__ bool elect_one() {
 __device__ __forceinline__ void tmem_ld_wait() {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+// 32-byte store: one full sector per lane (sm_100 has 256-bit global stores)
+__device__ __forceinline__ void st_global_v8(void* ptr, uint32_t a0, uint32_t a1, uint32_t a2,
+                                             uint32_t a3, uint32_t a4, uint32_t a5, uint32_t a6,
+                                             uint32_t a7) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(ptr), "r"(a0),
+               "r"(a1), "r"(a2), "r"(a3), "r"(a4), "r"(a5), "r"(a6), "r"(a7)
+               : "memory");
+}
 __device__ __forceinline__ uint32_t pack_bf16x2(uint32_t lo_f32_bits, uint32_t hi_f32_bits) {
   const __nv_bfloat162 v =
       __floats2bfloat162_rn(__uint_as_float(lo_f32_bits), __uint_as_float(hi_f32_bits));
   return *reinterpret_cast<const uint32_t*>(&v);
 }
 
-constexpr int kThreads = 224;
-// warp 0: Image TMA producer, warp 1: MMA issuer, warps 2-5: epilogue, warp 6: Filter producer
+constexpr int kThreads = 288;
+// warp 1: MMA issuer, warps 2-5: epilogue, warps 0 and 7: Image producers (TMA), warps 6 and 8:
+// Filter producers (bulk copies).  One thread's asynchronous copies run one after the other
+// (about 730 cycles each, whatever the size -- measured), so each ring is fed by two threads that
+// take alternate stages; that keeps four copies in flight per CTA.
+constexpr int kProducersPerRing = 2;
 
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes,
                                           uint32_t bar) {
@@ -331,6 +343,181 @@ cudaError_t launch_pack_filter(const void* filter, void* packed, const Dims& d, 
 }
 
 // ------------------------------------------------------------------------------------------------
+// MMA issuer role (warp 1 of cconv_halo_kernel).
+// The whole warp walks the loops (descriptor arithmetic stays warp-uniform) and one fixed lane
+// issues the tcgen05 instructions.  BH > 0 fixes b_h at compile time; TAPS = 9 / 1 unrolls 3x3 /
+// 1x1 filters (0 = any R x S, offsets advanced arithmetically).
+// ------------------------------------------------------------------------------------------------
+struct MmaCtx {
+  uint32_t bar_ifull, bar_iempty, bar_ffull, bar_fempty, bar_tfull, bar_tempty, bar_drain;
+  uint32_t img_ring, filt_ring, tmem_base;
+  volatile int* abort_flag;
+  int* status;
+  uint64_t limit;
+};
+
+template <int BH>
+__device__ __forceinline__ void issue_unit(bool leader, int bh, uint32_t d, uint32_t n_mma,
+                                           uint64_t a_desc, uint32_t b_hi, uint32_t b_lo0,
+                                           uint32_t b16, uint32_t hstep16, uint32_t idesc,
+                                           uint32_t acc) {
+  if constexpr (BH > 0) {
+#pragma unroll
+    for (int hh = 0; hh < BH; ++hh)
+      umma_bf16_if(leader, d + uint32_t(hh) * n_mma, a_desc,
+                   (uint64_t(b_hi) << 32) | (b_lo0 | (b16 + uint32_t(hh) * hstep16)), idesc, acc);
+  } else {
+    for (int hh = 0; hh < bh; ++hh, b16 += hstep16, d += n_mma)
+      umma_bf16_if(leader, d, a_desc, (uint64_t(b_hi) << 32) | (b_lo0 | b16), idesc, acc);
+  }
+}
+
+template <int BH, int TAPS>
+__device__ __forceinline__ void mma_role(const HaloKernelParams& p, const MmaCtx& cx) {
+  const int lane = threadIdx.x & 31;
+  const bool leader = elect_one();
+  uint32_t is = 0, iph = 0, fs = 0, fph = 0, abuf = 0, aph = 0;
+  bool ok = true, first_tile = true;
+  const int R = p.R, S = p.S, units = p.units, units_per_img = p.units_per_img;
+  const uint32_t slab16 = p.slab_bytes >> 4, row16 = uint32_t(p.halo_w) * slab16;
+  uint32_t off9[9];  // 3x3: halo offset of tap (r, s) = r*3 + s, in 16 B units
+#pragma unroll
+  for (int t = 0; t < 9; ++t) off9[t] = uint32_t(t % 3) * row16 + uint32_t(t / 3) * slab16;
+  // Descriptors differ only in their low word (start address >> 4, bits [0,14)); all
+  // per-instruction arithmetic below is on 32-bit "address >> 4" quantities.
+  const uint32_t a_lo0 = uint32_t(p.a_desc), a_hi = uint32_t(p.a_desc >> 32);
+  const uint32_t b_lo0 = uint32_t(p.b_desc), b_hi = uint32_t(p.b_desc >> 32);
+  const uint32_t hstep16 = uint32_t(p.sh * p.halo_w) * slab16;  // next output row
+  const uint32_t kstep16 = p.b_kstep_bytes >> 4;
+  const uint32_t img16 = p.img_stage_bytes >> 4, filt16 = p.filt_stage_bytes >> 4;
+  const uint32_t img_ring16 = cx.img_ring >> 4, filt_ring16 = cx.filt_ring >> 4;
+  const uint32_t idesc = p.idesc, n_mma = uint32_t(p.n_mma);
+  const uint32_t n_ist = uint32_t(p.i_stages), n_fst = uint32_t(p.f_stages);
+  const int bh = p.bh, uf = p.uf;
+  constexpr uint32_t kBlk16 = kPackedBlockBytes >> 4;
+  for (int tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
+    if (!mbar_wait_warp(cx.bar_tempty + 8u * abuf, aph ^ 1u, cx.abort_flag, cx.status,
+                        kStatMmaWaitTmem, cx.limit))
+      break;
+    tc_fence_after();
+    const uint32_t d_base = cx.tmem_base + abuf * uint32_t(p.acc_cols);
+    uint32_t acc = 0;
+    int f_left = 0, i_left = 0;   // units left in the current Filter / Image stage
+    int sx = 0, tap_r = 0;
+    uint32_t tap_off = 0, col_off = 0;  // halo offset of the current tap, in 16 B units
+    uint32_t a16 = 0, img_kk16 = 0;
+    int units_left = units;
+    while (units_left > 0) {
+      if (i_left == 0) {
+        if (!mbar_wait_warp(cx.bar_ifull + 8u * is, iph, cx.abort_flag, cx.status, kStatMmaWaitFull,
+                            cx.limit)) {
+          ok = false;
+          break;
+        }
+        tc_fence_after();
+        img_kk16 = img_ring16 + is * img16;
+        i_left = units_left < units_per_img ? units_left : units_per_img;
+      }
+      if (f_left == 0) {
+        if (!mbar_wait_warp(cx.bar_ffull + 8u * fs, fph, cx.abort_flag, cx.status, kStatMmaWaitFull,
+                            cx.limit)) {
+          ok = false;
+          break;
+        }
+        tc_fence_after();
+        a16 = filt_ring16 + fs * filt16;
+        f_left = units_left < uf ? units_left : uf;
+      }
+      // Issue every unit both resident stages cover, with no barrier work in between.
+      // Descriptors are built by the whole warp (uniform values); only the issue is elected.
+      const int n = i_left < f_left ? i_left : f_left;
+      int issued = 0;
+      if (TAPS == 9 && sx == 0 && tap_r == 0) {
+        // whole 16-channel steps of a 3x3 filter, the nine tap offsets held in registers
+        for (; issued + 9 <= n; issued += 9) {
+#pragma unroll
+          for (int t = 0; t < 9; ++t) {
+            const uint64_t a_desc = (uint64_t(a_hi) << 32) | (a_lo0 | (a16 + uint32_t(t) * kBlk16));
+            issue_unit<BH>(leader, bh, d_base, n_mma, a_desc, b_hi, b_lo0, img_kk16 + off9[t],
+                           hstep16, idesc, acc);
+            acc = 1;
+          }
+          a16 += 9u * kBlk16;
+          img_kk16 += kstep16;
+        }
+      } else if (TAPS == 1) {
+        // 1x1 filter: one unit per 16 channels
+        for (; issued < n; ++issued) {
+          const uint64_t a_desc = (uint64_t(a_hi) << 32) | (a_lo0 | a16);
+          issue_unit<BH>(leader, bh, d_base, n_mma, a_desc, b_hi, b_lo0, img_kk16, hstep16, idesc,
+                         acc);
+          acc = 1;
+          a16 += kBlk16;
+          img_kk16 += kstep16;
+        }
+      }
+      for (; issued < n; ++issued) {
+        const uint64_t a_desc = (uint64_t(a_hi) << 32) | (a_lo0 | a16);
+        issue_unit<BH>(leader, bh, d_base, n_mma, a_desc, b_hi, b_lo0, img_kk16 + tap_off, hstep16,
+                       idesc, acc);
+        acc = 1;
+        a16 += kBlk16;
+        // next tap: one halo row down; after S rows, one pixel to the right; after R*S taps, the
+        // next 16 channels of the same Image stage
+        tap_off += row16;
+        if (++sx == S) {
+          sx = 0;
+          col_off += slab16;
+          tap_off = col_off;
+          if (++tap_r == R) {
+            tap_r = 0;
+            col_off = 0;
+            tap_off = 0;
+            img_kk16 += kstep16;
+          }
+        }
+      }
+      i_left -= n;
+      f_left -= n;
+      units_left -= n;
+      if (f_left == 0) {
+        // the Filter stage is free once the MMAs issued so far have read it
+        if (leader) umma_commit(cx.bar_fempty + 8u * fs);
+        if (++fs == n_fst) {
+          fs = 0;
+          fph ^= 1u;
+        }
+      }
+      if (i_left == 0) {
+        if (leader) umma_commit(cx.bar_iempty + 8u * is);
+        if (++is == n_ist) {
+          is = 0;
+          iph ^= 1u;
+        }
+      }
+    }
+    if (!ok) break;
+    if (leader) umma_commit(cx.bar_tfull + 8u * abuf);  // accumulator complete
+    if (first_tile && lane == 0 && p.trace) p.trace[blockIdx.x * 16 + 6] = globaltimer_ns();
+    first_tile = false;
+    if (++abuf == uint32_t(p.acc_bufs)) {
+      abuf = 0;
+      aph ^= 1u;
+    }
+  }
+  // All MMAs must have retired before TMEM is released.
+  if (lane == 0 && p.trace) p.trace[blockIdx.x * 16 + 7] = globaltimer_ns();
+  if (leader) umma_commit(cx.bar_drain);
+  const uint64_t t0 = globaltimer_ns();
+  while (!mbar_try_wait(cx.bar_drain, 0)) {
+    if (globaltimer_ns() - t0 > cx.limit) {
+      atomicOr(cx.status, kStatDrainWait);
+      break;
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
 // Halo-tile tcgen05 kernel
 // ------------------------------------------------------------------------------------------------
 template <typename OutT>
@@ -395,13 +582,19 @@ __global__ void __launch_bounds__(kThreads, 1)
 
   // Ring positions advance by increment-and-wrap; a runtime division per stage would cost more
   // single-thread issue time than the stage's tensor-core work.
-  if (warp == 0) {
-    // ===================== Image halo producer (TMA) =====================
-    if (lane == 0) {
-      uint32_t it = 0, s = 0, ph = 0;
+  if (warp == 0 || warp == 7) {
+    // ===================== Image halo producers (TMA) =====================
+    // Producer j of the ring issues the stages j, j+2, j+4, ... of the CTA's stage sequence.
+    // (A one-stage ring is fed by the first producer alone: with parity waits a thread may be at
+    // most one phase ahead of a barrier, and two producers sharing one slot would break that.)
+    const uint32_t i_prod = p.i_stages >= 2 ? uint32_t(kProducersPerRing) : 1u;
+    if (lane == 0 && ((warp == 0) ? 0u : 1u) < i_prod) {
+      const uint32_t me = (warp == 0) ? 0u : 1u;
+      const uint32_t n_st = uint32_t(p.i_stages);
+      uint32_t seq = 0;             // stages of this CTA so far, both producers count all of them
+      uint32_t s = 0, ph = 0;       // ring slot and phase of stage `seq`
       bool ok = true;
       const int cchunks = (p.C + p.bc - 1) / p.bc;
-      const uint32_t n_st = uint32_t(p.i_stages);
       for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
         int t = tile / p.tiles_k;
         const int bt = t % p.tiles_b; t /= p.tiles_b;
@@ -409,44 +602,50 @@ __global__ void __launch_bounds__(kThreads, 1)
         const int ht = t;
         const int b0 = bt * p.bb;
         const int x0 = wt * p.bw * p.sw, y0 = ht * p.bh * p.sh;
-        for (int cc = 0, c0 = 0; cc < cchunks; ++cc, c0 += p.bc, ++it) {
-          if (!mbar_wait(bar_iempty + 8u * s, ph ^ 1u, abort_flag, status, kStatProducerWait,
-                         limit)) {
-            ok = false;
-            break;
+        for (int cc = 0, c0 = 0; cc < cchunks; ++cc, c0 += p.bc, ++seq) {
+          if ((seq & (i_prod - 1u)) == me) {
+            if (!mbar_wait(bar_iempty + 8u * s, ph ^ 1u, abort_flag, status, kStatProducerWait,
+                           limit)) {
+              ok = false;
+              break;
+            }
+            const uint32_t full = bar_ifull + 8u * s;
+            mbar_arrive_expect_tx(full, p.img_stage_bytes);
+            tma_load_4d(img_ring + s * p.img_stage_bytes, &tm_image, b0, c0, x0, y0, full);
+            if (seq == 0) CCONV_TRACE(2);
           }
-          const uint32_t full = bar_ifull + 8u * s;
-          mbar_arrive_expect_tx(full, p.img_stage_bytes);
-          tma_load_4d(img_ring + s * p.img_stage_bytes, &tm_image, b0, c0, x0, y0, full);
-          if (it == 0) CCONV_TRACE(2);
           if (++s == n_st) {
             s = 0;
             ph ^= 1u;
           }
         }
       }
-      CCONV_TRACE(3);
-      drain_ring(bar_ifull, it, n_st, status, limit);
+      if (me == 0) CCONV_TRACE(3);
+      drain_ring(bar_ifull, seq, n_st, status, limit);
     }
-  } else if (warp == 6) {
-    // ===================== Filter producer (bulk copies of packed blocks) =====================
-    if (lane == 0) {
-      uint32_t it = 0, s = 0, ph = 0;
-      bool ok = true;
+  } else if (warp == 6 || warp == 8) {
+    // ===================== Filter producers (bulk copies of packed blocks) =====================
+    const uint32_t f_prod = p.f_stages >= 2 ? uint32_t(kProducersPerRing) : 1u;
+    if (lane == 0 && ((warp == 6) ? 0u : 1u) < f_prod) {
+      const uint32_t me = (warp == 6) ? 0u : 1u;
       const uint32_t n_st = uint32_t(p.f_stages);
+      uint32_t seq = 0, s = 0, ph = 0;
+      bool ok = true;
       for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
         const int kt = tile % p.tiles_k;
         const uint8_t* src = packed_filter + (size_t)kt * p.units * kPackedBlockBytes;
-        for (int left = p.units; left > 0; left -= p.uf, ++it) {
+        for (int left = p.units; left > 0; left -= p.uf, ++seq) {
           const uint32_t bytes = uint32_t(left < p.uf ? left : p.uf) * kPackedBlockBytes;
-          if (!mbar_wait(bar_fempty + 8u * s, ph ^ 1u, abort_flag, status, kStatFilterWait,
-                         limit)) {
-            ok = false;
-            break;
+          if ((seq & (f_prod - 1u)) == me) {
+            if (!mbar_wait(bar_fempty + 8u * s, ph ^ 1u, abort_flag, status, kStatFilterWait,
+                           limit)) {
+              ok = false;
+              break;
+            }
+            const uint32_t full = bar_ffull + 8u * s;
+            mbar_arrive_expect_tx(full, bytes);
+            bulk_load(filt_ring + s * p.filt_stage_bytes, src, bytes, full);
           }
-          const uint32_t full = bar_ffull + 8u * s;
-          mbar_arrive_expect_tx(full, bytes);
-          bulk_load(filt_ring + s * p.filt_stage_bytes, src, bytes, full);
           src += bytes;
           if (++s == n_st) {
             s = 0;
@@ -454,151 +653,26 @@ __global__ void __launch_bounds__(kThreads, 1)
           }
         }
       }
-      CCONV_TRACE(4);
-      drain_ring(bar_ffull, it, n_st, status, limit);
+      if (me == 0) CCONV_TRACE(4);
+      drain_ring(bar_ffull, seq, n_st, status, limit);
     }
   } else if (warp == 1) {
     // ===================== MMA issuer =====================
-    // The whole warp walks the loops (descriptor arithmetic stays warp-uniform) and one fixed lane
-    // issues the tcgen05 instructions.  Per unit the loop does one table read (the tap's halo
-    // offset), b_h MMAs and a few counter updates.
-    {
-      const bool leader = elect_one();
-      uint32_t is = 0, iph = 0, fs = 0, fph = 0, abuf = 0, aph = 0;
-      bool ok = true, first_tile = true;
-      const int R = p.R, S = p.S, units = p.units, units_per_img = p.units_per_img;
-      const uint32_t slab16 = p.slab_bytes >> 4, row16 = uint32_t(p.halo_w) * slab16;
-      const bool taps9 = (R == 3 && S == 3);
-      uint32_t off9[9];  // halo offset of tap (r, s) = r*3 + s, in 16 B units
-#pragma unroll
-      for (int t = 0; t < 9; ++t) off9[t] = uint32_t(t % 3) * row16 + uint32_t(t / 3) * slab16;
-      // Descriptors differ only in their low word (start address >> 4, bits [0,14)); all
-      // per-instruction arithmetic below is on 32-bit "address >> 4" quantities.
-      const uint32_t a_lo0 = uint32_t(p.a_desc), a_hi = uint32_t(p.a_desc >> 32);
-      const uint32_t b_lo0 = uint32_t(p.b_desc), b_hi = uint32_t(p.b_desc >> 32);
-      const uint32_t hstep16 = uint32_t(p.sh * p.halo_w) * (p.slab_bytes >> 4);  // next output row
-      const uint32_t kstep16 = p.b_kstep_bytes >> 4;
-      const uint32_t img16 = p.img_stage_bytes >> 4, filt16 = p.filt_stage_bytes >> 4;
-      const uint32_t img_ring16 = img_ring >> 4, filt_ring16 = filt_ring >> 4;
-      const uint32_t idesc = p.idesc, n_mma = uint32_t(p.n_mma);
-      const uint32_t n_ist = uint32_t(p.i_stages), n_fst = uint32_t(p.f_stages);
-      const int bh = p.bh, uf = p.uf;
-      for (int tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
-        if (!mbar_wait_warp(bar_tempty + 8u * abuf, aph ^ 1u, abort_flag, status, kStatMmaWaitTmem,
-                            limit))
-          break;
-        tc_fence_after();
-        const uint32_t d_base = tmem_base + abuf * uint32_t(p.acc_cols);
-        uint32_t acc = 0;
-        int f_left = 0, i_left = 0;   // units left in the current Filter / Image stage
-        int sx = 0, tap_r = 0;
-        uint32_t tap_off = 0, col_off = 0;  // halo offset of the current tap, in 16 B units
-        uint32_t a16 = 0, img_kk16 = 0;
-        int units_left = units;
-        while (units_left > 0) {
-          if (i_left == 0) {
-            if (!mbar_wait_warp(bar_ifull + 8u * is, iph, abort_flag, status, kStatMmaWaitFull,
-                                limit)) {
-              ok = false;
-              break;
-            }
-            tc_fence_after();
-            img_kk16 = img_ring16 + is * img16;
-            i_left = units_left < units_per_img ? units_left : units_per_img;
-          }
-          if (f_left == 0) {
-            if (!mbar_wait_warp(bar_ffull + 8u * fs, fph, abort_flag, status, kStatMmaWaitFull,
-                                limit)) {
-              ok = false;
-              break;
-            }
-            tc_fence_after();
-            a16 = filt_ring16 + fs * filt16;
-            f_left = units_left < uf ? units_left : uf;
-          }
-          // Issue every unit both resident stages cover, with no barrier work in between.
-          // Descriptors are built by the whole warp (uniform values); only the issue is elected.
-          const int n = i_left < f_left ? i_left : f_left;
-          if (taps9 && sx == 0 && tap_r == 0 && n >= 9) {
-            // 3x3 filters: whole 16-channel steps, the nine tap offsets held in registers
-            for (int done = 0; done + 9 <= n; done += 9) {
-#pragma unroll
-              for (int t = 0; t < 9; ++t) {
-                const uint64_t a_desc = (uint64_t(a_hi) << 32) | (a_lo0 | (a16 + uint32_t(t) * 256u));
-                uint32_t b16 = img_kk16 + off9[t], d = d_base;
-                for (int hh = 0; hh < bh; ++hh, b16 += hstep16, d += n_mma)
-                  umma_bf16_if(leader, d, a_desc, (uint64_t(b_hi) << 32) | (b_lo0 | b16), idesc, acc);
-                acc = 1;
-              }
-              a16 += 9u * 256u;
-              img_kk16 += kstep16;
-            }
-            const int issued = n - n % 9;
-            i_left -= issued;
-            f_left -= issued;
-            units_left -= issued;
-          } else {
-            for (int j = 0; j < n; ++j) {
-              const uint64_t a_desc = (uint64_t(a_hi) << 32) | (a_lo0 | a16);
-              uint32_t b16 = img_kk16 + tap_off, d = d_base;
-              for (int hh = 0; hh < bh; ++hh, b16 += hstep16, d += n_mma)
-                umma_bf16_if(leader, d, a_desc, (uint64_t(b_hi) << 32) | (b_lo0 | b16), idesc, acc);
-              acc = 1;
-              a16 += kPackedBlockBytes >> 4;
-              // next tap: one halo row down; after S rows, one pixel to the right; after R*S taps,
-              // the next 16 channels of the same Image stage
-              tap_off += row16;
-              if (++sx == S) {
-                sx = 0;
-                col_off += slab16;
-                tap_off = col_off;
-                if (++tap_r == R) {
-                  tap_r = 0;
-                  col_off = 0;
-                  tap_off = 0;
-                  img_kk16 += kstep16;
-                }
-              }
-            }
-            i_left -= n;
-            f_left -= n;
-            units_left -= n;
-          }
-          if (f_left == 0) {
-            // the Filter stage is free once the MMAs issued so far have read it
-            if (leader) umma_commit(bar_fempty + 8u * fs);
-            if (++fs == n_fst) {
-              fs = 0;
-              fph ^= 1u;
-            }
-          }
-          if (i_left == 0) {
-            if (leader) umma_commit(bar_iempty + 8u * is);
-            if (++is == n_ist) {
-              is = 0;
-              iph ^= 1u;
-            }
-          }
-        }
-        if (!ok) break;
-        if (leader) umma_commit(bar_tfull + 8u * abuf);  // accumulator complete
-        if (first_tile && lane == 0) CCONV_TRACE(6);
-        first_tile = false;
-        if (++abuf == uint32_t(p.acc_bufs)) {
-          abuf = 0;
-          aph ^= 1u;
-        }
-      }
-      // All MMAs must have retired before TMEM is released.
-      if (lane == 0) CCONV_TRACE(7);
-      if (leader) umma_commit(bar_drain);
-      const uint64_t t0 = globaltimer_ns();
-      while (!mbar_try_wait(bar_drain, 0)) {
-        if (globaltimer_ns() - t0 > limit) {
-          atomicOr(status, kStatDrainWait);
-          break;
-        }
-      }
+    const MmaCtx cx{bar_ifull, bar_iempty, bar_ffull, bar_fempty, bar_tfull, bar_tempty, bar_drain,
+                    img_ring, filt_ring, tmem_base, abort_flag, status, limit};
+    const int taps = p.R * p.S;
+    // Straight-line issue code for the common shapes (a loop branch costs a lone warp ~20 cycles):
+    // b_h in {1,2} and 1x1 / 3x3 filters; everything else takes the generic loops.
+    if (p.R == 3 && p.S == 3) {
+      if (p.bh == 1) mma_role<1, 9>(p, cx);
+      else if (p.bh == 2) mma_role<2, 9>(p, cx);
+      else mma_role<0, 9>(p, cx);
+    } else if (taps == 1) {
+      if (p.bh == 1) mma_role<1, 1>(p, cx);
+      else if (p.bh == 2) mma_role<2, 1>(p, cx);
+      else mma_role<0, 1>(p, cx);
+    } else {
+      mma_role<0, 0>(p, cx);
     }
   } else {
     // ===================== epilogue: TMEM -> registers -> Out =====================
@@ -629,22 +703,25 @@ __global__ void __launch_bounds__(kThreads, 1)
             tmem_ld_32x32b_x32(t_base + uint32_t(hh * p.n_mma + ww * p.bb + ch * 32), v);
             tmem_ld_wait();
             if (valid) {
-              uint4* dst = reinterpret_cast<uint4*>(
-                  out + (((long long)k * p.H + h) * p.W + w) * p.B + b0 + ch * 32);
+              // 32 consecutive images of one (k, h, w): 64 B (bf16) or 128 B (fp32), written as
+              // whole 32-byte sectors
+              OutT* dst = out + (((long long)k * p.H + h) * p.W + w) * p.B + b0 + ch * 32;
               if constexpr (sizeof(OutT) == 4) {
 #pragma unroll
-                for (int j = 0; j < 8; ++j)
-                  dst[j] = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                for (int j = 0; j < 4; ++j)
+                  st_global_v8(dst + 8 * j, v[8 * j], v[8 * j + 1], v[8 * j + 2], v[8 * j + 3],
+                               v[8 * j + 4], v[8 * j + 5], v[8 * j + 6], v[8 * j + 7]);
               } else {
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                  uint4 o;
-                  o.x = pack_bf16x2(v[8 * j + 0], v[8 * j + 1]);
-                  o.y = pack_bf16x2(v[8 * j + 2], v[8 * j + 3]);
-                  o.z = pack_bf16x2(v[8 * j + 4], v[8 * j + 5]);
-                  o.w = pack_bf16x2(v[8 * j + 6], v[8 * j + 7]);
-                  dst[j] = o;
-                }
+                for (int j = 0; j < 2; ++j)
+                  st_global_v8(dst + 16 * j, pack_bf16x2(v[16 * j + 0], v[16 * j + 1]),
+                               pack_bf16x2(v[16 * j + 2], v[16 * j + 3]),
+                               pack_bf16x2(v[16 * j + 4], v[16 * j + 5]),
+                               pack_bf16x2(v[16 * j + 6], v[16 * j + 7]),
+                               pack_bf16x2(v[16 * j + 8], v[16 * j + 9]),
+                               pack_bf16x2(v[16 * j + 10], v[16 * j + 11]),
+                               pack_bf16x2(v[16 * j + 12], v[16 * j + 13]),
+                               pack_bf16x2(v[16 * j + 14], v[16 * j + 15]));
               }
             }
           }

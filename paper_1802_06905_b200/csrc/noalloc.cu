@@ -77,8 +77,8 @@ extern "C" int cconv_forward_noalloc(const void* Image, const void* Filter, void
   const Dims d{B, C, K, W, H, R, S, sw, sh};
   if (!d.positive()) return CCONV_EINVAL;
   if (out_dtype != CCONV_OUT_BF16 && out_dtype != CCONV_OUT_F32) return CCONV_EINVAL;
-  if ((reinterpret_cast<uintptr_t>(Image) | reinterpret_cast<uintptr_t>(Filter) |
-       reinterpret_cast<uintptr_t>(Out)) & 15u)
+  if (((reinterpret_cast<uintptr_t>(Image) | reinterpret_cast<uintptr_t>(Filter)) & 15u) ||
+      (reinterpret_cast<uintptr_t>(Out) & 31u))
     return CCONV_EINVAL;
   if (!halo_supported(d, nullptr)) return CCONV_EUNSUPPORTED;
 

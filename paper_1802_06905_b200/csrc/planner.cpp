@@ -133,7 +133,7 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[5], HaloT
   //    (8 TB/s in aggregate), at most ~60 B/clk for one SM -- this, the paper's "words moved into
   //    fast memory", is what binds the large 3x3 shapes;
   //  * one elected thread issues a unit (b_h MMAs) in about 130 + 60*b_h cycles at best;
-  //  * the epilogue drains an accumulator at about 24 cycles per TMEM column.
+  //  * the epilogue drains an accumulator at about 14 cycles per TMEM column.
   const double l2_total_bytes_per_clk = 30.0 * m.sm_count, l2_sm_max_bytes_per_clk = 60.0;
   const int RS = d.R * d.S;
   const int c16 = (d.C + 15) / 16;
@@ -196,7 +196,7 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[5], HaloT
           const double l2_rate = std::min(l2_sm_max_bytes_per_clk, l2_total_bytes_per_clk / t.grid);
           // 64-byte rows (bb = 32) use the copy engine and the swizzle half as well as 128-byte rows
           const double cyc_copy = tile_bytes / l2_rate * (bb == 32 ? 1.08 : 1.0);
-          const double cyc_epi = 24.0 * acc_cols;
+          const double cyc_epi = 14.0 * acc_cols;
           double tile_cyc = (t.acc_bufs == 2) ? std::max({cyc_mma, cyc_copy, cyc_epi})
                                               : std::max(cyc_mma, cyc_copy) + cyc_epi;
           if (t.i_stages == 1) tile_cyc = cyc_mma + cyc_copy + cyc_epi;
