@@ -302,6 +302,9 @@ __device__ __forceinline__ void drain_ring(uint32_t bar_full0, uint32_t it, uint
 __global__ void __launch_bounds__(256)
     cconv_pack_filter_kernel(const __nv_bfloat16* __restrict__ filter, uint4* __restrict__ packed,
                              Dims d, int c16, long long slots) {
+  // Let the convolution kernel (launched with programmatic stream serialization) start its set-up
+  // and its Image copies while this kernel runs; it waits for our stores before reading them.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const long long slot = blockIdx.x * (long long)blockDim.x + threadIdx.x;
   if (slot >= slots) return;
   const int RS = d.R * d.S;
@@ -631,6 +634,8 @@ __global__ void __launch_bounds__(kThreads, 1)
       const uint32_t n_st = uint32_t(p.f_stages);
       uint32_t seq = 0, s = 0, ph = 0;
       bool ok = true;
+      // the packed Filter is written by the kernel launched just before this one
+      asm volatile("griddepcontrol.wait;" ::: "memory");
       for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
         const int kt = tile % p.tiles_k;
         const uint8_t* src = packed_filter + (size_t)kt * p.units * kPackedBlockBytes;
@@ -763,13 +768,23 @@ cudaError_t launch_halo(const CUtensorMap& tm_image, const void* packed_filter, 
                         bool out_f32, const HaloKernelParams& p, int grid, int smem_bytes,
                         int* status, cudaStream_t stream) {
   const uint8_t* pf = static_cast<const uint8_t*>(packed_filter);
+  // Programmatic dependent launch: this kernel may begin while the Filter-packing kernel in front
+  // of it is still running; only its Filter producers wait for that kernel's results.
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(unsigned(grid));
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = size_t(smem_bytes);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
   if (out_f32)
-    cconv_halo_kernel<float><<<grid, kThreads, smem_bytes, stream>>>(
-        tm_image, pf, static_cast<float*>(out), p, status);
-  else
-    cconv_halo_kernel<__nv_bfloat16><<<grid, kThreads, smem_bytes, stream>>>(
-        tm_image, pf, static_cast<__nv_bfloat16*>(out), p, status);
-  return cudaGetLastError();
+    return cudaLaunchKernelEx(&cfg, cconv_halo_kernel<float>, tm_image, pf,
+                              static_cast<float*>(out), p, status);
+  return cudaLaunchKernelEx(&cfg, cconv_halo_kernel<__nv_bfloat16>, tm_image, pf,
+                            static_cast<__nv_bfloat16*>(out), p, status);
 }
 
 }  // namespace cconv
