@@ -50,6 +50,8 @@ struct cconv_plan {
   double lp_G = 0, lp_words = 0;
   HaloTile tile{};
   HaloKernelParams kp{};
+  StemTile stile{};
+  StemKernelParams skp{};
   int* d_status = nullptr;
   void* d_packed = nullptr;  // scratch: the packed Filter (rewritten by every forward call)
   unsigned long long* d_trace = nullptr;  // diagnostics: [grid][16] device time stamps
@@ -114,7 +116,7 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
   *plan_out = nullptr;
   const Dims d{B, C, K, W, H, R, S, sw, sh};
   if (!d.positive()) return CCONV_EINVAL;
-  if (variant < CCONV_VARIANT_AUTO || variant > CCONV_VARIANT_HALO) return CCONV_EINVAL;
+  if (variant < CCONV_VARIANT_AUTO || variant > CCONV_VARIANT_STEM) return CCONV_EINVAL;
   if (out_dtype != CCONV_OUT_BF16 && out_dtype != CCONV_OUT_F32) return CCONV_EINVAL;
   // element counts must fit the kernels' index arithmetic
   const double lim = 9.0e18;
@@ -137,7 +139,7 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
     pl->m.sm_count = prop.multiProcessorCount;
     pl->m.smem_optin_bytes = int(prop.sharedMemPerBlockOptin);
     pl->m.l2_bytes = prop.l2CacheSize;
-    if (prop.major != 10 && variant == CCONV_VARIANT_HALO) {
+    if (prop.major != 10 && variant >= CCONV_VARIANT_HALO) {
       delete pl;
       return CCONV_EUNSUPPORTED;
     }
@@ -150,16 +152,23 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
   if (const char* f = std::getenv("CCONV_FORCE_TILE"))
     std::sscanf(f, "%d,%d,%d,%d,%d", &force[0], &force[1], &force[2], &force[3], &force[4]);
   const int env_variant = env_int("CCONV_VARIANT", 0);
-  if (variant == CCONV_VARIANT_AUTO && env_variant >= 1 && env_variant <= 2) variant = env_variant;
+  if (variant == CCONV_VARIANT_AUTO && env_variant >= 1 && env_variant <= 3) variant = env_variant;
 
   const bool halo_ok = halo_supported(d, nullptr) && choose_halo_tile(d, pl->m, force, &pl->tile);
-  if (variant == CCONV_VARIANT_HALO && !halo_ok) {
+  const bool stem_ok = choose_stem_tile(d, pl->m, &pl->stile);
+  if ((variant == CCONV_VARIANT_HALO && !halo_ok) || (variant == CCONV_VARIANT_STEM && !stem_ok)) {
     delete pl;
     return CCONV_EUNSUPPORTED;
   }
-  if (variant == CCONV_VARIANT_AUTO) variant = halo_ok ? CCONV_VARIANT_HALO : CCONV_VARIANT_SIMT;
+  if (variant == CCONV_VARIANT_AUTO) {
+    // Fewer than 8 channels: a 16-channel K step of the halo kernel is mostly zero padding, so
+    // the kernel that folds (s, c) into the contraction wins where it applies.
+    if (stem_ok && d.C < 8) variant = CCONV_VARIANT_STEM;
+    else variant = halo_ok ? CCONV_VARIANT_HALO : CCONV_VARIANT_SIMT;
+  }
   pl->variant = variant;
   if (variant == CCONV_VARIANT_HALO) build_halo_params(pl->d, pl->tile, &pl->kp);
+  if (variant == CCONV_VARIANT_STEM) build_stem_params(pl->d, pl->stile, &pl->skp);
 
   if (device >= 0) {
     int prev = 0;
@@ -171,6 +180,10 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
       e = halo_kernel_prepare(pl->tile.smem_bytes);
     if (e == cudaSuccess && variant == CCONV_VARIANT_HALO)
       e = cudaMalloc(&pl->d_packed, size_t(pl->tile.packed_filter_bytes));
+    if (e == cudaSuccess && variant == CCONV_VARIANT_STEM)
+      e = stem_kernel_prepare(pl->stile.smem_bytes);
+    if (e == cudaSuccess && variant == CCONV_VARIANT_STEM)
+      e = cudaMalloc(&pl->d_packed, size_t(pl->stile.packed_filter_bytes));
     if (e == cudaSuccess && variant == CCONV_VARIANT_HALO && env_int("CCONV_TRACE", 0)) {
       e = cudaMalloc(reinterpret_cast<void**>(&pl->d_trace), size_t(pl->tile.grid + 16) * 16 * 8);
       if (e == cudaSuccess) e = cudaMemset(pl->d_trace, 0, size_t(pl->tile.grid + 16) * 16 * 8);
@@ -184,7 +197,14 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
       return cuda_fail(e, "plan device setup");
     }
   }
-  if (env_int("CCONV_LOG", 0)) {
+  if (env_int("CCONV_LOG", 0) && variant == CCONV_VARIANT_STEM) {
+    const StemTile& t = pl->stile;
+    std::fprintf(stderr,
+                 "[cconv] B%d C%d K%d W%d H%d R%d S%d s%dx%d variant=3 tile bw=%d kw=%d ndelta=%d "
+                 "n_out=%d i_stages=%d tmem=%d tiles=%lld grid=%d smem=%d filt=%u\n",
+                 B, C, K, W, H, R, S, sw, sh, t.bw, t.kw, t.ndelta, t.n_out, t.i_stages, t.tmem_cols,
+                 t.tiles, t.grid, t.smem_bytes, t.filt_bytes);
+  } else if (env_int("CCONV_LOG", 0)) {
     const HaloTile& t = pl->tile;
     std::fprintf(stderr,
                  "[cconv] B%d C%d K%d W%d H%d R%d S%d s%dx%d variant=%d tile bb=%d bw=%d bh=%d "
@@ -217,6 +237,15 @@ int cconv_plan_info_get(const cconv_plan* pl, cconv_plan_info* o) {
   const Dims& d = pl->d;
   o->compulsory_words =
       double(d.Wi()) * d.Hi() * d.C * d.B + double(d.K) * d.R * d.S * d.C + double(d.K) * d.H * d.W * d.B;
+  if (pl->variant == CCONV_VARIANT_STEM) {
+    const StemTile& t = pl->stile;
+    o->bb = 64; o->bc = d.C; o->bk = t.n_out; o->bw = t.bw; o->bh = 1;
+    o->halo_w = t.halo_w; o->halo_h = d.S;
+    o->stages = t.i_stages; o->filter_stages = 1; o->grid = t.grid; o->tiles = int(t.tiles);
+    o->smem_bytes = t.smem_bytes; o->tmem_cols = t.tmem_cols;
+    o->tile_words_smem = t.words_smem;
+    o->scratch_bytes = double(t.packed_filter_bytes);
+  }
   if (pl->variant == CCONV_VARIANT_HALO) {
     const HaloTile& t = pl->tile;
     o->bb = t.bb; o->bc = t.bc; o->bk = t.bk; o->bw = t.bw; o->bh = t.bh;
@@ -262,11 +291,20 @@ int cconv_forward_planned(const cconv_plan* pl, const void* Image, const void* F
     // the tensor map is rebuilt only when the Image pointer changes
     std::lock_guard<std::mutex> lk(pl->mu);
     if (pl->tm_image_ptr != Image) {
-      int rc = encode_image_map(pl->d, pl->tile, Image, &pl->tm_image);
+      int rc = pl->variant == CCONV_VARIANT_STEM
+                   ? encode_stem_image_map(pl->d, pl->stile, Image, &pl->tm_image)
+                   : encode_image_map(pl->d, pl->tile, Image, &pl->tm_image);
       if (rc != CCONV_OK) return rc;
       pl->tm_image_ptr = Image;
     }
     tmi = pl->tm_image;
+  }
+  if (pl->variant == CCONV_VARIANT_STEM) {
+    cudaError_t es = launch_pack_filter_stem(Filter, pl->d_packed, pl->d, pl->skp, stream);
+    if (es != cudaSuccess) return cuda_fail(es, "launch_pack_filter_stem");
+    es = launch_stem(tmi, pl->d_packed, Out, pl->out_dtype == CCONV_OUT_F32, pl->skp,
+                     pl->stile.grid, pl->stile.smem_bytes, pl->d_status, stream);
+    return es == cudaSuccess ? CCONV_OK : cuda_fail(es, "launch_stem");
   }
   cudaError_t e = launch_pack_filter(Filter, pl->d_packed, pl->d, pl->tile.c16, pl->tile.tiles_k,
                                      stream);

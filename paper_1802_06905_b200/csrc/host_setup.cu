@@ -117,6 +117,56 @@ int encode_image_map(const Dims& d, const HaloTile& t, const void* image, CUtens
   return CCONV_OK;
 }
 
+void build_stem_params(const Dims& d, const StemTile& t, StemKernelParams* out) {
+  StemKernelParams& p = *out;
+  p.K = d.K; p.H = d.H; p.W = d.W; p.B = d.B; p.C = d.C;
+  p.R = d.R; p.S = d.S; p.sw = d.sw; p.sh = d.sh;
+  p.bw = t.bw; p.kw = t.kw; p.khalves = t.khalves; p.dstep = t.dstep; p.ndelta = t.ndelta;
+  p.halo_w = t.halo_w; p.n_out = t.n_out;
+  p.tiles_w = t.tiles_w; p.tiles_b = t.tiles_b; p.total_tiles = int(t.tiles);
+  p.i_stages = t.i_stages;
+  p.acc_cols = (t.bw / 2) * t.n_out;
+  p.tmem_cols = t.tmem_cols;
+  p.img_stage_bytes = t.img_stage_bytes;
+  p.filt_bytes = t.filt_bytes;
+  p.xslab_bytes = uint32_t(t.kw) * 128u;       // one Image column: kw rows of 64 images
+  p.fblock_bytes = uint32_t(t.n_out) * 32u;    // one Filter block: n_out x 16
+  // instruction descriptor: D=f32, A=B=bf16, A MN-major [15]=1, B K-major [16]=0, N = n_out, M = 128
+  p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (0u << 16) |
+            (uint32_t(t.n_out >> 3) << 17) | (uint32_t(128 >> 4) << 24);
+  // A = Image window [16 rows][2 pixels x 64 images], MN-major, 128-byte swizzle (layout type 2):
+  // SBO = 1024 B from one group of 8 rows to the next; LBO = from pixel 1's 64 images to pixel 2's,
+  // sw Image columns further.
+  p.a_desc = make_smem_desc(uint32_t(d.sw) * p.xslab_bytes, 1024, 2);
+  // B = Filter block [n_out rows][16], K-major, no swizzle: LBO = 128 B, SBO = 256 B.
+  p.b_desc = make_smem_desc(128, 256, 0);
+  p.wait_limit_ns = uint64_t(env_int("CCONV_WAIT_LIMIT_MS", 1000)) * 1000000ull;
+  p.trace = nullptr;
+}
+
+int encode_stem_image_map(const Dims& d, const StemTile& t, const void* image, CUtensorMap* tm) {
+  EncodeTiledFn enc = encode_tiled_fn();
+  if (!enc) {
+    set_last_cuda_error("cuTensorMapEncodeTiled is not available from this driver");
+    return CCONV_ECUDA;
+  }
+  // Image[x][y][c][b] viewed as (b, m, x) with m = y*C + c: for a fixed x the (y,c) rows are
+  // contiguous, B images each.  A box lands as [x][m][64 images].
+  const cuuint64_t dims[3] = {cuuint64_t(d.B), cuuint64_t(d.Hi()) * d.C, cuuint64_t(d.Wi())};
+  const cuuint64_t strides[2] = {cuuint64_t(d.B) * 2, cuuint64_t(d.Hi()) * d.C * d.B * 2};
+  const cuuint32_t box[3] = {64u, cuuint32_t(t.kw), cuuint32_t(t.halo_w)};
+  const cuuint32_t es[3] = {1, 1, 1};
+  CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(image), dims, strides,
+                   box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    set_last_cuda_error("cuTensorMapEncodeTiled(Image, stem view) failed with CUresult " +
+                        std::to_string(int(r)));
+    return CCONV_ECUDA;
+  }
+  return CCONV_OK;
+}
+
 void set_last_cuda_error(const std::string& msg) { g_last_cuda_error = msg; }
 const char* last_cuda_error() { return g_last_cuda_error.c_str(); }
 

@@ -20,4 +20,8 @@ void build_halo_params(const Dims& d, const HaloTile& t, HaloKernelParams* p);
 // (CCONV_ECUDA) with the last-error text set.  A pure host-side encode.
 int encode_image_map(const Dims& d, const HaloTile& t, const void* image, CUtensorMap* tm);
 
+// The same two pieces for the small-C ("stem") kernel: Image viewed as (b, m = y*C + c, x).
+void build_stem_params(const Dims& d, const StemTile& t, StemKernelParams* p);
+int encode_stem_image_map(const Dims& d, const StemTile& t, const void* image, CUtensorMap* tm);
+
 }  // namespace cconv

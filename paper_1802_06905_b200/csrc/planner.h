@@ -56,6 +56,19 @@ struct HaloTile {
   double words_smem = 0;   // words staged into shared memory over the whole problem + |Out|
 };
 
+// Tile of the small-C ("stem") kernel: one output row, bw pixels, all K (<= 256) channels, 64 images.
+struct StemTile {
+  int bw = 0, kw = 0, khalves = 0, dstep = 0, ndelta = 0, halo_w = 0, n_out = 0;
+  int i_stages = 2, tmem_cols = 0;
+  int tiles_w = 0, tiles_b = 0;
+  long long tiles = 0;
+  int grid = 0;
+  uint32_t img_stage_bytes = 0, filt_bytes = 0;
+  long long packed_filter_bytes = 0;
+  int smem_bytes = 0;
+  double words_smem = 0;
+};
+
 void theorem1_terms(const Dims& d, double M, double t[5]);
 
 // Dense primal simplex on the LP of Section 5 in log_M space.  tiles[9] in the order
@@ -68,5 +81,9 @@ bool halo_supported(const Dims& d, const char** why);
 // Enumerate legal tiles and keep the one with the least estimated time (ties: fewer staged words).
 // `force` may carry "bw,bh,bc,stages,bb" (0 = free) from the CCONV_FORCE_TILE environment variable.
 bool choose_halo_tile(const Dims& d, const Machine& m, const int force[5], HaloTile* out);
+
+// The stem kernel needs B % 64 == 0, K <= 256, and the shifted (s,c) window, the resident Filter
+// and two Image stages to fit in shared memory.
+bool choose_stem_tile(const Dims& d, const Machine& m, StemTile* out);
 
 }  // namespace cconv

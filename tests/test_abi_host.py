@@ -125,6 +125,10 @@ def test_inspection_plans_are_hardware_legal():
             assert info["scratch_bytes"] == -(-cfg.K // 128) * units * 4096
             # the staged words can never undercut the bound at the shared-memory size
             assert info["tile_words_smem"] >= max(exp_terms) * 0.999 or max(exp_terms) < info["M_words"]
+        elif info["variant"] == binding.VARIANT_STEM:
+            assert cfg.B % 64 == 0 and cfg.C < 8 and cfg.K <= 256
+            assert info["bw"] % 2 == 0 and info["bw"] // 2 * info["bk"] * 2 <= 512   # two TMEM buffers
+            assert info["smem_bytes"] <= 232448 and info["stages"] >= 2
         else:
             assert info["variant"] == binding.VARIANT_SIMT
         # forward on an inspection plan is refused on the host, before any launch

@@ -32,6 +32,8 @@ def test_config_full_parity(name, out_dtype):
     info = check_full(BY[name], out_dtype=out_dtype)
     if name in ("cfg2_resnet_3x3", "cfg4_pointwise_1x1"):
         assert info["variant"] == binding.VARIANT_HALO     # the tensor-core path is the one that ran
+    if name == "cfg3_stem_7x7_s2":
+        assert info["variant"] == binding.VARIANT_STEM
 
 
 @pytest.mark.parametrize("out_dtype", DTYPES, ids=DT_IDS)
@@ -101,6 +103,24 @@ HALO_SHAPES = [
 def test_halo_shapes(c, out_dtype):
     info = check_full(c, variant=binding.VARIANT_HALO, out_dtype=out_dtype)
     assert info["variant"] == binding.VARIANT_HALO
+
+
+# ---- small-C tensor-core kernel: (s,c) folded into the contraction ----------------------------------
+
+STEM_SHAPES = [
+    cs("st_c3_7x7_s2", 64, 3, 64, 20, 18, 7, 7, 2, 2),      # four window offsets (sh*C = 6)
+    cs("st_c4_k40", 64, 4, 40, 9, 6, 3, 3),                 # odd W: ragged pixel pair; K < 64
+    cs("st_c1", 128, 1, 16, 10, 7, 5, 5, 1, 2),             # two batch tiles, one channel
+    cs("st_c6_s3", 64, 6, 100, 7, 5, 3, 4, 3, 1),           # K = 100 -> N = 112; sw = 3
+    cs("st_c2_wide", 64, 2, 24, 33, 3, 2, 9, 2, 1),         # S*C = 18 with offsets 0..6
+]
+
+
+@pytest.mark.parametrize("out_dtype", DTYPES, ids=DT_IDS)
+@pytest.mark.parametrize("c", STEM_SHAPES, ids=lambda c: c.name)
+def test_stem_shapes(c, out_dtype):
+    info = check_full(c, variant=binding.VARIANT_STEM, out_dtype=out_dtype)
+    assert info["variant"] == binding.VARIANT_STEM
 
 
 def test_halo_matches_simt_kernel_on_device():
