@@ -212,12 +212,13 @@ def roofline_for(cfg, info, secs_per_launch, peaks, binding):
     """Roofline of the dominant kernel: tensor-bound where the tcgen05 kernel ran (dense
     contraction), HBM-bound for the CUDA-core kernel (reported against compulsory bytes)."""
     traffic = dram_traffic_from_profiles(cfg.name)
-    if info["variant"] == binding.VARIANT_HALO:
+    if info["variant"] in (binding.VARIANT_HALO, binding.VARIANT_STEM):
         ach = cfg.flops / secs_per_launch / 1e12
         peak = peaks["bf16_tflops"]
+        kernel = "cconv_halo_kernel" if info["variant"] == binding.VARIANT_HALO else "cconv_stem_kernel"
         return {"bound": "tensor", "achieved": ach, "peak": peak, "unit": "TFLOP/s",
                 "frac": ach / peak, "traffic": traffic, "peak_source": peaks["source"],
-                "kernel": "cconv_halo_kernel"}
+                "kernel": kernel}
     byts = 2.0 * info["compulsory_words"]
     ach = byts / secs_per_launch / 1e9
     return {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",

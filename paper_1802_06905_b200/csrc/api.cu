@@ -63,6 +63,8 @@ struct cconv_plan {
   mutable std::mutex mu;
   mutable const void* tm_image_ptr = nullptr;
   mutable CUtensorMap tm_image{};
+  mutable const void* tm_out_ptr = nullptr;
+  mutable CUtensorMap tm_out{};  // stem kernel, bf16 Out only
 };
 
 namespace {
@@ -300,9 +302,20 @@ int cconv_forward_planned(const cconv_plan* pl, const void* Image, const void* F
     tmi = pl->tm_image;
   }
   if (pl->variant == CCONV_VARIANT_STEM) {
+    CUtensorMap tmo;
+    {
+      std::lock_guard<std::mutex> lk(pl->mu);
+      if (pl->tm_out_ptr != Out) {
+        // fp32 Out is stored without TMA; the map is then built over the same bytes and not used
+        int rc = encode_stem_out_map(pl->d, Out, &pl->tm_out);
+        if (rc != CCONV_OK) return rc;
+        pl->tm_out_ptr = Out;
+      }
+      tmo = pl->tm_out;
+    }
     cudaError_t es = launch_pack_filter_stem(Filter, pl->d_packed, pl->d, pl->skp, stream);
     if (es != cudaSuccess) return cuda_fail(es, "launch_pack_filter_stem");
-    es = launch_stem(tmi, pl->d_packed, Out, pl->out_dtype == CCONV_OUT_F32, pl->skp,
+    es = launch_stem(tmi, tmo, pl->d_packed, Out, pl->out_dtype == CCONV_OUT_F32, pl->skp,
                      pl->stile.grid, pl->stile.smem_bytes, pl->d_status, stream);
     return es == cudaSuccess ? CCONV_OK : cuda_fail(es, "launch_stem");
   }

@@ -167,6 +167,27 @@ int encode_stem_image_map(const Dims& d, const StemTile& t, const void* image, C
   return CCONV_OK;
 }
 
+int encode_stem_out_map(const Dims& d, void* out, CUtensorMap* tm) {
+  EncodeTiledFn enc = encode_tiled_fn();
+  if (!enc) {
+    set_last_cuda_error("cuTensorMapEncodeTiled is not available from this driver");
+    return CCONV_ECUDA;
+  }
+  const cuuint64_t dims[4] = {cuuint64_t(d.B), cuuint64_t(d.W), cuuint64_t(d.H), cuuint64_t(d.K)};
+  const cuuint64_t strides[3] = {cuuint64_t(d.B) * 2, cuuint64_t(d.W) * d.B * 2,
+                                 cuuint64_t(d.H) * d.W * d.B * 2};
+  const cuuint32_t box[4] = {64u, 1u, 1u, 32u};
+  const cuuint32_t es[4] = {1, 1, 1, 1};
+  CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, out, dims, strides, box, es,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                   CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    set_last_cuda_error("cuTensorMapEncodeTiled(Out) failed with CUresult " + std::to_string(int(r)));
+    return CCONV_ECUDA;
+  }
+  return CCONV_OK;
+}
+
 void set_last_cuda_error(const std::string& msg) { g_last_cuda_error = msg; }
 const char* last_cuda_error() { return g_last_cuda_error.c_str(); }
 

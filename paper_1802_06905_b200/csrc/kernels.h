@@ -81,7 +81,8 @@ cudaError_t launch_pack_filter(const void* filter, void* packed, const Dims& d, 
 cudaError_t launch_pack_filter_stem(const void* filter, void* packed, const Dims& d,
                                     const StemKernelParams& p, cudaStream_t stream);
 cudaError_t stem_kernel_prepare(int smem_bytes);
-cudaError_t launch_stem(const CUtensorMap& tm_image, const void* packed_filter, void* out,
+cudaError_t launch_stem(const CUtensorMap& tm_image, const CUtensorMap& tm_out,
+                        const void* packed_filter, void* out,
                         bool out_f32, const StemKernelParams& p, int grid, int smem_bytes,
                         int* status, cudaStream_t stream);
 

@@ -219,6 +219,8 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[5], HaloT
 }
 
 bool choose_stem_tile(const Dims& d, const Machine& m, StemTile* out) {
+  // two 4 KB buffers from which the epilogue's TMA stores read (one per pixel of a pair)
+  constexpr int kStemStagingBytes = 8192;
   if (d.B % 64 != 0 || d.K > 256) return false;
   const int reserve = 2048;
   const int cap = m.smem_optin_bytes - reserve;
@@ -251,11 +253,11 @@ bool choose_stem_tile(const Dims& d, const Machine& m, StemTile* out) {
     const int halo_w = d.sw * (bw - 1) + d.R;
     if (halo_w > 256) continue;
     const long long img = 1ll * halo_w * t.kw * 128;
-    if (2 * img + t.filt_bytes > cap) continue;
+    if (2 * img + t.filt_bytes + kStemStagingBytes > cap) continue;
     t.bw = bw;
     t.halo_w = halo_w;
     t.img_stage_bytes = uint32_t(img);
-    t.i_stages = int(std::min<long long>(4, (cap - t.filt_bytes) / img));
+    t.i_stages = int(std::min<long long>(4, (cap - t.filt_bytes - kStemStagingBytes) / img));
     found = true;
     break;
   }
@@ -268,7 +270,7 @@ bool choose_stem_tile(const Dims& d, const Machine& m, StemTile* out) {
   t.tiles = 1ll * t.tiles_b * d.H * t.tiles_w;
   if (t.tiles > 0x7fffffffll) return false;
   t.grid = int(std::min<long long>(t.tiles, m.sm_count));
-  t.smem_bytes = std::max(int(t.i_stages * t.img_stage_bytes + t.filt_bytes) + reserve, 117760);
+  t.smem_bytes = std::max(int(t.i_stages * t.img_stage_bytes + t.filt_bytes) + kStemStagingBytes + reserve, 117760);
   t.words_smem = double(t.tiles) * (t.img_stage_bytes / 2) + double(t.grid) * (t.filt_bytes / 2) +
                  double(d.K) * d.H * d.W * d.B;
   *out = t;

@@ -36,9 +36,32 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm,
       : "memory");
 }
 
-__device__ __forceinline__ void store_scalar(__nv_bfloat16* p, uint32_t f32_bits) {
-  *p = __float2bfloat16_rn(__uint_as_float(f32_bits));
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* tm, int c0, int c1, int c2, int c3,
+                                             uint32_t src) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%1, %2, %3, %4}], [%5];" ::
+          "l"(reinterpret_cast<uint64_t>(tm)),
+      "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(src)
+      : "memory");
 }
+__device__ __forceinline__ void bulk_commit() {
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// until the bulk stores issued so far by this thread have READ their shared-memory source
+__device__ __forceinline__ void bulk_wait_read_all() {
+  asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+}
+// until they have completed altogether
+__device__ __forceinline__ void bulk_wait_all() {
+  asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async_smem() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
 __device__ __forceinline__ void store_scalar(float* p, uint32_t f32_bits) {
   *p = __uint_as_float(f32_bits);
 }
@@ -104,13 +127,15 @@ cudaError_t launch_pack_filter_stem(const void* filter, void* packed, const Dims
 template <typename OutT>
 __global__ void __launch_bounds__(kStemThreads, 1)
     cconv_stem_kernel(const __grid_constant__ CUtensorMap tm_image,
+                      const __grid_constant__ CUtensorMap tm_out,
                       const uint8_t* __restrict__ packed_filter, OutT* __restrict__ out,
                       const StemKernelParams p, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t img_ring = smem0;
   const uint32_t filt_smem = img_ring + uint32_t(p.i_stages) * p.img_stage_bytes;
-  const uint32_t bars = filt_smem + p.filt_bytes;
+  const uint32_t stage_smem = filt_smem + p.filt_bytes;  // 2 x 4 KB: sources of the TMA stores
+  const uint32_t bars = stage_smem + 8192u;
   const uint32_t bar_ifull = bars;
   const uint32_t bar_iempty = bar_ifull + 8u * p.i_stages;
   const uint32_t bar_filt = bar_iempty + 8u * p.i_stages;
@@ -139,6 +164,7 @@ __global__ void __launch_bounds__(kStemThreads, 1)
     *abort_flag = 0;
     fence_barrier_init();
     prefetch_tensormap(&tm_image);
+    prefetch_tensormap(&tm_out);
   }
   if (warp == 1) {
     tmem_alloc(slot_addr, uint32_t(p.tmem_cols));
@@ -269,16 +295,37 @@ __global__ void __launch_bounds__(kStemThreads, 1)
       const uint32_t t_base = tmem_base + (uint32_t(q * 32) << 16) + abuf * uint32_t(p.acc_cols);
       for (int g = 0; g < pairs; ++g) {
         const int w = wt * p.bw + 2 * g + pix;
-        OutT* dst = out + ((long long)h * p.W + w) * p.B + bt * 64 + b_in;
         for (int k0 = 0; k0 < p.n_out; k0 += 32) {
           uint32_t v[32];
           tmem_ld_32x32b_x32(t_base + uint32_t(g * p.n_out + k0), v);
           tmem_ld_wait();
-          if (w < p.W) {
-            // a warp writes 32 consecutive images of one (k, h, w): 64 or 128 contiguous bytes
+          if constexpr (sizeof(OutT) == 2) {
+            // bf16: the two warps that hold one pixel (images 0-31 and 32-63) transpose their
+            // 32 x 32 blocks through a [32 k][64 images] staging buffer, and one TMA store writes
+            // it as 32 full 128-byte lines of Out.
+            const uint32_t buf = stage_smem + uint32_t(pix) * 4096u;
+            const bool issuer = (q & 1) == 0 && lane == 0;
+            if (issuer) bulk_wait_read_all();       // the previous store has read the buffer
+            named_bar_sync(1 + pix, 64);
+            uint8_t* row0 = gen0 + (buf - smem0) + b_in * 2;
 #pragma unroll
             for (int j = 0; j < 32; ++j)
-              if (k0 + j < p.K) store_scalar(dst + (long long)(k0 + j) * k_stride, v[j]);
+              *reinterpret_cast<__nv_bfloat16*>(row0 + j * 128) =
+                  __float2bfloat16_rn(__uint_as_float(v[j]));
+            fence_proxy_async_smem();
+            named_bar_sync(1 + pix, 64);
+            if (issuer && w < p.W && k0 < p.K) {
+              tma_store_4d(&tm_out, bt * 64, w, h, k0, buf);   // rows k >= K are clipped
+              bulk_commit();
+            }
+          } else {
+            if (w < p.W) {
+              // fp32: a warp writes 32 consecutive images of one (k, h, w), 128 contiguous bytes
+              OutT* dst = out + ((long long)h * p.W + w) * p.B + bt * 64 + b_in;
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (k0 + j < p.K) store_scalar(dst + (long long)(k0 + j) * k_stride, v[j]);
+            }
           }
         }
       }
@@ -288,6 +335,7 @@ __global__ void __launch_bounds__(kStemThreads, 1)
       abuf ^= 1u;
       if (abuf == 0) aph ^= 1u;
     }
+    if ((q & 1) == 0 && lane == 0) bulk_wait_all();  // Out is written before the CTA leaves
   }
 
   // ===================== teardown =====================
@@ -307,7 +355,8 @@ cudaError_t stem_kernel_prepare(int smem_bytes) {
                               smem_bytes);
 }
 
-cudaError_t launch_stem(const CUtensorMap& tm_image, const void* packed_filter, void* out,
+cudaError_t launch_stem(const CUtensorMap& tm_image, const CUtensorMap& tm_out,
+                        const void* packed_filter, void* out,
                         bool out_f32, const StemKernelParams& p, int grid, int smem_bytes,
                         int* status, cudaStream_t stream) {
   const uint8_t* pf = static_cast<const uint8_t*>(packed_filter);
@@ -322,9 +371,9 @@ cudaError_t launch_stem(const CUtensorMap& tm_image, const void* packed_filter, 
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   if (out_f32)
-    return cudaLaunchKernelEx(&cfg, cconv_stem_kernel<float>, tm_image, pf, static_cast<float*>(out),
+    return cudaLaunchKernelEx(&cfg, cconv_stem_kernel<float>, tm_image, tm_out, pf, static_cast<float*>(out),
                               p, status);
-  return cudaLaunchKernelEx(&cfg, cconv_stem_kernel<__nv_bfloat16>, tm_image, pf,
+  return cudaLaunchKernelEx(&cfg, cconv_stem_kernel<__nv_bfloat16>, tm_image, tm_out, pf,
                             static_cast<__nv_bfloat16*>(out), p, status);
 }
 
