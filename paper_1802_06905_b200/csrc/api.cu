@@ -55,6 +55,9 @@ struct cconv_plan {
   int* d_status = nullptr;
   void* d_packed = nullptr;  // scratch: the packed Filter (rewritten by every forward call)
   unsigned long long* d_trace = nullptr;  // diagnostics: [grid][16] device time stamps
+  int trace_rows = 0;
+  mutable const void* tm_out_ptr = nullptr;
+  mutable CUtensorMap tm_out{};  // stem kernel: Out is written with TMA stores
   // host-buffer entry point: device staging owned by the plan
   void* st_image = nullptr;
   void* st_filter = nullptr;
@@ -63,8 +66,6 @@ struct cconv_plan {
   mutable std::mutex mu;
   mutable const void* tm_image_ptr = nullptr;
   mutable CUtensorMap tm_image{};
-  mutable const void* tm_out_ptr = nullptr;
-  mutable CUtensorMap tm_out{};  // stem kernel, bf16 Out only
 };
 
 namespace {
@@ -184,12 +185,12 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
       e = cudaMalloc(&pl->d_packed, size_t(pl->tile.packed_filter_bytes));
     if (e == cudaSuccess && variant == CCONV_VARIANT_STEM)
       e = stem_kernel_prepare(pl->stile.smem_bytes);
-    if (e == cudaSuccess && variant == CCONV_VARIANT_STEM)
-      e = cudaMalloc(&pl->d_packed, size_t(pl->stile.packed_filter_bytes));
-    if (e == cudaSuccess && variant == CCONV_VARIANT_HALO && env_int("CCONV_TRACE", 0)) {
-      e = cudaMalloc(reinterpret_cast<void**>(&pl->d_trace), size_t(pl->tile.grid + 16) * 16 * 8);
-      if (e == cudaSuccess) e = cudaMemset(pl->d_trace, 0, size_t(pl->tile.grid + 16) * 16 * 8);
+    if (e == cudaSuccess && variant >= CCONV_VARIANT_HALO && env_int("CCONV_TRACE", 0)) {
+      pl->trace_rows = (variant == CCONV_VARIANT_HALO ? pl->tile.grid : pl->stile.grid) + 16;
+      e = cudaMalloc(reinterpret_cast<void**>(&pl->d_trace), size_t(pl->trace_rows) * 16 * 8);
+      if (e == cudaSuccess) e = cudaMemset(pl->d_trace, 0, size_t(pl->trace_rows) * 16 * 8);
       pl->kp.trace = pl->d_trace;
+      pl->skp.trace = pl->d_trace;
     }
     cudaSetDevice(prev);
     if (e != cudaSuccess) {
@@ -202,9 +203,9 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
   if (env_int("CCONV_LOG", 0) && variant == CCONV_VARIANT_STEM) {
     const StemTile& t = pl->stile;
     std::fprintf(stderr,
-                 "[cconv] B%d C%d K%d W%d H%d R%d S%d s%dx%d variant=3 tile bw=%d kw=%d ndelta=%d "
-                 "n_out=%d i_stages=%d tmem=%d tiles=%lld grid=%d smem=%d filt=%u\n",
-                 B, C, K, W, H, R, S, sw, sh, t.bw, t.kw, t.ndelta, t.n_out, t.i_stages, t.tmem_cols,
+                 "[cconv] B%d C%d K%d W%d H%d R%d S%d s%dx%d variant=3 tile bw=%d bhm=%d kpad=%d "
+                 "kw=%d i_stages=%d tmem=%d tiles=%lld grid=%d smem=%d filt=%u\n",
+                 B, C, K, W, H, R, S, sw, sh, t.bw, t.bhm, t.kpad, t.kw, t.i_stages, t.tmem_cols,
                  t.tiles, t.grid, t.smem_bytes, t.filt_bytes);
   } else if (env_int("CCONV_LOG", 0)) {
     const HaloTile& t = pl->tile;
@@ -241,8 +242,8 @@ int cconv_plan_info_get(const cconv_plan* pl, cconv_plan_info* o) {
       double(d.Wi()) * d.Hi() * d.C * d.B + double(d.K) * d.R * d.S * d.C + double(d.K) * d.H * d.W * d.B;
   if (pl->variant == CCONV_VARIANT_STEM) {
     const StemTile& t = pl->stile;
-    o->bb = 64; o->bc = d.C; o->bk = t.n_out; o->bw = t.bw; o->bh = 1;
-    o->halo_w = t.halo_w; o->halo_h = d.S;
+    o->bb = 64; o->bc = d.C; o->bk = t.kpad; o->bw = t.bw; o->bh = t.bhm;
+    o->halo_w = t.halo_w; o->halo_h = d.sh * (t.bhm - 1) + d.S;
     o->stages = t.i_stages; o->filter_stages = 1; o->grid = t.grid; o->tiles = int(t.tiles);
     o->smem_bytes = t.smem_bytes; o->tmem_cols = t.tmem_cols;
     o->tile_words_smem = t.words_smem;
@@ -306,17 +307,14 @@ int cconv_forward_planned(const cconv_plan* pl, const void* Image, const void* F
     {
       std::lock_guard<std::mutex> lk(pl->mu);
       if (pl->tm_out_ptr != Out) {
-        // fp32 Out is stored without TMA; the map is then built over the same bytes and not used
-        int rc = encode_stem_out_map(pl->d, Out, &pl->tm_out);
+        int rc = encode_stem_out_map(pl->d, Out, pl->out_dtype == CCONV_OUT_F32, &pl->tm_out);
         if (rc != CCONV_OK) return rc;
         pl->tm_out_ptr = Out;
       }
       tmo = pl->tm_out;
     }
-    cudaError_t es = launch_pack_filter_stem(Filter, pl->d_packed, pl->d, pl->skp, stream);
-    if (es != cudaSuccess) return cuda_fail(es, "launch_pack_filter_stem");
-    es = launch_stem(tmi, tmo, pl->d_packed, Out, pl->out_dtype == CCONV_OUT_F32, pl->skp,
-                     pl->stile.grid, pl->stile.smem_bytes, pl->d_status, stream);
+    cudaError_t es = launch_stem(tmi, tmo, Filter, pl->out_dtype == CCONV_OUT_F32, pl->skp,
+                                 pl->stile.grid, pl->stile.smem_bytes, pl->d_status, stream);
     return es == cudaSuccess ? CCONV_OK : cuda_fail(es, "launch_stem");
   }
   cudaError_t e = launch_pack_filter(Filter, pl->d_packed, pl->d, pl->tile.c16, pl->tile.tiles_k,
@@ -373,7 +371,7 @@ int cconv_forward_host(cconv_plan* pl, const void* hImage, const void* hFilter, 
 int cconv_plan_trace_read(const cconv_plan* pl, unsigned long long* host_out, int max_u64) {
   if (!pl || !host_out || max_u64 <= 0) return CCONV_EINVAL;
   if (!pl->d_trace) return 0;
-  const int n = std::min(max_u64, (pl->tile.grid + 16) * 16);
+  const int n = std::min(max_u64, pl->trace_rows * 16);
   CCONV_CUDA(cudaMemcpy(host_out, pl->d_trace, size_t(n) * 8, cudaMemcpyDeviceToHost));
   return n;
 }

@@ -121,25 +121,25 @@ void build_stem_params(const Dims& d, const StemTile& t, StemKernelParams* out) 
   StemKernelParams& p = *out;
   p.K = d.K; p.H = d.H; p.W = d.W; p.B = d.B; p.C = d.C;
   p.R = d.R; p.S = d.S; p.sw = d.sw; p.sh = d.sh;
-  p.bw = t.bw; p.kw = t.kw; p.khalves = t.khalves; p.dstep = t.dstep; p.ndelta = t.ndelta;
-  p.halo_w = t.halo_w; p.n_out = t.n_out;
-  p.tiles_w = t.tiles_w; p.tiles_b = t.tiles_b; p.total_tiles = int(t.tiles);
+  p.bw = t.bw; p.kpad = t.kpad; p.bhm = t.bhm; p.kw = t.kw; p.khalves = t.khalves;
+  p.units = d.R * t.khalves;
+  p.halo_w = t.halo_w;
+  p.tiles_k = t.tiles_k; p.tiles_w = t.tiles_w; p.tiles_h = t.tiles_h; p.tiles_b = t.tiles_b;
+  p.total_tiles = int(t.tiles);
   p.i_stages = t.i_stages;
-  p.acc_cols = (t.bw / 2) * t.n_out;
+  p.acc_cols = 64 * t.bw;
   p.tmem_cols = t.tmem_cols;
   p.img_stage_bytes = t.img_stage_bytes;
   p.filt_bytes = t.filt_bytes;
-  p.xslab_bytes = uint32_t(t.kw) * 128u;       // one Image column: kw rows of 64 images
-  p.fblock_bytes = uint32_t(t.n_out) * 32u;    // one Filter block: n_out x 16
-  // instruction descriptor: D=f32, A=B=bf16, A MN-major [15]=1, B K-major [16]=0, N = n_out, M = 128
-  p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (0u << 16) |
-            (uint32_t(t.n_out >> 3) << 17) | (uint32_t(128 >> 4) << 24);
-  // A = Image window [16 rows][2 pixels x 64 images], MN-major, 128-byte swizzle (layout type 2):
-  // SBO = 1024 B from one group of 8 rows to the next; LBO = from pixel 1's 64 images to pixel 2's,
-  // sw Image columns further.
-  p.a_desc = make_smem_desc(uint32_t(d.sw) * p.xslab_bytes, 1024, 2);
-  // B = Filter block [n_out rows][16], K-major, no swizzle: LBO = 128 B, SBO = 256 B.
-  p.b_desc = make_smem_desc(128, 256, 0);
+  // instruction descriptor: D=f32, A=B=bf16, A K-major [15]=0, B MN-major [16]=1, N = 64*bw, M = 128
+  p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
+            (uint32_t((64 * t.bw) >> 3) << 17) | (uint32_t(128 >> 4) << 24);
+  // A = Filter block [128 rows][16], K-major, no swizzle: LBO = 128 B, SBO = 256 B.
+  p.a_desc = make_smem_desc(128, 256, 0);
+  // B = Image window [16 rows][bw pixels x 64 images], MN-major, 128-byte swizzle (layout type 2):
+  // SBO = 1024 B from one group of 8 rows to the next; LBO = from one pixel's 64 images to the next
+  // pixel's, sw Image columns (of kw rows x 128 B) further.
+  p.b_desc = make_smem_desc(uint32_t(d.sw) * uint32_t(t.kw) * 128u, 1024, 2);
   p.wait_limit_ns = uint64_t(env_int("CCONV_WAIT_LIMIT_MS", 1000)) * 1000000ull;
   p.trace = nullptr;
 }
@@ -167,20 +167,24 @@ int encode_stem_image_map(const Dims& d, const StemTile& t, const void* image, C
   return CCONV_OK;
 }
 
-int encode_stem_out_map(const Dims& d, void* out, CUtensorMap* tm) {
+int encode_stem_out_map(const Dims& d, void* out, bool out_f32, CUtensorMap* tm) {
   EncodeTiledFn enc = encode_tiled_fn();
   if (!enc) {
     set_last_cuda_error("cuTensorMapEncodeTiled is not available from this driver");
     return CCONV_ECUDA;
   }
+  // Out[k][h][w][b] viewed as (b, w, h, k).  One store = 32 out-channels x 128 bytes of images
+  // (64 bf16 or 32 fp32) of one pixel, read from 128-byte-swizzled shared-memory rows.
+  const cuuint64_t es_bytes = out_f32 ? 4 : 2;
   const cuuint64_t dims[4] = {cuuint64_t(d.B), cuuint64_t(d.W), cuuint64_t(d.H), cuuint64_t(d.K)};
-  const cuuint64_t strides[3] = {cuuint64_t(d.B) * 2, cuuint64_t(d.W) * d.B * 2,
-                                 cuuint64_t(d.H) * d.W * d.B * 2};
-  const cuuint32_t box[4] = {64u, 1u, 1u, 32u};
+  const cuuint64_t strides[3] = {cuuint64_t(d.B) * es_bytes, cuuint64_t(d.W) * d.B * es_bytes,
+                                 cuuint64_t(d.H) * d.W * d.B * es_bytes};
+  const cuuint32_t box[4] = {out_f32 ? 32u : 64u, 1u, 1u, 32u};
   const cuuint32_t es[4] = {1, 1, 1, 1};
-  CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, out, dims, strides, box, es,
-                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
-                   CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  CUresult r = enc(tm, out_f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+                   4, out, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
     set_last_cuda_error("cuTensorMapEncodeTiled(Out) failed with CUresult " + std::to_string(int(r)));
     return CCONV_ECUDA;

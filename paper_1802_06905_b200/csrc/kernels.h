@@ -48,21 +48,20 @@ struct HaloKernelParams {
 // tensor core's K-major no-swizzle core-matrix order.
 constexpr int kPackedBlockBytes = 4096;
 
-// Parameters of the small-C ("stem") tensor-core kernel.  Roles are swapped with respect to the halo
-// kernel: MMA rows = 2 output pixels x 64 images, MMA columns = output channels, and the
-// contraction dimension of one MMA runs over consecutive (s, c) rows of the Image, which are
-// contiguous in memory for a fixed first subscript.
+// Parameters of the small-C ("stem") tensor-core kernel.  The contraction dimension of one MMA
+// runs over consecutive (s, c) rows of the Image, which are contiguous in memory for a fixed first
+// subscript; MMA rows = (stacked output row j, out-channel), MMA columns = bw pixels x 64 images.
 struct StemKernelParams {
   int K, H, W, B, C, R, S, sw, sh;
-  int bw;                 // output pixels per tile along w (even); pairs = bw/2 accumulators
+  int bw;                 // output pixels per tile along w; MMA N = 64*bw
+  int kpad, bhm;          // MMA row = j*kpad + k: bhm output rows stacked in M (kpad*bhm <= 128)
   int kw, khalves;        // rows of the (s,c) window (multiple of 16) and kw/16
-  int dstep, ndelta;      // window offsets delta = (sh*C*h) % 8 are multiples of dstep; 8/dstep of them
+  int units;              // MMAs per tile: R * khalves
   int halo_w;             // sw*(bw-1)+R Image columns per tile
-  int n_out;              // MMA N: K rounded up to 16
-  int tiles_w, tiles_b, total_tiles;
+  int tiles_k, tiles_w, tiles_h, tiles_b, total_tiles;
   int i_stages;
   int acc_cols, tmem_cols;
-  uint32_t img_stage_bytes, filt_bytes, xslab_bytes, fblock_bytes;
+  uint32_t img_stage_bytes, filt_bytes;
   uint32_t idesc;
   uint64_t a_desc, b_desc;
   uint64_t wait_limit_ns;
@@ -76,13 +75,9 @@ cudaError_t launch_simt(const void* image, const void* filter, void* out, bool o
 cudaError_t launch_pack_filter(const void* filter, void* packed, const Dims& d, int c16,
                                int tiles_k, cudaStream_t stream);
 
-// Filter [K][R][S][C] -> stem blocks [r][delta][k-half][n_out x 16], the (s,c) run of each r shifted
-// by delta rows and zero padded.
-cudaError_t launch_pack_filter_stem(const void* filter, void* packed, const Dims& d,
-                                    const StemKernelParams& p, cudaStream_t stream);
 cudaError_t stem_kernel_prepare(int smem_bytes);
-cudaError_t launch_stem(const CUtensorMap& tm_image, const CUtensorMap& tm_out,
-                        const void* packed_filter, void* out,
+// `filter` is the caller's Filter [K][R][S][C]; Out is reached through its tensor map only.
+cudaError_t launch_stem(const CUtensorMap& tm_image, const CUtensorMap& tm_out, const void* filter,
                         bool out_f32, const StemKernelParams& p, int grid, int smem_bytes,
                         int* status, cudaStream_t stream);
 

@@ -219,58 +219,58 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[5], HaloT
 }
 
 bool choose_stem_tile(const Dims& d, const Machine& m, StemTile* out) {
-  // two 4 KB buffers from which the epilogue's TMA stores read (one per pixel of a pair)
-  constexpr int kStemStagingBytes = 8192;
-  if (d.B % 64 != 0 || d.K > 256) return false;
+  // 8 epilogue warps x 2 x 4 KB sources of the TMA stores; the raw Filter passes through the same
+  // bytes (at least one whole zero-padded out-channel at a time) while it is repacked
+  constexpr int kStemStagingBytes = 65536;
+  if (d.B % 64 != 0) return false;
   const int reserve = 2048;
-  const int cap = m.smem_optin_bytes - reserve;
+  const int cap = m.smem_optin_bytes - reserve - kStemStagingBytes;
+  const int shc = d.sh * d.C;
   StemTile t;
-  // Row offset of output row h inside an 8-row swizzle atom: delta = (sh*C*h) % 8, a multiple of
-  // gcd(sh*C, 8).
-  int ga = (d.sh * d.C) % 8, gb = 8;
-  while (ga != 0) {
-    const int r = gb % ga;
-    gb = ga;
-    ga = r;
-  }
-  const int g = gb;  // gcd(sh*C mod 8, 8); 8 when sh*C is a multiple of 8
-  t.dstep = g;
-  t.ndelta = 8 / g;
-  const int dmax = 8 - g;
-  t.kw = (dmax + d.S * d.C + 15) / 16 * 16;
-  if (t.kw > 256) return false;
-  t.khalves = t.kw / 16;
-  t.n_out = (d.K + 15) / 16 * 16;
-  t.filt_bytes = uint32_t(d.R) * t.ndelta * t.khalves * t.n_out * 32u;
-  t.packed_filter_bytes = t.filt_bytes;
-  if (int(t.filt_bytes) > cap / 2) return false;
-  // The epilogue reads TMEM 32 columns at a time; when n_out is not a multiple of 32 its last read
-  // runs up to 16 columns past the accumulators, which must still be allocated columns.
-  const int tmem_pad = (t.n_out % 32) ? 32 : 0;
+  // Few out-channels leave MMA rows free: stack consecutive output rows there (row j*kpad + k).
+  t.kpad = d.K <= 32 ? 32 : d.K <= 64 ? 64 : 128;
+  t.tiles_k = (d.K + 127) / 128;
   bool found = false;
-  for (int bw = 8; bw >= 2; bw -= 2) {
-    if (bw / 2 * t.n_out * 2 + tmem_pad > m.tmem_cols) continue;  // two accumulator buffers
-    const int halo_w = d.sw * (bw - 1) + d.R;
-    if (halo_w > 256) continue;
-    const long long img = 1ll * halo_w * t.kw * 128;
-    if (2 * img + t.filt_bytes + kStemStagingBytes > cap) continue;
-    t.bw = bw;
-    t.halo_w = halo_w;
-    t.img_stage_bytes = uint32_t(img);
-    t.i_stages = int(std::min<long long>(4, (cap - t.filt_bytes - kStemStagingBytes) / img));
-    found = true;
-    break;
+  for (int bhm = 128 / t.kpad; bhm >= 1 && !found; bhm /= 2) {
+    if (bhm > 1 && bhm / 2 >= d.H) continue;  // rows past H would only widen the window
+    const int kw = (shc * (bhm - 1) + d.S * d.C + 15) / 16 * 16;
+    if (kw > 256) continue;
+    const long long filt = 1ll * t.tiles_k * d.R * (kw / 16) * 4096;
+    if (filt > cap) continue;
+    const int padded_run = (shc * (bhm - 1) + kw + 7) / 8 * 8;
+    if (2ll * d.R * (padded_run + d.S * d.C) > kStemStagingBytes - 32) continue;
+    for (int bw = 4; bw >= 1; --bw) {
+      if (bw > 1 && bw - 1 >= d.W) continue;  // no wider than the output row
+      const int halo_w = d.sw * (bw - 1) + d.R;
+      if (halo_w > 256) continue;
+      const long long img = 1ll * halo_w * kw * 128;
+      if (2 * img + filt > cap) continue;
+      t.bhm = bhm;
+      t.kw = kw;
+      t.khalves = kw / 16;
+      t.filt_bytes = uint32_t(filt);
+      t.bw = bw;
+      t.halo_w = halo_w;
+      t.img_stage_bytes = uint32_t(img);
+      t.i_stages = int(std::min<long long>(4, (cap - filt) / img));
+      found = true;
+      break;
+    }
   }
   if (!found) return false;
+  t.packed_filter_bytes = 0;  // every CTA repacks the Filter itself
   int cols = 32;
-  while (cols < t.bw / 2 * t.n_out * 2 + tmem_pad) cols *= 2;
+  while (cols < 2 * 64 * t.bw) cols *= 2;  // two accumulator buffers of 64*bw columns
   t.tmem_cols = cols;
   t.tiles_w = (d.W + t.bw - 1) / t.bw;
+  t.tiles_h = (d.H + t.bhm - 1) / t.bhm;
   t.tiles_b = d.B / 64;
-  t.tiles = 1ll * t.tiles_b * d.H * t.tiles_w;
+  t.tiles = 1ll * t.tiles_b * t.tiles_h * t.tiles_w * t.tiles_k;
   if (t.tiles > 0x7fffffffll) return false;
   t.grid = int(std::min<long long>(t.tiles, m.sm_count));
-  t.smem_bytes = std::max(int(t.i_stages * t.img_stage_bytes + t.filt_bytes) + kStemStagingBytes + reserve, 117760);
+  t.smem_bytes =
+      std::max(int(t.i_stages * t.img_stage_bytes + t.filt_bytes) + kStemStagingBytes + reserve,
+               117760);
   t.words_smem = double(t.tiles) * (t.img_stage_bytes / 2) + double(t.grid) * (t.filt_bytes / 2) +
                  double(d.K) * d.H * d.W * d.B;
   *out = t;

@@ -56,11 +56,12 @@ struct HaloTile {
   double words_smem = 0;   // words staged into shared memory over the whole problem + |Out|
 };
 
-// Tile of the small-C ("stem") kernel: one output row, bw pixels, all K (<= 256) channels, 64 images.
+// Tile of the small-C ("stem") kernel: 128 MMA rows = bhm stacked output rows x kpad out-channels,
+// bw pixels, 64 images; the whole (shifted, zero-padded) Filter stays in shared memory.
 struct StemTile {
-  int bw = 0, kw = 0, khalves = 0, dstep = 0, ndelta = 0, halo_w = 0, n_out = 0;
+  int bw = 0, kpad = 0, bhm = 0, kw = 0, khalves = 0, halo_w = 0;
   int i_stages = 2, tmem_cols = 0;
-  int tiles_w = 0, tiles_b = 0;
+  int tiles_k = 0, tiles_w = 0, tiles_h = 0, tiles_b = 0;
   long long tiles = 0;
   int grid = 0;
   uint32_t img_stage_bytes = 0, filt_bytes = 0;
@@ -82,8 +83,8 @@ bool halo_supported(const Dims& d, const char** why);
 // `force` may carry "bw,bh,bc,stages,bb" (0 = free) from the CCONV_FORCE_TILE environment variable.
 bool choose_halo_tile(const Dims& d, const Machine& m, const int force[5], HaloTile* out);
 
-// The stem kernel needs B % 64 == 0, K <= 256, and the shifted (s,c) window, the resident Filter
-// and two Image stages to fit in shared memory.
+// The stem kernel needs B % 64 == 0 and the resident Filter plus two Image windows to fit in shared
+// memory.
 bool choose_stem_tile(const Dims& d, const Machine& m, StemTile* out);
 
 }  // namespace cconv

@@ -126,8 +126,10 @@ def test_inspection_plans_are_hardware_legal():
             # the staged words can never undercut the bound at the shared-memory size
             assert info["tile_words_smem"] >= max(exp_terms) * 0.999 or max(exp_terms) < info["M_words"]
         elif info["variant"] == binding.VARIANT_STEM:
-            assert cfg.B % 64 == 0 and cfg.C < 8 and cfg.K <= 256
-            assert info["bw"] % 2 == 0 and info["bw"] // 2 * info["bk"] * 2 <= 512   # two TMEM buffers
+            assert cfg.B % 64 == 0 and cfg.C < 8
+            assert 1 <= info["bw"] <= 4 and 2 * 64 * info["bw"] <= info["tmem_cols"] <= 512
+            assert info["bk"] * info["bh"] <= 128            # stacked output rows share the MMA's M
+            assert info["halo_h"] == cfg.sh * (info["bh"] - 1) + cfg.S
             assert info["smem_bytes"] <= 232448 and info["stages"] >= 2
         else:
             assert info["variant"] == binding.VARIANT_SIMT

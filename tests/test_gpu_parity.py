@@ -108,11 +108,13 @@ def test_halo_shapes(c, out_dtype):
 # ---- small-C tensor-core kernel: (s,c) folded into the contraction ----------------------------------
 
 STEM_SHAPES = [
-    cs("st_c3_7x7_s2", 64, 3, 64, 20, 18, 7, 7, 2, 2),      # four window offsets (sh*C = 6)
-    cs("st_c4_k40", 64, 4, 40, 9, 6, 3, 3),                 # odd W: ragged pixel pair; K < 64
-    cs("st_c1", 128, 1, 16, 10, 7, 5, 5, 1, 2),             # two batch tiles, one channel
-    cs("st_c6_s3", 64, 6, 100, 7, 5, 3, 4, 3, 1),           # K = 100 -> N = 112; sw = 3
-    cs("st_c2_wide", 64, 2, 24, 33, 3, 2, 9, 2, 1),         # S*C = 18 with offsets 0..6
+    cs("st_c3_7x7_s2", 64, 3, 64, 20, 19, 7, 7, 2, 2),      # two stacked rows (shift sh*C = 6), odd H
+    cs("st_c4_k40", 64, 4, 40, 9, 6, 3, 3),                 # ragged W tile; K < 64
+    cs("st_c1", 128, 1, 16, 10, 7, 5, 5, 1, 2),             # two batch tiles, one channel, 4 stacked rows
+    cs("st_c6_s3", 64, 6, 100, 7, 5, 3, 4, 3, 1),           # K = 100: no stacking; sw = 3
+    cs("st_c2_wide", 64, 2, 24, 33, 3, 2, 9, 2, 1),         # S*C = 18; four stacked rows, H = 3
+    cs("st_c3_k200", 64, 3, 200, 6, 5, 3, 3),               # two out-channel tiles
+    cs("st_c5_h1", 64, 5, 64, 3, 1, 4, 2, 1, 3),            # one output row, W < bw
 ]
 
 
