@@ -88,7 +88,8 @@ typedef struct {
    * fast-memory level = shared memory of one CTA; slow side = L2/HBM. */
   double tile_words_smem; /* words staged into shared memory over the whole problem + Out words */
   double compulsory_words; /* |Image| + |Filter| + |Out| with the real Image extent             */
-  double scratch_bytes;   /* device scratch the plan owns (the packed Filter)                   */
+  double scratch_bytes;   /* one packed Filter; the plan owns two such device buffers and
+                             alternates between them from call to call                          */
 } cconv_plan_info;
 
 /* Theorem 1 (Section 4.1): the five lower-bound terms, in words, for a fast memory of M_words.
@@ -108,8 +109,9 @@ int cconv_tiling_lp(int B, int C, int K, int W, int H, int R, int S, int sw, int
 /* Plan: evaluate the bound, solve the LP, pick a hardware-legal tile and kernel variant for
  * `device`, and build the TMA descriptors' shape data.  M_words <= 0 means "the shared memory one
  * CTA can use, in bf16 words".  variant: CCONV_VARIANT_*; out_dtype: CCONV_OUT_*.  device >= 0 is a
- * CUDA ordinal (a status word and, for the HALO variant, scratch for the repacked Filter are
- * allocated there; every forward call rewrites that scratch); device = -1 plans for a nominal
+ * CUDA ordinal (a status word and, for the tensor-core variants, two scratch buffers for the
+ * repacked Filter are allocated there; forward calls rewrite them in turn, and the repacking of
+ * one call may overlap the convolution of the call before it); device = -1 plans for a nominal
  * B200 without any CUDA call, for inspection only (forward calls on such a plan return EINVAL).
  * The plan is immutable afterwards and may be used from any stream of that device, one launch at a
  * time per plan (launches of one plan share its status word). */

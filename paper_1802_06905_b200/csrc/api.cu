@@ -53,11 +53,13 @@ struct cconv_plan {
   StemTile stile{};
   StemKernelParams skp{};
   int* d_status = nullptr;
-  void* d_packed = nullptr;  // scratch: the packed Filter (rewritten by every forward call)
+  // Scratch: the packed Filter, rewritten by every forward call.  Two buffers, used alternately:
+  // the packing kernel of call n+1 may run while the convolution of call n still reads its buffer.
+  void* d_packed = nullptr;  // 2 x packed_bytes
+  size_t packed_bytes = 0;
+  mutable unsigned calls = 0;
   unsigned long long* d_trace = nullptr;  // diagnostics: [grid][16] device time stamps
   int trace_rows = 0;
-  mutable const void* tm_out_ptr = nullptr;
-  mutable CUtensorMap tm_out{};  // stem kernel: Out is written with TMA stores
   // host-buffer entry point: device staging owned by the plan
   void* st_image = nullptr;
   void* st_filter = nullptr;
@@ -181,8 +183,11 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
     if (e == cudaSuccess) e = cudaMemset(pl->d_status, 0, 256);
     if (e == cudaSuccess && variant == CCONV_VARIANT_HALO)
       e = halo_kernel_prepare(pl->tile.smem_bytes);
-    if (e == cudaSuccess && variant == CCONV_VARIANT_HALO)
-      e = cudaMalloc(&pl->d_packed, size_t(pl->tile.packed_filter_bytes));
+    if (variant == CCONV_VARIANT_HALO) pl->packed_bytes = size_t(pl->tile.packed_filter_bytes);
+    if (variant == CCONV_VARIANT_STEM) pl->packed_bytes = size_t(pl->stile.packed_filter_bytes);
+    pl->packed_bytes = (pl->packed_bytes + 255) & ~size_t(255);
+    if (e == cudaSuccess && variant >= CCONV_VARIANT_HALO)
+      e = cudaMalloc(&pl->d_packed, 2 * pl->packed_bytes);
     if (e == cudaSuccess && variant == CCONV_VARIANT_STEM)
       e = stem_kernel_prepare(pl->stile.smem_bytes);
     if (e == cudaSuccess && variant >= CCONV_VARIANT_HALO && env_int("CCONV_TRACE", 0)) {
@@ -290,6 +295,7 @@ int cconv_forward_planned(const cconv_plan* pl, const void* Image, const void* F
     return e == cudaSuccess ? CCONV_OK : cuda_fail(e, "launch_simt");
   }
   CUtensorMap tmi;
+  void* packed = nullptr;
   {
     // the tensor map is rebuilt only when the Image pointer changes
     std::lock_guard<std::mutex> lk(pl->mu);
@@ -301,26 +307,19 @@ int cconv_forward_planned(const cconv_plan* pl, const void* Image, const void* F
       pl->tm_image_ptr = Image;
     }
     tmi = pl->tm_image;
+    packed = static_cast<char*>(pl->d_packed) + (pl->calls++ & 1u) * pl->packed_bytes;
   }
   if (pl->variant == CCONV_VARIANT_STEM) {
-    CUtensorMap tmo;
-    {
-      std::lock_guard<std::mutex> lk(pl->mu);
-      if (pl->tm_out_ptr != Out) {
-        int rc = encode_stem_out_map(pl->d, Out, pl->out_dtype == CCONV_OUT_F32, &pl->tm_out);
-        if (rc != CCONV_OK) return rc;
-        pl->tm_out_ptr = Out;
-      }
-      tmo = pl->tm_out;
-    }
-    cudaError_t es = launch_stem(tmi, tmo, Filter, pl->out_dtype == CCONV_OUT_F32, pl->skp,
-                                 pl->stile.grid, pl->stile.smem_bytes, pl->d_status, stream);
+    cudaError_t es = launch_pack_filter_stem(Filter, packed, pl->d, pl->skp, stream);
+    if (es != cudaSuccess) return cuda_fail(es, "launch_pack_filter_stem");
+    es = launch_stem(tmi, packed, Out, pl->out_dtype == CCONV_OUT_F32, pl->skp, pl->stile.grid,
+                     pl->stile.smem_bytes, pl->d_status, stream);
     return es == cudaSuccess ? CCONV_OK : cuda_fail(es, "launch_stem");
   }
-  cudaError_t e = launch_pack_filter(Filter, pl->d_packed, pl->d, pl->tile.c16, pl->tile.tiles_k,
-                                     stream);
+  cudaError_t e = launch_pack_filter(Filter, packed, pl->d, pl->tile.c16, pl->tile.tiles_k,
+                                     /*overlap_prev=*/true, stream);
   if (e != cudaSuccess) return cuda_fail(e, "launch_pack_filter");
-  e = launch_halo(tmi, pl->d_packed, Out, pl->out_dtype == CCONV_OUT_F32, pl->kp, pl->tile.grid,
+  e = launch_halo(tmi, packed, Out, pl->out_dtype == CCONV_OUT_F32, pl->kp, pl->tile.grid,
                   pl->tile.smem_bytes, pl->d_status, stream);
   return e == cudaSuccess ? CCONV_OK : cuda_fail(e, "launch_halo");
 }

@@ -167,31 +167,6 @@ int encode_stem_image_map(const Dims& d, const StemTile& t, const void* image, C
   return CCONV_OK;
 }
 
-int encode_stem_out_map(const Dims& d, void* out, bool out_f32, CUtensorMap* tm) {
-  EncodeTiledFn enc = encode_tiled_fn();
-  if (!enc) {
-    set_last_cuda_error("cuTensorMapEncodeTiled is not available from this driver");
-    return CCONV_ECUDA;
-  }
-  // Out[k][h][w][b] viewed as (b, w, h, k).  One store = 32 out-channels x 128 bytes of images
-  // (64 bf16 or 32 fp32) of one pixel, read from 128-byte-swizzled shared-memory rows.
-  const cuuint64_t es_bytes = out_f32 ? 4 : 2;
-  const cuuint64_t dims[4] = {cuuint64_t(d.B), cuuint64_t(d.W), cuuint64_t(d.H), cuuint64_t(d.K)};
-  const cuuint64_t strides[3] = {cuuint64_t(d.B) * es_bytes, cuuint64_t(d.W) * d.B * es_bytes,
-                                 cuuint64_t(d.H) * d.W * d.B * es_bytes};
-  const cuuint32_t box[4] = {out_f32 ? 32u : 64u, 1u, 1u, 32u};
-  const cuuint32_t es[4] = {1, 1, 1, 1};
-  CUresult r = enc(tm, out_f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
-                   4, out, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
-                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) {
-    set_last_cuda_error("cuTensorMapEncodeTiled(Out) failed with CUresult " + std::to_string(int(r)));
-    return CCONV_ECUDA;
-  }
-  return CCONV_OK;
-}
-
 void set_last_cuda_error(const std::string& msg) { g_last_cuda_error = msg; }
 const char* last_cuda_error() { return g_last_cuda_error.c_str(); }
 

@@ -22,9 +22,6 @@ int encode_image_map(const Dims& d, const HaloTile& t, const void* image, CUtens
 
 // The same two pieces for the small-C ("stem") kernel: Image viewed as (b, m = y*C + c, x).
 void build_stem_params(const Dims& d, const StemTile& t, StemKernelParams* p);
-// Out [K][H][W][B] viewed as (b, w, h, k) with a 128-byte x 1 x 1 x 32 box: the stem kernel's
-// epilogue stores 32 output channels of 64 (bf16) or 32 (fp32) images of one pixel per TMA store.
-int encode_stem_out_map(const Dims& d, void* out, bool out_f32, CUtensorMap* tm);
 int encode_stem_image_map(const Dims& d, const StemTile& t, const void* image, CUtensorMap* tm);
 
 }  // namespace cconv

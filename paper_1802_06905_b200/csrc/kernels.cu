@@ -102,6 +102,10 @@ constexpr int kProducersPerRing = 2;
 // (no swizzle, LBO = 128 B between the two channel halves, SBO = 256 B between 8-row groups).
 // Rows k >= K and channels c >= C are zero.  One thread writes 16 bytes.
 // ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void pack_filter_slot(const __nv_bfloat16* __restrict__ filter,
+                                                 uint4* __restrict__ packed, const Dims& d, int c16,
+                                                 long long slot);
+
 __global__ void __launch_bounds__(256)
     cconv_pack_filter_kernel(const __nv_bfloat16* __restrict__ filter, uint4* __restrict__ packed,
                              Dims d, int c16, long long slots) {
@@ -109,7 +113,16 @@ __global__ void __launch_bounds__(256)
   // and its Image copies while this kernel runs; it waits for our stores before reading them.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const long long slot = blockIdx.x * (long long)blockDim.x + threadIdx.x;
-  if (slot >= slots) return;
+  if (slot < slots) pack_filter_slot(filter, packed, d, c16, slot);
+  // Launched with programmatic stream serialization (overlap_prev), this kernel may run while the
+  // kernel in front of it is still executing; it then ends only after that kernel has, so that
+  // "this kernel is complete" still implies "everything older in the stream is complete".
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+__device__ __forceinline__ void pack_filter_slot(const __nv_bfloat16* __restrict__ filter,
+                                                 uint4* __restrict__ packed, const Dims& d, int c16,
+                                                 long long slot) {
   const int RS = d.R * d.S;
   const int j = int(slot & 255);
   long long unit = slot >> 8;
@@ -140,12 +153,21 @@ __global__ void __launch_bounds__(256)
 }
 
 cudaError_t launch_pack_filter(const void* filter, void* packed, const Dims& d, int c16,
-                               int tiles_k, cudaStream_t stream) {
+                               int tiles_k, bool overlap_prev, cudaStream_t stream) {
   const long long slots = 1ll * tiles_k * c16 * d.R * d.S * (kPackedBlockBytes / 16);
   const long long blocks = (slots + 255) / 256;
-  cconv_pack_filter_kernel<<<(unsigned)blocks, 256, 0, stream>>>(
-      static_cast<const __nv_bfloat16*>(filter), static_cast<uint4*>(packed), d, c16, slots);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(unsigned(blocks));
+  cfg.blockDim = dim3(256);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = overlap_prev ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, cconv_pack_filter_kernel,
+                            static_cast<const __nv_bfloat16*>(filter), static_cast<uint4*>(packed), d,
+                            c16, slots);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -437,8 +459,11 @@ __global__ void __launch_bounds__(kThreads, 1)
       const uint32_t n_st = uint32_t(p.f_stages);
       uint32_t seq = 0, s = 0, ph = 0;
       bool ok = true;
-      // the packed Filter is written by the kernel launched just before this one
+      // The packed Filter is written by the kernel launched just before this one.  Once that
+      // kernel is complete (and with it everything older in the stream), the next packing kernel
+      // may start: it writes the other scratch buffer while this kernel runs.
       asm volatile("griddepcontrol.wait;" ::: "memory");
+      if (me == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
       for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
         const int kt = tile % p.tiles_k;
         const uint8_t* src = packed_filter + (size_t)kt * p.units * kPackedBlockBytes;

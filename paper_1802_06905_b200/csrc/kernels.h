@@ -72,12 +72,20 @@ cudaError_t launch_simt(const void* image, const void* filter, void* out, bool o
                         const Dims& d, cudaStream_t stream);
 
 // Filter [K][R][S][C] -> packed [k-tile][16-channel chunk][tap][4 KB block], zero padded.
+// overlap_prev: launch with programmatic stream serialization, so that the packing may run while
+// the kernel in front of it in the stream (normally the previous convolution, which signals early)
+// is still executing.  Only for callers that alternate between two `packed` buffers: the previous
+// convolution still reads the other one.  The packing kernel always ends after its predecessor.
 cudaError_t launch_pack_filter(const void* filter, void* packed, const Dims& d, int c16,
-                               int tiles_k, cudaStream_t stream);
+                               int tiles_k, bool overlap_prev, cudaStream_t stream);
 
+// Filter [K][R][S][C] -> stem blocks [k-tile][r][16-row slice][128 x 16], the (s,c) run of each r
+// repeated once per stacked output row, shifted by that row's window offset, zero padded.  Always
+// launched with programmatic stream serialization (callers alternate between two buffers).
+cudaError_t launch_pack_filter_stem(const void* filter, void* packed, const Dims& d,
+                                    const StemKernelParams& p, cudaStream_t stream);
 cudaError_t stem_kernel_prepare(int smem_bytes);
-// `filter` is the caller's Filter [K][R][S][C]; Out is reached through its tensor map only.
-cudaError_t launch_stem(const CUtensorMap& tm_image, const CUtensorMap& tm_out, const void* filter,
+cudaError_t launch_stem(const CUtensorMap& tm_image, const void* packed_filter, void* out,
                         bool out_f32, const StemKernelParams& p, int grid, int smem_bytes,
                         int* status, cudaStream_t stream);
 

@@ -113,7 +113,7 @@ extern "C" int cconv_forward_noalloc(const void* Image, const void* Filter, void
   // Filter is rewritten in full (zero padding included) by the packing kernel.
   e = cudaMemsetAsync(status, 0, sizeof(int), stream);
   if (e != cudaSuccess) return fail(e, "cudaMemsetAsync(status)");
-  e = launch_pack_filter(Filter, packed, d, tile.c16, tile.tiles_k, stream);
+  e = launch_pack_filter(Filter, packed, d, tile.c16, tile.tiles_k, /*overlap_prev=*/false, stream);
   if (e != cudaSuccess) return fail(e, "launch_pack_filter");
   e = launch_halo(tm, packed, Out, out_dtype == CCONV_OUT_F32, kp, tile.grid, tile.smem_bytes, status,
                   stream);

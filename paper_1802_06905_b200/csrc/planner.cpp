@@ -219,12 +219,9 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[5], HaloT
 }
 
 bool choose_stem_tile(const Dims& d, const Machine& m, StemTile* out) {
-  // 8 epilogue warps x 2 x 4 KB sources of the TMA stores; the raw Filter passes through the same
-  // bytes (at least one whole zero-padded out-channel at a time) while it is repacked
-  constexpr int kStemStagingBytes = 65536;
   if (d.B % 64 != 0) return false;
   const int reserve = 2048;
-  const int cap = m.smem_optin_bytes - reserve - kStemStagingBytes;
+  const int cap = m.smem_optin_bytes - reserve;
   const int shc = d.sh * d.C;
   StemTile t;
   // Few out-channels leave MMA rows free: stack consecutive output rows there (row j*kpad + k).
@@ -237,8 +234,6 @@ bool choose_stem_tile(const Dims& d, const Machine& m, StemTile* out) {
     if (kw > 256) continue;
     const long long filt = 1ll * t.tiles_k * d.R * (kw / 16) * 4096;
     if (filt > cap) continue;
-    const int padded_run = (shc * (bhm - 1) + kw + 7) / 8 * 8;
-    if (2ll * d.R * (padded_run + d.S * d.C) > kStemStagingBytes - 32) continue;
     for (int bw = 4; bw >= 1; --bw) {
       if (bw > 1 && bw - 1 >= d.W) continue;  // no wider than the output row
       const int halo_w = d.sw * (bw - 1) + d.R;
@@ -258,7 +253,7 @@ bool choose_stem_tile(const Dims& d, const Machine& m, StemTile* out) {
     }
   }
   if (!found) return false;
-  t.packed_filter_bytes = 0;  // every CTA repacks the Filter itself
+  t.packed_filter_bytes = t.filt_bytes;
   int cols = 32;
   while (cols < 2 * 64 * t.bw) cols *= 2;  // two accumulator buffers of 64*bw columns
   t.tmem_cols = cols;
@@ -269,8 +264,7 @@ bool choose_stem_tile(const Dims& d, const Machine& m, StemTile* out) {
   if (t.tiles > 0x7fffffffll) return false;
   t.grid = int(std::min<long long>(t.tiles, m.sm_count));
   t.smem_bytes =
-      std::max(int(t.i_stages * t.img_stage_bytes + t.filt_bytes) + kStemStagingBytes + reserve,
-               117760);
+      std::max(int(t.i_stages * t.img_stage_bytes + t.filt_bytes) + reserve, 117760);
   t.words_smem = double(t.tiles) * (t.img_stage_bytes / 2) + double(t.grid) * (t.filt_bytes / 2) +
                  double(d.K) * d.H * d.W * d.B;
   *out = t;

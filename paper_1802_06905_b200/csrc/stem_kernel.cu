@@ -8,8 +8,7 @@
 // a block (c) is merged with its neighbour (s) so that the block is full.
 //
 // One MMA (M = 128, N = 64*bw, K = 16):
-//   A (rows)  = Filter column r, K-major, repacked by every CTA at its start and resident in
-//               shared memory for the whole kernel (no packing kernel, no scratch).  When
+//   A (rows)  = Filter column r, K-major, resident in shared memory for the whole kernel.  When
 //               K <= 64 the 128 rows are STACKED output rows: row j*kpad + k holds filter k shifted
 //               down by j*sh*C window rows, so one MMA over one Image window yields the bhm = 128/kpad
 //               consecutive output rows h0 .. h0+bhm-1 (their windows overlap almost entirely);
@@ -39,7 +38,6 @@ namespace {
 // taking every other pixel of a tile)
 constexpr int kStemThreads = 320;
 constexpr int kStemEpiThreads = 256;
-constexpr uint32_t kStemStagingBytes = 65536;
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, int c0, int c1,
                                             int c2, uint32_t bar) {
@@ -50,51 +48,97 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm,
       : "memory");
 }
 
-__device__ __forceinline__ void tma_store_4d(const CUtensorMap* tm, int c0, int c1, int c2, int c3,
-                                             uint32_t src) {
-  asm volatile(
-      "cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%1, %2, %3, %4}], [%5];" ::
-          "l"(reinterpret_cast<uint64_t>(tm)),
-      "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(src)
-      : "memory");
-}
-__device__ __forceinline__ void bulk_commit() {
-  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-}
-// until all but the newest bulk-store group of this thread have READ their shared-memory source
-__device__ __forceinline__ void bulk_wait_read_1() {
-  asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-}
-// until every bulk store of this thread has completed altogether
-__device__ __forceinline__ void bulk_wait_all() {
-  asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-}
-__device__ __forceinline__ void fence_proxy_async_smem() {
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-}
-__device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
-}
-__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c,
-                                             uint32_t d) {
-  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d)
-               : "memory");
-}
-__device__ __forceinline__ void st_shared_u16(uint32_t addr, unsigned short v) {
-  asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"(v) : "memory");
-}
-__device__ __forceinline__ uint32_t ld_shared_u32(uint32_t addr) {
-  uint32_t v;
-  asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(addr));
-  return v;
-}
-__device__ __forceinline__ uint32_t ld_shared_u16(uint32_t addr) {
-  uint32_t v;
-  asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(addr));
-  return v;
+// 32 consecutive images of one (k, h, w): 64 B (bf16) or 128 B (fp32), written as whole 32-byte sectors
+template <typename OutT>
+__device__ __forceinline__ void store_run(OutT* dst, const uint32_t (&v)[32]) {
+  if constexpr (sizeof(OutT) == 4) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      st_global_v8(dst + 8 * i, v[8 * i], v[8 * i + 1], v[8 * i + 2], v[8 * i + 3], v[8 * i + 4],
+                   v[8 * i + 5], v[8 * i + 6], v[8 * i + 7]);
+  } else {
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+      st_global_v8(dst + 16 * i, pack_bf16x2(v[16 * i + 0], v[16 * i + 1]),
+                   pack_bf16x2(v[16 * i + 2], v[16 * i + 3]),
+                   pack_bf16x2(v[16 * i + 4], v[16 * i + 5]),
+                   pack_bf16x2(v[16 * i + 6], v[16 * i + 7]),
+                   pack_bf16x2(v[16 * i + 8], v[16 * i + 9]),
+                   pack_bf16x2(v[16 * i + 10], v[16 * i + 11]),
+                   pack_bf16x2(v[16 * i + 12], v[16 * i + 13]),
+                   pack_bf16x2(v[16 * i + 14], v[16 * i + 15]));
+  }
 }
 
 }  // namespace
+
+// ------------------------------------------------------------------------------------------------
+// Filter packing for the stem kernel.  Block (kt, r, kh) holds 128 rows x 16 window rows: row
+// j*kpad + kk, column jj carries Filter[kt*128 + kk][r][s][c] with s*C + c = kh*16 + jj - j*sh*C
+// (zero outside 0 .. S*C-1, for k >= K and for j >= bhm), in K-major no-swizzle core-matrix order:
+// element (row, jj) at ((row/8)*2 + jj/8)*128 + (row%8)*16 + (jj%8)*2 bytes.  Since (s, c) is
+// contiguous in Filter, the value is element q = kh*16 + jj - j*sh*C of the run Filter[k][r][.][.].
+// One thread writes 16 bytes.  The kernel lets its dependent (the convolution) start at once and
+// does not finish before the kernel in front of it has (see launch_pack_filter).
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+    cconv_pack_filter_stem_kernel(const unsigned short* __restrict__ filter,
+                                  uint4* __restrict__ packed, Dims d, int kpad, int bhm, int khalves,
+                                  long long slots) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const long long slot = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+  if (slot < slots) {
+    const int j16 = int(slot & 255);  // 16-byte slot inside the 4 KB block
+    long long blk = slot >> 8;
+    const int kh = int(blk % khalves);
+    blk /= khalves;
+    const int r = int(blk % d.R);
+    const int kt = int(blk / d.R);
+    const int core = j16 >> 3, row8 = j16 & 7;
+    const int row = (core >> 1) * 8 + row8;
+    const int jj0 = (core & 1) * 8;
+    const int j = row / kpad, kk = row - j * kpad;
+    const int k = kt * 128 + kk;
+    const int SC = d.S * d.C;
+    const int q0 = kh * 16 + jj0 - j * d.sh * d.C;
+    unsigned short e[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) e[i] = 0;
+    if (k < d.K && j < bhm && q0 + 8 > 0 && q0 < SC) {
+      const unsigned short* run = filter + ((long long)k * d.R + r) * SC;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int q = q0 + i;
+        if (q >= 0 && q < SC) e[i] = __ldg(run + q);
+      }
+    }
+    uint4 o;
+    o.x = e[0] | (uint32_t(e[1]) << 16);
+    o.y = e[2] | (uint32_t(e[3]) << 16);
+    o.z = e[4] | (uint32_t(e[5]) << 16);
+    o.w = e[6] | (uint32_t(e[7]) << 16);
+    packed[slot] = o;
+  }
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+cudaError_t launch_pack_filter_stem(const void* filter, void* packed, const Dims& d,
+                                    const StemKernelParams& p, cudaStream_t stream) {
+  const long long slots = (long long)p.filt_bytes / 16;
+  const long long blocks = (slots + 255) / 256;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(unsigned(blocks));
+  cfg.blockDim = dim3(256);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, cconv_pack_filter_stem_kernel,
+                            static_cast<const unsigned short*>(filter), static_cast<uint4*>(packed), d,
+                            p.kpad, p.bhm, p.khalves, slots);
+}
 
 // ------------------------------------------------------------------------------------------------
 // The kernel.  Persistent; tile = (128 out-channels) x (64 images) x (bhm output rows) x (bw pixels).
@@ -102,17 +146,13 @@ __device__ __forceinline__ uint32_t ld_shared_u16(uint32_t addr) {
 template <typename OutT>
 __global__ void __launch_bounds__(kStemThreads, 1)
     cconv_stem_kernel(const __grid_constant__ CUtensorMap tm_image,
-                      const __grid_constant__ CUtensorMap tm_out,
-                      const unsigned short* __restrict__ filter, const StemKernelParams p,
-                      int* __restrict__ status) {
+                      const uint8_t* __restrict__ packed_filter, OutT* __restrict__ out,
+                      const StemKernelParams p, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t img_ring = smem0;
   const uint32_t filt_smem = img_ring + uint32_t(p.i_stages) * p.img_stage_bytes;
-  // 8 epilogue warps x 2 buffers x 4 KB: sources of the TMA stores; before the first tile the same
-  // bytes hold the raw Filter while it is repacked
-  const uint32_t stage_smem = filt_smem + p.filt_bytes;
-  const uint32_t bars = stage_smem + kStemStagingBytes;
+  const uint32_t bars = filt_smem + p.filt_bytes;
   const uint32_t bar_ifull = bars;
   const uint32_t bar_iempty = bar_ifull + 8u * p.i_stages;
   const uint32_t bar_filt = bar_iempty + 8u * p.i_stages;
@@ -135,7 +175,7 @@ __global__ void __launch_bounds__(kStemThreads, 1)
       mbar_init(bar_ifull + 8u * s, 1);
       mbar_init(bar_iempty + 8u * s, 1);
     }
-    mbar_init(bar_filt, kStemEpiThreads);  // every thread of the epilogue warps arrives once
+    mbar_init(bar_filt, 1);
     for (int a = 0; a < 2; ++a) {
       mbar_init(bar_tfull + 8u * a, 1);
       mbar_init(bar_tempty + 8u * a, kStemEpiThreads / 32);  // one arrival per epilogue warp
@@ -144,7 +184,6 @@ __global__ void __launch_bounds__(kStemThreads, 1)
     *abort_flag = 0;
     fence_barrier_init();
     prefetch_tensormap(&tm_image);
-    prefetch_tensormap(&tm_out);
   }
   if (warp == 1) {
     tmem_alloc(slot_addr, uint32_t(p.tmem_cols));
@@ -164,6 +203,16 @@ __global__ void __launch_bounds__(kStemThreads, 1)
       bool ok = true;
       long long t_wait = 0;
       const uint32_t n_st = uint32_t(p.i_stages);
+      // The packed Filter is written by the kernel launched just before this one.  Once that
+      // kernel is complete (and with it everything older in the stream), the next packing kernel
+      // may start: it writes the other scratch buffer while this kernel runs.
+      asm volatile("griddepcontrol.wait;" ::: "memory");
+      asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+      mbar_arrive_expect_tx(bar_filt, p.filt_bytes);
+      for (uint32_t off = 0; off < p.filt_bytes; off += 16384u) {
+        const uint32_t n = p.filt_bytes - off < 16384u ? p.filt_bytes - off : 16384u;
+        bulk_load(filt_smem + off, packed_filter + off, n, bar_filt);
+      }
       for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x, ++it) {
         int t = tile / p.tiles_k;
         const int wt = t % p.tiles_w;
@@ -186,6 +235,13 @@ __global__ void __launch_bounds__(kStemThreads, 1)
       }
       if (tr) tr[2] = (unsigned long long)t_wait;
       drain_ring(bar_ifull, it, n_st, status, limit);
+      const uint64_t t0 = globaltimer_ns();
+      while (!mbar_try_wait(bar_filt, 0)) {
+        if (globaltimer_ns() - t0 > limit) {
+          atomicOr(status, kStatDrainWait);
+          break;
+        }
+      }
     }
   } else if (warp == 1) {
     // ===================== MMA issuer (whole warp walks, one lane issues) =====================
@@ -259,146 +315,13 @@ __global__ void __launch_bounds__(kStemThreads, 1)
     // ===================== epilogue warps =====================
     const int q = warp & 3;            // this warp may touch TMEM lanes [32q, 32q+32)
     const int eset = (warp - 2) >> 2;  // 0: even pixels of a tile, 1: odd pixels
-    const int et = (warp - 2) * 32 + lane;  // 0..255
-    // ---- phase 0: repack the Filter into the resident MMA blocks ----
-    // Block (kt, r, kh) holds 128 rows x 16 window rows: row j*kpad + kk, column jj carries
-    // Filter[kt*128 + kk][r][s][c] with s*C + c = kh*16 + jj - j*sh*C (zero outside 0 .. S*C-1, for
-    // k >= K and for j >= bhm), in K-major no-swizzle core-matrix order: element (row, jj) at
-    // ((row/8)*2 + jj/8)*128 + (row%8)*16 + (jj%8)*2 bytes.  Since (s, c) is contiguous in Filter,
-    // the value is simply element q = kh*16 + jj - j*sh*C of the run Filter[k][r][.][.].  The raw
-    // Filter passes through shared memory in chunks of whole out-channels, every run padded with
-    // `lead` zeros in front and zeros behind up to P elements, so that any 8 consecutive window rows
-    // of any stacked row are 8 consecutive elements there, with no bounds to test.
-    {
-      const long long pk0 = tr ? clock64() : 0;
-      for (uint32_t off = uint32_t(et) * 16u; off < p.filt_bytes; off += 16u * kStemEpiThreads)
-        st_shared_v4(filt_smem + off, 0u, 0u, 0u, 0u);
-      const int SC = p.S * p.C;
-      const int lead = shc * (p.bhm - 1);
-      const int P = (lead + p.kw + 7) & ~7;  // padded run length, elements
-      // per out-channel: R raw runs of SC elements and R padded runs of P elements
-      const int kc_max = int((kStemStagingBytes - 32u) / (2u * uint32_t(p.R * (SC + P))));  // >= 1
-      const int kc = p.K < kc_max ? p.K : kc_max;
-      const uint32_t pad_smem = stage_smem;                              // [runs][P]
-      const uint32_t raw_base = stage_smem + 2u * uint32_t(kc * p.R * P);  // 16-byte aligned
-      for (int k0 = 0; k0 < p.K; k0 += kc) {
-        const int nk = p.K - k0 < kc ? p.K - k0 : kc;
-        const int runs = nk * p.R;
-        named_bar_sync(1, kStemEpiThreads);  // previous chunk no longer read
-        // (a) the chunk's raw bytes, as 16-byte vectors; shared and global addresses stay congruent
-        //     mod 16 so that the vectors line up
-        const unsigned short* g = filter + (long long)k0 * p.R * SC;
-        const uint32_t mis = uint32_t(reinterpret_cast<uintptr_t>(g) & 15u);
-        const uint32_t raw = raw_base + mis;  // address of element 0 of the chunk
-        const int n = runs * SC;
-        int head = int(((16u - mis) & 15u) >> 1);
-        if (head > n) head = n;
-        const int nvec = (n - head) >> 3;
-        const int tail0 = head + nvec * 8;
-        if (et < head) st_shared_u16(raw + 2u * et, __ldg(g + et));
-        const uint4* gv = reinterpret_cast<const uint4*>(g + head);
-        for (int i0 = 0; i0 < nvec; i0 += 4 * kStemEpiThreads) {
-          uint4 v[4];
-#pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            const int i = i0 + u * kStemEpiThreads + et;
-            if (i < nvec) v[u] = __ldg(gv + i);
-          }
-#pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            const int i = i0 + u * kStemEpiThreads + et;
-            if (i < nvec) st_shared_v4(raw + 2u * head + 16u * i, v[u].x, v[u].y, v[u].z, v[u].w);
-          }
-        }
-        if (et < n - tail0) st_shared_u16(raw + 2u * (tail0 + et), __ldg(g + tail0 + et));
-        // (b) zero the padded runs
-        for (uint32_t off = uint32_t(et) * 16u; off < uint32_t(runs * P) * 2u;
-             off += 16u * kStemEpiThreads)
-          st_shared_v4(pad_smem + off, 0u, 0u, 0u, 0u);
-        named_bar_sync(1, kStemEpiThreads);
-        if (tr && et == 64) tr[15] = (unsigned long long)(clock64() - pk0);
-        // (c) raw run -> padded run, `lead` elements in
-        for (int run = et; run < runs; run += kStemEpiThreads) {
-          const uint32_t src = raw + 2u * uint32_t(run * SC);
-          const uint32_t dst = pad_smem + 2u * uint32_t(run * P + lead);
-#pragma unroll 4
-          for (int i = 0; i < SC; ++i)
-            st_shared_u16(dst + 2u * i, (unsigned short)ld_shared_u16(src + 2u * i));
-        }
-        named_bar_sync(1, kStemEpiThreads);
-        if (tr && et == 64) tr[12] = (unsigned long long)(clock64() - pk0);
-        const int combos = nk * p.bhm * 2;
-        for (int ci = et; ci < combos; ci += kStemEpiThreads) {
-          const int half = ci & 1, rest = ci >> 1;
-          const int j = rest / nk, kl = rest - j * nk;
-          const int k = k0 + kl;
-          const int kt = k >> 7, kk = k & 127;  // kpad is 128 whenever K > 128
-          const int row = j * p.kpad + kk;
-          uint32_t dst = filt_smem + uint32_t(kt * p.units) * 4096u +
-                         uint32_t(((row >> 3) * 2 + half) * 128 + (row & 7) * 16);
-          const int qbase = half * 8 - j * shc;  // window row -> element of the run
-          const bool even = ((lead + qbase) & 1) == 0;
-          uint32_t src_r = pad_smem + 2u * uint32_t(kl * p.R * P + lead + qbase);
-          for (int r = 0; r < p.R; ++r, src_r += 2u * P) {
-            uint32_t src = src_r;
-            for (int kh = 0; kh < p.khalves; ++kh, dst += 4096u, src += 32u) {
-              const int q0 = kh * 16 + qbase;
-              if (q0 + 8 <= 0 || q0 >= SC) continue;  // stays zero
-              if (even) {
-                st_shared_v4(dst, ld_shared_u32(src), ld_shared_u32(src + 4u), ld_shared_u32(src + 8u),
-                             ld_shared_u32(src + 12u));
-              } else {
-                uint32_t e[8];
-#pragma unroll
-                for (int i = 0; i < 8; ++i) e[i] = ld_shared_u16(src + 2u * i);
-                st_shared_v4(dst, e[0] | (e[1] << 16), e[2] | (e[3] << 16), e[4] | (e[5] << 16),
-                             e[6] | (e[7] << 16));
-              }
-            }
-          }
-        }
-      }
-      fence_proxy_async_smem();  // the MMAs read these generic-proxy writes through the async proxy
-      if (tr && et == 64) tr[14] = (unsigned long long)(clock64() - pk0);
-      mbar_arrive(bar_filt);
-      named_bar_sync(1, kStemEpiThreads);  // the raw area becomes the store staging buffers
-    }
-
-    // ---- tiles: TMEM -> registers -> swizzled staging rows -> TMA store ----
-    // TMEM lane = j*kpad + kk: stacked output row j (uniform in a warp), out-channel kk (32
-    // consecutive ones in a warp).  One staging buffer = [32 out-channels][128 B] = the 64 (bf16) or
-    // 32 (fp32) images of one pixel, 16-byte chunks XOR-swizzled by the row as the store's tensor
-    // map expects, so that the 8 lanes of a store phase hit 8 different bank groups.
-    const int j = (q * 32) / p.kpad;
-    const int kk0 = q * 32 - j * p.kpad;
-    const uint32_t my_stage = stage_smem + uint32_t(warp - 2) * 8192u;
-    const uint32_t row_addr = uint32_t(lane) * 128u, x7 = uint32_t(lane & 7) << 4;
-    uint32_t cnt = 0, abuf = 0, aph = 0;
-    long long t_wf = 0, t_busy = 0, t_ld = 0, t_rd = 0, t_fence = 0, t_issue = 0;
-    auto emit = [&](const uint32_t(&r)[32], bool ok, int b0, int w, int h, int k0) {
-      const uint32_t buf = my_stage + (cnt & 1u) * 4096u;
-      const long long e0 = tr ? clock64() : 0;
-      if (lane == 0) bulk_wait_read_1();  // the store issued two buffers ago has read this one
-      __syncwarp();
-      if (tr) t_rd += clock64() - e0;
-#pragma unroll
-      for (int c = 0; c < 8; ++c)
-        st_shared_v4(buf + row_addr + (uint32_t(c << 4) ^ x7), r[4 * c], r[4 * c + 1], r[4 * c + 2],
-                     r[4 * c + 3]);
-      const long long e1 = tr ? clock64() : 0;
-      fence_proxy_async_smem();
-      __syncwarp();
-      const long long e2 = tr ? clock64() : 0;
-      if (lane == 0) {
-        if (ok) tma_store_4d(&tm_out, b0, w, h, k0, buf);  // rows k >= K are clipped by the map
-        bulk_commit();
-      }
-      if (tr) {
-        t_fence += e2 - e1;
-        t_issue += clock64() - e2;
-      }
-      ++cnt;
-    };
+    // TMEM lane = j*kpad + kk: stacked output row j (uniform in a warp), out-channel kk.  A lane
+    // reads the 64 images of one pixel and writes them as one 128-byte (bf16) or 256-byte (fp32) run
+    // of Out, in whole 32-byte sectors.
+    const int L = q * 32 + lane;
+    const int j = L / p.kpad, kk = L - j * p.kpad;
+    uint32_t abuf = 0, aph = 0;
+    long long t_wf = 0, t_busy = 0, t_ld = 0;
     for (int tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
       int t = tile;
       const int kt = t % p.tiles_k;
@@ -406,7 +329,7 @@ __global__ void __launch_bounds__(kStemThreads, 1)
       const int wt = t % p.tiles_w;
       t /= p.tiles_w;
       const int ht = t % p.tiles_h, bt = t / p.tiles_h;
-      const int k0 = kt * 128 + kk0;
+      const int k = kt * 128 + kk;
       const int h = ht * p.bhm + j;
       const long long c0 = tr ? clock64() : 0;
       if (!mbar_wait_warp(bar_tfull + 8u * abuf, aph, abort_flag, status, kStatEpilogueWait, limit))
@@ -414,7 +337,8 @@ __global__ void __launch_bounds__(kStemThreads, 1)
       const long long c1 = tr ? clock64() : 0;
       tc_fence_after();
       const uint32_t t_base = tmem_base + (uint32_t(q * 32) << 16) + abuf * uint32_t(p.acc_cols);
-      const bool row_ok = (k0 < p.K) && (j < p.bhm) && (h < p.H);
+      const bool row_ok = (k < p.K) && (j < p.bhm) && (h < p.H);
+      OutT* row = out + (((long long)k * p.H + h) * p.W + wt * p.bw) * p.B + bt * 64;
       for (int px = eset; px < p.bw; px += 2) {
         uint32_t va[32], vb[32];
         const long long l0 = tr ? clock64() : 0;
@@ -422,19 +346,10 @@ __global__ void __launch_bounds__(kStemThreads, 1)
         tmem_ld_32x32b_x32(t_base + uint32_t(px * 64 + 32), vb);
         tmem_ld_wait();
         if (tr) t_ld += clock64() - l0;
-        const int w = wt * p.bw + px;
-        const bool ok = row_ok && w < p.W;
-        if constexpr (sizeof(OutT) == 4) {
-          emit(va, ok, bt * 64, w, h, k0);
-          emit(vb, ok, bt * 64 + 32, w, h, k0);
-        } else {
-          uint32_t pk[32];
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            pk[i] = pack_bf16x2(va[2 * i], va[2 * i + 1]);
-            pk[16 + i] = pack_bf16x2(vb[2 * i], vb[2 * i + 1]);
-          }
-          emit(pk, ok, bt * 64, w, h, k0);
+        if (row_ok && wt * p.bw + px < p.W) {
+          OutT* dst = row + (long long)px * p.B;
+          store_run(dst, va);
+          store_run(dst + 32, vb);
         }
       }
       tc_fence_before();
@@ -451,10 +366,7 @@ __global__ void __launch_bounds__(kStemThreads, 1)
       tr[6] = (unsigned long long)t_wf;
       tr[7] = (unsigned long long)t_busy;
       tr[10] = (unsigned long long)t_ld;
-      tr[11] = (unsigned long long)t_rd;
-      tr[13] = (unsigned long long)t_issue;
     }
-    if (lane == 0) bulk_wait_all();  // Out is written before the CTA leaves
   }
 
   // ===================== teardown =====================
@@ -475,16 +387,27 @@ cudaError_t stem_kernel_prepare(int smem_bytes) {
                               smem_bytes);
 }
 
-cudaError_t launch_stem(const CUtensorMap& tm_image, const CUtensorMap& tm_out, const void* filter,
+cudaError_t launch_stem(const CUtensorMap& tm_image, const void* packed_filter, void* out,
                         bool out_f32, const StemKernelParams& p, int grid, int smem_bytes,
                         int* status, cudaStream_t stream) {
-  const unsigned short* f = static_cast<const unsigned short*>(filter);
+  const uint8_t* pf = static_cast<const uint8_t*>(packed_filter);
+  // Programmatic dependent launch: the kernel may begin while the Filter-packing kernel in front of
+  // it is still running; only its producer waits for that kernel's results.
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(unsigned(grid));
+  cfg.blockDim = dim3(kStemThreads);
+  cfg.dynamicSmemBytes = size_t(smem_bytes);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
   if (out_f32)
-    cconv_stem_kernel<float><<<grid, kStemThreads, smem_bytes, stream>>>(tm_image, tm_out, f, p, status);
-  else
-    cconv_stem_kernel<__nv_bfloat16><<<grid, kStemThreads, smem_bytes, stream>>>(tm_image, tm_out, f, p,
-                                                                                status);
-  return cudaGetLastError();
+    return cudaLaunchKernelEx(&cfg, cconv_stem_kernel<float>, tm_image, pf, static_cast<float*>(out),
+                              p, status);
+  return cudaLaunchKernelEx(&cfg, cconv_stem_kernel<__nv_bfloat16>, tm_image, pf,
+                            static_cast<__nv_bfloat16*>(out), p, status);
 }
 
 }  // namespace cconv
