@@ -88,6 +88,11 @@ typedef struct {
    * fast-memory level = shared memory of one CTA; slow side = L2/HBM. */
   double tile_words_smem; /* words staged into shared memory over the whole problem + Out words */
   double compulsory_words; /* |Image| + |Filter| + |Out| with the real Image extent             */
+  /* Wave-quantisation tail (HALO variant): when the main tiling would fill its last wave of CTAs
+   * only partly, output rows h >= tail_h0 run as a second launch with the tile below, started
+   * while the first is in its last wave.  tail_h0 == H: no tail; `tiles` and `grid` above then
+   * describe the only launch, otherwise the main one. */
+  int tail_h0, tail_bb, tail_bc, tail_bw, tail_bh, tail_tiles, tail_grid;
   double scratch_bytes;   /* one packed Filter; the plan owns two such device buffers and
                              alternates between them from call to call                          */
 } cconv_plan_info;

@@ -50,6 +50,9 @@ class PlanInfo(ctypes.Structure):
         ("tiles", ctypes.c_int),
         ("smem_bytes", ctypes.c_int), ("tmem_cols", ctypes.c_int),
         ("tile_words_smem", ctypes.c_double), ("compulsory_words", ctypes.c_double),
+        ("tail_h0", ctypes.c_int), ("tail_bb", ctypes.c_int), ("tail_bc", ctypes.c_int),
+        ("tail_bw", ctypes.c_int), ("tail_bh", ctypes.c_int), ("tail_tiles", ctypes.c_int),
+        ("tail_grid", ctypes.c_int),
         ("scratch_bytes", ctypes.c_double),
     ]
 

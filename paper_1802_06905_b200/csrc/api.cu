@@ -50,6 +50,11 @@ struct cconv_plan {
   double lp_G = 0, lp_words = 0;
   HaloTile tile{};
   HaloKernelParams kp{};
+  // Optional second launch of a call: the last output rows with a smaller tile, filling the SMs
+  // that the last wave of the main launch leaves idle.
+  bool has_tail = false;
+  HaloTile tail{};
+  HaloKernelParams kp_tail{};
   StemTile stile{};
   StemKernelParams skp{};
   int* d_status = nullptr;
@@ -68,6 +73,7 @@ struct cconv_plan {
   mutable std::mutex mu;
   mutable const void* tm_image_ptr = nullptr;
   mutable CUtensorMap tm_image{};
+  mutable CUtensorMap tm_image_tail{};
 };
 
 namespace {
@@ -172,7 +178,34 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
     else variant = halo_ok ? CCONV_VARIANT_HALO : CCONV_VARIANT_SIMT;
   }
   pl->variant = variant;
-  if (variant == CCONV_VARIANT_HALO) build_halo_params(pl->d, pl->tile, &pl->kp);
+  if (variant == CCONV_VARIANT_HALO) {
+    const bool forced = force[0] || force[1] || force[2] || force[3] || force[4];
+    int keep = 0;
+    bool tail_ok = !forced && !env_int("CCONV_NO_TAIL", 0) &&
+                   choose_halo_tail(pl->d, pl->m, pl->tile, &keep, &pl->tail);
+    if (const char* f = std::getenv("CCONV_FORCE_TAIL")) {
+      // diagnostics: "rows of tiles kept,bw,bh,bc,stages,bb" for the tail
+      int tf[5] = {0, 0, 0, 0, 0};
+      tail_ok = false;
+      if (std::sscanf(f, "%d,%d,%d,%d,%d,%d", &keep, &tf[0], &tf[1], &tf[2], &tf[3], &tf[4]) >= 1 &&
+          keep >= 1 && keep < pl->tile.tiles_h) {
+        Dims dr = pl->d;
+        dr.H = pl->d.H - keep * pl->tile.bh;
+        tail_ok = dr.H > 0 && choose_halo_tile(dr, pl->m, tf, &pl->tail);
+      }
+    }
+    if (tail_ok) {
+      pl->has_tail = true;
+      const long long per_row = pl->tile.tiles / pl->tile.tiles_h;
+      pl->tile.tiles_h = keep;
+      pl->tile.tiles = per_row * keep;
+      pl->tile.grid = int(std::min<long long>(pl->tile.tiles, pl->m.sm_count));
+      build_halo_params(pl->d, pl->tail, &pl->kp_tail);
+      pl->kp_tail.h0 = keep * pl->tile.bh;
+      pl->kp_tail.tail = 1;
+    }
+    build_halo_params(pl->d, pl->tile, &pl->kp);
+  }
   if (variant == CCONV_VARIANT_STEM) build_stem_params(pl->d, pl->stile, &pl->skp);
 
   if (device >= 0) {
@@ -182,7 +215,7 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
     if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&pl->d_status), 256);
     if (e == cudaSuccess) e = cudaMemset(pl->d_status, 0, 256);
     if (e == cudaSuccess && variant == CCONV_VARIANT_HALO)
-      e = halo_kernel_prepare(pl->tile.smem_bytes);
+      e = halo_kernel_prepare(std::max(pl->tile.smem_bytes, pl->has_tail ? pl->tail.smem_bytes : 0));
     if (variant == CCONV_VARIANT_HALO) pl->packed_bytes = size_t(pl->tile.packed_filter_bytes);
     if (variant == CCONV_VARIANT_STEM) pl->packed_bytes = size_t(pl->stile.packed_filter_bytes);
     pl->packed_bytes = (pl->packed_bytes + 255) & ~size_t(255);
@@ -221,6 +254,11 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
                  B, C, K, W, H, R, S, sw, sh, variant, t.bb, t.bw, t.bh, t.bc, t.i_stages,
                  t.f_stages, t.uf, t.acc_bufs, t.tmem_cols, t.tiles, t.grid, t.smem_bytes,
                  t.est_cycles);
+    if (pl->has_tail)
+      std::fprintf(stderr, "[cconv]   tail from h=%d: tile bb=%d bw=%d bh=%d bc=%d i_stages=%d tiles=%lld "
+                           "grid=%d smem=%d\n",
+                   pl->kp_tail.h0, pl->tail.bb, pl->tail.bw, pl->tail.bh, pl->tail.bc,
+                   pl->tail.i_stages, pl->tail.tiles, pl->tail.grid, pl->tail.smem_bytes);
   }
   *plan_out = pl;
   return CCONV_OK;
@@ -243,6 +281,7 @@ int cconv_plan_info_get(const cconv_plan* pl, cconv_plan_info* o) {
   o->variant = pl->variant;
   o->out_dtype = pl->out_dtype;
   const Dims& d = pl->d;
+  o->tail_h0 = d.H;
   o->compulsory_words =
       double(d.Wi()) * d.Hi() * d.C * d.B + double(d.K) * d.R * d.S * d.C + double(d.K) * d.H * d.W * d.B;
   if (pl->variant == CCONV_VARIANT_STEM) {
@@ -262,6 +301,18 @@ int cconv_plan_info_get(const cconv_plan* pl, cconv_plan_info* o) {
     o->smem_bytes = t.smem_bytes; o->tmem_cols = t.tmem_cols;
     o->tile_words_smem = t.words_smem;
     o->scratch_bytes = double(t.packed_filter_bytes);
+    if (pl->has_tail) {
+      const HaloTile& u = pl->tail;
+      o->tail_h0 = pl->kp_tail.h0;
+      o->tail_bb = u.bb; o->tail_bc = u.bc; o->tail_bw = u.bw; o->tail_bh = u.bh;
+      o->tail_tiles = int(u.tiles); o->tail_grid = u.grid;
+      // rows kept by the main tiling: scale its staged words; then add the tail's (minus the Out
+      // words both estimates include)
+      const double out_words = double(d.K) * d.H * d.W * d.B;
+      o->tile_words_smem = double(t.tiles) * ((t.words_smem - out_words) /
+                                              (double(t.tiles) / t.tiles_h * ((d.H + t.bh - 1) / t.bh))) +
+                           (u.words_smem - double(d.K) * (d.H - pl->kp_tail.h0) * d.W * d.B) + out_words;
+    }
   }
   return CCONV_OK;
 }
@@ -294,7 +345,7 @@ int cconv_forward_planned(const cconv_plan* pl, const void* Image, const void* F
     cudaError_t e = launch_simt(Image, Filter, Out, pl->out_dtype == CCONV_OUT_F32, pl->d, stream);
     return e == cudaSuccess ? CCONV_OK : cuda_fail(e, "launch_simt");
   }
-  CUtensorMap tmi;
+  CUtensorMap tmi, tmi_tail;
   void* packed = nullptr;
   {
     // the tensor map is rebuilt only when the Image pointer changes
@@ -303,10 +354,13 @@ int cconv_forward_planned(const cconv_plan* pl, const void* Image, const void* F
       int rc = pl->variant == CCONV_VARIANT_STEM
                    ? encode_stem_image_map(pl->d, pl->stile, Image, &pl->tm_image)
                    : encode_image_map(pl->d, pl->tile, Image, &pl->tm_image);
+      if (rc == CCONV_OK && pl->has_tail)
+        rc = encode_image_map(pl->d, pl->tail, Image, &pl->tm_image_tail);
       if (rc != CCONV_OK) return rc;
       pl->tm_image_ptr = Image;
     }
     tmi = pl->tm_image;
+    if (pl->has_tail) tmi_tail = pl->tm_image_tail;
     packed = static_cast<char*>(pl->d_packed) + (pl->calls++ & 1u) * pl->packed_bytes;
   }
   if (pl->variant == CCONV_VARIANT_STEM) {
@@ -321,6 +375,9 @@ int cconv_forward_planned(const cconv_plan* pl, const void* Image, const void* F
   if (e != cudaSuccess) return cuda_fail(e, "launch_pack_filter");
   e = launch_halo(tmi, packed, Out, pl->out_dtype == CCONV_OUT_F32, pl->kp, pl->tile.grid,
                   pl->tile.smem_bytes, pl->d_status, stream);
+  if (e == cudaSuccess && pl->has_tail)
+    e = launch_halo(tmi_tail, packed, Out, pl->out_dtype == CCONV_OUT_F32, pl->kp_tail,
+                    pl->tail.grid, pl->tail.smem_bytes, pl->d_status, stream);
   return e == cudaSuccess ? CCONV_OK : cuda_fail(e, "launch_halo");
 }
 

@@ -429,7 +429,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         const int wt = t % p.tiles_w; t /= p.tiles_w;
         const int ht = t;
         const int b0 = bt * p.bb;
-        const int x0 = wt * p.bw * p.sw, y0 = ht * p.bh * p.sh;
+        const int x0 = wt * p.bw * p.sw, y0 = (p.h0 + ht * p.bh) * p.sh;
         for (int cc = 0, c0 = 0; cc < cchunks; ++cc, c0 += p.bc, ++seq) {
           if ((seq & (i_prod - 1u)) == me) {
             if (!mbar_wait(bar_iempty + 8u * s, ph ^ 1u, abort_flag, status, kStatProducerWait,
@@ -462,7 +462,9 @@ __global__ void __launch_bounds__(kThreads, 1)
       // The packed Filter is written by the kernel launched just before this one.  Once that
       // kernel is complete (and with it everything older in the stream), the next packing kernel
       // may start: it writes the other scratch buffer while this kernel runs.
-      asm volatile("griddepcontrol.wait;" ::: "memory");
+      // (A tail launch starts only after every CTA of the main launch has passed this point, so
+      // the packed Filter is known to be complete; it waits at its end instead, see below.)
+      if (!p.tail) asm volatile("griddepcontrol.wait;" ::: "memory");
       if (me == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
       for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
         const int kt = tile % p.tiles_k;
@@ -527,7 +529,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       if (first_tile && threadIdx.x == 64) CCONV_TRACE(8);
       const uint32_t t_base = tmem_base + (uint32_t(q * 32) << 16) + abuf * uint32_t(p.acc_cols);
       for (int hh = 0; hh < p.bh; ++hh) {
-        const int h = ht * p.bh + hh;
+        const int h = p.h0 + ht * p.bh + hh;
         for (int ww = 0; ww < p.bw; ++ww) {
           const int w = wt * p.bw + ww;
           const bool valid = (k < p.K) && (h < p.H) && (w < p.W);
@@ -580,6 +582,9 @@ __global__ void __launch_bounds__(kThreads, 1)
     tc_fence_after();
     tmem_dealloc(tmem_base, uint32_t(p.tmem_cols));
   }
+  // A tail launch runs beside the main launch of the same call; it ends only after that one has,
+  // so that "the last kernel of a call is complete" implies that the whole call is.
+  if (p.tail && threadIdx.x == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
   if (threadIdx.x == 0) CCONV_TRACE(11);
 #undef CCONV_TRACE
 }

@@ -33,6 +33,8 @@ struct HaloKernelParams {
   int i_stages, f_stages;       // ring depths
   int tiles_k, tiles_b, tiles_w, tiles_h;
   int total_tiles;
+  int h0;                       // first output row of this launch (tiles_h counts rows from there)
+  int tail;                     // 1: second launch of a call, started while the first still runs
   int n_mma;                    // N of one MMA = bb*bw
   int acc_cols, acc_bufs, tmem_cols;
   uint32_t img_stage_bytes, filt_stage_bytes;

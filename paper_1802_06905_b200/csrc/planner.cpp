@@ -201,6 +201,7 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[5], HaloT
                                               : std::max(cyc_mma, cyc_copy) + cyc_epi;
           if (t.i_stages == 1) tile_cyc = cyc_mma + cyc_copy + cyc_epi;
           const double waves = std::ceil(double(t.tiles) / t.grid);
+          t.tile_cycles = tile_cyc;
           t.est_cycles = waves * tile_cyc + cyc_epi + 4000.0;
           t.words_smem = double(t.tiles) * (double(t.cchunks) * (img / 2) + double(units) * 2048.0) +
                          double(d.K) * d.H * d.W * d.B;
@@ -215,6 +216,36 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[5], HaloT
     }
   }
   if (found) *out = best;
+  return found;
+}
+
+bool choose_halo_tail(const Dims& d, const Machine& m, const HaloTile& main, int* main_tiles_h,
+                      HaloTile* tail) {
+  if (main.tiles <= main.grid || main.tiles_h < 2) return false;
+  const double waves = double(main.tiles) / main.grid;
+  const double frac = waves - std::floor(waves);
+  if (frac < 1e-9 || frac > 0.75) return false;  // the last wave is full enough
+  const long long per_row = main.tiles / main.tiles_h;
+  const int no_force[5] = {0, 0, 0, 0, 0};
+  bool found = false;
+  double best = main.est_cycles * 0.97;  // must beat the single launch by 3 %
+  for (int keep = main.tiles_h - 1; keep >= 1 && keep >= main.tiles_h - 4; --keep) {
+    Dims dr = d;
+    dr.H = d.H - keep * main.bh;
+    if (dr.H <= 0) continue;
+    HaloTile t;
+    if (!choose_halo_tile(dr, m, no_force, &t)) continue;
+    if (t.tiles > m.sm_count) continue;  // the tail is one partial wave
+    const double main_cyc = std::ceil(double(per_row * keep) / main.grid) * main.tile_cycles;
+    // the tail's CTAs start as SMs fall idle: it costs its own tile time after the main waves
+    const double est = main_cyc + t.tile_cycles + 14.0 * t.bb * t.bw * t.bh + 4000.0;
+    if (est < best) {
+      best = est;
+      *main_tiles_h = keep;
+      *tail = t;
+      found = true;
+    }
+  }
   return found;
 }
 

@@ -53,6 +53,7 @@ struct HaloTile {
   long long packed_filter_bytes = 0;  // scratch: tiles_k * c16 * R*S blocks of 4 KB
   int smem_bytes = 0;
   double est_cycles = 0;   // cost-model estimate for the whole problem, SM cycles
+  double tile_cycles = 0;  // cost-model estimate for one tile on one SM
   double words_smem = 0;   // words staged into shared memory over the whole problem + |Out|
 };
 
@@ -82,6 +83,15 @@ bool halo_supported(const Dims& d, const char** why);
 // Enumerate legal tiles and keep the one with the least estimated time (ties: fewer staged words).
 // `force` may carry "bw,bh,bc,stages,bb" (0 = free) from the CCONV_FORCE_TILE environment variable.
 bool choose_halo_tile(const Dims& d, const Machine& m, const int force[5], HaloTile* out);
+
+// Wave quantisation: when the tiles of the best tiling fill the last wave of the persistent grid
+// only partly, the last output rows may be cheaper as a second launch with a smaller tile whose
+// CTAs fill the SMs that the first launch leaves idle.  Returns true and sets *main_tiles_h (rows of
+// tiles the main tiling keeps, counted from h = 0) and *tail (tiling of the remaining output rows,
+// planned as a problem with H = the remaining rows) when the model predicts a gain; `main` is the
+// whole-problem tile from choose_halo_tile.
+bool choose_halo_tail(const Dims& d, const Machine& m, const HaloTile& main, int* main_tiles_h,
+                      HaloTile* tail);
 
 // The stem kernel needs B % 64 == 0 and the resident Filter plus two Image windows to fit in shared
 // memory.
