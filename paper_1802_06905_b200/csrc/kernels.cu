@@ -50,6 +50,7 @@ __global__ void __launch_bounds__(256) cconv_simt_kernel(const __nv_bfloat16* __
         const __nv_bfloat16* ip =
             image + (((long long)(r + d.sw * w) * Hi + (s + d.sh * h)) * d.C) * d.B + b;
         const __nv_bfloat16* fp = filter + (((long long)k0 * d.R + r) * d.S + s) * d.C;
+#pragma unroll 4
         for (int c = 0; c < d.C; ++c) {
           const float x = __bfloat162float(ip[(long long)c * d.B]);
 #pragma unroll
@@ -67,20 +68,33 @@ __global__ void __launch_bounds__(256) cconv_simt_kernel(const __nv_bfloat16* __
 
 cudaError_t launch_simt(const void* image, const void* filter, void* out, bool out_f32,
                         const Dims& d, cudaStream_t stream) {
-  constexpr int KT = 4;
+  // Four out-channels per thread reuse each Image value four times; problems too small to fill
+  // the SMs that way take one out-channel per thread and smaller blocks instead (more threads,
+  // shorter dependent chains per thread).
+  const long long outputs = (long long)d.K * d.H * d.W * d.B;
+  const bool small = outputs < 148ll * 1024 * 4;
+  const int KT = small ? 1 : 4;
   const long long total = (long long)((d.K + KT - 1) / KT) * d.H * d.W * d.B;
-  const int threads = 256;
+  const int threads = small ? 64 : 256;
   long long blocks = (total + threads - 1) / threads;
   if (blocks > 148ll * 64) blocks = 148ll * 64;
   if (blocks < 1) blocks = 1;
   const __nv_bfloat16* im = static_cast<const __nv_bfloat16*>(image);
   const __nv_bfloat16* fl = static_cast<const __nv_bfloat16*>(filter);
-  if (out_f32)
-    cconv_simt_kernel<KT, float><<<(unsigned)blocks, threads, 0, stream>>>(
+  if (small) {
+    if (out_f32)
+      cconv_simt_kernel<1, float><<<(unsigned)blocks, threads, 0, stream>>>(
+          im, fl, static_cast<float*>(out), d);
+    else
+      cconv_simt_kernel<1, __nv_bfloat16><<<(unsigned)blocks, threads, 0, stream>>>(
+          im, fl, static_cast<__nv_bfloat16*>(out), d);
+  } else if (out_f32) {
+    cconv_simt_kernel<4, float><<<(unsigned)blocks, threads, 0, stream>>>(
         im, fl, static_cast<float*>(out), d);
-  else
-    cconv_simt_kernel<KT, __nv_bfloat16><<<(unsigned)blocks, threads, 0, stream>>>(
+  } else {
+    cconv_simt_kernel<4, __nv_bfloat16><<<(unsigned)blocks, threads, 0, stream>>>(
         im, fl, static_cast<__nv_bfloat16*>(out), d);
+  }
   return cudaGetLastError();
 }
 

@@ -123,6 +123,17 @@ def test_inspection_plans_are_hardware_legal():
             assert info["stages"] * img_stage + info["filter_stages"] * 4096 <= info["smem_bytes"]
             units = -(-cfg.C // 16) * cfg.R * cfg.S
             assert info["scratch_bytes"] == -(-cfg.K // 128) * units * 4096
+            # wave-quantisation tail: whole rows of main tiles, the rest in one partial wave
+            if info["tail_h0"] < cfg.H:
+                assert info["tail_h0"] % info["bh"] == 0 and info["tail_h0"] > 0
+                per_row = -(-cfg.K // 128) * (cfg.B // info["bb"]) * -(-cfg.W // info["bw"])
+                assert info["tiles"] == per_row * (info["tail_h0"] // info["bh"])
+                rows = cfg.H - info["tail_h0"]
+                assert info["tail_tiles"] == (-(-cfg.K // 128) * (cfg.B // info["tail_bb"]) *
+                                              -(-cfg.W // info["tail_bw"]) * -(-rows // info["tail_bh"]))
+                assert info["tail_tiles"] <= 148
+            else:
+                assert info["tail_tiles"] == 0
             # the staged words can never undercut the bound at the shared-memory size
             assert info["tile_words_smem"] >= max(exp_terms) * 0.999 or max(exp_terms) < info["M_words"]
         elif info["variant"] == binding.VARIANT_STEM:

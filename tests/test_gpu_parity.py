@@ -125,6 +125,28 @@ def test_stem_shapes(c, out_dtype):
     assert info["variant"] == binding.VARIANT_STEM
 
 
+@pytest.mark.parametrize("out_dtype", DTYPES, ids=DT_IDS)
+def test_halo_tail_launch(monkeypatch, out_dtype):
+    """The wave-quantisation tail: output rows h >= tail_h0 come from a second launch with its own
+    tile, running beside the first; every output must still be Eq. 1."""
+    monkeypatch.setenv("CCONV_FORCE_TILE", "2,2,16,0,64")      # main: 2 x 2 pixels, 5 rows of tiles
+    monkeypatch.setenv("CCONV_FORCE_TAIL", "3,4,1,16,0,64")    # keep 3 rows; rows h >= 6: 4 x 1 pixels
+    c = cs("tail", 64, 40, 160, 8, 9, 3, 3)
+    info = check_full(c, variant=binding.VARIANT_HALO, out_dtype=out_dtype)
+    assert info["tail_h0"] == 6 and info["tail_bw"] == 4 and info["tail_bh"] == 1
+    assert info["tiles"] == 2 * 1 * 4 * 3 and info["tail_tiles"] == 2 * 1 * 2 * 3
+
+
+def test_tail_is_planned_for_the_large_config():
+    cfg = synth.CONFIGS[4]
+    p = binding.Plan(*cfg.dims(), device=0)
+    info = p.info()
+    p.close()
+    assert info["variant"] == binding.VARIANT_HALO
+    assert 0 < info["tail_h0"] < cfg.H and info["tail_h0"] % info["bh"] == 0
+    assert info["tail_tiles"] <= 148 and info["tiles"] % info["grid"] != 1
+
+
 def test_halo_matches_simt_kernel_on_device():
     c = cs("cross", 64, 48, 160, 9, 8, 3, 3)
     ib, fb = synth.make_inputs(c)
