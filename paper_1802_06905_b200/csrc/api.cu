@@ -159,9 +159,10 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
   theorem1_terms(d, pl->M_words, pl->terms);
   if (pl->M_words > 1.0) tiling_lp(d, pl->M_words, false, pl->lp_tile, &pl->lp_G, &pl->lp_words);
 
-  int force[5] = {0, 0, 0, 0, 0};
+  int force[6] = {0, 0, 0, 0, 0, 0};
   if (const char* f = std::getenv("CCONV_FORCE_TILE"))
-    std::sscanf(f, "%d,%d,%d,%d,%d", &force[0], &force[1], &force[2], &force[3], &force[4]);
+    std::sscanf(f, "%d,%d,%d,%d,%d,%d", &force[0], &force[1], &force[2], &force[3], &force[4],
+                &force[5]);
   const int env_variant = env_int("CCONV_VARIANT", 0);
   if (variant == CCONV_VARIANT_AUTO && env_variant >= 1 && env_variant <= 3) variant = env_variant;
 
@@ -179,13 +180,13 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
   }
   pl->variant = variant;
   if (variant == CCONV_VARIANT_HALO) {
-    const bool forced = force[0] || force[1] || force[2] || force[3] || force[4];
+    const bool forced = force[0] || force[1] || force[2] || force[3] || force[4] || force[5];
     int keep = 0;
     bool tail_ok = !forced && !env_int("CCONV_NO_TAIL", 0) &&
                    choose_halo_tail(pl->d, pl->m, pl->tile, &keep, &pl->tail);
     if (const char* f = std::getenv("CCONV_FORCE_TAIL")) {
       // diagnostics: "rows of tiles kept,bw,bh,bc,stages,bb" for the tail
-      int tf[5] = {0, 0, 0, 0, 0};
+      int tf[6] = {0, 0, 0, 0, 0, 1};
       tail_ok = false;
       if (std::sscanf(f, "%d,%d,%d,%d,%d,%d", &keep, &tf[0], &tf[1], &tf[2], &tf[3], &tf[4]) >= 1 &&
           keep >= 1 && keep < pl->tile.tiles_h) {
@@ -249,9 +250,9 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
     const HaloTile& t = pl->tile;
     std::fprintf(stderr,
                  "[cconv] B%d C%d K%d W%d H%d R%d S%d s%dx%d variant=%d tile bb=%d bw=%d bh=%d "
-                 "bc=%d i_stages=%d f_stages=%d uf=%d acc_bufs=%d tmem=%d tiles=%lld grid=%d smem=%d "
+                 "bc=%d split=%d i_stages=%d f_stages=%d uf=%d acc_bufs=%d tmem=%d tiles=%lld grid=%d smem=%d "
                  "est_cyc=%.0f\n",
-                 B, C, K, W, H, R, S, sw, sh, variant, t.bb, t.bw, t.bh, t.bc, t.i_stages,
+                 B, C, K, W, H, R, S, sw, sh, variant, t.bb, t.bw, t.bh, t.bc, t.split, t.i_stages,
                  t.f_stages, t.uf, t.acc_bufs, t.tmem_cols, t.tiles, t.grid, t.smem_bytes,
                  t.est_cycles);
     if (pl->has_tail)

@@ -64,6 +64,9 @@ void build_halo_params(const Dims& d, const HaloTile& t, HaloKernelParams* out) 
   p.i_stages = t.i_stages; p.f_stages = t.f_stages;
   p.tiles_k = t.tiles_k; p.tiles_b = t.tiles_b; p.tiles_w = t.tiles_w; p.tiles_h = t.tiles_h;
   p.total_tiles = int(t.tiles);
+  p.split = t.split;
+  p.units_cta = p.units / t.split;
+  p.cchunks_cta = t.cchunks / t.split;
   p.h0 = 0;
   p.tail = 0;
   p.n_mma = t.bb * t.bw;

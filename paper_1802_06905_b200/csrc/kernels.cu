@@ -196,6 +196,7 @@ struct MmaCtx {
   volatile int* abort_flag;
   int* status;
   uint64_t limit;
+  int tile_first, tile_step;  // this CTA's tiles: tile_first, tile_first + tile_step, ...
 };
 
 template <int BH>
@@ -220,7 +221,7 @@ __device__ __forceinline__ void mma_role(const HaloKernelParams& p, const MmaCtx
   const bool leader = elect_one();
   uint32_t is = 0, iph = 0, fs = 0, fph = 0, abuf = 0, aph = 0;
   bool ok = true, first_tile = true;
-  const int R = p.R, S = p.S, units = p.units, units_per_img = p.units_per_img;
+  const int R = p.R, S = p.S, units = p.units_cta, units_per_img = p.units_per_img;
   const uint32_t slab16 = p.slab_bytes >> 4, row16 = uint32_t(p.halo_w) * slab16;
   uint32_t off9[9];  // 3x3: halo offset of tap (r, s) = r*3 + s, in 16 B units
 #pragma unroll
@@ -232,12 +233,15 @@ __device__ __forceinline__ void mma_role(const HaloKernelParams& p, const MmaCtx
   const uint32_t hstep16 = uint32_t(p.sh * p.halo_w) * slab16;  // next output row
   const uint32_t kstep16 = p.b_kstep_bytes >> 4;
   const uint32_t img16 = p.img_stage_bytes >> 4, filt16 = p.filt_stage_bytes >> 4;
-  const uint32_t img_ring16 = cx.img_ring >> 4, filt_ring16 = cx.filt_ring >> 4;
+  // A descriptor holds address bits [4,18) of the CTA's own window.  In a cluster launch the
+  // shared-memory addresses of CTA rank r carry r above bit 24; left in, those bits would run into
+  // the descriptor's leading-byte-offset field.
+  const uint32_t img_ring16 = (cx.img_ring >> 4) & 0x3FFFu, filt_ring16 = (cx.filt_ring >> 4) & 0x3FFFu;
   const uint32_t idesc = p.idesc, n_mma = uint32_t(p.n_mma);
   const uint32_t n_ist = uint32_t(p.i_stages), n_fst = uint32_t(p.f_stages);
   const int bh = p.bh, uf = p.uf;
   constexpr uint32_t kBlk16 = kPackedBlockBytes >> 4;
-  for (int tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
+  for (int tile = cx.tile_first; tile < p.total_tiles; tile += cx.tile_step) {
     if (!mbar_wait_warp(cx.bar_tempty + 8u * abuf, aph ^ 1u, cx.abort_flag, cx.status,
                         kStatMmaWaitTmem, cx.limit))
       break;
@@ -359,6 +363,29 @@ __device__ __forceinline__ void mma_role(const HaloKernelParams& p, const MmaCtx
   }
 }
 
+// 32 consecutive images of one (k, h, w): 64 B (bf16) or 128 B (fp32), written as whole 32-byte
+// sectors.
+template <typename OutT>
+__device__ __forceinline__ void store_run32(OutT* dst, const uint32_t (&v)[32]) {
+  if constexpr (sizeof(OutT) == 4) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      st_global_v8(dst + 8 * j, v[8 * j], v[8 * j + 1], v[8 * j + 2], v[8 * j + 3], v[8 * j + 4],
+                   v[8 * j + 5], v[8 * j + 6], v[8 * j + 7]);
+  } else {
+#pragma unroll
+    for (int j = 0; j < 2; ++j)
+      st_global_v8(dst + 16 * j, pack_bf16x2(v[16 * j + 0], v[16 * j + 1]),
+                   pack_bf16x2(v[16 * j + 2], v[16 * j + 3]),
+                   pack_bf16x2(v[16 * j + 4], v[16 * j + 5]),
+                   pack_bf16x2(v[16 * j + 6], v[16 * j + 7]),
+                   pack_bf16x2(v[16 * j + 8], v[16 * j + 9]),
+                   pack_bf16x2(v[16 * j + 10], v[16 * j + 11]),
+                   pack_bf16x2(v[16 * j + 12], v[16 * j + 13]),
+                   pack_bf16x2(v[16 * j + 14], v[16 * j + 15]));
+  }
+}
+
 // ------------------------------------------------------------------------------------------------
 // Halo-tile tcgen05 kernel
 // ------------------------------------------------------------------------------------------------
@@ -380,6 +407,7 @@ __global__ void __launch_bounds__(kThreads, 1)
   const uint32_t bar_tempty = bar_tfull + 16u;
   const uint32_t bar_drain = bar_tempty + 16u;
   const uint32_t slot_addr = bar_drain + 8u;
+  const uint32_t bar_xchg = slot_addr + 8u;  // split launch: the peer's partial sums have arrived
   uint8_t* gen0 = smem_raw + (smem0 - smem_u32(smem_raw));
   volatile uint32_t* tmem_slot =
       reinterpret_cast<volatile uint32_t*>(gen0 + (slot_addr - smem0));
@@ -407,8 +435,11 @@ __global__ void __launch_bounds__(kThreads, 1)
       mbar_init(bar_tempty + 8u * a, 4);  // one arrival per epilogue warp
     }
     mbar_init(bar_drain, 1);
+    mbar_init(bar_xchg, 1);
     *abort_flag = 0;
     fence_barrier_init();
+    // split launch: the peer will copy 128 rows of acc_cols/2 fp32 partial sums into this CTA
+    if (p.split > 1) mbar_arrive_expect_tx(bar_xchg, 128u * uint32_t(p.acc_cols >> 1) * 4u);
     prefetch_tensormap(&tm_image);
   }
   if (warp == 1) {
@@ -421,6 +452,11 @@ __global__ void __launch_bounds__(kThreads, 1)
   const uint32_t tmem_base = *tmem_slot;
   const uint64_t limit = p.wait_limit_ns;
   if (threadIdx.x == 0) CCONV_TRACE(1);
+  // Persistent launch: CTA i takes tiles i, i + grid, ...  Split launch: the two CTAs of cluster i
+  // take tile i once, rank r contracting the r-th half of the channels.
+  const int crank = p.split > 1 ? int(cluster_ctarank()) : 0;
+  const int tile_first = p.split > 1 ? int(blockIdx.x) / p.split : int(blockIdx.x);
+  const int tile_step = p.split > 1 ? p.total_tiles : int(gridDim.x);
 
   // Ring positions advance by increment-and-wrap; a runtime division per stage would cost more
   // single-thread issue time than the stage's tensor-core work.
@@ -436,15 +472,16 @@ __global__ void __launch_bounds__(kThreads, 1)
       uint32_t seq = 0;             // stages of this CTA so far, both producers count all of them
       uint32_t s = 0, ph = 0;       // ring slot and phase of stage `seq`
       bool ok = true;
-      const int cchunks = (p.C + p.bc - 1) / p.bc;
-      for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
+      const int cchunks = p.cchunks_cta;
+      const int c_first = crank * p.cchunks_cta * p.bc;
+      for (int tile = tile_first; ok && tile < p.total_tiles; tile += tile_step) {
         int t = tile / p.tiles_k;
         const int bt = t % p.tiles_b; t /= p.tiles_b;
         const int wt = t % p.tiles_w; t /= p.tiles_w;
         const int ht = t;
         const int b0 = bt * p.bb;
         const int x0 = wt * p.bw * p.sw, y0 = (p.h0 + ht * p.bh) * p.sh;
-        for (int cc = 0, c0 = 0; cc < cchunks; ++cc, c0 += p.bc, ++seq) {
+        for (int cc = 0, c0 = c_first; cc < cchunks; ++cc, c0 += p.bc, ++seq) {
           if ((seq & (i_prod - 1u)) == me) {
             if (!mbar_wait(bar_iempty + 8u * s, ph ^ 1u, abort_flag, status, kStatProducerWait,
                            limit)) {
@@ -480,10 +517,11 @@ __global__ void __launch_bounds__(kThreads, 1)
       // the packed Filter is known to be complete; it waits at its end instead, see below.)
       if (!p.tail) asm volatile("griddepcontrol.wait;" ::: "memory");
       if (me == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-      for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
+      for (int tile = tile_first; ok && tile < p.total_tiles; tile += tile_step) {
         const int kt = tile % p.tiles_k;
-        const uint8_t* src = packed_filter + (size_t)kt * p.units * kPackedBlockBytes;
-        for (int left = p.units; left > 0; left -= p.uf, ++seq) {
+        const uint8_t* src = packed_filter +
+                             ((size_t)kt * p.units + (size_t)crank * p.units_cta) * kPackedBlockBytes;
+        for (int left = p.units_cta; left > 0; left -= p.uf, ++seq) {
           const uint32_t bytes = uint32_t(left < p.uf ? left : p.uf) * kPackedBlockBytes;
           if ((seq & (f_prod - 1u)) == me) {
             if (!mbar_wait(bar_fempty + 8u * s, ph ^ 1u, abort_flag, status, kStatFilterWait,
@@ -508,7 +546,7 @@ __global__ void __launch_bounds__(kThreads, 1)
   } else if (warp == 1) {
     // ===================== MMA issuer =====================
     const MmaCtx cx{bar_ifull, bar_iempty, bar_ffull, bar_fempty, bar_tfull, bar_tempty, bar_drain,
-                    img_ring, filt_ring, tmem_base, abort_flag, status, limit};
+                    img_ring, filt_ring, tmem_base, abort_flag, status, limit, tile_first, tile_step};
     const int taps = p.R * p.S;
     // Straight-line issue code for the common shapes (a loop branch costs a lone warp ~20 cycles):
     // b_h in {1,2} and 1x1 / 3x3 filters; everything else takes the generic loops.
@@ -523,7 +561,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     } else {
       mma_role<0, 0>(p, cx);
     }
-  } else {
+  } else if (p.split == 1) {
     // ===================== epilogue: TMEM -> registers -> Out =====================
     const int q = warp & 3;  // this warp may touch TMEM lanes [32q, 32q+32)
     uint32_t abuf = 0, aph = 0;
@@ -552,26 +590,8 @@ __global__ void __launch_bounds__(kThreads, 1)
             tmem_ld_32x32b_x32(t_base + uint32_t(hh * p.n_mma + ww * p.bb + ch * 32), v);
             tmem_ld_wait();
             if (valid) {
-              // 32 consecutive images of one (k, h, w): 64 B (bf16) or 128 B (fp32), written as
-              // whole 32-byte sectors
               OutT* dst = out + (((long long)k * p.H + h) * p.W + w) * p.B + b0 + ch * 32;
-              if constexpr (sizeof(OutT) == 4) {
-#pragma unroll
-                for (int j = 0; j < 4; ++j)
-                  st_global_v8(dst + 8 * j, v[8 * j], v[8 * j + 1], v[8 * j + 2], v[8 * j + 3],
-                               v[8 * j + 4], v[8 * j + 5], v[8 * j + 6], v[8 * j + 7]);
-              } else {
-#pragma unroll
-                for (int j = 0; j < 2; ++j)
-                  st_global_v8(dst + 16 * j, pack_bf16x2(v[16 * j + 0], v[16 * j + 1]),
-                               pack_bf16x2(v[16 * j + 2], v[16 * j + 3]),
-                               pack_bf16x2(v[16 * j + 4], v[16 * j + 5]),
-                               pack_bf16x2(v[16 * j + 6], v[16 * j + 7]),
-                               pack_bf16x2(v[16 * j + 8], v[16 * j + 9]),
-                               pack_bf16x2(v[16 * j + 10], v[16 * j + 11]),
-                               pack_bf16x2(v[16 * j + 12], v[16 * j + 13]),
-                               pack_bf16x2(v[16 * j + 14], v[16 * j + 15]));
-              }
+              store_run32(dst, v);
             }
           }
         }
@@ -587,6 +607,102 @@ __global__ void __launch_bounds__(kThreads, 1)
       }
     }
     if (threadIdx.x == 64) CCONV_TRACE(10);
+  }
+
+  // ===================== split launch: exchange partial sums, then store =====================
+  // Both CTAs of the cluster hold a full 128 x acc_cols accumulator over their half of the
+  // channels.  Rank r owns the columns [r*half, (r+1)*half): it receives the peer's partial sums
+  // for them in its own shared memory (the rings are idle by then), adds its own and stores.
+  // The partial sums travel as four 16 KB asynchronous shared-memory-to-shared-memory copies per
+  // CTA (one per epilogue warp), credited to the receiver's mbarrier; single remote stores from
+  // 32 lanes to 32 different rows were measured 5x slower.
+  // Every thread of both CTAs reaches both cluster barriers, whatever happened before.
+  if (p.split > 1) {
+    const bool epi = warp >= 2 && warp <= 5;
+    const int q = warp & 3;
+    bool acc_ok = true;
+    if (epi) {
+      acc_ok = mbar_wait_warp(bar_tfull, 0, abort_flag, status, kStatEpilogueWait, limit);
+      acc_ok = __all_sync(0xffffffffu, acc_ok);  // the TMEM loads below need a uniform decision
+      tc_fence_after();
+    }
+    __syncwarp();
+    cluster_sync_all();  // both accumulators complete: neither CTA's rings are read any more
+    if (threadIdx.x == 64) CCONV_TRACE(8);
+    const int half = p.acc_cols >> 1;                 // columns per owner, a multiple of 32
+    const uint32_t row_bytes = uint32_t(half) * 4u;   // one accumulator row of fp32 partial sums
+    const uint32_t t_lane = tmem_base + (uint32_t(q * 32) << 16);
+    // Incoming area: row L = 32q + lane at smem0 + L*row_bytes; outgoing staging area right behind
+    // it, same layout.  16-byte chunk c of a row is stored at chunk c ^ (lane & 7), so that the
+    // eight lanes of a store phase hit eight different bank groups.
+    const uint32_t in_row = smem0 + uint32_t(q * 32 + lane) * row_bytes;
+    const uint32_t out_area = smem0 + 128u * row_bytes;
+    const uint32_t out_row = out_area + uint32_t(q * 32 + lane) * row_bytes;
+    const uint32_t x7 = uint32_t(lane & 7);
+    if (epi && acc_ok) {
+      const int col0 = (crank ^ 1) * half;  // the peer's columns
+      for (int g = 0; g < half; g += 32) {
+        uint32_t v[32];
+        tmem_ld_32x32b_x32(t_lane + uint32_t(col0 + g), v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+          st_shared_v4(out_row + ((uint32_t(g / 4 + c) ^ x7) << 4), v[4 * c], v[4 * c + 1],
+                       v[4 * c + 2], v[4 * c + 3]);
+      }
+      fence_proxy_async_shared();  // the copy engine reads these generic-proxy writes
+      __syncwarp();
+      if (lane == 0) {
+        const uint32_t peer = uint32_t(crank ^ 1);
+        const uint32_t warp_rows = uint32_t(q * 32) * row_bytes;
+        bulk_copy_to_peer(cluster_map_shared(smem0 + warp_rows, peer), out_area + warp_rows,
+                          32u * row_bytes, cluster_map_shared(bar_xchg, peer));
+      }
+    }
+    if (threadIdx.x == 64) CCONV_TRACE(9);
+    if (epi && acc_ok) {
+      acc_ok = mbar_wait_warp(bar_xchg, 0, abort_flag, status, kStatEpilogueWait, limit);
+      acc_ok = __all_sync(0xffffffffu, acc_ok);
+    }
+    if (threadIdx.x == 64) CCONV_TRACE(12);
+    if (epi && acc_ok) {
+      const int tile = tile_first;
+      int t = tile;
+      const int kt = t % p.tiles_k; t /= p.tiles_k;
+      const int bt = t % p.tiles_b; t /= p.tiles_b;
+      const int wt = t % p.tiles_w; t /= p.tiles_w;
+      const int ht = t;
+      const int k = kt * 128 + q * 32 + lane;
+      const int col0 = crank * half;
+      for (int g = 0; g < half; g += 32) {
+        uint32_t v[32];
+        tmem_ld_32x32b_x32(t_lane + uint32_t(col0 + g), v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          uint32_t a0, a1, a2, a3;
+          ld_shared_v4(in_row + ((uint32_t(g / 4 + c) ^ x7) << 4), a0, a1, a2, a3);
+          v[4 * c] = __float_as_uint(__uint_as_float(v[4 * c]) + __uint_as_float(a0));
+          v[4 * c + 1] = __float_as_uint(__uint_as_float(v[4 * c + 1]) + __uint_as_float(a1));
+          v[4 * c + 2] = __float_as_uint(__uint_as_float(v[4 * c + 2]) + __uint_as_float(a2));
+          v[4 * c + 3] = __float_as_uint(__uint_as_float(v[4 * c + 3]) + __uint_as_float(a3));
+        }
+        // column -> (output row, pixel, 32 images)
+        const int col = col0 + g;
+        const int hh = col / p.n_mma, rem = col - hh * p.n_mma;
+        const int ww = rem / p.bb, ch = (rem - ww * p.bb) >> 5;
+        const int h = p.h0 + ht * p.bh + hh, w = wt * p.bw + ww;
+        if (k < p.K && h < p.H && w < p.W) {
+          OutT* dst = out + (((long long)k * p.H + h) * p.W + w) * p.B + bt * p.bb + ch * 32;
+          store_run32(dst, v);
+        }
+      }
+    }
+    if (threadIdx.x == 64) CCONV_TRACE(10);
+    // Neither CTA may leave while a copy still reads its staging area or writes its incoming
+    // area: both have consumed their incoming rows only past this barrier.
+    __syncwarp();
+    cluster_sync_all();
   }
 
   // ===================== teardown =====================
@@ -622,11 +738,19 @@ cudaError_t launch_halo(const CUtensorMap& tm_image, const void* packed_filter, 
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = size_t(smem_bytes);
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  if (p.split > 1) {
+    // the grid is tiles x split CTAs; consecutive CTAs form the cluster that shares a tile
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = unsigned(p.split);
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.numAttrs = 2;
+  }
   if (out_f32)
     return cudaLaunchKernelEx(&cfg, cconv_halo_kernel<float>, tm_image, pf,
                               static_cast<float*>(out), p, status);

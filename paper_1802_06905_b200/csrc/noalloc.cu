@@ -91,7 +91,7 @@ extern "C" int cconv_forward_noalloc(const void* Image, const void* Filter, void
   if (rc != CCONV_OK) return rc;
 
   HaloTile tile;
-  const int no_force[5] = {0, 0, 0, 0, 0};
+  const int no_force[6] = {0, 0, 0, 0, 0, 0};
   if (!choose_halo_tile(d, ds->machine, no_force, &tile)) return CCONV_EUNSUPPORTED;
   if (tile.packed_filter_bytes > (long long)CCONV_NOALLOC_MAX_SCRATCH_BYTES) return CCONV_ETOOLARGE;
 

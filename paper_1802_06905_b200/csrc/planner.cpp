@@ -124,7 +124,7 @@ bool halo_supported(const Dims& d, const char** why) {
   return w == nullptr;
 }
 
-bool choose_halo_tile(const Dims& d, const Machine& m, const int force[5], HaloTile* out) {
+bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloTile* out) {
   if (!halo_supported(d, nullptr)) return false;
   const int reserve = 2048;  // barriers, TMEM slot, 1024-byte alignment slack
   const int cap = m.smem_optin_bytes - reserve;
@@ -151,65 +151,87 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[5], HaloT
         const int N = bb * bw;
         for (int bh = 1; bh <= d.H && N * bh <= m.tmem_cols; ++bh) {
           if (force[1] && bh != force[1]) continue;
-          HaloTile t;
-          t.bb = bb; t.bw = bw; t.bh = bh; t.bc = bc; t.bk = 128;
-          t.halo_w = d.sw * (bw - 1) + d.R;
-          t.halo_h = d.sh * (bh - 1) + d.S;
-          if (t.halo_w > 256 || t.halo_h > 256) continue;  // TMA box extents
-          t.c16 = c16;
-          t.cchunks = (d.C + bc - 1) / bc;
-          t.uf = int(std::min<long long>(units, 9));
-          t.filt_stage_bytes = uint32_t(t.uf) * 4096u;
-          t.f_stages = (t.filt_stage_bytes <= 24576u) ? 3 : 2;
-          const long long img = 1ll * t.halo_w * t.halo_h * bc * bb * 2;
-          if (img > cap) continue;
-          t.img_stage_bytes = uint32_t(img);
-          const long long left = cap - 1ll * t.f_stages * t.filt_stage_bytes;
-          int is = int(std::min<long long>(6, left / img));
-          if (force[3]) {
-            if (is < force[3]) continue;
-            is = force[3];
-          }
-          if (is < 1) continue;
-          t.i_stages = is;  // a single Image stage (huge filters only) runs without overlap
-          const int acc_cols = N * bh;
-          t.acc_bufs = (2 * acc_cols <= m.tmem_cols) ? 2 : 1;
-          int cols = 32;
-          while (cols < acc_cols * t.acc_bufs) cols *= 2;
-          t.tmem_cols = cols;
-          t.tiles_k = (d.K + t.bk - 1) / t.bk;
-          t.tiles_b = d.B / bb;
-          t.tiles_w = (d.W + bw - 1) / bw;
-          t.tiles_h = (d.H + bh - 1) / bh;
-          t.tiles = 1ll * t.tiles_k * t.tiles_b * t.tiles_w * t.tiles_h;
-          if (t.tiles > 0x7fffffffll) continue;
-          t.grid = int(std::min<long long>(t.tiles, m.sm_count));
-          t.packed_filter_bytes = 1ll * t.tiles_k * units * 4096;
-          // at least ~115 KB so that two CTAs never share an SM (each would want the tensor memory)
-          t.smem_bytes = std::max(int(t.i_stages * t.img_stage_bytes +
-                                      t.f_stages * t.filt_stage_bytes) + reserve, 117760);
-          // ---- cycle model (per SM) ------------------------------------------------------
-          const double exec = std::max(N / 2.0, (4096.0 + 32.0 * N) / 128.0);  // math vs operand reads
-          const double unit_clk = std::max(bh * exec, 130.0 + 60.0 * bh);      // issue-rate floor
-          const double cyc_mma = double(units) * unit_clk;
-          const double tile_bytes = double(t.cchunks) * double(img) + double(units) * 4096.0;
-          const double l2_rate = std::min(l2_sm_max_bytes_per_clk, l2_total_bytes_per_clk / t.grid);
-          // 64-byte rows (bb = 32) use the copy engine and the swizzle half as well as 128-byte rows
-          const double cyc_copy = tile_bytes / l2_rate * (bb == 32 ? 1.08 : 1.0);
-          const double cyc_epi = 14.0 * acc_cols;
-          double tile_cyc = (t.acc_bufs == 2) ? std::max({cyc_mma, cyc_copy, cyc_epi})
-                                              : std::max(cyc_mma, cyc_copy) + cyc_epi;
-          if (t.i_stages == 1) tile_cyc = cyc_mma + cyc_copy + cyc_epi;
-          const double waves = std::ceil(double(t.tiles) / t.grid);
-          t.tile_cycles = tile_cyc;
-          t.est_cycles = waves * tile_cyc + cyc_epi + 4000.0;
-          t.words_smem = double(t.tiles) * (double(t.cchunks) * (img / 2) + double(units) * 2048.0) +
-                         double(d.K) * d.H * d.W * d.B;
-          if (!found || t.est_cycles < best.est_cycles * (1 - 1e-9) ||
-              (std::fabs(t.est_cycles - best.est_cycles) <= 1e-9 * best.est_cycles &&
-               t.words_smem < best.words_smem)) {
-            best = t;
-            found = true;
+          // split = 2 (two CTAs per tile, half of the channels each) is built and tested, but the
+          // exchange of partial sums costs more than the shorter main loop saves on every shape
+          // measured so far, so the planner takes it only on request (force[5] == 2).
+          for (int split = 1; split <= 2; ++split) {
+            if (split != (force[5] == 2 ? 2 : 1)) continue;
+            HaloTile t;
+            t.bb = bb; t.bw = bw; t.bh = bh; t.bc = bc; t.bk = 128;
+            t.halo_w = d.sw * (bw - 1) + d.R;
+            t.halo_h = d.sh * (bh - 1) + d.S;
+            if (t.halo_w > 256 || t.halo_h > 256) continue;  // TMA box extents
+            t.c16 = c16;
+            t.cchunks = (d.C + bc - 1) / bc;
+            t.split = split;
+            // halves must be whole Image stages of whole 16-channel chunks, and whole 32-column groups
+            if (split == 2 && (c16 % (2 * (bc / 16)) != 0 || (N * bh / 2) % 32 != 0)) continue;
+            t.uf = int(std::min<long long>(units, 9));
+            t.filt_stage_bytes = uint32_t(t.uf) * 4096u;
+            t.f_stages = (t.filt_stage_bytes <= 24576u) ? 3 : 2;
+            const long long img = 1ll * t.halo_w * t.halo_h * bc * bb * 2;
+            if (img > cap) continue;
+            t.img_stage_bytes = uint32_t(img);
+            const long long left = cap - 1ll * t.f_stages * t.filt_stage_bytes;
+            int is = int(std::min<long long>(6, left / img));
+            if (force[3]) {
+              if (is < force[3]) continue;
+              is = force[3];
+            }
+            if (is < 1) continue;
+            t.i_stages = is;  // a single Image stage (huge filters only) runs without overlap
+            const int acc_cols = N * bh;
+            // a split tile parks the peer's partial sums (128 rows x acc_cols/2 fp32) and stages its
+            // own outgoing ones in the idle rings
+            if (split == 2 &&
+                1ll * is * img + 1ll * t.f_stages * t.filt_stage_bytes < 512ll * acc_cols)
+              continue;
+            t.acc_bufs = (split == 1 && 2 * acc_cols <= m.tmem_cols) ? 2 : 1;
+            int cols = 32;
+            while (cols < acc_cols * t.acc_bufs) cols *= 2;
+            t.tmem_cols = cols;
+            t.tiles_k = (d.K + t.bk - 1) / t.bk;
+            t.tiles_b = d.B / bb;
+            t.tiles_w = (d.W + bw - 1) / bw;
+            t.tiles_h = (d.H + bh - 1) / bh;
+            t.tiles = 1ll * t.tiles_k * t.tiles_b * t.tiles_w * t.tiles_h;
+            if (t.tiles > 0x7fffffffll) continue;
+            if (split == 2 && 2 * t.tiles > m.sm_count) continue;  // split tiles run as one wave
+            t.grid = split == 2 ? int(2 * t.tiles) : int(std::min<long long>(t.tiles, m.sm_count));
+            t.packed_filter_bytes = 1ll * t.tiles_k * units * 4096;
+            // at least ~115 KB so that two CTAs never share an SM (each would want the tensor memory)
+            t.smem_bytes = std::max(int(t.i_stages * t.img_stage_bytes +
+                                        t.f_stages * t.filt_stage_bytes) + reserve, 117760);
+            // ---- cycle model (per SM) ------------------------------------------------------
+            const double exec = std::max(N / 2.0, (4096.0 + 32.0 * N) / 128.0);  // math vs operand reads
+            const double unit_clk = std::max(bh * exec, 130.0 + 60.0 * bh);      // issue-rate floor
+            const double cyc_mma = double(units) / split * unit_clk;
+            const double tile_bytes =
+                (double(t.cchunks) * double(img) + double(units) * 4096.0) / split;
+            const double l2_rate = std::min(l2_sm_max_bytes_per_clk, l2_total_bytes_per_clk / t.grid);
+            // 64-byte rows (bb = 32) use the copy engine and the swizzle half as well as 128-byte rows
+            const double cyc_copy = tile_bytes / l2_rate * (bb == 32 ? 1.08 : 1.0);
+            const double cyc_epi = 14.0 * acc_cols;
+            double tile_cyc = (t.acc_bufs == 2) ? std::max({cyc_mma, cyc_copy, cyc_epi})
+                                                : std::max(cyc_mma, cyc_copy) + cyc_epi;
+            if (t.i_stages == 1) tile_cyc = cyc_mma + cyc_copy + cyc_epi;
+            if (split == 2) {
+              // two cluster barriers, acc_cols/2 columns of fp32 pushed to the peer (about 32 B/clk),
+              // then half an epilogue
+              tile_cyc = (t.i_stages == 1 ? cyc_mma + cyc_copy : std::max(cyc_mma, cyc_copy)) +
+                         1000.0 + 256.0 * acc_cols / 32.0 + 0.5 * cyc_epi + 4.0 * acc_cols;
+            }
+            const double waves = split == 2 ? 1.0 : std::ceil(double(t.tiles) / t.grid);
+            t.tile_cycles = tile_cyc;
+            t.est_cycles = waves * tile_cyc + cyc_epi + 4000.0;
+            t.words_smem = double(t.tiles) * (double(t.cchunks) * (img / 2) + double(units) * 2048.0) +
+                           double(d.K) * d.H * d.W * d.B;
+            if (!found || t.est_cycles < best.est_cycles * (1 - 1e-9) ||
+                (std::fabs(t.est_cycles - best.est_cycles) <= 1e-9 * best.est_cycles &&
+                 t.words_smem < best.words_smem)) {
+              best = t;
+              found = true;
+            }
           }
         }
       }
@@ -226,7 +248,7 @@ bool choose_halo_tail(const Dims& d, const Machine& m, const HaloTile& main, int
   const double frac = waves - std::floor(waves);
   if (frac < 1e-9 || frac > 0.75) return false;  // the last wave is full enough
   const long long per_row = main.tiles / main.tiles_h;
-  const int no_force[5] = {0, 0, 0, 0, 0};
+  const int no_force[6] = {0, 0, 0, 0, 0, 1};  // the tail is never split
   bool found = false;
   double best = main.est_cycles * 0.97;  // must beat the single launch by 3 %
   for (int keep = main.tiles_h - 1; keep >= 1 && keep >= main.tiles_h - 4; --keep) {

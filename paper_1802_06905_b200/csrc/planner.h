@@ -43,6 +43,7 @@ struct HaloTile {
   int f_stages = 0;   // Filter ring depth
   int uf = 0;         // units per Filter stage
   int acc_bufs = 1;   // TMEM accumulator buffers (2 when two fit in 512 columns)
+  int split = 1;      // 2: two CTAs (a cluster) share each tile, half of the channels each
   int tmem_cols = 0;
   int c16 = 0;        // 16-channel chunks: ceil(C/16)
   int cchunks = 0;    // Image stages per tile: ceil(C/bc)
@@ -81,8 +82,9 @@ bool tiling_lp(const Dims& d, double M, bool pooling, double tiles[9], double* G
 bool halo_supported(const Dims& d, const char** why);
 
 // Enumerate legal tiles and keep the one with the least estimated time (ties: fewer staged words).
-// `force` may carry "bw,bh,bc,stages,bb" (0 = free) from the CCONV_FORCE_TILE environment variable.
-bool choose_halo_tile(const Dims& d, const Machine& m, const int force[5], HaloTile* out);
+// `force` may carry "bw,bh,bc,stages,bb,split" (0 = free) from the CCONV_FORCE_TILE environment
+// variable; split: 1 = never split the channels over a CTA pair, 2 = always.
+bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloTile* out);
 
 // Wave quantisation: when the tiles of the best tiling fill the last wave of the persistent grid
 // only partly, the last output rows may be cheaper as a second launch with a smaller tile whose

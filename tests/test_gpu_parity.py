@@ -137,6 +137,21 @@ def test_halo_tail_launch(monkeypatch, out_dtype):
     assert info["tiles"] == 2 * 1 * 4 * 3 and info["tail_tiles"] == 2 * 1 * 2 * 3
 
 
+@pytest.mark.parametrize("out_dtype", DTYPES, ids=DT_IDS)
+@pytest.mark.parametrize("force,c", [
+    ("4,2,16,0,32,2", cs("split_3x3", 32, 64, 160, 8, 5, 3, 3)),        # b_h = 2: one output row per CTA
+    ("8,1,32,0,32,2", cs("split_w", 32, 128, 128, 13, 3, 3, 3)),        # b_h = 1: pixels split; ragged w
+    ("2,2,64,0,64,2", cs("split_1x1", 64, 256, 200, 6, 6, 1, 1)),       # 1x1, K not a multiple of 128
+    ("4,1,16,0,64,2", cs("split_s2", 64, 32, 64, 7, 4, 5, 3, 2, 1)),    # stride 2, 5x3 filter
+], ids=lambda v: v.name if hasattr(v, "name") else None)
+def test_halo_split_channels_over_a_cta_pair(monkeypatch, force, c, out_dtype):
+    """split = 2: a cluster of two CTAs shares each tile, half of the channels each; the partial sums
+    cross through distributed shared memory.  Every output must still be Eq. 1."""
+    monkeypatch.setenv("CCONV_FORCE_TILE", force)
+    info = check_full(c, variant=binding.VARIANT_HALO, out_dtype=out_dtype)
+    assert info["grid"] == 2 * info["tiles"]
+
+
 def test_tail_is_planned_for_the_large_config():
     cfg = synth.CONFIGS[4]
     p = binding.Plan(*cfg.dims(), device=0)
