@@ -185,6 +185,61 @@ def time_config(cfg, torch, binding, dev, steps, warmup, dist=None, sampler=None
     return secs, info, nsets
 
 
+def time_repeats(cfg, torch, binding, dev, launches, repeats=5):
+    """Per-configuration table: median over `repeats` of the CUDA-event time of `launches`
+    back-to-back forward calls, L2-cold (rotating buffer sets larger than L2) and L2-warm (one
+    buffer set).  Returns (cold seconds per call, warm seconds per call, plan info)."""
+    ib, fb = make_inputs(cfg)
+    set_bytes = 2 * (cfg.image_words + cfg.filter_words + cfg.out_words)
+    nsets = max(2, min(64, -(-int(1.5 * L2_BYTES) // set_bytes)))
+    base_i, base_f = to_dev(ib, torch, dev), to_dev(fb, torch, dev)
+    imgs = [base_i] + [base_i.clone() for _ in range(nsets - 1)]
+    flts = [base_f] + [base_f.clone() for _ in range(nsets - 1)]
+    outs = [torch.empty(cfg.out_shape, dtype=torch.bfloat16, device=dev) for _ in range(nsets)]
+    plan = binding.Plan(*cfg.dims(), device=dev.index, out_dtype=binding.OUT_BF16)
+    stream = torch.cuda.current_stream()
+    sp = stream.cuda_stream
+    ptrs = [(imgs[i].data_ptr(), flts[i].data_ptr(), outs[i].data_ptr()) for i in range(nsets)]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    result = []
+    for rotate in (True, False):
+        times = []
+        for rep in range(repeats + 1):            # the first repeat is warm-up
+            torch.cuda.synchronize()
+            e0.record(stream)
+            for i in range(launches):
+                a, b, c = ptrs[i % nsets] if rotate else ptrs[0]
+                plan.forward_ptrs(a, b, c, sp)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            if rep:
+                times.append(e0.elapsed_time(e1) * 1e-3 / launches)
+        result.append(float(np.median(times)))
+    plan.check()
+    info = plan.info()
+    plan.close()
+    return result[0], result[1], info
+
+
+def oracle_sample(cfg, budget_s=2.5):
+    """The CPU oracle on a bounded k-slice of one configuration: (TFLOP/s, cores, seconds, sample)."""
+    from oracle import cnn as ocnn
+    ib, fb = make_inputs(cfg)
+    threads = ocnn.max_threads()
+    k_probe = min(cfg.K, max(1, threads))
+    shp = ocnn.Shape(cfg.B, cfg.C, k_probe, cfg.W, cfg.H, cfg.R, cfg.S, cfg.sw, cfg.sh)
+    t0 = time.perf_counter()
+    ocnn.cnn_bf16(ib, fb[:k_probe], shp)
+    t_probe = time.perf_counter() - t0
+    k_sub = int(min(cfg.K, max(k_probe, k_probe * budget_s // max(t_probe, 1e-9))))
+    shp = ocnn.Shape(cfg.B, cfg.C, k_sub, cfg.W, cfg.H, cfg.R, cfg.S, cfg.sw, cfg.sh)
+    t0 = time.perf_counter()
+    ocnn.cnn_bf16(ib, fb[:k_sub], shp)
+    t = time.perf_counter() - t0
+    return {"tflops": 2.0 * shp.macs / t / 1e12, "cores": threads, "seconds": t,
+            "sample": f"out-channels 0..{k_sub - 1} of {cfg.K}"}
+
+
 def time_e2e(cfg, torch, binding, dev, steps):
     """The same metric through the host-buffer entry point: H2D of Image and Filter from pinned
     memory, the kernel, D2H of Out, every step."""
@@ -413,19 +468,25 @@ def main():
             line["applicable_roofline"]["write_only_stream_gbs"] = wgbs
             rows = []
             for i, c in enumerate(CONFIGS):
-                if i == args.config:
-                    s_i, info_i = secs, info
-                    n_i = steps
-                else:
-                    n_i = 200 if c.flops < 1e11 else 20
-                    s_i, info_i, _ = time_config(c, torch, binding, dev, n_i, 3)
+                # median of 5 repeats of >= 100 back-to-back calls (20 for the 0.3 ms shape)
+                n_i = 100 if c.flops < 1e11 else 20
+                cold, warm, info_i = time_repeats(c, torch, binding, dev, n_i)
                 tr, lbb = applicable_roofline_seconds(c, info_i, peaks)
+                m_cta = binding.lower_bound(*c.dims(), info_i["M_words"])
                 rows.append({"workload": c.name, "variant": info_i["variant"],
-                             "us_per_launch": s_i / n_i * 1e6,
+                             "us_per_launch": cold * 1e6, "us_per_launch_l2_warm": warm * 1e6,
                              "t_write_out_us": 2.0 * c.out_words / (wgbs * 1e9) * 1e6,
-                             "tflops": c.flops * n_i / s_i / 1e12,
-                             "t_roof_us": tr * 1e6, "roofline_frac": tr / (s_i / n_i),
-                             "tile": [info_i[k] for k in ("bb", "bw", "bh", "bc", "stages")]})
+                             "tflops": c.flops / cold / 1e12,
+                             "tflops_vs_sustained_peak": c.flops / cold / 1e12 /
+                                                         peaks["bf16_tflops_sustained"],
+                             "t_roof_us": tr * 1e6, "roofline_frac": tr / cold,
+                             "roofline_frac_l2_warm": tr / warm,
+                             "lower_bound_bytes_at_L2": lbb,
+                             "lower_bound_bytes_at_cta_smem": 2.0 * max(m_cta),
+                             "planned_bytes_into_smem": 2.0 * info_i["tile_words_smem"],
+                             "dram_bytes_ncu": dram_traffic_from_profiles(c.name),
+                             "tile": [info_i[k] for k in ("bb", "bw", "bh", "bc", "stages")],
+                             "oracle": oracle_sample(c)})
             line["all_configs"] = rows
             line["cpu_baseline"] = cpu_baseline(cfg)
     if rank == 0:
