@@ -274,6 +274,8 @@ __device__ __forceinline__ void mma_role(const HaloKernelParams& p, const MmaCtx
         a16 = filt_ring16 + fs * filt16;
         f_left = units_left < uf ? units_left : uf;
       }
+      if (first_tile && units_left == units && lane == 0 && p.trace)
+        p.trace[blockIdx.x * 16 + 5] = globaltimer_ns();  // operands of the first MMA are resident
       // Issue every unit both resident stages cover, with no barrier work in between.
       // Descriptors are built by the whole warp (uniform values); only the issue is elected.
       const int n = i_left < f_left ? i_left : f_left;
