@@ -52,7 +52,8 @@ extern "C" {
 /* Kernel variants (cconv_plan_create's `variant`). */
 #define CCONV_VARIANT_AUTO 0
 #define CCONV_VARIANT_SIMT 1 /* CUDA-core kernel: any shape, any alignment                      */
-#define CCONV_VARIANT_HALO 2 /* TMA halo tiles -> tcgen05.mma -> TMEM; needs B % 32 == 0         */
+#define CCONV_VARIANT_HALO 2 /* TMA halo tiles -> tcgen05.mma -> TMEM; needs B % 8 == 0 (a batch
+                                block of 32 images is zero padded past B when B % 32 != 0)      */
 #define CCONV_VARIANT_STEM 3 /* small C: (s,c) folded into the MMA contraction; needs B % 64 == 0,
                                 K <= 256 and the whole Filter resident in shared memory          */
 
@@ -150,7 +151,7 @@ int cconv_forward_host(cconv_plan* plan, const void* hImage, const void* hFilter
  * Eq. 1 on device buffers for callers that cannot allocate device memory at the time of the call:
  * code running inside a CUDA-graph capture, a serving callback whose memory was handed out at
  * start-up, a process whose allocator may not be entered from this thread.  It runs the same
- * tensor-core kernels as cconv_forward_planned (HALO variant, so B % 32 == 0 is required; other
+ * tensor-core kernels as cconv_forward_planned (HALO variant, so B % 8 == 0 is required; other
  * shapes return CCONV_EUNSUPPORTED), but keeps the repacked Filter and the status word in a fixed
  * array inside the library (CCONV_NOALLOC_MAX_SCRATCH_BYTES + 256 bytes of device memory on every
  * GPU that loads the library, held until the process exits) instead of plan-owned cudaMalloc'd

@@ -367,6 +367,24 @@ __device__ __forceinline__ void mma_role(const HaloKernelParams& p, const MmaCtx
 
 // 32 consecutive images of one (k, h, w): 64 B (bf16) or 128 B (fp32), written as whole 32-byte
 // sectors.
+// The same run cut off after `n` images (n a multiple of 8, as B is), in pieces of 8 images.
+template <typename OutT>
+__device__ __forceinline__ void store_run_partial(OutT* dst, const uint32_t (&v)[32], int n) {
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    if (8 * j < n) {
+      if constexpr (sizeof(OutT) == 4) {
+        st_global_v8(dst + 8 * j, v[8 * j], v[8 * j + 1], v[8 * j + 2], v[8 * j + 3], v[8 * j + 4],
+                     v[8 * j + 5], v[8 * j + 6], v[8 * j + 7]);
+      } else {
+        *reinterpret_cast<uint4*>(dst + 8 * j) =
+            make_uint4(pack_bf16x2(v[8 * j], v[8 * j + 1]), pack_bf16x2(v[8 * j + 2], v[8 * j + 3]),
+                       pack_bf16x2(v[8 * j + 4], v[8 * j + 5]), pack_bf16x2(v[8 * j + 6], v[8 * j + 7]));
+      }
+    }
+  }
+}
+
 template <typename OutT>
 __device__ __forceinline__ void store_run32(OutT* dst, const uint32_t (&v)[32]) {
   if constexpr (sizeof(OutT) == 4) {
@@ -453,6 +471,7 @@ __global__ void __launch_bounds__(kThreads, 1)
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   const uint64_t limit = p.wait_limit_ns;
+  const bool wide_rows = (size_t(p.B) * sizeof(OutT)) % 32 == 0;
   if (threadIdx.x == 0) CCONV_TRACE(1);
   // Persistent launch: CTA i takes tiles i, i + grid, ...  Split launch: the two CTAs of cluster i
   // take tile i once, rank r contracting the r-th half of the channels.
@@ -593,7 +612,10 @@ __global__ void __launch_bounds__(kThreads, 1)
             tmem_ld_wait();
             if (valid) {
               OutT* dst = out + (((long long)k * p.H + h) * p.W + w) * p.B + b0 + ch * 32;
-              store_run32(dst, v);
+              const int nb = p.B - (b0 + ch * 32);  // images left in the batch (block padded past B)
+              // 32-byte stores need rows of Out that are multiples of 32 bytes (bf16: B % 16 == 0)
+              if (nb >= 32 && wide_rows) store_run32(dst, v);
+              else if (nb > 0) store_run_partial(dst, v, nb < 32 ? nb : 32);
             }
           }
         }
@@ -696,7 +718,9 @@ __global__ void __launch_bounds__(kThreads, 1)
         const int h = p.h0 + ht * p.bh + hh, w = wt * p.bw + ww;
         if (k < p.K && h < p.H && w < p.W) {
           OutT* dst = out + (((long long)k * p.H + h) * p.W + w) * p.B + bt * p.bb + ch * 32;
-          store_run32(dst, v);
+          const int nb = p.B - (bt * p.bb + ch * 32);
+          if (nb >= 32 && wide_rows) store_run32(dst, v);
+          else if (nb > 0) store_run_partial(dst, v, nb < 32 ? nb : 32);
         }
       }
     }

@@ -118,8 +118,8 @@ bool tiling_lp(const Dims& d, double M, bool pooling, double tiles[9], double* G
 
 bool halo_supported(const Dims& d, const char** why) {
   const char* w = nullptr;
-  if (d.B % 32 != 0)
-    w = "B must be a multiple of 32 (one swizzled shared-memory row of images)";
+  if (d.B % 8 != 0)
+    w = "B must be a multiple of 8 (the Image's channel stride must be a multiple of 16 bytes for TMA)";
   if (why) *why = w;
   return w == nullptr;
 }
@@ -141,7 +141,9 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloT
   bool found = false;
   HaloTile best;
   for (int bb : {64, 32}) {
-    if (d.B % bb) continue;
+    // a batch block that does not divide B is padded by the TMA's out-of-bounds zero fill; take
+    // such a block only when no exact one exists
+    if (d.B % bb != 0 && !(bb == 32 && d.B % 32 != 0)) continue;
     if (force[4] && bb != force[4]) continue;
     for (int bc : {64, 32, 16}) {
       if (bc > c16 * 16 && bc != 16) continue;
@@ -191,7 +193,7 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloT
             while (cols < acc_cols * t.acc_bufs) cols *= 2;
             t.tmem_cols = cols;
             t.tiles_k = (d.K + t.bk - 1) / t.bk;
-            t.tiles_b = d.B / bb;
+            t.tiles_b = (d.B + bb - 1) / bb;
             t.tiles_w = (d.W + bw - 1) / bw;
             t.tiles_h = (d.H + bh - 1) / bh;
             t.tiles = 1ll * t.tiles_k * t.tiles_b * t.tiles_w * t.tiles_h;

@@ -110,7 +110,7 @@ def test_inspection_plans_are_hardware_legal():
         assert info["lp_words"] == pytest.approx(ob.tiling_lp(*cfg.dims(), info["M_words"])[2], rel=1e-7)
         assert info["compulsory_words"] == cfg.image_words + cfg.filter_words + cfg.out_words
         if info["variant"] == binding.VARIANT_HALO:
-            assert cfg.B % 32 == 0
+            assert cfg.B % 8 == 0
             n = info["bb"] * info["bw"]
             assert n % 16 == 0 and 16 <= n <= 256                      # tcgen05 N rule at M=128
             assert n * info["bh"] <= 512 and info["tmem_cols"] <= 512   # tensor memory
@@ -155,11 +155,18 @@ def test_plan_create_rejects_bad_arguments(lib):
     assert lib.cconv_plan_create(ctypes.byref(h), 2, 8, 8, 4, 4, 3, 3, 1, 1, -1, 0.0, 7, 0) == binding.EINVAL
     assert lib.cconv_plan_create(None, 2, 8, 8, 4, 4, 3, 3, 1, 1, -1, 0.0, 0, 0) == binding.EINVAL
     assert lib.cconv_plan_create(ctypes.byref(h), 2, 8, 8, 4, 4, 3, 3, 1, 1, -1, 0.0, 0, 5) == binding.EINVAL
-    # the tensor-core variant refuses shapes it cannot tile (B not a multiple of 32)
+    # the tensor-core variant refuses shapes it cannot tile (B not a multiple of 8)
     assert lib.cconv_plan_create(ctypes.byref(h), 2, 8, 16, 14, 14, 3, 3, 1, 1, -1, 0.0,
                                  binding.VARIANT_HALO, 0) == binding.EUNSUPPORTED
-    assert lib.cconv_plan_create(ctypes.byref(h), 48, 8, 64, 12, 12, 3, 3, 1, 1, -1, 0.0,
+    assert lib.cconv_plan_create(ctypes.byref(h), 36, 8, 64, 12, 12, 3, 3, 1, 1, -1, 0.0,
                                  binding.VARIANT_HALO, 0) == binding.EUNSUPPORTED
+    # B = 48: a multiple of 8 but not of 32 -> blocks of 32 images, the last one zero padded
+    assert lib.cconv_plan_create(ctypes.byref(h), 48, 8, 64, 12, 12, 3, 3, 1, 1, -1, 0.0,
+                                 binding.VARIANT_HALO, 0) == binding.OK
+    info = binding.PlanInfo()
+    assert lib.cconv_plan_info_get(h, ctypes.byref(info)) == binding.OK
+    assert info.bb == 32 and info.tiles == 1 * 2 * -(-12 // info.bw) * -(-12 // info.bh)
+    lib.cconv_plan_destroy(h)
 
 
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):

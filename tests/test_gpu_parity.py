@@ -162,6 +162,20 @@ def test_tail_is_planned_for_the_large_config():
     assert info["tail_tiles"] <= 148 and info["tiles"] % info["grid"] != 1
 
 
+@pytest.mark.parametrize("out_dtype", DTYPES, ids=DT_IDS)
+@pytest.mark.parametrize("c", [
+    cs("b8", 8, 32, 64, 6, 5, 3, 3),            # a quarter of one batch block
+    cs("b24_1x1", 24, 48, 130, 5, 4, 1, 1),     # 24 of 32 images, K and C ragged too
+    cs("b40_s2", 40, 16, 32, 7, 6, 3, 5, 2, 1),  # one full block + 8 images
+    cs("b72", 72, 64, 128, 4, 9, 3, 3),         # two full blocks + 8 images
+], ids=lambda c: c.name)
+def test_halo_batch_not_a_multiple_of_the_block(c, out_dtype):
+    """B % 8 == 0 but B % 32 != 0: the last batch block is zero padded by the TMA loads and its
+    stores stop at B; nothing beyond Out's end may be touched (guard bands in run_gpu)."""
+    info = check_full(c, variant=binding.VARIANT_HALO, out_dtype=out_dtype)
+    assert info["bb"] == 32 and c.B % 32 != 0
+
+
 def test_halo_matches_simt_kernel_on_device():
     c = cs("cross", 64, 48, 160, 9, 8, 3, 3)
     ib, fb = synth.make_inputs(c)

@@ -81,7 +81,7 @@ def test_noalloc_rejects_what_it_cannot_hold_or_run():
     rc = lib.cconv_forward_noalloc(p, p, p, 32, 1024, 1024, 8, 8, 3, 3, 1, 1, binding.OUT_BF16, None, None)
     assert rc == binding.ETOOLARGE
     assert b"scratch" in lib.cconv_strerror(rc)
-    # B not a multiple of 32: the tensor-core kernel cannot tile it
+    # B not a multiple of 8: the tensor-core kernel cannot tile it
     rc = lib.cconv_forward_noalloc(p, p, p, 2, 8, 16, 14, 14, 3, 3, 1, 1, binding.OUT_BF16, None, None)
     assert rc == binding.EUNSUPPORTED
     rc = lib.cconv_forward_noalloc(None, p, p, 32, 8, 16, 14, 14, 3, 3, 1, 1, binding.OUT_BF16, None, None)
