@@ -176,6 +176,36 @@ def test_halo_batch_not_a_multiple_of_the_block(c, out_dtype):
     assert info["bb"] == 32 and c.B % 32 != 0
 
 
+@pytest.mark.parametrize("variant,c", [
+    (binding.VARIANT_HALO, cs("chain_halo", 64, 64, 256, 20, 18, 3, 3)),     # several tiles per CTA
+    (binding.VARIANT_STEM, cs("chain_stem", 64, 3, 64, 40, 38, 7, 7, 2, 2)),
+], ids=["halo", "stem"])
+def test_back_to_back_calls_with_changing_filters(variant, c):
+    """The Filter packing of call n+1 runs while the convolution of call n is still executing (two
+    scratch buffers, programmatic dependent launch).  Twelve unsynchronised calls that alternate
+    between three Filters and two Images, each into its own Out: every one must be Eq. 1 of ITS
+    inputs.  A packing kernel that overwrote a buffer still being read, or a convolution that
+    started before its packing kernel finished, would show here."""
+    inputs = [synth.make_inputs(c, seed=1000 + i) for i in range(3)]
+    imgs = [to_dev(inputs[i][0]) for i in range(2)]
+    flts = [to_dev(inputs[i][1]) for i in range(3)]
+    exp = {}
+    for i in range(2):
+        for f in range(3):
+            exp[(i, f)] = ocnn.cnn_bf16(inputs[i][0], inputs[f][1], oshape(c))
+    plan = binding.Plan(*c.dims(), device=torch.cuda.current_device(), variant=variant,
+                        out_dtype=binding.OUT_F32)
+    calls = [(n % 2, (n * 2 + n // 3) % 3) for n in range(12)]
+    outs = [torch.full(c.out_shape, float("nan"), dtype=torch.float32, device="cuda") for _ in calls]
+    for (i, f), o in zip(calls, outs):
+        plan.forward(imgs[i], flts[f], o)          # no synchronisation in between
+    plan.check()
+    plan.close()
+    for n, ((i, f), o) in enumerate(zip(calls, outs)):
+        e, ab = exp[(i, f)]
+        assert_close(o.cpu().numpy().astype(np.float64), e, ab, f"call {n} (image {i}, filter {f})")
+
+
 def test_halo_matches_simt_kernel_on_device():
     c = cs("cross", 64, 48, 160, 9, 8, 3, 3)
     ib, fb = synth.make_inputs(c)
