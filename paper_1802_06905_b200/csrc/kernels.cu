@@ -253,23 +253,29 @@ __device__ __forceinline__ void mma_role(const HaloKernelParams& p, const MmaCtx
     uint32_t tap_off = 0, col_off = 0;  // halo offset of the current tap, in 16 B units
     uint32_t a16 = 0, img_kk16 = 0;
     int units_left = units;
+    long long tw_i = 0, tw_f = 0;
+    const long long tl0 = p.trace ? clock64() : 0;
     while (units_left > 0) {
       if (i_left == 0) {
+        const long long w0 = p.trace ? clock64() : 0;
         if (!mbar_wait_warp(cx.bar_ifull + 8u * is, iph, cx.abort_flag, cx.status, kStatMmaWaitFull,
                             cx.limit)) {
           ok = false;
           break;
         }
+        if (p.trace) tw_i += clock64() - w0;
         tc_fence_after();
         img_kk16 = img_ring16 + is * img16;
         i_left = units_left < units_per_img ? units_left : units_per_img;
       }
       if (f_left == 0) {
+        const long long w0 = p.trace ? clock64() : 0;
         if (!mbar_wait_warp(cx.bar_ffull + 8u * fs, fph, cx.abort_flag, cx.status, kStatMmaWaitFull,
                             cx.limit)) {
           ok = false;
           break;
         }
+        if (p.trace) tw_f += clock64() - w0;
         tc_fence_after();
         a16 = filt_ring16 + fs * filt16;
         f_left = units_left < uf ? units_left : uf;
@@ -345,6 +351,11 @@ __device__ __forceinline__ void mma_role(const HaloKernelParams& p, const MmaCtx
       }
     }
     if (!ok) break;
+    if (first_tile && lane == 0 && p.trace) {
+      p.trace[blockIdx.x * 16 + 13] = (unsigned long long)tw_i;
+      p.trace[blockIdx.x * 16 + 14] = (unsigned long long)tw_f;
+      p.trace[blockIdx.x * 16 + 15] = (unsigned long long)(clock64() - tl0);
+    }
     if (leader) umma_commit(cx.bar_tfull + 8u * abuf);  // accumulator complete
     if (first_tile && lane == 0 && p.trace) p.trace[blockIdx.x * 16 + 6] = globaltimer_ns();
     first_tile = false;

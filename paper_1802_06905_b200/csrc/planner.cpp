@@ -129,12 +129,13 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloT
   const int reserve = 2048;  // barriers, TMEM slot, 1024-byte alignment slack
   const int cap = m.smem_optin_bytes - reserve;
   // Cost-model constants, measured on B200 with this kernel (SM cycles):
-  //  * words staged into shared memory are served by L2 at about 30 B/clk per SM when all SMs pull
-  //    (8 TB/s in aggregate), at most ~60 B/clk for one SM -- this, the paper's "words moved into
-  //    fast memory", is what binds the large 3x3 shapes;
+  //  * words staged into shared memory arrive at about 45 B/clk per SM in this kernel, with 98, 112
+  //    or 140 CTAs pulling alike (tile sweeps on the 14x14 shapes; the copy engines alone reach
+  //    about 88 B/clk per SM in a micro-benchmark, so this constant stands for the whole
+  //    producer/consumer pipeline, not for L2) -- it rewards tiles that fill all SMs;
   //  * one elected thread issues a unit (b_h MMAs) in about 130 + 60*b_h cycles at best;
   //  * the epilogue drains an accumulator at about 14 cycles per TMEM column.
-  const double l2_total_bytes_per_clk = 30.0 * m.sm_count, l2_sm_max_bytes_per_clk = 60.0;
+  const double l2_total_bytes_per_clk = 45.0 * m.sm_count, l2_sm_max_bytes_per_clk = 45.0;
   const int RS = d.R * d.S;
   const int c16 = (d.C + 15) / 16;
   const long long units = 1ll * c16 * RS;
@@ -207,7 +208,11 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloT
             // ---- cycle model (per SM) ------------------------------------------------------
             const double exec = std::max(N / 2.0, (4096.0 + 32.0 * N) / 128.0);  // math vs operand reads
             const double unit_clk = std::max(bh * exec, 130.0 + 60.0 * bh);      // issue-rate floor
-            const double cyc_mma = double(units) / split * unit_clk;
+            // every stage of either ring costs the issuing thread a barrier wait and a commit
+            const double stage_clk = 150.0;
+            const double cyc_mma =
+                (double(units) * unit_clk + (double(t.cchunks) + std::ceil(double(units) / t.uf)) * stage_clk) /
+                split;
             const double tile_bytes =
                 (double(t.cchunks) * double(img) + double(units) * 4096.0) / split;
             const double l2_rate = std::min(l2_sm_max_bytes_per_clk, l2_total_bytes_per_clk / t.grid);
@@ -225,7 +230,9 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloT
             }
             const double waves = split == 2 ? 1.0 : std::ceil(double(t.tiles) / t.grid);
             t.tile_cycles = tile_cyc;
-            t.est_cycles = waves * tile_cyc + cyc_epi + 4000.0;
+            // pipeline fill: nothing is issued before the first Image and Filter stages have landed
+            const double fill = (double(img) + double(t.filt_stage_bytes)) / l2_rate;
+            t.est_cycles = waves * tile_cyc + fill + cyc_epi + 4000.0;
             t.words_smem = double(t.tiles) * (double(t.cchunks) * (img / 2) + double(units) * 2048.0) +
                            double(d.K) * d.H * d.W * d.B;
             if (!found || t.est_cycles < best.est_cycles * (1 - 1e-9) ||
