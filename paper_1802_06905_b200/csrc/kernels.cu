@@ -289,18 +289,40 @@ __device__ __forceinline__ void mma_role(const HaloKernelParams& p, const MmaCtx
       if (TAPS == 9 && sx == 0 && tap_r == 0) {
         // whole 16-channel steps of a 3x3 filter, the nine tap offsets held in registers
         for (; issued + 9 <= n; issued += 9) {
+          if constexpr (BH == 1) {
+            umma_taps9_bh1(leader, d_base, a_lo0 | a16, a_hi, b_lo0 | img_kk16, b_hi, idesc, acc, off9);
+          } else if constexpr (BH == 2) {
+            umma_taps9_bh2(leader, d_base, a_lo0 | a16, a_hi, b_lo0 | img_kk16, b_hi, idesc, acc, off9,
+                           hstep16, n_mma);
+          } else {
 #pragma unroll
-          for (int t = 0; t < 9; ++t) {
-            const uint64_t a_desc = (uint64_t(a_hi) << 32) | (a_lo0 | (a16 + uint32_t(t) * kBlk16));
-            issue_unit<BH>(leader, bh, d_base, n_mma, a_desc, b_hi, b_lo0, img_kk16 + off9[t],
-                           hstep16, idesc, acc);
-            acc = 1;
+            for (int t = 0; t < 9; ++t) {
+              const uint64_t a_desc =
+                  (uint64_t(a_hi) << 32) | (a_lo0 | (a16 + uint32_t(t) * kBlk16));
+              issue_unit<BH>(leader, bh, d_base, n_mma, a_desc, b_hi, b_lo0, img_kk16 + off9[t],
+                             hstep16, idesc, acc);
+              acc = 1;
+            }
           }
+          acc = 1;
           a16 += 9u * kBlk16;
           img_kk16 += kstep16;
         }
       } else if (TAPS == 1) {
-        // 1x1 filter: one unit per 16 channels
+        // 1x1 filter: one unit per 16 channels, four at a time while both stages last
+        if constexpr (BH == 1 || BH == 2) {
+          for (; issued + 4 <= n; issued += 4) {
+            if constexpr (BH == 1)
+              umma_run4_bh1(leader, d_base, a_lo0 | a16, a_hi, b_lo0 | img_kk16, b_hi, idesc, acc,
+                            kstep16);
+            else
+              umma_run4_bh2(leader, d_base, a_lo0 | a16, a_hi, b_lo0 | img_kk16, b_hi, idesc, acc,
+                            kstep16, hstep16, n_mma);
+            acc = 1;
+            a16 += 4u * kBlk16;
+            img_kk16 += 4u * kstep16;
+          }
+        }
         for (; issued < n; ++issued) {
           const uint64_t a_desc = (uint64_t(a_hi) << 32) | (a_lo0 | a16);
           issue_unit<BH>(leader, bh, d_base, n_mma, a_desc, b_hi, b_lo0, img_kk16, hstep16, idesc,

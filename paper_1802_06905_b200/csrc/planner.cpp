@@ -146,7 +146,7 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloT
     // such a block only when no exact one exists
     if (d.B % bb != 0 && !(bb == 32 && d.B % 32 != 0)) continue;
     if (force[4] && bb != force[4]) continue;
-    for (int bc : {64, 32, 16}) {
+    for (int bc : {128, 64, 32, 16}) {
       if (bc > c16 * 16 && bc != 16) continue;
       if (force[2] && bc != force[2]) continue;
       for (int bw = 1; bw <= std::min(d.W, 256 / bb); ++bw) {
@@ -169,7 +169,12 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloT
             t.split = split;
             // halves must be whole Image stages of whole 16-channel chunks, and whole 32-column groups
             if (split == 2 && (c16 % (2 * (bc / 16)) != 0 || (N * bh / 2) % 32 != 0)) continue;
-            t.uf = int(std::min<long long>(units, 9));
+            // about nine units per Filter stage, a whole number of Image stages where those are
+            // shorter (1x1 filters), so that stage boundaries of the two rings coincide
+            const int upi = (bc / 16) * RS;
+            int uf = 9;
+            if (upi < 9 && 9 % upi != 0) uf = (9 / upi) * upi;
+            t.uf = int(std::min<long long>(units, uf));
             t.filt_stage_bytes = uint32_t(t.uf) * 4096u;
             t.f_stages = (t.filt_stage_bytes <= 24576u) ? 3 : 2;
             const long long img = 1ll * t.halo_w * t.halo_h * bc * bb * 2;

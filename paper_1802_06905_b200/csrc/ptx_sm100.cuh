@@ -135,6 +135,240 @@ __device__ __forceinline__ void umma_bf16_if(bool issue, uint32_t d_tmem, uint64
       : "memory");
 }
 // Arrives on the mbarrier once every tcgen05.mma issued so far by this thread has completed.
+// ---- straight-line groups of MMAs: two adds per instruction instead of rebuilding both descriptors ----
+// Nine taps of one 16-channel step of a 3x3 filter in one instruction block: Filter blocks
+// a_lo + t*4 KB, Image views b_lo + off[t].  a_lo / b_lo are descriptor low words (address >> 4 already merged
+// with the constant fields); only lane `issue` issues; `accumulate` applies to tap 0, the rest add.
+__device__ __forceinline__ void umma_taps9_bh1(
+    bool issue, uint32_t d, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+    uint32_t idesc, uint32_t accumulate, const uint32_t (&off)[9]) {
+  asm volatile(
+      "{\n\t.reg .pred p, q, pt;\n\t.reg .b64 ad, bd;\n\t.reg .b32 a, b, d2;\n\t"
+      "setp.ne.b32 p, %6, 0;\n\t"
+      "setp.ne.b32 q, %7, 0;\n\t"
+      "setp.eq.b32 pt, %5, %5;\n\t"
+      "mov.b64 ad, {%1, %2};\n\t"
+      "mov.b64 bd, {%3, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %5, p;\n\t"
+      "add.u32 a, %1, 256;\n\t"
+      "add.u32 b, %3, %8;\n\t"
+      "mov.b64 ad, {a, %2};\n\t"
+      "mov.b64 bd, {b, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %5, pt;\n\t"
+      "add.u32 a, %1, 512;\n\t"
+      "add.u32 b, %3, %9;\n\t"
+      "mov.b64 ad, {a, %2};\n\t"
+      "mov.b64 bd, {b, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %5, pt;\n\t"
+      "add.u32 a, %1, 768;\n\t"
+      "add.u32 b, %3, %10;\n\t"
+      "mov.b64 ad, {a, %2};\n\t"
+      "mov.b64 bd, {b, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %5, pt;\n\t"
+      "add.u32 a, %1, 1024;\n\t"
+      "add.u32 b, %3, %11;\n\t"
+      "mov.b64 ad, {a, %2};\n\t"
+      "mov.b64 bd, {b, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %5, pt;\n\t"
+      "add.u32 a, %1, 1280;\n\t"
+      "add.u32 b, %3, %12;\n\t"
+      "mov.b64 ad, {a, %2};\n\t"
+      "mov.b64 bd, {b, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %5, pt;\n\t"
+      "add.u32 a, %1, 1536;\n\t"
+      "add.u32 b, %3, %13;\n\t"
+      "mov.b64 ad, {a, %2};\n\t"
+      "mov.b64 bd, {b, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %5, pt;\n\t"
+      "add.u32 a, %1, 1792;\n\t"
+      "add.u32 b, %3, %14;\n\t"
+      "mov.b64 ad, {a, %2};\n\t"
+      "mov.b64 bd, {b, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %5, pt;\n\t"
+      "add.u32 a, %1, 2048;\n\t"
+      "add.u32 b, %3, %15;\n\t"
+      "mov.b64 ad, {a, %2};\n\t"
+      "mov.b64 bd, {b, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %5, pt;\n\t"
+      "}"
+      ::"r"(d), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate),
+      "r"(uint32_t(issue)), "r"(off[1]), "r"(off[2]), "r"(off[3]), "r"(off[4]), "r"(off[5]), "r"(off[6]),
+      "r"(off[7]), "r"(off[8])
+      : "memory");
+}
+
+// Nine taps of one 16-channel step of a 3x3 filter in one instruction block: Filter blocks
+// a_lo + t*4 KB, Image views b_lo + off[t] and b_lo + off[t] + hstep (second output row, accumulator
+// d + n_mma).  a_lo / b_lo are descriptor low words (address >> 4 already merged
+// with the constant fields); only lane `issue` issues; `accumulate` applies to tap 0, the rest add.
+__device__ __forceinline__ void umma_taps9_bh2(
+    bool issue, uint32_t d, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+    uint32_t idesc, uint32_t accumulate, const uint32_t (&off)[9], uint32_t hstep, uint32_t n_mma) {
+  asm volatile(
+      "{\n\t.reg .pred p, q, pt;\n\t.reg .b64 ad, bd;\n\t.reg .b32 a, b, d2;\n\t"
+      "setp.ne.b32 p, %6, 0;\n\t"
+      "setp.ne.b32 q, %7, 0;\n\t"
+      "setp.eq.b32 pt, %5, %5;\n\t"
+      "add.u32 d2, %0, %17;\n\t"
+      "mov.b64 ad, {%1, %2};\n\t"
+      "mov.b64 bd, {%3, %4};\n\t"
+      "mov.b32 b, %3;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %5, p;\n\t"
+      "add.u32 b, b, %16;\n\t"
+      "mov.b64 bd, {b, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [d2], ad, bd, %5, p;\n\t"
+      "add.u32 a, %1, 256;\n\t"
+      "add.u32 b, %3, %8;\n\t"
+      "mov.b64 ad, {a, %2};\n\t"
+      "mov.b64 bd, {b, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %5, pt;\n\t"
+      "add.u32 b, b, %16;\n\t"
+      "mov.b64 bd, {b, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [d2], ad, bd, %5, pt;\n\t"
+      "add.u32 a, %1, 512;\n\t"
+      "add.u32 b, %3, %9;\n\t"
+      "mov.b64 ad, {a, %2};\n\t"
+      "mov.b64 bd, {b, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %5, pt;\n\t"
+      "add.u32 b, b, %16;\n\t"
+      "mov.b64 bd, {b, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [d2], ad, bd, %5, pt;\n\t"
+      "add.u32 a, %1, 768;\n\t"
+      "add.u32 b, %3, %10;\n\t"
+      "mov.b64 ad, {a, %2};\n\t"
+      "mov.b64 bd, {b, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %5, pt;\n\t"
+      "add.u32 b, b, %16;\n\t"
+      "mov.b64 bd, {b, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [d2], ad, bd, %5, pt;\n\t"
+      "add.u32 a, %1, 1024;\n\t"
+      "add.u32 b, %3, %11;\n\t"
+      "mov.b64 ad, {a, %2};\n\t"
+      "mov.b64 bd, {b, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %5, pt;\n\t"
+      "add.u32 b, b, %16;\n\t"
+      "mov.b64 bd, {b, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [d2], ad, bd, %5, pt;\n\t"
+      "add.u32 a, %1, 1280;\n\t"
+      "add.u32 b, %3, %12;\n\t"
+      "mov.b64 ad, {a, %2};\n\t"
+      "mov.b64 bd, {b, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %5, pt;\n\t"
+      "add.u32 b, b, %16;\n\t"
+      "mov.b64 bd, {b, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [d2], ad, bd, %5, pt;\n\t"
+      "add.u32 a, %1, 1536;\n\t"
+      "add.u32 b, %3, %13;\n\t"
+      "mov.b64 ad, {a, %2};\n\t"
+      "mov.b64 bd, {b, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %5, pt;\n\t"
+      "add.u32 b, b, %16;\n\t"
+      "mov.b64 bd, {b, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [d2], ad, bd, %5, pt;\n\t"
+      "add.u32 a, %1, 1792;\n\t"
+      "add.u32 b, %3, %14;\n\t"
+      "mov.b64 ad, {a, %2};\n\t"
+      "mov.b64 bd, {b, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %5, pt;\n\t"
+      "add.u32 b, b, %16;\n\t"
+      "mov.b64 bd, {b, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [d2], ad, bd, %5, pt;\n\t"
+      "add.u32 a, %1, 2048;\n\t"
+      "add.u32 b, %3, %15;\n\t"
+      "mov.b64 ad, {a, %2};\n\t"
+      "mov.b64 bd, {b, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %5, pt;\n\t"
+      "add.u32 b, b, %16;\n\t"
+      "mov.b64 bd, {b, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [d2], ad, bd, %5, pt;\n\t"
+      "}"
+      ::"r"(d), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate),
+      "r"(uint32_t(issue)), "r"(off[1]), "r"(off[2]), "r"(off[3]), "r"(off[4]), "r"(off[5]), "r"(off[6]),
+      "r"(off[7]), "r"(off[8]), "r"(hstep), "r"(n_mma)
+      : "memory");
+}
+
+// 4 consecutive K=16 steps of a 1x1 filter: Filter blocks a_lo + u*4 KB, Image views b_lo + u*kstep.
+__device__ __forceinline__ void umma_run4_bh1(
+    bool issue, uint32_t d, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+    uint32_t idesc, uint32_t accumulate, uint32_t kstep) {
+  asm volatile(
+      "{\n\t.reg .pred p, q, pt;\n\t.reg .b64 ad, bd;\n\t.reg .b32 a, b, b2, d2;\n\t"
+      "setp.ne.b32 p, %6, 0;\n\t"
+      "setp.ne.b32 q, %7, 0;\n\t"
+      "setp.eq.b32 pt, %5, %5;\n\t"
+      "mov.b32 b, %3;\n\t"
+      "mov.b64 ad, {%1, %2};\n\t"
+      "mov.b64 bd, {b, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %5, p;\n\t"
+      "add.u32 a, %1, 256;\n\t"
+      "add.u32 b, b, %8;\n\t"
+      "mov.b64 ad, {a, %2};\n\t"
+      "mov.b64 bd, {b, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %5, pt;\n\t"
+      "add.u32 a, %1, 512;\n\t"
+      "add.u32 b, b, %8;\n\t"
+      "mov.b64 ad, {a, %2};\n\t"
+      "mov.b64 bd, {b, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %5, pt;\n\t"
+      "add.u32 a, %1, 768;\n\t"
+      "add.u32 b, b, %8;\n\t"
+      "mov.b64 ad, {a, %2};\n\t"
+      "mov.b64 bd, {b, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %5, pt;\n\t"
+      "}"
+      ::"r"(d), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate),
+      "r"(uint32_t(issue)), "r"(kstep)
+      : "memory");
+}
+
+// 4 consecutive K=16 steps of a 1x1 filter: Filter blocks a_lo + u*4 KB, Image views b_lo + u*kstep (and + hstep into d + n_mma).
+__device__ __forceinline__ void umma_run4_bh2(
+    bool issue, uint32_t d, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+    uint32_t idesc, uint32_t accumulate, uint32_t kstep, uint32_t hstep, uint32_t n_mma) {
+  asm volatile(
+      "{\n\t.reg .pred p, q, pt;\n\t.reg .b64 ad, bd;\n\t.reg .b32 a, b, b2, d2;\n\t"
+      "setp.ne.b32 p, %6, 0;\n\t"
+      "setp.ne.b32 q, %7, 0;\n\t"
+      "setp.eq.b32 pt, %5, %5;\n\t"
+      "mov.b32 b, %3;\n\t"
+      "add.u32 d2, %0, %10;\n\t"
+      "mov.b64 ad, {%1, %2};\n\t"
+      "mov.b64 bd, {b, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %5, p;\n\t"
+      "add.u32 b2, b, %9;\n\t"
+      "mov.b64 bd, {b2, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [d2], ad, bd, %5, p;\n\t"
+      "add.u32 a, %1, 256;\n\t"
+      "add.u32 b, b, %8;\n\t"
+      "mov.b64 ad, {a, %2};\n\t"
+      "mov.b64 bd, {b, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %5, pt;\n\t"
+      "add.u32 b2, b, %9;\n\t"
+      "mov.b64 bd, {b2, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [d2], ad, bd, %5, pt;\n\t"
+      "add.u32 a, %1, 512;\n\t"
+      "add.u32 b, b, %8;\n\t"
+      "mov.b64 ad, {a, %2};\n\t"
+      "mov.b64 bd, {b, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %5, pt;\n\t"
+      "add.u32 b2, b, %9;\n\t"
+      "mov.b64 bd, {b2, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [d2], ad, bd, %5, pt;\n\t"
+      "add.u32 a, %1, 768;\n\t"
+      "add.u32 b, b, %8;\n\t"
+      "mov.b64 ad, {a, %2};\n\t"
+      "mov.b64 bd, {b, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %5, pt;\n\t"
+      "add.u32 b2, b, %9;\n\t"
+      "mov.b64 bd, {b2, %4};\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [d2], ad, bd, %5, pt;\n\t"
+      "}"
+      ::"r"(d), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate),
+      "r"(uint32_t(issue)), "r"(kstep), "r"(hstep), "r"(n_mma)
+      : "memory");
+}
+
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
                    bar)
