@@ -176,10 +176,21 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloT
             if (upi < 9 && 9 % upi != 0) uf = (9 / upi) * upi;
             t.uf = int(std::min<long long>(units, uf));
             t.filt_stage_bytes = uint32_t(t.uf) * 4096u;
-            t.f_stages = (t.filt_stage_bytes <= 24576u) ? 3 : 2;
             const long long img = 1ll * t.halo_w * t.halo_h * bc * bb * 2;
             if (img > cap) continue;
             t.img_stage_bytes = uint32_t(img);
+            // Ring depths: shared memory is split between the rings in proportion to the bytes
+            // each must deliver per unit (4 KB of Filter, img/upi of Image), since the bytes a ring
+            // keeps in flight bound its delivery rate; 2..4 Filter stages, and two Image stages
+            // wherever two fit (measured on the 14x14 shapes: 3x3 wants 4 Filter stages, 1x1 two).
+            {
+              const double per_unit_img = double(img) / upi;
+              const double share_f = 4096.0 / (4096.0 + per_unit_img);
+              int fs = int(share_f * cap / t.filt_stage_bytes);
+              fs = std::max(2, std::min(4, fs));
+              while (fs > 2 && (cap - 1ll * fs * t.filt_stage_bytes) / img < 2) --fs;
+              t.f_stages = fs;
+            }
             const long long left = cap - 1ll * t.f_stages * t.filt_stage_bytes;
             int is = int(std::min<long long>(6, left / img));
             if (force[3]) {
