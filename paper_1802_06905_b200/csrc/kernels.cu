@@ -442,7 +442,9 @@ __device__ __forceinline__ void store_run32(OutT* dst, const uint32_t (&v)[32]) 
 // ------------------------------------------------------------------------------------------------
 // Halo-tile tcgen05 kernel
 // ------------------------------------------------------------------------------------------------
-template <typename OutT>
+// BH, TAPS: the issuer's compile-time shape (see mma_role).  One kernel per shape: the issuing loop
+// is sensitive to the size of the code around it, so a launch carries only the loops it runs.
+template <typename OutT, int BH, int TAPS>
 __global__ void __launch_bounds__(kThreads, 1)
     cconv_halo_kernel(const __grid_constant__ CUtensorMap tm_image,
                       const uint8_t* __restrict__ packed_filter, OutT* __restrict__ out,
@@ -601,20 +603,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     // ===================== MMA issuer =====================
     const MmaCtx cx{bar_ifull, bar_iempty, bar_ffull, bar_fempty, bar_tfull, bar_tempty, bar_drain,
                     img_ring, filt_ring, tmem_base, abort_flag, status, limit, tile_first, tile_step};
-    const int taps = p.R * p.S;
-    // Straight-line issue code for the common shapes (a loop branch costs a lone warp ~20 cycles):
-    // b_h in {1,2} and 1x1 / 3x3 filters; everything else takes the generic loops.
-    if (p.R == 3 && p.S == 3) {
-      if (p.bh == 1) mma_role<1, 9>(p, cx);
-      else if (p.bh == 2) mma_role<2, 9>(p, cx);
-      else mma_role<0, 9>(p, cx);
-    } else if (taps == 1) {
-      if (p.bh == 1) mma_role<1, 1>(p, cx);
-      else if (p.bh == 2) mma_role<2, 1>(p, cx);
-      else mma_role<0, 1>(p, cx);
-    } else {
-      mma_role<0, 0>(p, cx);
-    }
+    mma_role<BH, TAPS>(p, cx);
   } else if (p.split == 1) {
     // ===================== epilogue: TMEM -> registers -> Out =====================
     const int q = warp & 3;  // this warp may touch TMEM lanes [32q, 32q+32)
@@ -778,12 +767,42 @@ __global__ void __launch_bounds__(kThreads, 1)
 #undef CCONV_TRACE
 }
 
+namespace {
+
+// Straight-line issue code for the common shapes (a loop branch costs a lone warp ~20 cycles):
+// b_h in {1,2} and 1x1 / 3x3 filters; everything else takes the generic loops.
+template <typename OutT>
+using HaloFn = void (*)(CUtensorMap, const uint8_t*, OutT*, HaloKernelParams, int*);
+
+template <typename OutT>
+HaloFn<OutT> halo_fn(int R, int S, int bh) {
+  const int b = bh == 1 ? 1 : bh == 2 ? 2 : 0;
+  if (R == 3 && S == 3)
+    return b == 1 ? cconv_halo_kernel<OutT, 1, 9> : b == 2 ? cconv_halo_kernel<OutT, 2, 9>
+                                                           : cconv_halo_kernel<OutT, 0, 9>;
+  if (R * S == 1)
+    return b == 1 ? cconv_halo_kernel<OutT, 1, 1> : b == 2 ? cconv_halo_kernel<OutT, 2, 1>
+                                                           : cconv_halo_kernel<OutT, 0, 1>;
+  return cconv_halo_kernel<OutT, 0, 0>;
+}
+
+template <typename OutT>
+cudaError_t prepare_all(int smem_bytes) {
+  const int shapes[7][3] = {{3, 3, 1}, {3, 3, 2}, {3, 3, 3}, {1, 1, 1}, {1, 1, 2}, {1, 1, 3}, {5, 5, 1}};
+  for (const auto& sh : shapes) {
+    cudaError_t e = cudaFuncSetAttribute(halo_fn<OutT>(sh[0], sh[1], sh[2]),
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
+}
+
+}  // namespace
+
 cudaError_t halo_kernel_prepare(int smem_bytes) {
-  cudaError_t e = cudaFuncSetAttribute(cconv_halo_kernel<__nv_bfloat16>,
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+  cudaError_t e = prepare_all<__nv_bfloat16>(smem_bytes);
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(cconv_halo_kernel<float>,
-                              cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+  return prepare_all<float>(smem_bytes);
 }
 
 cudaError_t launch_halo(const CUtensorMap& tm_image, const void* packed_filter, void* out,
@@ -811,9 +830,9 @@ cudaError_t launch_halo(const CUtensorMap& tm_image, const void* packed_filter, 
     cfg.numAttrs = 2;
   }
   if (out_f32)
-    return cudaLaunchKernelEx(&cfg, cconv_halo_kernel<float>, tm_image, pf,
+    return cudaLaunchKernelEx(&cfg, halo_fn<float>(p.R, p.S, p.bh), tm_image, pf,
                               static_cast<float*>(out), p, status);
-  return cudaLaunchKernelEx(&cfg, cconv_halo_kernel<__nv_bfloat16>, tm_image, pf,
+  return cudaLaunchKernelEx(&cfg, halo_fn<__nv_bfloat16>(p.R, p.S, p.bh), tm_image, pf,
                             static_cast<__nv_bfloat16*>(out), p, status);
 }
 
