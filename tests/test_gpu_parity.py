@@ -206,6 +206,39 @@ def test_back_to_back_calls_with_changing_filters(variant, c):
         assert_close(o.cpu().numpy().astype(np.float64), e, ab, f"call {n} (image {i}, filter {f})")
 
 
+def test_random_shapes_tensor_kernels_match_the_cuda_core_kernel():
+    """Forty seeded random shapes (batch multiples of 8, 1x1 to 7x7 filters, strides up to 3, ragged
+    channel counts, tails, batch padding): whatever kernel the planner picks must agree with the
+    CUDA-core kernel to fp32-accumulation noise; every fifth shape is also checked against the
+    oracle with the stated tolerance."""
+    import random
+    rng = random.Random(20260)
+    done = 0
+    it = 0
+    while done < 40:
+        it += 1
+        B = rng.choice([8, 16, 24, 32, 40, 64, 64, 96, 128])
+        R = rng.choice([1, 1, 2, 3, 3, 3, 5, 7])
+        S = rng.choice([1, 3, 3, R, R, 4])
+        C = rng.choice([1, 3, 4, 8, 16, 24, 32, 48, 64, 100, 128, 192, 256])
+        K = rng.choice([8, 16, 40, 64, 100, 128, 160, 256, 300])
+        W, H = rng.randint(1, 17), rng.randint(1, 17)
+        sw, sh = rng.choice([1, 1, 1, 2, 3]), rng.choice([1, 1, 1, 2])
+        c = cs(f"rnd{it}", B, C, K, W, H, R, S, sw, sh)
+        if c.macs > 1.5e9:
+            continue
+        done += 1
+        ib, fb = synth.make_inputs(c, seed=7000 + it)
+        ref, _ = run_gpu(c, ib, fb, binding.VARIANT_SIMT, binding.OUT_F32)
+        got, info = run_gpu(c, ib, fb, binding.VARIANT_AUTO, binding.OUT_F32)
+        assert info["variant"] != binding.VARIANT_SIMT, c
+        scale = np.abs(ref).max() + 1e-30
+        assert np.abs(got - ref).max() <= 2e-5 * scale * np.sqrt(C * R * S), (c, info)
+        if done % 5 == 0:
+            exp, ab = ocnn.cnn_bf16(ib, fb, oshape(c))
+            assert_close(got, exp, ab, f"{c.name} {c.dims()}")
+
+
 def test_halo_matches_simt_kernel_on_device():
     c = cs("cross", 64, 48, 160, 9, 8, 3, 3)
     ib, fb = synth.make_inputs(c)
