@@ -54,8 +54,8 @@ extern "C" {
 #define CCONV_VARIANT_SIMT 1 /* CUDA-core kernel: any shape, any alignment                      */
 #define CCONV_VARIANT_HALO 2 /* TMA halo tiles -> tcgen05.mma -> TMEM; needs B % 8 == 0 (a batch
                                 block of 32 images is zero padded past B when B % 32 != 0)      */
-#define CCONV_VARIANT_STEM 3 /* small C: (s,c) folded into the MMA contraction; needs B % 64 == 0,
-                                K <= 256 and the whole Filter resident in shared memory          */
+#define CCONV_VARIANT_STEM 3 /* small C: (s,c) folded into the MMA contraction; needs B % 8 == 0
+                                and the whole (shifted, padded) Filter resident in shared memory */
 
 /* Element type of Out (cconv_plan_create's `out_dtype`). */
 #define CCONV_OUT_BF16 0

@@ -297,7 +297,9 @@ bool choose_halo_tail(const Dims& d, const Machine& m, const HaloTile& main, int
 }
 
 bool choose_stem_tile(const Dims& d, const Machine& m, StemTile* out) {
-  if (d.B % 64 != 0) return false;
+  // the Image's row stride must be a multiple of 16 bytes for TMA; a block of 64 images is zero
+  // padded past B
+  if (d.B % 8 != 0) return false;
   const int reserve = 2048;
   const int cap = m.smem_optin_bytes - reserve;
   const int shc = d.sh * d.C;
@@ -337,7 +339,7 @@ bool choose_stem_tile(const Dims& d, const Machine& m, StemTile* out) {
   t.tmem_cols = cols;
   t.tiles_w = (d.W + t.bw - 1) / t.bw;
   t.tiles_h = (d.H + t.bhm - 1) / t.bhm;
-  t.tiles_b = d.B / 64;
+  t.tiles_b = (d.B + 63) / 64;
   t.tiles = 1ll * t.tiles_b * t.tiles_h * t.tiles_w * t.tiles_k;
   if (t.tiles > 0x7fffffffll) return false;
   t.grid = int(std::min<long long>(t.tiles, m.sm_count));

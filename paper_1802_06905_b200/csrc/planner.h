@@ -95,7 +95,7 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloT
 bool choose_halo_tail(const Dims& d, const Machine& m, const HaloTile& main, int* main_tiles_h,
                       HaloTile* tail);
 
-// The stem kernel needs B % 64 == 0 and the resident Filter plus two Image windows to fit in shared
+// The stem kernel needs B % 8 == 0 and the resident Filter plus two Image windows to fit in shared
 // memory.
 bool choose_stem_tile(const Dims& d, const Machine& m, StemTile* out);
 

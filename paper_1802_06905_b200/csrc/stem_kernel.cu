@@ -143,6 +143,25 @@ cudaError_t launch_pack_filter_stem(const void* filter, void* packed, const Dims
 // ------------------------------------------------------------------------------------------------
 // The kernel.  Persistent; tile = (128 out-channels) x (64 images) x (bhm output rows) x (bw pixels).
 // ------------------------------------------------------------------------------------------------
+// The same run cut off after `n` images (n a multiple of 8, as B is), in pieces of 8 images: for a
+// batch block padded past B, and for rows of Out that are not multiples of 32 bytes.
+template <typename OutT>
+__device__ __forceinline__ void store_run_partial(OutT* dst, const uint32_t (&v)[32], int n) {
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    if (8 * j < n) {
+      if constexpr (sizeof(OutT) == 4) {
+        st_global_v8(dst + 8 * j, v[8 * j], v[8 * j + 1], v[8 * j + 2], v[8 * j + 3], v[8 * j + 4],
+                     v[8 * j + 5], v[8 * j + 6], v[8 * j + 7]);
+      } else {
+        *reinterpret_cast<uint4*>(dst + 8 * j) =
+            make_uint4(pack_bf16x2(v[8 * j], v[8 * j + 1]), pack_bf16x2(v[8 * j + 2], v[8 * j + 3]),
+                       pack_bf16x2(v[8 * j + 4], v[8 * j + 5]), pack_bf16x2(v[8 * j + 6], v[8 * j + 7]));
+      }
+    }
+  }
+}
+
 template <typename OutT>
 __global__ void __launch_bounds__(kStemThreads, 1)
     cconv_stem_kernel(const __grid_constant__ CUtensorMap tm_image,
@@ -194,6 +213,7 @@ __global__ void __launch_bounds__(kStemThreads, 1)
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   const uint64_t limit = p.wait_limit_ns;
+  const bool wide_rows = (size_t(p.B) * sizeof(OutT)) % 32 == 0;  // 32-byte stores stay aligned
   const int shc = p.sh * p.C;  // Image rows (of the merged (y,c) axis) per output row
 
   if (warp == 0) {
@@ -348,8 +368,14 @@ __global__ void __launch_bounds__(kStemThreads, 1)
         if (tr) t_ld += clock64() - l0;
         if (row_ok && wt * p.bw + px < p.W) {
           OutT* dst = row + (long long)px * p.B;
-          store_run(dst, va);
-          store_run(dst + 32, vb);
+          const int nb = p.B - bt * 64;  // images left in the batch (the block is padded past B)
+          if (nb >= 64 && wide_rows) {
+            store_run(dst, va);
+            store_run(dst + 32, vb);
+          } else {
+            store_run_partial(dst, va, nb < 32 ? nb : 32);
+            if (nb > 32) store_run_partial(dst + 32, vb, nb - 32 < 32 ? nb - 32 : 32);
+          }
         }
       }
       tc_fence_before();

@@ -115,6 +115,8 @@ STEM_SHAPES = [
     cs("st_c2_wide", 64, 2, 24, 33, 3, 2, 9, 2, 1),         # S*C = 18; four stacked rows, H = 3
     cs("st_c3_k200", 64, 3, 200, 6, 5, 3, 3),               # two out-channel tiles
     cs("st_c5_h1", 64, 5, 64, 3, 1, 4, 2, 1, 3),            # one output row, W < bw
+    cs("st_b32", 32, 3, 64, 9, 8, 7, 7, 2, 2),              # half a batch block (zero padded)
+    cs("st_b72", 72, 4, 48, 6, 5, 3, 3),                    # one block + 8 images; 144-byte Out rows
 ]
 
 
