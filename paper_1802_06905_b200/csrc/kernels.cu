@@ -5,10 +5,10 @@
 // cconv_halo_kernel realises the blocked loop nest of Section 5 on one SM:
 //   outer loops  {b,k,w,h}_1 : the persistent tile loop (k innermost so CTAs that run at the same
 //                              time share one Image block in L2),
-//   outer loop   c_1         : the shared-memory ring, one stage per block of b_c channels,
-//   inner loops  {b,k,w,h,c,r,s}_2 : tcgen05.mma instructions.  One stage holds the Image block
-//                              b_b x b_c x (sw(b_w-1)+R) x (sh(b_h-1)+S) -- the halo tile -- and the
-//                              Filter block b_k x R x S x b_c.  Every (r,s) tap reads the SAME
+//   outer loop   c_1         : two shared-memory rings: an Image stage per block of b_c channels
+//                              (the halo tile b_b x b_c x (sw(b_w-1)+R) x (sh(b_h-1)+S)) and a Filter
+//                              stage per group of about nine packed b_k x 16 blocks,
+//   inner loops  {b,k,w,h,c,r,s}_2 : tcgen05.mma instructions.  Every (r,s) tap reads the SAME
 //                              resident halo tile through a shifted shared-memory descriptor, so
 //                              an Image word fetched once serves all R*S taps and all b_k channels
 //                              (the reuse behind the fifth term of Theorem 1).
