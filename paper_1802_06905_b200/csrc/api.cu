@@ -40,6 +40,7 @@ int env_int(const char* name, int dflt) {
 
 struct cconv_plan {
   Dims d{};
+  ImageView view{};  // what the tensor-core kernels run: `d`, or its unstrided 1x1 equivalent
   int device = -1;
   int variant = CCONV_VARIANT_SIMT;
   int out_dtype = CCONV_OUT_BF16;
@@ -137,6 +138,8 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
   cconv_plan* pl = new (std::nothrow) cconv_plan();
   if (!pl) return CCONV_ENOMEM;
   pl->d = d;
+  pl->view = image_view(d);
+  const Dims& dk = pl->view.dk;
   pl->device = device;
   pl->out_dtype = out_dtype;
   if (device >= 0) {
@@ -166,7 +169,7 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
   const int env_variant = env_int("CCONV_VARIANT", 0);
   if (variant == CCONV_VARIANT_AUTO && env_variant >= 1 && env_variant <= 3) variant = env_variant;
 
-  const bool halo_ok = halo_supported(d, nullptr) && choose_halo_tile(d, pl->m, force, &pl->tile);
+  const bool halo_ok = halo_supported(dk, nullptr) && choose_halo_tile(dk, pl->m, force, &pl->tile);
   const bool stem_ok = choose_stem_tile(d, pl->m, &pl->stile);
   if ((variant == CCONV_VARIANT_HALO && !halo_ok) || (variant == CCONV_VARIANT_STEM && !stem_ok)) {
     delete pl;
@@ -183,15 +186,15 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
     const bool forced = force[0] || force[1] || force[2] || force[3] || force[4] || force[5];
     int keep = 0;
     bool tail_ok = !forced && !env_int("CCONV_NO_TAIL", 0) &&
-                   choose_halo_tail(pl->d, pl->m, pl->tile, &keep, &pl->tail);
+                   choose_halo_tail(dk, pl->m, pl->tile, &keep, &pl->tail);
     if (const char* f = std::getenv("CCONV_FORCE_TAIL")) {
       // diagnostics: "rows of tiles kept,bw,bh,bc,stages,bb" for the tail
       int tf[6] = {0, 0, 0, 0, 0, 1};
       tail_ok = false;
       if (std::sscanf(f, "%d,%d,%d,%d,%d,%d", &keep, &tf[0], &tf[1], &tf[2], &tf[3], &tf[4]) >= 1 &&
           keep >= 1 && keep < pl->tile.tiles_h) {
-        Dims dr = pl->d;
-        dr.H = pl->d.H - keep * pl->tile.bh;
+        Dims dr = dk;
+        dr.H = dk.H - keep * pl->tile.bh;
         tail_ok = dr.H > 0 && choose_halo_tile(dr, pl->m, tf, &pl->tail);
       }
     }
@@ -201,11 +204,11 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
       pl->tile.tiles_h = keep;
       pl->tile.tiles = per_row * keep;
       pl->tile.grid = int(std::min<long long>(pl->tile.tiles, pl->m.sm_count));
-      build_halo_params(pl->d, pl->tail, &pl->kp_tail);
+      build_halo_params(dk, pl->tail, &pl->kp_tail);
       pl->kp_tail.h0 = keep * pl->tile.bh;
       pl->kp_tail.tail = 1;
     }
-    build_halo_params(pl->d, pl->tile, &pl->kp);
+    build_halo_params(dk, pl->tile, &pl->kp);
   }
   if (variant == CCONV_VARIANT_STEM) build_stem_params(pl->d, pl->stile, &pl->skp);
 
@@ -354,9 +357,9 @@ int cconv_forward_planned(const cconv_plan* pl, const void* Image, const void* F
     if (pl->tm_image_ptr != Image) {
       int rc = pl->variant == CCONV_VARIANT_STEM
                    ? encode_stem_image_map(pl->d, pl->stile, Image, &pl->tm_image)
-                   : encode_image_map(pl->d, pl->tile, Image, &pl->tm_image);
+                   : encode_image_map(pl->view, pl->tile, Image, &pl->tm_image);
       if (rc == CCONV_OK && pl->has_tail)
-        rc = encode_image_map(pl->d, pl->tail, Image, &pl->tm_image_tail);
+        rc = encode_image_map(pl->view, pl->tail, Image, &pl->tm_image_tail);
       if (rc != CCONV_OK) return rc;
       pl->tm_image_ptr = Image;
     }

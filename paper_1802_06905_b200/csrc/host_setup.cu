@@ -95,7 +95,8 @@ void build_halo_params(const Dims& d, const HaloTile& t, HaloKernelParams* out) 
   p.trace = nullptr;
 }
 
-int encode_image_map(const Dims& d, const HaloTile& t, const void* image, CUtensorMap* tm) {
+int encode_image_map(const ImageView& v, const HaloTile& t, const void* image, CUtensorMap* tm) {
+  const Dims& d = v.dk;
   EncodeTiledFn enc = encode_tiled_fn();
   if (!enc) {
     set_last_cuda_error("cuTensorMapEncodeTiled is not available from this driver");
@@ -105,8 +106,8 @@ int encode_image_map(const Dims& d, const HaloTile& t, const void* image, CUtens
   // A box lands in shared memory as [y][x][c][b]: one slab of b_c x b_b per halo pixel.
   const cuuint64_t dims[4] = {cuuint64_t(d.B), cuuint64_t(d.C), cuuint64_t(d.Wi()),
                               cuuint64_t(d.Hi())};
-  const cuuint64_t strides[3] = {cuuint64_t(d.B) * 2, cuuint64_t(d.Hi()) * d.C * d.B * 2,
-                                 cuuint64_t(d.C) * d.B * 2};
+  const cuuint64_t strides[3] = {cuuint64_t(d.B) * 2, cuuint64_t(v.stride_w) * 2,
+                                 cuuint64_t(v.stride_h) * 2};
   const cuuint32_t box[4] = {cuuint32_t(t.bb), cuuint32_t(t.bc), cuuint32_t(t.halo_w),
                              cuuint32_t(t.halo_h)};
   const cuuint32_t es[4] = {1, 1, 1, 1};

@@ -80,7 +80,9 @@ extern "C" int cconv_forward_noalloc(const void* Image, const void* Filter, void
   if (((reinterpret_cast<uintptr_t>(Image) | reinterpret_cast<uintptr_t>(Filter)) & 15u) ||
       (reinterpret_cast<uintptr_t>(Out) & 31u))
     return CCONV_EINVAL;
-  if (!halo_supported(d, nullptr)) return CCONV_EUNSUPPORTED;
+  const ImageView view = image_view(d);
+  const Dims& dk = view.dk;
+  if (!halo_supported(dk, nullptr)) return CCONV_EUNSUPPORTED;
 
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
@@ -92,13 +94,13 @@ extern "C" int cconv_forward_noalloc(const void* Image, const void* Filter, void
 
   HaloTile tile;
   const int no_force[6] = {0, 0, 0, 0, 0, 0};
-  if (!choose_halo_tile(d, ds->machine, no_force, &tile)) return CCONV_EUNSUPPORTED;
+  if (!choose_halo_tile(dk, ds->machine, no_force, &tile)) return CCONV_EUNSUPPORTED;
   if (tile.packed_filter_bytes > (long long)CCONV_NOALLOC_MAX_SCRATCH_BYTES) return CCONV_ETOOLARGE;
 
   HaloKernelParams kp;
-  build_halo_params(d, tile, &kp);
+  build_halo_params(dk, tile, &kp);
   CUtensorMap tm;
-  rc = encode_image_map(d, tile, Image, &tm);
+  rc = encode_image_map(view, tile, Image, &tm);
   if (rc != CCONV_OK) return rc;
   if (tile.smem_bytes > ds->prepared_smem) {
     e = halo_kernel_prepare(tile.smem_bytes);

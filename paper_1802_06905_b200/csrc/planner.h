@@ -15,6 +15,24 @@ struct Dims {
   }
 };
 
+// How the tensor-core kernels see the Image.  A 1x1 filter with strides touches only every sw-th
+// column and sh-th row, so those kernels run the unstrided problem `dk` on a strided view of the
+// array (same Filter, same Out) and never fetch the skipped pixels.  Strides are in elements,
+// between consecutive view rows (the h direction) and view columns (the w direction).
+struct ImageView {
+  Dims dk;
+  long long stride_h, stride_w;
+};
+inline ImageView image_view(const Dims& d) {
+  ImageView v{d, (long long)d.C * d.B, (long long)d.Hi() * d.C * d.B};
+  if (d.R == 1 && d.S == 1 && (d.sw > 1 || d.sh > 1)) {
+    v.stride_h *= d.sh;
+    v.stride_w *= d.sw;
+    v.dk.sw = v.dk.sh = 1;
+  }
+  return v;
+}
+
 // What the device offers; filled from cudaGetDeviceProperties (or defaults for a B200 when a plan
 // is only inspected on a machine without a GPU).
 struct Machine {

@@ -174,3 +174,16 @@ def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(binding, "_LIB_PATH", str(tmp_path / "nope.so"))
     with pytest.raises(RuntimeError, match="no CPU fallback"):
         binding.load_library()
+
+
+def test_strided_1x1_is_planned_on_a_subsampled_view():
+    """A 1x1 filter with strides skips Image pixels: the tile's halo is the tile itself."""
+    plan = binding.Plan(64, 1024, 2048, 7, 7, 1, 1, 2, 2, device=-1)
+    info = plan.info()
+    plan.close()
+    assert info["variant"] == binding.VARIANT_HALO
+    assert info["halo_w"] == info["bw"] and info["halo_h"] == info["bh"]
+    plan = binding.Plan(64, 64, 128, 7, 7, 3, 3, 2, 2, device=-1)
+    info = plan.info()
+    plan.close()
+    assert info["halo_w"] == 2 * (info["bw"] - 1) + 3

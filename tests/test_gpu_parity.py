@@ -95,6 +95,9 @@ HALO_SHAPES = [
     cs("h_asym", 96, 40, 130, 5, 13, 2, 4, 1, 3),          # B = 3 batch blocks of 32; sh > 1
     cs("h_big_c", 32, 520, 128, 3, 3, 3, 3),               # many channel chunks: ring wraps often
     cs("h_many_tiles", 128, 64, 384, 20, 18, 3, 3),        # more tiles than SMs: persistent loop
+    cs("h_1x1_s2", 64, 48, 136, 9, 7, 1, 1, 2, 2),         # 1x1 with strides: strided Image view
+    cs("h_1x1_s3x1", 32, 32, 64, 6, 11, 1, 1, 3, 1),
+    cs("h_1x1_s1x2", 40, 16, 128, 13, 5, 1, 1, 1, 2),
 ]
 
 
