@@ -124,6 +124,14 @@ bool halo_supported(const Dims& d, const char** why) {
   return w == nullptr;
 }
 
+// Cycles that the compulsory HBM traffic of one call takes: reads at the copy rate (about
+// 3400 B/clk) plus bf16 Out writes at the write-only rate: about 1900 B/clk in 128-byte runs
+// (b_b = 64), about 1400 B/clk in 64-byte runs (b_b = 32; measured on a write-bound 1x1 shape).
+static double hbm_floor_cycles(const Dims& d, int bb) {
+  return 2.0 * (double(d.Wi()) * d.Hi() * d.C * d.B + double(d.K) * d.R * d.S * d.C) / 3400.0 +
+         2.0 * double(d.K) * d.H * d.W * d.B / (bb >= 64 ? 1900.0 : 1400.0);
+}
+
 bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloTile* out) {
   if (!halo_supported(d, nullptr)) return false;
   const int reserve = 2048;  // barriers, TMEM slot, 1024-byte alignment slack
@@ -133,8 +141,12 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloT
   //    or 140 CTAs pulling alike (tile sweeps on the 14x14 shapes; the copy engines alone reach
   //    about 88 B/clk per SM in a micro-benchmark, so this constant stands for the whole
   //    producer/consumer pipeline, not for L2) -- it rewards tiles that fill all SMs;
-  //  * one elected thread issues a unit (b_h MMAs) in about 130 + 60*b_h cycles at best;
-  //  * the epilogue drains an accumulator at about 14 cycles per TMEM column.
+  //  * one elected thread issues a unit (b_h MMAs) in about 130 + 60*b_h cycles at best with the
+  //    straight-line issue blocks (3x3 and 1x1 filters), 170 + 60*b_h with the generic tap loop;
+  //  * the epilogue drains an accumulator at about 14 cycles per TMEM column;
+  //  * HBM: a call cannot end before its compulsory reads (about 3400 B/clk, the copy rate) and its
+  //    Out writes (about 1900 B/clk, the write-only rate) have passed; on write-heavy 1x1 shapes the
+  //    two add up rather than overlap.
   const double l2_total_bytes_per_clk = 45.0 * m.sm_count, l2_sm_max_bytes_per_clk = 45.0;
   const int RS = d.R * d.S;
   const int c16 = (d.C + 15) / 16;
@@ -223,7 +235,8 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloT
                                         t.f_stages * t.filt_stage_bytes) + reserve, 117760);
             // ---- cycle model (per SM) ------------------------------------------------------
             const double exec = std::max(N / 2.0, (4096.0 + 32.0 * N) / 128.0);  // math vs operand reads
-            const double unit_clk = std::max(bh * exec, 130.0 + 60.0 * bh);      // issue-rate floor
+            const double issue0 = (RS == 9 && d.R == 3) || RS == 1 ? 130.0 : 170.0;
+            const double unit_clk = std::max(bh * exec, issue0 + 60.0 * bh);     // issue-rate floor
             // every stage of either ring costs the issuing thread a barrier wait and a commit
             const double stage_clk = 150.0;
             const double cyc_mma =
@@ -244,16 +257,22 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloT
               tile_cyc = (t.i_stages == 1 ? cyc_mma + cyc_copy : std::max(cyc_mma, cyc_copy)) +
                          1000.0 + 256.0 * acc_cols / 32.0 + 0.5 * cyc_epi + 4.0 * acc_cols;
             }
+            tile_cyc += 400.0;  // hand-overs at a tile boundary (accumulator full/empty, ring restart)
             const double waves = split == 2 ? 1.0 : std::ceil(double(t.tiles) / t.grid);
             t.tile_cycles = tile_cyc;
             // pipeline fill: nothing is issued before the first Image and Filter stages have landed
             const double fill = (double(img) + double(t.filt_stage_bytes)) / l2_rate;
-            t.est_cycles = waves * tile_cyc + fill + cyc_epi + 4000.0;
+            t.model_cycles = waves * tile_cyc + fill + cyc_epi + 4000.0;
+            t.est_cycles = std::max(t.model_cycles, hbm_floor_cycles(d, bb) + 4000.0);
             t.words_smem = double(t.tiles) * (double(t.cchunks) * (img / 2) + double(units) * 2048.0) +
                            double(d.K) * d.H * d.W * d.B;
-            if (!found || t.est_cycles < best.est_cycles * (1 - 1e-9) ||
-                (std::fabs(t.est_cycles - best.est_cycles) <= 1e-9 * best.est_cycles &&
-                 t.words_smem < best.words_smem)) {
+            // among tiles that the HBM floor makes equal, the one whose own pipeline is fastest
+            const bool tie = found && std::fabs(t.est_cycles - best.est_cycles) <= 1e-9 * best.est_cycles;
+            const bool tie2 = tie && std::fabs(t.model_cycles - best.model_cycles) <= 1e-9 * best.model_cycles;
+            if (!found || (!tie && t.est_cycles < best.est_cycles) ||
+                (tie && !tie2 && t.model_cycles < best.model_cycles) ||
+                (tie2 && (t.words_smem < best.words_smem ||
+                          (t.words_smem == best.words_smem && t.bh < best.bh)))) {
               best = t;
               found = true;
             }
@@ -285,7 +304,8 @@ bool choose_halo_tail(const Dims& d, const Machine& m, const HaloTile& main, int
     if (t.tiles > m.sm_count) continue;  // the tail is one partial wave
     const double main_cyc = std::ceil(double(per_row * keep) / main.grid) * main.tile_cycles;
     // the tail's CTAs start as SMs fall idle: it costs its own tile time after the main waves
-    const double est = main_cyc + t.tile_cycles + 14.0 * t.bb * t.bw * t.bh + 4000.0;
+    const double est = std::max(main_cyc + t.tile_cycles + 14.0 * t.bb * t.bw * t.bh,
+                                hbm_floor_cycles(d, main.bb)) + 4000.0;
     if (est < best) {
       best = est;
       *main_tiles_h = keep;

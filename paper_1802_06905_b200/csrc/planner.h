@@ -72,6 +72,7 @@ struct HaloTile {
   long long packed_filter_bytes = 0;  // scratch: tiles_k * c16 * R*S blocks of 4 KB
   int smem_bytes = 0;
   double est_cycles = 0;   // cost-model estimate for the whole problem, SM cycles
+  double model_cycles = 0; // the same before the HBM floor is applied
   double tile_cycles = 0;  // cost-model estimate for one tile on one SM
   double words_smem = 0;   // words staged into shared memory over the whole problem + |Out|
 };
