@@ -42,6 +42,16 @@ def theorem1_bound(B, C, K, W, H, R, S, sw, sh, M):
     return max(t), int(np.argmax(t)) + 1
 
 
+def pooling_terms(B, C, K, W, H, R, S, sw, sh, M):
+    """The three expressions whose maximum bounds the words moved by pooling (Section 6):
+    |Out|, |Image| (asymptotic form) and the HBL term of the nest without its Filter."""
+    return [
+        float(B * K * W * H),
+        float(sw * sh * B * C * W * H),
+        float(B * C * K * W * H) * R * S / M,
+    ]
+
+
 def tiling_lp(B, C, K, W, H, R, S, sw, sh, M, pooling=False):
     """Solve the Section-5 LP at the concrete parameters.
 
