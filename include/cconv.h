@@ -172,6 +172,36 @@ int cconv_forward_noalloc(const void* Image, const void* Filter, void* Out, int 
                           int W, int H, int R, int S, int sw, int sh, int out_dtype,
                           void* cuda_stream, int* device_status_out);
 
+/* ---- Pooling (Section 6) ---------------------------------------------------------------------
+ * The loop nest of Eq. 1 without its Filter,
+ *
+ *     for b<B, c<C, k<K, w<W, h<H, r<R, s<S:   Out(k,h,w,b) (+)= Image(r + sw*w, s + sh*h, c, b)
+ *
+ * where a (+) b is a + b/(R*S) with Out starting from 0 (CCONV_POOL_AVG) or max(a, b) with Out
+ * starting from -infinity (CCONV_POOL_MAX).  The nest is taken literally: k does not occur on the
+ * right-hand side, so the reduction runs over the channel c as well as over the window (r,s), and
+ * all K planes of Out receive the same values:
+ *     AVG:  Out(k,h,w,b) = (1/(R*S)) * sum_{c,r,s} Image(...)       MAX:  max_{c,r,s} Image(...)
+ * The usual per-channel pooling layer is the case C = K = 1 with the channels folded into B.
+ * Layouts, element types and alignment are those of the convolution (Image bf16 [Wi][Hi][C][B],
+ * Out [K][H][W][B] bf16 or fp32, overwritten); sums are accumulated in fp32, the maximum is exact.
+ * Any positive bounds are accepted (B % 8 == 0 takes the 16-byte vector path). */
+#define CCONV_POOL_AVG 0
+#define CCONV_POOL_MAX 1
+
+/* The three terms, in words, whose maximum bounds the communication of pooling (Section 6):
+ * BKWH, sw*sh*BCWH, BCKWHRS/M.  Pure host arithmetic; CCONV_EINVAL for non-positive arguments. */
+int cconv_pool_lower_bound(int B, int C, int K, int W, int H, int R, int S, int sw, int sh,
+                           double M_words, double terms_out[3]);
+
+/* Pooling on device buffers of the current device, asynchronous on `cuda_stream`; one kernel, no
+ * scratch memory, no device-side waits (so there is no status word to read).  op: CCONV_POOL_*;
+ * out_dtype: CCONV_OUT_*.  Returns CCONV_EINVAL for null or misaligned pointers, non-positive
+ * bounds or unknown op / out_dtype, CCONV_EUNSUPPORTED when H*W*B exceeds the grid limit
+ * (about 5e11 elements), CCONV_ECUDA when the launch fails. */
+int cconv_pool_forward(const void* Image, void* Out, int B, int C, int K, int W, int H, int R,
+                       int S, int sw, int sh, int op, int out_dtype, void* cuda_stream);
+
 /* Synchronises `cuda_stream`, reads the plan's device status word and clears it.  Returns CCONV_OK,
  * CCONV_EDEVICE_TIMEOUT (and *detail_out = bit mask of the waits that expired) or CCONV_ECUDA. */
 int cconv_plan_status(const cconv_plan* plan, void* cuda_stream, int* detail_out);

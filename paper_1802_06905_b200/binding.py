@@ -19,11 +19,12 @@ EINVAL, EUNSUPPORTED, ECUDA, EDEVICE_TIMEOUT, ENOMEM, ETOOLARGE = -1, -2, -3, -4
 NOALLOC_MAX_SCRATCH_BYTES = 8 * 1024 * 1024
 VARIANT_AUTO, VARIANT_SIMT, VARIANT_HALO, VARIANT_STEM = 0, 1, 2, 3
 OUT_BF16, OUT_F32 = 0, 1
+POOL_AVG, POOL_MAX = 0, 1
 
 EXPORTS = (
     "cconv_lower_bound", "cconv_tiling_lp", "cconv_plan_create", "cconv_plan_info_get",
     "cconv_plan_destroy", "cconv_forward_planned", "cconv_forward", "cconv_forward_host",
-    "cconv_forward_noalloc",
+    "cconv_forward_noalloc", "cconv_pool_lower_bound", "cconv_pool_forward",
     "cconv_plan_status", "cconv_plan_trace_read", "cconv_strerror", "cconv_last_cuda_error", "cconv_version",
 )
 
@@ -99,6 +100,10 @@ def load_library():
     lib.cconv_forward_noalloc.argtypes = [vp, vp, vp] + nine + [i, vp, ctypes.POINTER(i)]
     lib.cconv_forward_host.restype = i
     lib.cconv_forward_host.argtypes = [vp, vp, vp, vp, vp]
+    lib.cconv_pool_lower_bound.restype = i
+    lib.cconv_pool_lower_bound.argtypes = nine + [d, dp]
+    lib.cconv_pool_forward.restype = i
+    lib.cconv_pool_forward.argtypes = [vp, vp] + nine + [i, i, vp]
     lib.cconv_plan_status.restype = i
     lib.cconv_plan_status.argtypes = [vp, vp, ctypes.POINTER(i)]
     lib.cconv_plan_trace_read.restype = i
@@ -122,6 +127,38 @@ def lower_bound(B, C, K, W, H, R, S, sw, sh, M_words):
     _check(load_library().cconv_lower_bound(B, C, K, W, H, R, S, sw, sh, float(M_words), t),
            "cconv_lower_bound")
     return list(t)
+
+
+def pool_lower_bound(B, C, K, W, H, R, S, sw, sh, M_words):
+    """cconv_pool_lower_bound: the three terms of the pooling bound (Section 6)."""
+    t = (ctypes.c_double * 3)()
+    _check(load_library().cconv_pool_lower_bound(B, C, K, W, H, R, S, sw, sh, float(M_words), t),
+           "cconv_pool_lower_bound")
+    return list(t)
+
+
+def pool_forward_ptrs(image_ptr, out_ptr, B, C, K, W, H, R, S, sw, sh, op, out_dtype=0, stream=0):
+    """cconv_pool_forward on raw device addresses (asynchronous on ``stream``)."""
+    _check(load_library().cconv_pool_forward(ctypes.c_void_p(image_ptr), ctypes.c_void_p(out_ptr),
+                                             B, C, K, W, H, R, S, sw, sh, int(op), int(out_dtype),
+                                             ctypes.c_void_p(stream)), "cconv_pool_forward")
+
+
+def pool_forward(image, out, B, C, K, W, H, R, S, sw=1, sh=1, op=0, stream=None):
+    """cconv_pool_forward on torch CUDA tensors: Image bf16 [Wi][Hi][C][B], Out [K][H][W][B] bf16 or
+    fp32 (its dtype selects the output type).  Argument marshalling only."""
+    import torch
+    Wi, Hi = sw * (W - 1) + R, sh * (H - 1) + S
+    if tuple(image.shape) != (Wi, Hi, C, B) or image.dtype != torch.bfloat16:
+        raise ValueError(f"Image must be bf16 {(Wi, Hi, C, B)}")
+    if tuple(out.shape) != (K, H, W, B) or out.dtype not in (torch.bfloat16, torch.float32):
+        raise ValueError(f"Out must be bf16 or fp32 {(K, H, W, B)}")
+    if not (image.is_cuda and out.is_cuda and image.is_contiguous() and out.is_contiguous()):
+        raise ValueError("dense CUDA tensors are required")
+    sp = (stream or torch.cuda.current_stream(image.device)).cuda_stream
+    with torch.cuda.device(image.device):
+        pool_forward_ptrs(image.data_ptr(), out.data_ptr(), B, C, K, W, H, R, S, sw, sh, op,
+                          OUT_F32 if out.dtype == torch.float32 else OUT_BF16, sp)
 
 
 def tiling_lp(B, C, K, W, H, R, S, sw, sh, M_words, pooling=False):

@@ -1,0 +1,214 @@
+// Pooling (Section 6): the loop nest of Eq. 1 without its Filter,
+//
+//     for b,c,k,w,h,r,s:   Out(k,h,w,b) (+)= Image(r + sw*w, s + sh*h, c, b)
+//
+// read literally: k does not occur on the right-hand side, so the reduction runs over (c, r, s) and
+// every k-plane of Out holds the same values.  The kernel therefore reduces once per output pixel
+// and writes the result K times: Image is read once from HBM (window overlaps are served by L1/L2),
+// Out is written once, which is the first two terms of the section's bound; the third term
+// (B*C*K*W*H*R*S/M) never binds here because the reduction is shared by all k.
+//
+// The work is HBM-bound (no contraction, no tensor cores): b is the fastest subscript of both
+// arrays, so a thread owns 8 consecutive images (one 16-byte vector) of one output pixel, a warp
+// reads/writes 512 contiguous bytes per pixel group.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstdint>
+#include <string>
+
+#include "../../include/cconv.h"
+#include "host_setup.h"
+
+namespace cconv {
+namespace {
+
+struct PoolParams {
+  int B, C, K, W, H, R, S, sw, sh;
+  int Hi;
+  int nb;             // vectors per pixel: B / VEC
+  long long total_v;  // H * W * nb output vectors per k-plane
+  int kper;           // k-planes written by one blockIdx.y
+  int terms;          // C * R * S
+  float inv_rs;       // 1 / (R*S)
+};
+
+template <int VEC>
+__device__ __forceinline__ void load_vec(const __nv_bfloat16* p, float (&x)[VEC]) {
+  if constexpr (VEC == 8) {
+    const uint4 q = __ldg(reinterpret_cast<const uint4*>(p));
+    const uint32_t u[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      x[2 * i] = __uint_as_float(u[i] << 16);
+      x[2 * i + 1] = __uint_as_float(u[i] & 0xffff0000u);
+    }
+  } else {
+    x[0] = __bfloat162float(*p);
+  }
+}
+
+template <typename OutT, int VEC>
+__device__ __forceinline__ void store_vec(OutT* p, const float (&x)[VEC]) {
+  if constexpr (VEC == 8 && sizeof(OutT) == 2) {
+    uint32_t u[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const __nv_bfloat162 h2 = __floats2bfloat162_rn(x[2 * i], x[2 * i + 1]);
+      u[i] = *reinterpret_cast<const uint32_t*>(&h2);
+    }
+    __stcs(reinterpret_cast<uint4*>(p), make_uint4(u[0], u[1], u[2], u[3]));
+  } else if constexpr (VEC == 8) {
+    __stcs(reinterpret_cast<float4*>(p), make_float4(x[0], x[1], x[2], x[3]));
+    __stcs(reinterpret_cast<float4*>(p) + 1, make_float4(x[4], x[5], x[6], x[7]));
+  } else if constexpr (sizeof(OutT) == 2) {
+    *reinterpret_cast<__nv_bfloat16*>(p) = __float2bfloat16_rn(x[0]);
+  } else {
+    *reinterpret_cast<float*>(p) = x[0];
+  }
+}
+
+// COOP: a block owns 32 output vectors; its 8 warps split the C*R*S terms of the reduction, combine
+// through shared memory (fixed order: the result does not depend on timing), then split the K
+// planes of the write.  Otherwise (few terms and few planes) a thread does all of it for its own
+// vector and a block owns 256 vectors.
+template <typename OutT, int VEC, bool MAX, bool COOP>
+__global__ void __launch_bounds__(256) cconv_pool_kernel(const __nv_bfloat16* __restrict__ image,
+                                                         OutT* __restrict__ out, PoolParams p) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const long long v = COOP ? (long long)blockIdx.x * 32 + lane
+                           : (long long)blockIdx.x * 256 + threadIdx.x;
+  const bool valid = v < p.total_v;
+  const long long vv = valid ? v : 0;
+  const int bv = int(vv % p.nb);
+  const long long pix = vv / p.nb;
+  const int w = int(pix % p.W), h = int(pix / p.W);
+  const int RS = p.R * p.S;
+  // Image element offset of (x = sw*w, y = sh*h, c = 0, b = bv*VEC)
+  const long long base = (((long long)p.sw * w * p.Hi + (long long)p.sh * h) * p.C) * p.B + (long long)bv * VEC;
+  const long long xstride = (long long)p.Hi * p.C * p.B, ystride = (long long)p.C * p.B;
+
+  float acc[VEC];
+#pragma unroll
+  for (int i = 0; i < VEC; ++i) acc[i] = MAX ? -INFINITY : 0.f;
+  const int t0 = COOP ? warp : 0, tstep = COOP ? 8 : 1;
+  for (int t = t0; t < p.terms; t += tstep) {
+    const int c = t / RS, rs = t - c * RS;
+    const int r = rs / p.S, s = rs - r * p.S;
+    float x[VEC];
+    load_vec<VEC>(image + base + r * xstride + s * ystride + (long long)c * p.B, x);
+#pragma unroll
+    for (int i = 0; i < VEC; ++i) acc[i] = MAX ? fmaxf(acc[i], x[i]) : acc[i] + x[i];
+  }
+
+  if constexpr (COOP) {
+    __shared__ float part[8][32][VEC];
+#pragma unroll
+    for (int i = 0; i < VEC; ++i) part[warp][lane][i] = acc[i];
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < VEC; ++i) acc[i] = part[0][lane][i];
+    for (int j = 1; j < 8; ++j) {
+#pragma unroll
+      for (int i = 0; i < VEC; ++i)
+        acc[i] = MAX ? fmaxf(acc[i], part[j][lane][i]) : acc[i] + part[j][lane][i];
+    }
+  }
+  if (!MAX) {
+#pragma unroll
+    for (int i = 0; i < VEC; ++i) acc[i] *= p.inv_rs;
+  }
+  if (!valid) return;
+  const int k0 = blockIdx.y * p.kper;
+  const int k1 = min(p.K, k0 + p.kper);
+  for (int k = k0 + (COOP ? warp : 0); k < k1; k += COOP ? 8 : 1)
+    store_vec<OutT, VEC>(out + ((long long)k * p.total_v + v) * VEC, acc);
+}
+
+template <typename OutT, int VEC, bool MAX>
+cudaError_t launch_pool_t(const void* image, void* out, const PoolParams& p, bool coop, dim3 grid,
+                          cudaStream_t stream) {
+  const __nv_bfloat16* im = static_cast<const __nv_bfloat16*>(image);
+  OutT* o = static_cast<OutT*>(out);
+  if (coop)
+    cconv_pool_kernel<OutT, VEC, MAX, true><<<grid, 256, 0, stream>>>(im, o, p);
+  else
+    cconv_pool_kernel<OutT, VEC, MAX, false><<<grid, 256, 0, stream>>>(im, o, p);
+  return cudaGetLastError();
+}
+
+}  // namespace
+}  // namespace cconv
+
+using namespace cconv;
+
+extern "C" int cconv_pool_lower_bound(int B, int C, int K, int W, int H, int R, int S, int sw,
+                                      int sh, double M_words, double terms_out[3]) {
+  if (B <= 0 || C <= 0 || K <= 0 || W <= 0 || H <= 0 || R <= 0 || S <= 0 || sw <= 0 || sh <= 0 ||
+      !(M_words > 0) || !terms_out)
+    return CCONV_EINVAL;
+  const double bwh = double(B) * W * H;
+  terms_out[0] = bwh * K;
+  terms_out[1] = bwh * C * sw * sh;
+  terms_out[2] = bwh * C * K * R * S / M_words;
+  return CCONV_OK;
+}
+
+extern "C" int cconv_pool_forward(const void* Image, void* Out, int B, int C, int K, int W, int H,
+                                  int R, int S, int sw, int sh, int op, int out_dtype,
+                                  void* cuda_stream) {
+  if (!Image || !Out) return CCONV_EINVAL;
+  if (B <= 0 || C <= 0 || K <= 0 || W <= 0 || H <= 0 || R <= 0 || S <= 0 || sw <= 0 || sh <= 0)
+    return CCONV_EINVAL;
+  if (op != CCONV_POOL_AVG && op != CCONV_POOL_MAX) return CCONV_EINVAL;
+  if (out_dtype != CCONV_OUT_BF16 && out_dtype != CCONV_OUT_F32) return CCONV_EINVAL;
+  if ((reinterpret_cast<uintptr_t>(Image) & 15u) || (reinterpret_cast<uintptr_t>(Out) & 31u))
+    return CCONV_EINVAL;
+  const double Wi = double(sw) * (W - 1) + R, Hi = double(sh) * (H - 1) + S;
+  if (Wi * Hi * C * B > 9.0e18 || double(K) * H * W * B > 9.0e18 || double(C) * R * S > 2.0e9 ||
+      Hi > 2.0e9)
+    return CCONV_EINVAL;
+
+  PoolParams p;
+  p.B = B; p.C = C; p.K = K; p.W = W; p.H = H; p.R = R; p.S = S; p.sw = sw; p.sh = sh;
+  p.Hi = int(Hi);
+  const int vec = B % 8 == 0 ? 8 : 1;
+  p.nb = B / vec;
+  p.total_v = (long long)H * W * p.nb;
+  p.terms = C * R * S;
+  p.inv_rs = 1.0f / (float(R) * float(S));
+  const bool coop = p.terms + K >= 64;
+  const long long blocks_x = (p.total_v + (coop ? 31 : 255)) / (coop ? 32 : 256);
+  if (blocks_x > 0x7fffffffll) return CCONV_EUNSUPPORTED;
+  // Few pixel groups and many planes: split the planes over blockIdx.y (each slice repeats the
+  // reduction, whose reads hit L2) until the grid fills the machine a few times over.
+  int ksplit = 1;
+  if (coop && blocks_x < 1184) {
+    ksplit = int((1184 + blocks_x - 1) / blocks_x);
+    ksplit = std::max(1, std::min(ksplit, (K + 7) / 8));
+  }
+  p.kper = (K + ksplit - 1) / ksplit;
+  ksplit = (K + p.kper - 1) / p.kper;
+  const dim3 grid{unsigned(blocks_x), unsigned(ksplit), 1u};
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const bool f32 = out_dtype == CCONV_OUT_F32, mx = op == CCONV_POOL_MAX;
+  cudaError_t e;
+  if (vec == 8) {
+    if (f32) e = mx ? launch_pool_t<float, 8, true>(Image, Out, p, coop, grid, stream)
+                    : launch_pool_t<float, 8, false>(Image, Out, p, coop, grid, stream);
+    else e = mx ? launch_pool_t<__nv_bfloat16, 8, true>(Image, Out, p, coop, grid, stream)
+                : launch_pool_t<__nv_bfloat16, 8, false>(Image, Out, p, coop, grid, stream);
+  } else {
+    if (f32) e = mx ? launch_pool_t<float, 1, true>(Image, Out, p, coop, grid, stream)
+                    : launch_pool_t<float, 1, false>(Image, Out, p, coop, grid, stream);
+    else e = mx ? launch_pool_t<__nv_bfloat16, 1, true>(Image, Out, p, coop, grid, stream)
+                : launch_pool_t<__nv_bfloat16, 1, false>(Image, Out, p, coop, grid, stream);
+  }
+  if (e != cudaSuccess) {
+    set_last_cuda_error(std::string("cconv_pool_kernel launch: ") + cudaGetErrorString(e));
+    return CCONV_ECUDA;
+  }
+  return CCONV_OK;
+}

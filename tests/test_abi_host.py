@@ -187,3 +187,15 @@ def test_strided_1x1_is_planned_on_a_subsampled_view():
     info = plan.info()
     plan.close()
     assert info["halo_w"] == 2 * (info["bw"] - 1) + 3
+
+
+def test_pool_lower_bound_matches_the_oracle_terms():
+    for dims in [(64, 64, 256, 27, 27, 3, 3, 2, 2), (8, 3, 5, 6, 5, 3, 2, 1, 3)]:
+        for M in (512.0, 116224.0):
+            got = binding.pool_lower_bound(*dims, M)
+            exp = ob.pooling_terms(*dims, M)
+            assert got == pytest.approx(exp, rel=1e-12)
+    lib = binding.load_library()
+    t = (ctypes.c_double * 3)()
+    assert lib.cconv_pool_lower_bound(0, 1, 1, 1, 1, 1, 1, 1, 1, 4.0, t) == -1
+    assert lib.cconv_pool_lower_bound(1, 1, 1, 1, 1, 1, 1, 1, 1, 0.0, t) == -1
