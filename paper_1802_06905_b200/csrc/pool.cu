@@ -17,6 +17,8 @@
 #include <algorithm>
 #include <cmath>
 #include <cstdint>
+#include <cstdio>
+#include <cstdlib>
 #include <string>
 
 #include "../../include/cconv.h"
@@ -70,51 +72,122 @@ __device__ __forceinline__ void store_vec(OutT* p, const float (&x)[VEC]) {
   }
 }
 
-// COOP: a block owns 32 output vectors; its 8 warps split the C*R*S terms of the reduction, combine
-// through shared memory (fixed order: the result does not depend on timing), then split the K
-// planes of the write.  Otherwise (few terms and few planes) a thread does all of it for its own
-// vector and a block owns 256 vectors.
-template <typename OutT, int VEC, bool MAX, bool COOP>
+// A block of 256 threads owns VPB consecutive output vectors; its G = 256/VPB thread groups split the
+// C*R*S terms of the reduction (thread t: vector t % VPB, group t / VPB), combine through shared
+// memory in a fixed order (the result does not depend on timing), then split the K planes of the
+// write.  VPB = 256 (G = 1): a thread does everything for its own vector (few terms, few planes).
+// Eight loads are kept in flight per thread: the loop is bound by memory latency otherwise.
+template <typename OutT, int VEC, bool MAX, int VPB>
 __global__ void __launch_bounds__(256) cconv_pool_kernel(const __nv_bfloat16* __restrict__ image,
                                                          OutT* __restrict__ out, PoolParams p) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const long long v = COOP ? (long long)blockIdx.x * 32 + lane
-                           : (long long)blockIdx.x * 256 + threadIdx.x;
+  constexpr int G = 256 / VPB;
+  const int vi = threadIdx.x % VPB, g = threadIdx.x / VPB;
+  const long long v = (long long)blockIdx.x * VPB + vi;
   const bool valid = v < p.total_v;
   const long long vv = valid ? v : 0;
-  const int bv = int(vv % p.nb);
-  const long long pix = vv / p.nb;
-  const int w = int(pix % p.W), h = int(pix / p.W);
-  const int RS = p.R * p.S;
+  int bv, w, h;
+  if (p.total_v <= 0x7fffffffll) {  // the usual case: 32-bit divisions
+    const unsigned u = unsigned(vv), pix = u / unsigned(p.nb);
+    bv = int(u - pix * unsigned(p.nb));
+    h = int(pix / unsigned(p.W));
+    w = int(pix - unsigned(h) * unsigned(p.W));
+  } else {
+    bv = int(vv % p.nb);
+    const long long pix = vv / p.nb;
+    w = int(pix % p.W);
+    h = int(pix / p.W);
+  }
   // Image element offset of (x = sw*w, y = sh*h, c = 0, b = bv*VEC)
-  const long long base = (((long long)p.sw * w * p.Hi + (long long)p.sh * h) * p.C) * p.B + (long long)bv * VEC;
+  const __nv_bfloat16* base =
+      image + (((long long)p.sw * w * p.Hi + (long long)p.sh * h) * p.C) * p.B + (long long)bv * VEC;
   const long long xstride = (long long)p.Hi * p.C * p.B, ystride = (long long)p.C * p.B;
+  // Term t = (c*R + r)*S + s, stepped by G = dc*R*S + dr*S + ds with no division or multiplication
+  // in the loop: the pointer moves by a constant, plus a correction whenever s or r wraps.
+  const int RS = p.R * p.S;
+  const int dc = G / RS, dr = (G - dc * RS) / p.S, ds = G - dc * RS - dr * p.S;
+  const int c0 = g / RS;
+  int r = (g - c0 * RS) / p.S, s = g - c0 * RS - r * p.S;
+  const __nv_bfloat16* ptr = base + r * xstride + s * ystride + (long long)c0 * p.B;
+  const long long step = ds * ystride + dr * xstride + (long long)dc * p.B;
+  const long long wrap_s = xstride - p.S * ystride, wrap_r = (long long)p.B - p.R * xstride;
+  auto next_ptr = [&]() {
+    const __nv_bfloat16* cur = ptr;
+    ptr += step;
+    s += ds;
+    if (s >= p.S) { s -= p.S; ptr += wrap_s; ++r; }
+    r += dr;
+    if (r >= p.R) { r -= p.R; ptr += wrap_r; }
+    return cur;
+  };
 
   float acc[VEC];
 #pragma unroll
   for (int i = 0; i < VEC; ++i) acc[i] = MAX ? -INFINITY : 0.f;
-  const int t0 = COOP ? warp : 0, tstep = COOP ? 8 : 1;
-  for (int t = t0; t < p.terms; t += tstep) {
-    const int c = t / RS, rs = t - c * RS;
-    const int r = rs / p.S, s = rs - r * p.S;
-    float x[VEC];
-    load_vec<VEC>(image + base + r * xstride + s * ystride + (long long)c * p.B, x);
+  constexpr int U = 8;  // loads in flight per thread
+  int t = g;
+  if constexpr (MAX && VEC == 8) {
+    // the maximum of bf16 values is taken on the packed pairs themselves (exact), 4 ops per vector
+    const __nv_bfloat162 ninf = __floats2bfloat162_rn(-INFINITY, -INFINITY);
+    __nv_bfloat162 m[4] = {ninf, ninf, ninf, ninf};
+    for (; t + (U - 1) * G < p.terms; t += U * G) {
+      uint4 q[U];
 #pragma unroll
-    for (int i = 0; i < VEC; ++i) acc[i] = MAX ? fmaxf(acc[i], x[i]) : acc[i] + x[i];
+      for (int u = 0; u < U; ++u) q[u] = __ldg(reinterpret_cast<const uint4*>(next_ptr()));
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        m[0] = __hmax2(m[0], *reinterpret_cast<const __nv_bfloat162*>(&q[u].x));
+        m[1] = __hmax2(m[1], *reinterpret_cast<const __nv_bfloat162*>(&q[u].y));
+        m[2] = __hmax2(m[2], *reinterpret_cast<const __nv_bfloat162*>(&q[u].z));
+        m[3] = __hmax2(m[3], *reinterpret_cast<const __nv_bfloat162*>(&q[u].w));
+      }
+    }
+    for (; t < p.terms; t += G) {
+      const uint4 q = __ldg(reinterpret_cast<const uint4*>(next_ptr()));
+      m[0] = __hmax2(m[0], *reinterpret_cast<const __nv_bfloat162*>(&q.x));
+      m[1] = __hmax2(m[1], *reinterpret_cast<const __nv_bfloat162*>(&q.y));
+      m[2] = __hmax2(m[2], *reinterpret_cast<const __nv_bfloat162*>(&q.z));
+      m[3] = __hmax2(m[3], *reinterpret_cast<const __nv_bfloat162*>(&q.w));
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      acc[2 * i] = __low2float(m[i]);
+      acc[2 * i + 1] = __high2float(m[i]);
+    }
+  } else {
+    for (; t + (U - 1) * G < p.terms; t += U * G) {
+      float x[U][VEC];
+#pragma unroll
+      for (int u = 0; u < U; ++u) load_vec<VEC>(next_ptr(), x[u]);
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) acc[i] = MAX ? fmaxf(acc[i], x[u][i]) : acc[i] + x[u][i];
+      }
+    }
+    for (; t < p.terms; t += G) {
+      float x[VEC];
+      load_vec<VEC>(next_ptr(), x);
+#pragma unroll
+      for (int i = 0; i < VEC; ++i) acc[i] = MAX ? fmaxf(acc[i], x[i]) : acc[i] + x[i];
+    }
   }
 
-  if constexpr (COOP) {
-    __shared__ float part[8][32][VEC];
+  if constexpr (G > 1) {
+    // Combine the G partial results of each output element: thread o < VPB*VEC owns element o and
+    // reads part[j][o] for j = 0..G-1 (consecutive threads, consecutive words: no bank conflicts).
+    __shared__ float part[G][VPB * VEC];
+    __shared__ float total[VPB * VEC];
 #pragma unroll
-    for (int i = 0; i < VEC; ++i) part[warp][lane][i] = acc[i];
+    for (int i = 0; i < VEC; ++i) part[g][vi * VEC + i] = acc[i];
+    __syncthreads();
+    for (int o = threadIdx.x; o < VPB * VEC; o += 256) {
+      float a = part[0][o];
+      for (int j = 1; j < G; ++j) a = MAX ? fmaxf(a, part[j][o]) : a + part[j][o];
+      total[o] = a;
+    }
     __syncthreads();
 #pragma unroll
-    for (int i = 0; i < VEC; ++i) acc[i] = part[0][lane][i];
-    for (int j = 1; j < 8; ++j) {
-#pragma unroll
-      for (int i = 0; i < VEC; ++i)
-        acc[i] = MAX ? fmaxf(acc[i], part[j][lane][i]) : acc[i] + part[j][lane][i];
-    }
+    for (int i = 0; i < VEC; ++i) acc[i] = total[vi * VEC + i];
   }
   if (!MAX) {
 #pragma unroll
@@ -123,19 +196,21 @@ __global__ void __launch_bounds__(256) cconv_pool_kernel(const __nv_bfloat16* __
   if (!valid) return;
   const int k0 = blockIdx.y * p.kper;
   const int k1 = min(p.K, k0 + p.kper);
-  for (int k = k0 + (COOP ? warp : 0); k < k1; k += COOP ? 8 : 1)
+  for (int k = k0 + g; k < k1; k += G)
     store_vec<OutT, VEC>(out + ((long long)k * p.total_v + v) * VEC, acc);
 }
 
 template <typename OutT, int VEC, bool MAX>
-cudaError_t launch_pool_t(const void* image, void* out, const PoolParams& p, bool coop, dim3 grid,
+cudaError_t launch_pool_t(const void* image, void* out, const PoolParams& p, int vpb, dim3 grid,
                           cudaStream_t stream) {
   const __nv_bfloat16* im = static_cast<const __nv_bfloat16*>(image);
   OutT* o = static_cast<OutT*>(out);
-  if (coop)
-    cconv_pool_kernel<OutT, VEC, MAX, true><<<grid, 256, 0, stream>>>(im, o, p);
+  if (vpb == 256)
+    cconv_pool_kernel<OutT, VEC, MAX, 256><<<grid, 256, 0, stream>>>(im, o, p);
+  else if (vpb == 32)
+    cconv_pool_kernel<OutT, VEC, MAX, 32><<<grid, 256, 0, stream>>>(im, o, p);
   else
-    cconv_pool_kernel<OutT, VEC, MAX, false><<<grid, 256, 0, stream>>>(im, o, p);
+    cconv_pool_kernel<OutT, VEC, MAX, 8><<<grid, 256, 0, stream>>>(im, o, p);
   return cudaGetLastError();
 }
 
@@ -179,32 +254,45 @@ extern "C" int cconv_pool_forward(const void* Image, void* Out, int B, int C, in
   p.total_v = (long long)H * W * p.nb;
   p.terms = C * R * S;
   p.inv_rs = 1.0f / (float(R) * float(S));
-  const bool coop = p.terms + K >= 64;
-  const long long blocks_x = (p.total_v + (coop ? 31 : 255)) / (coop ? 32 : 256);
+  // Vectors per block: a thread per vector when there is little to share (few terms, few planes);
+  // otherwise 32, or 8 when 32 would leave most SMs without a block and the reduction outweighs
+  // the writes (8 lanes per plane make 128-byte write runs instead of 512-byte ones).
+  int vpb = 256;
+  if (p.terms + K >= 64) vpb = ((p.total_v + 31) / 32 >= 1184 || K >= 4 * p.terms) ? 32 : 8;
+  const long long blocks_x = (p.total_v + vpb - 1) / vpb;
   if (blocks_x > 0x7fffffffll) return CCONV_EUNSUPPORTED;
-  // Few pixel groups and many planes: split the planes over blockIdx.y (each slice repeats the
-  // reduction, whose reads hit L2) until the grid fills the machine a few times over.
+  // Few blocks, and writes that outweigh the reduction: split the planes over blockIdx.y (each
+  // slice repeats the reduction, whose reads hit L2) until the grid fills the machine a few times.
   int ksplit = 1;
-  if (coop && blocks_x < 1184) {
+  if (vpb == 32 && blocks_x < 1184) {
     ksplit = int((1184 + blocks_x - 1) / blocks_x);
-    ksplit = std::max(1, std::min(ksplit, (K + 7) / 8));
+    ksplit = std::max(1, std::min(ksplit, (K + 63) / 64));
   }
+  if (const char* f = std::getenv("CCONV_POOL_FORCE")) {  // diagnostics: "vectors per block,k slices"
+    int fv = 0, fk = 0;
+    if (std::sscanf(f, "%d,%d", &fv, &fk) == 2 && (fv == 8 || fv == 32 || fv == 256) && fk >= 1 &&
+        fk <= 65535 && (p.total_v + fv - 1) / fv <= 0x7fffffffll) {
+      vpb = fv;
+      ksplit = std::min(fk, K);
+    }
+  }
+  const long long blocks = (p.total_v + vpb - 1) / vpb;
   p.kper = (K + ksplit - 1) / ksplit;
   ksplit = (K + p.kper - 1) / p.kper;
-  const dim3 grid{unsigned(blocks_x), unsigned(ksplit), 1u};
+  const dim3 grid{unsigned(blocks), unsigned(ksplit), 1u};
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   const bool f32 = out_dtype == CCONV_OUT_F32, mx = op == CCONV_POOL_MAX;
   cudaError_t e;
   if (vec == 8) {
-    if (f32) e = mx ? launch_pool_t<float, 8, true>(Image, Out, p, coop, grid, stream)
-                    : launch_pool_t<float, 8, false>(Image, Out, p, coop, grid, stream);
-    else e = mx ? launch_pool_t<__nv_bfloat16, 8, true>(Image, Out, p, coop, grid, stream)
-                : launch_pool_t<__nv_bfloat16, 8, false>(Image, Out, p, coop, grid, stream);
+    if (f32) e = mx ? launch_pool_t<float, 8, true>(Image, Out, p, vpb, grid, stream)
+                    : launch_pool_t<float, 8, false>(Image, Out, p, vpb, grid, stream);
+    else e = mx ? launch_pool_t<__nv_bfloat16, 8, true>(Image, Out, p, vpb, grid, stream)
+                : launch_pool_t<__nv_bfloat16, 8, false>(Image, Out, p, vpb, grid, stream);
   } else {
-    if (f32) e = mx ? launch_pool_t<float, 1, true>(Image, Out, p, coop, grid, stream)
-                    : launch_pool_t<float, 1, false>(Image, Out, p, coop, grid, stream);
-    else e = mx ? launch_pool_t<__nv_bfloat16, 1, true>(Image, Out, p, coop, grid, stream)
-                : launch_pool_t<__nv_bfloat16, 1, false>(Image, Out, p, coop, grid, stream);
+    if (f32) e = mx ? launch_pool_t<float, 1, true>(Image, Out, p, vpb, grid, stream)
+                    : launch_pool_t<float, 1, false>(Image, Out, p, vpb, grid, stream);
+    else e = mx ? launch_pool_t<__nv_bfloat16, 1, true>(Image, Out, p, vpb, grid, stream)
+                : launch_pool_t<__nv_bfloat16, 1, false>(Image, Out, p, vpb, grid, stream);
   }
   if (e != cudaSuccess) {
     set_last_cuda_error(std::string("cconv_pool_kernel launch: ") + cudaGetErrorString(e));
