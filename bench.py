@@ -221,6 +221,49 @@ def time_repeats(cfg, torch, binding, dev, launches, repeats=5):
     return result[0], result[1], info
 
 
+def time_pooling(torch, binding, dev, peaks, launches=50, repeats=5):
+    """Pooling (Section 6) rows: median CUDA-event time of back-to-back cconv_pool_forward calls over
+    rotating buffer sets larger than L2.  Algorithmic bytes = Image + Out, each moved once; the
+    roofline is the measured HBM copy rate."""
+    from paper_1802_06905_b200.synth import POOL_SHAPES
+    stream = torch.cuda.current_stream()
+    sp = stream.cuda_stream
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    rows = []
+    gen = torch.Generator(device="cpu").manual_seed(0x18020690 + 60)
+    for name, B, C, K, W, H, R, S, sw, sh in POOL_SHAPES:
+        Wi, Hi = sw * (W - 1) + R, sh * (H - 1) + S
+        ibytes, obytes = 2 * Wi * Hi * C * B, 2 * K * H * W * B
+        nsets = max(2, min(16, -(-int(1.5 * L2_BYTES) // (ibytes + obytes))))
+        base = torch.randn((Wi, Hi, C, B), generator=gen).to(torch.bfloat16).to(dev)
+        imgs = [base] + [base.clone() for _ in range(nsets - 1)]
+        outs = [torch.empty((K, H, W, B), dtype=torch.bfloat16, device=dev) for _ in range(nsets)]
+        terms = binding.pool_lower_bound(B, C, K, W, H, R, S, sw, sh, L2_BYTES / 4.0)
+        for op, opname in ((binding.POOL_AVG, "avg"), (binding.POOL_MAX, "max")):
+            times = []
+            for rep in range(repeats + 1):        # the first repeat is warm-up
+                torch.cuda.synchronize()
+                e0.record(stream)
+                for i in range(launches):
+                    binding.pool_forward_ptrs(imgs[i % nsets].data_ptr(), outs[i % nsets].data_ptr(),
+                                              B, C, K, W, H, R, S, sw, sh, op, binding.OUT_BF16, sp)
+                e1.record(stream)
+                torch.cuda.synchronize()
+                if rep:
+                    times.append(e0.elapsed_time(e1) * 1e-3 / launches)
+            t = float(np.median(times))
+            rows.append({"workload": name, "op": opname,
+                         "dims": dict(zip("B C K W H R S sw sh".split(), (B, C, K, W, H, R, S, sw, sh))),
+                         "us_per_launch": t * 1e6, "algorithmic_bytes": ibytes + obytes,
+                         "gbs": (ibytes + obytes) / t / 1e9,
+                         "roofline": {"bound": "hbm", "achieved": (ibytes + obytes) / t / 1e9,
+                                      "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                      "frac": (ibytes + obytes) / t / 1e9 / peaks["hbm_gbs"]},
+                         "lower_bound_bytes_at_L2": 2.0 * max(terms), "launches": launches})
+        del imgs, outs, base
+    return rows
+
+
 def oracle_sample(cfg, budget_s=2.5):
     """The CPU oracle on a bounded k-slice of one configuration: (TFLOP/s, cores, seconds, sample)."""
     from oracle import cnn as ocnn
@@ -488,6 +531,7 @@ def main():
                              "tile": [info_i[k] for k in ("bb", "bw", "bh", "bc", "stages")],
                              "oracle": oracle_sample(c)})
             line["all_configs"] = rows
+            line["pooling"] = time_pooling(torch, binding, dev, peaks)
             line["cpu_baseline"] = cpu_baseline(cfg)
     if rank == 0:
         print(json.dumps(line))

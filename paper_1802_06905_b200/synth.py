@@ -93,6 +93,16 @@ CONFIGS = (
     ConvShape("cfg5_large_3x3", B=128, C=512, K=512, W=28, H=28, R=3, S=3, seed=SEED_BASE + 5),
 )
 
+# Pooling shapes (Section 6) timed by the benchmark: (name, B, C, K, W, H, R, S, sw, sh).  The first
+# is the usual per-channel layer behind a stem convolution (64 channels folded into b); the second
+# the paper's seven-loop form with a channel reduction and K equal planes; the third writes many
+# planes from a small Image.
+POOL_SHAPES = (
+    ("pool_per_channel_3x3_s2", 4096, 1, 1, 55, 55, 3, 3, 2, 2),
+    ("pool_seven_loop_c64_k256", 64, 64, 256, 27, 27, 3, 3, 2, 2),
+    ("pool_many_planes_2x2_s2", 64, 16, 1024, 28, 28, 2, 2, 2, 2),
+)
+
 
 def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
     """Round float32 to bf16 (nearest, ties to even); returns uint16 bit patterns.  Finite inputs."""
