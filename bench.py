@@ -317,20 +317,36 @@ def kernels_per_step(info, binding):
 
 
 def write_only_gbs(torch, dev):
-    """HBM bandwidth of a write-only stream (device memset over rotating 256 MB buffers): the
-    floor for a kernel whose traffic is dominated by writing Out.  The copy figure in
-    MEASURED_PEAKS.json counts bytes read plus bytes written."""
+    """HBM bandwidth of a write-only stream: cudaMemsetAsync over rotating 256 MB buffers (the CUDA
+    runtime that torch has loaded, called through ctypes; torch's own fill kernel reaches only about
+    two thirds of this rate and is used only if the runtime cannot be reached).  The copy figure
+    in MEASURED_PEAKS.json counts bytes read plus bytes written; a kernel that mostly writes Out is
+    bounded by this figure instead."""
+    import ctypes
     n = 256 * 1024 * 1024
     bufs = [torch.empty(n, dtype=torch.uint8, device=dev) for _ in range(3)]
     for b in bufs:
         b.zero_()
+    stream = torch.cuda.current_stream()
+    memset = None
+    try:
+        rt = ctypes.CDLL("libcudart.so.12")
+        rt.cudaMemsetAsync.restype = ctypes.c_int
+        rt.cudaMemsetAsync.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t, ctypes.c_void_p]
+        if rt.cudaMemsetAsync(bufs[0].data_ptr(), 0, n, stream.cuda_stream) == 0:
+            memset = rt.cudaMemsetAsync
+    except (OSError, AttributeError):
+        memset = None
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
-    e0.record()
+    e0.record(stream)
     reps = 12
     for i in range(reps):
-        bufs[i % 3].zero_()
-    e1.record()
+        if memset is not None:
+            memset(bufs[i % 3].data_ptr(), 0, n, stream.cuda_stream)
+        else:
+            bufs[i % 3].zero_()
+    e1.record(stream)
     torch.cuda.synchronize()
     return n * reps / (e0.elapsed_time(e1) * 1e-3) / 1e9
 

@@ -125,8 +125,9 @@ bool halo_supported(const Dims& d, const char** why) {
 }
 
 // Cycles that the compulsory HBM traffic of one call takes: reads at the copy rate (about
-// 3400 B/clk) plus bf16 Out writes at the write-only rate: about 1900 B/clk in 128-byte runs
-// (b_b = 64), about 1400 B/clk in 64-byte runs (b_b = 32; measured on a write-bound 1x1 shape).
+// 3400 B/clk) plus bf16 Out writes at the rate the epilogue's stores (one 32-byte sector per lane
+// and out-channel plane) are absorbed: about 1900 B/clk in 128-byte runs (b_b = 64), about
+// 1400 B/clk in 64-byte runs (b_b = 32); both measured on write-bound 1x1 shapes.
 static double hbm_floor_cycles(const Dims& d, int bb) {
   return 2.0 * (double(d.Wi()) * d.Hi() * d.C * d.B + double(d.K) * d.R * d.S * d.C) / 3400.0 +
          2.0 * double(d.K) * d.H * d.W * d.B / (bb >= 64 ? 1900.0 : 1400.0);
@@ -145,8 +146,8 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloT
   //    straight-line issue blocks (3x3 and 1x1 filters), 170 + 60*b_h with the generic tap loop;
   //  * the epilogue drains an accumulator at about 14 cycles per TMEM column;
   //  * HBM: a call cannot end before its compulsory reads (about 3400 B/clk, the copy rate) and its
-  //    Out writes (about 1900 B/clk, the write-only rate) have passed; on write-heavy 1x1 shapes the
-  //    two add up rather than overlap.
+  //    Out writes (about 1900 B/clk with this epilogue's stores) have passed; on write-heavy 1x1
+  //    shapes the two add up rather than overlap.
   const double l2_total_bytes_per_clk = 45.0 * m.sm_count, l2_sm_max_bytes_per_clk = 45.0;
   const int RS = d.R * d.S;
   const int c16 = (d.C + 15) / 16;
