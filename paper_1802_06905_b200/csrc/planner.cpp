@@ -249,9 +249,20 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloT
             // 64-byte rows (bb = 32) use the copy engine and the swizzle half as well as 128-byte rows
             const double cyc_copy = tile_bytes / l2_rate * (bb == 32 ? 1.08 : 1.0);
             const double cyc_epi = 14.0 * acc_cols;
-            double tile_cyc = (t.acc_bufs == 2) ? std::max({cyc_mma, cyc_copy, cyc_epi})
-                                                : std::max(cyc_mma, cyc_copy) + cyc_epi;
-            if (t.i_stages == 1) tile_cyc = cyc_mma + cyc_copy + cyc_epi;
+            // every asynchronous copy costs its issuing thread about 700 cycles whatever its
+            // size, and a ring's stages are consumed in order: many small stages starve the MMAs
+            const double cyc_issue_copies =
+                700.0 * std::max(double(t.cchunks), std::ceil(double(units) / t.uf)) / split;
+            double tile_cyc = (t.acc_bufs == 2)
+                                  ? std::max({cyc_mma, cyc_copy, cyc_epi, cyc_issue_copies})
+                                  : std::max({cyc_mma, cyc_copy, cyc_issue_copies}) + cyc_epi;
+            if (t.i_stages == 1) {
+              // one Image stage: the copy of a channel chunk cannot start before the MMAs on the
+              // chunk in front of it are done (Filter copies still run ahead)
+              const double cyc_img = double(t.cchunks) * double(img) / split / l2_rate;
+              tile_cyc = std::max(cyc_mma + cyc_img, cyc_copy) + (t.acc_bufs == 2 ? 0.0 : cyc_epi);
+              if (t.acc_bufs == 2) tile_cyc = std::max(tile_cyc, cyc_epi);
+            }
             if (split == 2) {
               // two cluster barriers, acc_cols/2 columns of fp32 pushed to the peer (about 32 B/clk),
               // then half an epilogue
@@ -305,8 +316,9 @@ bool choose_halo_tail(const Dims& d, const Machine& m, const HaloTile& main, int
     if (t.tiles > m.sm_count) continue;  // the tail is one partial wave
     const double main_cyc = std::ceil(double(per_row * keep) / main.grid) * main.tile_cycles;
     // the tail's CTAs start as SMs fall idle: it costs its own tile time after the main waves
+    // (the second launch has costs of its own -- launch, set-up, first copies -- of about 6000 cycles)
     const double est = std::max(main_cyc + t.tile_cycles + 14.0 * t.bb * t.bw * t.bh,
-                                hbm_floor_cycles(d, main.bb)) + 4000.0;
+                                hbm_floor_cycles(d, main.bb)) + 4000.0 + 6000.0;
     if (est < best) {
       best = est;
       *main_tiles_h = keep;
