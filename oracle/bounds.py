@@ -52,6 +52,32 @@ def pooling_terms(B, C, K, W, H, R, S, sw, sh, M):
     ]
 
 
+def parallel_terms(B, C, K, W, H, R, S, sw, sh, M, aB, aK, aH, aW):
+    """The five terms of the bound for p processors behind one shared memory of M words when the
+    output is cut into aB x aK x aH x aW equal blocks, one per processor (Section 8, "Parallel
+    Algorithm"): p times Theorem 1 on the sub-problem B/aB, K/aK, H/aH, W/aW, which leaves terms
+    1, 4 and 5 as they are, multiplies the Image term by aK and the Filter term by aB*aW*aH."""
+    t = theorem1_terms(B, C, K, W, H, R, S, sw, sh, M)
+    return [t[0], aK * t[1], aB * aW * aH * t[2], t[3], t[4]]
+
+
+def parallel_partition(B, C, K, W, H, R, S, sw, sh, M, p):
+    """Brute force over all (aB, aK, aH, aW) with aX <= X and product <= p.  Reading (the paper only
+    says "choose those values in order to minimize"): use as many processors as the output allows
+    (largest product first), then the smallest bound, then the least replicated traffic (terms 2+3),
+    then the lexicographically smallest tuple.  Returns ((aB, aK, aH, aW), bound)."""
+    best = None
+    for aB in range(1, min(B, p) + 1):
+        for aK in range(1, min(K, p // aB) + 1):
+            for aH in range(1, min(H, p // (aB * aK)) + 1):
+                for aW in range(1, min(W, p // (aB * aK * aH)) + 1):
+                    t = parallel_terms(B, C, K, W, H, R, S, sw, sh, M, aB, aK, aH, aW)
+                    key = (-(aB * aK * aH * aW), max(t), t[1] + t[2], (aB, aK, aH, aW))
+                    if best is None or key < best:
+                        best = key
+    return best[3], best[1]
+
+
 def tiling_lp(B, C, K, W, H, R, S, sw, sh, M, pooling=False):
     """Solve the Section-5 LP at the concrete parameters.
 

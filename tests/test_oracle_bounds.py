@@ -174,3 +174,45 @@ def test_pooling_lp_drops_filter_constraint():
     g_conv = ob.tiling_lp(*d.dims(), M)[1]
     g_pool = ob.tiling_lp(*d.dims(), M, pooling=True)[1]
     assert g_pool >= g_conv * (1 - 1e-9)
+
+
+# ---- parallel sketch (Section 8): p processors, output cut into aB x aK x aH x aW blocks ----------
+
+def test_parallel_terms_are_p_times_theorem1_on_the_subproblem():
+    # the definition the section starts from: p * (Theorem 1 with B, K, H, W divided by the a's)
+    dims = (32, 24, 48, 12, 8, 3, 3, 2, 1)
+    B, C, K, W, H, R, S, sw, sh = dims
+    M = 4096.0
+    for (aB, aK, aH, aW) in [(1, 1, 1, 1), (2, 1, 1, 1), (1, 4, 1, 1), (2, 2, 2, 3), (4, 3, 4, 2)]:
+        p = aB * aK * aH * aW
+        sub = ob.theorem1_terms(B // aB, C, K // aK, W // aW, H // aH, R, S, sw, sh, M)
+        got = ob.parallel_terms(*dims, M, aB, aK, aH, aW)
+        np.testing.assert_allclose(got, [p * x for x in sub], rtol=1e-12)
+    # one processor: Theorem 1 itself
+    assert ob.parallel_terms(*dims, M, 1, 1, 1, 1) == ob.theorem1_terms(*dims, M)
+
+
+def test_parallel_partition_prefers_the_cut_that_replicates_the_smaller_array():
+    M = 116224.0
+    # large 3x3 shape (B128 C512 K512 28x28): Filter is 2.4 M words, Image 51 M: cutting the batch
+    # in 8 replicates only the Filter (8 * 2.4 M < |Out|), so the bound does not move
+    dims = (128, 512, 512, 28, 28, 3, 3, 1, 1)
+    one = max(ob.theorem1_terms(*dims, M))
+    (aB, aK, aH, aW), bound = ob.parallel_partition(*dims, M, 8)
+    assert aK == 1 and aB * aH * aW == 8
+    assert bound == pytest.approx(one)
+    # cutting the out-channels instead multiplies the Image term: strictly worse once it passes the max
+    t_k = ob.parallel_terms(*dims, M, 1, 8, 1, 1)
+    assert t_k[1] == pytest.approx(8 * 128 * 512 * 28 * 28) and max(t_k) > bound
+    # a huge Filter and a single small image: now the out-channels are what to cut
+    dims2 = (1, 64, 4096, 2, 2, 7, 7, 1, 1)
+    (aB, aK, aH, aW), _ = ob.parallel_partition(*dims2, 1024.0, 4)
+    assert (aB, aK, aH, aW) == (1, 4, 1, 1)
+
+
+def test_parallel_partition_uses_all_processors_the_output_allows():
+    dims = (2, 8, 3, 2, 2, 3, 3, 1, 1)      # only 2*3*2*2 = 24 output blocks exist
+    (aB, aK, aH, aW), _ = ob.parallel_partition(*dims, 512.0, 64)
+    assert aB * aK * aH * aW == 24
+    (aB, aK, aH, aW), _ = ob.parallel_partition(*dims, 512.0, 5)
+    assert aB * aK * aH * aW == 4           # 5 is prime and > every extent: 4 is the largest product
