@@ -104,6 +104,21 @@ typedef struct {
 int cconv_lower_bound(int B, int C, int K, int W, int H, int R, int S, int sw, int sh,
                       double M_words, double terms_out[5]);
 
+/* Section 8, "Parallel Algorithm": p processors that share one memory of M_words, the output cut
+ * into aB x aK x aH x aW equal blocks (one per processor, 1 <= aX <= X).  terms_out[0..4] are the
+ * five terms of the resulting bound on the total traffic: Theorem 1's, with the Image term times aK
+ * and the Filter term times aB*aH*aW.  Pure host arithmetic. */
+int cconv_parallel_lower_bound(int B, int C, int K, int W, int H, int R, int S, int sw, int sh,
+                               double M_words, int aB, int aK, int aH, int aW, double terms_out[5]);
+
+/* The cut for p processors (1 <= p <= 65536): among all (aB, aK, aH, aW) with aX <= X and product
+ * <= p, the one that uses the most processors, then gives the smallest bound, then replicates the
+ * least traffic (terms 2 + 3), then is lexicographically smallest (the paper only says to choose
+ * the values that minimise the bound).  a_out = {aB, aK, aH, aW}; *bound_out (may be NULL) = the
+ * bound in words.  Exhaustive search on the host. */
+int cconv_parallel_partition(int B, int C, int K, int W, int H, int R, int S, int sw, int sh,
+                             double M_words, int p, int a_out[4], double* bound_out);
+
 /* Section 5 tiling LP (maximise the sum of log_M block sizes subject to the block-fits-in-M
  * constraints), solved at the concrete parameters with a dense simplex.  Pure host.
  * tiles_out: b_b,b_c,b_k,b_w,b_h,b_r',b_r'',b_s',b_s'' (real numbers >= 1); *G_out their product;

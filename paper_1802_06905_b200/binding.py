@@ -25,6 +25,7 @@ EXPORTS = (
     "cconv_lower_bound", "cconv_tiling_lp", "cconv_plan_create", "cconv_plan_info_get",
     "cconv_plan_destroy", "cconv_forward_planned", "cconv_forward", "cconv_forward_host",
     "cconv_forward_noalloc", "cconv_pool_lower_bound", "cconv_pool_forward",
+    "cconv_parallel_lower_bound", "cconv_parallel_partition",
     "cconv_plan_status", "cconv_plan_trace_read", "cconv_strerror", "cconv_last_cuda_error", "cconv_version",
 )
 
@@ -100,6 +101,10 @@ def load_library():
     lib.cconv_forward_noalloc.argtypes = [vp, vp, vp] + nine + [i, vp, ctypes.POINTER(i)]
     lib.cconv_forward_host.restype = i
     lib.cconv_forward_host.argtypes = [vp, vp, vp, vp, vp]
+    lib.cconv_parallel_lower_bound.restype = i
+    lib.cconv_parallel_lower_bound.argtypes = nine + [d, i, i, i, i, dp]
+    lib.cconv_parallel_partition.restype = i
+    lib.cconv_parallel_partition.argtypes = nine + [d, i, ctypes.POINTER(i), dp]
     lib.cconv_pool_lower_bound.restype = i
     lib.cconv_pool_lower_bound.argtypes = nine + [d, dp]
     lib.cconv_pool_forward.restype = i
@@ -127,6 +132,25 @@ def lower_bound(B, C, K, W, H, R, S, sw, sh, M_words):
     _check(load_library().cconv_lower_bound(B, C, K, W, H, R, S, sw, sh, float(M_words), t),
            "cconv_lower_bound")
     return list(t)
+
+
+def parallel_lower_bound(B, C, K, W, H, R, S, sw, sh, M_words, aB, aK, aH, aW):
+    """cconv_parallel_lower_bound: the five terms for an aB x aK x aH x aW cut (Section 8)."""
+    t = (ctypes.c_double * 5)()
+    _check(load_library().cconv_parallel_lower_bound(B, C, K, W, H, R, S, sw, sh, float(M_words),
+                                                     aB, aK, aH, aW, t),
+           "cconv_parallel_lower_bound")
+    return list(t)
+
+
+def parallel_partition(B, C, K, W, H, R, S, sw, sh, M_words, p):
+    """cconv_parallel_partition: ((aB, aK, aH, aW), bound in words) for p processors."""
+    a = (ctypes.c_int * 4)()
+    bound = ctypes.c_double()
+    _check(load_library().cconv_parallel_partition(B, C, K, W, H, R, S, sw, sh, float(M_words),
+                                                   int(p), a, ctypes.byref(bound)),
+           "cconv_parallel_partition")
+    return tuple(a), bound.value
 
 
 def pool_lower_bound(B, C, K, W, H, R, S, sw, sh, M_words):

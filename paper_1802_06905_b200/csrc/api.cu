@@ -114,6 +114,23 @@ int cconv_lower_bound(int B, int C, int K, int W, int H, int R, int S, int sw, i
   return CCONV_OK;
 }
 
+int cconv_parallel_lower_bound(int B, int C, int K, int W, int H, int R, int S, int sw, int sh,
+                               double M_words, int aB, int aK, int aH, int aW, double terms_out[5]) {
+  const Dims d{B, C, K, W, H, R, S, sw, sh};
+  if (!d.positive() || !(M_words > 0) || !terms_out) return CCONV_EINVAL;
+  if (aB < 1 || aK < 1 || aH < 1 || aW < 1 || aB > B || aK > K || aH > H || aW > W) return CCONV_EINVAL;
+  const int a[4] = {aB, aK, aH, aW};
+  parallel_terms(d, M_words, a, terms_out);
+  return CCONV_OK;
+}
+
+int cconv_parallel_partition(int B, int C, int K, int W, int H, int R, int S, int sw, int sh,
+                             double M_words, int p, int a_out[4], double* bound_out) {
+  const Dims d{B, C, K, W, H, R, S, sw, sh};
+  if (!d.positive() || !(M_words > 0) || !a_out) return CCONV_EINVAL;
+  return choose_partition(d, M_words, p, a_out, bound_out) ? CCONV_OK : CCONV_EINVAL;
+}
+
 int cconv_tiling_lp(int B, int C, int K, int W, int H, int R, int S, int sw, int sh,
                     double M_words, int pooling, double tiles_out[9], double* G_out,
                     double* words_out) {

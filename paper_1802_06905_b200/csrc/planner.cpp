@@ -27,6 +27,48 @@ void theorem1_terms(const Dims& d, double M, double t[5]) {
   t[4] = F * std::sqrt(double(d.R) * d.S * d.sw * d.sh / M);
 }
 
+void parallel_terms(const Dims& d, double M, const int a[4], double t[5]) {
+  theorem1_terms(d, M, t);
+  t[1] *= double(a[1]);
+  t[2] *= double(a[0]) * a[2] * a[3];
+}
+
+bool choose_partition(const Dims& d, double M, int p, int a_out[4], double* bound_out) {
+  if (p < 1 || p > 65536) return false;
+  double base[5];
+  theorem1_terms(d, M, base);
+  bool found = false;
+  long long best_prod = 0;
+  double best_bound = 0, best_repl = 0;
+  int best[4] = {1, 1, 1, 1};
+  for (int aB = 1; aB <= std::min(d.B, p); ++aB)
+    for (int aK = 1; aK <= std::min(d.K, p / aB); ++aK)
+      for (int aH = 1; aH <= std::min(d.H, p / (aB * aK)); ++aH) {
+        // for fixed aB, aK, aH every term grows with aW, but more processors come first
+        for (int aW = 1; aW <= std::min(d.W, p / (aB * aK * aH)); ++aW) {
+          const long long prod = 1ll * aB * aK * aH * aW;
+          const double t2 = base[1] * aK, t3 = base[2] * aB * aH * aW;
+          const double bound = std::max({base[0], t2, t3, base[3], base[4]});
+          const double repl = t2 + t3;
+          const int cand[4] = {aB, aK, aH, aW};
+          bool better = !found || prod > best_prod;
+          if (!better && prod == best_prod) {
+            if (bound != best_bound) better = bound < best_bound;
+            else if (repl != best_repl) better = repl < best_repl;
+            else better = std::lexicographical_compare(cand, cand + 4, best, best + 4);
+          }
+          if (better) {
+            found = true;
+            best_prod = prod; best_bound = bound; best_repl = repl;
+            std::copy(cand, cand + 4, best);
+          }
+        }
+      }
+  std::copy(best, best + 4, a_out);
+  if (bound_out) *bound_out = best_bound;
+  return found;
+}
+
 namespace {
 
 // maximise sum(x) s.t. A x <= b (b >= 0), x >= 0.  Tableau simplex, Bland's anti-cycling rule.

@@ -93,6 +93,15 @@ struct StemTile {
 
 void theorem1_terms(const Dims& d, double M, double t[5]);
 
+// Section 8, "Parallel Algorithm": p processors behind one shared memory of M words, the output cut
+// into a[0] x a[1] x a[2] x a[3] = aB x aK x aH x aW equal blocks, one per processor.  The bound is p
+// times Theorem 1 on a block, i.e. the Image term times aK and the Filter term times aB*aH*aW.
+void parallel_terms(const Dims& d, double M, const int a[4], double t[5]);
+// The cut with aX <= X and product <= p that uses the most processors, then has the smallest
+// bound, then the least replicated traffic (terms 2 + 3), then is lexicographically smallest.
+// Returns false for p < 1 or p > 65536.
+bool choose_partition(const Dims& d, double M, int p, int a_out[4], double* bound_out);
+
 // Dense primal simplex on the LP of Section 5 in log_M space.  tiles[9] in the order
 // b_b,b_c,b_k,b_w,b_h,b_r',b_r'',b_s',b_s''.  Returns false on non-positive arguments.
 bool tiling_lp(const Dims& d, double M, bool pooling, double tiles[9], double* G, double* words);

@@ -199,3 +199,38 @@ def test_pool_lower_bound_matches_the_oracle_terms():
     t = (ctypes.c_double * 3)()
     assert lib.cconv_pool_lower_bound(0, 1, 1, 1, 1, 1, 1, 1, 1, 4.0, t) == -1
     assert lib.cconv_pool_lower_bound(1, 1, 1, 1, 1, 1, 1, 1, 1, 0.0, t) == -1
+
+
+def test_parallel_bound_and_partition_match_the_oracle():
+    rng = np.random.default_rng(17)
+    for _ in range(40):
+        B, C, K = (int(v) for v in rng.integers(1, 40, size=3))
+        W, H = (int(v) for v in rng.integers(1, 12, size=2))
+        R, S = (int(v) for v in rng.integers(1, 6, size=2))
+        sw, sh = (int(v) for v in rng.integers(1, 3, size=2))
+        M = float(rng.integers(64, 10 ** 5))
+        p = int(rng.integers(1, 40))
+        a, bound = binding.parallel_partition(B, C, K, W, H, R, S, sw, sh, M, p)
+        a_exp, bound_exp = ob.parallel_partition(B, C, K, W, H, R, S, sw, sh, M, p)
+        assert a == a_exp
+        assert bound == pytest.approx(bound_exp, rel=1e-12)
+        got = binding.parallel_lower_bound(B, C, K, W, H, R, S, sw, sh, M, *a)
+        assert got == pytest.approx(ob.parallel_terms(B, C, K, W, H, R, S, sw, sh, M, *a), rel=1e-12)
+        assert max(got) == pytest.approx(bound, rel=1e-12)
+    lib = binding.load_library()
+    t = (ctypes.c_double * 5)()
+    assert lib.cconv_parallel_lower_bound(4, 4, 4, 4, 4, 1, 1, 1, 1, 64.0, 5, 1, 1, 1, t) == -1  # aB > B
+    a = (ctypes.c_int * 4)()
+    assert lib.cconv_parallel_partition(4, 4, 4, 4, 4, 1, 1, 1, 1, 64.0, 0, a, None) == -1
+
+
+def test_batch_sharding_is_the_partition_the_bound_prefers_on_the_benchmark_shapes():
+    """Multi-GPU runs shard the batch: for the large shapes the paper's own criterion picks a cut
+    without aK (the Image is the big array), and with 8 processors the bound stays at |Out|."""
+    for cfg in CONFIGS[1:]:
+        dims = cfg.dims()
+        a, bound = binding.parallel_partition(*dims, 116224.0, 8)
+        one = max(binding.lower_bound(*dims, 116224.0))
+        batch_cut = max(binding.parallel_lower_bound(*dims, 116224.0, 8, 1, 1, 1))
+        assert batch_cut <= 1.0001 * max(one, 8 * dims[1] * dims[2] * dims[5] * dims[6])
+        assert bound <= batch_cut * (1 + 1e-12)
