@@ -104,6 +104,14 @@ typedef struct {
 int cconv_lower_bound(int B, int C, int K, int W, int H, int R, int S, int sw, int sh,
                       double M_words, double terms_out[5]);
 
+/* Theorem 2 (Appendix A), strides 1: the leaf of the decision tree that says which expression of
+ * Theorem 1 a tiling can attain for these loop bounds and a fast memory of M_words.  *leaf_out is the
+ * leaf's name written as an integer (1, 21, 221, 2221, 2222 for Cases 1, 2.1, 2.2.1, 2.2.2.1,
+ * 2.2.2.2); *alb_words_out (may be NULL) the attainable lower bound in words, constants dropped as
+ * in the theorem.  Pure host arithmetic. */
+int cconv_theorem2_case(int B, int C, int K, int W, int H, int R, int S, double M_words,
+                        int* leaf_out, double* alb_words_out);
+
 /* Section 8, "Parallel Algorithm": p processors that share one memory of M_words, the output cut
  * into aB x aK x aH x aW equal blocks (one per processor, 1 <= aX <= X).  terms_out[0..4] are the
  * five terms of the resulting bound on the total traffic: Theorem 1's, with the Image term times aK

@@ -25,7 +25,7 @@ EXPORTS = (
     "cconv_lower_bound", "cconv_tiling_lp", "cconv_plan_create", "cconv_plan_info_get",
     "cconv_plan_destroy", "cconv_forward_planned", "cconv_forward", "cconv_forward_host",
     "cconv_forward_noalloc", "cconv_pool_lower_bound", "cconv_pool_forward",
-    "cconv_parallel_lower_bound", "cconv_parallel_partition",
+    "cconv_parallel_lower_bound", "cconv_parallel_partition", "cconv_theorem2_case",
     "cconv_plan_status", "cconv_plan_trace_read", "cconv_strerror", "cconv_last_cuda_error", "cconv_version",
 )
 
@@ -101,6 +101,8 @@ def load_library():
     lib.cconv_forward_noalloc.argtypes = [vp, vp, vp] + nine + [i, vp, ctypes.POINTER(i)]
     lib.cconv_forward_host.restype = i
     lib.cconv_forward_host.argtypes = [vp, vp, vp, vp, vp]
+    lib.cconv_theorem2_case.restype = i
+    lib.cconv_theorem2_case.argtypes = [i] * 7 + [d, ctypes.POINTER(i), dp]
     lib.cconv_parallel_lower_bound.restype = i
     lib.cconv_parallel_lower_bound.argtypes = nine + [d, i, i, i, i, dp]
     lib.cconv_parallel_partition.restype = i
@@ -132,6 +134,15 @@ def lower_bound(B, C, K, W, H, R, S, sw, sh, M_words):
     _check(load_library().cconv_lower_bound(B, C, K, W, H, R, S, sw, sh, float(M_words), t),
            "cconv_lower_bound")
     return list(t)
+
+
+def theorem2_case(B, C, K, W, H, R, S, M_words):
+    """cconv_theorem2_case: (leaf name as a string such as "2.2.2.1", attainable bound in words)."""
+    leaf, alb = ctypes.c_int(), ctypes.c_double()
+    _check(load_library().cconv_theorem2_case(B, C, K, W, H, R, S, float(M_words),
+                                              ctypes.byref(leaf), ctypes.byref(alb)),
+           "cconv_theorem2_case")
+    return ".".join(str(leaf.value)), alb.value
 
 
 def parallel_lower_bound(B, C, K, W, H, R, S, sw, sh, M_words, aB, aK, aH, aW):

@@ -114,6 +114,14 @@ int cconv_lower_bound(int B, int C, int K, int W, int H, int R, int S, int sw, i
   return CCONV_OK;
 }
 
+int cconv_theorem2_case(int B, int C, int K, int W, int H, int R, int S, double M_words,
+                        int* leaf_out, double* alb_words_out) {
+  const Dims d{B, C, K, W, H, R, S, 1, 1};
+  if (!d.positive() || !(M_words > 0) || !leaf_out) return CCONV_EINVAL;
+  *leaf_out = theorem2_leaf(d, M_words, alb_words_out);
+  return CCONV_OK;
+}
+
 int cconv_parallel_lower_bound(int B, int C, int K, int W, int H, int R, int S, int sw, int sh,
                                double M_words, int aB, int aK, int aH, int aW, double terms_out[5]) {
   const Dims d{B, C, K, W, H, R, S, sw, sh};

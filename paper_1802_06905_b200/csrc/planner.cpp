@@ -27,6 +27,34 @@ void theorem1_terms(const Dims& d, double M, double t[5]) {
   t[4] = F * std::sqrt(double(d.R) * d.S * d.sw * d.sh / M);
 }
 
+int theorem2_leaf(const Dims& d, double M, double* alb_words) {
+  const double image = double(d.C) * d.H * d.W * d.B;   // CHWB (strides 1: the Image term)
+  const double filter = double(d.K) * d.C * d.R * d.S;  // KCRS
+  const double out = double(d.K) * d.H * d.W * d.B;     // KHWB
+  const double rs = double(d.R) * d.S, bhw = double(d.B) * d.H * d.W;
+  const double work = out * d.C;                        // KCHWB
+  int leaf;
+  double alb;
+  if (std::min({image, filter, out}) <= M) {
+    leaf = 1;      // one array fits: stream the other two once
+    alb = std::max({image, filter, out});
+  } else if (rs >= M) {
+    leaf = 21;     // the filter window alone overflows the fast memory: no reuse at all
+    alb = work * rs / M;
+  } else if (M * rs >= bhw * bhw) {
+    leaf = 221;    // few output positions: the Filter is the array to read once
+    alb = filter;
+  } else if (std::min(double(d.C), double(d.K)) >= std::sqrt(M / rs)) {
+    leaf = 2221;   // the small-filter term of Theorem 1 is reached
+    alb = work * std::sqrt(rs / M);
+  } else {
+    leaf = 2222;   // too few channels to fill a square block: an array-size term is reached
+    alb = std::max(out, image);
+  }
+  if (alb_words) *alb_words = alb;
+  return leaf;
+}
+
 void parallel_terms(const Dims& d, double M, const int a[4], double t[5]) {
   theorem1_terms(d, M, t);
   t[1] *= double(a[1]);

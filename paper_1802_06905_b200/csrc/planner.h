@@ -93,6 +93,11 @@ struct StemTile {
 
 void theorem1_terms(const Dims& d, double M, double t[5]);
 
+// Theorem 2 (Appendix A; strides 1): which expression of Theorem 1 is attainable.  Returns the leaf
+// of the decision tree as the digits of its name (1, 21, 221, 2221, 2222) and stores the attainable
+// lower bound in words.
+int theorem2_leaf(const Dims& d, double M, double* alb_words);
+
 // Section 8, "Parallel Algorithm": p processors behind one shared memory of M words, the output cut
 // into a[0] x a[1] x a[2] x a[3] = aB x aK x aH x aW equal blocks, one per processor.  The bound is p
 // times Theorem 1 on a block, i.e. the Image term times aK and the Filter term times aB*aH*aW.

@@ -234,3 +234,25 @@ def test_batch_sharding_is_the_partition_the_bound_prefers_on_the_benchmark_shap
         batch_cut = max(binding.parallel_lower_bound(*dims, 116224.0, 8, 1, 1, 1))
         assert batch_cut <= 1.0001 * max(one, 8 * dims[1] * dims[2] * dims[5] * dims[6])
         assert bound <= batch_cut * (1 + 1e-12)
+
+
+def test_theorem2_leaf_matches_the_oracle_and_the_benchmark_shapes():
+    rng = np.random.default_rng(23)
+    seen = set()
+    for _ in range(400):
+        B, C, K = (int(v) for v in rng.integers(1, 300, size=3))
+        W, H = (int(v) for v in rng.integers(1, 40, size=2))
+        R, S = (int(v) for v in rng.integers(1, 12, size=2))
+        M = float(2 ** rng.integers(1, 20))
+        leaf, alb = binding.theorem2_case(B, C, K, W, H, R, S, M)
+        leaf_exp, alb_exp = ob.theorem2_case(B, C, K, W, H, R, S, M)
+        assert leaf == leaf_exp
+        assert alb == pytest.approx(alb_exp, rel=1e-12)
+        seen.add(leaf)
+    assert seen == {"1", "2.1", "2.2.1", "2.2.2.1", "2.2.2.2"}
+    # the stride-1 benchmark shapes at the shared memory of one CTA
+    M = 116224.0
+    assert binding.theorem2_case(*CONFIGS[0].dims()[:7], M)[0] == "1"
+    assert binding.theorem2_case(*CONFIGS[1].dims()[:7], M)[0] == "2.2.2.1"
+    assert binding.theorem2_case(*CONFIGS[3].dims()[:7], M)[0] == "2.2.2.2"
+    assert binding.theorem2_case(*CONFIGS[4].dims()[:7], M)[0] == "2.2.2.1"
