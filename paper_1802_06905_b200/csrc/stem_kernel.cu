@@ -48,28 +48,6 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm,
       : "memory");
 }
 
-// 32 consecutive images of one (k, h, w): 64 B (bf16) or 128 B (fp32), written as whole 32-byte sectors
-template <typename OutT>
-__device__ __forceinline__ void store_run(OutT* dst, const uint32_t (&v)[32]) {
-  if constexpr (sizeof(OutT) == 4) {
-#pragma unroll
-    for (int i = 0; i < 4; ++i)
-      st_global_v8(dst + 8 * i, v[8 * i], v[8 * i + 1], v[8 * i + 2], v[8 * i + 3], v[8 * i + 4],
-                   v[8 * i + 5], v[8 * i + 6], v[8 * i + 7]);
-  } else {
-#pragma unroll
-    for (int i = 0; i < 2; ++i)
-      st_global_v8(dst + 16 * i, pack_bf16x2(v[16 * i + 0], v[16 * i + 1]),
-                   pack_bf16x2(v[16 * i + 2], v[16 * i + 3]),
-                   pack_bf16x2(v[16 * i + 4], v[16 * i + 5]),
-                   pack_bf16x2(v[16 * i + 6], v[16 * i + 7]),
-                   pack_bf16x2(v[16 * i + 8], v[16 * i + 9]),
-                   pack_bf16x2(v[16 * i + 10], v[16 * i + 11]),
-                   pack_bf16x2(v[16 * i + 12], v[16 * i + 13]),
-                   pack_bf16x2(v[16 * i + 14], v[16 * i + 15]));
-  }
-}
-
 }  // namespace
 
 // ------------------------------------------------------------------------------------------------
@@ -143,21 +121,30 @@ cudaError_t launch_pack_filter_stem(const void* filter, void* packed, const Dims
 // ------------------------------------------------------------------------------------------------
 // The kernel.  Persistent; tile = (128 out-channels) x (64 images) x (bhm output rows) x (bw pixels).
 // ------------------------------------------------------------------------------------------------
-// The same run cut off after `n` images (n a multiple of 8, as B is), in pieces of 8 images: for a
-// batch block padded past B, and for rows of Out that are not multiples of 32 bytes.
-template <typename OutT>
-__device__ __forceinline__ void store_run_partial(OutT* dst, const uint32_t (&v)[32], int n) {
+// Four lanes of a quad each hold four 8-word (32-byte) sectors of their own accumulator row.
+// After the call lane q of the quad holds sector q of the quad's rows 0..3 (slot j = row j): a 4x4
+// transpose of sectors in two butterfly stages of warp shuffles.  With it the four lanes of a quad
+// write one whole 128-byte line of ONE row per store instruction, and a warp eight whole lines,
+// instead of 32 lanes writing one sector each to 32 different lines (one per out-channel plane),
+// which the memory system absorbs at well under half the rate.
+__device__ __forceinline__ void quad_transpose_sectors(uint32_t (&s)[4][8], int lane) {
+  const bool b0 = lane & 1, b1 = lane & 2;
 #pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    if (8 * j < n) {
-      if constexpr (sizeof(OutT) == 4) {
-        st_global_v8(dst + 8 * j, v[8 * j], v[8 * j + 1], v[8 * j + 2], v[8 * j + 3], v[8 * j + 4],
-                     v[8 * j + 5], v[8 * j + 6], v[8 * j + 7]);
-      } else {
-        *reinterpret_cast<uint4*>(dst + 8 * j) =
-            make_uint4(pack_bf16x2(v[8 * j], v[8 * j + 1]), pack_bf16x2(v[8 * j + 2], v[8 * j + 3]),
-                       pack_bf16x2(v[8 * j + 4], v[8 * j + 5]), pack_bf16x2(v[8 * j + 6], v[8 * j + 7]));
-      }
+  for (int c = 0; c < 4; c += 2) {
+#pragma unroll
+    for (int w = 0; w < 8; ++w) {
+      const uint32_t send = b0 ? s[c][w] : s[c + 1][w];
+      const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 1);
+      if (b0) s[c][w] = recv; else s[c + 1][w] = recv;
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+#pragma unroll
+    for (int w = 0; w < 8; ++w) {
+      const uint32_t send = b1 ? s[i][w] : s[2 + i][w];
+      const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 2);
+      if (b1) s[i][w] = recv; else s[2 + i][w] = recv;
     }
   }
 }
@@ -335,11 +322,14 @@ __global__ void __launch_bounds__(kStemThreads, 1)
     // ===================== epilogue warps =====================
     const int q = warp & 3;            // this warp may touch TMEM lanes [32q, 32q+32)
     const int eset = (warp - 2) >> 2;  // 0: even pixels of a tile, 1: odd pixels
-    // TMEM lane = j*kpad + kk: stacked output row j (uniform in a warp), out-channel kk.  A lane
-    // reads the 64 images of one pixel and writes them as one 128-byte (bf16) or 256-byte (fp32) run
-    // of Out, in whole 32-byte sectors.
-    const int L = q * 32 + lane;
-    const int j = L / p.kpad, kk = L - j * p.kpad;
+    // TMEM lane L = j*kpad + kk: stacked output row j, out-channel kk (kpad is a power of two).  A
+    // lane reads the 64 images of one pixel of its row; the sectors are then transposed within
+    // quads of lanes (quad_transpose_sectors) so that a quad writes whole lines of Out.
+    constexpr int kSectorElems = 32 / int(sizeof(OutT));  // images per 32-byte sector: 16 / 8
+    constexpr int kPasses = int(sizeof(OutT)) / 2;         // 128-byte row pieces per pixel: 1 / 2
+    const int kpad_log2 = 31 - __clz(p.kpad);
+    const int sector = lane & 3;                           // the sector this lane stores
+    const long long plane_row = (long long)p.W * p.B;      // elements per (k, h) row of Out
     uint32_t abuf = 0, aph = 0;
     long long t_wf = 0, t_busy = 0, t_ld = 0;
     for (int tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
@@ -349,16 +339,25 @@ __global__ void __launch_bounds__(kStemThreads, 1)
       const int wt = t % p.tiles_w;
       t /= p.tiles_w;
       const int ht = t % p.tiles_h, bt = t / p.tiles_h;
-      const int k = kt * 128 + kk;
-      const int h = ht * p.bhm + j;
+      // the four rows of this lane's quad: accumulator rows 4*(lane/4) + j of the warp's 32
+      OutT* rowp[4];
+      uint32_t row_ok = 0;
+      const long long tile_off = (long long)(wt * p.bw) * p.B + bt * 64 + sector * kSectorElems;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int L = q * 32 + 4 * (lane >> 2) + j;
+        const int jr = L >> kpad_log2, kk = L & (p.kpad - 1);
+        const int k = kt * 128 + kk, h = ht * p.bhm + jr;
+        if (k < p.K && jr < p.bhm && h < p.H) row_ok |= 1u << j;
+        rowp[j] = out + ((long long)k * p.H + h) * plane_row + tile_off;
+      }
+      const int nb = p.B - bt * 64;  // images left in the batch (the block is padded past B)
       const long long c0 = tr ? clock64() : 0;
       if (!mbar_wait_warp(bar_tfull + 8u * abuf, aph, abort_flag, status, kStatEpilogueWait, limit))
         break;
       const long long c1 = tr ? clock64() : 0;
       tc_fence_after();
       const uint32_t t_base = tmem_base + (uint32_t(q * 32) << 16) + abuf * uint32_t(p.acc_cols);
-      const bool row_ok = (k < p.K) && (j < p.bhm) && (h < p.H);
-      OutT* row = out + (((long long)k * p.H + h) * p.W + wt * p.bw) * p.B + bt * 64;
       for (int px = eset; px < p.bw; px += 2) {
         uint32_t va[32], vb[32];
         const long long l0 = tr ? clock64() : 0;
@@ -366,15 +365,41 @@ __global__ void __launch_bounds__(kStemThreads, 1)
         tmem_ld_32x32b_x32(t_base + uint32_t(px * 64 + 32), vb);
         tmem_ld_wait();
         if (tr) t_ld += clock64() - l0;
-        if (row_ok && wt * p.bw + px < p.W) {
-          OutT* dst = row + (long long)px * p.B;
-          const int nb = p.B - bt * 64;  // images left in the batch (the block is padded past B)
-          if (nb >= 64 && wide_rows) {
-            store_run(dst, va);
-            store_run(dst + 32, vb);
+        const bool px_ok = wt * p.bw + px < p.W;
+#pragma unroll
+        for (int pass = 0; pass < kPasses; ++pass) {
+          uint32_t sec[4][8];  // this lane's 128-byte row piece as four sectors
+          if constexpr (sizeof(OutT) == 2) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              sec[0][i] = pack_bf16x2(va[2 * i], va[2 * i + 1]);
+              sec[1][i] = pack_bf16x2(va[16 + 2 * i], va[17 + 2 * i]);
+              sec[2][i] = pack_bf16x2(vb[2 * i], vb[2 * i + 1]);
+              sec[3][i] = pack_bf16x2(vb[16 + 2 * i], vb[17 + 2 * i]);
+            }
           } else {
-            store_run_partial(dst, va, nb < 32 ? nb : 32);
-            if (nb > 32) store_run_partial(dst + 32, vb, nb - 32 < 32 ? nb - 32 : 32);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) sec[i >> 3][i & 7] = pass == 0 ? va[i] : vb[i];
+          }
+          quad_transpose_sectors(sec, lane);
+          // first image (within the block of 64) of the sector this lane stores
+          const int first = sector * kSectorElems + pass * 32;
+          const int left = nb - first;  // images of the sector inside the batch (a multiple of 8)
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            if (!px_ok || !((row_ok >> j) & 1u) || left <= 0) continue;
+            OutT* dst = rowp[j] + (long long)px * p.B + pass * 32;
+            if (left >= kSectorElems && wide_rows) {
+              st_global_v8(dst, sec[j][0], sec[j][1], sec[j][2], sec[j][3], sec[j][4], sec[j][5],
+                           sec[j][6], sec[j][7]);
+            } else {
+              // rows of Out that are not multiples of 32 bytes, or a sector cut by the end of the
+              // batch (bf16 only: half a sector = 8 images): 16-byte pieces
+              *reinterpret_cast<uint4*>(dst) = make_uint4(sec[j][0], sec[j][1], sec[j][2], sec[j][3]);
+              if (left >= kSectorElems)
+                *reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(dst) + 16) =
+                    make_uint4(sec[j][4], sec[j][5], sec[j][6], sec[j][7]);
+            }
           }
         }
       }
