@@ -38,6 +38,7 @@ namespace {
 // taking every other pixel of a tile)
 constexpr int kStemThreads = 320;
 constexpr int kStemEpiThreads = 256;
+constexpr int kFiltBars = 16;  // 16 KB Filter pieces: at most 14 fit in shared memory
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, int c0, int c1,
                                             int c2, uint32_t bar) {
@@ -162,7 +163,7 @@ __global__ void __launch_bounds__(kStemThreads, 1)
   const uint32_t bar_ifull = bars;
   const uint32_t bar_iempty = bar_ifull + 8u * p.i_stages;
   const uint32_t bar_filt = bar_iempty + 8u * p.i_stages;
-  const uint32_t bar_tfull = bar_filt + 8u;
+  const uint32_t bar_tfull = bar_filt + 8u * kFiltBars;  // one Filter barrier per 16 KB piece
   const uint32_t bar_tempty = bar_tfull + 16u;
   const uint32_t bar_drain = bar_tempty + 16u;
   const uint32_t slot_addr = bar_drain + 8u;
@@ -181,7 +182,7 @@ __global__ void __launch_bounds__(kStemThreads, 1)
       mbar_init(bar_ifull + 8u * s, 1);
       mbar_init(bar_iempty + 8u * s, 1);
     }
-    mbar_init(bar_filt, 1);
+    for (int f = 0; f < kFiltBars; ++f) mbar_init(bar_filt + 8u * f, 1);
     for (int a = 0; a < 2; ++a) {
       mbar_init(bar_tfull + 8u * a, 1);
       mbar_init(bar_tempty + 8u * a, kStemEpiThreads / 32);  // one arrival per epilogue warp
@@ -215,11 +216,8 @@ __global__ void __launch_bounds__(kStemThreads, 1)
       // may start: it writes the other scratch buffer while this kernel runs.
       asm volatile("griddepcontrol.wait;" ::: "memory");
       asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-      mbar_arrive_expect_tx(bar_filt, p.filt_bytes);
-      for (uint32_t off = 0; off < p.filt_bytes; off += 16384u) {
-        const uint32_t n = p.filt_bytes - off < 16384u ? p.filt_bytes - off : 16384u;
-        bulk_load(filt_smem + off, packed_filter + off, n, bar_filt);
-      }
+      // The first Image window goes out before the Filter: the first MMA needs both, and one
+      // thread's copies are issued one after the other.
       for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x, ++it) {
         int t = tile / p.tiles_k;
         const int wt = t % p.tiles_w;
@@ -239,14 +237,25 @@ __global__ void __launch_bounds__(kStemThreads, 1)
           s = 0;
           ph ^= 1u;
         }
+        if (it == 0) {
+          // the Filter in 16 KB pieces (four 4 KB blocks), each with its own barrier: the MMAs of
+          // the first tile start on the first piece while the others are still in flight
+          for (uint32_t off = 0, f = 0; off < p.filt_bytes; off += 16384u, ++f) {
+            const uint32_t n = p.filt_bytes - off < 16384u ? p.filt_bytes - off : 16384u;
+            mbar_arrive_expect_tx(bar_filt + 8u * f, n);
+            bulk_load(filt_smem + off, packed_filter + off, n, bar_filt + 8u * f);
+          }
+        }
       }
       if (tr) tr[2] = (unsigned long long)t_wait;
       drain_ring(bar_ifull, it, n_st, status, limit);
       const uint64_t t0 = globaltimer_ns();
-      while (!mbar_try_wait(bar_filt, 0)) {
-        if (globaltimer_ns() - t0 > limit) {
-          atomicOr(status, kStatDrainWait);
-          break;
+      for (uint32_t f = 0; f < (p.filt_bytes + 16383u) / 16384u; ++f) {
+        while (!mbar_try_wait(bar_filt + 8u * f, 0)) {
+          if (globaltimer_ns() - t0 > limit) {
+            atomicOr(status, kStatDrainWait);
+            break;
+          }
         }
       }
     }
@@ -262,10 +271,9 @@ __global__ void __launch_bounds__(kStemThreads, 1)
     const uint32_t idesc = p.idesc;
     const int units = p.units;
     const uint32_t kt_step16 = uint32_t(units) * 256u;  // one k-tile of the Filter: units x 4 KB
-    long long t_filt = tr ? clock64() : 0, t_wt = 0, t_wi = 0, t_issue = 0, n_tiles = 0;
-    bool ok = mbar_wait_warp(bar_filt, 0, abort_flag, status, kStatMmaWaitFull, limit);
-    if (tr) t_filt = clock64() - t_filt;
-    tc_fence_after();
+    long long t_filt = 0, t_wt = 0, t_wi = 0, t_issue = 0, n_tiles = 0;
+    bool ok = true, filt_ready = false;
+    const uint32_t filt_pieces = (p.filt_bytes + 16383u) / 16384u;
     for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
       const uint32_t kt = uint32_t(tile % p.tiles_k);
       const long long c0 = tr ? clock64() : 0;
@@ -280,13 +288,38 @@ __global__ void __launch_bounds__(kStemThreads, 1)
       const uint32_t d = tmem_base + abuf * uint32_t(p.acc_cols);
       uint32_t a16 = a_lo0 | (filt16 + kt * kt_step16);   // +256 per unit (4 KB Filter block)
       uint32_t b16 = b_lo0 | (img_ring16 + is * img16);   // +128 per unit (16 window rows)
-      umma_bf16_if(leader, d, (uint64_t(a_hi) << 32) | a16, (uint64_t(b_hi) << 32) | b16, idesc, 0u);
+      if (!filt_ready) {
+        // first tile of this CTA: wait for each 16 KB piece of the Filter when its first block is
+        // due, then (after the last MMA is issued) for the rest of the Filter
+        const long long f0 = tr ? clock64() : 0;
+        uint32_t blk = kt * uint32_t(units), waited = 0xffffffffu;
+        for (int u = 0; ok && u < units; ++u, ++blk) {
+          if ((blk >> 2) != waited) {
+            waited = blk >> 2;
+            ok = mbar_wait_warp(bar_filt + 8u * waited, 0, abort_flag, status, kStatMmaWaitFull, limit);
+            tc_fence_after();
+          }
+          if (ok)
+            umma_bf16_if(leader, d, (uint64_t(a_hi) << 32) | a16, (uint64_t(b_hi) << 32) | b16, idesc,
+                         u ? 1u : 0u);
+          a16 += 256u;
+          b16 += 128u;
+        }
+        for (uint32_t f = 0; ok && f < filt_pieces; ++f)
+          ok = mbar_wait_warp(bar_filt + 8u * f, 0, abort_flag, status, kStatMmaWaitFull, limit);
+        tc_fence_after();
+        filt_ready = true;
+        if (tr) t_filt = clock64() - f0;
+        if (!ok) break;
+      } else {
+        umma_bf16_if(leader, d, (uint64_t(a_hi) << 32) | a16, (uint64_t(b_hi) << 32) | b16, idesc, 0u);
 #pragma unroll 2
-      for (int u = 1; u < units; ++u) {
-        a16 += 256u;
-        b16 += 128u;
-        umma_bf16_if(leader, d, (uint64_t(a_hi) << 32) | a16, (uint64_t(b_hi) << 32) | b16, idesc,
-                     1u);
+        for (int u = 1; u < units; ++u) {
+          a16 += 256u;
+          b16 += 128u;
+          umma_bf16_if(leader, d, (uint64_t(a_hi) << 32) | a16, (uint64_t(b_hi) << 32) | b16, idesc,
+                       1u);
+        }
       }
       if (leader) umma_commit(bar_iempty + 8u * is);
       if (leader) umma_commit(bar_tfull + 8u * abuf);
