@@ -195,7 +195,7 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
   if (variant == CCONV_VARIANT_AUTO && env_variant >= 1 && env_variant <= 3) variant = env_variant;
 
   const bool halo_ok = halo_supported(dk, nullptr) && choose_halo_tile(dk, pl->m, force, &pl->tile);
-  const bool stem_ok = choose_stem_tile(d, pl->m, &pl->stile);
+  const bool stem_ok = choose_stem_tile(d, pl->m, &pl->stile, env_int("CCONV_STEM_BW", 0));
   if ((variant == CCONV_VARIANT_HALO && !halo_ok) || (variant == CCONV_VARIANT_STEM && !stem_ok)) {
     delete pl;
     return CCONV_EUNSUPPORTED;

@@ -3,6 +3,7 @@
 
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cstdlib>
 
 #include "../../include/cconv.h"
@@ -135,6 +136,7 @@ void build_stem_params(const Dims& d, const StemTile& t, StemKernelParams* out) 
   p.i_stages = t.i_stages;
   p.acc_cols = 64 * t.bw;
   p.tmem_cols = t.tmem_cols;
+  p.acc_bufs = std::min(8, t.tmem_cols / p.acc_cols);
   p.img_stage_bytes = t.img_stage_bytes;
   p.filt_bytes = t.filt_bytes;
   // instruction descriptor: D=f32, A=B=bf16, A K-major [15]=0, B MN-major [16]=1, N = 64*bw, M = 128

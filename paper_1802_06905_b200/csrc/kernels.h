@@ -68,6 +68,7 @@ struct StemKernelParams {
   int tiles_k, tiles_w, tiles_h, tiles_b, total_tiles;
   int i_stages;
   int acc_cols, tmem_cols;
+  int acc_bufs;           // accumulator buffers of acc_cols columns in tensor memory (2..8)
   uint32_t img_stage_bytes, filt_bytes;
   uint32_t idesc;
   uint64_t a_desc, b_desc;

@@ -399,7 +399,7 @@ bool choose_halo_tail(const Dims& d, const Machine& m, const HaloTile& main, int
   return found;
 }
 
-bool choose_stem_tile(const Dims& d, const Machine& m, StemTile* out) {
+bool choose_stem_tile(const Dims& d, const Machine& m, StemTile* out, int force_bw) {
   // the Image's row stride must be a multiple of 16 bytes for TMA; a block of 64 images is zero
   // padded past B
   if (d.B % 8 != 0) return false;
@@ -418,6 +418,7 @@ bool choose_stem_tile(const Dims& d, const Machine& m, StemTile* out) {
     const long long filt = 1ll * t.tiles_k * d.R * (kw / 16) * 4096;
     if (filt > cap) continue;
     for (int bw = 4; bw >= 1; --bw) {
+      if (force_bw > 0 && bw != force_bw) continue;
       if (bw > 1 && bw - 1 >= d.W) continue;  // no wider than the output row
       const int halo_w = d.sw * (bw - 1) + d.R;
       if (halo_w > 256) continue;
@@ -437,9 +438,7 @@ bool choose_stem_tile(const Dims& d, const Machine& m, StemTile* out) {
   }
   if (!found) return false;
   t.packed_filter_bytes = t.filt_bytes;
-  int cols = 32;
-  while (cols < 2 * 64 * t.bw) cols *= 2;  // two accumulator buffers of 64*bw columns
-  t.tmem_cols = cols;
+  t.tmem_cols = 512;  // all of it: 512 / (64*bw) accumulator buffers (2 for bw = 3 or 4, 4 for bw = 2)
   t.tiles_w = (d.W + t.bw - 1) / t.bw;
   t.tiles_h = (d.H + t.bhm - 1) / t.bhm;
   t.tiles_b = (d.B + 63) / 64;

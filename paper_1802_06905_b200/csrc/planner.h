@@ -130,6 +130,6 @@ bool choose_halo_tail(const Dims& d, const Machine& m, const HaloTile& main, int
 
 // The stem kernel needs B % 8 == 0 and the resident Filter plus two Image windows to fit in shared
 // memory.
-bool choose_stem_tile(const Dims& d, const Machine& m, StemTile* out);
+bool choose_stem_tile(const Dims& d, const Machine& m, StemTile* out, int force_bw = 0);
 
 }  // namespace cconv

@@ -39,6 +39,7 @@ namespace {
 constexpr int kStemThreads = 320;
 constexpr int kStemEpiThreads = 256;
 constexpr int kFiltBars = 16;  // 16 KB Filter pieces: at most 14 fit in shared memory
+constexpr int kMaxAccBufs = 8;  // accumulator buffers in tensor memory: tmem_cols / acc_cols
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, int c0, int c1,
                                             int c2, uint32_t bar) {
@@ -164,8 +165,8 @@ __global__ void __launch_bounds__(kStemThreads, 1)
   const uint32_t bar_iempty = bar_ifull + 8u * p.i_stages;
   const uint32_t bar_filt = bar_iempty + 8u * p.i_stages;
   const uint32_t bar_tfull = bar_filt + 8u * kFiltBars;  // one Filter barrier per 16 KB piece
-  const uint32_t bar_tempty = bar_tfull + 16u;
-  const uint32_t bar_drain = bar_tempty + 16u;
+  const uint32_t bar_tempty = bar_tfull + 8u * kMaxAccBufs;
+  const uint32_t bar_drain = bar_tempty + 8u * kMaxAccBufs;
   const uint32_t slot_addr = bar_drain + 8u;
   uint8_t* gen0 = smem_raw + (smem0 - smem_u32(smem_raw));
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen0 + (slot_addr - smem0));
@@ -183,7 +184,7 @@ __global__ void __launch_bounds__(kStemThreads, 1)
       mbar_init(bar_iempty + 8u * s, 1);
     }
     for (int f = 0; f < kFiltBars; ++f) mbar_init(bar_filt + 8u * f, 1);
-    for (int a = 0; a < 2; ++a) {
+    for (int a = 0; a < kMaxAccBufs; ++a) {
       mbar_init(bar_tfull + 8u * a, 1);
       mbar_init(bar_tempty + 8u * a, kStemEpiThreads / 32);  // one arrival per epilogue warp
     }
@@ -263,7 +264,7 @@ __global__ void __launch_bounds__(kStemThreads, 1)
     // ===================== MMA issuer (whole warp walks, one lane issues) =====================
     const bool leader = elect_one();
     uint32_t is = 0, iph = 0, abuf = 0, aph = 0;
-    const uint32_t n_ist = uint32_t(p.i_stages);
+    const uint32_t n_ist = uint32_t(p.i_stages), n_acc = uint32_t(p.acc_bufs);
     const uint32_t a_lo0 = uint32_t(p.a_desc), a_hi = uint32_t(p.a_desc >> 32);
     const uint32_t b_lo0 = uint32_t(p.b_desc), b_hi = uint32_t(p.b_desc >> 32);
     const uint32_t img16 = p.img_stage_bytes >> 4;
@@ -333,8 +334,10 @@ __global__ void __launch_bounds__(kStemThreads, 1)
         is = 0;
         iph ^= 1u;
       }
-      abuf ^= 1u;
-      if (abuf == 0) aph ^= 1u;
+      if (++abuf == n_acc) {
+        abuf = 0;
+        aph ^= 1u;
+      }
     }
     if (tr && lane == 0) {
       tr[3] = (unsigned long long)t_wt;
@@ -364,6 +367,7 @@ __global__ void __launch_bounds__(kStemThreads, 1)
     const int sector = lane & 3;                           // the sector this lane stores
     const long long plane_row = (long long)p.W * p.B;      // elements per (k, h) row of Out
     uint32_t abuf = 0, aph = 0;
+    const uint32_t n_acc = uint32_t(p.acc_bufs);
     long long t_wf = 0, t_busy = 0, t_ld = 0;
     for (int tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
       int t = tile;
@@ -439,8 +443,10 @@ __global__ void __launch_bounds__(kStemThreads, 1)
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_tempty + 8u * abuf);
-      abuf ^= 1u;
-      if (abuf == 0) aph ^= 1u;
+      if (++abuf == n_acc) {
+        abuf = 0;
+        aph ^= 1u;
+      }
       if (tr) {
         t_wf += c1 - c0;
         t_busy += clock64() - c1;
