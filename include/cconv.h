@@ -25,8 +25,9 @@
  * Ownership: the caller owns Image, Filter and Out.  Unless a function says "host", they are
  * DEVICE pointers on the plan's device, 16-byte aligned (Out: 32-byte aligned), and Out must not
  * overlap the inputs.
- * The library keeps no caller pointer after a call returns.  Device calls are asynchronous on the
- * given stream and never synchronise it.
+ * The library never dereferences a caller pointer after a call returns (it remembers the address
+ * range of the last call's Out, to order a following call whose Image overlaps it).  Device calls are
+ * asynchronous on the given stream, obey stream order, and never synchronise the stream.
  *
  * Errors: every function returns CCONV_OK (0) or a negative code; nothing throws, aborts or traps.
  * All positive loop bounds are accepted, also those outside the paper's assumptions

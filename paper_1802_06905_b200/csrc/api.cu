@@ -36,6 +36,38 @@ int env_int(const char* name, int dflt) {
   return (v && *v) ? std::atoi(v) : dflt;
 }
 
+// Out of the most recent tensor-core convolution launched through a plan, and its stream (see
+// cconv_forward_planned).
+struct LastOut {
+  bool valid = false;
+  void* stream = nullptr;
+  const char* lo = nullptr;
+  const char* hi = nullptr;
+};
+LastOut g_last_out;
+std::mutex g_last_out_mu;
+
+// Records this call's Out as the latest one and says whether its Image overlaps the Out of the
+// tensor-core convolution launched just before it on the same stream.  Those kernels let their
+// successors start while they are still in their last tiles (that hides the launch gap), and the
+// halo kernel's Image producers read at once: wrong only in that one case, which the two layouts
+// make useless but do not forbid; the producers are then told to wait for the earlier call.
+bool note_call_and_check_overlap(const Dims& d, int out_dtype, const void* Image, const void* Out,
+                                 void* stream, bool early_start_kernel) {
+  const char* img_lo = static_cast<const char*>(Image);
+  const char* img_hi = img_lo + size_t(d.Wi()) * d.Hi() * d.C * d.B * 2;
+  const char* out_lo = static_cast<const char*>(Out);
+  const char* out_hi = out_lo + size_t(d.K) * d.H * d.W * d.B * (out_dtype == CCONV_OUT_F32 ? 4 : 2);
+  std::lock_guard<std::mutex> lk(g_last_out_mu);
+  const bool overlap = g_last_out.valid && g_last_out.stream == stream && g_last_out.lo < img_hi &&
+                       img_lo < g_last_out.hi;
+  g_last_out.valid = early_start_kernel;
+  g_last_out.stream = stream;
+  g_last_out.lo = out_lo;
+  g_last_out.hi = out_hi;
+  return overlap;
+}
+
 }  // namespace
 
 struct cconv_plan {
@@ -370,6 +402,8 @@ int cconv_forward_planned(const cconv_plan* pl, const void* Image, const void* F
   if (!aligned16(Image) || !aligned16(Filter) || (reinterpret_cast<uintptr_t>(Out) & 31u))
     return CCONV_EINVAL;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const bool image_overlaps_last_out = note_call_and_check_overlap(
+      pl->d, pl->out_dtype, Image, Out, cuda_stream, pl->variant != CCONV_VARIANT_SIMT);
   if (pl->variant == CCONV_VARIANT_SIMT) {
     cudaError_t e = launch_simt(Image, Filter, Out, pl->out_dtype == CCONV_OUT_F32, pl->d, stream);
     return e == cudaSuccess ? CCONV_OK : cuda_fail(e, "launch_simt");
@@ -399,10 +433,12 @@ int cconv_forward_planned(const cconv_plan* pl, const void* Image, const void* F
                      pl->stile.smem_bytes, pl->d_status, stream);
     return es == cudaSuccess ? CCONV_OK : cuda_fail(es, "launch_stem");
   }
+  HaloKernelParams kp = pl->kp;
+  kp.image_wait = image_overlaps_last_out ? 1 : 0;
   cudaError_t e = launch_pack_filter(Filter, packed, pl->d, pl->tile.c16, pl->tile.tiles_k,
                                      /*overlap_prev=*/true, stream);
   if (e != cudaSuccess) return cuda_fail(e, "launch_pack_filter");
-  e = launch_halo(tmi, packed, Out, pl->out_dtype == CCONV_OUT_F32, pl->kp, pl->tile.grid,
+  e = launch_halo(tmi, packed, Out, pl->out_dtype == CCONV_OUT_F32, kp, pl->tile.grid,
                   pl->tile.smem_bytes, pl->d_status, stream);
   if (e == cudaSuccess && pl->has_tail)
     e = launch_halo(tmi_tail, packed, Out, pl->out_dtype == CCONV_OUT_F32, pl->kp_tail,

@@ -70,6 +70,7 @@ void build_halo_params(const Dims& d, const HaloTile& t, HaloKernelParams* out) 
   p.cchunks_cta = t.cchunks / t.split;
   p.h0 = 0;
   p.tail = 0;
+  p.image_wait = 0;
   p.n_mma = t.bb * t.bw;
   p.acc_cols = p.n_mma * t.bh;
   p.acc_bufs = t.acc_bufs;

@@ -530,6 +530,10 @@ __global__ void __launch_bounds__(kThreads, 1)
       bool ok = true;
       const int cchunks = p.cchunks_cta;
       const int c_first = crank * p.cchunks_cta * p.bc;
+      // This kernel may start while the convolution of the call in front of it is still running
+      // (that kernel is the only kind that lets its successors start early).  If that call's Out
+      // overlaps this call's Image -- the host checks -- nothing is read before it is complete.
+      if (p.image_wait) asm volatile("griddepcontrol.wait;" ::: "memory");
       for (int tile = tile_first; ok && tile < p.total_tiles; tile += tile_step) {
         int t = tile / p.tiles_k;
         const int bt = t % p.tiles_b; t /= p.tiles_b;
@@ -799,10 +803,18 @@ cudaError_t prepare_all(int smem_bytes) {
 
 }  // namespace
 
+// The attribute is a per-kernel ceiling, and the value set last wins: several plans (and the
+// non-allocating entry point) share these kernels, so it is always raised to the device's limit,
+// never to one plan's need (a second plan with a smaller tile would otherwise break the first).
 cudaError_t halo_kernel_prepare(int smem_bytes) {
-  cudaError_t e = prepare_all<__nv_bfloat16>(smem_bytes);
+  int dev = 0, cap = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&cap, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
   if (e != cudaSuccess) return e;
-  return prepare_all<float>(smem_bytes);
+  if (smem_bytes > cap) return cudaErrorInvalidValue;
+  e = prepare_all<__nv_bfloat16>(cap);
+  if (e != cudaSuccess) return e;
+  return prepare_all<float>(cap);
 }
 
 cudaError_t launch_halo(const CUtensorMap& tm_image, const void* packed_filter, void* out,

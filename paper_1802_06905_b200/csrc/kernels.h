@@ -40,6 +40,8 @@ struct HaloKernelParams {
   int cchunks_cta;              // Image stages one CTA loads per tile: ceil(C/bc) / split
   int h0;                       // first output row of this launch (tiles_h counts rows from there)
   int tail;                     // 1: second launch of a call, started while the first still runs
+  int image_wait;               // 1: Image overlaps the Out of the call in front of this one on the
+                                // stream: the Image producers wait for that call to complete
   int n_mma;                    // N of one MMA = bb*bw
   int acc_cols, acc_bufs, tmem_cols;
   uint32_t img_stage_bytes, filt_stage_bytes;

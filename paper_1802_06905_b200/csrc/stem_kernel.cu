@@ -469,12 +469,19 @@ __global__ void __launch_bounds__(kStemThreads, 1)
   if (tr && threadIdx.x == 0) tr[1] = globaltimer_ns();
 }
 
+// (The attribute is a per-kernel ceiling and the value set last wins: it is raised to the device's
+// limit, never to one plan's need, since several plans share the kernel.)
 cudaError_t stem_kernel_prepare(int smem_bytes) {
-  cudaError_t e = cudaFuncSetAttribute(cconv_stem_kernel<__nv_bfloat16>,
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+  int dev = 0, cap = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&cap, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+  if (e != cudaSuccess) return e;
+  if (smem_bytes > cap) return cudaErrorInvalidValue;
+  e = cudaFuncSetAttribute(cconv_stem_kernel<__nv_bfloat16>,
+                           cudaFuncAttributeMaxDynamicSharedMemorySize, cap);
   if (e != cudaSuccess) return e;
   return cudaFuncSetAttribute(cconv_stem_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              smem_bytes);
+                              cap);
 }
 
 cudaError_t launch_stem(const CUtensorMap& tm_image, const void* packed_filter, void* out,

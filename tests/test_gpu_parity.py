@@ -336,3 +336,51 @@ def test_repeated_launches_are_deterministic():
     np.testing.assert_array_equal(outs[0], outs[1])
     np.testing.assert_array_equal(outs[0], outs[2])
     plan.close()
+
+
+def test_out_of_one_call_read_as_image_by_the_next_call_on_the_stream():
+    """The convolution kernel of a call may start while the previous call's kernel is in its last
+    tiles.  If the previous call's Out IS this call's Image (the layouts differ, but shapes can be
+    made to agree: (K,H,W,B) of call A = (Wi,Hi,C,B) of call B), call B must still see all of it."""
+    a = cs("chain_a", 64, 96, 128, 28, 28, 3, 3)                  # Out (128, 28, 28, 64)
+    b = cs("chain_b", 64, 28, 64, 126, 26, 3, 3)                  # Image (128, 28, 28, 64)
+    assert a.out_shape == b.image_shape
+    ia, fa = synth.make_inputs(a)
+    _, fb = synth.make_inputs(b)
+    img_a, flt_a, flt_b = to_dev(ia), to_dev(fa), to_dev(fb)
+    plan_a = binding.Plan(*a.dims(), device=0, variant=binding.VARIANT_HALO, out_dtype=binding.OUT_BF16)
+    plan_b = binding.Plan(*b.dims(), device=0, variant=binding.VARIANT_HALO, out_dtype=binding.OUT_F32)
+    mid = torch.zeros(a.out_shape, dtype=torch.bfloat16, device="cuda")
+    out_b = torch.empty(b.out_shape, dtype=torch.float32, device="cuda")
+    for rep in range(6):
+        mid.zero_()                                               # stale values would be zeros
+        out_b.fill_(float("nan"))
+        plan_a.forward(img_a, flt_a, mid)
+        plan_b.forward(mid, flt_b, out_b)
+        plan_a.check()
+        plan_b.check()
+        exp, ab = ocnn.cnn_bf16(to_bits(mid), fb, oshape(b))      # oracle on what call A really wrote
+        assert_close(out_b.cpu().numpy().astype(np.float64), exp, ab, what=f"chained call, repeat {rep}")
+    # call A itself is checked elsewhere; here only that it wrote something
+    assert float(mid.float().abs().max()) > 0
+    plan_a.close()
+    plan_b.close()
+
+
+def test_two_plans_with_different_shared_memory_needs_stay_usable():
+    """Plans share the kernels: creating a second plan with a smaller tile must not lower the
+    shared-memory ceiling the first one needs."""
+    big = cs("two_plans_big", 64, 64, 128, 12, 10, 3, 3)
+    small = cs("two_plans_small", 32, 16, 64, 4, 3, 1, 1)
+    plan_big = binding.Plan(*big.dims(), device=0, variant=binding.VARIANT_HALO, out_dtype=binding.OUT_F32)
+    plan_small = binding.Plan(*small.dims(), device=0, variant=binding.VARIANT_HALO, out_dtype=binding.OUT_F32)
+    assert plan_small.info()["smem_bytes"] <= plan_big.info()["smem_bytes"]
+    for shp, plan in ((big, plan_big), (small, plan_small), (big, plan_big)):
+        ib, fb = synth.make_inputs(shp)
+        out = torch.full(shp.out_shape, float("nan"), dtype=torch.float32, device="cuda")
+        plan.forward(to_dev(ib), to_dev(fb), out)
+        plan.check()
+        exp, ab = ocnn.cnn_bf16(ib, fb, oshape(shp))
+        assert_close(out.cpu().numpy().astype(np.float64), exp, ab, what=shp.name)
+    plan_big.close()
+    plan_small.close()
