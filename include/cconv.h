@@ -151,7 +151,7 @@ int cconv_plan_info_get(const cconv_plan* plan, cconv_plan_info* info_out);
 void cconv_plan_destroy(cconv_plan* plan);
 
 /* Eq. 1 on device buffers (layouts above), asynchronous on `cuda_stream` (a cudaStream_t, may be
- * NULL for the default stream).  Launch errors are returned; device-side guards are read back by
+ * NULL for the default stream).  The plan's device must be the current device (else CCONV_EINVAL).  Launch errors are returned; device-side guards are read back by
  * cconv_plan_status. */
 int cconv_forward_planned(const cconv_plan* plan, const void* Image, const void* Filter, void* Out,
                           void* cuda_stream);

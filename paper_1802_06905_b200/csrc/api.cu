@@ -399,6 +399,8 @@ int cconv_forward_planned(const cconv_plan* pl, const void* Image, const void* F
                           void* cuda_stream) {
   if (!pl || !Image || !Filter || !Out) return CCONV_EINVAL;
   if (pl->device < 0) return CCONV_EINVAL;  // inspection-only plan
+  int cur = -1;
+  if (cudaGetDevice(&cur) != cudaSuccess || cur != pl->device) return CCONV_EINVAL;  // wrong current device
   if (!aligned16(Image) || !aligned16(Filter) || (reinterpret_cast<uintptr_t>(Out) & 31u))
     return CCONV_EINVAL;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
