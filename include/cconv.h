@@ -152,7 +152,8 @@ void cconv_plan_destroy(cconv_plan* plan);
 
 /* Eq. 1 on device buffers (layouts above), asynchronous on `cuda_stream` (a cudaStream_t, may be
  * NULL for the default stream).  The plan's device must be the current device (else CCONV_EINVAL).  Launch errors are returned; device-side guards are read back by
- * cconv_plan_status. */
+ * cconv_plan_status.  A forward call allocates nothing (plans allocate at creation), so it may be
+ * made while the stream is being captured into a CUDA graph. */
 int cconv_forward_planned(const cconv_plan* plan, const void* Image, const void* Filter, void* Out,
                           void* cuda_stream);
 

@@ -384,3 +384,43 @@ def test_two_plans_with_different_shared_memory_needs_stay_usable():
         assert_close(out.cpu().numpy().astype(np.float64), exp, ab, what=shp.name)
     plan_big.close()
     plan_small.close()
+
+
+def test_planned_forward_and_pooling_inside_a_cuda_graph():
+    """Plans allocate at creation only: a planned forward call (packing kernel + convolution,
+    programmatic dependent launch) and a pooling call can be captured into a CUDA graph and
+    replayed on new contents of the same buffers."""
+    from oracle import pool as opool
+    c = cs("graph_planned", 64, 32, 128, 12, 9, 3, 3)
+    ib, fb = synth.make_inputs(c)
+    img, flt = to_dev(ib), to_dev(fb)
+    out = torch.full(c.out_shape, float("nan"), device="cuda", dtype=torch.float32)
+    # pooling reads the same Image: (Wi, Hi, C, B) -> 2x2 stride-2 windows, channel reduction, 3 planes
+    pdims = (c.B, c.C, 3, (c.Wi - 2) // 2 + 1, (c.Hi - 2) // 2 + 1, 2, 2, 2, 2)
+    pshape = ocnn.Shape(*pdims)
+    pimg = img[:pshape.Wi, :pshape.Hi].contiguous()
+    pout = torch.full(pshape.out_shape, float("nan"), device="cuda", dtype=torch.float32)
+    plan = binding.Plan(*c.dims(), device=0, variant=binding.VARIANT_HALO, out_dtype=binding.OUT_F32)
+    plan.forward(img, flt, out)               # warm-up outside the capture
+    plan.check()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.graph(graph, stream=side):
+        plan.forward(img, flt, out)
+        binding.pool_forward(pimg, pout, *pdims, op=binding.POOL_MAX)
+    for seed in (81, 82):
+        ib2, fb2 = synth.make_inputs(ConvShape("graph_planned", *c.dims(), seed=seed))
+        img.copy_(to_dev(ib2))
+        flt.copy_(to_dev(fb2))
+        pimg.copy_(img[:pshape.Wi, :pshape.Hi])
+        out.fill_(float("nan"))
+        pout.fill_(float("nan"))
+        graph.replay()
+        torch.cuda.synchronize()
+        exp, ab = ocnn.cnn_bf16(ib2, fb2, oshape(c))
+        assert_close(out.cpu().numpy().astype(np.float64), exp, ab, what=f"graph replay, seed {seed}")
+        pexp, _ = opool.pool_bf16(to_bits(pimg), pshape, opool.MAX)
+        np.testing.assert_array_equal(pout.cpu().numpy().astype(np.float64), pexp)
+    plan.check()
+    plan.close()

@@ -87,3 +87,31 @@ def test_noalloc_rejects_what_it_cannot_hold_or_run():
     rc = lib.cconv_forward_noalloc(None, p, p, 32, 8, 16, 14, 14, 3, 3, 1, 1, binding.OUT_BF16, None, None)
     assert rc == binding.EINVAL
     torch.cuda.synchronize()
+
+
+def test_noalloc_inside_a_cuda_graph_capture_and_replay():
+    """The call is made while a stream is being captured (no allocation may happen there), then the
+    graph is replayed on new contents of the same buffers."""
+    c = ConvShape("na_graph", 32, 48, 136, 10, 8, 3, 3, seed=74)
+    ib, fb = synth.make_inputs(c)
+    img, flt = to_dev(ib), to_dev(fb)
+    out = torch.full(c.out_shape, float("nan"), device="cuda", dtype=torch.float32)
+    # first call on this device outside any capture (it looks up the scratch array's address)
+    binding.conv_forward_noalloc(img, flt, out, *c.dims(), out_dtype=binding.OUT_F32, sync=True)
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.graph(graph, stream=side):
+        binding.conv_forward_noalloc(img, flt, out, *c.dims(), out_dtype=binding.OUT_F32,
+                                     stream=torch.cuda.current_stream())
+    for seed in (75, 76):
+        ib2, fb2 = synth.make_inputs(ConvShape("na_graph", *c.dims(), seed=seed))
+        img.copy_(to_dev(ib2))
+        flt.copy_(to_dev(fb2))
+        out.fill_(float("nan"))
+        graph.replay()
+        torch.cuda.synchronize()
+        exp, ab = ocnn.cnn_bf16(ib2, fb2, oshape(c))
+        got = out.cpu().numpy().astype(np.float64)
+        assert not np.isnan(got).any()
+        assert np.all(np.abs(got - exp) <= TOL * ab), f"replay with seed {seed}: mismatch"
