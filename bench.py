@@ -188,7 +188,8 @@ def time_config(cfg, torch, binding, dev, steps, warmup, dist=None, sampler=None
 def time_repeats(cfg, torch, binding, dev, launches, repeats=5):
     """Per-configuration table: median over `repeats` of the CUDA-event time of `launches`
     back-to-back forward calls, L2-cold (rotating buffer sets larger than L2) and L2-warm (one
-    buffer set).  Returns (cold seconds per call, warm seconds per call, plan info)."""
+    buffer set), and L2-cold again with the calls captured once into a CUDA graph and replayed.
+    Returns (cold seconds per call, warm seconds per call, plan info, graph seconds per call)."""
     ib, fb = make_inputs(cfg)
     set_bytes = 2 * (cfg.image_words + cfg.filter_words + cfg.out_words)
     nsets = max(2, min(64, -(-int(1.5 * L2_BYTES) // set_bytes)))
@@ -215,10 +216,34 @@ def time_repeats(cfg, torch, binding, dev, launches, repeats=5):
             if rep:
                 times.append(e0.elapsed_time(e1) * 1e-3 / launches)
         result.append(float(np.median(times)))
+    # the same rotation captured once into a CUDA graph and replayed (no host work per call)
+    graph_s = None
+    try:
+        side = torch.cuda.Stream()
+        side.wait_stream(stream)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            cap = torch.cuda.current_stream().cuda_stream
+            for i in range(launches):
+                a, b, c = ptrs[i % nsets]
+                plan.forward_ptrs(a, b, c, cap)
+        g.replay()
+        torch.cuda.synchronize()
+        times = []
+        for rep in range(repeats):
+            e0.record(stream)
+            g.replay()
+            e1.record(stream)
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1) * 1e-3 / launches)
+        graph_s = float(np.median(times))
+        del g
+    except RuntimeError:
+        graph_s = None
     plan.check()
     info = plan.info()
     plan.close()
-    return result[0], result[1], info
+    return result[0], result[1], info, graph_s
 
 
 def time_pooling(torch, binding, dev, peaks, launches=50, repeats=5):
@@ -529,11 +554,12 @@ def main():
             for i, c in enumerate(CONFIGS):
                 # median of 5 repeats of >= 100 back-to-back calls (20 for the 0.3 ms shape)
                 n_i = 100 if c.flops < 1e11 else 20
-                cold, warm, info_i = time_repeats(c, torch, binding, dev, n_i)
+                cold, warm, info_i, graph_s = time_repeats(c, torch, binding, dev, n_i)
                 tr, lbb = applicable_roofline_seconds(c, info_i, peaks)
                 m_cta = binding.lower_bound(*c.dims(), info_i["M_words"])
                 rows.append({"workload": c.name, "variant": info_i["variant"],
                              "us_per_launch": cold * 1e6, "us_per_launch_l2_warm": warm * 1e6,
+                             "us_per_launch_cuda_graph": None if graph_s is None else graph_s * 1e6,
                              "t_write_out_us": 2.0 * c.out_words / (wgbs * 1e9) * 1e6,
                              "tflops": c.flops / cold / 1e12,
                              "tflops_vs_sustained_peak": c.flops / cold / 1e12 /
