@@ -424,3 +424,55 @@ def test_planned_forward_and_pooling_inside_a_cuda_graph():
         np.testing.assert_array_equal(pout.cpu().numpy().astype(np.float64), pexp)
     plan.check()
     plan.close()
+
+
+def test_mixed_plans_and_pooling_back_to_back_without_synchronisation():
+    """Sixty calls of five plans (three kernel variants) and a pooling kernel on one stream, in a
+    seeded random order, each with its own Filter and Out and no synchronisation in between: every
+    kernel may start while its predecessors are still running (programmatic dependent launch), and
+    every plan alternates its two scratch buffers.  All sixty results are checked afterwards."""
+    from oracle import pool as opool
+    rng = np.random.default_rng(1234)
+    shapes = [
+        (cs("mix_halo_3x3", 64, 32, 136, 9, 7, 3, 3), binding.VARIANT_HALO),
+        (cs("mix_halo_1x1", 32, 64, 64, 6, 5, 1, 1, 2, 2), binding.VARIANT_HALO),
+        (cs("mix_halo_big", 64, 64, 256, 14, 14, 3, 3), binding.VARIANT_HALO),   # several tiles per CTA
+        (cs("mix_stem", 64, 3, 64, 11, 9, 5, 5, 2, 2), binding.VARIANT_STEM),
+        (cs("mix_simt", 3, 5, 7, 6, 5, 3, 2), binding.VARIANT_SIMT),
+    ]
+    plans = [binding.Plan(*c.dims(), device=0, variant=v, out_dtype=binding.OUT_F32) for c, v in shapes]
+    images = [to_dev(synth.make_inputs(c)[0]) for c, _ in shapes]
+    pool_shape = ocnn.Shape(32, 4, 3, 5, 4, 3, 3, 2, 2)
+    pool_bits = synth.make_inputs(ConvShape("mix_pool", *pool_shape.args(), seed=99))[0]
+    pool_img = to_dev(pool_bits)
+    jobs = []
+    for n in range(60):
+        i = int(rng.integers(0, len(shapes) + 1))
+        if i == len(shapes):
+            out = torch.full(pool_shape.out_shape, float("nan"), device="cuda", dtype=torch.float32)
+            jobs.append(("pool", None, None, out))
+        else:
+            c = shapes[i][0]
+            fb = synth.make_inputs(ConvShape(c.name, *c.dims(), seed=7000 + n))[1]
+            out = torch.full(c.out_shape, float("nan"), device="cuda", dtype=torch.float32)
+            jobs.append((i, fb, to_dev(fb), out))
+    for kind, _, flt, out in jobs:                       # launch everything, no synchronisation
+        if kind == "pool":
+            binding.pool_forward(pool_img, out, *pool_shape.args(), op=binding.POOL_AVG)
+        else:
+            plans[kind].forward(images[kind], flt, out)
+    for pl in plans:
+        pl.check()
+    pexp, pab = opool.pool_bf16(pool_bits, pool_shape, opool.AVG)
+    cache = {}
+    for n, (kind, fb, _, out) in enumerate(jobs):
+        got = out.cpu().numpy().astype(np.float64)
+        if kind == "pool":
+            assert_close(got, pexp, pab, what=f"job {n}: pooling")
+            continue
+        c = shapes[kind][0]
+        ib = cache.setdefault(kind, synth.make_inputs(c)[0])
+        exp, ab = ocnn.cnn_bf16(ib, fb, oshape(c))
+        assert_close(got, exp, ab, what=f"job {n}: {c.name}")
+    for pl in plans:
+        pl.close()
