@@ -53,10 +53,14 @@ extern "C" {
 /* Kernel variants (cconv_plan_create's `variant`). */
 #define CCONV_VARIANT_AUTO 0
 #define CCONV_VARIANT_SIMT 1 /* CUDA-core kernel: any shape, any alignment                      */
-#define CCONV_VARIANT_HALO 2 /* TMA halo tiles -> tcgen05.mma -> TMEM; needs B % 8 == 0 (a batch
-                                block of 32 images is zero padded past B when B % 32 != 0)      */
-#define CCONV_VARIANT_STEM 3 /* small C: (s,c) folded into the MMA contraction; needs B % 8 == 0
-                                and the whole (shifted, padded) Filter resident in shared memory */
+#define CCONV_VARIANT_HALO 2 /* TMA halo tiles -> tcgen05.mma -> TMEM (a batch block of 32 images
+                                is zero padded past B when B % 32 != 0)                          */
+#define CCONV_VARIANT_STEM 3 /* small C: (s,c) folded into the MMA contraction; needs the whole
+                                (shifted, padded) Filter resident in shared memory               */
+/* The tensor-core kernels need B % 8 == 0.  For other batch sizes a plan runs them on copies of
+ * Image and Out padded to the next multiple of 8 (plan-owned scratch, one padding and one compaction
+ * kernel per call); AUTO does so unless the problem is tiny (then SIMT) or the scratch would exceed
+ * 4 GiB.  cconv_forward_noalloc, which owns no such scratch, still requires B % 8 == 0. */
 
 /* Element type of Out (cconv_plan_create's `out_dtype`). */
 #define CCONV_OUT_BF16 0

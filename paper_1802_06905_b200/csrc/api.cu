@@ -38,6 +38,39 @@ int env_int(const char* name, int dflt) {
 
 // Out of the most recent tensor-core convolution launched through a plan, and its stream (see
 // cconv_forward_planned).
+// rows x B  ->  rows x Bp (Bp >= B): copies the B real elements of every row and zero-fills the rest
+// (element size `es` bytes; used on the bf16 Image, 2 bytes)
+__global__ void __launch_bounds__(256) cconv_pad_batch_kernel(const unsigned short* __restrict__ src,
+                                                              unsigned short* __restrict__ dst,
+                                                              long long rows, int B, int Bp) {
+  const long long n = rows * Bp;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n;
+       i += (long long)gridDim.x * blockDim.x) {
+    const long long r = i / Bp;
+    const int b = int(i - r * Bp);
+    dst[i] = b < B ? src[r * B + b] : (unsigned short)0;
+  }
+}
+
+// rows x Bp  ->  rows x B: drops the padding images of every row (T = bf16 bits or fp32)
+template <typename T>
+__global__ void __launch_bounds__(256) cconv_compact_batch_kernel(const T* __restrict__ src,
+                                                                  T* __restrict__ dst, long long rows,
+                                                                  int B, int Bp) {
+  const long long n = rows * B;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n;
+       i += (long long)gridDim.x * blockDim.x) {
+    const long long r = i / B;
+    const int b = int(i - r * B);
+    dst[i] = src[r * Bp + b];
+  }
+}
+
+unsigned grid_for(long long n) {
+  const long long blocks = (n + 255) / 256;
+  return unsigned(std::max<long long>(1, std::min<long long>(blocks, 148ll * 32)));
+}
+
 struct LastOut {
   bool valid = false;
   void* stream = nullptr;
@@ -72,7 +105,15 @@ bool note_call_and_check_overlap(const Dims& d, int out_dtype, const void* Image
 
 struct cconv_plan {
   Dims d{};
-  ImageView view{};  // what the tensor-core kernels run: `d`, or its unstrided 1x1 equivalent
+  // What the tensor-core kernels run.  They need B % 8 == 0 (16-byte TMA strides, 16-byte pieces of
+  // Out): for any other batch size they run `drun` = `d` with B rounded up to a multiple of 8 on
+  // plan-owned zero-padded copies of Image and Out (`d_img_pad`, `d_out_pad`); a padding kernel in
+  // front and a compaction kernel behind move the real images in and out.
+  Dims drun{};
+  bool padded = false;
+  void* d_img_pad = nullptr;
+  void* d_out_pad = nullptr;
+  ImageView view{};  // `drun`, or its unstrided equivalent for 1x1 filters with strides
   int device = -1;
   int variant = CCONV_VARIANT_SIMT;
   int out_dtype = CCONV_OUT_BF16;
@@ -117,6 +158,47 @@ std::mutex g_cache_mu;
 std::map<std::tuple<int, int, int, int, int, int, int, int, int, int, int>, cconv_plan*> g_cache;
 
 }  // namespace
+
+// The tensor-core launches of one forward call (Image and Out already padded if need be).
+static int launch_tensor_core(const cconv_plan* pl, const void* Image, const void* Filter, void* Out,
+                              bool image_overlaps_last_out, cudaStream_t stream) {
+  CUtensorMap tmi, tmi_tail;
+  void* packed = nullptr;
+  {
+    // the tensor map is rebuilt only when the Image pointer changes
+    std::lock_guard<std::mutex> lk(pl->mu);
+    if (pl->tm_image_ptr != Image) {
+      int rc = pl->variant == CCONV_VARIANT_STEM
+                   ? encode_stem_image_map(pl->drun, pl->stile, Image, &pl->tm_image)
+                   : encode_image_map(pl->view, pl->tile, Image, &pl->tm_image);
+      if (rc == CCONV_OK && pl->has_tail)
+        rc = encode_image_map(pl->view, pl->tail, Image, &pl->tm_image_tail);
+      if (rc != CCONV_OK) return rc;
+      pl->tm_image_ptr = Image;
+    }
+    tmi = pl->tm_image;
+    if (pl->has_tail) tmi_tail = pl->tm_image_tail;
+    packed = static_cast<char*>(pl->d_packed) + (pl->calls++ & 1u) * pl->packed_bytes;
+  }
+  if (pl->variant == CCONV_VARIANT_STEM) {
+    cudaError_t es = launch_pack_filter_stem(Filter, packed, pl->d, pl->skp, stream);
+    if (es != cudaSuccess) return cuda_fail(es, "launch_pack_filter_stem");
+    es = launch_stem(tmi, packed, Out, pl->out_dtype == CCONV_OUT_F32, pl->skp, pl->stile.grid,
+                     pl->stile.smem_bytes, pl->d_status, stream);
+    return es == cudaSuccess ? CCONV_OK : cuda_fail(es, "launch_stem");
+  }
+  HaloKernelParams kp = pl->kp;
+  kp.image_wait = image_overlaps_last_out ? 1 : 0;
+  cudaError_t e = launch_pack_filter(Filter, packed, pl->d, pl->tile.c16, pl->tile.tiles_k,
+                                     /*overlap_prev=*/true, stream);
+  if (e != cudaSuccess) return cuda_fail(e, "launch_pack_filter");
+  e = launch_halo(tmi, packed, Out, pl->out_dtype == CCONV_OUT_F32, kp, pl->tile.grid,
+                  pl->tile.smem_bytes, pl->d_status, stream);
+  if (e == cudaSuccess && pl->has_tail)
+    e = launch_halo(tmi_tail, packed, Out, pl->out_dtype == CCONV_OUT_F32, pl->kp_tail,
+                    pl->tail.grid, pl->tail.smem_bytes, pl->d_status, stream);
+  return e == cudaSuccess ? CCONV_OK : cuda_fail(e, "launch_halo");
+}
 
 extern "C" {
 
@@ -195,7 +277,10 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
   cconv_plan* pl = new (std::nothrow) cconv_plan();
   if (!pl) return CCONV_ENOMEM;
   pl->d = d;
-  pl->view = image_view(d);
+  pl->drun = d;
+  pl->drun.B = (d.B + 7) / 8 * 8;
+  pl->padded = pl->drun.B != d.B;
+  pl->view = image_view(pl->drun);
   const Dims& dk = pl->view.dk;
   pl->device = device;
   pl->out_dtype = out_dtype;
@@ -227,7 +312,7 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
   if (variant == CCONV_VARIANT_AUTO && env_variant >= 1 && env_variant <= 3) variant = env_variant;
 
   const bool halo_ok = halo_supported(dk, nullptr) && choose_halo_tile(dk, pl->m, force, &pl->tile);
-  const bool stem_ok = choose_stem_tile(d, pl->m, &pl->stile, env_int("CCONV_STEM_BW", 0));
+  const bool stem_ok = choose_stem_tile(pl->drun, pl->m, &pl->stile, env_int("CCONV_STEM_BW", 0));
   if ((variant == CCONV_VARIANT_HALO && !halo_ok) || (variant == CCONV_VARIANT_STEM && !stem_ok)) {
     delete pl;
     return CCONV_EUNSUPPORTED;
@@ -237,6 +322,14 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
     // the kernel that folds (s, c) into the contraction wins where it applies.
     if (stem_ok && d.C < 8) variant = CCONV_VARIANT_STEM;
     else variant = halo_ok ? CCONV_VARIANT_HALO : CCONV_VARIANT_SIMT;
+    // A padded batch costs two more kernels (about 15 us per call in all, measured) and two scratch
+    // arrays: worth it unless the problem is tiny (the CUDA-core kernel needs 8 us for 0.5 M
+    // multiply-adds, 25-50 us for 7-15 M), and only within 4 GiB of scratch.
+    if (pl->padded && variant != CCONV_VARIANT_SIMT) {
+      const double scratch = 2.0 * pl->drun.Wi() * pl->drun.Hi() * d.C * pl->drun.B +
+                             double(d.K) * d.H * d.W * pl->drun.B * (out_dtype == CCONV_OUT_F32 ? 4 : 2);
+      if (d.macs() < 4.0e6 || scratch > 4.0 * 1024 * 1024 * 1024) variant = CCONV_VARIANT_SIMT;
+    }
   }
   pl->variant = variant;
   if (variant == CCONV_VARIANT_HALO) {
@@ -267,7 +360,7 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
     }
     build_halo_params(dk, pl->tile, &pl->kp);
   }
-  if (variant == CCONV_VARIANT_STEM) build_stem_params(pl->d, pl->stile, &pl->skp);
+  if (variant == CCONV_VARIANT_STEM) build_stem_params(pl->drun, pl->stile, &pl->skp);
 
   if (device >= 0) {
     int prev = 0;
@@ -282,6 +375,12 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
     pl->packed_bytes = (pl->packed_bytes + 255) & ~size_t(255);
     if (e == cudaSuccess && variant >= CCONV_VARIANT_HALO)
       e = cudaMalloc(&pl->d_packed, 2 * pl->packed_bytes);
+    if (e == cudaSuccess && variant >= CCONV_VARIANT_HALO && pl->padded) {
+      const Dims& r = pl->drun;
+      e = cudaMalloc(&pl->d_img_pad, size_t(r.Wi()) * r.Hi() * r.C * r.B * 2);
+      if (e == cudaSuccess)
+        e = cudaMalloc(&pl->d_out_pad, size_t(r.K) * r.H * r.W * r.B * (out_dtype == CCONV_OUT_F32 ? 4 : 2));
+    }
     if (e == cudaSuccess && variant == CCONV_VARIANT_STEM)
       e = stem_kernel_prepare(pl->stile.smem_bytes);
     if (e == cudaSuccess && variant >= CCONV_VARIANT_HALO && env_int("CCONV_TRACE", 0)) {
@@ -295,6 +394,8 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
     if (e != cudaSuccess) {
       if (pl->d_status) cudaFree(pl->d_status);
       if (pl->d_packed) cudaFree(pl->d_packed);
+      if (pl->d_img_pad) cudaFree(pl->d_img_pad);
+      if (pl->d_out_pad) cudaFree(pl->d_out_pad);
       delete pl;
       return cuda_fail(e, "plan device setup");
     }
@@ -387,6 +488,8 @@ void cconv_plan_destroy(cconv_plan* pl) {
     if (pl->d_status) cudaFree(pl->d_status);
     if (pl->d_packed) cudaFree(pl->d_packed);
     if (pl->d_trace) cudaFree(pl->d_trace);
+    if (pl->d_img_pad) cudaFree(pl->d_img_pad);
+    if (pl->d_out_pad) cudaFree(pl->d_out_pad);
     if (pl->st_image) cudaFree(pl->st_image);
     if (pl->st_filter) cudaFree(pl->st_filter);
     if (pl->st_out) cudaFree(pl->st_out);
@@ -410,42 +513,38 @@ int cconv_forward_planned(const cconv_plan* pl, const void* Image, const void* F
     cudaError_t e = launch_simt(Image, Filter, Out, pl->out_dtype == CCONV_OUT_F32, pl->d, stream);
     return e == cudaSuccess ? CCONV_OK : cuda_fail(e, "launch_simt");
   }
-  CUtensorMap tmi, tmi_tail;
-  void* packed = nullptr;
+  // Batch sizes that are not multiples of 8: the kernels run on zero-padded copies (see cconv_plan).
+  void* const user_out = Out;
+  if (pl->padded) {
+    const Dims& r = pl->drun;
+    const long long rows = (long long)r.Wi() * r.Hi() * r.C;
+    cconv_pad_batch_kernel<<<grid_for(rows * r.B), 256, 0, stream>>>(
+        static_cast<const unsigned short*>(Image), static_cast<unsigned short*>(pl->d_img_pad), rows,
+        pl->d.B, r.B);
+    cudaError_t ep = cudaGetLastError();
+    if (ep != cudaSuccess) return cuda_fail(ep, "cconv_pad_batch_kernel");
+    Image = pl->d_img_pad;
+    Out = pl->d_out_pad;
+  }
+  const int rc_run = launch_tensor_core(pl, Image, Filter, Out, image_overlaps_last_out, stream);
+  if (rc_run != CCONV_OK || !pl->padded) return rc_run;
   {
-    // the tensor map is rebuilt only when the Image pointer changes
-    std::lock_guard<std::mutex> lk(pl->mu);
-    if (pl->tm_image_ptr != Image) {
-      int rc = pl->variant == CCONV_VARIANT_STEM
-                   ? encode_stem_image_map(pl->d, pl->stile, Image, &pl->tm_image)
-                   : encode_image_map(pl->view, pl->tile, Image, &pl->tm_image);
-      if (rc == CCONV_OK && pl->has_tail)
-        rc = encode_image_map(pl->view, pl->tail, Image, &pl->tm_image_tail);
-      if (rc != CCONV_OK) return rc;
-      pl->tm_image_ptr = Image;
-    }
-    tmi = pl->tm_image;
-    if (pl->has_tail) tmi_tail = pl->tm_image_tail;
-    packed = static_cast<char*>(pl->d_packed) + (pl->calls++ & 1u) * pl->packed_bytes;
+    const Dims& r = pl->drun;
+    const long long rows = (long long)r.K * r.H * r.W;
+    if (pl->out_dtype == CCONV_OUT_F32)
+      cconv_compact_batch_kernel<float><<<grid_for(rows * pl->d.B), 256, 0, stream>>>(
+          static_cast<const float*>(Out), static_cast<float*>(user_out), rows, pl->d.B, r.B);
+    else
+      cconv_compact_batch_kernel<unsigned short><<<grid_for(rows * pl->d.B), 256, 0, stream>>>(
+          static_cast<const unsigned short*>(Out), static_cast<unsigned short*>(user_out), rows,
+          pl->d.B, r.B);
+    cudaError_t ec = cudaGetLastError();
+    if (ec != cudaSuccess) return cuda_fail(ec, "cconv_compact_batch_kernel");
+    // the compaction kernel is an ordinary launch: nothing behind it starts before it is complete
+    std::lock_guard<std::mutex> lk(g_last_out_mu);
+    g_last_out.valid = false;
   }
-  if (pl->variant == CCONV_VARIANT_STEM) {
-    cudaError_t es = launch_pack_filter_stem(Filter, packed, pl->d, pl->skp, stream);
-    if (es != cudaSuccess) return cuda_fail(es, "launch_pack_filter_stem");
-    es = launch_stem(tmi, packed, Out, pl->out_dtype == CCONV_OUT_F32, pl->skp, pl->stile.grid,
-                     pl->stile.smem_bytes, pl->d_status, stream);
-    return es == cudaSuccess ? CCONV_OK : cuda_fail(es, "launch_stem");
-  }
-  HaloKernelParams kp = pl->kp;
-  kp.image_wait = image_overlaps_last_out ? 1 : 0;
-  cudaError_t e = launch_pack_filter(Filter, packed, pl->d, pl->tile.c16, pl->tile.tiles_k,
-                                     /*overlap_prev=*/true, stream);
-  if (e != cudaSuccess) return cuda_fail(e, "launch_pack_filter");
-  e = launch_halo(tmi, packed, Out, pl->out_dtype == CCONV_OUT_F32, kp, pl->tile.grid,
-                  pl->tile.smem_bytes, pl->d_status, stream);
-  if (e == cudaSuccess && pl->has_tail)
-    e = launch_halo(tmi_tail, packed, Out, pl->out_dtype == CCONV_OUT_F32, pl->kp_tail,
-                    pl->tail.grid, pl->tail.smem_bytes, pl->d_status, stream);
-  return e == cudaSuccess ? CCONV_OK : cuda_fail(e, "launch_halo");
+  return CCONV_OK;
 }
 
 int cconv_forward(const void* Image, const void* Filter, void* Out, int B, int C, int K, int W,

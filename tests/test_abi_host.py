@@ -155,11 +155,11 @@ def test_plan_create_rejects_bad_arguments(lib):
     assert lib.cconv_plan_create(ctypes.byref(h), 2, 8, 8, 4, 4, 3, 3, 1, 1, -1, 0.0, 7, 0) == binding.EINVAL
     assert lib.cconv_plan_create(None, 2, 8, 8, 4, 4, 3, 3, 1, 1, -1, 0.0, 0, 0) == binding.EINVAL
     assert lib.cconv_plan_create(ctypes.byref(h), 2, 8, 8, 4, 4, 3, 3, 1, 1, -1, 0.0, 0, 5) == binding.EINVAL
-    # the tensor-core variant refuses shapes it cannot tile (B not a multiple of 8)
-    assert lib.cconv_plan_create(ctypes.byref(h), 2, 8, 16, 14, 14, 3, 3, 1, 1, -1, 0.0,
-                                 binding.VARIANT_HALO, 0) == binding.EUNSUPPORTED
-    assert lib.cconv_plan_create(ctypes.byref(h), 36, 8, 64, 12, 12, 3, 3, 1, 1, -1, 0.0,
-                                 binding.VARIANT_HALO, 0) == binding.EUNSUPPORTED
+    # B not a multiple of 8: the tensor-core variants run on a batch padded to the next multiple of 8
+    for B in (2, 36):
+        assert lib.cconv_plan_create(ctypes.byref(h), B, 8, 64, 12, 12, 3, 3, 1, 1, -1, 0.0,
+                                     binding.VARIANT_HALO, 0) == binding.OK
+        lib.cconv_plan_destroy(h)
     # B = 48: a multiple of 8 but not of 32 -> blocks of 32 images, the last one zero padded
     assert lib.cconv_plan_create(ctypes.byref(h), 48, 8, 64, 12, 12, 3, 3, 1, 1, -1, 0.0,
                                  binding.VARIANT_HALO, 0) == binding.OK
@@ -256,3 +256,17 @@ def test_theorem2_leaf_matches_the_oracle_and_the_benchmark_shapes():
     assert binding.theorem2_case(*CONFIGS[1].dims()[:7], M)[0] == "2.2.2.1"
     assert binding.theorem2_case(*CONFIGS[3].dims()[:7], M)[0] == "2.2.2.2"
     assert binding.theorem2_case(*CONFIGS[4].dims()[:7], M)[0] == "2.2.2.1"
+
+
+def test_auto_variant_for_batches_that_are_not_multiples_of_8():
+    """Small problems stay on the CUDA-core kernel (a padded batch costs two more kernels); large ones
+    take the tensor-core path on a padded batch."""
+    small = binding.Plan(2, 8, 16, 14, 14, 3, 3, 1, 1, device=-1)        # the tiny benchmark shape
+    assert small.info()["variant"] == binding.VARIANT_SIMT
+    small.close()
+    big = binding.Plan(1, 64, 64, 14, 14, 3, 3, 1, 1, device=-1)        # 7 M multiply-adds, one image
+    assert big.info()["variant"] == binding.VARIANT_HALO
+    big.close()
+    stem = binding.Plan(20, 3, 64, 56, 56, 7, 7, 2, 2, device=-1)
+    assert stem.info()["variant"] == binding.VARIANT_STEM
+    stem.close()

@@ -476,3 +476,34 @@ def test_mixed_plans_and_pooling_back_to_back_without_synchronisation():
         assert_close(got, exp, ab, what=f"job {n}: {c.name}")
     for pl in plans:
         pl.close()
+
+
+@pytest.mark.parametrize("out_dtype", DTYPES, ids=DT_IDS)
+@pytest.mark.parametrize("variant,c", [
+    (binding.VARIANT_HALO, cs("pad_b3", 3, 24, 72, 7, 6, 3, 3)),
+    (binding.VARIANT_HALO, cs("pad_b12_s2", 12, 16, 136, 9, 8, 3, 3, 2, 2)),
+    (binding.VARIANT_HALO, cs("pad_b100_1x1", 100, 32, 64, 5, 4, 1, 1)),
+    (binding.VARIANT_HALO, cs("pad_b1", 1, 64, 128, 14, 14, 3, 3)),
+    (binding.VARIANT_STEM, cs("pad_stem_b5", 5, 3, 64, 12, 11, 7, 7, 2, 2)),
+    (binding.VARIANT_STEM, cs("pad_stem_b70", 70, 4, 40, 8, 6, 3, 3)),
+], ids=lambda v: v.name if hasattr(v, "name") else str(v))
+def test_batches_that_are_not_multiples_of_8_on_the_tensor_core_kernels(variant, c, out_dtype):
+    info = check_full(c, variant=variant, out_dtype=out_dtype)
+    assert info["variant"] == variant
+
+
+def test_padded_batch_calls_back_to_back_with_changing_inputs():
+    c = cs("pad_b2b", 6, 32, 128, 10, 9, 3, 3)
+    plan = binding.Plan(*c.dims(), device=0, variant=binding.VARIANT_HALO, out_dtype=binding.OUT_F32)
+    jobs = []
+    for n in range(6):
+        ib, fb = synth.make_inputs(ConvShape(c.name, *c.dims(), seed=8100 + n))
+        out = torch.full(c.out_shape, float("nan"), device="cuda", dtype=torch.float32)
+        jobs.append((ib, fb, to_dev(ib), to_dev(fb), out))
+    for _, _, img, flt, out in jobs:
+        plan.forward(img, flt, out)
+    plan.check()
+    for n, (ib, fb, _, _, out) in enumerate(jobs):
+        exp, ab = ocnn.cnn_bf16(ib, fb, oshape(c))
+        assert_close(out.cpu().numpy().astype(np.float64), exp, ab, what=f"padded call {n}")
+    plan.close()
