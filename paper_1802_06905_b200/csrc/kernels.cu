@@ -333,11 +333,35 @@ __device__ __forceinline__ void mma_role(const HaloKernelParams& p, const MmaCtx
         }
       }
       for (; issued < n; ++issued) {
-        const uint64_t a_desc = (uint64_t(a_hi) << 32) | (a_lo0 | a16);
-        issue_unit<BH>(leader, bh, d_base, n_mma, a_desc, b_hi, b_lo0, img_kk16 + tap_off, hstep16,
-                       idesc, acc);
-        acc = 1;
-        a16 += kBlk16;
+        if constexpr (TAPS == 0 && (BH == 1 || BH == 2)) {
+          // other filter sizes: four taps of one filter column (s, s+1, s+2, s+3: one halo row
+          // apart) per straight-line block while the column and both stages last
+          if (sx + 4 <= S && issued + 4 <= n) {
+            if constexpr (BH == 1)
+              umma_run4_bh1(leader, d_base, a_lo0 | a16, a_hi, b_lo0 | (img_kk16 + tap_off), b_hi, idesc,
+                            acc, row16);
+            else
+              umma_run4_bh2(leader, d_base, a_lo0 | a16, a_hi, b_lo0 | (img_kk16 + tap_off), b_hi, idesc,
+                            acc, row16, hstep16, n_mma);
+            acc = 1;
+            a16 += 4u * kBlk16;
+            tap_off += 3u * row16;  // the common tail below adds the fourth step
+            sx += 3;
+            issued += 3;
+          } else {
+            const uint64_t a_desc = (uint64_t(a_hi) << 32) | (a_lo0 | a16);
+            issue_unit<BH>(leader, bh, d_base, n_mma, a_desc, b_hi, b_lo0, img_kk16 + tap_off, hstep16,
+                           idesc, acc);
+            acc = 1;
+            a16 += kBlk16;
+          }
+        } else {
+          const uint64_t a_desc = (uint64_t(a_hi) << 32) | (a_lo0 | a16);
+          issue_unit<BH>(leader, bh, d_base, n_mma, a_desc, b_hi, b_lo0, img_kk16 + tap_off, hstep16,
+                         idesc, acc);
+          acc = 1;
+          a16 += kBlk16;
+        }
         // next tap: one halo row down; after S rows, one pixel to the right; after R*S taps, the
         // next 16 channels of the same Image stage
         tap_off += row16;
@@ -787,12 +811,14 @@ HaloFn<OutT> halo_fn(int R, int S, int bh) {
   if (R * S == 1)
     return b == 1 ? cconv_halo_kernel<OutT, 1, 1> : b == 2 ? cconv_halo_kernel<OutT, 2, 1>
                                                            : cconv_halo_kernel<OutT, 0, 1>;
-  return cconv_halo_kernel<OutT, 0, 0>;
+  return b == 1 ? cconv_halo_kernel<OutT, 1, 0> : b == 2 ? cconv_halo_kernel<OutT, 2, 0>
+                                                         : cconv_halo_kernel<OutT, 0, 0>;
 }
 
 template <typename OutT>
 cudaError_t prepare_all(int smem_bytes) {
-  const int shapes[7][3] = {{3, 3, 1}, {3, 3, 2}, {3, 3, 3}, {1, 1, 1}, {1, 1, 2}, {1, 1, 3}, {5, 5, 1}};
+  const int shapes[9][3] = {{3, 3, 1}, {3, 3, 2}, {3, 3, 3}, {1, 1, 1}, {1, 1, 2},
+                            {1, 1, 3}, {5, 5, 1}, {5, 5, 2}, {5, 5, 3}};
   for (const auto& sh : shapes) {
     cudaError_t e = cudaFuncSetAttribute(halo_fn<OutT>(sh[0], sh[1], sh[2]),
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
