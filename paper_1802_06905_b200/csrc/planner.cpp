@@ -213,7 +213,8 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloT
   //    about 88 B/clk per SM in a micro-benchmark, so this constant stands for the whole
   //    producer/consumer pipeline, not for L2) -- it rewards tiles that fill all SMs;
   //  * one elected thread issues a unit (b_h MMAs) in about 130 + 60*b_h cycles at best with the
-  //    straight-line issue blocks (3x3 and 1x1 filters), 170 + 60*b_h with the generic tap loop;
+  //    straight-line issue blocks (3x3 and 1x1 filters), 170 + 60*b_h with the generic tap loop
+  //    (about 145 + 60*b_h where a filter column has four or more taps, which go out in blocks of four);
   //  * the epilogue drains an accumulator at about 14 cycles per TMEM column;
   //  * HBM: a call cannot end before its compulsory reads (about 3400 B/clk, the copy rate) and its
   //    Out writes (about 1900 B/clk with this epilogue's stores) have passed; on write-heavy 1x1
@@ -306,7 +307,7 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloT
                                         t.f_stages * t.filt_stage_bytes) + reserve, 117760);
             // ---- cycle model (per SM) ------------------------------------------------------
             const double exec = std::max(N / 2.0, (4096.0 + 32.0 * N) / 128.0);  // math vs operand reads
-            const double issue0 = (RS == 9 && d.R == 3) || RS == 1 ? 130.0 : 170.0;
+            const double issue0 = (RS == 9 && d.R == 3) || RS == 1 ? 130.0 : (d.S >= 4 ? 145.0 : 170.0);
             const double unit_clk = std::max(bh * exec, issue0 + 60.0 * bh);     // issue-rate floor
             // every stage of either ring costs the issuing thread a barrier wait and a commit
             const double stage_clk = 150.0;
