@@ -319,7 +319,8 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloT
             const double l2_rate = std::min(l2_sm_max_bytes_per_clk, l2_total_bytes_per_clk / t.grid);
             // 64-byte rows (bb = 32) use the copy engine and the swizzle half as well as 128-byte rows
             const double cyc_copy = tile_bytes / l2_rate * (bb == 32 ? 1.08 : 1.0);
-            const double cyc_epi = 14.0 * acc_cols;
+            // (64-byte runs of Out, b_b = 32, are absorbed more slowly than 128-byte runs)
+            const double cyc_epi = (bb == 32 ? 17.0 : 14.0) * acc_cols;
             // every asynchronous copy costs its issuing thread about 700 cycles whatever its
             // size, and a ring's stages are consumed in order: many small stages starve the MMAs
             const double cyc_issue_copies =
