@@ -334,6 +334,28 @@ __device__ __forceinline__ void mma_role(const HaloKernelParams& p, const MmaCtx
       }
       for (; issued < n; ++issued) {
         if constexpr (TAPS == 0 && (BH == 1 || BH == 2)) {
+          // R x 1 filters: four taps of the filter row (r .. r+3: one halo pixel apart)
+          if (S == 1 && tap_r + 4 <= R && issued + 4 <= n) {
+            if constexpr (BH == 1)
+              umma_run4_bh1(leader, d_base, a_lo0 | a16, a_hi, b_lo0 | (img_kk16 + tap_off), b_hi, idesc,
+                            acc, slab16);
+            else
+              umma_run4_bh2(leader, d_base, a_lo0 | a16, a_hi, b_lo0 | (img_kk16 + tap_off), b_hi, idesc,
+                            acc, slab16, hstep16, n_mma);
+            acc = 1;
+            a16 += 4u * kBlk16;
+            issued += 3;
+            tap_r += 4;
+            col_off += 4u * slab16;
+            tap_off = col_off;
+            if (tap_r == R) {
+              tap_r = 0;
+              col_off = 0;
+              tap_off = 0;
+              img_kk16 += kstep16;
+            }
+            continue;
+          }
           // other filter sizes: four taps of one filter column (s, s+1, s+2, s+3: one halo row
           // apart) per straight-line block while the column and both stages last
           if (sx + 4 <= S && issued + 4 <= n) {

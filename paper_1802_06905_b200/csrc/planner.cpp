@@ -307,7 +307,7 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloT
                                         t.f_stages * t.filt_stage_bytes) + reserve, 117760);
             // ---- cycle model (per SM) ------------------------------------------------------
             const double exec = std::max(N / 2.0, (4096.0 + 32.0 * N) / 128.0);  // math vs operand reads
-            const double issue0 = (RS == 9 && d.R == 3) || RS == 1 ? 130.0 : (d.S >= 4 ? 145.0 : 170.0);
+            const double issue0 = (RS == 9 && d.R == 3) || RS == 1 ? 130.0 : (d.S >= 4 || (d.S == 1 && d.R >= 4) ? 145.0 : 170.0);
             const double unit_clk = std::max(bh * exec, issue0 + 60.0 * bh);     // issue-rate floor
             // every stage of either ring costs the issuing thread a barrier wait and a commit
             const double stage_clk = 150.0;

@@ -507,3 +507,17 @@ def test_padded_batch_calls_back_to_back_with_changing_inputs():
         exp, ab = ocnn.cnn_bf16(ib, fb, oshape(c))
         assert_close(out.cpu().numpy().astype(np.float64), exp, ab, what=f"padded call {n}")
     plan.close()
+
+
+@pytest.mark.parametrize("out_dtype", DTYPES, ids=DT_IDS)
+@pytest.mark.parametrize("c", [
+    cs("taps_7x1", 32, 40, 136, 9, 8, 7, 1),            # R x 1: four-tap blocks along the filter row
+    cs("taps_9x1_bh2", 64, 16, 128, 12, 10, 9, 1),
+    cs("taps_1x7", 32, 24, 64, 8, 9, 1, 7),             # 1 x S: four-tap blocks along the filter column
+    cs("taps_5x5", 64, 32, 128, 9, 9, 5, 5),
+    cs("taps_6x4_s2", 32, 16, 72, 7, 6, 6, 4, 2, 2),
+    cs("taps_4x8", 32, 8, 64, 6, 5, 4, 8),
+], ids=lambda c: c.name)
+def test_filters_that_use_the_four_tap_issue_blocks(c, out_dtype):
+    info = check_full(c, variant=binding.VARIANT_HALO, out_dtype=out_dtype)
+    assert info["variant"] == binding.VARIANT_HALO
