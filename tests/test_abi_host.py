@@ -270,3 +270,46 @@ def test_auto_variant_for_batches_that_are_not_multiples_of_8():
     stem = binding.Plan(20, 3, 64, 56, 56, 7, 7, 2, 2, device=-1)
     assert stem.info()["variant"] == binding.VARIANT_STEM
     stem.close()
+
+
+def test_random_shapes_plan_to_hardware_legal_tiles():
+    """A thousand seeded random shapes (any batch size, filters up to 11x11, strides up to 4): every
+    plan for a nominal B200 obeys the limits of the SM, whichever variant AUTO picks."""
+    rng = np.random.default_rng(2718)
+    seen = {binding.VARIANT_SIMT: 0, binding.VARIANT_HALO: 0, binding.VARIANT_STEM: 0}
+    for _ in range(1000):
+        B = int(rng.choice([1, 2, 3, 8, 12, 16, 24, 32, 40, 64, 100, 128, 256]))
+        C = int(rng.choice([1, 3, 4, 7, 8, 16, 24, 48, 64, 100, 128, 256, 512, 1024]))
+        K = int(rng.choice([1, 8, 16, 40, 64, 100, 128, 200, 256, 512, 1000]))
+        W, H = (int(v) for v in rng.integers(1, 60, size=2))
+        R = int(rng.choice([1, 1, 2, 3, 3, 5, 7, 11]))
+        S = int(rng.choice([1, 3, R, R, 4]))
+        sw, sh = (int(v) for v in rng.choice([1, 1, 2, 3, 4], size=2))
+        p = binding.Plan(B, C, K, W, H, R, S, sw, sh, device=-1)
+        info = p.info()
+        p.close()
+        seen[info["variant"]] += 1
+        Bp = -(-B // 8) * 8                       # the batch the tensor-core kernels run
+        if info["variant"] == binding.VARIANT_HALO:
+            n = info["bb"] * info["bw"]
+            assert info["bb"] in (32, 64) and info["bc"] in (16, 32, 64, 128)
+            assert n % 16 == 0 and 16 <= n <= 256
+            assert n * info["bh"] <= 512 and info["tmem_cols"] in (32, 64, 128, 256, 512)
+            assert 117760 <= info["smem_bytes"] <= 232448
+            assert 1 <= info["stages"] <= 6 and 2 <= info["filter_stages"] <= 4
+            assert 1 <= info["halo_w"] <= 256 and 1 <= info["halo_h"] <= 256
+            img_stage = info["halo_w"] * info["halo_h"] * info["bc"] * info["bb"] * 2
+            assert info["stages"] * img_stage + info["filter_stages"] * 4096 <= info["smem_bytes"]
+            assert 1 <= info["grid"] <= 148 and info["tiles"] >= info["grid"]
+            assert info["bw"] <= max(W, 1) and info["bh"] <= max(H, 1)
+            if info["tail_h0"] < H:
+                assert 0 < info["tail_h0"] and 1 <= info["tail_tiles"] <= 148
+        elif info["variant"] == binding.VARIANT_STEM:
+            assert C < 8
+            assert 1 <= info["bw"] <= 4 and info["bk"] in (32, 64, 128) and info["bk"] * info["bh"] <= 128
+            assert 117760 <= info["smem_bytes"] <= 232448 and info["stages"] >= 2
+            assert info["tmem_cols"] == 512 and 1 <= info["grid"] <= 148
+        else:
+            # the CUDA-core kernel is left only with tiny problems whose batch is not a multiple of 8
+            assert B % 8 != 0 and B * C * K * W * H * R * S < 4e6 or Bp != B
+    assert all(v > 0 for v in seen.values()), seen
