@@ -90,9 +90,13 @@ void build_halo_params(const Dims& d, const HaloTile& t, HaloKernelParams* out) 
   // B = Image halo view [channels][n = (w, b)], MN-major; row = bb*2 bytes = the swizzle span
   // (layout type 2 = 128B swizzle, 4 = 64B).  SBO: from one group of 8 channels to the next;
   // LBO: from one pixel's bb images to the next pixel along w, sw halo pixels further.
+  // (layout type 6 = 32B swizzle for blocks of 16 images, 0 = none for blocks of 8: 16-byte rows)
   const uint32_t b_row = uint32_t(t.bb) * 2;
-  const uint32_t b_layout = b_row == 128 ? 2u : 4u;
-  p.b_desc = make_smem_desc(uint32_t(d.sw) * p.slab_bytes, 8 * b_row, b_layout);
+  const uint32_t b_layout = b_row == 128 ? 2u : b_row == 64 ? 4u : b_row == 32 ? 6u : 0u;
+  // (Without a swizzle the two offsets change roles: the stride field then steps along n, from
+  // pixel to pixel, and the leading field from one group of 8 channels to the next.)
+  p.b_desc = b_layout != 0u ? make_smem_desc(uint32_t(d.sw) * p.slab_bytes, 8 * b_row, b_layout)
+                            : make_smem_desc(8 * b_row, uint32_t(d.sw) * p.slab_bytes, 0u);
   p.wait_limit_ns = uint64_t(env_int("CCONV_WAIT_LIMIT_MS", 1000)) * 1000000ull;
   p.trace = nullptr;
 }
@@ -113,7 +117,10 @@ int encode_image_map(const ImageView& v, const HaloTile& t, const void* image, C
   const cuuint32_t box[4] = {cuuint32_t(t.bb), cuuint32_t(t.bc), cuuint32_t(t.halo_w),
                              cuuint32_t(t.halo_h)};
   const cuuint32_t es[4] = {1, 1, 1, 1};
-  const CUtensorMapSwizzle sw = t.bb == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
+  const CUtensorMapSwizzle sw = t.bb == 64   ? CU_TENSOR_MAP_SWIZZLE_128B
+                                : t.bb == 32 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                : t.bb == 16 ? CU_TENSOR_MAP_SWIZZLE_32B
+                                             : CU_TENSOR_MAP_SWIZZLE_NONE;
   CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(image),
                    dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);

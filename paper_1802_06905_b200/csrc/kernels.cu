@@ -490,7 +490,7 @@ __device__ __forceinline__ void store_run32(OutT* dst, const uint32_t (&v)[32]) 
 // ------------------------------------------------------------------------------------------------
 // BH, TAPS: the issuer's compile-time shape (see mma_role).  One kernel per shape: the issuing loop
 // is sensitive to the size of the code around it, so a launch carries only the loops it runs.
-template <typename OutT, int BH, int TAPS>
+template <typename OutT, int BH, int TAPS, bool SB>
 __global__ void __launch_bounds__(kThreads, 1)
     cconv_halo_kernel(const __grid_constant__ CUtensorMap tm_image,
                       const uint8_t* __restrict__ packed_filter, OutT* __restrict__ out,
@@ -673,6 +673,42 @@ __global__ void __launch_bounds__(kThreads, 1)
       tc_fence_after();
       if (first_tile && threadIdx.x == 64) CCONV_TRACE(8);
       const uint32_t t_base = tmem_base + (uint32_t(q * 32) << 16) + abuf * uint32_t(p.acc_cols);
+      if constexpr (SB) {
+        // batch blocks of 16 or 8 images: 32 accumulator columns hold 2 or 4 pixels
+        const int per = 32 / p.bb;  // pixels per 32 columns
+        for (int hh = 0; hh < p.bh; ++hh) {
+          const int h = p.h0 + ht * p.bh + hh;
+          for (int c0 = 0; c0 < p.n_mma; c0 += 32) {
+            uint32_t v[32];
+            tmem_ld_32x32b_x32(t_base + uint32_t(hh * p.n_mma + c0), v);
+            tmem_ld_wait();
+            const int ww0 = c0 / p.bb;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              if (j >= per) break;
+              const int w = wt * p.bw + ww0 + j;
+              if (!(k < p.K && h < p.H && w < p.W && ww0 + j < p.bw)) continue;
+              OutT* dst = out + (((long long)k * p.H + h) * p.W + w) * p.B + b0;
+              const int nb = p.B - b0;  // images inside the batch (a multiple of 8)
+              // the pixel's images are v[j*bb .. j*bb + bb): 8 (per = 4) or 16 (per = 2) values
+#pragma unroll
+              for (int g = 0; g < 2; ++g) {
+                const int first = (per == 4 ? j * 8 : j * 16 + g * 8);
+                if ((per == 4 && g == 1) || g * 8 >= nb) continue;
+                OutT* d8 = dst + g * 8;
+                if constexpr (sizeof(OutT) == 4) {
+                  *reinterpret_cast<uint4*>(d8) = make_uint4(v[first], v[first + 1], v[first + 2], v[first + 3]);
+                  *reinterpret_cast<uint4*>(d8 + 4) = make_uint4(v[first + 4], v[first + 5], v[first + 6], v[first + 7]);
+                } else {
+                  *reinterpret_cast<uint4*>(d8) =
+                      make_uint4(pack_bf16x2(v[first], v[first + 1]), pack_bf16x2(v[first + 2], v[first + 3]),
+                                 pack_bf16x2(v[first + 4], v[first + 5]), pack_bf16x2(v[first + 6], v[first + 7]));
+                }
+              }
+            }
+          }
+        }
+      } else
       for (int hh = 0; hh < p.bh; ++hh) {
         const int h = p.h0 + ht * p.bh + hh;
         for (int ww = 0; ww < p.bw; ++ww) {
@@ -824,17 +860,24 @@ namespace {
 template <typename OutT>
 using HaloFn = void (*)(CUtensorMap, const uint8_t*, OutT*, HaloKernelParams, int*);
 
-template <typename OutT>
-HaloFn<OutT> halo_fn(int R, int S, int bh) {
+template <typename OutT, bool SB>
+HaloFn<OutT> halo_fn_sb(int R, int S, int bh) {
   const int b = bh == 1 ? 1 : bh == 2 ? 2 : 0;
   if (R == 3 && S == 3)
-    return b == 1 ? cconv_halo_kernel<OutT, 1, 9> : b == 2 ? cconv_halo_kernel<OutT, 2, 9>
-                                                           : cconv_halo_kernel<OutT, 0, 9>;
+    return b == 1 ? cconv_halo_kernel<OutT, 1, 9, SB> : b == 2 ? cconv_halo_kernel<OutT, 2, 9, SB>
+                                                               : cconv_halo_kernel<OutT, 0, 9, SB>;
   if (R * S == 1)
-    return b == 1 ? cconv_halo_kernel<OutT, 1, 1> : b == 2 ? cconv_halo_kernel<OutT, 2, 1>
-                                                           : cconv_halo_kernel<OutT, 0, 1>;
-  return b == 1 ? cconv_halo_kernel<OutT, 1, 0> : b == 2 ? cconv_halo_kernel<OutT, 2, 0>
-                                                         : cconv_halo_kernel<OutT, 0, 0>;
+    return b == 1 ? cconv_halo_kernel<OutT, 1, 1, SB> : b == 2 ? cconv_halo_kernel<OutT, 2, 1, SB>
+                                                               : cconv_halo_kernel<OutT, 0, 1, SB>;
+  return b == 1 ? cconv_halo_kernel<OutT, 1, 0, SB> : b == 2 ? cconv_halo_kernel<OutT, 2, 0, SB>
+                                                             : cconv_halo_kernel<OutT, 0, 0, SB>;
+}
+
+// One kernel per issuer shape (b_h, filter size) and per batch-block class (32/64 images, or 8/16
+// with its own epilogue), so that no instantiation carries another one's code.
+template <typename OutT>
+HaloFn<OutT> halo_fn(int R, int S, int bh, int bb) {
+  return bb < 32 ? halo_fn_sb<OutT, true>(R, S, bh) : halo_fn_sb<OutT, false>(R, S, bh);
 }
 
 template <typename OutT>
@@ -842,9 +885,11 @@ cudaError_t prepare_all(int smem_bytes) {
   const int shapes[9][3] = {{3, 3, 1}, {3, 3, 2}, {3, 3, 3}, {1, 1, 1}, {1, 1, 2},
                             {1, 1, 3}, {5, 5, 1}, {5, 5, 2}, {5, 5, 3}};
   for (const auto& sh : shapes) {
-    cudaError_t e = cudaFuncSetAttribute(halo_fn<OutT>(sh[0], sh[1], sh[2]),
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
-    if (e != cudaSuccess) return e;
+    for (int bb : {64, 8}) {
+      cudaError_t e = cudaFuncSetAttribute(halo_fn<OutT>(sh[0], sh[1], sh[2], bb),
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+      if (e != cudaSuccess) return e;
+    }
   }
   return cudaSuccess;
 }
@@ -890,9 +935,9 @@ cudaError_t launch_halo(const CUtensorMap& tm_image, const void* packed_filter, 
     cfg.numAttrs = 2;
   }
   if (out_f32)
-    return cudaLaunchKernelEx(&cfg, halo_fn<float>(p.R, p.S, p.bh), tm_image, pf,
+    return cudaLaunchKernelEx(&cfg, halo_fn<float>(p.R, p.S, p.bh, p.bb), tm_image, pf,
                               static_cast<float*>(out), p, status);
-  return cudaLaunchKernelEx(&cfg, halo_fn<__nv_bfloat16>(p.R, p.S, p.bh), tm_image, pf,
+  return cudaLaunchKernelEx(&cfg, halo_fn<__nv_bfloat16>(p.R, p.S, p.bh, p.bb), tm_image, pf,
                             static_cast<__nv_bfloat16*>(out), p, status);
 }
 

@@ -292,7 +292,8 @@ def test_random_shapes_plan_to_hardware_legal_tiles():
         Bp = -(-B // 8) * 8                       # the batch the tensor-core kernels run
         if info["variant"] == binding.VARIANT_HALO:
             n = info["bb"] * info["bw"]
-            assert info["bb"] in (32, 64) and info["bc"] in (16, 32, 64, 128)
+            assert info["bb"] in (8, 16, 32, 64) and info["bc"] in (16, 32, 64, 128)
+            assert info["bb"] >= 32 or (Bp <= info["bb"] and n % 32 == 0)
             assert n % 16 == 0 and 16 <= n <= 256
             assert n * info["bh"] <= 512 and info["tmem_cols"] in (32, 64, 128, 256, 512)
             assert 117760 <= info["smem_bytes"] <= 232448
@@ -301,7 +302,7 @@ def test_random_shapes_plan_to_hardware_legal_tiles():
             img_stage = info["halo_w"] * info["halo_h"] * info["bc"] * info["bb"] * 2
             assert info["stages"] * img_stage + info["filter_stages"] * 4096 <= info["smem_bytes"]
             assert 1 <= info["grid"] <= 148 and info["tiles"] >= info["grid"]
-            assert info["bw"] <= max(W, 1) and info["bh"] <= max(H, 1)
+            assert info["bw"] <= max(W, 1) + 3 and info["bh"] <= max(H, 1)
             if info["tail_h0"] < H:
                 assert 0 < info["tail_h0"] and 1 <= info["tail_tiles"] <= 148
         elif info["variant"] == binding.VARIANT_STEM:

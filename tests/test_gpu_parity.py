@@ -174,9 +174,11 @@ def test_tail_is_planned_for_the_large_config():
     cs("b40_s2", 40, 16, 32, 7, 6, 3, 5, 2, 1),  # one full block + 8 images
     cs("b72", 72, 64, 128, 4, 9, 3, 3),         # two full blocks + 8 images
 ], ids=lambda c: c.name)
-def test_halo_batch_not_a_multiple_of_the_block(c, out_dtype):
-    """B % 8 == 0 but B % 32 != 0: the last batch block is zero padded by the TMA loads and its
-    stores stop at B; nothing beyond Out's end may be touched (guard bands in run_gpu)."""
+def test_halo_batch_not_a_multiple_of_the_block(monkeypatch, c, out_dtype):
+    """B % 8 == 0 but B % 32 != 0 with blocks of 32 images (forced where the planner would take a
+    block of 8): the last batch block is zero padded by the TMA loads and its stores stop at B;
+    nothing beyond Out's end may be touched (guard bands in run_gpu)."""
+    monkeypatch.setenv("CCONV_FORCE_TILE", "0,0,0,0,32")
     info = check_full(c, variant=binding.VARIANT_HALO, out_dtype=out_dtype)
     assert info["bb"] == 32 and c.B % 32 != 0
 
@@ -521,3 +523,32 @@ def test_padded_batch_calls_back_to_back_with_changing_inputs():
 def test_filters_that_use_the_four_tap_issue_blocks(c, out_dtype):
     info = check_full(c, variant=binding.VARIANT_HALO, out_dtype=out_dtype)
     assert info["variant"] == binding.VARIANT_HALO
+
+
+@pytest.mark.parametrize("out_dtype", DTYPES, ids=DT_IDS)
+@pytest.mark.parametrize("c", [
+    cs("sb_b8_3x3", 8, 32, 136, 13, 7, 3, 3),              # batch block of 8 images (16-byte rows)
+    cs("sb_b8_1x1_s2", 8, 64, 64, 9, 6, 1, 1, 2, 2),
+    cs("sb_b16_3x3", 16, 24, 200, 11, 9, 3, 3),            # batch block of 16 images (32-byte swizzle)
+    cs("sb_b16_5x5_s2", 16, 16, 64, 8, 8, 5, 5, 2, 2),
+    cs("sb_b1_3x3", 1, 48, 128, 30, 9, 3, 3),              # padded to 8: ragged w tile, two rows
+    cs("sb_b3_w2", 3, 16, 64, 2, 5, 3, 3),                 # output row narrower than a 4-pixel group
+    cs("sb_b12_3x3", 12, 32, 72, 10, 10, 3, 3),            # padded to 16
+    cs("sb_b8_many_tiles", 8, 32, 384, 40, 36, 3, 3),      # more tiles than SMs
+], ids=lambda c: c.name)
+def test_small_batch_blocks(c, out_dtype):
+    info = check_full(c, variant=binding.VARIANT_HALO, out_dtype=out_dtype)
+    assert info["variant"] == binding.VARIANT_HALO
+
+
+@pytest.mark.parametrize("out_dtype", DTYPES, ids=DT_IDS)
+@pytest.mark.parametrize("force,c", [
+    ("4,1,16,0,8", cs("sbf_b8_1x1_s2", 8, 64, 64, 9, 6, 1, 1, 2, 2)),      # forced blocks of 8 ...
+    ("8,2,16,0,8", cs("sbf_b5_5x2", 5, 16, 72, 10, 7, 5, 2)),
+    ("2,2,16,0,16", cs("sbf_b12_3x3", 12, 32, 72, 10, 10, 3, 3)),          # ... and of 16 images
+    ("16,1,32,0,16", cs("sbf_b16_1x1", 16, 96, 128, 20, 3, 1, 1)),
+], ids=lambda v: v.name if hasattr(v, "name") else str(v))
+def test_forced_small_batch_blocks(monkeypatch, force, c, out_dtype):
+    monkeypatch.setenv("CCONV_FORCE_TILE", force)
+    info = check_full(c, variant=binding.VARIANT_HALO, out_dtype=out_dtype)
+    assert info["bb"] == int(force.split(",")[4])
