@@ -54,7 +54,7 @@ extern "C" {
 #define CCONV_VARIANT_AUTO 0
 #define CCONV_VARIANT_SIMT 1 /* CUDA-core kernel: any shape, any alignment                      */
 #define CCONV_VARIANT_HALO 2 /* TMA halo tiles -> tcgen05.mma -> TMEM; batch blocks of 64 or 32
-                                images (the last one zero padded past B), of 16 or 8 for B <= 16  */
+                                images (the last one zero padded past B), or of 16 or 8 images     */
 #define CCONV_VARIANT_STEM 3 /* small C: (s,c) folded into the MMA contraction; needs the whole
                                 (shifted, padded) Filter resident in shared memory               */
 /* The tensor-core kernels need B % 8 == 0.  For other batch sizes a plan runs them on copies of

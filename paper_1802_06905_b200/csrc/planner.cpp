@@ -228,9 +228,10 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloT
   for (int bb : {64, 32, 16, 8}) {
     // a batch block that does not divide B is padded by the TMA's out-of-bounds zero fill; take
     // such a block only when no exact one exists.  Blocks of 16 and 8 images (32-byte and 16-byte
-    // rows in shared memory: slower copies, more pixels per MMA) are for batches that small.
+    // rows in shared memory: slower copies, more pixels per MMA) are for batches that small ...
     if (bb >= 32 && d.B % bb != 0 && !(bb == 32 && d.B % 32 != 0)) continue;
-    if (bb < 32 && (d.B > bb || (bb == 16 && d.B <= 8))) continue;
+    // (also for larger batches whose last block of 32 would be partly empty: B = 40 runs five blocks of 8)
+    if (bb < 32 && (d.B % bb != 0 || (d.B > bb && d.B % 32 == 0) || (bb == 16 && d.B <= 8))) continue;
     if (force[4] && bb != force[4]) continue;
     for (int bc : {128, 64, 32, 16}) {
       if (bc > c16 * 16 && bc != 16) continue;
@@ -324,9 +325,9 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloT
                 (double(t.cchunks) * double(img) + double(units) * 4096.0) / split;
             const double l2_rate = std::min(l2_sm_max_bytes_per_clk, l2_total_bytes_per_clk / t.grid);
             // 64-byte rows (bb = 32) use the copy engine and the swizzle half as well as 128-byte rows
-            const double cyc_copy = tile_bytes / l2_rate * (bb >= 64 ? 1.0 : bb == 32 ? 1.08 : bb == 16 ? 1.3 : 1.6);
+            const double cyc_copy = tile_bytes / l2_rate * (bb >= 64 ? 1.0 : bb == 32 ? 1.08 : bb == 16 ? 1.4 : 2.0);
             // (64-byte runs of Out, b_b = 32, are absorbed more slowly than 128-byte runs)
-            const double cyc_epi = (bb >= 64 ? 14.0 : bb == 32 ? 17.0 : 20.0) * acc_cols;
+            const double cyc_epi = (bb >= 64 ? 14.0 : bb == 32 ? 17.0 : bb == 16 ? 20.0 : 24.0) * acc_cols;
             // every asynchronous copy costs its issuing thread about 700 cycles whatever its
             // size, and a ring's stages are consumed in order: many small stages starve the MMAs
             const double cyc_issue_copies =

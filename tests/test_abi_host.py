@@ -293,7 +293,7 @@ def test_random_shapes_plan_to_hardware_legal_tiles():
         if info["variant"] == binding.VARIANT_HALO:
             n = info["bb"] * info["bw"]
             assert info["bb"] in (8, 16, 32, 64) and info["bc"] in (16, 32, 64, 128)
-            assert info["bb"] >= 32 or (Bp <= info["bb"] and n % 32 == 0)
+            assert info["bb"] >= 32 or (Bp % info["bb"] == 0 and n % 32 == 0)
             assert n % 16 == 0 and 16 <= n <= 256
             assert n * info["bh"] <= 512 and info["tmem_cols"] in (32, 64, 128, 256, 512)
             assert 117760 <= info["smem_bytes"] <= 232448
