@@ -59,8 +59,9 @@ extern "C" {
                                 (shifted, padded) Filter resident in shared memory               */
 /* The tensor-core kernels need B % 8 == 0.  For other batch sizes a plan runs them on copies of
  * Image and Out padded to the next multiple of 8 (plan-owned scratch, one padding and one compaction
- * kernel per call); AUTO does so unless the problem is tiny (then SIMT) or the scratch would exceed
- * 4 GiB.  cconv_forward_noalloc, which owns no such scratch, still requires B % 8 == 0. */
+ * kernel per call); for B < 8 the copies also turn bands of output rows into images, so that a
+ * single image fills a block of 8 with real work (see cconv_plan_info.bands).  AUTO does so unless
+ * the problem is tiny (then SIMT) or the scratch would exceed 4 GiB.  cconv_forward_noalloc, which owns no such scratch, still requires B % 8 == 0. */
 
 /* Element type of Out (cconv_plan_create's `out_dtype`). */
 #define CCONV_OUT_BF16 0
@@ -96,11 +97,16 @@ typedef struct {
   double compulsory_words; /* |Image| + |Filter| + |Out| with the real Image extent             */
   /* Wave-quantisation tail (HALO variant): when the main tiling would fill its last wave of CTAs
    * only partly, output rows h >= tail_h0 run as a second launch with the tile below, started
-   * while the first is in its last wave.  tail_h0 == H: no tail; `tiles` and `grid` above then
+   * while the first is in its last wave.  tail_h0 == run_H (= H unless B < 8): no tail; `tiles` and `grid` above then
    * describe the only launch, otherwise the main one. */
   int tail_h0, tail_bb, tail_bc, tail_bw, tail_bh, tail_tiles, tail_grid;
   double scratch_bytes;   /* one packed Filter; the plan owns two such device buffers and
                              alternates between them from call to call                          */
+  /* What the tensor-core kernels run when B % 8 != 0 (else B, H, 1): the batch rounded up to a
+   * multiple of 8 and, for B < 8, the output rows cut into `bands` bands of run_H rows, each band
+   * of each image taking the place of one image (run_B = 8-multiple >= B * bands).  The tile and the
+   * tail above (tail_h0 included) then describe that run. */
+  int run_B, run_H, bands;
 } cconv_plan_info;
 
 /* Theorem 1 (Section 4.1): the five lower-bound terms, in words, for a fast memory of M_words.

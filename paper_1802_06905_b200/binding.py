@@ -56,6 +56,7 @@ class PlanInfo(ctypes.Structure):
         ("tail_bw", ctypes.c_int), ("tail_bh", ctypes.c_int), ("tail_tiles", ctypes.c_int),
         ("tail_grid", ctypes.c_int),
         ("scratch_bytes", ctypes.c_double),
+        ("run_B", ctypes.c_int), ("run_H", ctypes.c_int), ("bands", ctypes.c_int),
     ]
 
     def asdict(self):

@@ -38,31 +38,54 @@ int env_int(const char* name, int dflt) {
 
 // Out of the most recent tensor-core convolution launched through a plan, and its stream (see
 // cconv_forward_planned).
-// rows x B  ->  rows x Bp (Bp >= B): copies the B real elements of every row and zero-fills the rest
-// (element size `es` bytes; used on the bf16 Image, 2 bytes)
-__global__ void __launch_bounds__(256) cconv_pad_batch_kernel(const unsigned short* __restrict__ src,
+// What a padded plan runs on (see cconv_plan): Image [Wi][Hi][C][B] -> [Wi][Hir][C][Bp], where image
+// b' = band * B + b of the copy holds the rows of image b that output rows band*Hr .. band*Hr+Hr-1
+// need (Hir = sh*(Hr-1)+S of them, starting at row band*Hr*sh); rows past Hi, bands past `bands`
+// and the images that round Bp up to a multiple of 8 are zero.  bands == 1: batch padding alone.
+struct BandGeom {
+  long long Wi, Hi, Hir, C;  // Image extents of the caller's problem and rows of the banded copy
+  int B, Bp, bands;
+  int Hr, sh;                // output rows per band, stride along h
+};
+
+__global__ void __launch_bounds__(256) cconv_pad_bands_kernel(const unsigned short* __restrict__ src,
                                                               unsigned short* __restrict__ dst,
-                                                              long long rows, int B, int Bp) {
-  const long long n = rows * Bp;
+                                                              BandGeom g) {
+  const long long n = g.Wi * g.Hir * g.C * g.Bp;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n;
        i += (long long)gridDim.x * blockDim.x) {
-    const long long r = i / Bp;
-    const int b = int(i - r * Bp);
-    dst[i] = b < B ? src[r * B + b] : (unsigned short)0;
+    long long t = i / g.Bp;
+    const int bp = int(i - t * g.Bp);
+    const long long c = t % g.C;
+    t /= g.C;
+    const long long yr = t % g.Hir;
+    const long long x = t / g.Hir;
+    const int band = bp / g.B, b = bp - band * g.B;
+    const long long y = (long long)band * g.Hr * g.sh + yr;
+    unsigned short v = 0;
+    if (band < g.bands && y < g.Hi) v = src[((x * g.Hi + y) * g.C + c) * g.B + b];
+    dst[i] = v;
   }
 }
 
-// rows x Bp  ->  rows x B: drops the padding images of every row (T = bf16 bits or fp32)
+// The way back: Out [K][H][W][B] of the caller from [K][Hr][W][Bp] of the banded run (T = bf16 bits
+// or fp32); output row h is row h % Hr of band h / Hr.
 template <typename T>
-__global__ void __launch_bounds__(256) cconv_compact_batch_kernel(const T* __restrict__ src,
-                                                                  T* __restrict__ dst, long long rows,
-                                                                  int B, int Bp) {
-  const long long n = rows * B;
+__global__ void __launch_bounds__(256) cconv_compact_bands_kernel(const T* __restrict__ src,
+                                                                  T* __restrict__ dst, long long K,
+                                                                  long long H, long long W,
+                                                                  BandGeom g) {
+  const long long n = K * H * W * g.B;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n;
        i += (long long)gridDim.x * blockDim.x) {
-    const long long r = i / B;
-    const int b = int(i - r * B);
-    dst[i] = src[r * Bp + b];
+    long long t = i / g.B;
+    const int b = int(i - t * g.B);
+    const long long w = t % W;
+    t /= W;
+    const long long h = t % H;
+    const long long k = t / H;
+    const long long band = h / g.Hr, hr = h - band * g.Hr;
+    dst[i] = src[((k * g.Hr + hr) * W + w) * g.Bp + band * g.B + b];
   }
 }
 
@@ -109,8 +132,13 @@ struct cconv_plan {
   // Out): for any other batch size they run `drun` = `d` with B rounded up to a multiple of 8 on
   // plan-owned zero-padded copies of Image and Out (`d_img_pad`, `d_out_pad`); a padding kernel in
   // front and a compaction kernel behind move the real images in and out.
+  // Fewer than 8 images: instead of padding with up to 7 zero images, the output rows are cut into
+  // `bands` bands of drun.H rows, and each band of each image becomes one image of `drun` (Eq. 1 has
+  // no dependence between output rows; a band only needs S - sh more Image rows than it owns, which
+  // the padding kernel copies twice).  One image then fills a block of 8 with real work.
   Dims drun{};
   bool padded = false;
+  int bands = 1;
   void* d_img_pad = nullptr;
   void* d_out_pad = nullptr;
   ImageView view{};  // `drun`, or its unstrided equivalent for 1x1 filters with strides
@@ -278,8 +306,15 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
   if (!pl) return CCONV_ENOMEM;
   pl->d = d;
   pl->drun = d;
-  pl->drun.B = (d.B + 7) / 8 * 8;
-  pl->padded = pl->drun.B != d.B;
+  if (d.B < 8) {
+    int want = env_int("CCONV_BANDS", 0);
+    if (want < 1) want = 8 / d.B;
+    want = std::max(1, std::min(want, d.H));
+    pl->drun.H = (d.H + want - 1) / want;
+    pl->bands = (d.H + pl->drun.H - 1) / pl->drun.H;  // no empty band
+  }
+  pl->drun.B = (d.B * pl->bands + 7) / 8 * 8;
+  pl->padded = pl->drun.B != d.B || pl->bands > 1;
   pl->view = image_view(pl->drun);
   const Dims& dk = pl->view.dk;
   pl->device = device;
@@ -327,7 +362,7 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
     // multiply-adds, 25-50 us for 7-15 M), and only within 4 GiB of scratch.
     if (pl->padded && variant != CCONV_VARIANT_SIMT) {
       const double scratch = 2.0 * pl->drun.Wi() * pl->drun.Hi() * d.C * pl->drun.B +
-                             double(d.K) * d.H * d.W * pl->drun.B * (out_dtype == CCONV_OUT_F32 ? 4 : 2);
+                             double(d.K) * pl->drun.H * d.W * pl->drun.B * (out_dtype == CCONV_OUT_F32 ? 4 : 2);
       if (d.macs() < 4.0e6 || scratch > 4.0 * 1024 * 1024 * 1024) variant = CCONV_VARIANT_SIMT;
     }
   }
@@ -443,7 +478,10 @@ int cconv_plan_info_get(const cconv_plan* pl, cconv_plan_info* o) {
   o->variant = pl->variant;
   o->out_dtype = pl->out_dtype;
   const Dims& d = pl->d;
-  o->tail_h0 = d.H;
+  o->tail_h0 = pl->view.dk.H;
+  o->run_B = pl->drun.B;
+  o->run_H = pl->drun.H;
+  o->bands = pl->bands;
   o->compulsory_words =
       double(d.Wi()) * d.Hi() * d.C * d.B + double(d.K) * d.R * d.S * d.C + double(d.K) * d.H * d.W * d.B;
   if (pl->variant == CCONV_VARIANT_STEM) {
@@ -470,10 +508,11 @@ int cconv_plan_info_get(const cconv_plan* pl, cconv_plan_info* o) {
       o->tail_tiles = int(u.tiles); o->tail_grid = u.grid;
       // rows kept by the main tiling: scale its staged words; then add the tail's (minus the Out
       // words both estimates include)
-      const double out_words = double(d.K) * d.H * d.W * d.B;
+      const Dims& r = pl->view.dk;  // what the kernels run
+      const double out_words = double(r.K) * r.H * r.W * r.B;
       o->tile_words_smem = double(t.tiles) * ((t.words_smem - out_words) /
-                                              (double(t.tiles) / t.tiles_h * ((d.H + t.bh - 1) / t.bh))) +
-                           (u.words_smem - double(d.K) * (d.H - pl->kp_tail.h0) * d.W * d.B) + out_words;
+                                              (double(t.tiles) / t.tiles_h * ((r.H + t.bh - 1) / t.bh))) +
+                           (u.words_smem - double(r.K) * (r.H - pl->kp_tail.h0) * r.W * r.B) + out_words;
     }
   }
   return CCONV_OK;
@@ -515,31 +554,31 @@ int cconv_forward_planned(const cconv_plan* pl, const void* Image, const void* F
   }
   // Batch sizes that are not multiples of 8: the kernels run on zero-padded copies (see cconv_plan).
   void* const user_out = Out;
+  BandGeom g{};
   if (pl->padded) {
     const Dims& r = pl->drun;
-    const long long rows = (long long)r.Wi() * r.Hi() * r.C;
-    cconv_pad_batch_kernel<<<grid_for(rows * r.B), 256, 0, stream>>>(
-        static_cast<const unsigned short*>(Image), static_cast<unsigned short*>(pl->d_img_pad), rows,
-        pl->d.B, r.B);
+    g = BandGeom{pl->d.Wi(), pl->d.Hi(), r.Hi(), pl->d.C, pl->d.B, r.B, pl->bands, r.H, pl->d.sh};
+    cconv_pad_bands_kernel<<<grid_for(g.Wi * g.Hir * g.C * g.Bp), 256, 0, stream>>>(
+        static_cast<const unsigned short*>(Image), static_cast<unsigned short*>(pl->d_img_pad), g);
     cudaError_t ep = cudaGetLastError();
-    if (ep != cudaSuccess) return cuda_fail(ep, "cconv_pad_batch_kernel");
+    if (ep != cudaSuccess) return cuda_fail(ep, "cconv_pad_bands_kernel");
     Image = pl->d_img_pad;
     Out = pl->d_out_pad;
   }
   const int rc_run = launch_tensor_core(pl, Image, Filter, Out, image_overlaps_last_out, stream);
   if (rc_run != CCONV_OK || !pl->padded) return rc_run;
   {
-    const Dims& r = pl->drun;
-    const long long rows = (long long)r.K * r.H * r.W;
+    const Dims& d = pl->d;
+    const unsigned grid = grid_for((long long)d.K * d.H * d.W * d.B);
     if (pl->out_dtype == CCONV_OUT_F32)
-      cconv_compact_batch_kernel<float><<<grid_for(rows * pl->d.B), 256, 0, stream>>>(
-          static_cast<const float*>(Out), static_cast<float*>(user_out), rows, pl->d.B, r.B);
+      cconv_compact_bands_kernel<float><<<grid, 256, 0, stream>>>(
+          static_cast<const float*>(Out), static_cast<float*>(user_out), d.K, d.H, d.W, g);
     else
-      cconv_compact_batch_kernel<unsigned short><<<grid_for(rows * pl->d.B), 256, 0, stream>>>(
-          static_cast<const unsigned short*>(Out), static_cast<unsigned short*>(user_out), rows,
-          pl->d.B, r.B);
+      cconv_compact_bands_kernel<unsigned short><<<grid, 256, 0, stream>>>(
+          static_cast<const unsigned short*>(Out), static_cast<unsigned short*>(user_out), d.K, d.H,
+          d.W, g);
     cudaError_t ec = cudaGetLastError();
-    if (ec != cudaSuccess) return cuda_fail(ec, "cconv_compact_batch_kernel");
+    if (ec != cudaSuccess) return cuda_fail(ec, "cconv_compact_bands_kernel");
     // the compaction kernel is an ordinary launch: nothing behind it starts before it is complete
     std::lock_guard<std::mutex> lk(g_last_out_mu);
     g_last_out.valid = false;

@@ -289,7 +289,10 @@ def test_random_shapes_plan_to_hardware_legal_tiles():
         info = p.info()
         p.close()
         seen[info["variant"]] += 1
-        Bp = -(-B // 8) * 8                       # the batch the tensor-core kernels run
+        Bp, Hrun = info["run_B"], info["run_H"]   # the batch and rows the tensor-core kernels run
+        assert Bp % 8 == 0 and Bp >= B * info["bands"] and Bp - B * info["bands"] < 8
+        assert info["bands"] * Hrun >= H > (info["bands"] - 1) * Hrun
+        assert (info["bands"] == 1 and Hrun == H) if B >= 8 else info["bands"] <= 8 // B
         if info["variant"] == binding.VARIANT_HALO:
             n = info["bb"] * info["bw"]
             assert info["bb"] in (8, 16, 32, 64) and info["bc"] in (16, 32, 64, 128)
@@ -302,8 +305,8 @@ def test_random_shapes_plan_to_hardware_legal_tiles():
             img_stage = info["halo_w"] * info["halo_h"] * info["bc"] * info["bb"] * 2
             assert info["stages"] * img_stage + info["filter_stages"] * 4096 <= info["smem_bytes"]
             assert 1 <= info["grid"] <= 148 and info["tiles"] >= info["grid"]
-            assert info["bw"] <= max(W, 1) + 3 and info["bh"] <= max(H, 1)
-            if info["tail_h0"] < H:
+            assert info["bw"] <= max(W, 1) + 3 and info["bh"] <= max(Hrun, 1)
+            if info["tail_h0"] < Hrun:
                 assert 0 < info["tail_h0"] and 1 <= info["tail_tiles"] <= 148
         elif info["variant"] == binding.VARIANT_STEM:
             assert C < 8

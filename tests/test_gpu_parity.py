@@ -552,3 +552,42 @@ def test_forced_small_batch_blocks(monkeypatch, force, c, out_dtype):
     monkeypatch.setenv("CCONV_FORCE_TILE", force)
     info = check_full(c, variant=binding.VARIANT_HALO, out_dtype=out_dtype)
     assert info["bb"] == int(force.split(",")[4])
+
+
+# ---- fewer than 8 images: bands of output rows take the place of images -----------------------------
+@pytest.mark.parametrize("out_dtype", DTYPES, ids=DT_IDS)
+@pytest.mark.parametrize("variant,c,bands", [
+    (binding.VARIANT_HALO, cs("bands_b1_3x3", 1, 40, 136, 11, 23, 3, 3), 8),        # 8 bands of 3 rows, last one ragged
+    (binding.VARIANT_HALO, cs("bands_b1_5x4_s2x3", 1, 16, 64, 9, 17, 5, 4, 2, 3), 6),  # strides; 17 rows = 6 bands of 3
+    (binding.VARIANT_HALO, cs("bands_b2_1x1_s2", 2, 64, 72, 7, 9, 1, 1, 2, 2), 3),  # strided 1x1 view of 3-row bands
+    (binding.VARIANT_HALO, cs("bands_b3", 3, 24, 128, 10, 8, 3, 3), 2),             # 2 bands x 3 images + 2 zero images
+    (binding.VARIANT_HALO, cs("bands_b4_h1", 4, 32, 64, 12, 1, 3, 3), 1),           # one output row: nothing to cut
+    (binding.VARIANT_HALO, cs("bands_b1_h5", 1, 32, 64, 6, 5, 3, 3), 5),            # fewer rows than bands wanted
+    (binding.VARIANT_HALO, cs("bands_b7", 7, 16, 64, 6, 6, 3, 3), 1),               # 7 images: one band, one zero image
+    (binding.VARIANT_STEM, cs("bands_stem_b1", 1, 3, 64, 20, 21, 7, 7, 2, 2), 7),   # 21 rows = 7 bands of 3
+    (binding.VARIANT_STEM, cs("bands_stem_b2", 2, 4, 40, 9, 10, 3, 3), 4),
+], ids=lambda v: v.name if hasattr(v, "name") else str(v))
+def test_bands_of_output_rows_stand_in_for_images_when_the_batch_is_below_8(variant, c, bands, out_dtype):
+    info = check_full(c, variant=variant, out_dtype=out_dtype)
+    assert info["variant"] == variant and info["bands"] == bands
+    assert info["run_H"] == -(-c.H // bands) and info["run_B"] == -(-c.B * bands // 8) * 8
+
+
+def test_banded_calls_back_to_back_with_changing_inputs():
+    """The banded copies are plan-owned scratch that every call overwrites: calls queued without
+    synchronisation must not see one another's."""
+    c = cs("bands_b2b", 1, 32, 128, 12, 19, 3, 3)
+    plan = binding.Plan(*c.dims(), device=0, variant=binding.VARIANT_AUTO, out_dtype=binding.OUT_BF16)
+    assert plan.info()["variant"] == binding.VARIANT_HALO and plan.info()["bands"] == 7
+    jobs = []
+    for n in range(5):
+        ib, fb = synth.make_inputs(ConvShape(c.name, *c.dims(), seed=8300 + n))
+        out = torch.full(c.out_shape, float("nan"), device="cuda", dtype=torch.bfloat16)
+        jobs.append((ib, fb, to_dev(ib), to_dev(fb), out))
+    for _, _, img, flt, out in jobs:
+        plan.forward(img, flt, out)
+    plan.check()
+    for n, (ib, fb, _, _, out) in enumerate(jobs):
+        exp, ab = ocnn.cnn_bf16(ib, fb, oshape(c))
+        assert_close(out.float().cpu().numpy().astype(np.float64), exp, ab, what=f"banded call {n}", bf16_out=True)
+    plan.close()
