@@ -167,6 +167,19 @@ void cconv_plan_destroy(cconv_plan* plan);
 int cconv_forward_planned(const cconv_plan* plan, const void* Image, const void* Filter, void* Out,
                           void* cuda_stream);
 
+/* Eq. 1 with its "+=" taken at its word on an Out that already holds values:
+ *   Out(k,h,w,b) <- Out(k,h,w,b) + sum_{c,r,s} Image(r+sw*w, s+sh*h, c, b) * Filter(k,r,s,c).
+ * cconv_plan_reserve_accumulate allocates, once per plan, what such calls need (an fp32 array of Out's
+ * shape and a twin of the plan that writes it; CCONV_ECUDA when the allocation fails) so that the
+ * calls themselves allocate nothing.  cconv_forward_accumulate runs the twin's kernels into that array
+ * and then one kernel that adds it to Out: the sum is formed in fp32 and rounded once to Out's type
+ * (bf16: round to nearest even).  Same pointers, alignment, stream and device rules as
+ * cconv_forward_planned; CCONV_EINVAL when the plan has not reserved.  Calls of one plan share the
+ * fp32 array: issue them on one stream, or order them yourself. */
+int cconv_plan_reserve_accumulate(cconv_plan* plan);
+int cconv_forward_accumulate(const cconv_plan* plan, const void* Image, const void* Filter, void* Out,
+                             void* cuda_stream);
+
 /* Convenience: plan (cached per shape, device and out_dtype; variant AUTO) and launch on the
  * current device. */
 int cconv_forward(const void* Image, const void* Filter, void* Out, int B, int C, int K, int W,

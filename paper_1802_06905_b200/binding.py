@@ -23,7 +23,8 @@ POOL_AVG, POOL_MAX = 0, 1
 
 EXPORTS = (
     "cconv_lower_bound", "cconv_tiling_lp", "cconv_plan_create", "cconv_plan_info_get",
-    "cconv_plan_destroy", "cconv_forward_planned", "cconv_forward", "cconv_forward_host",
+    "cconv_plan_destroy", "cconv_plan_reserve_accumulate", "cconv_forward_accumulate",
+    "cconv_forward_planned", "cconv_forward", "cconv_forward_host",
     "cconv_forward_noalloc", "cconv_pool_lower_bound", "cconv_pool_forward",
     "cconv_parallel_lower_bound", "cconv_parallel_partition", "cconv_theorem2_case",
     "cconv_plan_status", "cconv_plan_trace_read", "cconv_strerror", "cconv_last_cuda_error", "cconv_version",
@@ -96,6 +97,10 @@ def load_library():
     lib.cconv_plan_destroy.argtypes = [vp]
     lib.cconv_forward_planned.restype = i
     lib.cconv_forward_planned.argtypes = [vp, vp, vp, vp, vp]
+    lib.cconv_plan_reserve_accumulate.restype = i
+    lib.cconv_plan_reserve_accumulate.argtypes = [vp]
+    lib.cconv_forward_accumulate.restype = i
+    lib.cconv_forward_accumulate.argtypes = [vp, vp, vp, vp, vp]
     lib.cconv_forward.restype = i
     lib.cconv_forward.argtypes = [vp, vp, vp] + nine + [i, vp]
     lib.cconv_forward_noalloc.restype = i
@@ -251,6 +256,17 @@ class Plan:
         pi, pf, po = _tensor_args(image, filt, out, self.dims, self.out_dtype)
         _check(self._lib.cconv_forward_planned(self._h, pi, pf, po, _stream_ptr(stream)),
                "cconv_forward_planned")
+        return out
+
+    def reserve_accumulate(self):
+        """cconv_plan_reserve_accumulate: allocate what forward_accumulate needs (once per plan)."""
+        _check(self._lib.cconv_plan_reserve_accumulate(self._h), "cconv_plan_reserve_accumulate")
+
+    def forward_accumulate(self, image, filt, out, stream=None):
+        """cconv_forward_accumulate on torch CUDA tensors: out += Eq. 1; asynchronous on ``stream``."""
+        pi, pf, po = _tensor_args(image, filt, out, self.dims, self.out_dtype)
+        _check(self._lib.cconv_forward_accumulate(self._h, pi, pf, po, _stream_ptr(stream)),
+               "cconv_forward_accumulate")
         return out
 
     def forward_ptrs(self, image_ptr, filt_ptr, out_ptr, stream_ptr):

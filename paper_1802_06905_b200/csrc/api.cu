@@ -2,6 +2,7 @@
 // launches.  No compute happens on the host; there is no CPU fallback.
 #include <cuda.h>
 #include <cuda_runtime.h>
+#include <cuda_bf16.h>
 
 #include <algorithm>
 #include <cstdio>
@@ -89,6 +90,25 @@ __global__ void __launch_bounds__(256) cconv_compact_bands_kernel(const T* __res
   }
 }
 
+// Eq. 1's "+=" on an Out that already holds values: Out <- Out + Conv, Conv in fp32 from the plan's
+// fp32 twin, one rounding to Out's type
+template <typename T>
+__device__ __forceinline__ T add_round(T old, float conv);
+template <>
+__device__ __forceinline__ float add_round<float>(float old, float conv) { return old + conv; }
+template <>
+__device__ __forceinline__ __nv_bfloat16 add_round<__nv_bfloat16>(__nv_bfloat16 old, float conv) {
+  return __float2bfloat16_rn(__bfloat162float(old) + conv);
+}
+template <typename T>
+__global__ void __launch_bounds__(256) cconv_accumulate_kernel(T* __restrict__ out,
+                                                               const float* __restrict__ conv,
+                                                               long long n) {
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n;
+       i += (long long)gridDim.x * blockDim.x)
+    out[i] = add_round<T>(out[i], conv[i]);
+}
+
 unsigned grid_for(long long n) {
   const long long blocks = (n + 255) / 256;
   return unsigned(std::max<long long>(1, std::min<long long>(blocks, 148ll * 32)));
@@ -141,6 +161,9 @@ struct cconv_plan {
   int bands = 1;
   void* d_img_pad = nullptr;
   void* d_out_pad = nullptr;
+  // cconv_plan_reserve_accumulate: the same plan with fp32 Out and an fp32 array of Out's shape
+  cconv_plan* acc_twin = nullptr;
+  float* d_acc = nullptr;
   ImageView view{};  // `drun`, or its unstrided equivalent for 1x1 filters with strides
   int device = -1;
   int variant = CCONV_VARIANT_SIMT;
@@ -532,9 +555,57 @@ void cconv_plan_destroy(cconv_plan* pl) {
     if (pl->st_image) cudaFree(pl->st_image);
     if (pl->st_filter) cudaFree(pl->st_filter);
     if (pl->st_out) cudaFree(pl->st_out);
+    if (pl->d_acc) cudaFree(pl->d_acc);
     cudaSetDevice(prev);
   }
+  if (pl->acc_twin) cconv_plan_destroy(pl->acc_twin);
   delete pl;
+}
+
+int cconv_plan_reserve_accumulate(cconv_plan* pl) {
+  if (!pl || pl->device < 0) return CCONV_EINVAL;
+  if (pl->acc_twin) return CCONV_OK;
+  const Dims& d = pl->d;
+  cconv_plan* twin = nullptr;
+  const int rc = cconv_plan_create(&twin, d.B, d.C, d.K, d.W, d.H, d.R, d.S, d.sw, d.sh, pl->device,
+                                   pl->M_words, pl->variant, CCONV_OUT_F32);
+  if (rc != CCONV_OK) return rc;
+  int prev = 0;
+  cudaGetDevice(&prev);
+  cudaError_t e = cudaSetDevice(pl->device);
+  if (e == cudaSuccess)
+    e = cudaMalloc(reinterpret_cast<void**>(&pl->d_acc), size_t(d.K) * d.H * d.W * d.B * sizeof(float));
+  cudaSetDevice(prev);
+  if (e != cudaSuccess) {
+    cconv_plan_destroy(twin);
+    pl->d_acc = nullptr;
+    return cuda_fail(e, "cconv_plan_reserve_accumulate");
+  }
+  pl->acc_twin = twin;
+  return CCONV_OK;
+}
+
+int cconv_forward_accumulate(const cconv_plan* pl, const void* Image, const void* Filter, void* Out,
+                             void* cuda_stream) {
+  if (!pl || !Image || !Filter || !Out) return CCONV_EINVAL;
+  if (!pl->acc_twin || !pl->d_acc) return CCONV_EINVAL;  // not reserved
+  if (reinterpret_cast<uintptr_t>(Out) & 31u) return CCONV_EINVAL;
+  const int rc = cconv_forward_planned(pl->acc_twin, Image, Filter, pl->d_acc, cuda_stream);
+  if (rc != CCONV_OK) return rc;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const Dims& d = pl->d;
+  const long long n = (long long)d.K * d.H * d.W * d.B;
+  if (pl->out_dtype == CCONV_OUT_F32)
+    cconv_accumulate_kernel<float><<<grid_for(n), 256, 0, stream>>>(static_cast<float*>(Out), pl->d_acc, n);
+  else
+    cconv_accumulate_kernel<__nv_bfloat16><<<grid_for(n), 256, 0, stream>>>(
+        static_cast<__nv_bfloat16*>(Out), pl->d_acc, n);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e, "cconv_accumulate_kernel");
+  // an ordinary launch: nothing behind it starts before it is complete
+  std::lock_guard<std::mutex> lk(g_last_out_mu);
+  g_last_out.valid = false;
+  return CCONV_OK;
 }
 
 int cconv_forward_planned(const cconv_plan* pl, const void* Image, const void* Filter, void* Out,
@@ -643,13 +714,18 @@ int cconv_plan_status(const cconv_plan* pl, void* cuda_stream, int* detail_out) 
   int st = 0;
   CCONV_CUDA(cudaMemcpyAsync(&st, pl->d_status, sizeof(int), cudaMemcpyDeviceToHost, stream));
   CCONV_CUDA(cudaStreamSynchronize(stream));
-  if (detail_out) *detail_out = st;
   if (st != 0) {
     CCONV_CUDA(cudaMemsetAsync(pl->d_status, 0, sizeof(int), stream));
     CCONV_CUDA(cudaStreamSynchronize(stream));
-    return CCONV_EDEVICE_TIMEOUT;
   }
-  return CCONV_OK;
+  if (pl->acc_twin) {  // the accumulating calls run on the twin
+    int st2 = 0;
+    const int rc2 = cconv_plan_status(pl->acc_twin, cuda_stream, &st2);
+    if (rc2 != CCONV_OK && rc2 != CCONV_EDEVICE_TIMEOUT) return rc2;
+    st |= st2;
+  }
+  if (detail_out) *detail_out = st;
+  return st != 0 ? CCONV_EDEVICE_TIMEOUT : CCONV_OK;
 }
 
 }  // extern "C"

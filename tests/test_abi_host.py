@@ -146,6 +146,9 @@ def test_inspection_plans_are_hardware_legal():
             assert info["variant"] == binding.VARIANT_SIMT
         # forward on an inspection plan is refused on the host, before any launch
         assert p._lib.cconv_forward_planned(p._h, 16, 16, 16, None) == binding.EINVAL
+        # ... and so are reserving for, and making, accumulating calls
+        assert p._lib.cconv_plan_reserve_accumulate(p._h) == binding.EINVAL
+        assert p._lib.cconv_forward_accumulate(p._h, 32, 32, 32, None) == binding.EINVAL
         p.close()
 
 

@@ -591,3 +591,44 @@ def test_banded_calls_back_to_back_with_changing_inputs():
         exp, ab = ocnn.cnn_bf16(ib, fb, oshape(c))
         assert_close(out.float().cpu().numpy().astype(np.float64), exp, ab, what=f"banded call {n}", bf16_out=True)
     plan.close()
+
+
+# ---- Eq. 1's "+=" on an Out that already holds values ----------------------------------------------
+@pytest.mark.parametrize("out_dtype", DTYPES, ids=DT_IDS)
+@pytest.mark.parametrize("variant,c", [
+    (binding.VARIANT_SIMT, cs("acc_simt", 3, 5, 7, 6, 5, 3, 2)),
+    (binding.VARIANT_HALO, cs("acc_halo", 32, 40, 136, 9, 8, 3, 3)),
+    (binding.VARIANT_HALO, cs("acc_halo_1x1_s2", 64, 64, 72, 7, 6, 1, 1, 2, 2)),
+    (binding.VARIANT_HALO, cs("acc_halo_bands", 1, 32, 64, 10, 13, 3, 3)),
+    (binding.VARIANT_STEM, cs("acc_stem", 64, 3, 64, 12, 11, 7, 7, 2, 2)),
+], ids=lambda v: v.name if hasattr(v, "name") else str(v))
+def test_accumulate_adds_the_convolution_to_what_out_holds(variant, c, out_dtype):
+    """Out0 + Conv against Out0 + oracle, twice in a row (Out0 + 2 Conv); the tolerance scales with
+    |Out0| + sum|Image*Filter|, and the stored bf16 value may be the rounding of any value inside it."""
+    f32 = out_dtype == binding.OUT_F32
+    ib, fb = synth.make_inputs(c)
+    rng = np.random.default_rng(4400 + c.B)
+    out0 = torch.from_numpy(rng.normal(0.0, 3.0, size=c.out_shape).astype(np.float32))
+    out = out0.cuda() if f32 else out0.to(torch.bfloat16).cuda()
+    start = out.float().cpu().numpy().astype(np.float64)
+    plan = binding.Plan(*c.dims(), device=0, variant=variant, out_dtype=out_dtype)
+    with pytest.raises(binding.CconvError):
+        plan.forward_accumulate(to_dev(ib), to_dev(fb), out)          # nothing reserved yet
+    plan.reserve_accumulate()
+    plan.reserve_accumulate()                                          # a second call changes nothing
+    img, flt = to_dev(ib), to_dev(fb)
+    exp, ab = ocnn.cnn_bf16(ib, fb, oshape(c))
+    plan.forward_accumulate(img, flt, out)
+    plan.check()
+    once = out.float().cpu().numpy().astype(np.float64)
+    assert_close(once, start + exp, np.abs(start) + ab, what=f"{c.name}: Out0 + Conv", bf16_out=not f32)
+    plan.forward_accumulate(img, flt, out)
+    plan.check()
+    twice = out.float().cpu().numpy().astype(np.float64)
+    assert_close(twice, once + exp, np.abs(once) + ab, what=f"{c.name}: second call", bf16_out=not f32)
+    # the plain call still overwrites
+    plan.forward(img, flt, out)
+    plan.check()
+    assert_close(out.float().cpu().numpy().astype(np.float64), exp, ab, what=f"{c.name}: plain",
+                 bf16_out=not f32)
+    plan.close()
