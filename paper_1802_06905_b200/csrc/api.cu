@@ -49,44 +49,65 @@ struct BandGeom {
   int Hr, sh;                // output rows per band, stride along h
 };
 
+// (one thread per 16 bytes of the copy: 8 images of one (x, y, c))
 __global__ void __launch_bounds__(256) cconv_pad_bands_kernel(const unsigned short* __restrict__ src,
-                                                              unsigned short* __restrict__ dst,
-                                                              BandGeom g) {
-  const long long n = g.Wi * g.Hir * g.C * g.Bp;
+                                                              uint4* __restrict__ dst, BandGeom g) {
+  const int gpb = g.Bp / 8;
+  const long long n = g.Wi * g.Hir * g.C * gpb;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n;
        i += (long long)gridDim.x * blockDim.x) {
-    long long t = i / g.Bp;
-    const int bp = int(i - t * g.Bp);
+    long long t = i / gpb;
+    const int grp = int(i - t * gpb);
     const long long c = t % g.C;
     t /= g.C;
     const long long yr = t % g.Hir;
     const long long x = t / g.Hir;
-    const int band = bp / g.B, b = bp - band * g.B;
-    const long long y = (long long)band * g.Hr * g.sh + yr;
-    unsigned short v = 0;
-    if (band < g.bands && y < g.Hi) v = src[((x * g.Hi + y) * g.C + c) * g.B + b];
-    dst[i] = v;
+    uint32_t e[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int bp = grp * 8 + j;
+      const int band = bp / g.B, b = bp - band * g.B;
+      const long long y = (long long)band * g.Hr * g.sh + yr;
+      e[j] = (band < g.bands && y < g.Hi) ? uint32_t(src[((x * g.Hi + y) * g.C + c) * g.B + b]) : 0u;
+    }
+    dst[i] = make_uint4(e[0] | (e[1] << 16), e[2] | (e[3] << 16), e[4] | (e[5] << 16),
+                        e[6] | (e[7] << 16));
   }
 }
 
 // The way back: Out [K][H][W][B] of the caller from [K][Hr][W][Bp] of the banded run (T = bf16 bits
-// or fp32); output row h is row h % Hr of band h / Hr.
+// or fp32); output row h is row h % Hr of band h / Hr.  One thread per 8 images of the banded Out:
+// consecutive threads hold consecutive w, so that the stores of one band run along an output row.
 template <typename T>
 __global__ void __launch_bounds__(256) cconv_compact_bands_kernel(const T* __restrict__ src,
                                                                   T* __restrict__ dst, long long K,
                                                                   long long H, long long W,
                                                                   BandGeom g) {
-  const long long n = K * H * W * g.B;
+  const int gpb = g.Bp / 8;
+  const long long n = K * g.Hr * W * gpb;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n;
        i += (long long)gridDim.x * blockDim.x) {
-    long long t = i / g.B;
-    const int b = int(i - t * g.B);
+    const int grp = int(i % gpb);
+    long long t = i / gpb;
     const long long w = t % W;
     t /= W;
-    const long long h = t % H;
-    const long long k = t / H;
-    const long long band = h / g.Hr, hr = h - band * g.Hr;
-    dst[i] = src[((k * g.Hr + hr) * W + w) * g.Bp + band * g.B + b];
+    const long long hr = t % g.Hr;
+    const long long k = t / g.Hr;
+    T v[8];
+    const T* s8 = src + ((k * g.Hr + hr) * W + w) * g.Bp + grp * 8;
+    if constexpr (sizeof(T) == 2) {
+      *reinterpret_cast<uint4*>(v) = *reinterpret_cast<const uint4*>(s8);
+    } else {
+      *reinterpret_cast<uint4*>(v) = *reinterpret_cast<const uint4*>(s8);
+      *reinterpret_cast<uint4*>(v + 4) = *reinterpret_cast<const uint4*>(s8 + 4);
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int bp = grp * 8 + j;
+      const int band = bp / g.B, b = bp - band * g.B;
+      const long long h = (long long)band * g.Hr + hr;
+      if (band < g.bands && h < H) dst[((k * H + h) * W + w) * g.B + b] = v[j];
+    }
   }
 }
 
@@ -629,8 +650,8 @@ int cconv_forward_planned(const cconv_plan* pl, const void* Image, const void* F
   if (pl->padded) {
     const Dims& r = pl->drun;
     g = BandGeom{pl->d.Wi(), pl->d.Hi(), r.Hi(), pl->d.C, pl->d.B, r.B, pl->bands, r.H, pl->d.sh};
-    cconv_pad_bands_kernel<<<grid_for(g.Wi * g.Hir * g.C * g.Bp), 256, 0, stream>>>(
-        static_cast<const unsigned short*>(Image), static_cast<unsigned short*>(pl->d_img_pad), g);
+    cconv_pad_bands_kernel<<<grid_for(g.Wi * g.Hir * g.C * (g.Bp / 8)), 256, 0, stream>>>(
+        static_cast<const unsigned short*>(Image), static_cast<uint4*>(pl->d_img_pad), g);
     cudaError_t ep = cudaGetLastError();
     if (ep != cudaSuccess) return cuda_fail(ep, "cconv_pad_bands_kernel");
     Image = pl->d_img_pad;
@@ -640,7 +661,7 @@ int cconv_forward_planned(const cconv_plan* pl, const void* Image, const void* F
   if (rc_run != CCONV_OK || !pl->padded) return rc_run;
   {
     const Dims& d = pl->d;
-    const unsigned grid = grid_for((long long)d.K * d.H * d.W * d.B);
+    const unsigned grid = grid_for((long long)d.K * g.Hr * d.W * (g.Bp / 8));
     if (pl->out_dtype == CCONV_OUT_F32)
       cconv_compact_bands_kernel<float><<<grid, 256, 0, stream>>>(
           static_cast<const float*>(Out), static_cast<float*>(user_out), d.K, d.H, d.W, g);
