@@ -107,6 +107,11 @@ typedef struct {
    * of each image taking the place of one image (run_B = 8-multiple >= B * bands).  The tile and the
    * tail above (tail_h0 included) then describe that run. */
   int run_B, run_H, bands;
+  /* HALO variant: 2 when every tile is shared by the two CTAs of a cluster, half of the channels
+   * each, partial sums exchanged through distributed shared memory (grid = 2 * tiles; the planner
+   * does so for 9-tap-or-longer filters with long channel loops whose tiles would leave half of the
+   * SMs idle), else 1. */
+  int split;
 } cconv_plan_info;
 
 /* Theorem 1 (Section 4.1): the five lower-bound terms, in words, for a fast memory of M_words.

@@ -58,6 +58,7 @@ class PlanInfo(ctypes.Structure):
         ("tail_grid", ctypes.c_int),
         ("scratch_bytes", ctypes.c_double),
         ("run_B", ctypes.c_int), ("run_H", ctypes.c_int), ("bands", ctypes.c_int),
+        ("split", ctypes.c_int),
     ]
 
     def asdict(self):

@@ -526,6 +526,7 @@ int cconv_plan_info_get(const cconv_plan* pl, cconv_plan_info* o) {
   o->run_B = pl->drun.B;
   o->run_H = pl->drun.H;
   o->bands = pl->bands;
+  o->split = pl->variant == CCONV_VARIANT_HALO ? pl->tile.split : 1;
   o->compulsory_words =
       double(d.Wi()) * d.Hi() * d.C * d.B + double(d.K) * d.R * d.S * d.C + double(d.K) * d.H * d.W * d.B;
   if (pl->variant == CCONV_VARIANT_STEM) {

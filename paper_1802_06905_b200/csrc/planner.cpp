@@ -245,9 +245,9 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloT
         if (bb < 32 && N % 32 != 0) continue;
         for (int bh = 1; bh <= d.H && N * bh <= m.tmem_cols; ++bh) {
           if (force[1] && bh != force[1]) continue;
-          // split = 2 (two CTAs per tile, half of the channels each) is built and tested, but the
-          // exchange of partial sums costs more than the shorter main loop saves on every shape
-          // measured so far, so the planner takes it only on request (force[5] == 2).
+          // split = 2 (two CTAs per tile, half of the channels each): the exchange of partial sums
+          // costs more than the shorter main loop saves wherever whole tiles fill the SMs, so this
+          // loop searches it only on request (force[5] == 2); see the end of the function.
           for (int split = 1; split <= 2; ++split) {
             if (split != (force[5] == 2 ? 2 : 1)) continue;
             HaloTile t;
@@ -260,6 +260,8 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloT
             t.split = split;
             // halves must be whole Image stages of whole 16-channel chunks, and whole 32-column groups
             if (split == 2 && (c16 % (2 * (bc / 16)) != 0 || (N * bh / 2) % 32 != 0)) continue;
+            // (the kernels for batch blocks of 8 and 16 images have no exchange of partial sums)
+            if (split == 2 && bb < 32) continue;
             // about nine units per Filter stage, a whole number of Image stages where those are
             // shorter (1x1 filters), so that stage boundaries of the two rings coincide
             const int upi = (bc / 16) * RS;
@@ -370,6 +372,24 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloT
           }
         }
       }
+    }
+  }
+  // Split tiles (two CTAs of a cluster take half of the channels each and exchange partial sums on
+  // chip) are searched on request, and for problems that leave at least half of the SMs idle while
+  // every CTA streams a long Filter slab: filters of 9 or more taps with at least 144 units per tile
+  // (C*R*S >= 2304).  Measured on 41 such shapes (B 8..32, C and K 128..2048, 4x4 to 14x14 outputs):
+  // where the model puts the split tile at 0.70 of the whole tile's time or below, and the split
+  // tile does not at most double the accumulator columns computed (a wider batch block on a small
+  // batch is mostly zero padding), the call takes 0.61-0.89 of the time; 1x1 filters and shorter
+  // slabs gain nothing or lose up to 30 %.
+  if (found && force[5] == 0 && !force[0] && !force[1] && !force[2] && !force[3] && !force[4] &&
+      2 * best.tiles <= m.sm_count && RS >= 9 && units >= 144) {
+    const int want_split[6] = {0, 0, 0, 0, 0, 2};
+    HaloTile sp;
+    if (choose_halo_tile(d, m, want_split, &sp)) {
+      const double cols_whole = double(best.tiles) * best.bb * best.bw * best.bh;
+      const double cols_split = double(sp.tiles) * sp.bb * sp.bw * sp.bh;
+      if (sp.est_cycles <= 0.70 * best.est_cycles && cols_split <= 2.0 * cols_whole) best = sp;
     }
   }
   if (found) *out = best;

@@ -632,3 +632,18 @@ def test_accumulate_adds_the_convolution_to_what_out_holds(variant, c, out_dtype
     assert_close(out.float().cpu().numpy().astype(np.float64), exp, ab, what=f"{c.name}: plain",
                  bf16_out=not f32)
     plan.close()
+
+
+# ---- split tiles chosen by the planner: small grids, long channel loops ------------------------------
+@pytest.mark.parametrize("out_dtype", DTYPES, ids=DT_IDS)
+@pytest.mark.parametrize("c", [
+    cs("autosplit_b16_3x3", 16, 256, 256, 7, 7, 3, 3),           # 28 whole tiles -> 56 tiles x 2 CTAs
+    cs("autosplit_b32_5x5", 32, 128, 200, 5, 4, 5, 5),           # K padded to 256, ragged w tile
+    cs("autosplit_b64_3x3", 64, 256, 128, 6, 5, 3, 3),           # blocks of 64 images, one pixel per tile
+    cs("autosplit_b24_s2", 24, 512, 64, 5, 4, 3, 3, 2, 1),       # B % 32 != 0, strides
+    cs("autosplit_b40_4x4", 40, 160, 136, 4, 4, 4, 4),           # C = 160: ten 16-channel chunks, five per CTA
+], ids=lambda c: c.name)
+def test_planner_splits_channels_over_cta_pairs_on_small_grids(c, out_dtype):
+    info = check_full(c, variant=binding.VARIANT_AUTO, out_dtype=out_dtype)
+    assert info["variant"] == binding.VARIANT_HALO and info["split"] == 2
+    assert info["grid"] == 2 * info["tiles"] and info["bb"] >= 32

@@ -43,6 +43,7 @@ def test_noalloc_matches_planned_entry_point_twice_in_a_row(out_dtype):
     # word in the shared array
     shapes = [ConvShape("na1", 64, 40, 200, 9, 7, 3, 3, seed=71),
               ConvShape("na2", 32, 256, 256, 14, 14, 3, 3, seed=72),
+              ConvShape("na_split", 16, 256, 256, 7, 7, 3, 3, seed=74),   # tiles shared by CTA pairs
               ConvShape("na1_again", 64, 40, 200, 9, 7, 3, 3, seed=73)]
     for c in shapes:
         ib, fb = synth.make_inputs(c)
