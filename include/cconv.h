@@ -109,7 +109,7 @@ typedef struct {
   int run_B, run_H, bands;
   /* HALO variant: 2 when every tile is shared by the two CTAs of a cluster, half of the channels
    * each, partial sums exchanged through distributed shared memory (grid = 2 * tiles; the planner
-   * does so for 9-tap-or-longer filters with long channel loops whose tiles would leave half of the
+   * does so for filters of 9 or more taps with long channel loops whose tiles would leave half of the
    * SMs idle), else 1. */
   int split;
 } cconv_plan_info;

@@ -819,16 +819,47 @@ __global__ void __launch_bounds__(kThreads, 1)
           v[4 * c + 2] = __float_as_uint(__uint_as_float(v[4 * c + 2]) + __uint_as_float(a2));
           v[4 * c + 3] = __float_as_uint(__uint_as_float(v[4 * c + 3]) + __uint_as_float(a3));
         }
-        // column -> (output row, pixel, 32 images)
-        const int col = col0 + g;
-        const int hh = col / p.n_mma, rem = col - hh * p.n_mma;
-        const int ww = rem / p.bb, ch = (rem - ww * p.bb) >> 5;
-        const int h = p.h0 + ht * p.bh + hh, w = wt * p.bw + ww;
-        if (k < p.K && h < p.H && w < p.W) {
-          OutT* dst = out + (((long long)k * p.H + h) * p.W + w) * p.B + bt * p.bb + ch * 32;
-          const int nb = p.B - (bt * p.bb + ch * 32);
-          if (nb >= 32 && wide_rows) store_run32(dst, v);
-          else if (nb > 0) store_run_partial(dst, v, nb < 32 ? nb : 32);
+        if constexpr (SB) {
+          // column -> (output row, 2 or 4 pixels, 16 or 8 images each), as in the epilogue above
+          const int col = col0 + g;
+          const int hh = col / p.n_mma, rem = col - hh * p.n_mma;
+          const int h = p.h0 + ht * p.bh + hh;
+          const int per = 32 / p.bb;
+          const int ww0 = rem / p.bb;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            if (j >= per) break;
+            const int w = wt * p.bw + ww0 + j;
+            if (!(k < p.K && h < p.H && w < p.W && ww0 + j < p.bw)) continue;
+            OutT* dst = out + (((long long)k * p.H + h) * p.W + w) * p.B + bt * p.bb;
+            const int nb = p.B - bt * p.bb;
+#pragma unroll
+            for (int g8 = 0; g8 < 2; ++g8) {
+              const int first = (per == 4 ? j * 8 : j * 16 + g8 * 8);
+              if ((per == 4 && g8 == 1) || g8 * 8 >= nb) continue;
+              OutT* d8 = dst + g8 * 8;
+              if constexpr (sizeof(OutT) == 4) {
+                *reinterpret_cast<uint4*>(d8) = make_uint4(v[first], v[first + 1], v[first + 2], v[first + 3]);
+                *reinterpret_cast<uint4*>(d8 + 4) = make_uint4(v[first + 4], v[first + 5], v[first + 6], v[first + 7]);
+              } else {
+                *reinterpret_cast<uint4*>(d8) =
+                    make_uint4(pack_bf16x2(v[first], v[first + 1]), pack_bf16x2(v[first + 2], v[first + 3]),
+                               pack_bf16x2(v[first + 4], v[first + 5]), pack_bf16x2(v[first + 6], v[first + 7]));
+              }
+            }
+          }
+        } else {
+          // column -> (output row, pixel, 32 images)
+          const int col = col0 + g;
+          const int hh = col / p.n_mma, rem = col - hh * p.n_mma;
+          const int ww = rem / p.bb, ch = (rem - ww * p.bb) >> 5;
+          const int h = p.h0 + ht * p.bh + hh, w = wt * p.bw + ww;
+          if (k < p.K && h < p.H && w < p.W) {
+            OutT* dst = out + (((long long)k * p.H + h) * p.W + w) * p.B + bt * p.bb + ch * 32;
+            const int nb = p.B - (bt * p.bb + ch * 32);
+            if (nb >= 32 && wide_rows) store_run32(dst, v);
+            else if (nb > 0) store_run_partial(dst, v, nb < 32 ? nb : 32);
+          }
         }
       }
     }

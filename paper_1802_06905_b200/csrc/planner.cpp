@@ -260,8 +260,6 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloT
             t.split = split;
             // halves must be whole Image stages of whole 16-channel chunks, and whole 32-column groups
             if (split == 2 && (c16 % (2 * (bc / 16)) != 0 || (N * bh / 2) % 32 != 0)) continue;
-            // (the kernels for batch blocks of 8 and 16 images have no exchange of partial sums)
-            if (split == 2 && bb < 32) continue;
             // about nine units per Filter stage, a whole number of Image stages where those are
             // shorter (1x1 filters), so that stage boundaries of the two rings coincide
             const int upi = (bc / 16) * RS;
@@ -379,8 +377,9 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloT
   // every CTA streams a long Filter slab: filters of 9 or more taps with at least 144 units per tile
   // (C*R*S >= 2304).  Measured on 41 such shapes (B 8..32, C and K 128..2048, 4x4 to 14x14 outputs):
   // where the model puts the split tile at 0.70 of the whole tile's time or below, and the split
-  // tile does not at most double the accumulator columns computed (a wider batch block on a small
-  // batch is mostly zero padding), the call takes 0.61-0.89 of the time; 1x1 filters and shorter
+  // tile at most doubles the accumulator columns computed (a wider batch block on a small batch is
+  // mostly zero padding; up to four times the columns where four times as many CTAs then work),
+  // the call takes 0.61-0.89 of the time; 1x1 filters and shorter
   // slabs gain nothing or lose up to 30 %.
   if (found && force[5] == 0 && !force[0] && !force[1] && !force[2] && !force[3] && !force[4] &&
       2 * best.tiles <= m.sm_count && RS >= 9 && units >= 144) {
@@ -389,7 +388,9 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloT
     if (choose_halo_tile(d, m, want_split, &sp)) {
       const double cols_whole = double(best.tiles) * best.bb * best.bw * best.bh;
       const double cols_split = double(sp.tiles) * sp.bb * sp.bw * sp.bh;
-      if (sp.est_cycles <= 0.70 * best.est_cycles && cols_split <= 2.0 * cols_whole) best = sp;
+      const bool cols_ok = cols_split <= 2.0 * cols_whole ||
+                           (cols_split <= 4.0 * cols_whole && sp.grid >= 4 * best.grid);
+      if (sp.est_cycles <= 0.70 * best.est_cycles && cols_ok) best = sp;
     }
   }
   if (found) *out = best;

@@ -642,8 +642,12 @@ def test_accumulate_adds_the_convolution_to_what_out_holds(variant, c, out_dtype
     cs("autosplit_b64_3x3", 64, 256, 128, 6, 5, 3, 3),           # blocks of 64 images, one pixel per tile
     cs("autosplit_b24_s2", 24, 512, 64, 5, 4, 3, 3, 2, 1),       # B % 32 != 0, strides
     cs("autosplit_b40_4x4", 40, 160, 136, 4, 4, 4, 4),           # C = 160: ten 16-channel chunks, five per CTA
+    cs("autosplit_b8_blocks_of_8", 8, 512, 512, 7, 7, 3, 3),     # batch blocks of 8 images: 4 pixels per 32 columns
+    cs("autosplit_b16_blocks_of_16", 16, 256, 136, 7, 6, 5, 5),  # ... of 16 images: 2 pixels per 32 columns
 ], ids=lambda c: c.name)
 def test_planner_splits_channels_over_cta_pairs_on_small_grids(c, out_dtype):
     info = check_full(c, variant=binding.VARIANT_AUTO, out_dtype=out_dtype)
     assert info["variant"] == binding.VARIANT_HALO and info["split"] == 2
-    assert info["grid"] == 2 * info["tiles"] and info["bb"] >= 32
+    assert info["grid"] == 2 * info["tiles"]
+    if "blocks_of" in c.name:
+        assert info["bb"] == int(c.name.rsplit("_", 1)[1])
