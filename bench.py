@@ -326,9 +326,23 @@ def time_e2e(cfg, torch, binding, dev, steps):
         plan.forward_host(hi, hf, ho, stream)
     e1.record(stream)
     torch.cuda.synchronize()
+    secs_sync = e0.elapsed_time(e1) * 1e-3
+    # the same steps through the pipelined entry point: every step still copies its Image and Filter
+    # in and its Out back, but the copies of neighbouring steps overlap (two staging sets, a copy
+    # stream per direction); the wait for the last Out is inside the timed region
+    for _ in range(3):
+        plan.forward_host_async(hi, hf, ho, stream)
+    plan.host_wait(stream)
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for _ in range(steps):
+        plan.forward_host_async(hi, hf, ho, stream)
+    plan.host_wait(stream)
+    e1.record(stream)
+    torch.cuda.synchronize()
     secs = e0.elapsed_time(e1) * 1e-3
     plan.close()
-    return secs, 2 * (cfg.image_words + cfg.filter_words), 2 * cfg.out_words
+    return secs, 2 * (cfg.image_words + cfg.filter_words), 2 * cfg.out_words, secs_sync
 
 
 def kernels_per_step(info, binding):
@@ -543,10 +557,15 @@ def main():
 
     if rank == 0 and not args.no_extras:
         e_steps = max(5, min(50, steps))
-        e_secs, h2d, d2h = time_e2e(cfg, torch, binding, dev, e_steps)
+        e_secs, h2d, d2h, e_sync = time_e2e(cfg, torch, binding, dev, e_steps)
         line["e2e"] = {"value": cfg.flops * e_steps / e_secs / 1e12, "unit": "TFLOP/s",
                        "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                       "ms_per_step": e_secs / e_steps * 1e3, "steps": e_steps}
+                       "ms_per_step": e_secs / e_steps * 1e3, "steps": e_steps,
+                       "call": "cconv_forward_host_async per step + one cconv_host_wait (copies of "
+                               "neighbouring steps overlap)",
+                       "one_call_at_a_time": {"call": "cconv_forward_host (waits every step)",
+                                              "value": cfg.flops * e_steps / e_sync / 1e12,
+                                              "ms_per_step": e_sync / e_steps * 1e3}}
         if world == 1:
             wgbs = write_only_gbs(torch, dev)
             line["applicable_roofline"]["write_only_stream_gbs"] = wgbs

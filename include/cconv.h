@@ -196,6 +196,19 @@ int cconv_forward(const void* Image, const void* Filter, void* Out, int B, int C
 int cconv_forward_host(cconv_plan* plan, const void* hImage, const void* hFilter, void* hOut,
                        void* cuda_stream);
 
+/* The same without the wait, for a loop of calls: cconv_forward_host_async returns once the work is
+ * queued -- the copy of Image and Filter (pinned host memory, else the copies are not asynchronous)
+ * on a copy stream of the plan, the kernels on `cuda_stream`, the copy of Out back on a second copy
+ * stream -- with two sets of plan-owned staging arrays (allocated on first use), so that one call's
+ * copies in either direction overlap the neighbouring calls' kernels and copies in the other
+ * direction.  Calls of one plan must come from one host thread at a time and use one `cuda_stream`.
+ * The host buffers of a call must stay untouched, and hOut is not valid, until cconv_host_wait has
+ * returned: it waits for every queued call of the plan and returns the device status like
+ * cconv_forward_host.  The plan's device must be current. */
+int cconv_forward_host_async(cconv_plan* plan, const void* hImage, const void* hFilter, void* hOut,
+                             void* cuda_stream);
+int cconv_host_wait(cconv_plan* plan, void* cuda_stream);
+
 /* Scratch held by cconv_forward_noalloc, in bytes (the repacked Filter must fit):
  * ceil(K/128) * ceil(C/16) * R*S * 4096 <= this. */
 #define CCONV_NOALLOC_MAX_SCRATCH_BYTES (8u * 1024u * 1024u)

@@ -25,6 +25,7 @@ EXPORTS = (
     "cconv_lower_bound", "cconv_tiling_lp", "cconv_plan_create", "cconv_plan_info_get",
     "cconv_plan_destroy", "cconv_plan_reserve_accumulate", "cconv_forward_accumulate",
     "cconv_forward_planned", "cconv_forward", "cconv_forward_host",
+    "cconv_forward_host_async", "cconv_host_wait",
     "cconv_forward_noalloc", "cconv_pool_lower_bound", "cconv_pool_forward",
     "cconv_parallel_lower_bound", "cconv_parallel_partition", "cconv_theorem2_case",
     "cconv_plan_status", "cconv_plan_trace_read", "cconv_strerror", "cconv_last_cuda_error", "cconv_version",
@@ -108,6 +109,10 @@ def load_library():
     lib.cconv_forward_noalloc.argtypes = [vp, vp, vp] + nine + [i, vp, ctypes.POINTER(i)]
     lib.cconv_forward_host.restype = i
     lib.cconv_forward_host.argtypes = [vp, vp, vp, vp, vp]
+    lib.cconv_forward_host_async.restype = i
+    lib.cconv_forward_host_async.argtypes = [vp, vp, vp, vp, vp]
+    lib.cconv_host_wait.restype = i
+    lib.cconv_host_wait.argtypes = [vp, vp]
     lib.cconv_theorem2_case.restype = i
     lib.cconv_theorem2_case.argtypes = [i] * 7 + [d, ctypes.POINTER(i), dp]
     lib.cconv_parallel_lower_bound.restype = i
@@ -281,6 +286,19 @@ class Plan:
                                             ctypes.c_void_p(h_out.data_ptr()), _stream_ptr(stream)),
                "cconv_forward_host")
         return h_out
+
+    def forward_host_async(self, h_image, h_filt, h_out, stream=None):
+        """cconv_forward_host_async on pinned CPU tensors: queues the copies and the kernels and
+        returns; ``host_wait`` makes ``h_out`` valid."""
+        _check(self._lib.cconv_forward_host_async(self._h, ctypes.c_void_p(h_image.data_ptr()),
+                                                  ctypes.c_void_p(h_filt.data_ptr()),
+                                                  ctypes.c_void_p(h_out.data_ptr()), _stream_ptr(stream)),
+               "cconv_forward_host_async")
+        return h_out
+
+    def host_wait(self, stream=None):
+        """cconv_host_wait: waits for every queued forward_host_async call; raises on a device status."""
+        _check(self._lib.cconv_host_wait(self._h, _stream_ptr(stream)), "cconv_host_wait")
 
     def status(self, stream=None):
         """cconv_plan_status: synchronises and returns (code, detail bit mask)."""

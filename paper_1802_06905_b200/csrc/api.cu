@@ -215,6 +215,16 @@ struct cconv_plan {
   void* st_image = nullptr;
   void* st_filter = nullptr;
   void* st_out = nullptr;
+  // cconv_forward_host_async: two sets of staging arrays, a copy stream per direction, and per set
+  // the events "inputs copied", "kernels done", "Out copied back"
+  bool pipe_ready = false;
+  unsigned pipe_calls = 0;
+  void* pp_image[2] = {nullptr, nullptr};
+  void* pp_filter[2] = {nullptr, nullptr};
+  void* pp_out[2] = {nullptr, nullptr};
+  cudaStream_t pp_h2d = nullptr, pp_h2d_f = nullptr, pp_d2h = nullptr;
+  cudaEvent_t ev_in_f[2] = {nullptr, nullptr};
+  cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_run[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr};
   // the tensor map is rebuilt only when the base pointer changes
   mutable std::mutex mu;
   mutable const void* tm_image_ptr = nullptr;
@@ -578,6 +588,21 @@ void cconv_plan_destroy(cconv_plan* pl) {
     if (pl->st_filter) cudaFree(pl->st_filter);
     if (pl->st_out) cudaFree(pl->st_out);
     if (pl->d_acc) cudaFree(pl->d_acc);
+    if (pl->pp_d2h) cudaStreamSynchronize(pl->pp_d2h);
+    if (pl->pp_h2d) cudaStreamSynchronize(pl->pp_h2d);
+    if (pl->pp_h2d_f) cudaStreamSynchronize(pl->pp_h2d_f);
+    for (int i = 0; i < 2; ++i) {
+      if (pl->ev_in_f[i]) cudaEventDestroy(pl->ev_in_f[i]);
+      if (pl->pp_image[i]) cudaFree(pl->pp_image[i]);
+      if (pl->pp_filter[i]) cudaFree(pl->pp_filter[i]);
+      if (pl->pp_out[i]) cudaFree(pl->pp_out[i]);
+      if (pl->ev_in[i]) cudaEventDestroy(pl->ev_in[i]);
+      if (pl->ev_run[i]) cudaEventDestroy(pl->ev_run[i]);
+      if (pl->ev_out[i]) cudaEventDestroy(pl->ev_out[i]);
+    }
+    if (pl->pp_h2d) cudaStreamDestroy(pl->pp_h2d);
+    if (pl->pp_h2d_f) cudaStreamDestroy(pl->pp_h2d_f);
+    if (pl->pp_d2h) cudaStreamDestroy(pl->pp_d2h);
     cudaSetDevice(prev);
   }
   if (pl->acc_twin) cconv_plan_destroy(pl->acc_twin);
@@ -718,6 +743,61 @@ int cconv_forward_host(cconv_plan* pl, const void* hImage, const void* hFilter, 
   int rc = cconv_forward_planned(pl, pl->st_image, pl->st_filter, pl->st_out, cuda_stream);
   if (rc != CCONV_OK) return rc;
   CCONV_CUDA(cudaMemcpyAsync(hOut, pl->st_out, no, cudaMemcpyDeviceToHost, stream));
+  int detail = 0;
+  return cconv_plan_status(pl, cuda_stream, &detail);
+}
+
+int cconv_forward_host_async(cconv_plan* pl, const void* hImage, const void* hFilter, void* hOut,
+                             void* cuda_stream) {
+  if (!pl || !hImage || !hFilter || !hOut || pl->device < 0) return CCONV_EINVAL;
+  int cur = -1;
+  if (cudaGetDevice(&cur) != cudaSuccess || cur != pl->device) return CCONV_EINVAL;
+  const Dims& d = pl->d;
+  const size_t ni = size_t(d.Wi()) * d.Hi() * d.C * d.B * 2;
+  const size_t nf = size_t(d.K) * d.R * d.S * d.C * 2;
+  const size_t no = size_t(d.K) * d.H * d.W * d.B * (pl->out_dtype == CCONV_OUT_F32 ? 4 : 2);
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (!pl->pipe_ready) {
+    CCONV_CUDA(cudaStreamCreateWithFlags(&pl->pp_h2d, cudaStreamNonBlocking));
+    CCONV_CUDA(cudaStreamCreateWithFlags(&pl->pp_h2d_f, cudaStreamNonBlocking));
+    CCONV_CUDA(cudaStreamCreateWithFlags(&pl->pp_d2h, cudaStreamNonBlocking));
+    for (int i = 0; i < 2; ++i) {
+      CCONV_CUDA(cudaEventCreateWithFlags(&pl->ev_in_f[i], cudaEventDisableTiming));
+      CCONV_CUDA(cudaMalloc(&pl->pp_image[i], ni));
+      CCONV_CUDA(cudaMalloc(&pl->pp_filter[i], nf));
+      CCONV_CUDA(cudaMalloc(&pl->pp_out[i], no));
+      CCONV_CUDA(cudaEventCreateWithFlags(&pl->ev_in[i], cudaEventDisableTiming));
+      CCONV_CUDA(cudaEventCreateWithFlags(&pl->ev_run[i], cudaEventDisableTiming));
+      CCONV_CUDA(cudaEventCreateWithFlags(&pl->ev_out[i], cudaEventDisableTiming));
+    }
+    pl->pipe_ready = true;
+  }
+  const int set = int(pl->pipe_calls++ & 1u);
+  // inputs: this set's arrays are free once the kernels of the call two back have run
+  // (Image and Filter on a stream each: a copy of this size is mostly fixed cost)
+  CCONV_CUDA(cudaStreamWaitEvent(pl->pp_h2d, pl->ev_run[set], 0));
+  CCONV_CUDA(cudaStreamWaitEvent(pl->pp_h2d_f, pl->ev_run[set], 0));
+  CCONV_CUDA(cudaMemcpyAsync(pl->pp_image[set], hImage, ni, cudaMemcpyHostToDevice, pl->pp_h2d));
+  CCONV_CUDA(cudaMemcpyAsync(pl->pp_filter[set], hFilter, nf, cudaMemcpyHostToDevice, pl->pp_h2d_f));
+  CCONV_CUDA(cudaEventRecord(pl->ev_in[set], pl->pp_h2d));
+  CCONV_CUDA(cudaEventRecord(pl->ev_in_f[set], pl->pp_h2d_f));
+  // kernels: after the inputs have landed and this set's Out of two calls back has been copied out
+  CCONV_CUDA(cudaStreamWaitEvent(stream, pl->ev_in[set], 0));
+  CCONV_CUDA(cudaStreamWaitEvent(stream, pl->ev_in_f[set], 0));
+  CCONV_CUDA(cudaStreamWaitEvent(stream, pl->ev_out[set], 0));
+  const int rc = cconv_forward_planned(pl, pl->pp_image[set], pl->pp_filter[set], pl->pp_out[set], cuda_stream);
+  if (rc != CCONV_OK) return rc;
+  CCONV_CUDA(cudaEventRecord(pl->ev_run[set], stream));
+  // Out: back to the host on the other copy stream
+  CCONV_CUDA(cudaStreamWaitEvent(pl->pp_d2h, pl->ev_run[set], 0));
+  CCONV_CUDA(cudaMemcpyAsync(hOut, pl->pp_out[set], no, cudaMemcpyDeviceToHost, pl->pp_d2h));
+  CCONV_CUDA(cudaEventRecord(pl->ev_out[set], pl->pp_d2h));
+  return CCONV_OK;
+}
+
+int cconv_host_wait(cconv_plan* pl, void* cuda_stream) {
+  if (!pl || pl->device < 0) return CCONV_EINVAL;
+  if (pl->pp_d2h) CCONV_CUDA(cudaStreamSynchronize(pl->pp_d2h));
   int detail = 0;
   return cconv_plan_status(pl, cuda_stream, &detail);
 }

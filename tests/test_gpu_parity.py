@@ -314,6 +314,33 @@ def test_forward_host_entry_point():
     plan.close()
 
 
+def test_pipelined_host_calls_keep_every_steps_result():
+    """cconv_forward_host_async: six queued steps with different inputs and their own Out buffers
+    (two staging sets inside the plan, so sets are re-used twice); each Out must be its own step's."""
+    c = cs("host_pipe", 32, 24, 72, 9, 8, 3, 3)
+    plan = binding.Plan(*c.dims(), device=0, out_dtype=binding.OUT_BF16)
+    steps = []
+    for n in range(6):
+        ib, fb = synth.make_inputs(ConvShape(c.name, *c.dims(), seed=8600 + n))
+        hi = torch.from_numpy(ib.view(np.int16)).view(torch.bfloat16).pin_memory()
+        hf = torch.from_numpy(fb.view(np.int16)).view(torch.bfloat16).pin_memory()
+        ho = torch.full(c.out_shape, float("nan"), dtype=torch.bfloat16).pin_memory()
+        steps.append((ib, fb, hi, hf, ho))
+    for _, _, hi, hf, ho in steps:
+        plan.forward_host_async(hi, hf, ho)
+    plan.host_wait()
+    for n, (ib, fb, _, _, ho) in enumerate(steps):
+        exp, ab = ocnn.cnn_bf16(ib, fb, oshape(c))
+        assert_close(ocnn.bf16_bits_to_f64(to_bits(ho)), exp, ab, f"pipelined step {n}", bf16_out=True)
+    # the synchronous call still works on the same plan afterwards
+    ib, fb, hi, hf, ho = steps[0]
+    ho.fill_(float("nan"))
+    plan.forward_host(hi, hf, ho)
+    exp, ab = ocnn.cnn_bf16(ib, fb, oshape(c))
+    assert_close(ocnn.bf16_bits_to_f64(to_bits(ho)), exp, ab, "synchronous call after the pipeline", bf16_out=True)
+    plan.close()
+
+
 def test_misaligned_and_null_pointers_are_rejected_on_the_host():
     c = BY["cfg1_tiny_3x3"]
     plan = binding.Plan(*c.dims(), device=0)
