@@ -373,16 +373,17 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloT
     }
   }
   // Split tiles (two CTAs of a cluster take half of the channels each and exchange partial sums on
-  // chip) are searched on request, and for problems that leave at least half of the SMs idle while
-  // every CTA streams a long Filter slab: filters of 9 or more taps with at least 144 units per tile
-  // (C*R*S >= 2304).  Measured on 41 such shapes (B 8..32, C and K 128..2048, 4x4 to 14x14 outputs):
-  // where the model puts the split tile at 0.70 of the whole tile's time or below, and the split
-  // tile at most doubles the accumulator columns computed (a wider batch block on a small batch is
-  // mostly zero padding; up to four times the columns where four times as many CTAs then work),
-  // the call takes 0.61-0.89 of the time; 1x1 filters and shorter
-  // slabs gain nothing or lose up to 30 %.
+  // chip) are searched on request, and for problems in which every CTA streams a long Filter slab
+  // past few output pixels: filters of 9 or more taps with at least 144 units per tile
+  // (C*R*S >= 2304), where a split tiling exists at all (its tiles run as one wave, so at most half
+  // as many tiles as SMs).  Measured on 52 such shapes (B 8..64, C and K 128..2048, 4x4 to 14x14
+  // outputs): where the model puts the split tile at 0.70 of the whole tile's time or below, and the
+  // split tile at most doubles the accumulator columns computed (a wider batch block on a small
+  // batch is mostly zero padding; up to four times the columns where four times as many CTAs then
+  // work), the call takes 0.61-0.90 of the time; above 0.70 (14x14 outputs with 256 channels, the
+  // benchmark shapes), with 1x1 filters and with shorter slabs it gains nothing or loses up to 30 %.
   if (found && force[5] == 0 && !force[0] && !force[1] && !force[2] && !force[3] && !force[4] &&
-      2 * best.tiles <= m.sm_count && RS >= 9 && units >= 144) {
+      RS >= 9 && units >= 144) {
     const int want_split[6] = {0, 0, 0, 0, 0, 2};
     HaloTile sp;
     if (choose_halo_tile(d, m, want_split, &sp)) {
