@@ -107,10 +107,10 @@ typedef struct {
    * of each image taking the place of one image (run_B = 8-multiple >= B * bands).  The tile and the
    * tail above (tail_h0 included) then describe that run. */
   int run_B, run_H, bands;
-  /* HALO variant: 2 when every tile is shared by the two CTAs of a cluster, half of the channels
-   * each, partial sums exchanged through distributed shared memory (grid = 2 * tiles; the planner
-   * does so for filters of 9 or more taps with long channel loops whose tiles would leave half of the
-   * SMs idle), else 1. */
+  /* HALO variant: 2 or 4 when every tile is shared by the CTAs of a cluster of that size, an equal
+   * share of the channels each, partial sums exchanged through distributed shared memory (grid =
+   * split * tiles; the planner does so for filters of 9 or more taps with long channel loops and few
+   * output pixels), else 1. */
   int split;
 } cconv_plan_info;
 

@@ -490,7 +490,7 @@ __device__ __forceinline__ void store_run32(OutT* dst, const uint32_t (&v)[32]) 
 // ------------------------------------------------------------------------------------------------
 // BH, TAPS: the issuer's compile-time shape (see mma_role).  One kernel per shape: the issuing loop
 // is sensitive to the size of the code around it, so a launch carries only the loops it runs.
-template <typename OutT, int BH, int TAPS, bool SB>
+template <typename OutT, int BH, int TAPS, bool SB, bool S4>
 __global__ void __launch_bounds__(kThreads, 1)
     cconv_halo_kernel(const __grid_constant__ CUtensorMap tm_image,
                       const uint8_t* __restrict__ packed_filter, OutT* __restrict__ out,
@@ -540,7 +540,12 @@ __global__ void __launch_bounds__(kThreads, 1)
     *abort_flag = 0;
     fence_barrier_init();
     // split launch: the peer will copy 128 rows of acc_cols/2 fp32 partial sums into this CTA
-    if (p.split > 1) mbar_arrive_expect_tx(bar_xchg, 128u * uint32_t(p.acc_cols >> 1) * 4u);
+    // (four CTAs per tile: each of three peers 128 rows of acc_cols/4)
+    if constexpr (S4) {
+      mbar_arrive_expect_tx(bar_xchg, 3u * 128u * uint32_t(p.acc_cols >> 2) * 4u);
+    } else {
+      if (p.split > 1) mbar_arrive_expect_tx(bar_xchg, 128u * uint32_t(p.acc_cols >> 1) * 4u);
+    }
     prefetch_tensormap(&tm_image);
   }
   if (warp == 1) {
@@ -742,13 +747,14 @@ __global__ void __launch_bounds__(kThreads, 1)
   }
 
   // ===================== split launch: exchange partial sums, then store =====================
-  // Both CTAs of the cluster hold a full 128 x acc_cols accumulator over their half of the
-  // channels.  Rank r owns the columns [r*half, (r+1)*half): it receives the peer's partial sums
-  // for them in its own shared memory (the rings are idle by then), adds its own and stores.
-  // The partial sums travel as four 16 KB asynchronous shared-memory-to-shared-memory copies per
-  // CTA (one per epilogue warp), credited to the receiver's mbarrier; single remote stores from
-  // 32 lanes to 32 different rows were measured 5x slower.
-  // Every thread of both CTAs reaches both cluster barriers, whatever happened before.
+  // The 2 or 4 CTAs of the cluster each hold a full 128 x acc_cols accumulator over their share of
+  // the channels.  Rank r owns the columns [r*half, (r+1)*half), half = acc_cols / split: it receives
+  // the peers' partial sums for them in its own shared memory (the rings are idle by then), adds its
+  // own and stores.  The partial sums travel as asynchronous shared-memory-to-shared-memory copies
+  // (one per epilogue warp and peer), credited to the receiver's mbarrier; single remote stores from
+  // 32 lanes to 32 different rows were measured 5x slower.  The order of the additions is fixed
+  // (own, then the slices in slot order), so results are reproducible run to run.
+  // Every thread of every CTA reaches both cluster barriers, whatever happened before.
   if (p.split > 1) {
     const bool epi = warp >= 2 && warp <= 5;
     const int q = warp & 3;
@@ -761,104 +767,220 @@ __global__ void __launch_bounds__(kThreads, 1)
     __syncwarp();
     cluster_sync_all();  // both accumulators complete: neither CTA's rings are read any more
     if (threadIdx.x == 64) CCONV_TRACE(8);
-    const int half = p.acc_cols >> 1;                 // columns per owner, a multiple of 32
-    const uint32_t row_bytes = uint32_t(half) * 4u;   // one accumulator row of fp32 partial sums
-    const uint32_t t_lane = tmem_base + (uint32_t(q * 32) << 16);
-    // Incoming area: row L = 32q + lane at smem0 + L*row_bytes; outgoing staging area right behind
-    // it, same layout.  16-byte chunk c of a row is stored at chunk c ^ (lane & 7), so that the
-    // eight lanes of a store phase hit eight different bank groups.
-    const uint32_t in_row = smem0 + uint32_t(q * 32 + lane) * row_bytes;
-    const uint32_t out_area = smem0 + 128u * row_bytes;
-    const uint32_t out_row = out_area + uint32_t(q * 32 + lane) * row_bytes;
-    const uint32_t x7 = uint32_t(lane & 7);
-    if (epi && acc_ok) {
-      const int col0 = (crank ^ 1) * half;  // the peer's columns
-      for (int g = 0; g < half; g += 32) {
-        uint32_t v[32];
-        tmem_ld_32x32b_x32(t_lane + uint32_t(col0 + g), v);
-        tmem_ld_wait();
-#pragma unroll
-        for (int c = 0; c < 8; ++c)
-          st_shared_v4(out_row + ((uint32_t(g / 4 + c) ^ x7) << 4), v[4 * c], v[4 * c + 1],
-                       v[4 * c + 2], v[4 * c + 3]);
-      }
-      fence_proxy_async_shared();  // the copy engine reads these generic-proxy writes
-      __syncwarp();
-      if (lane == 0) {
-        const uint32_t peer = uint32_t(crank ^ 1);
-        const uint32_t warp_rows = uint32_t(q * 32) * row_bytes;
-        bulk_copy_to_peer(cluster_map_shared(smem0 + warp_rows, peer), out_area + warp_rows,
-                          32u * row_bytes, cluster_map_shared(bar_xchg, peer));
-      }
-    }
-    if (threadIdx.x == 64) CCONV_TRACE(9);
-    if (epi && acc_ok) {
-      acc_ok = mbar_wait_warp(bar_xchg, 0, abort_flag, status, kStatEpilogueWait, limit);
-      acc_ok = __all_sync(0xffffffffu, acc_ok);
-    }
-    if (threadIdx.x == 64) CCONV_TRACE(12);
-    if (epi && acc_ok) {
-      const int tile = tile_first;
-      int t = tile;
-      const int kt = t % p.tiles_k; t /= p.tiles_k;
-      const int bt = t % p.tiles_b; t /= p.tiles_b;
-      const int wt = t % p.tiles_w; t /= p.tiles_w;
-      const int ht = t;
-      const int k = kt * 128 + q * 32 + lane;
-      const int col0 = crank * half;
-      for (int g = 0; g < half; g += 32) {
-        uint32_t v[32];
-        tmem_ld_32x32b_x32(t_lane + uint32_t(col0 + g), v);
-        tmem_ld_wait();
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          uint32_t a0, a1, a2, a3;
-          ld_shared_v4(in_row + ((uint32_t(g / 4 + c) ^ x7) << 4), a0, a1, a2, a3);
-          v[4 * c] = __float_as_uint(__uint_as_float(v[4 * c]) + __uint_as_float(a0));
-          v[4 * c + 1] = __float_as_uint(__uint_as_float(v[4 * c + 1]) + __uint_as_float(a1));
-          v[4 * c + 2] = __float_as_uint(__uint_as_float(v[4 * c + 2]) + __uint_as_float(a2));
-          v[4 * c + 3] = __float_as_uint(__uint_as_float(v[4 * c + 3]) + __uint_as_float(a3));
+    if constexpr (S4) {
+      const int nsp = p.split;                          // CTAs per tile: 2 or 4
+      const int half = p.acc_cols / nsp;                // columns per owner, a multiple of 32
+      const uint32_t row_bytes = uint32_t(half) * 4u;   // one accumulator row of fp32 partial sums
+      const uint32_t t_lane = tmem_base + (uint32_t(q * 32) << 16);
+      // Incoming area: one slice of 128 rows per peer, row L = 32q + lane of slice j at
+      // smem0 + (j*128 + L)*row_bytes; the outgoing staging slices right behind them, same layout.
+      // The sender of rank s writes slice (s - r - 1) mod nsp of the receiver of rank r.  16-byte
+      // chunk c of a row is stored at chunk c ^ (lane & 7), so that the eight lanes of a store phase
+      // hit eight different bank groups.
+      const uint32_t slice_bytes = 128u * row_bytes;
+      const uint32_t my_row = uint32_t(q * 32 + lane) * row_bytes;
+      const uint32_t out_area = smem0 + uint32_t(nsp - 1) * slice_bytes;
+      const uint32_t x7 = uint32_t(lane & 7);
+      if (epi && acc_ok) {
+        for (int j = 1; j < nsp; ++j) {
+          const int peer = (crank + j) % nsp;           // its slot for this CTA's slice is nsp - 1 - j ...
+          const uint32_t slot_there = uint32_t(nsp - 1 - j);  // ... = (crank - peer - 1) mod nsp
+          const uint32_t out_row = out_area + uint32_t(j - 1) * slice_bytes + my_row;
+          const int col0 = peer * half;                 // the peer's columns
+          for (int g = 0; g < half; g += 32) {
+            uint32_t v[32];
+            tmem_ld_32x32b_x32(t_lane + uint32_t(col0 + g), v);
+            tmem_ld_wait();
+  #pragma unroll
+            for (int c = 0; c < 8; ++c)
+              st_shared_v4(out_row + ((uint32_t(g / 4 + c) ^ x7) << 4), v[4 * c], v[4 * c + 1],
+                           v[4 * c + 2], v[4 * c + 3]);
+          }
+          fence_proxy_async_shared();  // the copy engine reads these generic-proxy writes
+          __syncwarp();
+          if (lane == 0) {
+            const uint32_t warp_rows = uint32_t(q * 32) * row_bytes;
+            bulk_copy_to_peer(cluster_map_shared(smem0 + slot_there * slice_bytes + warp_rows, uint32_t(peer)),
+                              out_area + uint32_t(j - 1) * slice_bytes + warp_rows, 32u * row_bytes,
+                              cluster_map_shared(bar_xchg, uint32_t(peer)));
+          }
         }
-        if constexpr (SB) {
-          // column -> (output row, 2 or 4 pixels, 16 or 8 images each), as in the epilogue above
-          const int col = col0 + g;
-          const int hh = col / p.n_mma, rem = col - hh * p.n_mma;
-          const int h = p.h0 + ht * p.bh + hh;
-          const int per = 32 / p.bb;
-          const int ww0 = rem / p.bb;
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            if (j >= per) break;
-            const int w = wt * p.bw + ww0 + j;
-            if (!(k < p.K && h < p.H && w < p.W && ww0 + j < p.bw)) continue;
-            OutT* dst = out + (((long long)k * p.H + h) * p.W + w) * p.B + bt * p.bb;
-            const int nb = p.B - bt * p.bb;
-#pragma unroll
-            for (int g8 = 0; g8 < 2; ++g8) {
-              const int first = (per == 4 ? j * 8 : j * 16 + g8 * 8);
-              if ((per == 4 && g8 == 1) || g8 * 8 >= nb) continue;
-              OutT* d8 = dst + g8 * 8;
-              if constexpr (sizeof(OutT) == 4) {
-                *reinterpret_cast<uint4*>(d8) = make_uint4(v[first], v[first + 1], v[first + 2], v[first + 3]);
-                *reinterpret_cast<uint4*>(d8 + 4) = make_uint4(v[first + 4], v[first + 5], v[first + 6], v[first + 7]);
-              } else {
-                *reinterpret_cast<uint4*>(d8) =
-                    make_uint4(pack_bf16x2(v[first], v[first + 1]), pack_bf16x2(v[first + 2], v[first + 3]),
-                               pack_bf16x2(v[first + 4], v[first + 5]), pack_bf16x2(v[first + 6], v[first + 7]));
-              }
+      }
+      if (threadIdx.x == 64) CCONV_TRACE(9);
+      if (epi && acc_ok) {
+        acc_ok = mbar_wait_warp(bar_xchg, 0, abort_flag, status, kStatEpilogueWait, limit);
+        acc_ok = __all_sync(0xffffffffu, acc_ok);
+      }
+      if (threadIdx.x == 64) CCONV_TRACE(12);
+      if (epi && acc_ok) {
+        const int tile = tile_first;
+        int t = tile;
+        const int kt = t % p.tiles_k; t /= p.tiles_k;
+        const int bt = t % p.tiles_b; t /= p.tiles_b;
+        const int wt = t % p.tiles_w; t /= p.tiles_w;
+        const int ht = t;
+        const int k = kt * 128 + q * 32 + lane;
+        const int col0 = crank * half;
+        for (int g = 0; g < half; g += 32) {
+          uint32_t v[32];
+          tmem_ld_32x32b_x32(t_lane + uint32_t(col0 + g), v);
+          tmem_ld_wait();
+          for (int j = 0; j < nsp - 1; ++j) {
+            const uint32_t in_row = smem0 + uint32_t(j) * slice_bytes + my_row;
+  #pragma unroll
+            for (int c = 0; c < 8; ++c) {
+              uint32_t a0, a1, a2, a3;
+              ld_shared_v4(in_row + ((uint32_t(g / 4 + c) ^ x7) << 4), a0, a1, a2, a3);
+              v[4 * c] = __float_as_uint(__uint_as_float(v[4 * c]) + __uint_as_float(a0));
+              v[4 * c + 1] = __float_as_uint(__uint_as_float(v[4 * c + 1]) + __uint_as_float(a1));
+              v[4 * c + 2] = __float_as_uint(__uint_as_float(v[4 * c + 2]) + __uint_as_float(a2));
+              v[4 * c + 3] = __float_as_uint(__uint_as_float(v[4 * c + 3]) + __uint_as_float(a3));
             }
           }
-        } else {
-          // column -> (output row, pixel, 32 images)
-          const int col = col0 + g;
-          const int hh = col / p.n_mma, rem = col - hh * p.n_mma;
-          const int ww = rem / p.bb, ch = (rem - ww * p.bb) >> 5;
-          const int h = p.h0 + ht * p.bh + hh, w = wt * p.bw + ww;
-          if (k < p.K && h < p.H && w < p.W) {
-            OutT* dst = out + (((long long)k * p.H + h) * p.W + w) * p.B + bt * p.bb + ch * 32;
-            const int nb = p.B - (bt * p.bb + ch * 32);
-            if (nb >= 32 && wide_rows) store_run32(dst, v);
-            else if (nb > 0) store_run_partial(dst, v, nb < 32 ? nb : 32);
+          if constexpr (SB) {
+            // column -> (output row, 2 or 4 pixels, 16 or 8 images each), as in the epilogue above
+            const int col = col0 + g;
+            const int hh = col / p.n_mma, rem = col - hh * p.n_mma;
+            const int h = p.h0 + ht * p.bh + hh;
+            const int per = 32 / p.bb;
+            const int ww0 = rem / p.bb;
+  #pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              if (j >= per) break;
+              const int w = wt * p.bw + ww0 + j;
+              if (!(k < p.K && h < p.H && w < p.W && ww0 + j < p.bw)) continue;
+              OutT* dst = out + (((long long)k * p.H + h) * p.W + w) * p.B + bt * p.bb;
+              const int nb = p.B - bt * p.bb;
+  #pragma unroll
+              for (int g8 = 0; g8 < 2; ++g8) {
+                const int first = (per == 4 ? j * 8 : j * 16 + g8 * 8);
+                if ((per == 4 && g8 == 1) || g8 * 8 >= nb) continue;
+                OutT* d8 = dst + g8 * 8;
+                if constexpr (sizeof(OutT) == 4) {
+                  *reinterpret_cast<uint4*>(d8) = make_uint4(v[first], v[first + 1], v[first + 2], v[first + 3]);
+                  *reinterpret_cast<uint4*>(d8 + 4) = make_uint4(v[first + 4], v[first + 5], v[first + 6], v[first + 7]);
+                } else {
+                  *reinterpret_cast<uint4*>(d8) =
+                      make_uint4(pack_bf16x2(v[first], v[first + 1]), pack_bf16x2(v[first + 2], v[first + 3]),
+                                 pack_bf16x2(v[first + 4], v[first + 5]), pack_bf16x2(v[first + 6], v[first + 7]));
+                }
+              }
+            }
+          } else {
+            // column -> (output row, pixel, 32 images)
+            const int col = col0 + g;
+            const int hh = col / p.n_mma, rem = col - hh * p.n_mma;
+            const int ww = rem / p.bb, ch = (rem - ww * p.bb) >> 5;
+            const int h = p.h0 + ht * p.bh + hh, w = wt * p.bw + ww;
+            if (k < p.K && h < p.H && w < p.W) {
+              OutT* dst = out + (((long long)k * p.H + h) * p.W + w) * p.B + bt * p.bb + ch * 32;
+              const int nb = p.B - (bt * p.bb + ch * 32);
+              if (nb >= 32 && wide_rows) store_run32(dst, v);
+              else if (nb > 0) store_run_partial(dst, v, nb < 32 ? nb : 32);
+            }
+          }
+        }
+      }
+    } else {
+      const int half = p.acc_cols >> 1;                 // columns per owner, a multiple of 32
+      const uint32_t row_bytes = uint32_t(half) * 4u;   // one accumulator row of fp32 partial sums
+      const uint32_t t_lane = tmem_base + (uint32_t(q * 32) << 16);
+      // Incoming area: row L = 32q + lane at smem0 + L*row_bytes; outgoing staging area right behind
+      // it, same layout.  16-byte chunk c of a row is stored at chunk c ^ (lane & 7), so that the
+      // eight lanes of a store phase hit eight different bank groups.
+      const uint32_t in_row = smem0 + uint32_t(q * 32 + lane) * row_bytes;
+      const uint32_t out_area = smem0 + 128u * row_bytes;
+      const uint32_t out_row = out_area + uint32_t(q * 32 + lane) * row_bytes;
+      const uint32_t x7 = uint32_t(lane & 7);
+      if (epi && acc_ok) {
+        const int col0 = (crank ^ 1) * half;  // the peer's columns
+        for (int g = 0; g < half; g += 32) {
+          uint32_t v[32];
+          tmem_ld_32x32b_x32(t_lane + uint32_t(col0 + g), v);
+          tmem_ld_wait();
+  #pragma unroll
+          for (int c = 0; c < 8; ++c)
+            st_shared_v4(out_row + ((uint32_t(g / 4 + c) ^ x7) << 4), v[4 * c], v[4 * c + 1],
+                         v[4 * c + 2], v[4 * c + 3]);
+        }
+        fence_proxy_async_shared();  // the copy engine reads these generic-proxy writes
+        __syncwarp();
+        if (lane == 0) {
+          const uint32_t peer = uint32_t(crank ^ 1);
+          const uint32_t warp_rows = uint32_t(q * 32) * row_bytes;
+          bulk_copy_to_peer(cluster_map_shared(smem0 + warp_rows, peer), out_area + warp_rows,
+                            32u * row_bytes, cluster_map_shared(bar_xchg, peer));
+        }
+      }
+      if (threadIdx.x == 64) CCONV_TRACE(9);
+      if (epi && acc_ok) {
+        acc_ok = mbar_wait_warp(bar_xchg, 0, abort_flag, status, kStatEpilogueWait, limit);
+        acc_ok = __all_sync(0xffffffffu, acc_ok);
+      }
+      if (threadIdx.x == 64) CCONV_TRACE(12);
+      if (epi && acc_ok) {
+        const int tile = tile_first;
+        int t = tile;
+        const int kt = t % p.tiles_k; t /= p.tiles_k;
+        const int bt = t % p.tiles_b; t /= p.tiles_b;
+        const int wt = t % p.tiles_w; t /= p.tiles_w;
+        const int ht = t;
+        const int k = kt * 128 + q * 32 + lane;
+        const int col0 = crank * half;
+        for (int g = 0; g < half; g += 32) {
+          uint32_t v[32];
+          tmem_ld_32x32b_x32(t_lane + uint32_t(col0 + g), v);
+          tmem_ld_wait();
+  #pragma unroll
+          for (int c = 0; c < 8; ++c) {
+            uint32_t a0, a1, a2, a3;
+            ld_shared_v4(in_row + ((uint32_t(g / 4 + c) ^ x7) << 4), a0, a1, a2, a3);
+            v[4 * c] = __float_as_uint(__uint_as_float(v[4 * c]) + __uint_as_float(a0));
+            v[4 * c + 1] = __float_as_uint(__uint_as_float(v[4 * c + 1]) + __uint_as_float(a1));
+            v[4 * c + 2] = __float_as_uint(__uint_as_float(v[4 * c + 2]) + __uint_as_float(a2));
+            v[4 * c + 3] = __float_as_uint(__uint_as_float(v[4 * c + 3]) + __uint_as_float(a3));
+          }
+          if constexpr (SB) {
+            // column -> (output row, 2 or 4 pixels, 16 or 8 images each), as in the epilogue above
+            const int col = col0 + g;
+            const int hh = col / p.n_mma, rem = col - hh * p.n_mma;
+            const int h = p.h0 + ht * p.bh + hh;
+            const int per = 32 / p.bb;
+            const int ww0 = rem / p.bb;
+  #pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              if (j >= per) break;
+              const int w = wt * p.bw + ww0 + j;
+              if (!(k < p.K && h < p.H && w < p.W && ww0 + j < p.bw)) continue;
+              OutT* dst = out + (((long long)k * p.H + h) * p.W + w) * p.B + bt * p.bb;
+              const int nb = p.B - bt * p.bb;
+  #pragma unroll
+              for (int g8 = 0; g8 < 2; ++g8) {
+                const int first = (per == 4 ? j * 8 : j * 16 + g8 * 8);
+                if ((per == 4 && g8 == 1) || g8 * 8 >= nb) continue;
+                OutT* d8 = dst + g8 * 8;
+                if constexpr (sizeof(OutT) == 4) {
+                  *reinterpret_cast<uint4*>(d8) = make_uint4(v[first], v[first + 1], v[first + 2], v[first + 3]);
+                  *reinterpret_cast<uint4*>(d8 + 4) = make_uint4(v[first + 4], v[first + 5], v[first + 6], v[first + 7]);
+                } else {
+                  *reinterpret_cast<uint4*>(d8) =
+                      make_uint4(pack_bf16x2(v[first], v[first + 1]), pack_bf16x2(v[first + 2], v[first + 3]),
+                                 pack_bf16x2(v[first + 4], v[first + 5]), pack_bf16x2(v[first + 6], v[first + 7]));
+                }
+              }
+            }
+          } else {
+            // column -> (output row, pixel, 32 images)
+            const int col = col0 + g;
+            const int hh = col / p.n_mma, rem = col - hh * p.n_mma;
+            const int ww = rem / p.bb, ch = (rem - ww * p.bb) >> 5;
+            const int h = p.h0 + ht * p.bh + hh, w = wt * p.bw + ww;
+            if (k < p.K && h < p.H && w < p.W) {
+              OutT* dst = out + (((long long)k * p.H + h) * p.W + w) * p.B + bt * p.bb + ch * 32;
+              const int nb = p.B - (bt * p.bb + ch * 32);
+              if (nb >= 32 && wide_rows) store_run32(dst, v);
+              else if (nb > 0) store_run_partial(dst, v, nb < 32 ? nb : 32);
+            }
           }
         }
       }
@@ -895,19 +1017,33 @@ template <typename OutT, bool SB>
 HaloFn<OutT> halo_fn_sb(int R, int S, int bh) {
   const int b = bh == 1 ? 1 : bh == 2 ? 2 : 0;
   if (R == 3 && S == 3)
-    return b == 1 ? cconv_halo_kernel<OutT, 1, 9, SB> : b == 2 ? cconv_halo_kernel<OutT, 2, 9, SB>
-                                                               : cconv_halo_kernel<OutT, 0, 9, SB>;
+    return b == 1 ? cconv_halo_kernel<OutT, 1, 9, SB, false> : b == 2 ? cconv_halo_kernel<OutT, 2, 9, SB, false>
+                                                                      : cconv_halo_kernel<OutT, 0, 9, SB, false>;
   if (R * S == 1)
-    return b == 1 ? cconv_halo_kernel<OutT, 1, 1, SB> : b == 2 ? cconv_halo_kernel<OutT, 2, 1, SB>
-                                                               : cconv_halo_kernel<OutT, 0, 1, SB>;
-  return b == 1 ? cconv_halo_kernel<OutT, 1, 0, SB> : b == 2 ? cconv_halo_kernel<OutT, 2, 0, SB>
-                                                             : cconv_halo_kernel<OutT, 0, 0, SB>;
+    return b == 1 ? cconv_halo_kernel<OutT, 1, 1, SB, false> : b == 2 ? cconv_halo_kernel<OutT, 2, 1, SB, false>
+                                                                      : cconv_halo_kernel<OutT, 0, 1, SB, false>;
+  return b == 1 ? cconv_halo_kernel<OutT, 1, 0, SB, false> : b == 2 ? cconv_halo_kernel<OutT, 2, 0, SB, false>
+                                                                    : cconv_halo_kernel<OutT, 0, 0, SB, false>;
 }
 
-// One kernel per issuer shape (b_h, filter size) and per batch-block class (32/64 images, or 8/16
-// with its own epilogue), so that no instantiation carries another one's code.
+// Four CTAs per tile: 3x3 filters unrolled, every other filter size (1x1 included) on the generic
+// tap loop.
+template <typename OutT, bool SB>
+HaloFn<OutT> halo_fn_s4(int R, int S, int bh) {
+  const int b = bh == 1 ? 1 : bh == 2 ? 2 : 0;
+  if (R == 3 && S == 3)
+    return b == 1 ? cconv_halo_kernel<OutT, 1, 9, SB, true> : b == 2 ? cconv_halo_kernel<OutT, 2, 9, SB, true>
+                                                                     : cconv_halo_kernel<OutT, 0, 9, SB, true>;
+  return b == 1 ? cconv_halo_kernel<OutT, 1, 0, SB, true> : b == 2 ? cconv_halo_kernel<OutT, 2, 0, SB, true>
+                                                                   : cconv_halo_kernel<OutT, 0, 0, SB, true>;
+}
+
+// One kernel per issuer shape (b_h, filter size), per batch-block class (32/64 images, or 8/16
+// with its own epilogue) and for the four-CTA exchange, so that no instantiation carries another
+// one's code.
 template <typename OutT>
-HaloFn<OutT> halo_fn(int R, int S, int bh, int bb) {
+HaloFn<OutT> halo_fn(int R, int S, int bh, int bb, int split) {
+  if (split == 4) return bb < 32 ? halo_fn_s4<OutT, true>(R, S, bh) : halo_fn_s4<OutT, false>(R, S, bh);
   return bb < 32 ? halo_fn_sb<OutT, true>(R, S, bh) : halo_fn_sb<OutT, false>(R, S, bh);
 }
 
@@ -917,9 +1053,11 @@ cudaError_t prepare_all(int smem_bytes) {
                             {1, 1, 3}, {5, 5, 1}, {5, 5, 2}, {5, 5, 3}};
   for (const auto& sh : shapes) {
     for (int bb : {64, 8}) {
-      cudaError_t e = cudaFuncSetAttribute(halo_fn<OutT>(sh[0], sh[1], sh[2], bb),
-                                           cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
-      if (e != cudaSuccess) return e;
+      for (int split : {1, 4}) {
+        cudaError_t e = cudaFuncSetAttribute(halo_fn<OutT>(sh[0], sh[1], sh[2], bb, split),
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+        if (e != cudaSuccess) return e;
+      }
     }
   }
   return cudaSuccess;
@@ -966,9 +1104,9 @@ cudaError_t launch_halo(const CUtensorMap& tm_image, const void* packed_filter, 
     cfg.numAttrs = 2;
   }
   if (out_f32)
-    return cudaLaunchKernelEx(&cfg, halo_fn<float>(p.R, p.S, p.bh, p.bb), tm_image, pf,
+    return cudaLaunchKernelEx(&cfg, halo_fn<float>(p.R, p.S, p.bh, p.bb, p.split), tm_image, pf,
                               static_cast<float*>(out), p, status);
-  return cudaLaunchKernelEx(&cfg, halo_fn<__nv_bfloat16>(p.R, p.S, p.bh, p.bb), tm_image, pf,
+  return cudaLaunchKernelEx(&cfg, halo_fn<__nv_bfloat16>(p.R, p.S, p.bh, p.bb, p.split), tm_image, pf,
                             static_cast<__nv_bfloat16*>(out), p, status);
 }
 

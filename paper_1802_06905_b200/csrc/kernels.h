@@ -33,9 +33,10 @@ struct HaloKernelParams {
   int i_stages, f_stages;       // ring depths
   int tiles_k, tiles_b, tiles_w, tiles_h;
   int total_tiles;
-  int split;                    // 1, or 2: a cluster of two CTAs shares one tile, each contracting
-                                // half of the channels; partial sums are exchanged through
-                                // distributed shared memory and each CTA stores half the columns
+  int split;                    // 1, or 2 / 4: a cluster of that many CTAs shares one tile, each
+                                // contracting an equal share of the channels; partial sums are
+                                // exchanged through distributed shared memory and each CTA stores
+                                // its share of the columns
   int units_cta;                // units one CTA contracts: units / split
   int cchunks_cta;              // Image stages one CTA loads per tile: ceil(C/bc) / split
   int h0;                       // first output row of this launch (tiles_h counts rows from there)

@@ -248,8 +248,8 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloT
           // split = 2 (two CTAs per tile, half of the channels each): the exchange of partial sums
           // costs more than the shorter main loop saves wherever whole tiles fill the SMs, so this
           // loop searches it only on request (force[5] == 2); see the end of the function.
-          for (int split = 1; split <= 2; ++split) {
-            if (split != (force[5] == 2 ? 2 : 1)) continue;
+          for (int split : {1, 2, 4}) {
+            if (split != (force[5] == 2 || force[5] == 4 ? force[5] : 1)) continue;
             HaloTile t;
             t.bb = bb; t.bw = bw; t.bh = bh; t.bc = bc; t.bk = 128;
             t.halo_w = d.sw * (bw - 1) + d.R;
@@ -259,7 +259,7 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloT
             t.cchunks = (d.C + bc - 1) / bc;
             t.split = split;
             // halves must be whole Image stages of whole 16-channel chunks, and whole 32-column groups
-            if (split == 2 && (c16 % (2 * (bc / 16)) != 0 || (N * bh / 2) % 32 != 0)) continue;
+            if (split > 1 && (c16 % (split * (bc / 16)) != 0 || (N * bh) % (32 * split) != 0)) continue;
             // about nine units per Filter stage, a whole number of Image stages where those are
             // shorter (1x1 filters), so that stage boundaries of the two rings coincide
             const int upi = (bc / 16) * RS;
@@ -293,8 +293,8 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloT
             const int acc_cols = N * bh;
             // a split tile parks the peer's partial sums (128 rows x acc_cols/2 fp32) and stages its
             // own outgoing ones in the idle rings
-            if (split == 2 &&
-                1ll * is * img + 1ll * t.f_stages * t.filt_stage_bytes < 512ll * acc_cols)
+            if (split > 1 && 1ll * is * img + 1ll * t.f_stages * t.filt_stage_bytes <
+                                 1024ll * acc_cols * (split - 1) / split)
               continue;
             t.acc_bufs = (split == 1 && 2 * acc_cols <= m.tmem_cols) ? 2 : 1;
             int cols = 32;
@@ -306,8 +306,10 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloT
             t.tiles_h = (d.H + bh - 1) / bh;
             t.tiles = 1ll * t.tiles_k * t.tiles_b * t.tiles_w * t.tiles_h;
             if (t.tiles > 0x7fffffffll) continue;
-            if (split == 2 && 2 * t.tiles > m.sm_count) continue;  // split tiles run as one wave
-            t.grid = split == 2 ? int(2 * t.tiles) : int(std::min<long long>(t.tiles, m.sm_count));
+            // split tiles run as one wave; clusters of four CTAs stay inside a group of SMs, which
+            // leaves some SMs of every group unused: 128 of 148 CTAs is what is counted on
+            if (split > 1 && split * t.tiles > (split == 4 ? std::min(m.sm_count, 128) : m.sm_count)) continue;
+            t.grid = split > 1 ? int(split * t.tiles) : int(std::min<long long>(t.tiles, m.sm_count));
             t.packed_filter_bytes = 1ll * t.tiles_k * units * 4096;
             // at least ~115 KB so that two CTAs never share an SM (each would want the tensor memory)
             t.smem_bytes = std::max(int(t.i_stages * t.img_stage_bytes +
@@ -342,14 +344,15 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloT
               tile_cyc = std::max(cyc_mma + cyc_img, cyc_copy) + (t.acc_bufs == 2 ? 0.0 : cyc_epi);
               if (t.acc_bufs == 2) tile_cyc = std::max(tile_cyc, cyc_epi);
             }
-            if (split == 2) {
-              // two cluster barriers, acc_cols/2 columns of fp32 pushed to the peer (about 32 B/clk),
-              // then half an epilogue
+            if (split > 1) {
+              // two cluster barriers, all but one share of the fp32 accumulator (128 rows) pushed to
+              // the peers (about 32 B/clk), then one share of an epilogue
               tile_cyc = (t.i_stages == 1 ? cyc_mma + cyc_copy : std::max(cyc_mma, cyc_copy)) +
-                         1000.0 + 256.0 * acc_cols / 32.0 + 0.5 * cyc_epi + 4.0 * acc_cols;
+                         1000.0 + 512.0 * acc_cols * (split - 1) / split / 32.0 + cyc_epi / split +
+                         4.0 * acc_cols;
             }
             tile_cyc += 400.0;  // hand-overs at a tile boundary (accumulator full/empty, ring restart)
-            const double waves = split == 2 ? 1.0 : std::ceil(double(t.tiles) / t.grid);
+            const double waves = split > 1 ? 1.0 : std::ceil(double(t.tiles) / t.grid);
             t.tile_cycles = tile_cyc;
             // pipeline fill: nothing is issued before the first Image and Filter stages have landed
             const double fill = (double(img) + double(t.filt_stage_bytes)) / l2_rate;
@@ -384,14 +387,17 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloT
   // benchmark shapes), with 1x1 filters and with shorter slabs it gains nothing or loses up to 30 %.
   if (found && force[5] == 0 && !force[0] && !force[1] && !force[2] && !force[3] && !force[4] &&
       RS >= 9 && units >= 144) {
-    const int want_split[6] = {0, 0, 0, 0, 0, 2};
-    HaloTile sp;
-    if (choose_halo_tile(d, m, want_split, &sp)) {
-      const double cols_whole = double(best.tiles) * best.bb * best.bw * best.bh;
+    const HaloTile whole = best;
+    for (int ways : {2, 4}) {
+      const int want_split[6] = {0, 0, 0, 0, 0, ways};
+      HaloTile sp;
+      if (!choose_halo_tile(d, m, want_split, &sp)) continue;
+      const double cols_whole = double(whole.tiles) * whole.bb * whole.bw * whole.bh;
       const double cols_split = double(sp.tiles) * sp.bb * sp.bw * sp.bh;
       const bool cols_ok = cols_split <= 2.0 * cols_whole ||
-                           (cols_split <= 4.0 * cols_whole && sp.grid >= 4 * best.grid);
-      if (sp.est_cycles <= 0.70 * best.est_cycles && cols_ok) best = sp;
+                           (cols_split <= 4.0 * cols_whole && sp.grid >= 4 * whole.grid);
+      if (sp.est_cycles <= 0.70 * whole.est_cycles && cols_ok && sp.est_cycles < best.est_cycles)
+        best = sp;
     }
   }
   if (found) *out = best;

@@ -61,7 +61,7 @@ struct HaloTile {
   int f_stages = 0;   // Filter ring depth
   int uf = 0;         // units per Filter stage
   int acc_bufs = 1;   // TMEM accumulator buffers (2 when two fit in 512 columns)
-  int split = 1;      // 2: two CTAs (a cluster) share each tile, half of the channels each
+  int split = 1;      // 2 or 4: the CTAs of a cluster share each tile, an equal share of the channels each
   int tmem_cols = 0;
   int c16 = 0;        // 16-channel chunks: ceil(C/16)
   int cchunks = 0;    // Image stages per tile: ceil(C/bc)

@@ -307,10 +307,11 @@ def test_random_shapes_plan_to_hardware_legal_tiles():
             assert 1 <= info["halo_w"] <= 256 and 1 <= info["halo_h"] <= 256
             img_stage = info["halo_w"] * info["halo_h"] * info["bc"] * info["bb"] * 2
             assert info["stages"] * img_stage + info["filter_stages"] * 4096 <= info["smem_bytes"]
-            assert 1 <= info["grid"] <= 148 and info["split"] in (1, 2)
-            if info["split"] == 2:   # a cluster of two CTAs per tile, one wave
-                assert info["grid"] == 2 * info["tiles"] and R * S >= 9
-                assert (n * info["bh"] // 2) % 32 == 0 and info["tail_h0"] == Hrun
+            assert 1 <= info["grid"] <= 148 and info["split"] in (1, 2, 4)
+            if info["split"] > 1:    # a cluster of two or four CTAs per tile, one wave
+                assert info["grid"] == info["split"] * info["tiles"] and R * S >= 9
+                assert (n * info["bh"]) % (32 * info["split"]) == 0 and info["tail_h0"] == Hrun
+                assert info["split"] == 2 or info["grid"] <= 128
             else:
                 assert info["tiles"] >= info["grid"]
             assert info["bw"] <= max(W, 1) + 3 and info["bh"] <= max(Hrun, 1)

@@ -148,13 +148,19 @@ def test_halo_tail_launch(monkeypatch, out_dtype):
     ("8,1,32,0,32,2", cs("split_w", 32, 128, 128, 13, 3, 3, 3)),        # b_h = 1: pixels split; ragged w
     ("2,2,64,0,64,2", cs("split_1x1", 64, 256, 200, 6, 6, 1, 1)),       # 1x1, K not a multiple of 128
     ("4,1,16,0,64,2", cs("split_s2", 64, 32, 64, 7, 4, 5, 3, 2, 1)),    # stride 2, 5x3 filter
+    ("4,1,16,0,32,4", cs("split4_3x3", 32, 128, 160, 7, 5, 3, 3)),      # four CTAs per tile, a quarter of the channels each
+    ("2,2,32,0,64,4", cs("split4_b64_bh2", 64, 256, 128, 6, 4, 3, 3)),  # b_h = 2: 256 columns, 64 per CTA
+    ("8,2,16,0,8,4", cs("split4_blocks_of_8", 8, 64, 72, 7, 6, 3, 3)),  # batch blocks of 8 images
+    ("4,1,32,0,16,2", cs("split2_blocks_of_16", 16, 128, 136, 7, 6, 3, 3)),  # ... and of 16
+    ("4,1,16,0,32,4", cs("split4_1x1_s2", 32, 192, 64, 5, 5, 1, 1, 2, 2)),  # strided 1x1 view, 12 chunks: 3 per CTA
 ], ids=lambda v: v.name if hasattr(v, "name") else None)
 def test_halo_split_channels_over_a_cta_pair(monkeypatch, force, c, out_dtype):
-    """split = 2: a cluster of two CTAs shares each tile, half of the channels each; the partial sums
-    cross through distributed shared memory.  Every output must still be Eq. 1."""
+    """split = 2 or 4: a cluster of that many CTAs shares each tile, an equal share of the channels
+    each; the partial sums cross through distributed shared memory.  Every output must still be
+    Eq. 1."""
     monkeypatch.setenv("CCONV_FORCE_TILE", force)
     info = check_full(c, variant=binding.VARIANT_HALO, out_dtype=out_dtype)
-    assert info["grid"] == 2 * info["tiles"]
+    assert info["split"] == int(force.split(",")[5]) and info["grid"] == info["split"] * info["tiles"]
 
 
 def test_tail_is_planned_for_the_large_config():
@@ -669,12 +675,10 @@ def test_accumulate_adds_the_convolution_to_what_out_holds(variant, c, out_dtype
     cs("autosplit_b64_3x3", 64, 256, 128, 6, 5, 3, 3),           # blocks of 64 images, one pixel per tile
     cs("autosplit_b24_s2", 24, 512, 64, 5, 4, 3, 3, 2, 1),       # B % 32 != 0, strides
     cs("autosplit_b40_4x4", 40, 160, 136, 4, 4, 4, 4),           # C = 160: ten 16-channel chunks, five per CTA
-    cs("autosplit_b8_blocks_of_8", 8, 512, 512, 7, 7, 3, 3),     # batch blocks of 8 images: 4 pixels per 32 columns
-    cs("autosplit_b16_blocks_of_16", 16, 256, 136, 7, 6, 5, 5),  # ... of 16 images: 2 pixels per 32 columns
+    cs("autosplit_b8", 8, 512, 512, 7, 7, 3, 3),                 # batch blocks of 8 images, four CTAs per tile
+    cs("autosplit_b16_5x5", 16, 256, 136, 7, 6, 5, 5),
 ], ids=lambda c: c.name)
 def test_planner_splits_channels_over_cta_pairs_on_small_grids(c, out_dtype):
     info = check_full(c, variant=binding.VARIANT_AUTO, out_dtype=out_dtype)
-    assert info["variant"] == binding.VARIANT_HALO and info["split"] == 2
-    assert info["grid"] == 2 * info["tiles"]
-    if "blocks_of" in c.name:
-        assert info["bb"] == int(c.name.rsplit("_", 1)[1])
+    assert info["variant"] == binding.VARIANT_HALO and info["split"] in (2, 4)
+    assert info["grid"] == info["split"] * info["tiles"]
