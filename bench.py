@@ -246,6 +246,60 @@ def time_repeats(cfg, torch, binding, dev, launches, repeats=5):
     return result[0], result[1], info, graph_s
 
 
+def time_general_shapes(torch, binding, dev, launches=30, repeats=3):
+    """Shapes outside the five benchmark configurations that exercise the planner's other paths:
+    tiles split over clusters of 2 or 4 CTAs (few output pixels, long channel loops) and bands of
+    output rows standing in for images (B < 8).  Each shape is timed twice, back-to-back calls on one
+    buffer set: as planned, and with that path switched off through the planner's diagnostic
+    environment variables (read at plan creation)."""
+    shapes = [("resnet50_conv5_3x3_b64", (64, 512, 512, 7, 7, 3, 3, 1, 1), "CCONV_FORCE_TILE", "0,0,0,0,0,1"),
+              ("deep_7x7_3x3_b16", (16, 1024, 256, 7, 7, 3, 3, 1, 1), "CCONV_FORCE_TILE", "0,0,0,0,0,1"),
+              ("deep_7x7_5x5_b8", (8, 512, 512, 7, 7, 5, 5, 1, 1), "CCONV_FORCE_TILE", "0,0,0,0,0,1"),
+              ("single_image_56x56_3x3", (1, 256, 256, 56, 56, 3, 3, 1, 1), "CCONV_BANDS", "1")]
+    stream = torch.cuda.current_stream()
+    sp = stream.cuda_stream
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    rows = []
+    for name, dims, var, off in shapes:
+        c = ConvShape(name, *dims)
+        ib, fb = make_inputs(c)
+        img, flt = to_dev(ib, torch, dev), to_dev(fb, torch, dev)
+        out = torch.empty(c.out_shape, dtype=torch.bfloat16, device=dev)
+        res = {}
+        for label, value in (("planned", None), ("path_off", off)):
+            saved = os.environ.get(var)
+            if value is None:
+                os.environ.pop(var, None)
+            else:
+                os.environ[var] = value
+            try:
+                plan = binding.Plan(*dims, device=dev.index, out_dtype=binding.OUT_BF16)
+            finally:
+                if saved is None:
+                    os.environ.pop(var, None)
+                else:
+                    os.environ[var] = saved
+            times = []
+            for rep in range(repeats + 1):
+                torch.cuda.synchronize()
+                e0.record(stream)
+                for _ in range(launches):
+                    plan.forward_ptrs(img.data_ptr(), flt.data_ptr(), out.data_ptr(), sp)
+                e1.record(stream)
+                torch.cuda.synchronize()
+                if rep:
+                    times.append(e0.elapsed_time(e1) * 1e3 / launches)
+            plan.check()
+            info = plan.info()
+            plan.close()
+            res[label] = {"us_per_launch": float(np.median(times)), "split": info["split"],
+                          "bands": info["bands"], "grid": info["grid"],
+                          "tile": [info[k] for k in ("bb", "bw", "bh", "bc")]}
+        rows.append({"workload": name, "dims": dict(zip("B C K W H R S sw sh".split(), dims)),
+                     "tflops": c.flops / res["planned"]["us_per_launch"] / 1e6, **res})
+    return rows
+
+
 def time_pooling(torch, binding, dev, peaks, launches=50, repeats=5):
     """Pooling (Section 6) rows: median CUDA-event time of back-to-back cconv_pool_forward calls over
     rotating buffer sets larger than L2.  Algorithmic bytes = Image + Out, each moved once; the
@@ -593,6 +647,7 @@ def main():
                              "oracle": oracle_sample(c)})
             line["all_configs"] = rows
             line["pooling"] = time_pooling(torch, binding, dev, peaks)
+            line["general_shapes"] = time_general_shapes(torch, binding, dev)
             line["cpu_baseline"] = cpu_baseline(cfg)
     if rank == 0:
         print(json.dumps(line))
