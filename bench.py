@@ -498,13 +498,22 @@ def cpu_baseline(cfg, budget_s=20.0):
                       f"pass(es), fp64 with the |.| sum"}
 
 
+def chosen_config(args):
+    if args.shape:
+        dims = tuple(int(v) for v in args.shape.split(","))
+        if len(dims) != 9 or min(dims) <= 0:
+            raise SystemExit("--shape wants nine positive integers: B,C,K,W,H,R,S,sw,sh")
+        return ConvShape("shape_" + "x".join(str(v) for v in dims), *dims)
+    return CONFIGS[args.config]
+
+
 def run_reference(args):
     """--impl reference: the CPU oracle on host cores, bounded sample per step."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return 0
     from oracle import cnn as ocnn
-    cfg = CONFIGS[args.config]
+    cfg = chosen_config(args)
     ib, fb = make_inputs(cfg)
     threads = ocnn.max_threads()
     total = args.steps + args.warmup
@@ -546,6 +555,9 @@ def main():
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--config", type=int, default=1, help="index into the five benchmark shapes")
+    ap.add_argument("--shape", default=None,
+                    help="B,C,K,W,H,R,S,sw,sh: time this shape instead of a benchmark configuration "
+                         "(same input recipe as the default configuration; no profile figures exist for it)")
     ap.add_argument("--impl", default="cconv", choices=["cconv", "reference"])
     ap.add_argument("--no-extras", action="store_true",
                     help="skip the per-configuration table, the e2e leg and the CPU baseline")
@@ -571,7 +583,7 @@ def main():
         dist = dist_mod
 
     peaks = measured_peaks()
-    cfg = CONFIGS[args.config]
+    cfg = chosen_config(args)
     steps, warmup = max(1, args.steps), max(3, args.warmup)
     sampler = ClockSampler(local)
     secs, info, nsets = time_config(cfg, torch, binding, dev, steps, warmup, dist, sampler)
