@@ -461,6 +461,51 @@ def test_planned_forward_and_pooling_inside_a_cuda_graph():
     plan.close()
 
 
+def test_split_banded_and_accumulating_calls_inside_a_cuda_graph():
+    """The other launch shapes survive capture too: a cluster launch of four CTAs per tile, a call on
+    banded copies (padding kernel, convolution, compaction kernel) and an accumulating call (the
+    twin's kernels plus the add kernel), captured once and replayed on new inputs."""
+    c4 = cs("graph_split4", 16, 512, 128, 7, 6, 3, 3)
+    c1 = cs("graph_bands", 1, 64, 64, 12, 16, 3, 3)
+    jobs = []
+    for c in (c4, c1):
+        ib, fb = synth.make_inputs(c)
+        jobs.append([c, to_dev(ib), to_dev(fb),
+                     torch.full(c.out_shape, float("nan"), device="cuda", dtype=torch.float32),
+                     binding.Plan(*c.dims(), device=0, out_dtype=binding.OUT_F32)])
+    assert jobs[0][4].info()["split"] == 4 and jobs[1][4].info()["bands"] == 8
+    acc = torch.zeros(c4.out_shape, device="cuda", dtype=torch.float32)
+    jobs[0][4].reserve_accumulate()
+    for c, img, flt, out, plan in jobs:
+        plan.forward(img, flt, out)           # warm-up outside the capture
+        plan.check()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.graph(graph, stream=side):
+        for c, img, flt, out, plan in jobs:
+            plan.forward(img, flt, out)
+        jobs[0][4].forward_accumulate(jobs[0][1], jobs[0][2], acc)
+    for seed in (91, 92):
+        exps = []
+        for c, img, flt, out, plan in jobs:
+            ib2, fb2 = synth.make_inputs(ConvShape(c.name, *c.dims(), seed=seed))
+            img.copy_(to_dev(ib2))
+            flt.copy_(to_dev(fb2))
+            out.fill_(float("nan"))
+            exps.append(ocnn.cnn_bf16(ib2, fb2, oshape(c)))
+        acc.fill_(2.5)
+        graph.replay()
+        torch.cuda.synchronize()
+        for (c, img, flt, out, plan), (exp, ab) in zip(jobs, exps):
+            assert_close(out.cpu().numpy().astype(np.float64), exp, ab, what=f"{c.name}, seed {seed}")
+        assert_close(acc.cpu().numpy().astype(np.float64), exps[0][0] + 2.5, exps[0][1] + 2.5,
+                     what=f"accumulate in a graph, seed {seed}")
+    for job in jobs:
+        job[4].check()
+        job[4].close()
+
+
 def test_mixed_plans_and_pooling_back_to_back_without_synchronisation():
     """Sixty calls of five plans (three kernel variants) and a pooling kernel on one stream, in a
     seeded random order, each with its own Filter and Out and no synchronisation in between: every
