@@ -50,8 +50,15 @@ struct BandGeom {
 };
 
 // (one thread per 16 bytes of the copy: 8 images of one (x, y, c))
+// Launched behind the Filter-packing kernel of the same call with programmatic stream
+// serialisation, so that the two (which share no data) run side by side; it ends with a dependency
+// wait, so that "this kernel is complete" implies that the packing kernel is, which is what the
+// convolution behind it relies on.  `wait_first`: the caller's Image may still be being written by
+// the kernel in front (the host's overlap check), so nothing is read before that one is complete.
 __global__ void __launch_bounds__(256) cconv_pad_bands_kernel(const unsigned short* __restrict__ src,
-                                                              uint4* __restrict__ dst, BandGeom g) {
+                                                              uint4* __restrict__ dst, BandGeom g,
+                                                              int wait_first) {
+  if (wait_first) asm volatile("griddepcontrol.wait;" ::: "memory");
   const int gpb = g.Bp / 8;
   const long long n = g.Wi * g.Hir * g.C * gpb;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n;
@@ -73,6 +80,7 @@ __global__ void __launch_bounds__(256) cconv_pad_bands_kernel(const unsigned sho
     dst[i] = make_uint4(e[0] | (e[1] << 16), e[2] | (e[3] << 16), e[4] | (e[5] << 16),
                         e[6] | (e[7] << 16));
   }
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 // The way back: Out [K][H][W][B] of the caller from [K][Hr][W][Bp] of the banded run (T = bf16 bits
@@ -242,8 +250,26 @@ std::map<std::tuple<int, int, int, int, int, int, int, int, int, int, int>, ccon
 }  // namespace
 
 // The tensor-core launches of one forward call (Image and Out already padded if need be).
+// `pad` (padded plans): the caller's Image is copied into the plan's padded array between the
+// packing kernel and the convolution, and `Image` is that array.
+static cudaError_t launch_pad(const void* user_image, void* padded, const BandGeom& g, bool wait_first,
+                              cudaStream_t stream) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid_for(g.Wi * g.Hir * g.C * (g.Bp / 8)));
+  cfg.blockDim = dim3(256);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, cconv_pad_bands_kernel, static_cast<const unsigned short*>(user_image),
+                            static_cast<uint4*>(padded), g, wait_first ? 1 : 0);
+}
+
 static int launch_tensor_core(const cconv_plan* pl, const void* Image, const void* Filter, void* Out,
-                              bool image_overlaps_last_out, cudaStream_t stream) {
+                              bool image_overlaps_last_out, cudaStream_t stream,
+                              const BandGeom* pad = nullptr, const void* user_image = nullptr) {
   CUtensorMap tmi, tmi_tail;
   void* packed = nullptr;
   {
@@ -265,15 +291,24 @@ static int launch_tensor_core(const cconv_plan* pl, const void* Image, const voi
   if (pl->variant == CCONV_VARIANT_STEM) {
     cudaError_t es = launch_pack_filter_stem(Filter, packed, pl->d, pl->skp, stream);
     if (es != cudaSuccess) return cuda_fail(es, "launch_pack_filter_stem");
+    if (pad) {
+      es = launch_pad(user_image, pl->d_img_pad, *pad, image_overlaps_last_out, stream);
+      if (es != cudaSuccess) return cuda_fail(es, "cconv_pad_bands_kernel");
+    }
     es = launch_stem(tmi, packed, Out, pl->out_dtype == CCONV_OUT_F32, pl->skp, pl->stile.grid,
                      pl->stile.smem_bytes, pl->d_status, stream);
     return es == cudaSuccess ? CCONV_OK : cuda_fail(es, "launch_stem");
   }
   HaloKernelParams kp = pl->kp;
-  kp.image_wait = image_overlaps_last_out ? 1 : 0;
+  // (a padded Image is written by the kernel right in front of the convolution)
+  kp.image_wait = (image_overlaps_last_out || pad) ? 1 : 0;
   cudaError_t e = launch_pack_filter(Filter, packed, pl->d, pl->tile.c16, pl->tile.tiles_k,
                                      /*overlap_prev=*/true, stream);
   if (e != cudaSuccess) return cuda_fail(e, "launch_pack_filter");
+  if (pad) {
+    e = launch_pad(user_image, pl->d_img_pad, *pad, image_overlaps_last_out, stream);
+    if (e != cudaSuccess) return cuda_fail(e, "cconv_pad_bands_kernel");
+  }
   e = launch_halo(tmi, packed, Out, pl->out_dtype == CCONV_OUT_F32, kp, pl->tile.grid,
                   pl->tile.smem_bytes, pl->d_status, stream);
   if (e == cudaSuccess && pl->has_tail)
@@ -672,18 +707,16 @@ int cconv_forward_planned(const cconv_plan* pl, const void* Image, const void* F
   }
   // Batch sizes that are not multiples of 8: the kernels run on zero-padded copies (see cconv_plan).
   void* const user_out = Out;
+  const void* const user_image = Image;
   BandGeom g{};
   if (pl->padded) {
     const Dims& r = pl->drun;
     g = BandGeom{pl->d.Wi(), pl->d.Hi(), r.Hi(), pl->d.C, pl->d.B, r.B, pl->bands, r.H, pl->d.sh};
-    cconv_pad_bands_kernel<<<grid_for(g.Wi * g.Hir * g.C * (g.Bp / 8)), 256, 0, stream>>>(
-        static_cast<const unsigned short*>(Image), static_cast<uint4*>(pl->d_img_pad), g);
-    cudaError_t ep = cudaGetLastError();
-    if (ep != cudaSuccess) return cuda_fail(ep, "cconv_pad_bands_kernel");
     Image = pl->d_img_pad;
     Out = pl->d_out_pad;
   }
-  const int rc_run = launch_tensor_core(pl, Image, Filter, Out, image_overlaps_last_out, stream);
+  const int rc_run = launch_tensor_core(pl, Image, Filter, Out, image_overlaps_last_out, stream,
+                                        pl->padded ? &g : nullptr, user_image);
   if (rc_run != CCONV_OK || !pl->padded) return rc_run;
   {
     const Dims& d = pl->d;
