@@ -91,6 +91,9 @@ __global__ void __launch_bounds__(256) cconv_compact_bands_kernel(const T* __res
                                                                   T* __restrict__ dst, long long K,
                                                                   long long H, long long W,
                                                                   BandGeom g) {
+  // launched with programmatic stream serialisation: resident early, working once the convolution
+  // in front is complete
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int gpb = g.Bp / 8;
   const long long n = K * g.Hr * W * gpb;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n;
@@ -720,17 +723,28 @@ int cconv_forward_planned(const cconv_plan* pl, const void* Image, const void* F
   if (rc_run != CCONV_OK || !pl->padded) return rc_run;
   {
     const Dims& d = pl->d;
-    const unsigned grid = grid_for((long long)d.K * g.Hr * d.W * (g.Bp / 8));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid_for((long long)d.K * g.Hr * d.W * (g.Bp / 8)));
+    cfg.blockDim = dim3(256);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t ec;
     if (pl->out_dtype == CCONV_OUT_F32)
-      cconv_compact_bands_kernel<float><<<grid, 256, 0, stream>>>(
-          static_cast<const float*>(Out), static_cast<float*>(user_out), d.K, d.H, d.W, g);
+      ec = cudaLaunchKernelEx(&cfg, cconv_compact_bands_kernel<float>, static_cast<const float*>(Out),
+                              static_cast<float*>(user_out), (long long)d.K, (long long)d.H,
+                              (long long)d.W, g);
     else
-      cconv_compact_bands_kernel<unsigned short><<<grid, 256, 0, stream>>>(
-          static_cast<const unsigned short*>(Out), static_cast<unsigned short*>(user_out), d.K, d.H,
-          d.W, g);
-    cudaError_t ec = cudaGetLastError();
+      ec = cudaLaunchKernelEx(&cfg, cconv_compact_bands_kernel<unsigned short>,
+                              static_cast<const unsigned short*>(Out),
+                              static_cast<unsigned short*>(user_out), (long long)d.K, (long long)d.H,
+                              (long long)d.W, g);
     if (ec != cudaSuccess) return cuda_fail(ec, "cconv_compact_bands_kernel");
-    // the compaction kernel is an ordinary launch: nothing behind it starts before it is complete
+    // the compaction kernel never releases its dependents early: nothing behind it starts before it
+    // is complete
     std::lock_guard<std::mutex> lk(g_last_out_mu);
     g_last_out.valid = false;
   }
