@@ -66,6 +66,59 @@ __global__ void __launch_bounds__(256) cconv_simt_kernel(const __nv_bfloat16* __
   }
 }
 
+// Tiny problems: the time of the kernel above is one thread's chain of dependent loads (C*R*S of
+// them, a few in flight at a time).  Here eight lanes share one output element, lane j taking the
+// filter taps j, j+8, ... with all channels of a tap loaded before the first use, and a three-step
+// shuffle tree adds the eight partial sums (fixed order: results are reproducible run to run).
+template <typename OutT>
+__global__ void __launch_bounds__(128) cconv_simt_taps_kernel(const __nv_bfloat16* __restrict__ image,
+                                                              const __nv_bfloat16* __restrict__ filter,
+                                                              OutT* __restrict__ out, Dims d) {
+  const long long total = (long long)d.K * d.H * d.W * d.B;
+  const long long Hi = (long long)d.sh * (d.H - 1) + d.S;
+  const int sub = threadIdx.x & 7;
+  const int RS = d.R * d.S;
+  const long long groups_per_grid = (long long)gridDim.x * (blockDim.x >> 3);
+  // the loop bound is the same for all lanes of a warp (its four groups are consecutive)
+  for (long long base = (blockIdx.x * (long long)blockDim.x + (threadIdx.x & ~31)) >> 3; base < total;
+       base += groups_per_grid) {
+    const long long idx = base + ((threadIdx.x & 31) >> 3);
+    const bool valid = idx < total;
+    float acc = 0.f;
+    if (valid) {
+      const int b = int(idx % d.B);
+      long long t = idx / d.B;
+      const int w = int(t % d.W);
+      t /= d.W;
+      const int h = int(t % d.H);
+      const int k = int(t / d.H);
+      for (int tap = sub; tap < RS; tap += 8) {
+        const int r = tap / d.S, s = tap - r * d.S;
+        const __nv_bfloat16* ip =
+            image + (((long long)(r + d.sw * w) * Hi + (s + d.sh * h)) * d.C) * d.B + b;
+        const __nv_bfloat16* fp = filter + ((long long)k * RS + tap) * d.C;
+        int c = 0;
+        for (; c + 8 <= d.C; c += 8) {
+          float x[8], f[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            x[j] = __bfloat162float(ip[(long long)(c + j) * d.B]);
+            f[j] = __bfloat162float(fp[c + j]);
+          }
+#pragma unroll
+          for (int j = 0; j < 8; ++j) acc = fmaf(x[j], f[j], acc);
+        }
+        for (; c < d.C; ++c)
+          acc = fmaf(__bfloat162float(ip[(long long)c * d.B]), __bfloat162float(fp[c]), acc);
+      }
+    }
+    acc += __shfl_xor_sync(0xffffffffu, acc, 4);
+    acc += __shfl_xor_sync(0xffffffffu, acc, 2);
+    acc += __shfl_xor_sync(0xffffffffu, acc, 1);
+    if (valid && sub == 0) store_out(out + idx, acc);
+  }
+}
+
 cudaError_t launch_simt(const void* image, const void* filter, void* out, bool out_f32,
                         const Dims& d, cudaStream_t stream) {
   // Four out-channels per thread reuse each Image value four times; problems too small to fill
@@ -81,6 +134,16 @@ cudaError_t launch_simt(const void* image, const void* filter, void* out, bool o
   if (blocks < 1) blocks = 1;
   const __nv_bfloat16* im = static_cast<const __nv_bfloat16*>(image);
   const __nv_bfloat16* fl = static_cast<const __nv_bfloat16*>(filter);
+  // eight lanes per output while that still leaves the SMs room for every thread at once
+  if (outputs * 8 <= 148ll * 2048 && d.R * d.S >= 4) {
+    const long long tblocks = (outputs * 8 + 127) / 128;
+    if (out_f32)
+      cconv_simt_taps_kernel<float><<<(unsigned)tblocks, 128, 0, stream>>>(im, fl, static_cast<float*>(out), d);
+    else
+      cconv_simt_taps_kernel<__nv_bfloat16><<<(unsigned)tblocks, 128, 0, stream>>>(
+          im, fl, static_cast<__nv_bfloat16*>(out), d);
+    return cudaGetLastError();
+  }
   if (small) {
     if (out_f32)
       cconv_simt_kernel<1, float><<<(unsigned)blocks, threads, 0, stream>>>(
