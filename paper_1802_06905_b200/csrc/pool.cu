@@ -129,10 +129,14 @@ __global__ void __launch_bounds__(256) cconv_pool_kernel(const __nv_bfloat16* __
     // the maximum of bf16 values is taken on the packed pairs themselves (exact), 4 ops per vector
     const __nv_bfloat162 ninf = __floats2bfloat162_rn(-INFINITY, -INFINITY);
     __nv_bfloat162 m[4] = {ninf, ninf, ninf, ninf};
-    for (; t + (U - 1) * G < p.terms; t += U * G) {
+    // (the last round is a full round with some loads switched off, not a loop of single loads:
+    // every round costs a memory latency)
+    const uint4 ninf4 = make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
+    for (; t < p.terms; t += U * G) {
       uint4 q[U];
 #pragma unroll
-      for (int u = 0; u < U; ++u) q[u] = __ldg(reinterpret_cast<const uint4*>(next_ptr()));
+      for (int u = 0; u < U; ++u)
+        q[u] = (t + u * G < p.terms) ? __ldg(reinterpret_cast<const uint4*>(next_ptr())) : ninf4;
 #pragma unroll
       for (int u = 0; u < U; ++u) {
         m[0] = __hmax2(m[0], *reinterpret_cast<const __nv_bfloat162*>(&q[u].x));
@@ -141,19 +145,14 @@ __global__ void __launch_bounds__(256) cconv_pool_kernel(const __nv_bfloat16* __
         m[3] = __hmax2(m[3], *reinterpret_cast<const __nv_bfloat162*>(&q[u].w));
       }
     }
-    for (; t < p.terms; t += G) {
-      const uint4 q = __ldg(reinterpret_cast<const uint4*>(next_ptr()));
-      m[0] = __hmax2(m[0], *reinterpret_cast<const __nv_bfloat162*>(&q.x));
-      m[1] = __hmax2(m[1], *reinterpret_cast<const __nv_bfloat162*>(&q.y));
-      m[2] = __hmax2(m[2], *reinterpret_cast<const __nv_bfloat162*>(&q.z));
-      m[3] = __hmax2(m[3], *reinterpret_cast<const __nv_bfloat162*>(&q.w));
-    }
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       acc[2 * i] = __low2float(m[i]);
       acc[2 * i + 1] = __high2float(m[i]);
     }
   } else {
+    // (sums: a predicated last round was measured slower here -- 14.9 -> 16.6 us on the seven-loop
+    // benchmark shape -- so the remainder goes load by load)
     for (; t + (U - 1) * G < p.terms; t += U * G) {
       float x[U][VEC];
 #pragma unroll
@@ -198,6 +197,70 @@ __global__ void __launch_bounds__(256) cconv_pool_kernel(const __nv_bfloat16* __
   const int k1 = min(p.K, k0 + p.kper);
   for (int k = k0 + g; k < k1; k += G)
     store_vec<OutT, VEC>(out + ((long long)k * p.total_v + v) * VEC, acc);
+}
+
+// The usual pooling layer (C = 1 with the channels folded into b, 8 images per thread, a 2x2 or
+// 3x3 window): a thread per output vector with the whole window loaded before the first use -- no
+// term stepping, 32-bit index arithmetic -- then the K planes written in turn.  The general kernel
+// above takes a 3x3 window in two rounds of loads (eight, then one) and ran 25 % slower on it.
+template <typename OutT, int R, int S, bool MAX>
+__global__ void __launch_bounds__(256) cconv_pool_window_kernel(const __nv_bfloat16* __restrict__ image,
+                                                                OutT* __restrict__ out, PoolParams p) {
+  const unsigned v = blockIdx.x * 256u + threadIdx.x;   // the host sends total_v < 2^31 here
+  if (v >= unsigned(p.total_v)) return;
+  const unsigned pix = v / unsigned(p.nb), bv = v - pix * unsigned(p.nb);
+  const unsigned h = pix / unsigned(p.W), w = pix - h * unsigned(p.W);
+  const long long ystride = (long long)p.B, xstride = (long long)p.Hi * p.B;
+  const __nv_bfloat16* base =
+      image + ((long long)p.sw * w * p.Hi + (long long)p.sh * h) * p.B + (long long)bv * 8;
+  uint4 q[R * S];
+#pragma unroll
+  for (int r = 0; r < R; ++r)
+#pragma unroll
+    for (int s = 0; s < S; ++s)
+      q[r * S + s] = __ldg(reinterpret_cast<const uint4*>(base + r * xstride + s * ystride));
+  float acc[8];
+  if constexpr (MAX) {
+    __nv_bfloat162 m[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) m[i] = reinterpret_cast<const __nv_bfloat162*>(&q[0])[i];
+#pragma unroll
+    for (int t = 1; t < R * S; ++t)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) m[i] = __hmax2(m[i], reinterpret_cast<const __nv_bfloat162*>(&q[t])[i]);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      acc[2 * i] = __low2float(m[i]);
+      acc[2 * i + 1] = __high2float(m[i]);
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+#pragma unroll
+    for (int t = 0; t < R * S; ++t) {
+      const uint32_t u[4] = {q[t].x, q[t].y, q[t].z, q[t].w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        acc[2 * i] += __uint_as_float(u[i] << 16);
+        acc[2 * i + 1] += __uint_as_float(u[i] & 0xffff0000u);
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc[i] *= p.inv_rs;
+  }
+  const int k0 = blockIdx.y * p.kper;
+  const int k1 = min(p.K, k0 + p.kper);
+  for (int k = k0; k < k1; ++k) store_vec<OutT, 8>(out + ((long long)k * p.total_v + v) * 8, acc);
+}
+
+template <typename OutT, int R, int S>
+cudaError_t launch_pool_window(const void* image, void* out, const PoolParams& p, bool mx, dim3 grid,
+                               cudaStream_t stream) {
+  const __nv_bfloat16* im = static_cast<const __nv_bfloat16*>(image);
+  OutT* o = static_cast<OutT*>(out);
+  if (mx) cconv_pool_window_kernel<OutT, R, S, true><<<grid, 256, 0, stream>>>(im, o, p);
+  else cconv_pool_window_kernel<OutT, R, S, false><<<grid, 256, 0, stream>>>(im, o, p);
+  return cudaGetLastError();
 }
 
 template <typename OutT, int VEC, bool MAX>
@@ -283,7 +346,16 @@ extern "C" int cconv_pool_forward(const void* Image, void* Out, int B, int C, in
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   const bool f32 = out_dtype == CCONV_OUT_F32, mx = op == CCONV_POOL_MAX;
   cudaError_t e;
-  if (vec == 8) {
+  const bool window33 = R == 3 && S == 3, window22 = R == 2 && S == 2;
+  if (C == 1 && vec == 8 && vpb == 256 && (window33 || window22) && p.total_v < 0x7fffffffll &&
+      !std::getenv("CCONV_POOL_FORCE")) {
+    if (window33)
+      e = f32 ? launch_pool_window<float, 3, 3>(Image, Out, p, mx, grid, stream)
+              : launch_pool_window<__nv_bfloat16, 3, 3>(Image, Out, p, mx, grid, stream);
+    else
+      e = f32 ? launch_pool_window<float, 2, 2>(Image, Out, p, mx, grid, stream)
+              : launch_pool_window<__nv_bfloat16, 2, 2>(Image, Out, p, mx, grid, stream);
+  } else if (vec == 8) {
     if (f32) e = mx ? launch_pool_t<float, 8, true>(Image, Out, p, vpb, grid, stream)
                     : launch_pool_t<float, 8, false>(Image, Out, p, vpb, grid, stream);
     else e = mx ? launch_pool_t<__nv_bfloat16, 8, true>(Image, Out, p, vpb, grid, stream)

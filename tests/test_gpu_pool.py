@@ -30,6 +30,9 @@ SHAPES = [
     Shape(B=3, C=40, K=70, W=4, H=4, R=2, S=3, sw=3, sh=1),      # scalar + cooperative + k split
     Shape(B=16, C=64, K=130, W=3, H=2, R=3, S=3, sw=1, sh=1),    # few pixels, many planes: k split
     Shape(B=128, C=2, K=3, W=33, H=17, R=5, S=4, sw=2, sh=3),    # several blocks of 256 vectors
+    Shape(B=72, C=1, K=1, W=13, H=9, R=3, S=3, sw=2, sh=2),      # window kernel: 3x3 stride 2, ragged last block
+    Shape(B=16, C=1, K=3, W=7, H=6, R=3, S=3, sw=1, sh=3),       # window kernel: overlapping columns, 3 planes
+    Shape(B=8, C=1, K=2, W=5, H=40, R=2, S=2, sw=1, sh=1),       # window kernel: 2x2 stride 1
 ]
 
 
