@@ -136,7 +136,29 @@ template <typename T>
 __global__ void __launch_bounds__(256) cconv_accumulate_kernel(T* __restrict__ out,
                                                                const float* __restrict__ conv,
                                                                long long n) {
-  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n;
+  // four elements per thread and step (Out is 32-byte aligned, the fp32 array 256), the last n % 4
+  // one by one
+  const long long n4 = n >> 2;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n4;
+       i += (long long)gridDim.x * blockDim.x) {
+    const float4 c = reinterpret_cast<const float4*>(conv)[i];
+    T* o = out + 4 * i;
+    if constexpr (sizeof(T) == 4) {
+      float4 v = *reinterpret_cast<float4*>(o);
+      v.x += c.x; v.y += c.y; v.z += c.z; v.w += c.w;
+      *reinterpret_cast<float4*>(o) = v;
+    } else {
+      uint2 raw = *reinterpret_cast<uint2*>(o);
+      __nv_bfloat162 a = *reinterpret_cast<__nv_bfloat162*>(&raw.x);
+      __nv_bfloat162 b = *reinterpret_cast<__nv_bfloat162*>(&raw.y);
+      a = __floats2bfloat162_rn(__low2float(a) + c.x, __high2float(a) + c.y);
+      b = __floats2bfloat162_rn(__low2float(b) + c.z, __high2float(b) + c.w);
+      raw.x = *reinterpret_cast<uint32_t*>(&a);
+      raw.y = *reinterpret_cast<uint32_t*>(&b);
+      *reinterpret_cast<uint2*>(o) = raw;
+    }
+  }
+  for (long long i = 4 * n4 + blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n;
        i += (long long)gridDim.x * blockDim.x)
     out[i] = add_round<T>(out[i], conv[i]);
 }
@@ -681,9 +703,9 @@ int cconv_forward_accumulate(const cconv_plan* pl, const void* Image, const void
   const Dims& d = pl->d;
   const long long n = (long long)d.K * d.H * d.W * d.B;
   if (pl->out_dtype == CCONV_OUT_F32)
-    cconv_accumulate_kernel<float><<<grid_for(n), 256, 0, stream>>>(static_cast<float*>(Out), pl->d_acc, n);
+    cconv_accumulate_kernel<float><<<grid_for((n + 3) / 4), 256, 0, stream>>>(static_cast<float*>(Out), pl->d_acc, n);
   else
-    cconv_accumulate_kernel<__nv_bfloat16><<<grid_for(n), 256, 0, stream>>>(
+    cconv_accumulate_kernel<__nv_bfloat16><<<grid_for((n + 3) / 4), 256, 0, stream>>>(
         static_cast<__nv_bfloat16*>(Out), pl->d_acc, n);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e, "cconv_accumulate_kernel");
