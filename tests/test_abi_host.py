@@ -326,3 +326,25 @@ def test_random_shapes_plan_to_hardware_legal_tiles():
             # the CUDA-core kernel is left only with tiny problems whose batch is not a multiple of 8
             assert B % 8 != 0 and B * C * K * W * H * R * S < 4e6 or Bp != B
     assert all(v > 0 for v in seen.values()), seen
+
+
+def test_planner_split_rule():
+    """Tiles are split over clusters of 2 or 4 CTAs only for filters of 9 or more taps with long channel
+    loops and few output pixels; the benchmark shapes, 1x1 filters and short loops stay whole; four
+    CTAs per tile need 288 units (C*R*S >= 4608)."""
+    def split_of(*dims):
+        p = binding.Plan(*dims, device=-1)
+        info = p.info()
+        p.close()
+        return info["split"], info
+    for cfg in CONFIGS:
+        assert split_of(*cfg.dims())[0] == 1, cfg.name
+    assert split_of(64, 512, 512, 7, 7, 3, 3, 1, 1)[0] == 2          # ResNet-50 conv5: 56 tiles x 2
+    assert split_of(16, 1024, 256, 7, 7, 3, 3, 1, 1)[0] == 4         # 576 units: a quarter each
+    assert split_of(16, 256, 256, 7, 7, 3, 3, 1, 1)[0] == 2          # 144 units: too short for four
+    assert split_of(8, 512, 512, 7, 7, 5, 5, 1, 1)[0] == 4
+    assert split_of(16, 128, 128, 7, 7, 3, 3, 1, 1)[0] == 1          # 72 units: stays whole
+    assert split_of(16, 2048, 512, 7, 7, 1, 1, 1, 1)[0] == 1         # 1x1 filters stay whole
+    assert split_of(64, 256, 256, 14, 14, 3, 3, 1, 1)[0] == 1        # enough pixels: whole tiles fill the SMs
+    s, info = split_of(32, 1024, 256, 4, 4, 3, 3, 1, 1)
+    assert s == 4 and info["grid"] == 4 * info["tiles"] <= 128
