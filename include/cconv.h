@@ -57,6 +57,9 @@ extern "C" {
                                 images (the last one zero padded past B), or of 16 or 8 images     */
 #define CCONV_VARIANT_STEM 3 /* small C: (s,c) folded into the MMA contraction; needs the whole
                                 (shifted, padded) Filter resident in shared memory               */
+#define CCONV_VARIANT_DIRECT 4 /* as HALO, but the Filter is staged straight from [K][R][S][C] by TMA:
+                                  one launch per call, no scratch; b_k = 128 or 256; needs B % 8 == 0
+                                  and C % 8 == 0 (no padded copies)                                */
 /* The tensor-core kernels need B % 8 == 0.  For other batch sizes a plan runs them on copies of
  * Image and Out padded to the next multiple of 8 (plan-owned scratch, one padding and one compaction
  * kernel per call); for B < 8 the copies also turn bands of output rows into images, so that a

@@ -17,7 +17,7 @@ _lib = None
 OK = 0
 EINVAL, EUNSUPPORTED, ECUDA, EDEVICE_TIMEOUT, ENOMEM, ETOOLARGE = -1, -2, -3, -4, -5, -6
 NOALLOC_MAX_SCRATCH_BYTES = 8 * 1024 * 1024
-VARIANT_AUTO, VARIANT_SIMT, VARIANT_HALO, VARIANT_STEM = 0, 1, 2, 3
+VARIANT_AUTO, VARIANT_SIMT, VARIANT_HALO, VARIANT_STEM, VARIANT_DIRECT = 0, 1, 2, 3, 4
 OUT_BF16, OUT_F32 = 0, 1
 POOL_AVG, POOL_MAX = 0, 1
 

@@ -13,7 +13,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcconv.so")
-SOURCES = ["kernels.cu", "stem_kernel.cu", "api.cu", "host_setup.cu", "noalloc.cu", "pool.cu", "planner.cpp"]
+SOURCES = ["kernels.cu", "direct_kernel.cu", "stem_kernel.cu", "api.cu", "host_setup.cu", "noalloc.cu", "pool.cu", "planner.cpp"]
 HEADERS = ["kernels.h", "planner.h", "host_setup.h", "ptx_sm100.cuh", os.path.join("..", "..", "include", "cconv.h")]
 
 

@@ -168,36 +168,6 @@ unsigned grid_for(long long n) {
   return unsigned(std::max<long long>(1, std::min<long long>(blocks, 148ll * 32)));
 }
 
-struct LastOut {
-  bool valid = false;
-  void* stream = nullptr;
-  const char* lo = nullptr;
-  const char* hi = nullptr;
-};
-LastOut g_last_out;
-std::mutex g_last_out_mu;
-
-// Records this call's Out as the latest one and says whether its Image overlaps the Out of the
-// tensor-core convolution launched just before it on the same stream.  Those kernels let their
-// successors start while they are still in their last tiles (that hides the launch gap), and the
-// halo kernel's Image producers read at once: wrong only in that one case, which the two layouts
-// make useless but do not forbid; the producers are then told to wait for the earlier call.
-bool note_call_and_check_overlap(const Dims& d, int out_dtype, const void* Image, const void* Out,
-                                 void* stream, bool early_start_kernel) {
-  const char* img_lo = static_cast<const char*>(Image);
-  const char* img_hi = img_lo + size_t(d.Wi()) * d.Hi() * d.C * d.B * 2;
-  const char* out_lo = static_cast<const char*>(Out);
-  const char* out_hi = out_lo + size_t(d.K) * d.H * d.W * d.B * (out_dtype == CCONV_OUT_F32 ? 4 : 2);
-  std::lock_guard<std::mutex> lk(g_last_out_mu);
-  const bool overlap = g_last_out.valid && g_last_out.stream == stream && g_last_out.lo < img_hi &&
-                       img_lo < g_last_out.hi;
-  g_last_out.valid = early_start_kernel;
-  g_last_out.stream = stream;
-  g_last_out.lo = out_lo;
-  g_last_out.hi = out_hi;
-  return overlap;
-}
-
 }  // namespace
 
 struct cconv_plan {
@@ -236,6 +206,8 @@ struct cconv_plan {
   HaloKernelParams kp_tail{};
   StemTile stile{};
   StemKernelParams skp{};
+  DirectTile dtile{};
+  DirectKernelParams dkp{};
   int* d_status = nullptr;
   // Scratch: the packed Filter, rewritten by every forward call.  Two buffers, used alternately:
   // the packing kernel of call n+1 may run while the convolution of call n still reads its buffer.
@@ -263,6 +235,8 @@ struct cconv_plan {
   mutable const void* tm_image_ptr = nullptr;
   mutable CUtensorMap tm_image{};
   mutable CUtensorMap tm_image_tail{};
+  mutable const void* tm_filter_ptr = nullptr;  // direct kernel: the Filter map
+  mutable CUtensorMap tm_filter{};
 };
 
 namespace {
@@ -293,7 +267,7 @@ static cudaError_t launch_pad(const void* user_image, void* padded, const BandGe
 }
 
 static int launch_tensor_core(const cconv_plan* pl, const void* Image, const void* Filter, void* Out,
-                              bool image_overlaps_last_out, cudaStream_t stream,
+                              bool inputs_hazard, cudaStream_t stream,
                               const BandGeom* pad = nullptr, const void* user_image = nullptr) {
   CUtensorMap tmi, tmi_tail;
   void* packed = nullptr;
@@ -314,10 +288,10 @@ static int launch_tensor_core(const cconv_plan* pl, const void* Image, const voi
     packed = static_cast<char*>(pl->d_packed) + (pl->calls++ & 1u) * pl->packed_bytes;
   }
   if (pl->variant == CCONV_VARIANT_STEM) {
-    cudaError_t es = launch_pack_filter_stem(Filter, packed, pl->d, pl->skp, stream);
+    cudaError_t es = launch_pack_filter_stem(Filter, packed, pl->d, pl->skp, !inputs_hazard, stream);
     if (es != cudaSuccess) return cuda_fail(es, "launch_pack_filter_stem");
     if (pad) {
-      es = launch_pad(user_image, pl->d_img_pad, *pad, image_overlaps_last_out, stream);
+      es = launch_pad(user_image, pl->d_img_pad, *pad, inputs_hazard, stream);
       if (es != cudaSuccess) return cuda_fail(es, "cconv_pad_bands_kernel");
     }
     es = launch_stem(tmi, packed, Out, pl->out_dtype == CCONV_OUT_F32, pl->skp, pl->stile.grid,
@@ -326,12 +300,13 @@ static int launch_tensor_core(const cconv_plan* pl, const void* Image, const voi
   }
   HaloKernelParams kp = pl->kp;
   // (a padded Image is written by the kernel right in front of the convolution)
-  kp.image_wait = (image_overlaps_last_out || pad) ? 1 : 0;
+  kp.image_wait = (inputs_hazard || pad) ? 1 : 0;
+  // (a Filter that the call in front may still be writing is not read before that call is complete)
   cudaError_t e = launch_pack_filter(Filter, packed, pl->d, pl->tile.c16, pl->tile.tiles_k,
-                                     /*overlap_prev=*/true, stream);
+                                     /*overlap_prev=*/!inputs_hazard, stream);
   if (e != cudaSuccess) return cuda_fail(e, "launch_pack_filter");
   if (pad) {
-    e = launch_pad(user_image, pl->d_img_pad, *pad, image_overlaps_last_out, stream);
+    e = launch_pad(user_image, pl->d_img_pad, *pad, inputs_hazard, stream);
     if (e != cudaSuccess) return cuda_fail(e, "cconv_pad_bands_kernel");
   }
   e = launch_halo(tmi, packed, Out, pl->out_dtype == CCONV_OUT_F32, kp, pl->tile.grid,
@@ -409,7 +384,7 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
   *plan_out = nullptr;
   const Dims d{B, C, K, W, H, R, S, sw, sh};
   if (!d.positive()) return CCONV_EINVAL;
-  if (variant < CCONV_VARIANT_AUTO || variant > CCONV_VARIANT_STEM) return CCONV_EINVAL;
+  if (variant < CCONV_VARIANT_AUTO || variant > CCONV_VARIANT_DIRECT) return CCONV_EINVAL;
   if (out_dtype != CCONV_OUT_BF16 && out_dtype != CCONV_OUT_F32) return CCONV_EINVAL;
   // element counts must fit the kernels' index arithmetic
   const double lim = 9.0e18;
@@ -458,11 +433,19 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
     std::sscanf(f, "%d,%d,%d,%d,%d,%d", &force[0], &force[1], &force[2], &force[3], &force[4],
                 &force[5]);
   const int env_variant = env_int("CCONV_VARIANT", 0);
-  if (variant == CCONV_VARIANT_AUTO && env_variant >= 1 && env_variant <= 3) variant = env_variant;
+  if (variant == CCONV_VARIANT_AUTO && env_variant >= 1 && env_variant <= 4) variant = env_variant;
+  int dforce[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
+  if (const char* f = std::getenv("CCONV_FORCE_DIRECT"))
+    std::sscanf(f, "%d,%d,%d,%d,%d,%d,%d,%d,%d", &dforce[0], &dforce[1], &dforce[2], &dforce[3],
+                &dforce[4], &dforce[5], &dforce[6], &dforce[7], &dforce[8]);
 
   const bool halo_ok = halo_supported(dk, nullptr) && choose_halo_tile(dk, pl->m, force, &pl->tile);
   const bool stem_ok = choose_stem_tile(pl->drun, pl->m, &pl->stile, env_int("CCONV_STEM_BW", 0));
-  if ((variant == CCONV_VARIANT_HALO && !halo_ok) || (variant == CCONV_VARIANT_STEM && !stem_ok)) {
+  // the direct-Filter kernel runs on the caller's arrays only (no padded copies)
+  const bool direct_ok = !pl->padded && direct_supported(dk, nullptr) &&
+                         choose_direct_tile(dk, pl->m, dforce, &pl->dtile);
+  if ((variant == CCONV_VARIANT_HALO && !halo_ok) || (variant == CCONV_VARIANT_STEM && !stem_ok) ||
+      (variant == CCONV_VARIANT_DIRECT && !direct_ok)) {
     delete pl;
     return CCONV_EUNSUPPORTED;
   }
@@ -510,6 +493,10 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
     build_halo_params(dk, pl->tile, &pl->kp);
   }
   if (variant == CCONV_VARIANT_STEM) build_stem_params(pl->drun, pl->stile, &pl->skp);
+  if (variant == CCONV_VARIANT_DIRECT) {
+    build_direct_params(dk, pl->dtile, &pl->dkp);
+    pl->dkp.skip_filter_stage = env_int("CCONV_DIAG_SKIP_FILTER_STAGE", -1);
+  }
 
   if (device >= 0) {
     int prev = 0;
@@ -522,8 +509,9 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
     if (variant == CCONV_VARIANT_HALO) pl->packed_bytes = size_t(pl->tile.packed_filter_bytes);
     if (variant == CCONV_VARIANT_STEM) pl->packed_bytes = size_t(pl->stile.packed_filter_bytes);
     pl->packed_bytes = (pl->packed_bytes + 255) & ~size_t(255);
-    if (e == cudaSuccess && variant >= CCONV_VARIANT_HALO)
+    if (e == cudaSuccess && (variant == CCONV_VARIANT_HALO || variant == CCONV_VARIANT_STEM))
       e = cudaMalloc(&pl->d_packed, 2 * pl->packed_bytes);
+    if (e == cudaSuccess && variant == CCONV_VARIANT_DIRECT) e = direct_kernel_prepare();
     if (e == cudaSuccess && variant >= CCONV_VARIANT_HALO && pl->padded) {
       const Dims& r = pl->drun;
       e = cudaMalloc(&pl->d_img_pad, size_t(r.Wi()) * r.Hi() * r.C * r.B * 2);
@@ -533,11 +521,14 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
     if (e == cudaSuccess && variant == CCONV_VARIANT_STEM)
       e = stem_kernel_prepare(pl->stile.smem_bytes);
     if (e == cudaSuccess && variant >= CCONV_VARIANT_HALO && env_int("CCONV_TRACE", 0)) {
-      pl->trace_rows = (variant == CCONV_VARIANT_HALO ? pl->tile.grid : pl->stile.grid) + 16;
+      pl->trace_rows = (variant == CCONV_VARIANT_HALO     ? pl->tile.grid
+                        : variant == CCONV_VARIANT_DIRECT ? pl->dtile.grid
+                                                          : pl->stile.grid) + 16;
       e = cudaMalloc(reinterpret_cast<void**>(&pl->d_trace), size_t(pl->trace_rows) * 16 * 8);
       if (e == cudaSuccess) e = cudaMemset(pl->d_trace, 0, size_t(pl->trace_rows) * 16 * 8);
       pl->kp.trace = pl->d_trace;
       pl->skp.trace = pl->d_trace;
+      pl->dkp.trace = pl->d_trace;
     }
     cudaSetDevice(prev);
     if (e != cudaSuccess) {
@@ -556,6 +547,13 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
                  "kw=%d i_stages=%d tmem=%d tiles=%lld grid=%d smem=%d filt=%u\n",
                  B, C, K, W, H, R, S, sw, sh, t.bw, t.bhm, t.kpad, t.kw, t.i_stages, t.tmem_cols,
                  t.tiles, t.grid, t.smem_bytes, t.filt_bytes);
+  } else if (env_int("CCONV_LOG", 0) && variant == CCONV_VARIANT_DIRECT) {
+    const DirectTile& t = pl->dtile;
+    std::fprintf(stderr,
+                 "[cconv] B%d C%d K%d W%d H%d R%d S%d s%dx%d variant=4 tile bb=%d bw=%d bh=%d kt=%d bc=%d "
+                 "tg=%d i_stages=%d f_stages=%d acc_bufs=%d tmem=%d tiles=%lld grid=%d smem=%d est_cyc=%.0f\n",
+                 B, C, K, W, H, R, S, sw, sh, t.bb, t.bw, t.bh, t.kt, t.bc, t.tg, t.i_stages, t.f_stages,
+                 t.acc_bufs, t.tmem_cols, t.tiles, t.grid, t.smem_bytes, t.est_cycles);
   } else if (env_int("CCONV_LOG", 0)) {
     const HaloTile& t = pl->tile;
     std::fprintf(stderr,
@@ -607,6 +605,15 @@ int cconv_plan_info_get(const cconv_plan* pl, cconv_plan_info* o) {
     o->smem_bytes = t.smem_bytes; o->tmem_cols = t.tmem_cols;
     o->tile_words_smem = t.words_smem;
     o->scratch_bytes = double(t.packed_filter_bytes);
+  }
+  if (pl->variant == CCONV_VARIANT_DIRECT) {
+    const DirectTile& t = pl->dtile;
+    o->bb = t.bb; o->bc = t.bc; o->bk = 128 * t.kt; o->bw = t.bw; o->bh = t.bh;
+    o->halo_w = t.halo_w; o->halo_h = t.halo_h;
+    o->stages = t.i_stages; o->filter_stages = t.f_stages; o->grid = t.grid; o->tiles = int(t.tiles);
+    o->smem_bytes = t.smem_bytes; o->tmem_cols = t.tmem_cols;
+    o->tile_words_smem = t.words_smem;
+    o->scratch_bytes = 0.0;
   }
   if (pl->variant == CCONV_VARIANT_HALO) {
     const HaloTile& t = pl->tile;
@@ -710,8 +717,7 @@ int cconv_forward_accumulate(const cconv_plan* pl, const void* Image, const void
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e, "cconv_accumulate_kernel");
   // an ordinary launch: nothing behind it starts before it is complete
-  std::lock_guard<std::mutex> lk(g_last_out_mu);
-  g_last_out.valid = false;
+  note_ordinary_launch(cuda_stream);
   return CCONV_OK;
 }
 
@@ -724,12 +730,38 @@ int cconv_forward_planned(const cconv_plan* pl, const void* Image, const void* F
   if (!aligned16(Image) || !aligned16(Filter) || (reinterpret_cast<uintptr_t>(Out) & 31u))
     return CCONV_EINVAL;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  const bool image_overlaps_last_out = note_call_and_check_overlap(
-      pl->d, pl->out_dtype, Image, Out, cuda_stream, pl->variant != CCONV_VARIANT_SIMT);
+  const CallSpans spans = spans_of(pl->d, pl->out_dtype, Image, Filter, Out);
   if (pl->variant == CCONV_VARIANT_SIMT) {
+    note_call(cuda_stream, spans, Overlap::kNone);
     cudaError_t e = launch_simt(Image, Filter, Out, pl->out_dtype == CCONV_OUT_F32, pl->d, stream);
     return e == cudaSuccess ? CCONV_OK : cuda_fail(e, "launch_simt");
   }
+  if (pl->variant == CCONV_VARIANT_DIRECT) {
+    const bool hazard = note_call(cuda_stream, spans, Overlap::kDeep);
+    CUtensorMap tmi, tmf;
+    {
+      // the tensor maps are rebuilt only when a base pointer changes
+      std::lock_guard<std::mutex> lk(pl->mu);
+      if (pl->tm_image_ptr != Image) {
+        const int rc = encode_direct_image_map(pl->view, pl->dtile, Image, &pl->tm_image);
+        if (rc != CCONV_OK) return rc;
+        pl->tm_image_ptr = Image;
+      }
+      if (pl->tm_filter_ptr != Filter) {
+        const int rc = encode_direct_filter_map(pl->view.dk, pl->dtile, Filter, &pl->tm_filter);
+        if (rc != CCONV_OK) return rc;
+        pl->tm_filter_ptr = Filter;
+      }
+      tmi = pl->tm_image;
+      tmf = pl->tm_filter;
+    }
+    DirectKernelParams kp = pl->dkp;
+    kp.wait_prev = hazard ? 1 : 0;
+    cudaError_t e = launch_direct(tmi, tmf, Out, pl->out_dtype == CCONV_OUT_F32, kp, pl->dtile.grid,
+                                  pl->dtile.smem_bytes, pl->d_status, stream);
+    return e == cudaSuccess ? CCONV_OK : cuda_fail(e, "launch_direct");
+  }
+  const bool inputs_hazard = note_call(cuda_stream, spans, Overlap::kInputsEarly);
   // Batch sizes that are not multiples of 8: the kernels run on zero-padded copies (see cconv_plan).
   void* const user_out = Out;
   const void* const user_image = Image;
@@ -740,7 +772,7 @@ int cconv_forward_planned(const cconv_plan* pl, const void* Image, const void* F
     Image = pl->d_img_pad;
     Out = pl->d_out_pad;
   }
-  const int rc_run = launch_tensor_core(pl, Image, Filter, Out, image_overlaps_last_out, stream,
+  const int rc_run = launch_tensor_core(pl, Image, Filter, Out, inputs_hazard, stream,
                                         pl->padded ? &g : nullptr, user_image);
   if (rc_run != CCONV_OK || !pl->padded) return rc_run;
   {
@@ -767,8 +799,7 @@ int cconv_forward_planned(const cconv_plan* pl, const void* Image, const void* F
     if (ec != cudaSuccess) return cuda_fail(ec, "cconv_compact_bands_kernel");
     // the compaction kernel never releases its dependents early: nothing behind it starts before it
     // is complete
-    std::lock_guard<std::mutex> lk(g_last_out_mu);
-    g_last_out.valid = false;
+    note_ordinary_launch(cuda_stream);
   }
   return CCONV_OK;
 }

@@ -1,0 +1,493 @@
+// Direct-Filter tensor-core kernel for the seven-nested-loop CNN (Eq. 1, Section 2):
+//   Out(k,h,w,b) = sum_{c,r,s} Image(r+sw*w, s+sh*h, c, b) * Filter(k,r,s,c)
+// Image [Wi][Hi][C][B], Filter [K][R][S][C], Out [K][H][W][B], bf16, last subscript fastest.
+//
+// The blocked loop nest of Section 5 on one SM, as in cconv_halo_kernel, with two differences:
+//   * the Filter block b_k x b_c of a tap is fetched straight from [K][R][S][C] by a 3-D TMA box
+//     (channels, out-channels, taps) into K-major swizzled rows, so a call is ONE launch with no
+//     scratch memory (the halo kernel repacks the Filter in a kernel of its own);
+//   * a CTA may own two blocks of 128 out-channels (b_k = 256) that share every staged Image block,
+//     which halves the Image words staged per multiply-add.
+// Outer loops {b,k,w,h}_1: the tile loop; outer loop c_1: the two shared-memory rings (an Image
+// stage = the halo block b_b x b_c x (sw(b_w-1)+R) x (sh(b_h-1)+S), shared by all R*S taps; a Filter
+// stage = tg taps of one channel block); inner loops: tcgen05.mma instructions whose B operand is
+// the SAME resident halo block seen through a descriptor shifted by (r, s).
+// Contraction order inside a tile: channel block -> tap (r major, s minor) -> 16-channel step.
+//
+// Calls overlap: the kernel lets the next kernel of the stream start at once
+// (griddepcontrol.launch_dependents at entry) and ends only after the kernel in front of it has
+// (griddepcontrol.wait before exit), so "kernel n complete" still implies "kernels < n complete".
+// Small problems therefore use few, large tiles: several calls run side by side on different SMs.
+// When an array of this call overlaps an array of a call that may still be running, the host sets
+// wait_prev and the producers start with griddepcontrol.wait.
+#include <cuda_bf16.h>
+
+#include "kernels.h"
+#include "ptx_sm100.cuh"
+
+namespace cconv {
+
+namespace {
+
+// warp 0: Image producer (TMA), warp 1: MMA issuer, warps 2-5: epilogue, warp 6: Filter producer
+constexpr int kDirectThreads = 224;
+
+// All MMAs of one tap: NC16 channel steps x KT out-channel blocks x b_h output rows.  Built by the
+// whole warp (uniform values), issued by the elected lane.  `acc` applies to the first channel
+// step; later steps always accumulate.
+template <int BH, int KT, int NC16>
+__device__ __forceinline__ void direct_issue_tap(bool leader, int bh, uint32_t d, uint32_t n_mma,
+                                                 uint32_t a_lo, uint32_t a_hi, uint32_t b_lo,
+                                                 uint32_t b_hi, uint32_t idesc, uint32_t acc,
+                                                 uint32_t ktile16, uint32_t kstep16,
+                                                 uint32_t hstep16) {
+#pragma unroll
+  for (int c = 0; c < NC16; ++c) {
+    const uint32_t accc = c == 0 ? acc : 1u;
+#pragma unroll
+    for (int kt = 0; kt < KT; ++kt) {
+      const uint64_t a_desc =
+          (uint64_t(a_hi) << 32) | (a_lo + uint32_t(c) * 2u + uint32_t(kt) * ktile16);
+      if constexpr (BH > 0) {
+#pragma unroll
+        for (int hh = 0; hh < BH; ++hh)
+          umma_bf16_if(leader, d + uint32_t(kt * BH + hh) * n_mma, a_desc,
+                       (uint64_t(b_hi) << 32) | (b_lo + uint32_t(c) * kstep16 + uint32_t(hh) * hstep16),
+                       idesc, accc);
+      } else {
+        for (int hh = 0; hh < bh; ++hh)
+          umma_bf16_if(leader, d + uint32_t(kt * bh + hh) * n_mma, a_desc,
+                       (uint64_t(b_hi) << 32) | (b_lo + uint32_t(c) * kstep16 + uint32_t(hh) * hstep16),
+                       idesc, accc);
+      }
+    }
+  }
+}
+
+template <typename OutT>
+__device__ __forceinline__ void direct_store_partial(OutT* dst, const uint32_t (&v)[32], int n) {
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    if (8 * j < n) {
+      if constexpr (sizeof(OutT) == 4) {
+        st_global_v8(dst + 8 * j, v[8 * j], v[8 * j + 1], v[8 * j + 2], v[8 * j + 3], v[8 * j + 4],
+                     v[8 * j + 5], v[8 * j + 6], v[8 * j + 7]);
+      } else {
+        *reinterpret_cast<uint4*>(dst + 8 * j) =
+            make_uint4(pack_bf16x2(v[8 * j], v[8 * j + 1]), pack_bf16x2(v[8 * j + 2], v[8 * j + 3]),
+                       pack_bf16x2(v[8 * j + 4], v[8 * j + 5]), pack_bf16x2(v[8 * j + 6], v[8 * j + 7]));
+      }
+    }
+  }
+}
+
+template <typename OutT>
+__device__ __forceinline__ void direct_store32(OutT* dst, const uint32_t (&v)[32]) {
+  if constexpr (sizeof(OutT) == 4) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      st_global_v8(dst + 8 * j, v[8 * j], v[8 * j + 1], v[8 * j + 2], v[8 * j + 3], v[8 * j + 4],
+                   v[8 * j + 5], v[8 * j + 6], v[8 * j + 7]);
+  } else {
+#pragma unroll
+    for (int j = 0; j < 2; ++j)
+      st_global_v8(dst + 16 * j, pack_bf16x2(v[16 * j + 0], v[16 * j + 1]),
+                   pack_bf16x2(v[16 * j + 2], v[16 * j + 3]), pack_bf16x2(v[16 * j + 4], v[16 * j + 5]),
+                   pack_bf16x2(v[16 * j + 6], v[16 * j + 7]), pack_bf16x2(v[16 * j + 8], v[16 * j + 9]),
+                   pack_bf16x2(v[16 * j + 10], v[16 * j + 11]),
+                   pack_bf16x2(v[16 * j + 12], v[16 * j + 13]),
+                   pack_bf16x2(v[16 * j + 14], v[16 * j + 15]));
+  }
+}
+
+}  // namespace
+
+// BH: b_h at compile time (0 = any); KT: blocks of 128 out-channels per CTA; NC16: 16-channel steps
+// per channel block (b_c / 16).
+template <typename OutT, int BH, int KT, int NC16>
+__global__ void __launch_bounds__(kDirectThreads, 1)
+    cconv_direct_kernel(const __grid_constant__ CUtensorMap tm_image,
+                        const __grid_constant__ CUtensorMap tm_filter, OutT* __restrict__ out,
+                        const DirectKernelParams p, int* __restrict__ status) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;  // swizzle atoms need 1024 B
+  const uint32_t img_ring = smem0;
+  const uint32_t filt_ring = img_ring + uint32_t(p.i_stages) * p.img_stage_bytes;
+  const uint32_t bars = filt_ring + uint32_t(p.f_stages) * p.filt_stage_bytes;
+  const uint32_t bar_ifull = bars;
+  const uint32_t bar_iempty = bar_ifull + 8u * p.i_stages;
+  const uint32_t bar_ffull = bar_iempty + 8u * p.i_stages;
+  const uint32_t bar_fempty = bar_ffull + 8u * p.f_stages;
+  const uint32_t bar_tfull = bar_fempty + 8u * p.f_stages;
+  const uint32_t bar_tempty = bar_tfull + 16u;
+  const uint32_t bar_drain = bar_tempty + 16u;
+  const uint32_t slot_addr = bar_drain + 8u;
+  uint8_t* gen0 = smem_raw + (smem0 - smem_u32(smem_raw));
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen0 + (slot_addr - smem0));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen0 + (slot_addr + 4u - smem0));
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+#define CCONV_TRACE(slot)                                                \
+  do {                                                                   \
+    if (p.trace) p.trace[blockIdx.x * 16 + (slot)] = globaltimer_ns();   \
+  } while (0)
+
+  if (threadIdx.x == 0) {
+    // The next kernel of the stream may start now: it takes SMs that this grid does not use.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    CCONV_TRACE(0);
+    for (int s = 0; s < p.i_stages; ++s) {
+      mbar_init(bar_ifull + 8u * s, 1);
+      mbar_init(bar_iempty + 8u * s, 1);
+    }
+    for (int s = 0; s < p.f_stages; ++s) {
+      mbar_init(bar_ffull + 8u * s, 1);
+      mbar_init(bar_fempty + 8u * s, 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(bar_tfull + 8u * a, 1);
+      mbar_init(bar_tempty + 8u * a, 4);  // one arrival per epilogue warp
+    }
+    mbar_init(bar_drain, 1);
+    *abort_flag = 0;
+    fence_barrier_init();
+    prefetch_tensormap(&tm_image);
+    prefetch_tensormap(&tm_filter);
+  }
+  if (warp == 1) {
+    tmem_alloc(slot_addr, uint32_t(p.tmem_cols));
+    tmem_relinquish();
+    tc_fence_before();
+  }
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint64_t limit = p.wait_limit_ns;
+  if (threadIdx.x == 0) CCONV_TRACE(1);
+
+  if (warp == 0) {
+    // ===================== Image halo producer (TMA) =====================
+    if (lane == 0) {
+      const uint32_t n_st = uint32_t(p.i_stages);
+      uint32_t seq = 0, s = 0, ph = 0;
+      bool ok = true;
+      if (p.wait_prev) asm volatile("griddepcontrol.wait;" ::: "memory");
+      for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
+        int t = tile / p.tiles_k;
+        const int bt = t % p.tiles_b; t /= p.tiles_b;
+        const int wt = t % p.tiles_w; t /= p.tiles_w;
+        const int ht = t;
+        const int b0 = bt * p.bb;
+        const int x0 = wt * p.bw * p.sw, y0 = ht * p.bh * p.sh;
+        for (int cc = 0, c0 = 0; cc < p.cchunks; ++cc, c0 += p.bc, ++seq) {
+          if (!mbar_wait(bar_iempty + 8u * s, ph ^ 1u, abort_flag, status, kStatProducerWait, limit)) {
+            ok = false;
+            break;
+          }
+          const uint32_t full = bar_ifull + 8u * s;
+          mbar_arrive_expect_tx(full, p.img_stage_bytes);
+          tma_load_4d(img_ring + s * p.img_stage_bytes, &tm_image, b0, c0, x0, y0, full);
+          if (seq == 0) CCONV_TRACE(2);
+          if (++s == n_st) {
+            s = 0;
+            ph ^= 1u;
+          }
+        }
+      }
+      CCONV_TRACE(3);
+      drain_ring(bar_ifull, seq, n_st, status, limit);
+    }
+  } else if (warp == 6) {
+    // ===================== Filter producer (TMA boxes of tg taps) =====================
+    if (lane == 0) {
+      const uint32_t n_st = uint32_t(p.f_stages);
+      uint32_t seq = 0, s = 0, ph = 0;
+      bool ok = true;
+      if (p.wait_prev) asm volatile("griddepcontrol.wait;" ::: "memory");
+      for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
+        const int k0 = (tile % p.tiles_k) * 128 * KT;
+        for (int cc = 0, c0 = 0; ok && cc < p.cchunks; ++cc, c0 += p.bc) {
+          for (int fg = 0, t0 = 0; fg < p.fgroups; ++fg, t0 += p.tg, ++seq) {
+            if (!mbar_wait(bar_fempty + 8u * s, ph ^ 1u, abort_flag, status, kStatFilterWait, limit)) {
+              ok = false;
+              break;
+            }
+            const uint32_t full = bar_ffull + 8u * s;
+            if (int(seq) != p.skip_filter_stage) {
+              mbar_arrive_expect_tx(full, p.filt_stage_bytes);
+              tma_load_3d(filt_ring + s * p.filt_stage_bytes, &tm_filter, c0, k0, t0, full);
+            }
+            if (++s == n_st) {
+              s = 0;
+              ph ^= 1u;
+            }
+          }
+        }
+      }
+      CCONV_TRACE(4);
+      // wait for the copies in flight (all but a stage left out on purpose, which never lands)
+      {
+        const uint32_t back = seq < n_st ? seq : n_st;
+        for (uint32_t j = 0; j < back; ++j) {
+          const uint32_t i2 = seq - 1 - j;
+          if (int(i2) == p.skip_filter_stage) continue;
+          const uint32_t t0s = i2 % n_st, phs = (i2 / n_st) & 1u;
+          const uint64_t t0 = globaltimer_ns();
+          while (!mbar_try_wait(bar_ffull + 8u * t0s, phs)) {
+            if (globaltimer_ns() - t0 > limit) {
+              atomicOr(status, kStatDrainWait);
+              break;
+            }
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ===================== MMA issuer =====================
+    const bool leader = elect_one();
+    uint32_t is = 0, iph = 0, fs = 0, fph = 0, abuf = 0, aph = 0;
+    bool ok = true, first_tile = true;
+    const int S = p.S, RS = p.R * p.S;
+    const uint32_t slab16 = p.slab_bytes >> 4, row16 = uint32_t(p.halo_w) * slab16;
+    const uint32_t a_lo0 = uint32_t(p.a_desc), a_hi = uint32_t(p.a_desc >> 32);
+    const uint32_t b_lo0 = uint32_t(p.b_desc), b_hi = uint32_t(p.b_desc >> 32);
+    const uint32_t hstep16 = uint32_t(p.sh * p.halo_w) * slab16;  // next output row
+    const uint32_t kstep16 = p.b_kstep_bytes >> 4;
+    const uint32_t img16 = p.img_stage_bytes >> 4, filt16 = p.filt_stage_bytes >> 4;
+    const uint32_t tap16 = p.filt_tap_bytes >> 4, ktile16 = p.filt_ktile_bytes >> 4;
+    const uint32_t img_ring16 = (img_ring >> 4) & 0x3FFFu, filt_ring16 = (filt_ring >> 4) & 0x3FFFu;
+    const uint32_t idesc = p.idesc, n_mma = uint32_t(p.n_mma);
+    const uint32_t n_ist = uint32_t(p.i_stages), n_fst = uint32_t(p.f_stages);
+    const int bh = p.bh, tg = p.tg;
+    long long tw_i = 0, tw_f = 0;
+    for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
+      if (!mbar_wait_warp(bar_tempty + 8u * abuf, aph ^ 1u, abort_flag, status, kStatMmaWaitTmem, limit))
+        break;
+      tc_fence_after();
+      const uint32_t d_base = tmem_base + abuf * uint32_t(p.acc_cols);
+      uint32_t acc = 0;
+      const long long tl0 = p.trace ? clock64() : 0;
+      for (int cc = 0; ok && cc < p.cchunks; ++cc) {
+        {
+          const long long w0 = p.trace ? clock64() : 0;
+          if (!mbar_wait_warp(bar_ifull + 8u * is, iph, abort_flag, status, kStatMmaWaitFull, limit)) {
+            ok = false;
+            break;
+          }
+          if (p.trace) tw_i += clock64() - w0;
+        }
+        tc_fence_after();
+        const uint32_t img_base16 = img_ring16 + is * img16;
+        int tap = 0, sx = 0;
+        uint32_t tap_off = 0, col_off = 0;  // halo offset of the current tap, in 16 B units
+        for (int fg = 0; fg < p.fgroups; ++fg) {
+          {
+            const long long w0 = p.trace ? clock64() : 0;
+            if (!mbar_wait_warp(bar_ffull + 8u * fs, fph, abort_flag, status, kStatMmaWaitFull, limit)) {
+              ok = false;
+              break;
+            }
+            if (p.trace) tw_f += clock64() - w0;
+          }
+          tc_fence_after();
+          if (first_tile && cc == 0 && fg == 0 && lane == 0) CCONV_TRACE(5);
+          uint32_t a16 = filt_ring16 + fs * filt16;
+          const int ntap = RS - tap < tg ? RS - tap : tg;
+          for (int j = 0; j < ntap; ++j) {
+            direct_issue_tap<BH, KT, NC16>(leader, bh, d_base, n_mma, a_lo0 | a16, a_hi,
+                                           b_lo0 | (img_base16 + tap_off), b_hi, idesc, acc, ktile16,
+                                           kstep16, hstep16);
+            acc = 1;
+            a16 += tap16;
+            // next tap: one halo row down (s); after S rows one halo pixel to the right (r)
+            tap_off += row16;
+            if (++sx == S) {
+              sx = 0;
+              col_off += slab16;
+              tap_off = col_off;
+            }
+          }
+          tap += ntap;
+          if (leader) umma_commit(bar_fempty + 8u * fs);  // free once the MMAs so far have read it
+          if (++fs == n_fst) {
+            fs = 0;
+            fph ^= 1u;
+          }
+        }
+        if (!ok) break;
+        if (leader) umma_commit(bar_iempty + 8u * is);
+        if (++is == n_ist) {
+          is = 0;
+          iph ^= 1u;
+        }
+      }
+      if (!ok) break;
+      if (first_tile && lane == 0 && p.trace) {
+        p.trace[blockIdx.x * 16 + 13] = (unsigned long long)tw_i;
+        p.trace[blockIdx.x * 16 + 14] = (unsigned long long)tw_f;
+        p.trace[blockIdx.x * 16 + 15] = (unsigned long long)(clock64() - tl0);
+      }
+      if (leader) umma_commit(bar_tfull + 8u * abuf);  // accumulator complete
+      if (first_tile && lane == 0) CCONV_TRACE(6);
+      first_tile = false;
+      if (++abuf == uint32_t(p.acc_bufs)) {
+        abuf = 0;
+        aph ^= 1u;
+      }
+    }
+    // All MMAs must have retired before TMEM is released.
+    if (lane == 0) CCONV_TRACE(7);
+    if (leader) umma_commit(bar_drain);
+    const uint64_t t0 = globaltimer_ns();
+    while (!mbar_try_wait(bar_drain, 0)) {
+      if (globaltimer_ns() - t0 > limit) {
+        atomicOr(status, kStatDrainWait);
+        break;
+      }
+    }
+  } else {
+    // ===================== epilogue: TMEM -> registers -> Out =====================
+    const int q = warp & 3;  // this warp may touch TMEM lanes [32q, 32q+32)
+    uint32_t abuf = 0, aph = 0;
+    bool first_tile = true;
+    const int chunks = p.bb / 32;
+    const bool wide_rows = (size_t(p.B) * sizeof(OutT)) % 32 == 0;
+    for (int tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
+      int t = tile;
+      const int ktile = t % p.tiles_k; t /= p.tiles_k;
+      const int bt = t % p.tiles_b; t /= p.tiles_b;
+      const int wt = t % p.tiles_w; t /= p.tiles_w;
+      const int ht = t;
+      const int b0 = bt * p.bb;
+      if (!mbar_wait_warp(bar_tfull + 8u * abuf, aph, abort_flag, status, kStatEpilogueWait, limit))
+        break;
+      tc_fence_after();
+      if (first_tile && threadIdx.x == 64) CCONV_TRACE(8);
+      const uint32_t t_base = tmem_base + (uint32_t(q * 32) << 16) + abuf * uint32_t(p.acc_cols);
+#pragma unroll
+      for (int kt = 0; kt < KT; ++kt) {
+        const int k = (ktile * KT + kt) * 128 + q * 32 + lane;
+        for (int hh = 0; hh < p.bh; ++hh) {
+          const int h = ht * p.bh + hh;
+          for (int ww = 0; ww < p.bw; ++ww) {
+            const int w = wt * p.bw + ww;
+            const bool valid = (k < p.K) && (h < p.H) && (w < p.W);
+            for (int ch = 0; ch < chunks; ++ch) {
+              uint32_t v[32];
+              tmem_ld_32x32b_x32(t_base + uint32_t((kt * p.bh + hh) * p.n_mma + ww * p.bb + ch * 32), v);
+              tmem_ld_wait();
+              if (valid) {
+                OutT* dst = out + (((long long)k * p.H + h) * p.W + w) * p.B + b0 + ch * 32;
+                const int nb = p.B - (b0 + ch * 32);  // images left in the batch (block padded past B)
+                if (nb >= 32 && wide_rows) direct_store32(dst, v);
+                else if (nb > 0) direct_store_partial(dst, v, nb < 32 ? nb : 32);
+              }
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_tempty + 8u * abuf);
+      if (first_tile && threadIdx.x == 64) CCONV_TRACE(9);
+      first_tile = false;
+      if (++abuf == uint32_t(p.acc_bufs)) {
+        abuf = 0;
+        aph ^= 1u;
+      }
+    }
+    if (threadIdx.x == 64) CCONV_TRACE(10);
+  }
+
+  // ===================== teardown =====================
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, uint32_t(p.tmem_cols));
+  }
+  // This kernel may have run beside the kernels in front of it; it ends only after they have.
+  if (threadIdx.x == 0) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    CCONV_TRACE(11);
+  }
+#undef CCONV_TRACE
+}
+
+namespace {
+
+template <typename OutT>
+using DirectFn = void (*)(CUtensorMap, CUtensorMap, OutT*, DirectKernelParams, int*);
+
+template <typename OutT, int KT, int NC16>
+DirectFn<OutT> direct_fn_bh(int bh) {
+  switch (bh) {
+    case 1: return cconv_direct_kernel<OutT, 1, KT, NC16>;
+    case 2: return cconv_direct_kernel<OutT, 2, KT, NC16>;
+    default: return cconv_direct_kernel<OutT, 0, KT, NC16>;
+  }
+}
+
+template <typename OutT, int KT>
+DirectFn<OutT> direct_fn_nc(int nc16, int bh) {
+  switch (nc16) {
+    case 1: return direct_fn_bh<OutT, KT, 1>(bh);
+    case 2: return direct_fn_bh<OutT, KT, 2>(bh);
+    default: return direct_fn_bh<OutT, KT, 4>(bh);
+  }
+}
+
+template <typename OutT>
+DirectFn<OutT> direct_fn(int kt, int nc16, int bh) {
+  return kt == 2 ? direct_fn_nc<OutT, 2>(nc16, bh) : direct_fn_nc<OutT, 1>(nc16, bh);
+}
+
+template <typename OutT>
+cudaError_t direct_prepare_all(int smem_bytes) {
+  for (int kt : {1, 2})
+    for (int nc : {1, 2, 4})
+      for (int bh : {1, 2, 3}) {
+        cudaError_t e = cudaFuncSetAttribute(direct_fn<OutT>(kt, nc, bh),
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+        if (e != cudaSuccess) return e;
+      }
+  return cudaSuccess;
+}
+
+}  // namespace
+
+// The dynamic shared-memory ceiling of every instantiation is raised to the device's limit (the
+// attribute is per kernel and the last value wins, so it is never set to one plan's need).
+cudaError_t direct_kernel_prepare() {
+  int dev = 0, cap = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&cap, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+  if (e != cudaSuccess) return e;
+  e = direct_prepare_all<__nv_bfloat16>(cap);
+  if (e != cudaSuccess) return e;
+  return direct_prepare_all<float>(cap);
+}
+
+cudaError_t launch_direct(const CUtensorMap& tm_image, const CUtensorMap& tm_filter, void* out,
+                          bool out_f32, const DirectKernelParams& p, int grid, int smem_bytes,
+                          int* status, cudaStream_t stream) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(unsigned(grid));
+  cfg.blockDim = dim3(kDirectThreads);
+  cfg.dynamicSmemBytes = size_t(smem_bytes);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const int nc16 = p.bc / 16;
+  if (out_f32)
+    return cudaLaunchKernelEx(&cfg, direct_fn<float>(p.kt, nc16, p.bh), tm_image, tm_filter,
+                              static_cast<float*>(out), p, status);
+  return cudaLaunchKernelEx(&cfg, direct_fn<__nv_bfloat16>(p.kt, nc16, p.bh), tm_image, tm_filter,
+                            static_cast<__nv_bfloat16*>(out), p, status);
+}
+
+}  // namespace cconv

@@ -5,6 +5,8 @@
 
 #include <algorithm>
 #include <cstdlib>
+#include <map>
+#include <mutex>
 
 #include "../../include/cconv.h"
 
@@ -132,6 +134,78 @@ int encode_image_map(const ImageView& v, const HaloTile& t, const void* image, C
   return CCONV_OK;
 }
 
+void build_direct_params(const Dims& d, const DirectTile& t, DirectKernelParams* out) {
+  DirectKernelParams& p = *out;
+  p.K = d.K; p.H = d.H; p.W = d.W; p.B = d.B; p.C = d.C;
+  p.R = d.R; p.S = d.S; p.sw = d.sw; p.sh = d.sh;
+  p.bb = t.bb; p.bw = t.bw; p.bh = t.bh; p.bc = t.bc; p.kt = t.kt;
+  p.halo_w = t.halo_w; p.halo_h = t.halo_h;
+  p.cchunks = t.cchunks;
+  p.tg = t.tg; p.fgroups = t.fgroups;
+  p.i_stages = t.i_stages; p.f_stages = t.f_stages;
+  p.tiles_k = t.tiles_k; p.tiles_b = t.tiles_b; p.tiles_w = t.tiles_w; p.tiles_h = t.tiles_h;
+  p.total_tiles = int(t.tiles);
+  p.n_mma = t.bb * t.bw;
+  p.acc_cols = p.n_mma * t.bh * t.kt;
+  p.acc_bufs = t.acc_bufs;
+  p.tmem_cols = t.tmem_cols;
+  p.wait_prev = 0;
+  p.img_stage_bytes = t.img_stage_bytes;
+  p.filt_stage_bytes = t.filt_stage_bytes;
+  p.filt_ktile_bytes = 128u * uint32_t(t.bc) * 2u;
+  p.filt_tap_bytes = uint32_t(t.kt) * p.filt_ktile_bytes;
+  p.slab_bytes = uint32_t(t.bc) * t.bb * 2;
+  p.b_kstep_bytes = 16u * t.bb * 2;
+  // instruction descriptor: D=f32, A=B=bf16, A K-major [15]=0, B MN-major [16]=1, N>>3, M=128>>4
+  p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
+            (uint32_t(p.n_mma >> 3) << 17) | (uint32_t(128 >> 4) << 24);
+  // A = Filter rows [128 out-channels][bc channels], K-major, one swizzle span per row (bc*2 = 128,
+  // 64 or 32 bytes: layout type 2, 4, 6); SBO = 8 rows; the leading offset is not used by swizzled
+  // K-major operands.  A 16-channel step advances the start address by 32 bytes inside the row.
+  const uint32_t a_row = uint32_t(t.bc) * 2;
+  const uint32_t a_layout = a_row == 128 ? 2u : a_row == 64 ? 4u : 6u;
+  p.a_desc = make_smem_desc(16, 8 * a_row, a_layout);
+  // B = Image halo view, as in the halo kernel: MN-major rows of bb*2 bytes (128- or 64-byte swizzle);
+  // SBO from one group of 8 channels to the next, LBO from one pixel to the next along w.
+  const uint32_t b_row = uint32_t(t.bb) * 2;
+  const uint32_t b_layout = b_row == 128 ? 2u : 4u;
+  p.b_desc = make_smem_desc(uint32_t(d.sw) * p.slab_bytes, 8 * b_row, b_layout);
+  p.wait_limit_ns = uint64_t(env_int("CCONV_WAIT_LIMIT_MS", 1000)) * 1000000ull;
+  p.skip_filter_stage = -1;
+  p.trace = nullptr;
+}
+
+int encode_direct_image_map(const ImageView& v, const DirectTile& t, const void* image, CUtensorMap* tm) {
+  HaloTile h;
+  h.bb = t.bb; h.bc = t.bc; h.halo_w = t.halo_w; h.halo_h = t.halo_h;
+  return encode_image_map(v, h, image, tm);
+}
+
+int encode_direct_filter_map(const Dims& d, const DirectTile& t, const void* filter, CUtensorMap* tm) {
+  EncodeTiledFn enc = encode_tiled_fn();
+  if (!enc) {
+    set_last_cuda_error("cuTensorMapEncodeTiled is not available from this driver");
+    return CCONV_ECUDA;
+  }
+  // Filter[k][r][s][c] viewed as (c, k, tap = r*S + s): a box lands as [tap][k][bc channels].
+  // Rows past K and channels past C are zero filled.
+  const cuuint64_t dims[3] = {cuuint64_t(d.C), cuuint64_t(d.K), cuuint64_t(d.R) * d.S};
+  const cuuint64_t strides[2] = {cuuint64_t(d.R) * d.S * d.C * 2, cuuint64_t(d.C) * 2};
+  const cuuint32_t box[3] = {cuuint32_t(t.bc), cuuint32_t(128 * t.kt), cuuint32_t(t.tg)};
+  const cuuint32_t es[3] = {1, 1, 1};
+  const CUtensorMapSwizzle sw = t.bc == 64   ? CU_TENSOR_MAP_SWIZZLE_128B
+                                : t.bc == 32 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                             : CU_TENSOR_MAP_SWIZZLE_32B;
+  CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(filter), dims, strides,
+                   box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    set_last_cuda_error("cuTensorMapEncodeTiled(Filter) failed with CUresult " + std::to_string(int(r)));
+    return CCONV_ECUDA;
+  }
+  return CCONV_OK;
+}
+
 void build_stem_params(const Dims& d, const StemTile& t, StemKernelParams* out) {
   StemKernelParams& p = *out;
   p.K = d.K; p.H = d.H; p.W = d.W; p.B = d.B; p.C = d.C;
@@ -181,6 +255,52 @@ int encode_stem_image_map(const Dims& d, const StemTile& t, const void* image, C
     return CCONV_ECUDA;
   }
   return CCONV_OK;
+}
+
+
+namespace {
+struct StreamCalls {
+  CallSpans calls[16];
+  int n = 0;
+};
+std::map<void*, StreamCalls> g_inflight;
+std::mutex g_inflight_mu;
+}  // namespace
+
+CallSpans spans_of(const Dims& d, int out_dtype, const void* Image, const void* Filter, const void* Out) {
+  CallSpans c;
+  c.image.lo = static_cast<const char*>(Image);
+  c.image.hi = c.image.lo + size_t(d.Wi()) * d.Hi() * d.C * d.B * 2;
+  c.filter.lo = static_cast<const char*>(Filter);
+  c.filter.hi = c.filter.lo + size_t(d.K) * d.R * d.S * d.C * 2;
+  c.out.lo = static_cast<const char*>(Out);
+  c.out.hi = c.out.lo + size_t(d.K) * d.H * d.W * d.B * (out_dtype == CCONV_OUT_F32 ? 4 : 2);
+  return c;
+}
+
+bool note_call(void* stream, const CallSpans& c, Overlap how) {
+  std::lock_guard<std::mutex> lk(g_inflight_mu);
+  StreamCalls& sc = g_inflight[stream];
+  if (how == Overlap::kNone) {
+    sc.n = 0;  // starts after, and is complete before, its neighbours
+    return false;
+  }
+  bool conflict = sc.n >= 16;  // bound the list: a waiting call completes everything before it
+  for (int i = 0; i < sc.n && !conflict; ++i) {
+    const CallSpans& e = sc.calls[i];
+    conflict = e.out.meets(c.image) || e.out.meets(c.filter);
+    if (how == Overlap::kDeep)
+      conflict = conflict || e.out.meets(c.out) || e.image.meets(c.out) || e.filter.meets(c.out);
+  }
+  if (conflict || how == Overlap::kInputsEarly) sc.n = 0;
+  sc.calls[sc.n++] = c;
+  return conflict;
+}
+
+void note_ordinary_launch(void* stream) {
+  std::lock_guard<std::mutex> lk(g_inflight_mu);
+  auto it = g_inflight.find(stream);
+  if (it != g_inflight.end()) it->second.n = 0;
 }
 
 void set_last_cuda_error(const std::string& msg) { g_last_cuda_error = msg; }

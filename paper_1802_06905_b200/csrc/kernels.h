@@ -79,6 +79,43 @@ struct StemKernelParams {
   unsigned long long* trace;
 };
 
+// Parameters of the direct-Filter tensor-core kernel (cconv_direct_kernel).  Same blocked nest as
+// the halo kernel, but the Filter is staged straight from [K][R][S][C] by TMA (no packing kernel, no
+// scratch): a Filter stage holds `tg` taps x kt*128 out-channels x bc channels as K-major swizzled
+// rows of bc*2 bytes.  Contraction order: channel chunk (bc) -> tap -> 16-channel step.
+struct DirectKernelParams {
+  int K, H, W, B, C, R, S, sw, sh;
+  int bb, bw, bh, bc;            // block sizes b_b, b_w, b_h; bc = channels per Image stage = per Filter row
+  int kt;                        // blocks of 128 out-channels per CTA (1 or 2): b_k = 128*kt
+  int halo_w, halo_h;
+  int cchunks;                   // ceil(C/bc)
+  int tg, fgroups;               // taps per Filter stage; Filter stages per channel chunk = ceil(R*S/tg)
+  int i_stages, f_stages;
+  int tiles_k, tiles_b, tiles_w, tiles_h, total_tiles;
+  int n_mma;                     // N of one MMA = bb*bw
+  int acc_cols;                  // accumulator columns of one tile = n_mma*bh*kt
+  int acc_bufs, tmem_cols;
+  int wait_prev;                 // 1: an array of this call overlaps one of a call that may still be
+                                 // running on the stream: nothing is read before the stream's
+                                 // earlier work is complete
+  uint32_t img_stage_bytes, filt_stage_bytes;
+  uint32_t filt_tap_bytes;       // one tap of a Filter stage: kt*128 rows of bc*2 bytes
+  uint32_t filt_ktile_bytes;     // 128 rows of bc*2 bytes
+  uint32_t slab_bytes;           // one Image pixel slab: bc*bb*2
+  uint32_t b_kstep_bytes;        // 16 channels of an Image slab: 16*bb*2
+  uint32_t idesc;
+  uint64_t a_desc, b_desc;       // shared-memory descriptors with a zero start address
+  uint64_t wait_limit_ns;
+  int skip_filter_stage;         // diagnostics: the Filter producer leaves out the stage with this
+                                 // sequence number (-1 = none), so that a bounded wait runs out
+  unsigned long long* trace;     // optional [grid][16] time stamps, or null
+};
+
+cudaError_t direct_kernel_prepare();
+cudaError_t launch_direct(const CUtensorMap& tm_image, const CUtensorMap& tm_filter, void* out,
+                          bool out_f32, const DirectKernelParams& p, int grid, int smem_bytes,
+                          int* status, cudaStream_t stream);
+
 cudaError_t launch_simt(const void* image, const void* filter, void* out, bool out_f32,
                         const Dims& d, cudaStream_t stream);
 
@@ -91,10 +128,12 @@ cudaError_t launch_pack_filter(const void* filter, void* packed, const Dims& d, 
                                int tiles_k, bool overlap_prev, cudaStream_t stream);
 
 // Filter [K][R][S][C] -> stem blocks [k-tile][r][16-row slice][128 x 16], the (s,c) run of each r
-// repeated once per stacked output row, shifted by that row's window offset, zero padded.  Always
-// launched with programmatic stream serialization (callers alternate between two buffers).
+// repeated once per stacked output row, shifted by that row's window offset, zero padded.
+// overlap_prev: as for launch_pack_filter (callers alternate between two buffers); off when the
+// Filter may still be being written by the call in front.
 cudaError_t launch_pack_filter_stem(const void* filter, void* packed, const Dims& d,
-                                    const StemKernelParams& p, cudaStream_t stream);
+                                    const StemKernelParams& p, bool overlap_prev,
+                                    cudaStream_t stream);
 cudaError_t stem_kernel_prepare(int smem_bytes);
 cudaError_t launch_stem(const CUtensorMap& tm_image, const void* packed_filter, void* out,
                         bool out_f32, const StemKernelParams& p, int grid, int smem_bytes,

@@ -407,6 +407,135 @@ bool choose_halo_tile(const Dims& d, const Machine& m, const int force[6], HaloT
   return found;
 }
 
+bool direct_supported(const Dims& d, const char** why) {
+  if (d.B % 8 != 0) {
+    if (why) *why = "B must be a multiple of 8 (16-byte TMA strides of the Image)";
+    return false;
+  }
+  if (d.C % 8 != 0) {
+    if (why) *why = "C must be a multiple of 8 (16-byte TMA strides of the Filter)";
+    return false;
+  }
+  return true;
+}
+
+bool choose_direct_tile(const Dims& d, const Machine& m, const int force[9], DirectTile* out) {
+  if (!direct_supported(d, nullptr)) return false;
+  const int reserve = 2048;  // barriers, TMEM slot, 1024-byte alignment slack
+  const int cap = m.smem_optin_bytes - reserve;
+  const int RS = d.R * d.S;
+  const int c16 = (d.C + 15) / 16;
+  // Cost model (SM cycles; constants measured on B200 with this kernel):
+  //  * an MMA of 128 x N x 16 occupies the tensor pipe for N/2 cycles; the issue loop sustains
+  //    about 90 % of that on tiles whose MMAs are 64 cycles or longer;
+  //  * operands arrive in shared memory at about 55 B/clk per SM when many SMs pull;
+  //  * a CTA spends about 4500 cycles before its first MMA (set-up, first copies from HBM) and
+  //    drains an accumulator at 14 (128-byte runs of Out) or 17 (64-byte runs) cycles per column;
+  //  * calls overlap (see cconv_direct_kernel): in a stream of calls the SMs stay busy, so the cost
+  //    of a call is its SM time divided by the SMs, rounded to whole grids per machine.
+  bool found = false;
+  DirectTile best;
+  for (int bb : {64, 32}) {
+    if (force[0] && bb != force[0]) continue;
+    if (!force[0] && bb == 64 && d.B <= 32) continue;  // half of the block would be padding
+    for (int bc : {64, 32, 16}) {
+      if (force[4] && bc != force[4]) continue;
+      if (bc > c16 * 16 && bc != 16) continue;
+      for (int kt : {1, 2}) {
+        if (force[3] && kt != force[3]) continue;
+        if (kt == 2 && d.K <= 128) continue;
+        for (int bw = 1; bw <= std::min(d.W, 256 / bb); ++bw) {
+          if (force[1] && bw != force[1]) continue;
+          const int N = bb * bw;
+          for (int bh = 1; bh <= d.H && N * bh * kt <= m.tmem_cols; ++bh) {
+            if (force[2] && bh != force[2]) continue;
+            DirectTile t;
+            t.bb = bb; t.bw = bw; t.bh = bh; t.bc = bc; t.kt = kt;
+            t.halo_w = d.sw * (bw - 1) + d.R;
+            t.halo_h = d.sh * (bh - 1) + d.S;
+            if (t.halo_w > 256 || t.halo_h > 256) continue;
+            t.cchunks = (d.C + bc - 1) / bc;
+            const long long img = 1ll * t.halo_w * t.halo_h * bc * bb * 2;
+            const long long tap_bytes = 1ll * kt * 128 * bc * 2;
+            // Filter stages of about 16 KB (whole taps)
+            int tg = int(std::max<long long>(1, 16384 / tap_bytes));
+            tg = std::min(tg, RS);
+            if (force[5]) tg = std::min(force[5], RS);
+            t.tg = tg;
+            t.fgroups = (RS + tg - 1) / tg;
+            const long long fst = tap_bytes * tg;
+            if (img + fst > cap) continue;
+            t.img_stage_bytes = uint32_t(img);
+            t.filt_stage_bytes = uint32_t(fst);
+            // Ring depths: shared memory split in proportion to the bytes each ring delivers per
+            // channel block, at least two stages each where they fit
+            const double per_chunk_f = double(tap_bytes) * RS;
+            const double share_f = per_chunk_f / (per_chunk_f + double(img));
+            int fs = int(share_f * cap / fst);
+            fs = std::max(2, std::min(12, fs));
+            while (fs > 2 && (cap - 1ll * fs * fst) / img < 2) --fs;
+            if (force[7]) fs = force[7];
+            long long left = cap - 1ll * fs * fst;
+            if (left < img) continue;
+            int is = int(std::min<long long>(6, left / img));
+            if (force[6]) {
+              if (is < force[6]) continue;
+              is = force[6];
+            }
+            t.i_stages = is;
+            t.f_stages = fs;
+            if (!force[7]) {
+              // left-over shared memory goes to the Filter ring
+              left = cap - 1ll * is * img - 1ll * fs * fst;
+              t.f_stages = int(std::min<long long>(12, fs + left / fst));
+            }
+            const int acc_cols = N * bh * kt;
+            t.tiles_k = (d.K + 128 * kt - 1) / (128 * kt);
+            t.tiles_b = (d.B + bb - 1) / bb;
+            t.tiles_w = (d.W + bw - 1) / bw;
+            t.tiles_h = (d.H + bh - 1) / bh;
+            t.tiles = 1ll * t.tiles_k * t.tiles_b * t.tiles_w * t.tiles_h;
+            if (t.tiles > 0x7fffffffll) continue;
+            t.grid = int(std::min<long long>(t.tiles, m.sm_count));
+            if (force[8]) t.grid = int(std::min<long long>(t.tiles, force[8]));
+            const double tiles_per_cta = std::ceil(double(t.tiles) / t.grid);
+            t.acc_bufs = (2 * acc_cols <= m.tmem_cols && tiles_per_cta > 1.0) ? 2 : 1;
+            int cols = 32;
+            while (cols < acc_cols * t.acc_bufs) cols *= 2;
+            t.tmem_cols = cols;
+            // CTAs that want more than half of the tensor memory must not share an SM
+            const int used = int(t.i_stages * t.img_stage_bytes + t.f_stages * t.filt_stage_bytes) + reserve;
+            t.smem_bytes = cols > 256 ? std::max(used, 117760) : used;
+            // ---- cycle model ----
+            const double units = double(c16) * RS;
+            const double cyc_mma = units * kt * bh * std::max(N / 2.0, 40.0) / 0.9;
+            const double tile_bytes = double(t.cchunks) * (double(img) + double(tap_bytes) * RS);
+            const double cyc_copy = tile_bytes / 55.0 * (bb >= 64 ? 1.0 : 1.08);
+            const double cyc_epi = (bb >= 64 ? 14.0 : 17.0) * acc_cols;
+            const double main_cyc = std::max(cyc_mma, cyc_copy);
+            const double cta_cyc = 4500.0 + (t.acc_bufs == 2
+                                                 ? tiles_per_cta * std::max(main_cyc, cyc_epi) + cyc_epi
+                                                 : tiles_per_cta * (main_cyc + cyc_epi));
+            t.tile_cycles = main_cyc;
+            t.sm_cycles = cta_cyc * t.grid;
+            // whole grids side by side on the machine
+            const double side = std::max(1.0, std::floor(double(m.sm_count) / t.grid));
+            t.est_cycles = cta_cyc / side;
+            t.words_smem = double(t.tiles) * tile_bytes / 2.0 + double(d.K) * d.H * d.W * d.B;
+            if (!found || t.est_cycles < best.est_cycles ||
+                (t.est_cycles == best.est_cycles && t.words_smem < best.words_smem)) {
+              best = t;
+              found = true;
+            }
+          }
+        }
+      }
+    }
+  }
+  if (found) *out = best;
+  return found;
+}
+
 bool choose_halo_tail(const Dims& d, const Machine& m, const HaloTile& main, int* main_tiles_h,
                       HaloTile* tail) {
   if (main.tiles <= main.grid || main.tiles_h < 2) return false;

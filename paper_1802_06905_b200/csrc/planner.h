@@ -91,6 +91,33 @@ struct StemTile {
   double words_smem = 0;
 };
 
+// Integer tile of the direct-Filter kernel.  As HaloTile, plus kt (b_k = 128*kt) and the Filter
+// stage shape; the Filter needs no scratch.
+struct DirectTile {
+  int bb = 0, bw = 0, bh = 0, bc = 0, kt = 1;
+  int halo_w = 0, halo_h = 0;
+  int tg = 1, fgroups = 1;
+  int i_stages = 0, f_stages = 0;
+  int acc_bufs = 1, tmem_cols = 0;
+  int cchunks = 0;
+  int tiles_k = 0, tiles_b = 0, tiles_w = 0, tiles_h = 0;
+  long long tiles = 0;
+  int grid = 0;
+  uint32_t img_stage_bytes = 0, filt_stage_bytes = 0;
+  int smem_bytes = 0;
+  double tile_cycles = 0;   // cost-model estimate for one tile on one SM
+  double sm_cycles = 0;     // tiles * tile_cycles: SM time of one call
+  double est_cycles = 0;    // estimate for one call in a stream of calls (calls overlap)
+  double words_smem = 0;
+};
+
+// True when the direct-Filter kernel can run this shape: B % 8 == 0 and C % 8 == 0 (16-byte TMA
+// strides of both tensor maps).
+bool direct_supported(const Dims& d, const char** why);
+// Enumerate legal tiles and keep the one with the least estimated SM time per call.  `force` may
+// carry "bb,bw,bh,kt,bc,tg,i_stages,f_stages,grid" (0 = free) from CCONV_FORCE_DIRECT.
+bool choose_direct_tile(const Dims& d, const Machine& m, const int force[9], DirectTile* out);
+
 void theorem1_terms(const Dims& d, double M, double t[5]);
 
 // Theorem 2 (Appendix A; strides 1): which expression of Theorem 1 is attainable.  Returns the leaf

@@ -41,15 +41,6 @@ constexpr int kStemEpiThreads = 256;
 constexpr int kFiltBars = 16;  // 16 KB Filter pieces: at most 14 fit in shared memory
 constexpr int kMaxAccBufs = 8;  // accumulator buffers in tensor memory: tmem_cols / acc_cols
 
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, int c0, int c1,
-                                            int c2, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
-      " [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
-      "l"(reinterpret_cast<uint64_t>(tm)), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
-      : "memory");
-}
-
 }  // namespace
 
 // ------------------------------------------------------------------------------------------------
@@ -103,7 +94,8 @@ __global__ void __launch_bounds__(256)
 }
 
 cudaError_t launch_pack_filter_stem(const void* filter, void* packed, const Dims& d,
-                                    const StemKernelParams& p, cudaStream_t stream) {
+                                    const StemKernelParams& p, bool overlap_prev,
+                                    cudaStream_t stream) {
   const long long slots = (long long)p.filt_bytes / 16;
   const long long blocks = (slots + 255) / 256;
   cudaLaunchConfig_t cfg = {};
@@ -114,7 +106,7 @@ cudaError_t launch_pack_filter_stem(const void* filter, void* packed, const Dims
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = overlap_prev ? 1 : 0;
   return cudaLaunchKernelEx(&cfg, cconv_pack_filter_stem_kernel,
                             static_cast<const unsigned short*>(filter), static_cast<uint4*>(packed), d,
                             p.kpad, p.bhm, p.khalves, slots);
