@@ -25,9 +25,13 @@
  * Ownership: the caller owns Image, Filter and Out.  Unless a function says "host", they are
  * DEVICE pointers on the plan's device, 16-byte aligned (Out: 32-byte aligned), and Out must not
  * overlap the inputs.
- * The library never dereferences a caller pointer after a call returns (it remembers the address
- * range of the last call's Out, to order a following call whose Image overlaps it).  Device calls are
- * asynchronous on the given stream, obey stream order, and never synchronise the stream.
+ * The library never dereferences a caller pointer after a call returns.  Device calls are
+ * asynchronous on the given stream, never synchronise it, and obey stream order although their
+ * kernels overlap on the GPU: per stream the library remembers the address ranges of the calls that
+ * may still be running, and a call whose Image or Filter overlaps the Out of one of them, or whose
+ * Out overlaps any array of one of them, starts only when the stream's earlier work is complete.
+ * Independent calls (other buffers) run side by side; "kernel n complete" always implies "kernels
+ * before n complete".  Calls of one explicit plan belong on one stream at a time.
  *
  * Errors: every function returns CCONV_OK (0) or a negative code; nothing throws, aborts or traps.
  * All positive loop bounds are accepted, also those outside the paper's assumptions
@@ -115,6 +119,17 @@ typedef struct {
    * split * tiles; the planner does so for filters of 9 or more taps with long channel loops and few
    * output pixels), else 1. */
   int split;
+  /* DIRECT variant: taps of the filter per Filter stage (a stage is filter_taps x bk x bc words). */
+  int filter_taps;
+  /* The paper's figure of merit for a tiling (Section 5): G = product of the block sizes, here
+   * bb*bc*bk*bw*bh*R*S (the kernels never cut r and s), and its ratio to the LP optimum lp_G at
+   * M_words.  bc is the channel block of one pipeline stage; the Out block stays in tensor memory
+   * across all channel blocks, which the two-level model behind lp_G has no notion of. */
+  double tile_G, tile_G_over_lp_G;
+  /* DIRECT variant, cost model in SM cycles: lifetime of one CTA (what a call that runs alone or
+   * must wait for the call in front takes) and the period of a stream of independent calls, which
+   * run side by side on the SMs. */
+  double est_cta_cycles, est_period_cycles;
 } cconv_plan_info;
 
 /* Theorem 1 (Section 4.1): the five lower-bound terms, in words, for a fast memory of M_words.
@@ -188,8 +203,11 @@ int cconv_plan_reserve_accumulate(cconv_plan* plan);
 int cconv_forward_accumulate(const cconv_plan* plan, const void* Image, const void* Filter, void* Out,
                              void* cuda_stream);
 
-/* Convenience: plan (cached per shape, device and out_dtype; variant AUTO) and launch on the
- * current device. */
+/* Convenience: plan (variant AUTO; cached per device, stream, shape and out_dtype, and kept until
+ * the process ends) and launch on the current device.  A plan owns scratch that its calls rewrite
+ * (HALO, STEM: the repacked Filter, padded copies), so calls of one plan belong on one stream; the
+ * cache therefore keeps a plan per stream, and two streams may run the same shape at once.  The
+ * first call of a (stream, shape) pair allocates: make it outside any stream capture. */
 int cconv_forward(const void* Image, const void* Filter, void* Out, int B, int C, int K, int W,
                   int H, int R, int S, int sw, int sh, int out_dtype, void* cuda_stream);
 

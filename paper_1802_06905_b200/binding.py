@@ -60,6 +60,9 @@ class PlanInfo(ctypes.Structure):
         ("scratch_bytes", ctypes.c_double),
         ("run_B", ctypes.c_int), ("run_H", ctypes.c_int), ("bands", ctypes.c_int),
         ("split", ctypes.c_int),
+        ("filter_taps", ctypes.c_int),
+        ("tile_G", ctypes.c_double), ("tile_G_over_lp_G", ctypes.c_double),
+        ("est_cta_cycles", ctypes.c_double), ("est_period_cycles", ctypes.c_double),
     ]
 
     def asdict(self):

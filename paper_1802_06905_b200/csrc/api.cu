@@ -208,6 +208,7 @@ struct cconv_plan {
   StemKernelParams skp{};
   DirectTile dtile{};
   DirectKernelParams dkp{};
+  mutable int diag_skip_once = -1;  // diagnostics: Filter stage the first call leaves out
   int* d_status = nullptr;
   // Scratch: the packed Filter, rewritten by every forward call.  Two buffers, used alternately:
   // the packing kernel of call n+1 may run while the convolution of call n still reads its buffer.
@@ -235,8 +236,18 @@ struct cconv_plan {
   mutable const void* tm_image_ptr = nullptr;
   mutable CUtensorMap tm_image{};
   mutable CUtensorMap tm_image_tail{};
-  mutable const void* tm_filter_ptr = nullptr;  // direct kernel: the Filter map
-  mutable CUtensorMap tm_filter{};
+  // direct kernel: tensor maps of the latest base pointers (callers rotate through a few buffers;
+  // encoding a map costs more host time than the rest of a call)
+  struct MapSlot {
+    const void* ptr = nullptr;
+    CUtensorMap tm{};
+  };
+  static constexpr int kMapSlots = 64;
+  mutable MapSlot img_maps[kMapSlots];
+  mutable MapSlot flt_maps[kMapSlots];
+  static int map_slot(const void* p) {
+    return int((reinterpret_cast<uintptr_t>(p) >> 8) * 0x9E3779B97F4A7C15ull >> 58);
+  }
 };
 
 namespace {
@@ -244,7 +255,7 @@ namespace {
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 std::mutex g_cache_mu;
-std::map<std::tuple<int, int, int, int, int, int, int, int, int, int, int>, cconv_plan*> g_cache;
+std::map<std::tuple<int, void*, int, int, int, int, int, int, int, int, int, int>, cconv_plan*> g_cache;
 
 }  // namespace
 
@@ -454,6 +465,16 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
     // the kernel that folds (s, c) into the contraction wins where it applies.
     if (stem_ok && d.C < 8) variant = CCONV_VARIANT_STEM;
     else variant = halo_ok ? CCONV_VARIANT_HALO : CCONV_VARIANT_SIMT;
+    // Problems whose tiles fit the SMs as one wave: the direct-Filter kernel (one launch, large
+    // tiles on few SMs, calls side by side) has about twice the throughput of the halo kernel in a
+    // stream of calls (measured on 16 layer shapes; it loses on problems of several waves).  A
+    // single call then takes longer (one CTA lifetime): CCONV_OBJECTIVE=latency keeps the halo
+    // kernel's many small tiles.
+    const char* objective = std::getenv("CCONV_OBJECTIVE");
+    const bool want_latency = objective && std::strcmp(objective, "latency") == 0;
+    if (variant == CCONV_VARIANT_HALO && direct_ok && !want_latency &&
+        pl->dtile.tiles <= pl->m.sm_count && d.macs() >= 4.0e6)
+      variant = CCONV_VARIANT_DIRECT;
     // A padded batch costs two more kernels (about 15 us per call in all, measured) and two scratch
     // arrays: worth it unless the problem is tiny (the CUDA-core kernel needs 8 us for 0.5 M
     // multiply-adds, 25-50 us for 7-15 M), and only within 4 GiB of scratch.
@@ -495,7 +516,7 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
   if (variant == CCONV_VARIANT_STEM) build_stem_params(pl->drun, pl->stile, &pl->skp);
   if (variant == CCONV_VARIANT_DIRECT) {
     build_direct_params(dk, pl->dtile, &pl->dkp);
-    pl->dkp.skip_filter_stage = env_int("CCONV_DIAG_SKIP_FILTER_STAGE", -1);
+    pl->diag_skip_once = env_int("CCONV_DIAG_SKIP_FILTER_STAGE", -1);
   }
 
   if (device >= 0) {
@@ -614,6 +635,9 @@ int cconv_plan_info_get(const cconv_plan* pl, cconv_plan_info* o) {
     o->smem_bytes = t.smem_bytes; o->tmem_cols = t.tmem_cols;
     o->tile_words_smem = t.words_smem;
     o->scratch_bytes = 0.0;
+    o->filter_taps = t.tg;
+    o->est_cta_cycles = t.cta_cycles;
+    o->est_period_cycles = t.est_cycles;
   }
   if (pl->variant == CCONV_VARIANT_HALO) {
     const HaloTile& t = pl->tile;
@@ -636,6 +660,10 @@ int cconv_plan_info_get(const cconv_plan* pl, cconv_plan_info* o) {
                                               (double(t.tiles) / t.tiles_h * ((r.H + t.bh - 1) / t.bh))) +
                            (u.words_smem - double(r.K) * (r.H - pl->kp_tail.h0) * r.W * r.B) + out_words;
     }
+  }
+  if (o->bb > 0 && pl->variant != CCONV_VARIANT_STEM) {
+    o->tile_G = double(o->bb) * o->bc * o->bk * o->bw * o->bh * d.R * d.S;
+    o->tile_G_over_lp_G = pl->lp_G > 0 ? o->tile_G / pl->lp_G : 0.0;
   }
   return CCONV_OK;
 }
@@ -730,38 +758,49 @@ int cconv_forward_planned(const cconv_plan* pl, const void* Image, const void* F
   if (!aligned16(Image) || !aligned16(Filter) || (reinterpret_cast<uintptr_t>(Out) & 31u))
     return CCONV_EINVAL;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  const CallSpans spans = spans_of(pl->d, pl->out_dtype, Image, Filter, Out);
+  CallSpans spans = spans_of(pl->d, pl->out_dtype, Image, Filter, Out);
   if (pl->variant == CCONV_VARIANT_SIMT) {
-    note_call(cuda_stream, spans, Overlap::kNone);
+    note_call(cuda_stream, spans, Overlap::kNone, pl->m.sm_count);
     cudaError_t e = launch_simt(Image, Filter, Out, pl->out_dtype == CCONV_OUT_F32, pl->d, stream);
     return e == cudaSuccess ? CCONV_OK : cuda_fail(e, "launch_simt");
   }
   if (pl->variant == CCONV_VARIANT_DIRECT) {
-    const bool hazard = note_call(cuda_stream, spans, Overlap::kDeep);
+    // SMs' worth of resident CTAs: CTAs that need more than half of an SM's shared memory or tensor
+    // memory have an SM each (under-counting only keeps calls on the list for longer)
+    spans.sms = double(pl->dtile.grid) /
+                std::max(1, std::min(pl->m.smem_optin_bytes / std::max(pl->dtile.smem_bytes, 1),
+                                     pl->m.tmem_cols / std::max(pl->dtile.tmem_cols, 1)));
+    const bool hazard = note_call(cuda_stream, spans, Overlap::kDeep, pl->m.sm_count);
     CUtensorMap tmi, tmf;
     {
-      // the tensor maps are rebuilt only when a base pointer changes
       std::lock_guard<std::mutex> lk(pl->mu);
-      if (pl->tm_image_ptr != Image) {
-        const int rc = encode_direct_image_map(pl->view, pl->dtile, Image, &pl->tm_image);
+      cconv_plan::MapSlot& si = pl->img_maps[cconv_plan::map_slot(Image)];
+      if (si.ptr != Image) {
+        const int rc = encode_direct_image_map(pl->view, pl->dtile, Image, &si.tm);
         if (rc != CCONV_OK) return rc;
-        pl->tm_image_ptr = Image;
+        si.ptr = Image;
       }
-      if (pl->tm_filter_ptr != Filter) {
-        const int rc = encode_direct_filter_map(pl->view.dk, pl->dtile, Filter, &pl->tm_filter);
+      cconv_plan::MapSlot& sf = pl->flt_maps[cconv_plan::map_slot(Filter)];
+      if (sf.ptr != Filter) {
+        const int rc = encode_direct_filter_map(pl->view.dk, pl->dtile, Filter, &sf.tm);
         if (rc != CCONV_OK) return rc;
-        pl->tm_filter_ptr = Filter;
+        sf.ptr = Filter;
       }
-      tmi = pl->tm_image;
-      tmf = pl->tm_filter;
+      tmi = si.tm;
+      tmf = sf.tm;
     }
     DirectKernelParams kp = pl->dkp;
+    {
+      std::lock_guard<std::mutex> lk(pl->mu);
+      kp.skip_filter_stage = pl->diag_skip_once;
+      pl->diag_skip_once = -1;
+    }
     kp.wait_prev = hazard ? 1 : 0;
     cudaError_t e = launch_direct(tmi, tmf, Out, pl->out_dtype == CCONV_OUT_F32, kp, pl->dtile.grid,
                                   pl->dtile.smem_bytes, pl->d_status, stream);
     return e == cudaSuccess ? CCONV_OK : cuda_fail(e, "launch_direct");
   }
-  const bool inputs_hazard = note_call(cuda_stream, spans, Overlap::kInputsEarly);
+  const bool inputs_hazard = note_call(cuda_stream, spans, Overlap::kInputsEarly, pl->m.sm_count);
   // Batch sizes that are not multiples of 8: the kernels run on zero-padded copies (see cconv_plan).
   void* const user_out = Out;
   const void* const user_image = Image;
@@ -811,7 +850,7 @@ int cconv_forward(const void* Image, const void* Filter, void* Out, int B, int C
   cconv_plan* pl = nullptr;
   {
     std::lock_guard<std::mutex> lk(g_cache_mu);
-    auto key = std::make_tuple(dev, B, C, K, W, H, R, S, sw, sh, out_dtype);
+    auto key = std::make_tuple(dev, cuda_stream, B, C, K, W, H, R, S, sw, sh, out_dtype);
     auto it = g_cache.find(key);
     if (it == g_cache.end()) {
       int rc = cconv_plan_create(&pl, B, C, K, W, H, R, S, sw, sh, dev, 0.0, CCONV_VARIANT_AUTO,

@@ -163,7 +163,10 @@ __global__ void __launch_bounds__(kDirectThreads, 1)
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const uint64_t limit = p.wait_limit_ns;
+  // The MMA issuer's wait for a stage is the one that names the cause when a copy never lands; the
+  // waits that depend on the issuer's progress (producers, epilogue) are given four times its
+  // limit, and leave as soon as the issuer has raised the abort flag.
+  const uint64_t limit = (warp == 1) ? p.wait_limit_ns : 4 * p.wait_limit_ns;
   if (threadIdx.x == 0) CCONV_TRACE(1);
 
   if (warp == 0) {
@@ -173,13 +176,17 @@ __global__ void __launch_bounds__(kDirectThreads, 1)
       uint32_t seq = 0, s = 0, ph = 0;
       bool ok = true;
       if (p.wait_prev) asm volatile("griddepcontrol.wait;" ::: "memory");
-      for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
+      auto coords = [&](int tile, int& b0, int& x0, int& y0) {
         int t = tile / p.tiles_k;
         const int bt = t % p.tiles_b; t /= p.tiles_b;
         const int wt = t % p.tiles_w; t /= p.tiles_w;
-        const int ht = t;
-        const int b0 = bt * p.bb;
-        const int x0 = wt * p.bw * p.sw, y0 = ht * p.bh * p.sh;
+        b0 = bt * p.bb;
+        x0 = wt * p.bw * p.sw;
+        y0 = t * p.bh * p.sh;
+      };
+      for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
+        int b0, x0, y0;
+        coords(tile, b0, x0, y0);
         for (int cc = 0, c0 = 0; cc < p.cchunks; ++cc, c0 += p.bc, ++seq) {
           if (!mbar_wait(bar_iempty + 8u * s, ph ^ 1u, abort_flag, status, kStatProducerWait, limit)) {
             ok = false;
@@ -360,8 +367,10 @@ __global__ void __launch_bounds__(kDirectThreads, 1)
       const int wt = t % p.tiles_w; t /= p.tiles_w;
       const int ht = t;
       const int b0 = bt * p.bb;
-      if (!mbar_wait_warp(bar_tfull + 8u * abuf, aph, abort_flag, status, kStatEpilogueWait, limit))
-        break;
+      // (every lane polls for itself and checks the abort flag each time; the decision to go on
+      // must be the same in all lanes because the TMEM loads below are warp-wide)
+      const bool got = mbar_wait(bar_tfull + 8u * abuf, aph, abort_flag, status, kStatEpilogueWait, limit);
+      if (!__all_sync(0xffffffffu, got)) break;
       tc_fence_after();
       if (first_tile && threadIdx.x == 64) CCONV_TRACE(8);
       const uint32_t t_base = tmem_base + (uint32_t(q * 32) << 16) + abuf * uint32_t(p.acc_cols);

@@ -259,8 +259,9 @@ int encode_stem_image_map(const Dims& d, const StemTile& t, const void* image, C
 
 
 namespace {
+constexpr int kMaxTracked = 160;
 struct StreamCalls {
-  CallSpans calls[16];
+  CallSpans calls[kMaxTracked];
   int n = 0;
 };
 std::map<void*, StreamCalls> g_inflight;
@@ -278,14 +279,29 @@ CallSpans spans_of(const Dims& d, int out_dtype, const void* Image, const void* 
   return c;
 }
 
-bool note_call(void* stream, const CallSpans& c, Overlap how) {
+bool note_call(void* stream, const CallSpans& c, Overlap how, int sm_count) {
   std::lock_guard<std::mutex> lk(g_inflight_mu);
   StreamCalls& sc = g_inflight[stream];
   if (how == Overlap::kNone) {
     sc.n = 0;  // starts after, and is complete before, its neighbours
     return false;
   }
-  bool conflict = sc.n >= 16;  // bound the list: a waiting call completes everything before it
+  // forget the calls that must be complete by the time this one starts: walking back from the
+  // latest call, everything behind more than sm_count SMs' worth of resident CTAs
+  {
+    double sms = 0;
+    int keep = 0;
+    for (int i = sc.n - 1; i >= 0; --i) {
+      ++keep;
+      sms += sc.calls[i].sms;
+      if (sms > double(sm_count)) break;
+    }
+    if (keep < sc.n) {
+      for (int i = 0; i < keep; ++i) sc.calls[i] = sc.calls[sc.n - keep + i];
+      sc.n = keep;
+    }
+  }
+  bool conflict = sc.n >= kMaxTracked;  // bound the list: a waiting call completes everything before it
   for (int i = 0; i < sc.n && !conflict; ++i) {
     const CallSpans& e = sc.calls[i];
     conflict = e.out.meets(c.image) || e.out.meets(c.filter);

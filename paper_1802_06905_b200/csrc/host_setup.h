@@ -47,6 +47,7 @@ struct Span {
 };
 struct CallSpans {
   Span image, filter, out;
+  double sms = 0;  // SMs' worth of CTAs the call keeps resident (grid / CTAs per SM)
 };
 CallSpans spans_of(const Dims& d, int out_dtype, const void* Image, const void* Filter, const void* Out);
 
@@ -58,8 +59,10 @@ enum class Overlap {
   kDeep,         // direct calls: reads and writes may overlap any number of earlier calls
 };
 // Registers a call and says whether it must wait for the stream's earlier work before touching
-// memory.
-bool note_call(void* stream, const CallSpans& c, Overlap how);
+// memory.  Calls known to be complete are forgotten: every CTA of an overlapping call stays
+// resident until the call in front of it is complete, so a call can still be running only while
+// the CTAs of all calls launched after it (but the newest) fit the `sm_count` SMs together.
+bool note_call(void* stream, const CallSpans& c, Overlap how, int sm_count);
 // An ordinary launch of this library (pooling, the accumulate pass, ...) went into the stream.
 void note_ordinary_launch(void* stream);
 

@@ -425,14 +425,18 @@ bool choose_direct_tile(const Dims& d, const Machine& m, const int force[9], Dir
   const int cap = m.smem_optin_bytes - reserve;
   const int RS = d.R * d.S;
   const int c16 = (d.C + 15) / 16;
-  // Cost model (SM cycles; constants measured on B200 with this kernel):
+  // Cost model (SM cycles; constants measured on B200 with this kernel on the 14x14 benchmark shapes):
   //  * an MMA of 128 x N x 16 occupies the tensor pipe for N/2 cycles; the issue loop sustains
-  //    about 90 % of that on tiles whose MMAs are 64 cycles or longer;
-  //  * operands arrive in shared memory at about 55 B/clk per SM when many SMs pull;
-  //  * a CTA spends about 4500 cycles before its first MMA (set-up, first copies from HBM) and
-  //    drains an accumulator at 14 (128-byte runs of Out) or 17 (64-byte runs) cycles per column;
+  //    about 87 % of that;
+  //  * operands arrive in shared memory at about 44 B/clk per SM when all SMs pull (1 MB per CTA in
+  //    21.7 k to 25 k cycles on four tilings);
+  //  * a CTA spends about 5300 cycles before its first MMA (set-up, first copies from HBM) and
+  //    drains an accumulator at about 15 cycles per column;
   //  * calls overlap (see cconv_direct_kernel): in a stream of calls the SMs stay busy, so the cost
-  //    of a call is its SM time divided by the SMs, rounded to whole grids per machine.
+  //    of a call is its SM time (CTAs x CTA lifetime) divided by the SMs; measured periods are that
+  //    figure / 0.85 for grids of 28 to 98 CTAs.
+  // Objective: the SM time of a call.  It favours few large tiles, whose lifetime is long: a call
+  // that runs alone (or must wait for the call in front) takes a CTA lifetime, not the period.
   bool found = false;
   DirectTile best;
   for (int bb : {64, 32}) {
@@ -508,19 +512,20 @@ bool choose_direct_tile(const Dims& d, const Machine& m, const int force[9], Dir
             t.smem_bytes = cols > 256 ? std::max(used, 117760) : used;
             // ---- cycle model ----
             const double units = double(c16) * RS;
-            const double cyc_mma = units * kt * bh * std::max(N / 2.0, 40.0) / 0.9;
+            const double cyc_mma = units * kt * bh * std::max(N / 2.0, 40.0) / 0.87;
             const double tile_bytes = double(t.cchunks) * (double(img) + double(tap_bytes) * RS);
-            const double cyc_copy = tile_bytes / 55.0 * (bb >= 64 ? 1.0 : 1.08);
-            const double cyc_epi = (bb >= 64 ? 14.0 : 17.0) * acc_cols;
-            const double main_cyc = std::max(cyc_mma, cyc_copy);
-            const double cta_cyc = 4500.0 + (t.acc_bufs == 2
+            const double cyc_copy = tile_bytes / 44.0;
+            const double cyc_epi = (bb >= 64 ? 14.6 : 15.6) * acc_cols;
+            // a single Image stage cannot be refilled while the MMAs on it run
+            const double main_cyc = t.i_stages == 1 ? cyc_mma + double(t.cchunks) * double(img) / 44.0
+                                                    : std::max(cyc_mma, cyc_copy);
+            const double cta_cyc = 5300.0 + (t.acc_bufs == 2
                                                  ? tiles_per_cta * std::max(main_cyc, cyc_epi) + cyc_epi
                                                  : tiles_per_cta * (main_cyc + cyc_epi));
             t.tile_cycles = main_cyc;
+            t.cta_cycles = cta_cyc;
             t.sm_cycles = cta_cyc * t.grid;
-            // whole grids side by side on the machine
-            const double side = std::max(1.0, std::floor(double(m.sm_count) / t.grid));
-            t.est_cycles = cta_cyc / side;
+            t.est_cycles = t.sm_cycles / m.sm_count / 0.85;
             t.words_smem = double(t.tiles) * tile_bytes / 2.0 + double(d.K) * d.H * d.W * d.B;
             if (!found || t.est_cycles < best.est_cycles ||
                 (t.est_cycles == best.est_cycles && t.words_smem < best.words_smem)) {

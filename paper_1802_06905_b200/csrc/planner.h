@@ -105,9 +105,10 @@ struct DirectTile {
   int grid = 0;
   uint32_t img_stage_bytes = 0, filt_stage_bytes = 0;
   int smem_bytes = 0;
-  double tile_cycles = 0;   // cost-model estimate for one tile on one SM
-  double sm_cycles = 0;     // tiles * tile_cycles: SM time of one call
-  double est_cycles = 0;    // estimate for one call in a stream of calls (calls overlap)
+  double tile_cycles = 0;   // cost-model estimate for the main loop of one tile
+  double cta_cycles = 0;    // lifetime of one CTA: what a call that runs alone takes
+  double sm_cycles = 0;     // grid * cta_cycles: SM time of one call
+  double est_cycles = 0;    // period of a stream of such calls (calls overlap on the SMs)
   double words_smem = 0;
 };
 

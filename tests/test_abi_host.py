@@ -136,6 +136,29 @@ def test_inspection_plans_are_hardware_legal():
                 assert info["tail_tiles"] == 0
             # the staged words can never undercut the bound at the shared-memory size
             assert info["tile_words_smem"] >= max(exp_terms) * 0.999 or max(exp_terms) < info["M_words"]
+        elif info["variant"] == binding.VARIANT_DIRECT:
+            assert cfg.B % 8 == 0 and cfg.C % 8 == 0                   # 16-byte TMA strides
+            n = info["bb"] * info["bw"]
+            assert n % 16 == 0 and 16 <= n <= 256                      # tcgen05 N rule at M=128
+            assert info["bk"] in (128, 256) and info["bc"] in (16, 32, 64)
+            kt = info["bk"] // 128
+            assert n * info["bh"] * kt <= info["tmem_cols"] <= 512     # tensor memory
+            assert info["smem_bytes"] <= 232448                        # 227 KB
+            assert info["halo_w"] == cfg.sw * (info["bw"] - 1) + cfg.R
+            assert info["halo_h"] == cfg.sh * (info["bh"] - 1) + cfg.S
+            img_stage = info["halo_w"] * info["halo_h"] * info["bc"] * info["bb"] * 2
+            filt_stage = info["filter_taps"] * info["bk"] * info["bc"] * 2
+            assert 1 <= info["filter_taps"] <= cfg.R * cfg.S
+            assert info["stages"] >= 1 and info["filter_stages"] >= 2
+            assert info["stages"] * img_stage + info["filter_stages"] * filt_stage <= info["smem_bytes"]
+            assert info["scratch_bytes"] == 0 and info["tail_tiles"] == 0
+            assert info["tiles"] == (-(-cfg.K // info["bk"]) * -(-cfg.B // info["bb"]) *
+                                     -(-cfg.W // info["bw"]) * -(-cfg.H // info["bh"]))
+            assert info["grid"] == min(info["tiles"], 148)
+            assert info["est_cta_cycles"] > 0 and info["est_period_cycles"] > 0
+            assert info["tile_G"] == (info["bb"] * info["bc"] * info["bk"] * info["bw"] * info["bh"] *
+                                      cfg.R * cfg.S)
+            assert info["tile_words_smem"] >= max(exp_terms) * 0.999 or max(exp_terms) < info["M_words"]
         elif info["variant"] == binding.VARIANT_STEM:
             assert cfg.B % 8 == 0 and cfg.C < 8
             assert 1 <= info["bw"] <= 4 and 2 * 64 * info["bw"] <= info["tmem_cols"] <= 512
@@ -184,7 +207,7 @@ def test_strided_1x1_is_planned_on_a_subsampled_view():
     plan = binding.Plan(64, 1024, 2048, 7, 7, 1, 1, 2, 2, device=-1)
     info = plan.info()
     plan.close()
-    assert info["variant"] == binding.VARIANT_HALO
+    assert info["variant"] in (binding.VARIANT_HALO, binding.VARIANT_DIRECT)
     assert info["halo_w"] == info["bw"] and info["halo_h"] == info["bh"]
     plan = binding.Plan(64, 64, 128, 7, 7, 3, 3, 2, 2, device=-1)
     info = plan.info()
@@ -279,7 +302,8 @@ def test_random_shapes_plan_to_hardware_legal_tiles():
     """A thousand seeded random shapes (any batch size, filters up to 11x11, strides up to 4): every
     plan for a nominal B200 obeys the limits of the SM, whichever variant AUTO picks."""
     rng = np.random.default_rng(2718)
-    seen = {binding.VARIANT_SIMT: 0, binding.VARIANT_HALO: 0, binding.VARIANT_STEM: 0}
+    seen = {binding.VARIANT_SIMT: 0, binding.VARIANT_HALO: 0, binding.VARIANT_STEM: 0,
+            binding.VARIANT_DIRECT: 0}
     for _ in range(1000):
         B = int(rng.choice([1, 2, 3, 8, 12, 16, 24, 32, 40, 64, 100, 128, 256]))
         C = int(rng.choice([1, 3, 4, 7, 8, 16, 24, 48, 64, 100, 128, 256, 512, 1024]))
@@ -317,6 +341,20 @@ def test_random_shapes_plan_to_hardware_legal_tiles():
             assert info["bw"] <= max(W, 1) + 3 and info["bh"] <= max(Hrun, 1)
             if info["tail_h0"] < Hrun:
                 assert 0 < info["tail_h0"] and 1 <= info["tail_tiles"] <= 148
+        elif info["variant"] == binding.VARIANT_DIRECT:
+            # one wave of large tiles on the caller's own arrays
+            n = info["bb"] * info["bw"]
+            kt = info["bk"] // 128
+            assert B % 8 == 0 and C % 8 == 0 and Bp == B
+            assert info["bb"] in (32, 64) and info["bc"] in (16, 32, 64) and kt in (1, 2)
+            assert n % 16 == 0 and 16 <= n <= 256
+            assert n * info["bh"] * kt <= info["tmem_cols"] <= 512
+            assert info["smem_bytes"] <= 232448 and (info["tmem_cols"] <= 256 or info["smem_bytes"] >= 117760)
+            assert 1 <= info["halo_w"] <= 256 and 1 <= info["halo_h"] <= 256
+            img_stage = info["halo_w"] * info["halo_h"] * info["bc"] * info["bb"] * 2
+            filt_stage = info["filter_taps"] * info["bk"] * info["bc"] * 2
+            assert info["stages"] * img_stage + info["filter_stages"] * filt_stage <= info["smem_bytes"]
+            assert info["tiles"] == info["grid"] <= 148 and info["scratch_bytes"] == 0
         elif info["variant"] == binding.VARIANT_STEM:
             assert C < 8
             assert 1 <= info["bw"] <= 4 and info["bk"] in (32, 64, 128) and info["bk"] * info["bh"] <= 128
@@ -333,7 +371,7 @@ def test_planner_split_rule():
     loops and few output pixels; the benchmark shapes, 1x1 filters and short loops stay whole; four
     CTAs per tile need 288 units (C*R*S >= 4608)."""
     def split_of(*dims):
-        p = binding.Plan(*dims, device=-1)
+        p = binding.Plan(*dims, device=-1, variant=binding.VARIANT_HALO)
         info = p.info()
         p.close()
         return info["split"], info

@@ -31,7 +31,7 @@ DT_IDS = ["f32out", "bf16out"]
 def test_config_full_parity(name, out_dtype):
     info = check_full(BY[name], out_dtype=out_dtype)
     if name in ("cfg2_resnet_3x3", "cfg4_pointwise_1x1"):
-        assert info["variant"] == binding.VARIANT_HALO     # the tensor-core path is the one that ran
+        assert info["variant"] == binding.VARIANT_DIRECT   # the tensor-core path is the one that ran
     if name == "cfg3_stem_7x7_s2":
         assert info["variant"] == binding.VARIANT_STEM
 
@@ -472,7 +472,8 @@ def test_split_banded_and_accumulating_calls_inside_a_cuda_graph():
         ib, fb = synth.make_inputs(c)
         jobs.append([c, to_dev(ib), to_dev(fb),
                      torch.full(c.out_shape, float("nan"), device="cuda", dtype=torch.float32),
-                     binding.Plan(*c.dims(), device=0, out_dtype=binding.OUT_F32)])
+                     binding.Plan(*c.dims(), device=0, out_dtype=binding.OUT_F32,
+                                  variant=binding.VARIANT_HALO)])
     assert jobs[0][4].info()["split"] == 4 and jobs[1][4].info()["bands"] == 8
     acc = torch.zeros(c4.out_shape, device="cuda", dtype=torch.float32)
     jobs[0][4].reserve_accumulate()
@@ -724,6 +725,6 @@ def test_accumulate_adds_the_convolution_to_what_out_holds(variant, c, out_dtype
     cs("autosplit_b16_5x5", 16, 256, 136, 7, 6, 5, 5),
 ], ids=lambda c: c.name)
 def test_planner_splits_channels_over_cta_pairs_on_small_grids(c, out_dtype):
-    info = check_full(c, variant=binding.VARIANT_AUTO, out_dtype=out_dtype)
+    info = check_full(c, variant=binding.VARIANT_HALO, out_dtype=out_dtype)
     assert info["variant"] == binding.VARIANT_HALO and info["split"] in (2, 4)
     assert info["grid"] == info["split"] * info["tiles"]
