@@ -247,17 +247,24 @@ int cconv_host_wait(cconv_plan* plan, void* cuda_stream);
  *   - Shapes whose repacked Filter exceeds the array return CCONV_ETOOLARGE; nothing is launched.
  *   - The first call on each device looks up the array's device address and the device limits
  *     (with that device current).  Make that first call outside any stream capture.
- *   - All calls share the one array, which keeps the previous call's contents: the call clears the
- *     status word and rewrites the Filter blocks it uses, so back-to-back calls on ONE stream are
- *     safe, but two calls whose kernels may overlap on the GPU (different streams, no dependency)
- *     race on the array and give wrong results.  Host-side, calls are serialised by a mutex.
+ *   - All calls share the one array, which keeps the previous call's contents: the call rewrites
+ *     the Filter blocks it uses, so back-to-back calls on ONE stream are safe (and ordered against
+ *     the planned calls around them like any other call), but two calls whose kernels may overlap
+ *     on the GPU (different streams, no dependency) race on the array and give wrong results.
+ *     Host-side, calls are serialised by a mutex.
  *   - Asynchronous on `cuda_stream` when device_status_out is NULL.  With a non-NULL
  *     device_status_out the call synchronises the stream, stores the device status word there
- *     (0 = fine, else a bit mask of the bounded waits that expired) and returns
- *     CCONV_EDEVICE_TIMEOUT if it is non-zero. */
+ *     (0 = fine, else a bit mask of the bounded waits that expired), clears it, and returns
+ *     CCONV_EDEVICE_TIMEOUT if it was non-zero. */
 int cconv_forward_noalloc(const void* Image, const void* Filter, void* Out, int B, int C, int K,
                           int W, int H, int R, int S, int sw, int sh, int out_dtype,
                           void* cuda_stream, int* device_status_out);
+/* (No counterpart in the paper either.)  The status word of the asynchronous cconv_forward_noalloc
+ * calls made so far on the current device: synchronises `cuda_stream`, stores the word in
+ * *detail_out (may be NULL), clears it, and returns CCONV_EDEVICE_TIMEOUT if it was non-zero.  The
+ * kernels only ever OR bits into the word, so a wait that expired in any earlier call stays
+ * visible until it is read.  Allocates nothing. */
+int cconv_noalloc_status(void* cuda_stream, int* detail_out);
 
 /* ---- Pooling (Section 6) ---------------------------------------------------------------------
  * The loop nest of Eq. 1 without its Filter,

@@ -26,7 +26,7 @@ EXPORTS = (
     "cconv_plan_destroy", "cconv_plan_reserve_accumulate", "cconv_forward_accumulate",
     "cconv_forward_planned", "cconv_forward", "cconv_forward_host",
     "cconv_forward_host_async", "cconv_host_wait",
-    "cconv_forward_noalloc", "cconv_pool_lower_bound", "cconv_pool_forward",
+    "cconv_forward_noalloc", "cconv_noalloc_status", "cconv_pool_lower_bound", "cconv_pool_forward",
     "cconv_parallel_lower_bound", "cconv_parallel_partition", "cconv_theorem2_case",
     "cconv_plan_status", "cconv_plan_trace_read", "cconv_strerror", "cconv_last_cuda_error", "cconv_version",
 )
@@ -110,6 +110,8 @@ def load_library():
     lib.cconv_forward.argtypes = [vp, vp, vp] + nine + [i, vp]
     lib.cconv_forward_noalloc.restype = i
     lib.cconv_forward_noalloc.argtypes = [vp, vp, vp] + nine + [i, vp, ctypes.POINTER(i)]
+    lib.cconv_noalloc_status.restype = i
+    lib.cconv_noalloc_status.argtypes = [vp, ctypes.POINTER(i)]
     lib.cconv_forward_host.restype = i
     lib.cconv_forward_host.argtypes = [vp, vp, vp, vp, vp]
     lib.cconv_forward_host_async.restype = i
@@ -358,3 +360,11 @@ def conv_forward_noalloc(image, filt, out, B, C, K, W, H, R, S, sw=1, sh=1, out_
                                               ctypes.byref(st) if sync else None)
     _check(rc, f"cconv_forward_noalloc (device status {st.value:#x})")
     return out
+
+
+def noalloc_status(stream=None):
+    """cconv_noalloc_status: synchronises, returns (code, detail bit mask) of the asynchronous
+    cconv_forward_noalloc calls made so far on the current device, and clears the word."""
+    st = ctypes.c_int(0)
+    code = load_library().cconv_noalloc_status(_stream_ptr(stream), ctypes.byref(st))
+    return code, st.value

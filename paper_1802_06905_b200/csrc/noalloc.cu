@@ -103,18 +103,23 @@ extern "C" int cconv_forward_noalloc(const void* Image, const void* Filter, void
   rc = encode_image_map(view, tile, Image, &tm);
   if (rc != CCONV_OK) return rc;
   if (tile.smem_bytes > ds->prepared_smem) {
+    // (raises every instantiation to the device's limit: needed once per device)
     e = halo_kernel_prepare(tile.smem_bytes);
     if (e != cudaSuccess) return fail(e, "cudaFuncSetAttribute(max dynamic shared memory)");
-    ds->prepared_smem = tile.smem_bytes;
+    ds->prepared_smem = ds->machine.smem_optin_bytes;
   }
 
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   int* status = reinterpret_cast<int*>(ds->scratch);
   unsigned char* packed = ds->scratch + kStatusBytes;
-  // The array keeps whatever the last call left.  The status word must start at zero; the packed
-  // Filter is rewritten in full (zero padding included) by the packing kernel.
-  e = cudaMemsetAsync(status, 0, sizeof(int), stream);
-  if (e != cudaSuccess) return fail(e, "cudaMemsetAsync(status)");
+  // The array keeps whatever the last call left.  The packed Filter is rewritten in full (zero
+  // padding included) by the packing kernel; the status word only ever has bits OR-ed into it by the
+  // kernels and is cleared by whoever reads it (below, or cconv_noalloc_status).
+  // Stream order: the packing kernel is an ordinary launch, so everything in front of this call is
+  // complete before it reads anything; the convolution lets the kernel behind it start early, so the
+  // call is registered like a planned one (a following call that reads this Out will wait).
+  note_call(cuda_stream, spans_of(d, out_dtype, Image, Filter, Out), Overlap::kInputsEarly,
+            ds->machine.sm_count);
   e = launch_pack_filter(Filter, packed, d, tile.c16, tile.tiles_k, /*overlap_prev=*/false, stream);
   if (e != cudaSuccess) return fail(e, "launch_pack_filter");
   e = launch_halo(tm, packed, Out, out_dtype == CCONV_OUT_F32, kp, tile.grid, tile.smem_bytes, status,
@@ -126,7 +131,34 @@ extern "C" int cconv_forward_noalloc(const void* Image, const void* Filter, void
     if (e != cudaSuccess) return fail(e, "cudaMemcpyAsync(status)");
     e = cudaStreamSynchronize(stream);
     if (e != cudaSuccess) return fail(e, "cudaStreamSynchronize");
-    if (*device_status_out != 0) return CCONV_EDEVICE_TIMEOUT;
+    if (*device_status_out != 0) {
+      e = cudaMemsetAsync(status, 0, sizeof(int), stream);
+      if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+      if (e != cudaSuccess) return fail(e, "clearing the status word");
+      return CCONV_EDEVICE_TIMEOUT;
+    }
   }
   return CCONV_OK;
+}
+
+extern "C" int cconv_noalloc_status(void* cuda_stream, int* detail_out) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return fail(e, "cudaGetDevice");
+  std::lock_guard<std::mutex> lk(g_mu);
+  DeviceSetup* ds = nullptr;
+  const int rc = setup_device(dev, &ds);
+  if (rc != CCONV_OK) return rc;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  int* status = reinterpret_cast<int*>(ds->scratch);
+  int st = 0;
+  e = cudaMemcpyAsync(&st, status, sizeof(int), cudaMemcpyDeviceToHost, stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+  if (e == cudaSuccess && st != 0) {
+    e = cudaMemsetAsync(status, 0, sizeof(int), stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+  }
+  if (e != cudaSuccess) return fail(e, "reading the status word");
+  if (detail_out) *detail_out = st;
+  return st != 0 ? CCONV_EDEVICE_TIMEOUT : CCONV_OK;
 }

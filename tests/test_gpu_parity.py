@@ -402,6 +402,38 @@ def test_out_of_one_call_read_as_image_by_the_next_call_on_the_stream():
     plan_b.close()
 
 
+def test_out_of_one_call_read_as_filter_by_the_next_call_on_the_stream():
+    """The Filter-packing kernel of a call normally runs beside the previous call's convolution.  If
+    the previous call's Out IS this call's Filter ((K,H,W,B) of call A = (K,R,S,C) of call B), the
+    packing must wait until all of it has been written."""
+    a = cs("fchain_a", 64, 256, 128, 4, 5, 3, 3)                  # Out (128, 5, 4, 64) bf16
+    b = cs("fchain_b", 32, 64, 128, 6, 5, 5, 4)                   # Filter (128, 5, 4, 64)
+    a3 = cs("fchain_a3", 8, 64, 64, 3, 7, 3, 3)                   # Out (64, 7, 3, 8) bf16
+    b3 = cs("fchain_b3", 64, 8, 64, 12, 11, 7, 3, 2, 2)           # Filter (64, 7, 3, 8)
+    assert a.out_shape == b.filter_shape and a3.out_shape == b3.filter_shape
+    for pa, pb in ((a, b), (a3, b3)):
+        ia, fa = synth.make_inputs(pa)
+        ib, _ = synth.make_inputs(pb)
+        img_a, flt_a, img_b = to_dev(ia), to_dev(fa), to_dev(ib)
+        plan_a = binding.Plan(*pa.dims(), device=0, variant=binding.VARIANT_HALO, out_dtype=binding.OUT_BF16)
+        plan_b = binding.Plan(*pb.dims(), device=0, variant=binding.VARIANT_HALO, out_dtype=binding.OUT_F32)
+        mid = torch.zeros(pa.out_shape, dtype=torch.bfloat16, device="cuda")
+        out_b = torch.empty(pb.out_shape, dtype=torch.float32, device="cuda")
+        for rep in range(6):
+            mid.zero_()                                           # a stale Filter would be zeros
+            out_b.fill_(float("nan"))
+            plan_a.forward(img_a, flt_a, mid)
+            plan_b.forward(img_b, mid, out_b)
+            plan_a.check()
+            plan_b.check()
+            exp, ab = ocnn.cnn_bf16(ib, to_bits(mid), oshape(pb))
+            assert_close(out_b.cpu().numpy().astype(np.float64), exp, ab,
+                         what=f"{pb.name}: Out as Filter, repeat {rep}")
+        assert float(mid.float().abs().max()) > 0
+        plan_a.close()
+        plan_b.close()
+
+
 def test_two_plans_with_different_shared_memory_needs_stay_usable():
     """Plans share the kernels: creating a second plan with a smaller tile must not lower the
     shared-memory ceiling the first one needs."""

@@ -7,7 +7,8 @@ scratch in a fixed array inside the library, shared by every call.
 
 The test calls it through the C ABI twice in a row (the array keeps the first call's contents, so
 the second call is the one that shows stale state) and compares each result with the existing
-planned entry point on the same inputs, within the tolerance the parity tests use.  It is collected
+planned entry point on the same inputs and with the CPU oracle, within the tolerance the parity
+tests use.  It is collected
 last (file name) so that a run which stops at the first failure has already run everything else;
 it passes alone in a fresh process as well.
 """
@@ -21,7 +22,7 @@ from oracle import cnn as ocnn
 from paper_1802_06905_b200 import binding, synth
 from paper_1802_06905_b200.synth import ConvShape
 
-from gpu_util import TOL, oshape, to_dev
+from gpu_util import TOL, assert_close, oshape, to_bits, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -49,7 +50,7 @@ def test_noalloc_matches_planned_entry_point_twice_in_a_row(out_dtype):
         ib, fb = synth.make_inputs(c)
         img, flt = to_dev(ib), to_dev(fb)
         ref = planned_reference(c, img, flt, out_dtype)
-        _, ab = ocnn.cnn_bf16(ib, fb, oshape(c))
+        exp, ab = ocnn.cnn_bf16(ib, fb, oshape(c))
         for call in range(2):
             out = torch.full(c.out_shape, float("nan"), device="cuda",
                              dtype=torch.float32 if out_dtype == binding.OUT_F32 else torch.bfloat16)
@@ -57,6 +58,8 @@ def test_noalloc_matches_planned_entry_point_twice_in_a_row(out_dtype):
             got = out.float().cpu().numpy().astype(np.float64)
             assert not np.isnan(got).any(), f"{c.name} call {call}: unwritten outputs"
             assert np.all(np.abs(got - ref) <= TOL * ab), f"{c.name} call {call}: differs from planned path"
+            assert_close(got, exp, ab, what=f"{c.name} call {call} against the oracle",
+                         bf16_out=out_dtype == binding.OUT_BF16)
 
 
 def test_noalloc_async_calls_on_one_stream_are_ordered():
@@ -64,13 +67,41 @@ def test_noalloc_async_calls_on_one_stream_are_ordered():
     ib, fb = synth.make_inputs(c)
     img, flt = to_dev(ib), to_dev(fb)
     ref = planned_reference(c, img, flt, binding.OUT_F32)
-    _, ab = ocnn.cnn_bf16(ib, fb, oshape(c))
+    exp, ab = ocnn.cnn_bf16(ib, fb, oshape(c))
     outs = [torch.full(c.out_shape, float("nan"), device="cuda") for _ in range(2)]
     for o in outs:                                   # no synchronisation between the two calls
         binding.conv_forward_noalloc(img, flt, o, *c.dims(), out_dtype=binding.OUT_F32)
-    torch.cuda.synchronize()
+    assert binding.noalloc_status() == (binding.OK, 0)       # synchronises; no wait expired
     for o in outs:
-        assert np.all(np.abs(o.cpu().numpy().astype(np.float64) - ref) <= TOL * ab)
+        got = o.cpu().numpy().astype(np.float64)
+        assert np.all(np.abs(got - ref) <= TOL * ab)
+        assert_close(got, exp, ab, what="asynchronous call against the oracle")
+
+
+@pytest.mark.parametrize("variant", [binding.VARIANT_HALO, binding.VARIANT_DIRECT], ids=["halo", "direct"])
+def test_a_planned_call_reads_the_out_of_the_noalloc_call_in_front_of_it(variant):
+    """The convolution of a noalloc call lets the kernel behind it start early; a planned call whose
+    Image is that call's Out (shapes made to agree) must still see all of it."""
+    a = ConvShape("na_chain_a", 64, 96, 128, 24, 28, 3, 3, seed=81)        # Out (128, 28, 24, 64)
+    b = ConvShape("na_chain_b", 64, 24, 64, 126, 26, 3, 3, seed=82)        # Image (128, 28, 24, 64)
+    assert a.out_shape == b.image_shape
+    ia, fa = synth.make_inputs(a)
+    _, fb = synth.make_inputs(b)
+    img_a, flt_a, flt_b = to_dev(ia), to_dev(fa), to_dev(fb)
+    plan_b = binding.Plan(*b.dims(), device=0, variant=variant, out_dtype=binding.OUT_F32)
+    mid = torch.zeros(a.out_shape, dtype=torch.bfloat16, device="cuda")
+    out_b = torch.empty(b.out_shape, dtype=torch.float32, device="cuda")
+    for rep in range(6):
+        mid.zero_()                                               # stale values would be zeros
+        out_b.fill_(float("nan"))
+        binding.conv_forward_noalloc(img_a, flt_a, mid, *a.dims(), out_dtype=binding.OUT_BF16)
+        plan_b.forward(mid, flt_b, out_b)
+        plan_b.check()
+        assert binding.noalloc_status() == (binding.OK, 0)
+        exp, ab = ocnn.cnn_bf16(to_bits(mid), fb, oshape(b))
+        assert_close(out_b.cpu().numpy().astype(np.float64), exp, ab, what=f"planned after noalloc, repeat {rep}")
+    assert float(mid.float().abs().max()) > 0
+    plan_b.close()
 
 
 def test_noalloc_rejects_what_it_cannot_hold_or_run():
