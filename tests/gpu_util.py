@@ -76,4 +76,5 @@ def check_full(cs, variant=binding.VARIANT_AUTO, out_dtype=binding.OUT_F32, seed
                      bf16_out=out_dtype == binding.OUT_BF16)
     if n:
         print(f"{cs.name}: {n} of {got.size} bf16 outputs pass through the rounding clause only")
+    info["rounding_clause_only"] = n     # elements inside the band only after the store's rounding
     return info

@@ -276,6 +276,10 @@ def test_theorem2_leaf_matches_the_oracle_and_the_benchmark_shapes():
         assert alb == pytest.approx(alb_exp, rel=1e-12)
         seen.add(leaf)
     assert seen == {"1", "2.1", "2.2.1", "2.2.2.1", "2.2.2.2"}
+    # the two leaves no benchmark shape reaches, multiplied out by hand (Theorem 2's tree)
+    assert binding.theorem2_case(2, 3, 5, 4, 4, 4, 4, 16.0) == ("2.1", 480.0)
+    assert binding.theorem2_case(1, 10, 8, 5, 4, 3, 3, 64.0) == ("2.2.1", 720.0)
+    assert binding.theorem2_case(2, 2, 8, 5, 4, 3, 3, 64.0) == ("2.2.2.2", 320.0)
     # the stride-1 benchmark shapes at the shared memory of one CTA
     M = 116224.0
     assert binding.theorem2_case(*CONFIGS[0].dims()[:7], M)[0] == "1"

@@ -153,6 +153,31 @@ def test_theorem2_leaves_for_the_benchmark_shapes():
     assert ob.theorem2_case(d.B, d.C, d.K, d.W, d.H, d.R, d.S, M)[0] == "1"
 
 
+def test_theorem2_leaves_21_and_221_by_hand():
+    """Theorem 2 (Appendix A), the two leaves no benchmark shape reaches, multiplied out by hand.
+    Case 2.1: every array exceeds M and R*S >= M; ALB = K*C*H*W*B*R*S / M.
+    Case 2.2.1: R*S < M and M*R*S >= (B*H*W)^2; ALB = K*C*R*S."""
+    # B=2 C=3 K=5 W=H=4 R=S=4, M=16: CHWB = 96, KCRS = 240, KHWB = 160, all > 16; RS = 16 >= 16
+    leaf, alb = ob.theorem2_case(2, 3, 5, 4, 4, 4, 4, 16.0)
+    assert leaf == "2.1" and alb == 480.0            # 5*3*4*4*2*16 / 16
+    # one word more of fast memory and R*S < M: (BHW)^2 = 1024 > M*RS = 272, min(C,K) = 3 >= sqrt(17/16)
+    leaf, alb = ob.theorem2_case(2, 3, 5, 4, 4, 4, 4, 17.0)
+    assert leaf == "2.2.2.1" and alb == pytest.approx(480.0 * math.sqrt(16.0 / 17.0), rel=1e-15)
+    # B=1 C=10 K=8 W=5 H=4 R=S=3, M=64: CHWB = 200, KCRS = 720, KHWB = 160, all > 64; RS = 9 < 64;
+    # M*RS = 576 >= (BHW)^2 = 400
+    leaf, alb = ob.theorem2_case(1, 10, 8, 5, 4, 3, 3, 64.0)
+    assert leaf == "2.2.1" and alb == 720.0          # 8*10*3*3
+    # two images: (BHW)^2 = 1600 > 576, min(C,K) = 8 >= sqrt(64/9): Case 2.2.2.1, 8*10*40*sqrt(9/64)
+    leaf, alb = ob.theorem2_case(2, 10, 8, 5, 4, 3, 3, 64.0)
+    assert leaf == "2.2.2.1" and alb == pytest.approx(1200.0, rel=1e-15)
+    # ... and with too few channels for that, Case 2.2.2.2: max(KHWB, CHWB) = max(320, 80)
+    leaf, alb = ob.theorem2_case(2, 2, 8, 5, 4, 3, 3, 64.0)
+    assert leaf == "2.2.2.2" and alb == 320.0
+    # an array that fits: Case 1 whatever the rest says (CHWB = 40 <= 64)
+    leaf, alb = ob.theorem2_case(1, 2, 8, 5, 4, 3, 3, 64.0)
+    assert leaf == "1" and alb == 160.0              # max(40, 144, 160)
+
+
 def test_case_2221_lemma_tiling_is_admissible_and_attains_term5():
     # Lemma for case 2.2.2.1: bK=bC=sqrt(M/RS), bR=R, bS=S, bH*bW*bB=sqrt(M*RS); G=M^1.5 (RS)^0.5
     d = [c for c in CONFIGS if c.name == "cfg5_large_3x3"][0]
