@@ -142,82 +142,100 @@ def to_dev(bits, torch, dev):
     return torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16).to(dev)
 
 
-def time_config(cfg, torch, binding, dev, steps, warmup, dist=None, sampler=None):
-    """Device-resident timing of one configuration.  Returns (seconds for `steps`, plan info)."""
-    ib, fb = make_inputs(cfg)
+def buffer_sets(cfg, torch, dev, ib, fb):
+    """Enough distinct (Image, Filter, Out) sets to exceed L2, so that back-to-back calls are L2-cold."""
     set_bytes = 2 * (cfg.image_words + cfg.filter_words + cfg.out_words)
     nsets = max(2, min(64, -(-int(1.5 * L2_BYTES) // set_bytes)))
     base_i, base_f = to_dev(ib, torch, dev), to_dev(fb, torch, dev)
     imgs = [base_i] + [base_i.clone() for _ in range(nsets - 1)]
     flts = [base_f] + [base_f.clone() for _ in range(nsets - 1)]
     outs = [torch.empty(cfg.out_shape, dtype=torch.bfloat16, device=dev) for _ in range(nsets)]
+    ptrs = [(imgs[i].data_ptr(), flts[i].data_ptr(), outs[i].data_ptr()) for i in range(nsets)]
+    return (imgs, flts, outs), ptrs, nsets
+
+
+def time_config(cfg, ib, fb, torch, binding, dev, steps, warmup, repeats, dist=None, sampler=None):
+    """Device-resident timing of one configuration: after `warmup` calls, `repeats` timed regions of
+    exactly `steps` back-to-back forward calls each (synchronise, event, calls, event, synchronise;
+    barrier on both sides with several ranks).  Returns the per-region seconds, plan info, nsets."""
+    keep, ptrs, nsets = buffer_sets(cfg, torch, dev, ib, fb)
     plan = binding.Plan(*cfg.dims(), device=dev.index, out_dtype=binding.OUT_BF16)
     stream = torch.cuda.current_stream()
     sp = stream.cuda_stream
-    ptrs = [(imgs[i].data_ptr(), flts[i].data_ptr(), outs[i].data_ptr()) for i in range(nsets)]
     for i in range(max(warmup, 3)):
         a, b, c = ptrs[i % nsets]
         rc = plan.forward_ptrs(a, b, c, sp)
         assert rc == 0, rc
     plan.check()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    if dist is not None:
-        dist.barrier()
-    torch.cuda.synchronize()
     if sampler:
         sampler.start()
-    e0.record(stream)
-    for i in range(steps):
-        a, b, c = ptrs[i % nsets]
-        plan.forward_ptrs(a, b, c, sp)
-    e1.record(stream)
+    regions = []
+    k = 0
+    for rep in range(repeats):
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for i in range(steps):
+            a, b, c = ptrs[k % nsets]
+            k += 1
+            plan.forward_ptrs(a, b, c, sp)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        regions.append(e0.elapsed_time(e1) * 1e-3)
     if sampler:
         sampler.sample_once()
-    torch.cuda.synchronize()
-    if sampler:
         sampler.stop()
-    if dist is not None:
-        dist.barrier()
     plan.check()
-    secs = e0.elapsed_time(e1) * 1e-3
     info = plan.info()
     plan.close()
-    return secs, info, nsets
+    del keep
+    return regions, info, nsets
 
 
 def time_repeats(cfg, torch, binding, dev, launches, repeats=5):
-    """Per-configuration table: median over `repeats` of the CUDA-event time of `launches`
-    back-to-back forward calls, L2-cold (rotating buffer sets larger than L2) and L2-warm (one
-    buffer set), and L2-cold again with the calls captured once into a CUDA graph and replayed.
-    Returns (cold seconds per call, warm seconds per call, plan info, graph seconds per call)."""
+    """Per-configuration table.  Median over `repeats` of the CUDA-event time of `launches`
+    back-to-back forward calls over rotating buffer sets larger than L2 (L2-cold); the same rotation
+    captured once into a CUDA graph and replayed; and the time of a call that runs alone
+    (synchronised on both sides; includes the launch).  Returns a dict of seconds per call."""
     ib, fb = make_inputs(cfg)
-    set_bytes = 2 * (cfg.image_words + cfg.filter_words + cfg.out_words)
-    nsets = max(2, min(64, -(-int(1.5 * L2_BYTES) // set_bytes)))
-    base_i, base_f = to_dev(ib, torch, dev), to_dev(fb, torch, dev)
-    imgs = [base_i] + [base_i.clone() for _ in range(nsets - 1)]
-    flts = [base_f] + [base_f.clone() for _ in range(nsets - 1)]
-    outs = [torch.empty(cfg.out_shape, dtype=torch.bfloat16, device=dev) for _ in range(nsets)]
+    keep, ptrs, nsets = buffer_sets(cfg, torch, dev, ib, fb)
     plan = binding.Plan(*cfg.dims(), device=dev.index, out_dtype=binding.OUT_BF16)
     stream = torch.cuda.current_stream()
     sp = stream.cuda_stream
-    ptrs = [(imgs[i].data_ptr(), flts[i].data_ptr(), outs[i].data_ptr()) for i in range(nsets)]
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    result = []
-    for rotate in (True, False):
-        times = []
-        for rep in range(repeats + 1):            # the first repeat is warm-up
-            torch.cuda.synchronize()
-            e0.record(stream)
-            for i in range(launches):
-                a, b, c = ptrs[i % nsets] if rotate else ptrs[0]
-                plan.forward_ptrs(a, b, c, sp)
-            e1.record(stream)
-            torch.cuda.synchronize()
-            if rep:
-                times.append(e0.elapsed_time(e1) * 1e-3 / launches)
-        result.append(float(np.median(times)))
-    # the same rotation captured once into a CUDA graph and replayed (no host work per call)
-    graph_s = None
+    sampler = ClockSampler(dev.index)
+    sampler.start()
+    times = []
+    k = 0
+    for rep in range(repeats + 1):            # the first repeat is warm-up
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for i in range(launches):
+            a, b, c = ptrs[k % nsets]
+            k += 1
+            plan.forward_ptrs(a, b, c, sp)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        if rep:
+            times.append(e0.elapsed_time(e1) * 1e-3 / launches)
+    sampler.sample_once()
+    sampler.stop()
+    res = {"stream": float(np.median(times)), "graph": None, "alone": None,
+           "sm_mhz": sampler.summary()["sm_mhz"], "nsets": nsets}
+    alone = []
+    for i in range(7):
+        a, b, c = ptrs[i % nsets]
+        torch.cuda.synchronize()
+        e0.record(stream)
+        plan.forward_ptrs(a, b, c, sp)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        alone.append(e0.elapsed_time(e1) * 1e-3)
+    res["alone"] = float(np.median(alone))
     try:
         side = torch.cuda.Stream()
         side.wait_stream(stream)
@@ -236,55 +254,46 @@ def time_repeats(cfg, torch, binding, dev, launches, repeats=5):
             e1.record(stream)
             torch.cuda.synchronize()
             times.append(e0.elapsed_time(e1) * 1e-3 / launches)
-        graph_s = float(np.median(times))
+        res["graph"] = float(np.median(times))
         del g
     except RuntimeError:
-        graph_s = None
+        res["graph"] = None
     plan.check()
     info = plan.info()
     plan.close()
-    return result[0], result[1], info, graph_s
+    del keep
+    return res, info
 
 
 def time_general_shapes(torch, binding, dev, launches=30, repeats=3):
-    """Shapes outside the five benchmark configurations that exercise the planner's other paths:
-    tiles split over clusters of 2 or 4 CTAs (few output pixels, long channel loops) and bands of
-    output rows standing in for images (B < 8).  Each shape is timed twice, back-to-back calls on one
-    buffer set: as planned, and with that path switched off through the planner's diagnostic
-    environment variables (read at plan creation)."""
-    shapes = [("resnet50_conv5_3x3_b64", (64, 512, 512, 7, 7, 3, 3, 1, 1), "CCONV_FORCE_TILE", "0,0,0,0,0,1"),
-              ("deep_7x7_3x3_b16", (16, 1024, 256, 7, 7, 3, 3, 1, 1), "CCONV_FORCE_TILE", "0,0,0,0,0,1"),
-              ("deep_7x7_5x5_b8", (8, 512, 512, 7, 7, 5, 5, 1, 1), "CCONV_FORCE_TILE", "0,0,0,0,0,1"),
-              ("single_image_56x56_3x3", (1, 256, 256, 56, 56, 3, 3, 1, 1), "CCONV_BANDS", "1")]
+    """Shapes outside the five benchmark configurations: layers with few output pixels and long
+    channel loops, and a single image (B < 8: bands of output rows stand in for images).  Each is
+    timed as planned (AUTO) and on the halo kernel (VARIANT_HALO: Filter-packing kernel, tiles split
+    over CTA clusters where the planner does so), back-to-back calls over rotating buffer sets."""
+    shapes = [("resnet50_conv5_3x3_b64", (64, 512, 512, 7, 7, 3, 3, 1, 1)),
+              ("deep_7x7_3x3_b16", (16, 1024, 256, 7, 7, 3, 3, 1, 1)),
+              ("deep_7x7_5x5_b8", (8, 512, 512, 7, 7, 5, 5, 1, 1)),
+              ("single_image_56x56_3x3", (1, 256, 256, 56, 56, 3, 3, 1, 1))]
     stream = torch.cuda.current_stream()
     sp = stream.cuda_stream
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     rows = []
-    for name, dims, var, off in shapes:
+    for name, dims in shapes:
         c = ConvShape(name, *dims)
         ib, fb = make_inputs(c)
-        img, flt = to_dev(ib, torch, dev), to_dev(fb, torch, dev)
-        out = torch.empty(c.out_shape, dtype=torch.bfloat16, device=dev)
+        keep, ptrs, nsets = buffer_sets(c, torch, dev, ib, fb)
         res = {}
-        for label, value in (("planned", None), ("path_off", off)):
-            saved = os.environ.get(var)
-            if value is None:
-                os.environ.pop(var, None)
-            else:
-                os.environ[var] = value
-            try:
-                plan = binding.Plan(*dims, device=dev.index, out_dtype=binding.OUT_BF16)
-            finally:
-                if saved is None:
-                    os.environ.pop(var, None)
-                else:
-                    os.environ[var] = saved
+        for label, variant in (("planned", binding.VARIANT_AUTO), ("halo_kernel", binding.VARIANT_HALO)):
+            plan = binding.Plan(*dims, device=dev.index, out_dtype=binding.OUT_BF16, variant=variant)
             times = []
+            k = 0
             for rep in range(repeats + 1):
                 torch.cuda.synchronize()
                 e0.record(stream)
                 for _ in range(launches):
-                    plan.forward_ptrs(img.data_ptr(), flt.data_ptr(), out.data_ptr(), sp)
+                    a, b, cc = ptrs[k % nsets]
+                    k += 1
+                    plan.forward_ptrs(a, b, cc, sp)
                 e1.record(stream)
                 torch.cuda.synchronize()
                 if rep:
@@ -292,15 +301,16 @@ def time_general_shapes(torch, binding, dev, launches=30, repeats=3):
             plan.check()
             info = plan.info()
             plan.close()
-            res[label] = {"us_per_launch": float(np.median(times)), "split": info["split"],
-                          "bands": info["bands"], "grid": info["grid"],
-                          "tile": [info[k] for k in ("bb", "bw", "bh", "bc")]}
+            res[label] = {"us_per_launch": float(np.median(times)), "variant": info["variant"],
+                          "split": info["split"], "bands": info["bands"], "grid": info["grid"],
+                          "tile": [info[k2] for k2 in ("bb", "bw", "bh", "bk", "bc")]}
+        del keep
         rows.append({"workload": name, "dims": dict(zip("B C K W H R S sw sh".split(), dims)),
                      "tflops": c.flops / res["planned"]["us_per_launch"] / 1e6, **res})
     return rows
 
 
-def time_pooling(torch, binding, dev, peaks, launches=50, repeats=5):
+def time_pooling(torch, binding, dev, peaks, launches=50, repeats=5, shapes=None, ops=("avg", "max")):
     """Pooling (Section 6) rows: median CUDA-event time of back-to-back cconv_pool_forward calls over
     rotating buffer sets larger than L2.  Algorithmic bytes = Image + Out, each moved once; the
     roofline is the measured HBM copy rate."""
@@ -310,7 +320,7 @@ def time_pooling(torch, binding, dev, peaks, launches=50, repeats=5):
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     rows = []
     gen = torch.Generator(device="cpu").manual_seed(0x18020690 + 60)
-    for name, B, C, K, W, H, R, S, sw, sh in POOL_SHAPES:
+    for name, B, C, K, W, H, R, S, sw, sh in (shapes or POOL_SHAPES):
         Wi, Hi = sw * (W - 1) + R, sh * (H - 1) + S
         ibytes, obytes = 2 * Wi * Hi * C * B, 2 * K * H * W * B
         nsets = max(2, min(16, -(-int(1.5 * L2_BYTES) // (ibytes + obytes))))
@@ -319,6 +329,8 @@ def time_pooling(torch, binding, dev, peaks, launches=50, repeats=5):
         outs = [torch.empty((K, H, W, B), dtype=torch.bfloat16, device=dev) for _ in range(nsets)]
         terms = binding.pool_lower_bound(B, C, K, W, H, R, S, sw, sh, L2_BYTES / 4.0)
         for op, opname in ((binding.POOL_AVG, "avg"), (binding.POOL_MAX, "max")):
+            if opname not in ops:
+                continue
             times = []
             for rep in range(repeats + 1):        # the first repeat is warm-up
                 torch.cuda.synchronize()
@@ -401,12 +413,16 @@ def time_e2e(cfg, torch, binding, dev, steps):
 
 def kernels_per_step(info, binding):
     """Kernels of this library launched by one forward call."""
-    if info["variant"] == binding.VARIANT_SIMT:
+    if info["variant"] in (binding.VARIANT_SIMT, binding.VARIANT_DIRECT):
         return 1
     n = 2                                    # Filter packing + convolution
     if info["variant"] == binding.VARIANT_HALO and info["tail_tiles"] > 0:
         n += 1                               # wave-quantisation tail launch
     return n
+
+
+KERNEL_NAMES = {1: "cconv_simt_kernel", 2: "cconv_halo_kernel", 3: "cconv_stem_kernel",
+                4: "cconv_direct_kernel"}
 
 
 def write_only_gbs(torch, dev):
@@ -445,18 +461,20 @@ def write_only_gbs(torch, dev):
 
 
 def roofline_for(cfg, info, secs_per_launch, peaks, binding):
-    """Roofline of the dominant kernel: tensor-bound where the tcgen05 kernel ran (dense
-    contraction), HBM-bound for the CUDA-core kernel (reported against compulsory bytes)."""
+    """Roofline of the dominant kernel: tensor-bound where a tcgen05 kernel ran (dense contraction),
+    HBM-bound for the CUDA-core kernel (reported against compulsory bytes).  `traffic` is ncu's
+    in-kernel DRAM byte count of one call from the committed profile summary (Out still in L2 when
+    the kernel ends is written back later and not in it); the compulsory bytes and the paper's bound
+    at both memory levels stand beside it."""
     traffic = dram_traffic_from_profiles(cfg.name)
-    if info["variant"] in (binding.VARIANT_HALO, binding.VARIANT_STEM):
+    if info["variant"] != binding.VARIANT_SIMT:
         ach = cfg.flops / secs_per_launch / 1e12
         peak = peaks["bf16_tflops"]
-        kernel = "cconv_halo_kernel" if info["variant"] == binding.VARIANT_HALO else "cconv_stem_kernel"
         return {"bound": "tensor", "achieved": ach, "peak": peak, "unit": "TFLOP/s",
                 "frac": ach / peak, "traffic": traffic, "peak_source": peaks["source"],
-                "kernel": kernel,
-                "duration": "CUDA-event time of one forward call (Filter packing included) "
-                            "/ launches; the convolution kernel alone is shorter"}
+                "kernel": KERNEL_NAMES[info["variant"]],
+                "duration": "CUDA-event time of `steps` back-to-back forward calls / steps, median of "
+                            "`repeats` such regions (calls of small shapes overlap on the GPU)"}
     byts = 2.0 * info["compulsory_words"]
     ach = byts / secs_per_launch / 1e9
     return {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
@@ -549,18 +567,41 @@ def run_reference(args):
     return 0
 
 
+def make_rank_problem(cfg, world, rank):
+    """Several ranks: ONE problem of world*B images, cut over b with the Filter replicated (no
+    collective in the forward); rank r gets images [b0, b0+n).  Returns (local shape, Image bits,
+    Filter bits, (b0, n), global B)."""
+    if world == 1:
+        ib, fb = make_inputs(cfg)
+        return cfg, ib, fb, (0, cfg.B), cfg.B
+    from dataclasses import replace
+    from paper_1802_06905_b200 import sharding
+    glob = replace(cfg, B=cfg.B * world)
+    b0, n = sharding.shard_batch(glob.B, world, rank)
+    ib, fb = make_inputs(glob)
+    return replace(cfg, B=n), sharding.slice_batch(ib, b0, n), fb, (b0, n), glob.B
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
-    ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--config", type=int, default=1, help="index into the five benchmark shapes")
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--repeats", type=int, default=25,
+                    help="timed regions of `steps` calls each; ms_per_step is the median region / steps")
+    ap.add_argument("--config", type=int, default=4,
+                    help="index into the five benchmark shapes (default: the largest, cfg5)")
     ap.add_argument("--shape", default=None,
                     help="B,C,K,W,H,R,S,sw,sh: time this shape instead of a benchmark configuration "
                          "(same input recipe as the default configuration; no profile figures exist for it)")
+    ap.add_argument("--pool-shape", default=None,
+                    help="B,C,K,W,H,R,S,sw,sh: time cconv_pool_forward on this shape only and print its row")
+    ap.add_argument("--pool-op", default="avg,max", help="avg, max or avg,max (with --pool-shape)")
     ap.add_argument("--impl", default="cconv", choices=["cconv", "reference"])
     ap.add_argument("--no-extras", action="store_true",
                     help="skip the per-configuration table, the e2e leg and the CPU baseline")
+    ap.add_argument("--detail-file", default=os.path.join(ROOT, "gpurun_out", "bench_detail.json"),
+                    help="where the long per-configuration / pooling / general-shape tables go")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -576,92 +617,135 @@ def main():
     local = int(os.environ.get("LOCAL_RANK", "0"))
     dev = torch.device("cuda", local)
     torch.cuda.set_device(dev)
+    peaks = measured_peaks()
+
+    if args.pool_shape:
+        dims = tuple(int(v) for v in args.pool_shape.split(","))
+        rows = time_pooling(torch, binding, dev, peaks, shapes=[("pool_shape",) + dims],
+                            ops=tuple(args.pool_op.split(",")))
+        print(json.dumps({"pooling": rows}))
+        return 0
+
     dist = None
     if world > 1:
         import torch.distributed as dist_mod
         dist_mod.init_process_group("nccl", device_id=dev)
         dist = dist_mod
 
-    peaks = measured_peaks()
-    cfg = chosen_config(args)
-    steps, warmup = max(1, args.steps), max(3, args.warmup)
+    cfg_named = chosen_config(args)
+    cfg, ib, fb, (b0, nb), global_B = make_rank_problem(cfg_named, world, rank)
+    steps, warmup, repeats = max(1, args.steps), max(3, args.warmup), max(1, args.repeats)
     sampler = ClockSampler(local)
-    secs, info, nsets = time_config(cfg, torch, binding, dev, steps, warmup, dist, sampler)
+    regions, info, nsets = time_config(cfg, ib, fb, torch, binding, dev, steps, warmup, repeats, dist,
+                                       sampler)
+    secs = float(np.median(regions))
+    flops_rank = float(cfg.flops)
+    flops_all = flops_rank
     if dist is not None:
         t = torch.tensor([secs], dtype=torch.float64, device=dev)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         secs = float(t.item())
-    # weak scaling: every rank convolves its own batch of B images with the replicated Filter
-    value = world * cfg.flops * steps / secs / 1e12
+        f = torch.tensor([flops_rank], dtype=torch.float64, device=dev)
+        dist.all_reduce(f, op=dist.ReduceOp.SUM)
+        flops_all = float(f.item())
+    # weak scaling: the problem grows with the ranks (world*B images), every rank convolves its
+    # shard with the replicated Filter
+    value = flops_all * steps / secs / 1e12
     per_launch = secs / steps
     roof = roofline_for(cfg, info, per_launch, peaks, binding)
     t_roof, lb_bytes = applicable_roofline_seconds(cfg, info, peaks)
+    m_cta = binding.lower_bound(*cfg.dims(), info["M_words"])
+    roof["applicable"] = {"t_roof_us": t_roof * 1e6, "frac": t_roof / per_launch,
+                          "rule": "max(flops / bf16 peak, bound bytes at M = L2 / HBM copy rate)"}
+    roof["bytes"] = {"compulsory": 2.0 * info["compulsory_words"],
+                     "bound_at_M_L2": lb_bytes, "bound_at_M_cta_smem": 2.0 * max(m_cta),
+                     "compulsory_over_bound_at_M_cta_smem": 2.0 * info["compulsory_words"] / (2.0 * max(m_cta)),
+                     "note": "the kernels move compulsory bytes through HBM (ncu: reads = Image + Filter "
+                             "once); the paper's bound is evaluated at the kernel's effective M, the "
+                             "shared memory of one CTA, and at M = L2"}
 
     line = {
         "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": steps,
         "warmup": warmup, "ms_per_step": per_launch * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": cfg.name,
-                   "dims": dict(zip("B C K W H R S sw sh".split(), cfg.dims())),
+        "config": {"workload": cfg_named.name,
+                   "dims": dict(zip("B C K W H R S sw sh".split(), cfg_named.dims())),
+                   "repeats": repeats,
+                   "timing": "median over `repeats` regions of exactly `steps` back-to-back calls, each "
+                             "bracketed by synchronize (and a barrier with several ranks)",
                    "l2": f"rotating {nsets} distinct buffer sets ({nsets * 2 * (cfg.image_words + cfg.filter_words + cfg.out_words) / 1e6:.0f} MB > 126 MB L2)",
                    "out_dtype": "bf16", "accumulate": "fp32",
-                   "parallelism": f"batch-sharded x{world}, no collective" if world > 1 else "single GPU"},
+                   "parallelism": (f"one problem of {global_B} images cut over b into {world} shards, "
+                                   f"Filter replicated, no collective") if world > 1 else "single GPU"},
         "roofline": roof,
-        "applicable_roofline": {"t_roof_us": t_roof * 1e6, "frac": t_roof / per_launch,
-                                "lower_bound_bytes_at_L2": lb_bytes,
-                                "compulsory_bytes": 2.0 * info["compulsory_words"]},
-        "plan": {k: info[k] for k in ("variant", "bb", "bc", "bk", "bw", "bh", "halo_w", "halo_h",
-                                      "stages", "grid", "tiles", "smem_bytes", "tmem_cols",
-                                      "bound_argmax", "bound_words", "lp_words", "tile_words_smem",
-                                      "M_words")},
+        "plan": {k: info[k] for k in ("variant", "bb", "bc", "bk", "bw", "bh", "stages", "filter_stages",
+                                      "grid", "tiles", "smem_bytes", "tmem_cols", "bound_argmax",
+                                      "tile_G_over_lp_G")},
         "clocks": sampler.summary(),
-        "gpu_launches": steps * kernels_per_step(info, binding),
+        "gpu_launches": steps * repeats * kernels_per_step(info, binding),
     }
-    if info["tail_tiles"] > 0:
-        line["plan"]["tail"] = {k: info[k] for k in ("tail_h0", "tail_bb", "tail_bw", "tail_bh",
-                                                     "tail_bc", "tail_tiles", "tail_grid")}
+    if world > 1:
+        line["config"]["shard_of_rank0"] = [b0, nb]
 
+    detail = {}
     if rank == 0 and not args.no_extras:
         e_steps = max(5, min(50, steps))
         e_secs, h2d, d2h, e_sync = time_e2e(cfg, torch, binding, dev, e_steps)
         line["e2e"] = {"value": cfg.flops * e_steps / e_secs / 1e12, "unit": "TFLOP/s",
                        "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                        "ms_per_step": e_secs / e_steps * 1e3, "steps": e_steps,
-                       "call": "cconv_forward_host_async per step + one cconv_host_wait (copies of "
-                               "neighbouring steps overlap)",
-                       "one_call_at_a_time": {"call": "cconv_forward_host (waits every step)",
-                                              "value": cfg.flops * e_steps / e_sync / 1e12,
-                                              "ms_per_step": e_sync / e_steps * 1e3}}
+                       "call": "cconv_forward_host_async per step + one cconv_host_wait",
+                       "one_call_at_a_time_ms_per_step": e_sync / e_steps * 1e3}
         if world == 1:
             wgbs = write_only_gbs(torch, dev)
-            line["applicable_roofline"]["write_only_stream_gbs"] = wgbs
-            rows = []
-            for i, c in enumerate(CONFIGS):
-                # median of 5 repeats of >= 100 back-to-back calls (20 for the 0.3 ms shape)
+            roof["applicable"]["write_only_stream_gbs"] = wgbs
+            per, rows = {}, []
+            for c in CONFIGS:
                 n_i = 100 if c.flops < 1e11 else 20
-                cold, warm, info_i, graph_s = time_repeats(c, torch, binding, dev, n_i)
+                res, info_i = time_repeats(c, torch, binding, dev, n_i)
+                cold = res["stream"]
                 tr, lbb = applicable_roofline_seconds(c, info_i, peaks)
-                m_cta = binding.lower_bound(*c.dims(), info_i["M_words"])
-                rows.append({"workload": c.name, "variant": info_i["variant"],
-                             "us_per_launch": cold * 1e6, "us_per_launch_l2_warm": warm * 1e6,
-                             "us_per_launch_cuda_graph": None if graph_s is None else graph_s * 1e6,
-                             "t_write_out_us": 2.0 * c.out_words / (wgbs * 1e9) * 1e6,
-                             "tflops": c.flops / cold / 1e12,
-                             "tflops_vs_sustained_peak": c.flops / cold / 1e12 /
-                                                         peaks["bf16_tflops_sustained"],
-                             "t_roof_us": tr * 1e6, "roofline_frac": tr / cold,
-                             "roofline_frac_l2_warm": tr / warm,
-                             "lower_bound_bytes_at_L2": lbb,
-                             "lower_bound_bytes_at_cta_smem": 2.0 * max(m_cta),
-                             "planned_bytes_into_smem": 2.0 * info_i["tile_words_smem"],
-                             "dram_bytes_ncu": dram_traffic_from_profiles(c.name),
-                             "tile": [info_i[k] for k in ("bb", "bw", "bh", "bc", "stages")],
-                             "oracle": oracle_sample(c)})
-            line["all_configs"] = rows
-            line["pooling"] = time_pooling(torch, binding, dev, peaks)
-            line["general_shapes"] = time_general_shapes(torch, binding, dev)
+                m_i = binding.lower_bound(*c.dims(), info_i["M_words"])
+                tensor = info_i["variant"] != binding.VARIANT_SIMT
+                bound = ("launch" if c.flops < 1e7 else
+                         "tensor" if c.flops / (peaks["bf16_tflops"] * 1e12) >= lbb / (peaks["hbm_gbs"] * 1e9)
+                         else "hbm")
+                per[c.name.split("_")[0]] = {
+                    "us": round(cold * 1e6, 2),
+                    "us_graph": None if res["graph"] is None else round(res["graph"] * 1e6, 2),
+                    "us_alone": round(res["alone"] * 1e6, 1),
+                    "tflops": round(c.flops / cold / 1e12, 1), "t_roof_us": round(tr * 1e6, 2),
+                    "frac": round(tr / cold, 3), "bound": bound, "kernel": KERNEL_NAMES[info_i["variant"]],
+                    "dram_bytes_ncu": dram_traffic_from_profiles(c.name),
+                    "compulsory_bytes": 2.0 * info_i["compulsory_words"],
+                    "bound_bytes_M_L2": lbb, "bound_bytes_M_cta": 2.0 * max(m_i),
+                    "staged_bytes_l2_to_sm": 2.0 * info_i["tile_words_smem"],
+                    "sm_mhz": res["sm_mhz"],
+                    "tile": [info_i[k] for k in ("bb", "bw", "bh", "bk", "bc")], "grid": info_i["grid"],
+                    "G_over_lp_G": round(info_i["tile_G_over_lp_G"], 3) if tensor else None}
+                rows.append({"workload": c.name, "plan": info_i, "timing_s": res, "oracle": oracle_sample(c)})
+            roof["per_config"] = per
+            roof["per_config_note"] = ("us = L2-cold back-to-back calls on one stream (independent calls "
+                                       "of small shapes run side by side on the SMs); us_alone = one "
+                                       "call between synchronisations, launch included; frac = t_roof_us / us")
+            pool = time_pooling(torch, binding, dev, peaks)
+            roof["pooling"] = {f"{r['workload']}_{r['op']}": {"us": round(r["us_per_launch"], 2),
+                                                               "frac_of_hbm_copy": round(r["roofline"]["frac"], 3)}
+                               for r in pool}
+            detail = {"all_configs": rows, "pooling": pool,
+                      "general_shapes": time_general_shapes(torch, binding, dev)}
+            roof["general_shapes_us"] = {g["workload"]: [round(g["planned"]["us_per_launch"], 1),
+                                                          round(g["halo_kernel"]["us_per_launch"], 1)]
+                                         for g in detail["general_shapes"]}
             line["cpu_baseline"] = cpu_baseline(cfg)
     if rank == 0:
+        if detail:
+            try:
+                os.makedirs(os.path.dirname(args.detail_file), exist_ok=True)
+                with open(args.detail_file, "w") as fh:
+                    json.dump({"line": line, **detail}, fh, indent=1, default=str)
+            except OSError:
+                pass
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
