@@ -27,6 +27,26 @@ def test_shard_batch_partitions_every_batch_size():
             assert covered == list(range(B))
 
 
+def test_bench_ranks_cut_one_batch_of_world_times_b_images():
+    """What `bench.py --gpus N` gives rank r: images [b0, b0+n) of ONE problem with N*B images (same
+    seeded data on every rank), the Filter whole.  The shards partition the batch, their dims carry
+    the shard's B, and their Image is the matching slice of the global Image."""
+    import bench
+    cfg = synth.CONFIGS[1]
+    for world in (1, 2, 4):
+        from dataclasses import replace
+        glob = replace(cfg, B=cfg.B * world)
+        gi, gf = synth.make_inputs(glob)
+        covered = []
+        for r in range(world):
+            local, ib, fb, (b0, n), gB = bench.make_rank_problem(cfg, world, r)
+            assert gB == cfg.B * world and local.B == n and local.dims()[1:] == cfg.dims()[1:]
+            assert ib.shape == local.image_shape and fb.shape == cfg.filter_shape
+            assert np.array_equal(ib, gi[..., b0:b0 + n]) and np.array_equal(fb, gf)
+            covered += list(range(b0, b0 + n))
+        assert covered == list(range(cfg.B * world))
+
+
 def _free_port():
     s = socket.socket()
     s.bind(("127.0.0.1", 0))
