@@ -11,7 +11,7 @@ import ctypes
 import os
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "libcconv.so")
+_LIB_PATH = os.environ.get("CCONV_LIB_PATH") or os.path.join(_HERE, "libcconv.so")
 _lib = None
 
 OK = 0

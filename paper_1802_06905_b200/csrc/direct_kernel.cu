@@ -29,8 +29,12 @@ namespace cconv {
 
 namespace {
 
-// warp 0: Image producer (TMA), warp 1: MMA issuer, warps 2-5: epilogue, warp 6: Filter producer
-constexpr int kDirectThreads = 224;
+// warp 0: Image producer (TMA), warp 1: MMA issuer, warps 2-9: epilogue (two per quarter of the TMEM
+// lanes, taking alternate 128-byte pieces of a row: the conversion and shuffle chain of one warp hides
+// behind the other's), warp 10: Filter producer
+constexpr int kEpiWarps = 8;
+constexpr int kFilterWarp = 2 + kEpiWarps;
+constexpr int kDirectThreads = 32 * (kFilterWarp + 1);
 
 // All MMAs of one tap: NC16 channel steps x KT out-channel blocks x b_h output rows.  Built by the
 // whole warp (uniform values), issued by the elected lane.  `acc` applies to the first channel
@@ -147,7 +151,7 @@ __global__ void __launch_bounds__(kDirectThreads, 1)
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(bar_tfull + 8u * a, 1);
-      mbar_init(bar_tempty + 8u * a, 4);  // one arrival per epilogue warp
+      mbar_init(bar_tempty + 8u * a, kEpiWarps);  // one arrival per epilogue warp
     }
     mbar_init(bar_drain, 1);
     *abort_flag = 0;
@@ -193,8 +197,12 @@ __global__ void __launch_bounds__(kDirectThreads, 1)
             break;
           }
           const uint32_t full = bar_ifull + 8u * s;
-          mbar_arrive_expect_tx(full, p.img_stage_bytes);
-          tma_load_4d(img_ring + s * p.img_stage_bytes, &tm_image, b0, c0, x0, y0, full);
+          if (p.diag_mode == 2) {
+            mbar_arrive(full);  // diagnostics: no copies, the MMAs run on whatever the ring holds
+          } else {
+            mbar_arrive_expect_tx(full, p.img_stage_bytes);
+            tma_load_4d(img_ring + s * p.img_stage_bytes, &tm_image, b0, c0, x0, y0, full);
+          }
           if (seq == 0) CCONV_TRACE(2);
           if (++s == n_st) {
             s = 0;
@@ -205,7 +213,7 @@ __global__ void __launch_bounds__(kDirectThreads, 1)
       CCONV_TRACE(3);
       drain_ring(bar_ifull, seq, n_st, status, limit);
     }
-  } else if (warp == 6) {
+  } else if (warp == kFilterWarp) {
     // ===================== Filter producer (TMA boxes of tg taps) =====================
     if (lane == 0) {
       const uint32_t n_st = uint32_t(p.f_stages);
@@ -221,7 +229,9 @@ __global__ void __launch_bounds__(kDirectThreads, 1)
               break;
             }
             const uint32_t full = bar_ffull + 8u * s;
-            if (int(seq) != p.skip_filter_stage) {
+            if (p.diag_mode == 2) {
+              mbar_arrive(full);
+            } else if (int(seq) != p.skip_filter_stage) {
               mbar_arrive_expect_tx(full, p.filt_stage_bytes);
               tma_load_3d(filt_ring + s * p.filt_stage_bytes, &tm_filter, c0, k0, t0, full);
             }
@@ -253,6 +263,7 @@ __global__ void __launch_bounds__(kDirectThreads, 1)
   } else if (warp == 1) {
     // ===================== MMA issuer =====================
     const bool leader = elect_one();
+    const bool issuer = leader && p.diag_mode != 1;  // diagnostics: stages are consumed without MMAs
     uint32_t is = 0, iph = 0, fs = 0, fph = 0, abuf = 0, aph = 0;
     bool ok = true, first_tile = true;
     const int S = p.S, RS = p.R * p.S;
@@ -302,7 +313,7 @@ __global__ void __launch_bounds__(kDirectThreads, 1)
           uint32_t a16 = filt_ring16 + fs * filt16;
           const int ntap = RS - tap < tg ? RS - tap : tg;
           for (int j = 0; j < ntap; ++j) {
-            direct_issue_tap<BH, KT, NC16>(leader, bh, d_base, n_mma, a_lo0 | a16, a_hi,
+            direct_issue_tap<BH, KT, NC16>(issuer, bh, d_base, n_mma, a_lo0 | a16, a_hi,
                                            b_lo0 | (img_base16 + tap_off), b_hi, idesc, acc, ktile16,
                                            kstep16, hstep16);
             acc = 1;
@@ -353,12 +364,13 @@ __global__ void __launch_bounds__(kDirectThreads, 1)
         break;
       }
     }
-  } else {
+  } else if (warp >= 2 && warp < 2 + kEpiWarps) {
     // ===================== epilogue: TMEM -> registers -> Out =====================
     const int q = warp & 3;  // this warp may touch TMEM lanes [32q, 32q+32)
+    const int part = (warp - 2) >> 2;   // which of the quarter's warps this is
+    constexpr int kParts = kEpiWarps / 4;
     uint32_t abuf = 0, aph = 0;
     bool first_tile = true;
-    const int chunks = p.bb / 32;
     const bool wide_rows = (size_t(p.B) * sizeof(OutT)) % 32 == 0;
     for (int tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
       int t = tile;
@@ -374,24 +386,81 @@ __global__ void __launch_bounds__(kDirectThreads, 1)
       tc_fence_after();
       if (first_tile && threadIdx.x == 64) CCONV_TRACE(8);
       const uint32_t t_base = tmem_base + (uint32_t(q * 32) << 16) + abuf * uint32_t(p.acc_cols);
+      // A lane holds one out-channel row of the accumulator.  Stored lane by lane, a warp's store
+      // instruction would touch 32 different lines (one sector per out-channel plane), which an SM
+      // gets rid of at about 20 B/clk; whole 128-byte lines leave at 32 B/clk (measured).  So the
+      // four lanes of a quad exchange 32-byte sectors by warp shuffles (a 4x4 transpose) and then
+      // write the 128-byte piece of ONE row per store instruction: lane j of the quad stores sector
+      // j of the quad's rows 0..3.  A piece is 64 columns (bf16) or 32 columns (fp32).
+      constexpr int kPiece = sizeof(OutT) == 2 ? 64 : 32;   // columns per 128-byte piece
+      constexpr int kSec = kPiece / 4;                       // columns per 32-byte sector
+      const long long plane = (long long)p.H * p.W * p.B;   // elements of one out-channel plane
+      const int bb_shift = p.bb == 64 ? 6 : 5;
+      const int sj = lane & 3;
 #pragma unroll
       for (int kt = 0; kt < KT; ++kt) {
-        const int k = (ktile * KT + kt) * 128 + q * 32 + lane;
+        const int kq = (ktile * KT + kt) * 128 + q * 32 + (lane & ~3);  // first row of this lane's quad
         for (int hh = 0; hh < p.bh; ++hh) {
           const int h = ht * p.bh + hh;
-          for (int ww = 0; ww < p.bw; ++ww) {
-            const int w = wt * p.bw + ww;
-            const bool valid = (k < p.K) && (h < p.H) && (w < p.W);
-            for (int ch = 0; ch < chunks; ++ch) {
-              uint32_t v[32];
-              tmem_ld_32x32b_x32(t_base + uint32_t((kt * p.bh + hh) * p.n_mma + ww * p.bb + ch * 32), v);
+          if (h >= p.H) continue;
+          OutT* const rowq = out + (((long long)kq * p.H + h) * p.W + wt * p.bw) * p.B + b0;
+          const uint32_t col0 = uint32_t((kt * p.bh + hh) * p.n_mma);
+          for (int c = part * kPiece; c + kPiece <= p.n_mma; c += kParts * kPiece) {
+            uint32_t va[32], sec[4][8];
+            tmem_ld_32x32b_x32(t_base + col0 + uint32_t(c), va);
+            if constexpr (sizeof(OutT) == 2) {
+              uint32_t vb[32];
+              tmem_ld_32x32b_x32(t_base + col0 + uint32_t(c + 32), vb);
               tmem_ld_wait();
-              if (valid) {
-                OutT* dst = out + (((long long)k * p.H + h) * p.W + w) * p.B + b0 + ch * 32;
-                const int nb = p.B - (b0 + ch * 32);  // images left in the batch (block padded past B)
-                if (nb >= 32 && wide_rows) direct_store32(dst, v);
-                else if (nb > 0) direct_store_partial(dst, v, nb < 32 ? nb : 32);
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                sec[0][i] = pack_bf16x2(va[2 * i], va[2 * i + 1]);
+                sec[1][i] = pack_bf16x2(va[16 + 2 * i], va[17 + 2 * i]);
+                sec[2][i] = pack_bf16x2(vb[2 * i], vb[2 * i + 1]);
+                sec[3][i] = pack_bf16x2(vb[16 + 2 * i], vb[17 + 2 * i]);
               }
+            } else {
+              tmem_ld_wait();
+#pragma unroll
+              for (int i = 0; i < 32; ++i) sec[i >> 3][i & 7] = va[i];
+            }
+            quad_transpose_sectors(sec, lane);
+            // the sector this lane stores: columns cc .. cc + kSec of the run = images b .. of pixel ww
+            const int cc = c + kSec * sj;
+            const int ww = cc >> bb_shift, b = cc - (ww << bb_shift);
+            const int left = p.B - (b0 + b);   // images of the sector inside the batch (a multiple of 8)
+            if (wt * p.bw + ww < p.W && left > 0) {
+              OutT* const d0 = rowq + (long long)ww * p.B + b;
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                if (kq + j >= p.K) break;
+                OutT* dst = d0 + j * plane;
+                if (left >= kSec && wide_rows) {
+                  st_global_v8(dst, sec[j][0], sec[j][1], sec[j][2], sec[j][3], sec[j][4], sec[j][5],
+                               sec[j][6], sec[j][7]);
+                } else {
+                  // rows of Out that are not multiples of 32 bytes, or (bf16) a sector cut in half by
+                  // the end of the batch: 16-byte pieces
+                  *reinterpret_cast<uint4*>(dst) = make_uint4(sec[j][0], sec[j][1], sec[j][2], sec[j][3]);
+                  if (left >= kSec)
+                    *reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(dst) + 16) =
+                        make_uint4(sec[j][4], sec[j][5], sec[j][6], sec[j][7]);
+                }
+              }
+            }
+          }
+          const int c = p.n_mma & ~(kPiece - 1);
+          if (c < p.n_mma && part == 0) {
+            // bf16, n_mma = 32 mod 64: the last 32 columns (one pixel of a 32-image block), lane by lane
+            uint32_t v[32];
+            tmem_ld_32x32b_x32(t_base + col0 + uint32_t(c), v);
+            tmem_ld_wait();
+            const int ww = c >> bb_shift, b = c - (ww << bb_shift);
+            const int k = kq + sj, nb = p.B - (b0 + b);
+            if (k < p.K && wt * p.bw + ww < p.W && nb > 0) {
+              OutT* dst = rowq + sj * plane + (long long)ww * p.B + b;
+              if (nb >= 32 && wide_rows) direct_store32(dst, v);
+              else direct_store_partial(dst, v, nb < 32 ? nb : 32);
             }
           }
         }

@@ -171,6 +171,7 @@ void build_direct_params(const Dims& d, const DirectTile& t, DirectKernelParams*
   const uint32_t b_layout = b_row == 128 ? 2u : 4u;
   p.b_desc = make_smem_desc(uint32_t(d.sw) * p.slab_bytes, 8 * b_row, b_layout);
   p.wait_limit_ns = uint64_t(env_int("CCONV_WAIT_LIMIT_MS", 1000)) * 1000000ull;
+  p.diag_mode = env_int("CCONV_DIAG_MODE", 0);
   p.skip_filter_stage = -1;
   p.trace = nullptr;
 }

@@ -115,34 +115,6 @@ cudaError_t launch_pack_filter_stem(const void* filter, void* packed, const Dims
 // ------------------------------------------------------------------------------------------------
 // The kernel.  Persistent; tile = (128 out-channels) x (64 images) x (bhm output rows) x (bw pixels).
 // ------------------------------------------------------------------------------------------------
-// Four lanes of a quad each hold four 8-word (32-byte) sectors of their own accumulator row.
-// After the call lane q of the quad holds sector q of the quad's rows 0..3 (slot j = row j): a 4x4
-// transpose of sectors in two butterfly stages of warp shuffles.  With it the four lanes of a quad
-// write one whole 128-byte line of ONE row per store instruction, and a warp eight whole lines,
-// instead of 32 lanes writing one sector each to 32 different lines (one per out-channel plane),
-// which the memory system absorbs at well under half the rate.
-__device__ __forceinline__ void quad_transpose_sectors(uint32_t (&s)[4][8], int lane) {
-  const bool b0 = lane & 1, b1 = lane & 2;
-#pragma unroll
-  for (int c = 0; c < 4; c += 2) {
-#pragma unroll
-    for (int w = 0; w < 8; ++w) {
-      const uint32_t send = b0 ? s[c][w] : s[c + 1][w];
-      const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 1);
-      if (b0) s[c][w] = recv; else s[c + 1][w] = recv;
-    }
-  }
-#pragma unroll
-  for (int i = 0; i < 2; ++i) {
-#pragma unroll
-    for (int w = 0; w < 8; ++w) {
-      const uint32_t send = b1 ? s[i][w] : s[2 + i][w];
-      const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 2);
-      if (b1) s[i][w] = recv; else s[2 + i][w] = recv;
-    }
-  }
-}
-
 template <typename OutT>
 __global__ void __launch_bounds__(kStemThreads, 1)
     cconv_stem_kernel(const __grid_constant__ CUtensorMap tm_image,
