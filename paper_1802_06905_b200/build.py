@@ -14,7 +14,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcconv.so")
 SOURCES = ["kernels.cu", "direct_kernel.cu", "stem_kernel.cu", "api.cu", "host_setup.cu", "noalloc.cu", "pool.cu", "planner.cpp"]
-HEADERS = ["kernels.h", "planner.h", "host_setup.h", "ptx_sm100.cuh", os.path.join("..", "..", "include", "cconv.h")]
+HEADERS = ["kernels.h", "planner.h", "host_setup.h", "ptx_sm100.cuh", "direct_issue.cuh", os.path.join("..", "..", "include", "cconv.h")]
 
 
 def _nvcc() -> str:

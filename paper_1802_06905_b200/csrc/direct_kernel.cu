@@ -22,6 +22,7 @@
 // wait_prev and the producers start with griddepcontrol.wait.
 #include <cuda_bf16.h>
 
+#include "direct_issue.cuh"
 #include "kernels.h"
 #include "ptx_sm100.cuh"
 
@@ -38,27 +39,35 @@ constexpr int kDirectThreads = 32 * (kFilterWarp + 1);
 
 // All MMAs of one tap: NC16 channel steps x KT out-channel blocks x b_h output rows.  Built by the
 // whole warp (uniform values), issued by the elected lane.  `acc` applies to the first channel
-// step; later steps always accumulate.
+// step; later steps always accumulate.  ob[c*BH + hh]: offset of channel step c, output row hh in the
+// Image operand; od[kt*BH + hh]: column offset of that accumulator (both hoisted out of the loops).
+// For b_h of 1 or 2 the tap goes out as one straight-line PTX block (direct_issue.cuh): the issuing
+// thread pays several cycles per instruction, and a tcgen05.mma of 128 x N x 16 occupies the tensor
+// pipe for max(N/2, 75) cycles only, so every instruction between two MMAs counts.
 template <int BH, int KT, int NC16>
 __device__ __forceinline__ void direct_issue_tap(bool leader, int bh, uint32_t d, uint32_t n_mma,
                                                  uint32_t a_lo, uint32_t a_hi, uint32_t b_lo,
                                                  uint32_t b_hi, uint32_t idesc, uint32_t acc,
-                                                 uint32_t ktile16, uint32_t kstep16,
-                                                 uint32_t hstep16) {
+                                                 uint32_t ktile16, uint32_t kstep16, uint32_t hstep16,
+                                                 const uint32_t (&ob)[NC16 * (BH > 0 ? BH : 1)],
+                                                 const uint32_t (&od)[KT * (BH > 0 ? BH : 1)]) {
+#define CCONV_TAP(B_, K_, N_)                                             \
+  if constexpr (BH == B_ && KT == K_ && NC16 == N_) {                     \
+    direct_tap_##B_##_##K_##_##N_(leader, d, a_lo, a_hi, b_lo, b_hi, idesc, acc, ob, od); \
+    return;                                                               \
+  }
+  CCONV_TAP(1, 1, 1) CCONV_TAP(1, 1, 2) CCONV_TAP(1, 1, 4) CCONV_TAP(1, 2, 1) CCONV_TAP(1, 2, 2)
+  CCONV_TAP(1, 2, 4) CCONV_TAP(2, 1, 1) CCONV_TAP(2, 1, 2) CCONV_TAP(2, 1, 4) CCONV_TAP(2, 2, 1)
+  CCONV_TAP(2, 2, 2) CCONV_TAP(2, 2, 4)
+#undef CCONV_TAP
+  if constexpr (BH == 0) {
 #pragma unroll
-  for (int c = 0; c < NC16; ++c) {
-    const uint32_t accc = c == 0 ? acc : 1u;
+    for (int c = 0; c < NC16; ++c) {
+      const uint32_t accc = c == 0 ? acc : 1u;
 #pragma unroll
-    for (int kt = 0; kt < KT; ++kt) {
-      const uint64_t a_desc =
-          (uint64_t(a_hi) << 32) | (a_lo + uint32_t(c) * 2u + uint32_t(kt) * ktile16);
-      if constexpr (BH > 0) {
-#pragma unroll
-        for (int hh = 0; hh < BH; ++hh)
-          umma_bf16_if(leader, d + uint32_t(kt * BH + hh) * n_mma, a_desc,
-                       (uint64_t(b_hi) << 32) | (b_lo + uint32_t(c) * kstep16 + uint32_t(hh) * hstep16),
-                       idesc, accc);
-      } else {
+      for (int kt = 0; kt < KT; ++kt) {
+        const uint64_t a_desc =
+            (uint64_t(a_hi) << 32) | (a_lo + uint32_t(c) * 2u + uint32_t(kt) * ktile16);
         for (int hh = 0; hh < bh; ++hh)
           umma_bf16_if(leader, d + uint32_t(kt * bh + hh) * n_mma, a_desc,
                        (uint64_t(b_hi) << 32) | (b_lo + uint32_t(c) * kstep16 + uint32_t(hh) * hstep16),
@@ -264,7 +273,7 @@ __global__ void __launch_bounds__(kDirectThreads, 1)
     // ===================== MMA issuer =====================
     const bool leader = elect_one();
     const bool issuer = leader && p.diag_mode != 1;  // diagnostics: stages are consumed without MMAs
-    uint32_t is = 0, iph = 0, fs = 0, fph = 0, abuf = 0, aph = 0;
+    uint32_t iph = 0, fph = 0, abuf = 0, aph = 0;
     bool ok = true, first_tile = true;
     const int S = p.S, RS = p.R * p.S;
     const uint32_t slab16 = p.slab_bytes >> 4, row16 = uint32_t(p.halo_w) * slab16;
@@ -278,7 +287,20 @@ __global__ void __launch_bounds__(kDirectThreads, 1)
     const uint32_t idesc = p.idesc, n_mma = uint32_t(p.n_mma);
     const uint32_t n_ist = uint32_t(p.i_stages), n_fst = uint32_t(p.f_stages);
     const int bh = p.bh, tg = p.tg;
-    long long tw_i = 0, tw_f = 0;
+    uint32_t ob[NC16 * (BH > 0 ? BH : 1)], od[KT * (BH > 0 ? BH : 1)];
+#pragma unroll
+    for (int c = 0; c < NC16; ++c)
+#pragma unroll
+      for (int hh = 0; hh < (BH > 0 ? BH : 1); ++hh)
+        ob[c * (BH > 0 ? BH : 1) + hh] = uint32_t(c) * kstep16 + uint32_t(hh) * hstep16;
+#pragma unroll
+    for (int i = 0; i < KT * (BH > 0 ? BH : 1); ++i) od[i] = uint32_t(i) * n_mma;
+    // Ring positions are kept as running addresses (no multiplications in the loop), and nothing
+    // but the waits, the issue blocks and the commits sits between two MMAs: the tensor pipe queues
+    // very little work, so every instruction of this warp between two issue blocks is idle time.
+    uint32_t i_addr16 = img_ring16, f_addr16 = filt_ring16;
+    uint32_t i_full = bar_ifull, i_empty = bar_iempty, f_full = bar_ffull, f_empty = bar_fempty;
+    const uint32_t i_full_end = bar_ifull + 8u * n_ist, f_full_end = bar_ffull + 8u * n_fst;
     for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
       if (!mbar_wait_warp(bar_tempty + 8u * abuf, aph ^ 1u, abort_flag, status, kStatMmaWaitTmem, limit))
         break;
@@ -286,36 +308,67 @@ __global__ void __launch_bounds__(kDirectThreads, 1)
       const uint32_t d_base = tmem_base + abuf * uint32_t(p.acc_cols);
       uint32_t acc = 0;
       const long long tl0 = p.trace ? clock64() : 0;
-      for (int cc = 0; ok && cc < p.cchunks; ++cc) {
-        {
-          const long long w0 = p.trace ? clock64() : 0;
-          if (!mbar_wait_warp(bar_ifull + 8u * is, iph, abort_flag, status, kStatMmaWaitFull, limit)) {
+      if (RS == 1) {
+        // 1x1 filters: one tap, one Filter stage per channel block -- the leanest loop
+        bool stamp = first_tile && lane == 0;
+        for (int cc = p.cchunks; cc > 0; --cc) {
+          if (!mbar_wait_warp(i_full, iph, abort_flag, status, kStatMmaWaitFull, limit) ||
+              !mbar_wait_warp(f_full, fph, abort_flag, status, kStatMmaWaitFull, limit)) {
             ok = false;
             break;
           }
-          if (p.trace) tw_i += clock64() - w0;
+          tc_fence_after();
+          if (stamp) {
+            CCONV_TRACE(5);
+            stamp = false;
+          }
+          direct_issue_tap<BH, KT, NC16>(issuer, bh, d_base, n_mma, a_lo0 | f_addr16, a_hi,
+                                         b_lo0 | i_addr16, b_hi, idesc, acc, ktile16, kstep16, hstep16,
+                                         ob, od);
+          acc = 1;
+          if (leader) {
+            umma_commit(f_empty);
+            umma_commit(i_empty);
+          }
+          f_full += 8u;
+          f_empty += 8u;
+          f_addr16 += filt16;
+          if (f_full == f_full_end) {
+            f_full = bar_ffull;
+            f_empty = bar_fempty;
+            f_addr16 = filt_ring16;
+            fph ^= 1u;
+          }
+          i_full += 8u;
+          i_empty += 8u;
+          i_addr16 += img16;
+          if (i_full == i_full_end) {
+            i_full = bar_ifull;
+            i_empty = bar_iempty;
+            i_addr16 = img_ring16;
+            iph ^= 1u;
+          }
         }
-        tc_fence_after();
-        const uint32_t img_base16 = img_ring16 + is * img16;
+      } else
+      for (int cc = 0; cc < p.cchunks; ++cc) {
+        if (!mbar_wait_warp(i_full, iph, abort_flag, status, kStatMmaWaitFull, limit)) {
+          ok = false;
+          break;
+        }
         int tap = 0, sx = 0;
-        uint32_t tap_off = 0, col_off = 0;  // halo offset of the current tap, in 16 B units
+        uint32_t tap_off = i_addr16, col_off = i_addr16;  // Image view of the current tap, in 16 B units
         for (int fg = 0; fg < p.fgroups; ++fg) {
-          {
-            const long long w0 = p.trace ? clock64() : 0;
-            if (!mbar_wait_warp(bar_ffull + 8u * fs, fph, abort_flag, status, kStatMmaWaitFull, limit)) {
-              ok = false;
-              break;
-            }
-            if (p.trace) tw_f += clock64() - w0;
+          if (!mbar_wait_warp(f_full, fph, abort_flag, status, kStatMmaWaitFull, limit)) {
+            ok = false;
+            break;
           }
           tc_fence_after();
           if (first_tile && cc == 0 && fg == 0 && lane == 0) CCONV_TRACE(5);
-          uint32_t a16 = filt_ring16 + fs * filt16;
+          uint32_t a16 = f_addr16;
           const int ntap = RS - tap < tg ? RS - tap : tg;
           for (int j = 0; j < ntap; ++j) {
-            direct_issue_tap<BH, KT, NC16>(issuer, bh, d_base, n_mma, a_lo0 | a16, a_hi,
-                                           b_lo0 | (img_base16 + tap_off), b_hi, idesc, acc, ktile16,
-                                           kstep16, hstep16);
+            direct_issue_tap<BH, KT, NC16>(issuer, bh, d_base, n_mma, a_lo0 | a16, a_hi, b_lo0 | tap_off,
+                                           b_hi, idesc, acc, ktile16, kstep16, hstep16, ob, od);
             acc = 1;
             a16 += tap16;
             // next tap: one halo row down (s); after S rows one halo pixel to the right (r)
@@ -327,25 +380,32 @@ __global__ void __launch_bounds__(kDirectThreads, 1)
             }
           }
           tap += ntap;
-          if (leader) umma_commit(bar_fempty + 8u * fs);  // free once the MMAs so far have read it
-          if (++fs == n_fst) {
-            fs = 0;
+          if (leader) umma_commit(f_empty);  // free once the MMAs so far have read it
+          f_full += 8u;
+          f_empty += 8u;
+          f_addr16 += filt16;
+          if (f_full == f_full_end) {
+            f_full = bar_ffull;
+            f_empty = bar_fempty;
+            f_addr16 = filt_ring16;
             fph ^= 1u;
           }
         }
         if (!ok) break;
-        if (leader) umma_commit(bar_iempty + 8u * is);
-        if (++is == n_ist) {
-          is = 0;
+        if (leader) umma_commit(i_empty);
+        i_full += 8u;
+        i_empty += 8u;
+        i_addr16 += img16;
+        if (i_full == i_full_end) {
+          i_full = bar_ifull;
+          i_empty = bar_iempty;
+          i_addr16 = img_ring16;
           iph ^= 1u;
         }
       }
       if (!ok) break;
-      if (first_tile && lane == 0 && p.trace) {
-        p.trace[blockIdx.x * 16 + 13] = (unsigned long long)tw_i;
-        p.trace[blockIdx.x * 16 + 14] = (unsigned long long)tw_f;
+      if (first_tile && lane == 0 && p.trace)
         p.trace[blockIdx.x * 16 + 15] = (unsigned long long)(clock64() - tl0);
-      }
       if (leader) umma_commit(bar_tfull + 8u * abuf);  // accumulator complete
       if (first_tile && lane == 0) CCONV_TRACE(6);
       first_tile = false;
@@ -381,8 +441,29 @@ __global__ void __launch_bounds__(kDirectThreads, 1)
       const int b0 = bt * p.bb;
       // (every lane polls for itself and checks the abort flag each time; the decision to go on
       // must be the same in all lanes because the TMEM loads below are warp-wide)
-      const bool got = mbar_wait(bar_tfull + 8u * abuf, aph, abort_flag, status, kStatEpilogueWait, limit);
-      if (!__all_sync(0xffffffffu, got)) break;
+      // One lane polls, with pauses: 256 threads polling shared memory while the main loop runs would
+      // compete with the tensor core's own operand reads.
+      bool got = true;
+      if (lane == 0) {
+        uint64_t t0 = 0;
+        while (!mbar_try_wait(bar_tfull + 8u * abuf, aph)) {
+          __nanosleep(256);
+          if (*abort_flag) {
+            got = false;
+            break;
+          }
+          const uint64_t t = globaltimer_ns();
+          if (t0 == 0) {
+            t0 = t;
+          } else if (t - t0 > limit) {
+            *abort_flag = 1;
+            atomicOr(status, kStatEpilogueWait);
+            got = false;
+            break;
+          }
+        }
+      }
+      if (!__shfl_sync(0xffffffffu, got, 0)) break;
       tc_fence_after();
       if (first_tile && threadIdx.x == 64) CCONV_TRACE(8);
       const uint32_t t_base = tmem_base + (uint32_t(q * 32) << 16) + abuf * uint32_t(p.acc_cols);
