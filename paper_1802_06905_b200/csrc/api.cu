@@ -215,6 +215,7 @@ struct cconv_plan {
   void* d_packed = nullptr;  // 2 x packed_bytes
   size_t packed_bytes = 0;
   mutable unsigned calls = 0;
+  mutable unsigned stem_uses[2] = {0, 0};  // calls that used each packed-Filter buffer (stem kernel)
   unsigned long long* d_trace = nullptr;  // diagnostics: [grid][16] device time stamps
   int trace_rows = 0;
   // host-buffer entry point: device staging owned by the plan
@@ -299,13 +300,24 @@ static int launch_tensor_core(const cconv_plan* pl, const void* Image, const voi
     packed = static_cast<char*>(pl->d_packed) + (pl->calls++ & 1u) * pl->packed_bytes;
   }
   if (pl->variant == CCONV_VARIANT_STEM) {
-    cudaError_t es = launch_pack_filter_stem(Filter, packed, pl->d, pl->skp, !inputs_hazard, stream);
+    // The packing kernel and the convolution of a call run side by side (and beside the previous
+    // call's last tiles); the packed Filter is handed over through a counter in plan-owned memory,
+    // one per scratch buffer (see StemKernelParams::filter_ready).
+    StemKernelParams skp = pl->skp;
+    {
+      std::lock_guard<std::mutex> lk(pl->mu);
+      const unsigned buf = (pl->calls - 1u) & 1u;  // the buffer `packed` points to
+      skp.filter_ready = reinterpret_cast<unsigned int*>(pl->d_status) + 16 + 16 * buf;
+      skp.ready_target = ++pl->stem_uses[buf] * pack_filter_stem_blocks(skp);
+    }
+    skp.wait_prev = (inputs_hazard || pad) ? 1 : 0;
+    cudaError_t es = launch_pack_filter_stem(Filter, packed, pl->d, skp, !inputs_hazard, stream);
     if (es != cudaSuccess) return cuda_fail(es, "launch_pack_filter_stem");
     if (pad) {
       es = launch_pad(user_image, pl->d_img_pad, *pad, inputs_hazard, stream);
       if (es != cudaSuccess) return cuda_fail(es, "cconv_pad_bands_kernel");
     }
-    es = launch_stem(tmi, packed, Out, pl->out_dtype == CCONV_OUT_F32, pl->skp, pl->stile.grid,
+    es = launch_stem(tmi, packed, Out, pl->out_dtype == CCONV_OUT_F32, skp, pl->stile.grid,
                      pl->stile.smem_bytes, pl->d_status, stream);
     return es == cudaSuccess ? CCONV_OK : cuda_fail(es, "launch_stem");
   }
@@ -800,7 +812,11 @@ int cconv_forward_planned(const cconv_plan* pl, const void* Image, const void* F
                                   pl->dtile.smem_bytes, pl->d_status, stream);
     return e == cudaSuccess ? CCONV_OK : cuda_fail(e, "launch_direct");
   }
-  const bool inputs_hazard = note_call(cuda_stream, spans, Overlap::kInputsEarly, pl->m.sm_count);
+  // (the stem kernel's calls overlap like the direct kernel's: reads and writes beside earlier calls)
+  if (pl->variant == CCONV_VARIANT_STEM) spans.sms = double(pl->stile.grid);
+  const bool inputs_hazard =
+      note_call(cuda_stream, spans,
+                pl->variant == CCONV_VARIANT_STEM ? Overlap::kDeep : Overlap::kInputsEarly, pl->m.sm_count);
   // Batch sizes that are not multiples of 8: the kernels run on zero-padded copies (see cconv_plan).
   void* const user_out = Out;
   const void* const user_image = Image;

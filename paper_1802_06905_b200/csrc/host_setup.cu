@@ -232,6 +232,9 @@ void build_stem_params(const Dims& d, const StemTile& t, StemKernelParams* out) 
   // pixel's, sw Image columns (of kw rows x 128 B) further.
   p.b_desc = make_smem_desc(uint32_t(d.sw) * uint32_t(t.kw) * 128u, 1024, 2);
   p.wait_limit_ns = uint64_t(env_int("CCONV_WAIT_LIMIT_MS", 1000)) * 1000000ull;
+  p.filter_ready = nullptr;
+  p.ready_target = 0;
+  p.wait_prev = 0;
   p.trace = nullptr;
 }
 
@@ -295,7 +298,7 @@ bool note_call(void* stream, const CallSpans& c, Overlap how, int sm_count) {
     for (int i = sc.n - 1; i >= 0; --i) {
       ++keep;
       sms += sc.calls[i].sms;
-      if (sms > double(sm_count)) break;
+      if (sms >= double(sm_count)) break;  // no SM left on which an older call could still have a CTA
     }
     if (keep < sc.n) {
       for (int i = 0; i < keep; ++i) sc.calls[i] = sc.calls[sc.n - keep + i];

@@ -76,6 +76,13 @@ struct StemKernelParams {
   uint32_t idesc;
   uint64_t a_desc, b_desc;
   uint64_t wait_limit_ns;
+  // Hand-over of the packed Filter between the packing kernel and the convolution of one call, which
+  // run side by side: every block of the packing kernel adds 1 to *filter_ready when its stores are
+  // visible, and the convolution reads the Filter once the counter has reached ready_target (the
+  // total over all calls that used this scratch buffer so far).
+  unsigned int* filter_ready;
+  unsigned int ready_target;
+  int wait_prev;          // 1: nothing is read before the stream's earlier work is complete
   unsigned long long* trace;
 };
 
@@ -136,6 +143,10 @@ cudaError_t launch_pack_filter(const void* filter, void* packed, const Dims& d, 
 cudaError_t launch_pack_filter_stem(const void* filter, void* packed, const Dims& d,
                                     const StemKernelParams& p, bool overlap_prev,
                                     cudaStream_t stream);
+// Blocks of that launch (each adds 1 to StemKernelParams::filter_ready).
+unsigned int pack_filter_stem_blocks(const StemKernelParams& p);
+// Blocks of that launch (each adds 1 to StemKernelParams::filter_ready).
+unsigned int pack_filter_stem_blocks(const StemKernelParams& p);
 cudaError_t stem_kernel_prepare(int smem_bytes);
 cudaError_t launch_stem(const CUtensorMap& tm_image, const void* packed_filter, void* out,
                         bool out_f32, const StemKernelParams& p, int grid, int smem_bytes,

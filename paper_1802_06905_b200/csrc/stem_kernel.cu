@@ -36,8 +36,8 @@ namespace {
 
 // warp 0: producer, warp 1: MMA issuer, warps 2-9: epilogue (two warps per TMEM lane quarter, each
 // taking every other pixel of a tile)
-constexpr int kStemThreads = 320;
-constexpr int kStemEpiThreads = 256;
+constexpr int kStemEpiThreads = 256;              // 8 warps: two per TMEM lane quarter (16 warps spill: 39 us)
+constexpr int kStemThreads = 64 + kStemEpiThreads;
 constexpr int kFiltBars = 16;  // 16 KB Filter pieces: at most 14 fit in shared memory
 constexpr int kMaxAccBufs = 8;  // accumulator buffers in tensor memory: tmem_cols / acc_cols
 
@@ -55,7 +55,7 @@ constexpr int kMaxAccBufs = 8;  // accumulator buffers in tensor memory: tmem_co
 __global__ void __launch_bounds__(256)
     cconv_pack_filter_stem_kernel(const unsigned short* __restrict__ filter,
                                   uint4* __restrict__ packed, Dims d, int kpad, int bhm, int khalves,
-                                  long long slots) {
+                                  long long slots, unsigned int* __restrict__ ready) {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const long long slot = blockIdx.x * (long long)blockDim.x + threadIdx.x;
   if (slot < slots) {
@@ -90,7 +90,18 @@ __global__ void __launch_bounds__(256)
     o.w = e[6] | (uint32_t(e[7]) << 16);
     packed[slot] = o;
   }
+  // This block's part of the packed Filter is written: make it visible and count the block in.  The
+  // convolution of the same call (already running beside this kernel) reads the Filter once every
+  // block has been counted.
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0 && ready != nullptr) atomicAdd(ready, 1u);
+  // The kernel ends only after the kernel in front of it has (completion stays in stream order).
   asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+unsigned int pack_filter_stem_blocks(const StemKernelParams& p) {
+  return unsigned(((long long)p.filt_bytes / 16 + 255) / 256);
 }
 
 cudaError_t launch_pack_filter_stem(const void* filter, void* packed, const Dims& d,
@@ -109,7 +120,7 @@ cudaError_t launch_pack_filter_stem(const void* filter, void* packed, const Dims
   cfg.numAttrs = overlap_prev ? 1 : 0;
   return cudaLaunchKernelEx(&cfg, cconv_pack_filter_stem_kernel,
                             static_cast<const unsigned short*>(filter), static_cast<uint4*>(packed), d,
-                            p.kpad, p.bhm, p.khalves, slots);
+                            p.kpad, p.bhm, p.khalves, slots, p.filter_ready);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -176,11 +187,9 @@ __global__ void __launch_bounds__(kStemThreads, 1)
       bool ok = true;
       long long t_wait = 0;
       const uint32_t n_st = uint32_t(p.i_stages);
-      // The packed Filter is written by the kernel launched just before this one.  Once that
-      // kernel is complete (and with it everything older in the stream), the next packing kernel
-      // may start: it writes the other scratch buffer while this kernel runs.
-      asm volatile("griddepcontrol.wait;" ::: "memory");
-      asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+      // An Image (or Filter) that a call still running may be writing: wait for the stream's
+      // earlier work first.  Otherwise this kernel runs beside the kernels in front of it.
+      if (p.wait_prev) asm volatile("griddepcontrol.wait;" ::: "memory");
       // The first Image window goes out before the Filter: the first MMA needs both, and one
       // thread's copies are issued one after the other.
       for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x, ++it) {
@@ -203,6 +212,26 @@ __global__ void __launch_bounds__(kStemThreads, 1)
           ph ^= 1u;
         }
         if (it == 0) {
+          // The packed Filter comes from the packing kernel of this call, which runs beside this
+          // kernel: wait (bounded) until all its blocks have counted themselves in, then order the
+          // copies below behind that observation.
+          if (p.filter_ready != nullptr) {
+            const uint64_t t0 = globaltimer_ns();
+            unsigned int seen;
+            for (;;) {
+              asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(p.filter_ready) : "memory");
+              if (int(seen - p.ready_target) >= 0) break;
+              if (*abort_flag || globaltimer_ns() - t0 > limit) {
+                *abort_flag = 1;
+                atomicOr(status, kStatFilterWait);
+                ok = false;
+                break;
+              }
+              __nanosleep(64);
+            }
+            if (!ok) break;
+            asm volatile("fence.proxy.async;" ::: "memory");
+          }
           // the Filter in 16 KB pieces (four 4 KB blocks), each with its own barrier: the MMAs of
           // the first tile start on the first piece while the others are still in flight
           for (uint32_t off = 0, f = 0; off < p.filt_bytes; off += 16384u, ++f) {
@@ -215,7 +244,7 @@ __global__ void __launch_bounds__(kStemThreads, 1)
       if (tr) tr[2] = (unsigned long long)t_wait;
       drain_ring(bar_ifull, it, n_st, status, limit);
       const uint64_t t0 = globaltimer_ns();
-      for (uint32_t f = 0; f < (p.filt_bytes + 16383u) / 16384u; ++f) {
+      for (uint32_t f = 0; ok && f < (p.filt_bytes + 16383u) / 16384u; ++f) {
         while (!mbar_try_wait(bar_filt + 8u * f, 0)) {
           if (globaltimer_ns() - t0 > limit) {
             atomicOr(status, kStatDrainWait);
@@ -274,6 +303,10 @@ __global__ void __launch_bounds__(kStemThreads, 1)
           ok = mbar_wait_warp(bar_filt + 8u * f, 0, abort_flag, status, kStatMmaWaitFull, limit);
         tc_fence_after();
         filt_ready = true;
+        // The Filter of this CTA is resident: once every CTA is that far, the scratch buffer may be
+        // rewritten, so the kernels behind this one may start (the next call's packing kernel and
+        // convolution run beside this kernel's remaining tiles).
+        if (lane == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
         if (tr) t_filt = clock64() - f0;
         if (!ok) break;
       } else {
@@ -321,7 +354,7 @@ __global__ void __launch_bounds__(kStemThreads, 1)
   } else {
     // ===================== epilogue warps =====================
     const int q = warp & 3;            // this warp may touch TMEM lanes [32q, 32q+32)
-    const int eset = (warp - 2) >> 2;  // 0: even pixels of a tile, 1: odd pixels
+    const int eset = (warp - 2) >> 2;  // which of the quarter's warps: pixels eset, eset + 2, ... of a tile
     // TMEM lane L = j*kpad + kk: stacked output row j, out-channel kk (kpad is a power of two).  A
     // lane reads the 64 images of one pixel of its row; the sectors are then transposed within
     // quads of lanes (quad_transpose_sectors) so that a quad writes whole lines of Out.
@@ -359,7 +392,7 @@ __global__ void __launch_bounds__(kStemThreads, 1)
       const long long c1 = tr ? clock64() : 0;
       tc_fence_after();
       const uint32_t t_base = tmem_base + (uint32_t(q * 32) << 16) + abuf * uint32_t(p.acc_cols);
-      for (int px = eset; px < p.bw; px += 2) {
+      for (int px = eset; px < p.bw; px += kStemEpiThreads / 128) {
         uint32_t va[32], vb[32];
         const long long l0 = tr ? clock64() : 0;
         tmem_ld_32x32b_x32(t_base + uint32_t(px * 64), va);
@@ -430,6 +463,8 @@ __global__ void __launch_bounds__(kStemThreads, 1)
     tc_fence_after();
     tmem_dealloc(tmem_base, uint32_t(p.tmem_cols));
   }
+  // This kernel ran beside the kernels in front of it; it ends only after they have.
+  if (threadIdx.x == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
   if (tr && threadIdx.x == 0) tr[1] = globaltimer_ns();
 }
 
