@@ -211,6 +211,25 @@ int cconv_forward_accumulate(const cconv_plan* plan, const void* Image, const vo
 int cconv_forward(const void* Image, const void* Filter, void* Out, int B, int C, int K, int W,
                   int H, int R, int S, int sw, int sh, int out_dtype, void* cuda_stream);
 
+/* Eq. 1 on arrays with EXPLICIT STRIDES.  Section 2 of the paper defines the three arrays by their
+ * subscripts only -- Image(x, y, c, b), Filter(k, r, s, c), Out(k, h, w, b) -- and says nothing about
+ * how they lie in memory; the rest of this ABI fixes dense row-major storage (last subscript fastest).
+ * This entry point takes the element stride of every subscript instead (in the order written above;
+ * all positive; distinct index tuples of Out must map to distinct addresses), so the column-major
+ * reading (first subscript fastest), transposed arrays and windows of larger arrays are served too:
+ *   - strides equal to the dense row-major layout, pointers aligned as for cconv_forward: the planned
+ *     path (cconv_forward);
+ *   - Image with contiguous images (stride of b = 1) and x, y, c strides that are multiples of 8
+ *     elements (16 bytes), B % 8 == 0, Filter and Out dense and aligned: the tensor-core kernels on a
+ *     tensor map built from the strides (plan cached like cconv_forward's; the first call allocates);
+ *   - anything else: a CUDA-core kernel, one thread per output element, threads running along the
+ *     subscript of Out with the smallest stride (pointers need only their element's alignment).
+ * Asynchronous on `cuda_stream`; same error codes as cconv_forward. */
+int cconv_forward_strided(const void* Image, const int64_t image_strides[4], const void* Filter,
+                          const int64_t filter_strides[4], void* Out, const int64_t out_strides[4],
+                          int B, int C, int K, int W, int H, int R, int S, int sw, int sh,
+                          int out_dtype, void* cuda_stream);
+
 /* Eq. 1 on HOST buffers (same layouts; pinned memory gives true asynchronous copies): copies Image
  * and Filter to device staging buffers owned by the plan (allocated on first use), launches, copies
  * Out back, all on `cuda_stream`, then synchronises that stream.  Returns the device status too. */

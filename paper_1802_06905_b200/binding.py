@@ -24,7 +24,7 @@ POOL_AVG, POOL_MAX = 0, 1
 EXPORTS = (
     "cconv_lower_bound", "cconv_tiling_lp", "cconv_plan_create", "cconv_plan_info_get",
     "cconv_plan_destroy", "cconv_plan_reserve_accumulate", "cconv_forward_accumulate",
-    "cconv_forward_planned", "cconv_forward", "cconv_forward_host",
+    "cconv_forward_planned", "cconv_forward", "cconv_forward_strided", "cconv_forward_host",
     "cconv_forward_host_async", "cconv_host_wait",
     "cconv_forward_noalloc", "cconv_noalloc_status", "cconv_pool_lower_bound", "cconv_pool_forward",
     "cconv_parallel_lower_bound", "cconv_parallel_partition", "cconv_theorem2_case",
@@ -108,6 +108,9 @@ def load_library():
     lib.cconv_forward_accumulate.argtypes = [vp, vp, vp, vp, vp]
     lib.cconv_forward.restype = i
     lib.cconv_forward.argtypes = [vp, vp, vp] + nine + [i, vp]
+    i64p = ctypes.POINTER(ctypes.c_int64)
+    lib.cconv_forward_strided.restype = i
+    lib.cconv_forward_strided.argtypes = [vp, i64p, vp, i64p, vp, i64p] + nine + [i, vp]
     lib.cconv_forward_noalloc.restype = i
     lib.cconv_forward_noalloc.argtypes = [vp, vp, vp] + nine + [i, vp, ctypes.POINTER(i)]
     lib.cconv_noalloc_status.restype = i
@@ -368,3 +371,21 @@ def noalloc_status(stream=None):
     st = ctypes.c_int(0)
     code = load_library().cconv_noalloc_status(_stream_ptr(stream), ctypes.byref(st))
     return code, st.value
+
+
+def conv_forward_strided(image, filt, out, B, C, K, W, H, R, S, sw=1, sh=1, out_dtype=OUT_BF16,
+                         stream=None):
+    """cconv_forward_strided on torch CUDA tensors of ANY strides: ``image`` indexed (x, y, c, b),
+    ``filt`` (k, r, s, c), ``out`` (k, h, w, b); the strides are taken from the tensors."""
+    Wi, Hi = sw * (W - 1) + R, sh * (H - 1) + S
+    for name, t, shp in (("Image", image, (Wi, Hi, C, B)), ("Filter", filt, (K, R, S, C)),
+                         ("Out", out, (K, H, W, B))):
+        if tuple(t.shape) != shp or not t.is_cuda:
+            raise ValueError(f"{name}: CUDA tensor of shape {shp} expected, got {tuple(t.shape)}")
+    arr = lambda t: (ctypes.c_int64 * 4)(*[int(v) if v > 0 else 1 for v in t.stride()])
+    rc = load_library().cconv_forward_strided(
+        ctypes.c_void_p(image.data_ptr()), arr(image), ctypes.c_void_p(filt.data_ptr()), arr(filt),
+        ctypes.c_void_p(out.data_ptr()), arr(out), B, C, K, W, H, R, S, sw, sh, int(out_dtype),
+        _stream_ptr(stream))
+    _check(rc, "cconv_forward_strided")
+    return out

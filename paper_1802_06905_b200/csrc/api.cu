@@ -189,6 +189,8 @@ struct cconv_plan {
   cconv_plan* acc_twin = nullptr;
   float* d_acc = nullptr;
   ImageView view{};  // `drun`, or its unstrided equivalent for 1x1 filters with strides
+  bool strided_image = false;     // the Image is a view with explicit strides (cconv_forward_strided)
+  size_t image_span_bytes = 0;    // bytes from the Image's first to one past its last element
   int device = -1;
   int variant = CCONV_VARIANT_SIMT;
   int out_dtype = CCONV_OUT_BF16;
@@ -257,6 +259,8 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 
 std::mutex g_cache_mu;
 std::map<std::tuple<int, void*, int, int, int, int, int, int, int, int, int, int>, cconv_plan*> g_cache;
+std::map<std::tuple<int, void*, int, int, int, int, int, int, int, int, int, int, long long, long long, long long>, cconv_plan*>
+    g_cache_strided;
 
 }  // namespace
 
@@ -401,8 +405,11 @@ int cconv_tiling_lp(int B, int C, int K, int W, int H, int R, int S, int sw, int
   return tiling_lp(d, M_words, pooling != 0, tiles_out, G_out, words_out) ? CCONV_OK : CCONV_EINVAL;
 }
 
-int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, int R, int S,
-                      int sw, int sh, int device, double M_words, int variant, int out_dtype) {
+// `image_strides` (may be null): element strides of Image's subscripts (x, y, c, b) with b contiguous;
+// the tensor-core kernels then read the Image through a strided tensor map (no padded copies).
+static int plan_create_impl(cconv_plan** plan_out, int B, int C, int K, int W, int H, int R, int S,
+                            int sw, int sh, int device, double M_words, int variant, int out_dtype,
+                            const long long* image_strides) {
   if (!plan_out) return CCONV_EINVAL;
   *plan_out = nullptr;
   const Dims d{B, C, K, W, H, R, S, sw, sh};
@@ -428,6 +435,20 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
   pl->drun.B = (d.B * pl->bands + 7) / 8 * 8;
   pl->padded = pl->drun.B != d.B || pl->bands > 1;
   pl->view = image_view(pl->drun);
+  pl->image_span_bytes = size_t(d.Wi()) * d.Hi() * d.C * d.B * 2;
+  if (image_strides) {
+    if (pl->padded) {
+      delete pl;
+      return CCONV_EUNSUPPORTED;
+    }
+    // (a strided 1x1 filter is already planned on a subsampled view: compose the two)
+    pl->view.stride_w = image_strides[0] * (pl->view.dk.sw != d.sw ? d.sw : 1);
+    pl->view.stride_h = image_strides[1] * (pl->view.dk.sh != d.sh ? d.sh : 1);
+    pl->view.stride_c = image_strides[2];
+    pl->strided_image = true;
+    pl->image_span_bytes = size_t((d.Wi() - 1) * image_strides[0] + (d.Hi() - 1) * image_strides[1] +
+                                  (d.C - 1) * image_strides[2] + d.B) * 2;
+  }
   const Dims& dk = pl->view.dk;
   pl->device = device;
   pl->out_dtype = out_dtype;
@@ -463,7 +484,9 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
                 &dforce[4], &dforce[5], &dforce[6], &dforce[7], &dforce[8]);
 
   const bool halo_ok = halo_supported(dk, nullptr) && choose_halo_tile(dk, pl->m, force, &pl->tile);
-  const bool stem_ok = choose_stem_tile(pl->drun, pl->m, &pl->stile, env_int("CCONV_STEM_BW", 0));
+  // (the stem kernel reads the Image through a map of its own that needs the dense layout)
+  const bool stem_ok = !image_strides &&
+                       choose_stem_tile(pl->drun, pl->m, &pl->stile, env_int("CCONV_STEM_BW", 0));
   // the direct-Filter kernel runs on the caller's arrays only (no padded copies)
   const bool direct_ok = !pl->padded && direct_supported(dk, nullptr) &&
                          choose_direct_tile(dk, pl->m, dforce, &pl->dtile);
@@ -495,6 +518,10 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
                              double(d.K) * pl->drun.H * d.W * pl->drun.B * (out_dtype == CCONV_OUT_F32 ? 4 : 2);
       if (d.macs() < 4.0e6 || scratch > 4.0 * 1024 * 1024 * 1024) variant = CCONV_VARIANT_SIMT;
     }
+  }
+  if (image_strides && variant != CCONV_VARIANT_HALO && variant != CCONV_VARIANT_DIRECT) {
+    delete pl;
+    return CCONV_EUNSUPPORTED;  // the caller falls back to the CUDA-core kernel for any strides
   }
   pl->variant = variant;
   if (variant == CCONV_VARIANT_HALO) {
@@ -604,6 +631,12 @@ int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, 
   }
   *plan_out = pl;
   return CCONV_OK;
+}
+
+int cconv_plan_create(cconv_plan** plan_out, int B, int C, int K, int W, int H, int R, int S,
+                      int sw, int sh, int device, double M_words, int variant, int out_dtype) {
+  return plan_create_impl(plan_out, B, C, K, W, H, R, S, sw, sh, device, M_words, variant, out_dtype,
+                          nullptr);
 }
 
 int cconv_plan_info_get(const cconv_plan* pl, cconv_plan_info* o) {
@@ -771,6 +804,7 @@ int cconv_forward_planned(const cconv_plan* pl, const void* Image, const void* F
     return CCONV_EINVAL;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   CallSpans spans = spans_of(pl->d, pl->out_dtype, Image, Filter, Out);
+  spans.image.hi = spans.image.lo + pl->image_span_bytes;
   if (pl->variant == CCONV_VARIANT_SIMT) {
     note_call(cuda_stream, spans, Overlap::kNone, pl->m.sm_count);
     cudaError_t e = launch_simt(Image, Filter, Out, pl->out_dtype == CCONV_OUT_F32, pl->d, stream);
@@ -878,6 +912,78 @@ int cconv_forward(const void* Image, const void* Filter, void* Out, int B, int C
     }
   }
   return cconv_forward_planned(pl, Image, Filter, Out, cuda_stream);
+}
+
+int cconv_forward_strided(const void* Image, const int64_t image_strides[4], const void* Filter,
+                          const int64_t filter_strides[4], void* Out, const int64_t out_strides[4],
+                          int B, int C, int K, int W, int H, int R, int S, int sw, int sh,
+                          int out_dtype, void* cuda_stream) {
+  if (!Image || !Filter || !Out || !image_strides || !filter_strides || !out_strides) return CCONV_EINVAL;
+  const Dims d{B, C, K, W, H, R, S, sw, sh};
+  if (!d.positive()) return CCONV_EINVAL;
+  if (out_dtype != CCONV_OUT_BF16 && out_dtype != CCONV_OUT_F32) return CCONV_EINVAL;
+  for (int i = 0; i < 4; ++i)
+    if (image_strides[i] <= 0 || filter_strides[i] <= 0 || out_strides[i] <= 0) return CCONV_EINVAL;
+  const size_t oel = out_dtype == CCONV_OUT_F32 ? 4 : 2;
+  if ((reinterpret_cast<uintptr_t>(Image) & 1u) || (reinterpret_cast<uintptr_t>(Filter) & 1u) ||
+      (reinterpret_cast<uintptr_t>(Out) & (oel - 1)))
+    return CCONV_EINVAL;
+  const int64_t dense_i[4] = {int64_t(d.Hi()) * C * B, int64_t(C) * B, B, 1};
+  const int64_t dense_f[4] = {int64_t(R) * S * C, int64_t(S) * C, C, 1};
+  const int64_t dense_o[4] = {int64_t(H) * W * B, int64_t(W) * B, B, 1};
+  bool img_dense = true, flt_dense = true, out_dense = true;
+  for (int i = 0; i < 4; ++i) {
+    // (the stride of a subscript with a single value is never used)
+    const int ext_i[4] = {d.Wi(), d.Hi(), C, B}, ext_f[4] = {K, R, S, C}, ext_o[4] = {K, H, W, B};
+    img_dense = img_dense && (ext_i[i] == 1 || image_strides[i] == dense_i[i]);
+    flt_dense = flt_dense && (ext_f[i] == 1 || filter_strides[i] == dense_f[i]);
+    out_dense = out_dense && (ext_o[i] == 1 || out_strides[i] == dense_o[i]);
+  }
+  const bool aligned = aligned16(Image) && aligned16(Filter) && !(reinterpret_cast<uintptr_t>(Out) & 31u);
+  // 1. the ABI's own dense layout: the planned path
+  if (img_dense && flt_dense && out_dense && aligned)
+    return cconv_forward(Image, Filter, Out, B, C, K, W, H, R, S, sw, sh, out_dtype, cuda_stream);
+  // 2. a strided view of the Image whose images are contiguous and whose other strides keep 16-byte
+  //    alignment (a window of a larger array, padded rows, a channel slice), Filter and Out dense:
+  //    the tensor-core kernels read it through a tensor map built from the strides
+  const bool img_tma = (B == 1 || image_strides[3] == 1) && image_strides[0] % 8 == 0 &&
+                       image_strides[1] % 8 == 0 && image_strides[2] % 8 == 0 && B % 8 == 0;
+  if (img_tma && flt_dense && out_dense && aligned) {
+    int dev = 0;
+    CCONV_CUDA(cudaGetDevice(&dev));
+    cconv_plan* pl = nullptr;
+    int rc = CCONV_OK;
+    {
+      std::lock_guard<std::mutex> lk(g_cache_mu);
+      auto key = std::make_tuple(dev, cuda_stream, B, C, K, W, H, R, S, sw, sh, out_dtype,
+                                 (long long)image_strides[0], (long long)image_strides[1],
+                                 (long long)image_strides[2]);
+      auto it = g_cache_strided.find(key);
+      if (it == g_cache_strided.end()) {
+        const long long ist[4] = {image_strides[0], image_strides[1], image_strides[2], 1};
+        rc = plan_create_impl(&pl, B, C, K, W, H, R, S, sw, sh, dev, 0.0, CCONV_VARIANT_AUTO, out_dtype, ist);
+        g_cache_strided[key] = rc == CCONV_OK ? pl : nullptr;  // remember a refusal too
+      } else {
+        pl = it->second;
+        if (!pl) rc = CCONV_EUNSUPPORTED;
+      }
+    }
+    if (rc == CCONV_OK) return cconv_forward_planned(pl, Image, Filter, Out, cuda_stream);
+    if (rc != CCONV_EUNSUPPORTED) return rc;
+  }
+  // 3. any other strides (column-major storage, transposed arrays, ...): the CUDA-core kernel
+  StridedLayout L;
+  for (int i = 0; i < 4; ++i) {
+    L.image[i] = image_strides[i];
+    L.filter[i] = filter_strides[i];
+    L.out[i] = out_strides[i];
+    L.order[i] = i;
+  }
+  std::sort(L.order, L.order + 4, [&](int a, int b) { return out_strides[a] < out_strides[b]; });
+  note_ordinary_launch(cuda_stream);
+  cudaError_t e = launch_simt_strided(Image, Filter, Out, out_dtype == CCONV_OUT_F32, d, L,
+                                      static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? CCONV_OK : cuda_fail(e, "launch_simt_strided");
 }
 
 int cconv_forward_host(cconv_plan* pl, const void* hImage, const void* hFilter, void* hOut,

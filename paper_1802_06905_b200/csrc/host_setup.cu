@@ -114,7 +114,7 @@ int encode_image_map(const ImageView& v, const HaloTile& t, const void* image, C
   // A box lands in shared memory as [y][x][c][b]: one slab of b_c x b_b per halo pixel.
   const cuuint64_t dims[4] = {cuuint64_t(d.B), cuuint64_t(d.C), cuuint64_t(d.Wi()),
                               cuuint64_t(d.Hi())};
-  const cuuint64_t strides[3] = {cuuint64_t(d.B) * 2, cuuint64_t(v.stride_w) * 2,
+  const cuuint64_t strides[3] = {cuuint64_t(v.stride_c) * 2, cuuint64_t(v.stride_w) * 2,
                                  cuuint64_t(v.stride_h) * 2};
   const cuuint32_t box[4] = {cuuint32_t(t.bb), cuuint32_t(t.bc), cuuint32_t(t.halo_w),
                              cuuint32_t(t.halo_h)};

@@ -119,6 +119,61 @@ __global__ void __launch_bounds__(128) cconv_simt_taps_kernel(const __nv_bfloat1
   }
 }
 
+// Eq. 1 on arrays with explicit element strides per subscript (any layout: column-major storage,
+// views of larger arrays, ...).  One thread per output element; consecutive threads run along the
+// subscript of Out with the smallest stride, so that stores coalesce whatever the layout.
+template <typename OutT>
+__global__ void __launch_bounds__(256) cconv_simt_strided_kernel(const __nv_bfloat16* __restrict__ image,
+                                                                 const __nv_bfloat16* __restrict__ filter,
+                                                                 OutT* __restrict__ out, Dims d,
+                                                                 StridedLayout L) {
+  const long long total = (long long)d.K * d.H * d.W * d.B;
+  // order[0] is the fastest-varying subscript of Out (0 = k, 1 = h, 2 = w, 3 = b)
+  const int ext[4] = {d.K, d.H, d.W, d.B};
+  for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
+       idx += (long long)gridDim.x * blockDim.x) {
+    int sub[4];
+    long long t = idx;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int a = L.order[j];
+      sub[a] = int(t % ext[a]);
+      t /= ext[a];
+    }
+    const int k = sub[0], h = sub[1], w = sub[2], b = sub[3];
+    float acc = 0.f;
+    for (int r = 0; r < d.R; ++r)
+      for (int s = 0; s < d.S; ++s) {
+        const __nv_bfloat16* ip = image + (long long)(r + d.sw * w) * L.image[0] +
+                                  (long long)(s + d.sh * h) * L.image[1] + (long long)b * L.image[3];
+        const __nv_bfloat16* fp = filter + (long long)k * L.filter[0] + (long long)r * L.filter[1] +
+                                  (long long)s * L.filter[2];
+        for (int c = 0; c < d.C; ++c)
+          acc = fmaf(__bfloat162float(ip[(long long)c * L.image[2]]),
+                     __bfloat162float(fp[(long long)c * L.filter[3]]), acc);
+      }
+    store_out(out + (long long)k * L.out[0] + (long long)h * L.out[1] + (long long)w * L.out[2] +
+                  (long long)b * L.out[3],
+              acc);
+  }
+}
+
+cudaError_t launch_simt_strided(const void* image, const void* filter, void* out, bool out_f32,
+                                const Dims& d, const StridedLayout& L, cudaStream_t stream) {
+  const long long total = (long long)d.K * d.H * d.W * d.B;
+  long long blocks = (total + 255) / 256;
+  if (blocks > 148ll * 64) blocks = 148ll * 64;
+  if (blocks < 1) blocks = 1;
+  const __nv_bfloat16* im = static_cast<const __nv_bfloat16*>(image);
+  const __nv_bfloat16* fl = static_cast<const __nv_bfloat16*>(filter);
+  if (out_f32)
+    cconv_simt_strided_kernel<float><<<unsigned(blocks), 256, 0, stream>>>(im, fl, static_cast<float*>(out), d, L);
+  else
+    cconv_simt_strided_kernel<__nv_bfloat16><<<unsigned(blocks), 256, 0, stream>>>(
+        im, fl, static_cast<__nv_bfloat16*>(out), d, L);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_simt(const void* image, const void* filter, void* out, bool out_f32,
                         const Dims& d, cudaStream_t stream) {
   // Four out-channels per thread reuse each Image value four times; problems too small to fill

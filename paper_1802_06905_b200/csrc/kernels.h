@@ -128,6 +128,16 @@ cudaError_t launch_direct(const CUtensorMap& tm_image, const CUtensorMap& tm_fil
 cudaError_t launch_simt(const void* image, const void* filter, void* out, bool out_f32,
                         const Dims& d, cudaStream_t stream);
 
+// Element strides of the four subscripts of each array, in the paper's subscript order:
+// Image(x, y, c, b), Filter(k, r, s, c), Out(k, h, w, b); `order` lists Out's subscripts
+// (0 = k, 1 = h, 2 = w, 3 = b) from the smallest stride to the largest.
+struct StridedLayout {
+  long long image[4], filter[4], out[4];
+  int order[4];
+};
+cudaError_t launch_simt_strided(const void* image, const void* filter, void* out, bool out_f32,
+                                const Dims& d, const StridedLayout& L, cudaStream_t stream);
+
 // Filter [K][R][S][C] -> packed [k-tile][16-channel chunk][tap][4 KB block], zero padded.
 // overlap_prev: launch with programmatic stream serialization, so that the packing may run while
 // the kernel in front of it in the stream (normally the previous convolution, which signals early)

@@ -22,9 +22,10 @@ struct Dims {
 struct ImageView {
   Dims dk;
   long long stride_h, stride_w;
+  long long stride_c;  // between consecutive channels (B for a dense Image; b itself is contiguous)
 };
 inline ImageView image_view(const Dims& d) {
-  ImageView v{d, (long long)d.C * d.B, (long long)d.Hi() * d.C * d.B};
+  ImageView v{d, (long long)d.C * d.B, (long long)d.Hi() * d.C * d.B, (long long)d.B};
   if (d.R == 1 && d.S == 1 && (d.sw > 1 || d.sh > 1)) {
     v.stride_h *= d.sh;
     v.stride_w *= d.sw;
