@@ -115,7 +115,8 @@ __device__ __forceinline__ void direct_store32(OutT* dst, const uint32_t (&v)[32
 
 }  // namespace
 
-// BH: b_h at compile time (0 = any); KT: blocks of 128 out-channels per CTA; NC16: 16-channel steps
+// BH: MMAs per tap, channel step and out-channel block (b_h, or 1 for merged rows) at compile time
+// (0 = any); KT: blocks of 128 out-channels per CTA; NC16: 16-channel steps
 // per channel block (b_c / 16).
 template <typename OutT, int BH, int KT, int NC16>
 __global__ void __launch_bounds__(kDirectThreads, 1)
@@ -284,9 +285,9 @@ __global__ void __launch_bounds__(kDirectThreads, 1)
     const uint32_t img16 = p.img_stage_bytes >> 4, filt16 = p.filt_stage_bytes >> 4;
     const uint32_t tap16 = p.filt_tap_bytes >> 4, ktile16 = p.filt_ktile_bytes >> 4;
     const uint32_t img_ring16 = (img_ring >> 4) & 0x3FFFu, filt_ring16 = (filt_ring >> 4) & 0x3FFFu;
-    const uint32_t idesc = p.idesc, n_mma = uint32_t(p.n_mma);
+    const uint32_t idesc = p.idesc, n_mma = uint32_t(p.mma_n);
     const uint32_t n_ist = uint32_t(p.i_stages), n_fst = uint32_t(p.f_stages);
-    const int bh = p.bh, tg = p.tg;
+    const int bh = p.mma_rows, tg = p.tg;  // BH is mma_rows at compile time
     uint32_t ob[NC16 * (BH > 0 ? BH : 1)], od[KT * (BH > 0 ? BH : 1)];
 #pragma unroll
     for (int c = 0; c < NC16; ++c)
@@ -478,13 +479,18 @@ __global__ void __launch_bounds__(kDirectThreads, 1)
       const long long plane = (long long)p.H * p.W * p.B;   // elements of one out-channel plane
       const int bb_shift = p.bb == 64 ? 6 : 5;
       const int sj = lane & 3;
+      const uint32_t stage = smem0 + uint32_t(warp - 2) * 4608u;  // 32 rows of 144 bytes per warp
+      const bool via_smem = p.total_tiles <= int(gridDim.x) &&
+                            uint32_t(kEpiWarps) * 4608u <= bars - smem0;
 #pragma unroll
       for (int kt = 0; kt < KT; ++kt) {
-        const int kq = (ktile * KT + kt) * 128 + q * 32 + (lane & ~3);  // first row of this lane's quad
+        const int kw = (ktile * KT + kt) * 128 + q * 32;  // first out-channel of this warp's 32 rows
+        const int kq = kw + (lane & ~3);                  // first row of this lane's quad
         for (int hh = 0; hh < p.bh; ++hh) {
           const int h = ht * p.bh + hh;
           if (h >= p.H) continue;
-          OutT* const rowq = out + (((long long)kq * p.H + h) * p.W + wt * p.bw) * p.B + b0;
+          OutT* const roww = out + (((long long)kw * p.H + h) * p.W + wt * p.bw) * p.B + b0;
+          OutT* const rowq = roww + (long long)(lane & ~3) * plane;
           const uint32_t col0 = uint32_t((kt * p.bh + hh) * p.n_mma);
           for (int c = part * kPiece; c + kPiece <= p.n_mma; c += kParts * kPiece) {
             uint32_t va[32], sec[4][8];
@@ -505,17 +511,43 @@ __global__ void __launch_bounds__(kDirectThreads, 1)
 #pragma unroll
               for (int i = 0; i < 32; ++i) sec[i >> 3][i & 7] = va[i];
             }
-            quad_transpose_sectors(sec, lane);
             // the sector this lane stores: columns cc .. cc + kSec of the run = images b .. of pixel ww
             const int cc = c + kSec * sj;
             const int ww = cc >> bb_shift, b = cc - (ww << bb_shift);
             const int left = p.B - (b0 + b);   // images of the sector inside the batch (a multiple of 8)
-            if (wt * p.bw + ww < p.W && left > 0) {
-              OutT* const d0 = rowq + (long long)ww * p.B + b;
+            int row0, row_step;                 // this lane stores rows row0 + j*row_step of the warp's 32
+            if (via_smem) {
+              // A CTA with a single tile: the rings are idle by now, so the 4x4 exchange of sectors
+              // goes through shared memory (16 vector accesses instead of 64 shuffles and as many
+              // selects): every lane parks its 128-byte piece in a row of 144 bytes (the pitch keeps
+              // both phases free of bank conflicts), then reads sector sj of rows 8j + lane/4.
+              const uint32_t wrow = stage + uint32_t(lane) * 144u;
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                st_shared_v4(wrow + 32u * i, sec[i][0], sec[i][1], sec[i][2], sec[i][3]);
+                st_shared_v4(wrow + 32u * i + 16u, sec[i][4], sec[i][5], sec[i][6], sec[i][7]);
+              }
+              __syncwarp();
 #pragma unroll
               for (int j = 0; j < 4; ++j) {
-                if (kq + j >= p.K) break;
-                OutT* dst = d0 + j * plane;
+                const uint32_t rrow = stage + uint32_t(8 * j + (lane >> 2)) * 144u + 32u * uint32_t(sj);
+                ld_shared_v4(rrow, sec[j][0], sec[j][1], sec[j][2], sec[j][3]);
+                ld_shared_v4(rrow + 16u, sec[j][4], sec[j][5], sec[j][6], sec[j][7]);
+              }
+              __syncwarp();
+              row0 = lane >> 2;
+              row_step = 8;
+            } else {
+              quad_transpose_sectors(sec, lane);
+              row0 = lane & ~3;
+              row_step = 1;
+            }
+            if (wt * p.bw + ww < p.W && left > 0) {
+              OutT* const d0 = roww + (long long)row0 * plane + (long long)ww * p.B + b;
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                if (kw + row0 + j * row_step >= p.K) continue;
+                OutT* dst = d0 + (long long)(j * row_step) * plane;
                 if (left >= kSec && wide_rows) {
                   st_global_v8(dst, sec[j][0], sec[j][1], sec[j][2], sec[j][3], sec[j][4], sec[j][5],
                                sec[j][6], sec[j][7]);
@@ -643,9 +675,9 @@ cudaError_t launch_direct(const CUtensorMap& tm_image, const CUtensorMap& tm_fil
   cfg.numAttrs = 1;
   const int nc16 = p.bc / 16;
   if (out_f32)
-    return cudaLaunchKernelEx(&cfg, direct_fn<float>(p.kt, nc16, p.bh), tm_image, tm_filter,
+    return cudaLaunchKernelEx(&cfg, direct_fn<float>(p.kt, nc16, p.mma_rows), tm_image, tm_filter,
                               static_cast<float*>(out), p, status);
-  return cudaLaunchKernelEx(&cfg, direct_fn<__nv_bfloat16>(p.kt, nc16, p.bh), tm_image, tm_filter,
+  return cudaLaunchKernelEx(&cfg, direct_fn<__nv_bfloat16>(p.kt, nc16, p.mma_rows), tm_image, tm_filter,
                             static_cast<__nv_bfloat16*>(out), p, status);
 }
 

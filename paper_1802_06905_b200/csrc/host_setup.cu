@@ -157,8 +157,15 @@ void build_direct_params(const Dims& d, const DirectTile& t, DirectKernelParams*
   p.slab_bytes = uint32_t(t.bc) * t.bb * 2;
   p.b_kstep_bytes = 16u * t.bb * 2;
   // instruction descriptor: D=f32, A=B=bf16, A K-major [15]=0, B MN-major [16]=1, N>>3, M=128>>4
+  // Output rows whose pixels continue at the same pitch in the stage (no halo columns between
+  // the rows: R = S = 1 at stride 1) form one operand of n_mma*bh columns: one MMA instead of bh
+  // reads the Filter block from shared memory once instead of bh times.
+  const bool rows_merge = t.bh > 1 && d.sh * t.halo_w == t.bw * d.sw && p.n_mma * t.bh <= 256 &&
+                          (p.n_mma * t.bh) % 16 == 0 && env_int("CCONV_DIRECT_MERGE_ROWS", 1) != 0;
+  p.mma_rows = rows_merge ? 1 : t.bh;
+  p.mma_n = rows_merge ? p.n_mma * t.bh : p.n_mma;
   p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
-            (uint32_t(p.n_mma >> 3) << 17) | (uint32_t(128 >> 4) << 24);
+            (uint32_t(p.mma_n >> 3) << 17) | (uint32_t(128 >> 4) << 24);
   // A = Filter rows [128 out-channels][bc channels], K-major, one swizzle span per row (bc*2 = 128,
   // 64 or 32 bytes: layout type 2, 4, 6); SBO = 8 rows; the leading offset is not used by swizzled
   // K-major operands.  A 16-channel step advances the start address by 32 bytes inside the row.

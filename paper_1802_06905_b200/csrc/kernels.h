@@ -99,7 +99,10 @@ struct DirectKernelParams {
   int tg, fgroups;               // taps per Filter stage; Filter stages per channel chunk = ceil(R*S/tg)
   int i_stages, f_stages;
   int tiles_k, tiles_b, tiles_w, tiles_h, total_tiles;
-  int n_mma;                     // N of one MMA = bb*bw
+  int n_mma;                     // columns of one output row of the tile = bb*bw
+  int mma_rows, mma_n;           // MMAs per (tap, 16 channels, out-channel block) and the N of each:
+                                 // bh of n_mma columns, or, where the rows of a tile lie at one
+                                 // pixel pitch in the stage (no halo between them), 1 of n_mma*bh
   int acc_cols;                  // accumulator columns of one tile = n_mma*bh*kt
   int acc_bufs, tmem_cols;
   int wait_prev;                 // 1: an array of this call overlaps one of a call that may still be
