@@ -308,7 +308,10 @@ int cconv_pool_lower_bound(int B, int C, int K, int W, int H, int R, int S, int 
                            double M_words, double terms_out[3]);
 
 /* Pooling on device buffers of the current device, asynchronous on `cuda_stream`; one kernel, no
- * scratch memory, no device-side waits (so there is no status word to read).  op: CCONV_POOL_*;
+ * scratch memory, no spin waits (so there is no status word to read).  Like the convolutions it
+ * overlaps independent neighbours on its stream and keeps stream order by the same address-range
+ * bookkeeping (CCONV_POOL_OVERLAP=0 in the environment makes it an ordinary launch).
+ * op: CCONV_POOL_*;
  * out_dtype: CCONV_OUT_*.  Returns CCONV_EINVAL for null or misaligned pointers, non-positive
  * bounds or unknown op / out_dtype, CCONV_EUNSUPPORTED when H*W*B exceeds the grid limit
  * (about 5e11 elements), CCONV_ECUDA when the launch fails. */

@@ -300,12 +300,14 @@ bool note_call(void* stream, const CallSpans& c, Overlap how, int sm_count) {
   // forget the calls that must be complete by the time this one starts: walking back from the
   // latest call, everything behind more than sm_count SMs' worth of resident CTAs
   {
-    double sms = 0;
+    double sms = 0, sms_by_threads = 0;
     int keep = 0;
     for (int i = sc.n - 1; i >= 0; --i) {
       ++keep;
       sms += sc.calls[i].sms;
-      if (sms >= double(sm_count)) break;  // no SM left on which an older call could still have a CTA
+      sms_by_threads += sc.calls[i].sms_by_threads;
+      // no SM left on which an older call could still have a CTA
+      if (sms >= double(sm_count) || sms_by_threads >= double(sm_count)) break;
     }
     if (keep < sc.n) {
       for (int i = 0; i < keep; ++i) sc.calls[i] = sc.calls[sc.n - keep + i];

@@ -47,7 +47,11 @@ struct Span {
 };
 struct CallSpans {
   Span image, filter, out;
-  double sms = 0;  // SMs' worth of CTAs the call keeps resident (grid / CTAs per SM)
+  // SMs' worth of CTAs the call keeps resident, counted on one resource each: by shared / tensor
+  // memory (grid / CTAs per SM: the tensor-core kernels) and by thread slots (pooling blocks).
+  // Either sum reaching the SM count proves that the calls behind it are complete; a call adds
+  // nothing to a resource it hardly uses, which only keeps older calls on the list for longer.
+  double sms = 0, sms_by_threads = 0;
 };
 CallSpans spans_of(const Dims& d, int out_dtype, const void* Image, const void* Filter, const void* Out);
 

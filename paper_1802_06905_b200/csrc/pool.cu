@@ -35,7 +35,23 @@ struct PoolParams {
   int kper;           // k-planes written by one blockIdx.y
   int terms;          // C * R * S
   float inv_rs;       // 1 / (R*S)
+  int overlap;        // 1: launched so that the stream's next kernel may start before this one ends
+  int wait_prev;      // 1: wait for the stream's earlier work before touching memory
 };
+
+// Overlap with the stream's neighbours (as the convolution kernels do it): the next kernel may be
+// launched as soon as every block of this one has started; a call whose arrays meet those of a call
+// that may still be running waits for the earlier work first; and thread 0 of every block leaves
+// only after the kernel in front is complete, so completion still follows stream order.
+__device__ __forceinline__ void pool_enter(const PoolParams& p) {
+  if (p.overlap) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (p.wait_prev) asm volatile("griddepcontrol.wait;" ::: "memory");
+  }
+}
+__device__ __forceinline__ void pool_leave(const PoolParams& p) {
+  if (p.overlap && !p.wait_prev && threadIdx.x == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
+}
 
 template <int VEC>
 __device__ __forceinline__ void load_vec(const __nv_bfloat16* p, float (&x)[VEC]) {
@@ -81,6 +97,7 @@ template <typename OutT, int VEC, bool MAX, int VPB>
 __global__ void __launch_bounds__(256) cconv_pool_kernel(const __nv_bfloat16* __restrict__ image,
                                                          OutT* __restrict__ out, PoolParams p) {
   constexpr int G = 256 / VPB;
+  pool_enter(p);
   const int vi = threadIdx.x % VPB, g = threadIdx.x / VPB;
   const long long v = (long long)blockIdx.x * VPB + vi;
   const bool valid = v < p.total_v;
@@ -192,11 +209,13 @@ __global__ void __launch_bounds__(256) cconv_pool_kernel(const __nv_bfloat16* __
 #pragma unroll
     for (int i = 0; i < VEC; ++i) acc[i] *= p.inv_rs;
   }
-  if (!valid) return;
-  const int k0 = blockIdx.y * p.kper;
-  const int k1 = min(p.K, k0 + p.kper);
-  for (int k = k0 + g; k < k1; k += G)
-    store_vec<OutT, VEC>(out + ((long long)k * p.total_v + v) * VEC, acc);
+  if (valid) {
+    const int k0 = blockIdx.y * p.kper;
+    const int k1 = min(p.K, k0 + p.kper);
+    for (int k = k0 + g; k < k1; k += G)
+      store_vec<OutT, VEC>(out + ((long long)k * p.total_v + v) * VEC, acc);
+  }
+  pool_leave(p);
 }
 
 // The usual pooling layer (C = 1 with the channels folded into b, 8 images per thread, a 2x2 or
@@ -206,8 +225,12 @@ __global__ void __launch_bounds__(256) cconv_pool_kernel(const __nv_bfloat16* __
 template <typename OutT, int R, int S, bool MAX>
 __global__ void __launch_bounds__(256) cconv_pool_window_kernel(const __nv_bfloat16* __restrict__ image,
                                                                 OutT* __restrict__ out, PoolParams p) {
+  pool_enter(p);
   const unsigned v = blockIdx.x * 256u + threadIdx.x;   // the host sends total_v < 2^31 here
-  if (v >= unsigned(p.total_v)) return;
+  if (v >= unsigned(p.total_v)) {
+    pool_leave(p);
+    return;
+  }
   const unsigned pix = v / unsigned(p.nb), bv = v - pix * unsigned(p.nb);
   const unsigned h = pix / unsigned(p.W), w = pix - h * unsigned(p.W);
   const long long ystride = (long long)p.B, xstride = (long long)p.Hi * p.B;
@@ -251,6 +274,22 @@ __global__ void __launch_bounds__(256) cconv_pool_window_kernel(const __nv_bfloa
   const int k0 = blockIdx.y * p.kper;
   const int k1 = min(p.K, k0 + p.kper);
   for (int k = k0; k < k1; ++k) store_vec<OutT, 8>(out + ((long long)k * p.total_v + v) * 8, acc);
+  pool_leave(p);
+}
+
+template <typename OutT>
+cudaError_t pool_launch(void (*kernel)(const __nv_bfloat16*, OutT*, PoolParams), dim3 grid,
+                        cudaStream_t stream, const __nv_bfloat16* im, OutT* o, const PoolParams& p) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(256);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = p.overlap ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, im, o, p);
 }
 
 template <typename OutT, int R, int S>
@@ -258,9 +297,8 @@ cudaError_t launch_pool_window(const void* image, void* out, const PoolParams& p
                                cudaStream_t stream) {
   const __nv_bfloat16* im = static_cast<const __nv_bfloat16*>(image);
   OutT* o = static_cast<OutT*>(out);
-  if (mx) cconv_pool_window_kernel<OutT, R, S, true><<<grid, 256, 0, stream>>>(im, o, p);
-  else cconv_pool_window_kernel<OutT, R, S, false><<<grid, 256, 0, stream>>>(im, o, p);
-  return cudaGetLastError();
+  if (mx) return pool_launch(cconv_pool_window_kernel<OutT, R, S, true>, grid, stream, im, o, p);
+  return pool_launch(cconv_pool_window_kernel<OutT, R, S, false>, grid, stream, im, o, p);
 }
 
 template <typename OutT, int VEC, bool MAX>
@@ -268,13 +306,9 @@ cudaError_t launch_pool_t(const void* image, void* out, const PoolParams& p, int
                           cudaStream_t stream) {
   const __nv_bfloat16* im = static_cast<const __nv_bfloat16*>(image);
   OutT* o = static_cast<OutT*>(out);
-  if (vpb == 256)
-    cconv_pool_kernel<OutT, VEC, MAX, 256><<<grid, 256, 0, stream>>>(im, o, p);
-  else if (vpb == 32)
-    cconv_pool_kernel<OutT, VEC, MAX, 32><<<grid, 256, 0, stream>>>(im, o, p);
-  else
-    cconv_pool_kernel<OutT, VEC, MAX, 8><<<grid, 256, 0, stream>>>(im, o, p);
-  return cudaGetLastError();
+  if (vpb == 256) return pool_launch(cconv_pool_kernel<OutT, VEC, MAX, 256>, grid, stream, im, o, p);
+  if (vpb == 32) return pool_launch(cconv_pool_kernel<OutT, VEC, MAX, 32>, grid, stream, im, o, p);
+  return pool_launch(cconv_pool_kernel<OutT, VEC, MAX, 8>, grid, stream, im, o, p);
 }
 
 }  // namespace
@@ -317,6 +351,9 @@ extern "C" int cconv_pool_forward(const void* Image, void* Out, int B, int C, in
   p.total_v = (long long)H * W * p.nb;
   p.terms = C * R * S;
   p.inv_rs = 1.0f / (float(R) * float(S));
+  p.overlap = 1;
+  if (const char* ov = std::getenv("CCONV_POOL_OVERLAP")) p.overlap = std::atoi(ov) != 0;
+  p.wait_prev = 0;
   // Vectors per block: a thread per vector when there is little to share (few terms, few planes);
   // otherwise 32, or 8 when 32 would leave most SMs without a block and the reduction outweighs
   // the writes (8 lanes per plane make 128-byte write runs instead of 512-byte ones).
@@ -346,6 +383,26 @@ extern "C" int cconv_pool_forward(const void* Image, void* Out, int B, int C, in
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   const bool f32 = out_dtype == CCONV_OUT_F32, mx = op == CCONV_POOL_MAX;
   cudaError_t e;
+  if (p.overlap) {
+    // stream order against the calls that may still be running: this call's blocks (256 threads of
+    // an SM's 2048 each) all stay resident until the kernel in front is complete
+    int dev = 0, sm_count = 0;
+    e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) {
+      set_last_cuda_error(std::string("cconv_pool_forward: ") + cudaGetErrorString(e));
+      return CCONV_ECUDA;
+    }
+    CallSpans spans;
+    spans.image.lo = static_cast<const char*>(Image);
+    spans.image.hi = spans.image.lo + size_t(Wi * Hi) * size_t(C) * size_t(B) * 2;
+    spans.out.lo = static_cast<const char*>(Out);
+    spans.out.hi = spans.out.lo + size_t(K) * H * W * size_t(B) * (f32 ? 4 : 2);
+    spans.sms_by_threads = double(blocks) * double(ksplit) / 8.0;
+    p.wait_prev = note_call(cuda_stream, spans, Overlap::kDeep, sm_count) ? 1 : 0;
+  } else {
+    note_ordinary_launch(cuda_stream);
+  }
   const bool window33 = R == 3 && S == 3, window22 = R == 2 && S == 2;
   if (C == 1 && vec == 8 && vpb == 256 && (window33 || window22) && p.total_v < 0x7fffffffll &&
       !std::getenv("CCONV_POOL_FORCE")) {
