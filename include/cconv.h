@@ -130,6 +130,12 @@ typedef struct {
    * must wait for the call in front takes) and the period of a stream of independent calls, which
    * run side by side on the SMs. */
   double est_cta_cycles, est_period_cycles;
+  /* The variant that runs a call which has to wait for the stream's earlier work because its arrays
+   * conflict with a call that may still be running (see the stream-order paragraph above).  AUTO
+   * plans that took DIRECT, whose tiling is chosen for a stream of independent calls, keep a HALO
+   * plan of the same problem for such calls, since one call alone finishes sooner on many small
+   * tiles (CCONV_WAIT_TWIN=0 at plan creation: no second plan); otherwise equal to `variant`. */
+  int wait_variant;
 } cconv_plan_info;
 
 /* Theorem 1 (Section 4.1): the five lower-bound terms, in words, for a fast memory of M_words.

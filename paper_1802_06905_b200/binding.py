@@ -63,6 +63,7 @@ class PlanInfo(ctypes.Structure):
         ("filter_taps", ctypes.c_int),
         ("tile_G", ctypes.c_double), ("tile_G_over_lp_G", ctypes.c_double),
         ("est_cta_cycles", ctypes.c_double), ("est_period_cycles", ctypes.c_double),
+        ("wait_variant", ctypes.c_int),
     ]
 
     def asdict(self):

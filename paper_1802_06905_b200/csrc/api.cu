@@ -187,6 +187,10 @@ struct cconv_plan {
   void* d_out_pad = nullptr;
   // cconv_plan_reserve_accumulate: the same plan with fp32 Out and an fp32 array of Out's shape
   cconv_plan* acc_twin = nullptr;
+  // AUTO plans that took the direct kernel (tiled for a stream of independent calls): the same
+  // problem planned for the halo kernel, whose many small tiles finish one call sooner.  A call
+  // that has to wait for the stream's earlier work cannot run beside it and takes this plan.
+  cconv_plan* wait_twin = nullptr;
   float* d_acc = nullptr;
   ImageView view{};  // `drun`, or its unstrided equivalent for 1x1 filters with strides
   bool strided_image = false;     // the Image is a view with explicit strides (cconv_forward_strided)
@@ -483,6 +487,7 @@ static int plan_create_impl(cconv_plan** plan_out, int B, int C, int K, int W, i
     std::sscanf(f, "%d,%d,%d,%d,%d,%d,%d,%d,%d", &dforce[0], &dforce[1], &dforce[2], &dforce[3],
                 &dforce[4], &dforce[5], &dforce[6], &dforce[7], &dforce[8]);
 
+  bool want_wait_twin = false;
   const bool halo_ok = halo_supported(dk, nullptr) && choose_halo_tile(dk, pl->m, force, &pl->tile);
   // (the stem kernel reads the Image through a map of its own that needs the dense layout)
   const bool stem_ok = !image_strides &&
@@ -508,8 +513,10 @@ static int plan_create_impl(cconv_plan** plan_out, int B, int C, int K, int W, i
     const char* objective = std::getenv("CCONV_OBJECTIVE");
     const bool want_latency = objective && std::strcmp(objective, "latency") == 0;
     if (variant == CCONV_VARIANT_HALO && direct_ok && !want_latency &&
-        pl->dtile.tiles <= pl->m.sm_count && d.macs() >= 4.0e6)
+        pl->dtile.tiles <= pl->m.sm_count && d.macs() >= 4.0e6) {
       variant = CCONV_VARIANT_DIRECT;
+      want_wait_twin = device >= 0 && env_int("CCONV_WAIT_TWIN", 1) != 0;
+    }
     // A padded batch costs two more kernels (about 15 us per call in all, measured) and two scratch
     // arrays: worth it unless the problem is tiny (the CUDA-core kernel needs 8 us for 0.5 M
     // multiply-adds, 25-50 us for 7-15 M), and only within 4 GiB of scratch.
@@ -629,6 +636,13 @@ static int plan_create_impl(cconv_plan** plan_out, int B, int C, int K, int W, i
                    pl->kp_tail.h0, pl->tail.bb, pl->tail.bw, pl->tail.bh, pl->tail.bc,
                    pl->tail.i_stages, pl->tail.tiles, pl->tail.grid, pl->tail.smem_bytes);
   }
+  if (want_wait_twin && pl->variant == CCONV_VARIANT_DIRECT) {
+    // (a plan without it still works: waiting calls then run the direct kernel)
+    cconv_plan* twin = nullptr;
+    if (plan_create_impl(&twin, B, C, K, W, H, R, S, sw, sh, device, M_words, CCONV_VARIANT_HALO,
+                         out_dtype, image_strides) == CCONV_OK)
+      pl->wait_twin = twin;
+  }
   *plan_out = pl;
   return CCONV_OK;
 }
@@ -654,6 +668,7 @@ int cconv_plan_info_get(const cconv_plan* pl, cconv_plan_info* o) {
   o->lp_G = pl->lp_G;
   o->lp_words = pl->lp_words;
   o->variant = pl->variant;
+  o->wait_variant = pl->wait_twin ? pl->wait_twin->variant : pl->variant;
   o->out_dtype = pl->out_dtype;
   const Dims& d = pl->d;
   o->tail_h0 = pl->view.dk.H;
@@ -679,7 +694,7 @@ int cconv_plan_info_get(const cconv_plan* pl, cconv_plan_info* o) {
     o->stages = t.i_stages; o->filter_stages = t.f_stages; o->grid = t.grid; o->tiles = int(t.tiles);
     o->smem_bytes = t.smem_bytes; o->tmem_cols = t.tmem_cols;
     o->tile_words_smem = t.words_smem;
-    o->scratch_bytes = 0.0;
+    o->scratch_bytes = pl->wait_twin ? double(pl->wait_twin->tile.packed_filter_bytes) : 0.0;
     o->filter_taps = t.tg;
     o->est_cta_cycles = t.cta_cycles;
     o->est_period_cycles = t.est_cycles;
@@ -746,6 +761,7 @@ void cconv_plan_destroy(cconv_plan* pl) {
     cudaSetDevice(prev);
   }
   if (pl->acc_twin) cconv_plan_destroy(pl->acc_twin);
+  if (pl->wait_twin) cconv_plan_destroy(pl->wait_twin);
   delete pl;
 }
 
@@ -816,7 +832,14 @@ int cconv_forward_planned(const cconv_plan* pl, const void* Image, const void* F
     spans.sms = double(pl->dtile.grid) /
                 std::max(1, std::min(pl->m.smem_optin_bytes / std::max(pl->dtile.smem_bytes, 1),
                                      pl->m.tmem_cols / std::max(pl->dtile.tmem_cols, 1)));
-    const bool hazard = note_call(cuda_stream, spans, Overlap::kDeep, pl->m.sm_count);
+    const int hazards = note_call_hazards(cuda_stream, spans, Overlap::kDeep, pl->m.sm_count);
+    const bool hazard = hazards != 0;
+    if (hazard && pl->wait_twin) {
+      // The call starts only when the stream's earlier work is complete, so it cannot run beside
+      // other calls: the halo kernel's tiling gives it the whole GPU.  That kernel writes Out only
+      // after every earlier kernel is complete; its inputs wait when they are what conflicts.
+      return launch_tensor_core(pl->wait_twin, Image, Filter, Out, (hazards & kHazardInputs) != 0, stream);
+    }
     CUtensorMap tmi, tmf;
     {
       std::lock_guard<std::mutex> lk(pl->mu);
@@ -1081,9 +1104,11 @@ int cconv_plan_status(const cconv_plan* pl, void* cuda_stream, int* detail_out) 
     CCONV_CUDA(cudaMemsetAsync(pl->d_status, 0, sizeof(int), stream));
     CCONV_CUDA(cudaStreamSynchronize(stream));
   }
-  if (pl->acc_twin) {  // the accumulating calls run on the twin
+  // (accumulating calls and calls that had to wait run on twin plans with status words of their own)
+  for (const cconv_plan* twin : {pl->acc_twin, pl->wait_twin}) {
+    if (!twin) continue;
     int st2 = 0;
-    const int rc2 = cconv_plan_status(pl->acc_twin, cuda_stream, &st2);
+    const int rc2 = cconv_plan_status(twin, cuda_stream, &st2);
     if (rc2 != CCONV_OK && rc2 != CCONV_EDEVICE_TIMEOUT) return rc2;
     st |= st2;
   }

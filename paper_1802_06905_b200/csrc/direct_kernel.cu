@@ -147,6 +147,10 @@ __global__ void __launch_bounds__(kDirectThreads, 1)
     if (p.trace) p.trace[blockIdx.x * 16 + (slot)] = globaltimer_ns();   \
   } while (0)
 
+  // Set-up is spread over three threads, and each producer issues its first stages as soon as its
+  // own barriers exist, before the CTA-wide barrier: the first operands are then on their way while
+  // tensor memory is allocated and the other roles get ready.
+  uint32_t pre_issued = 0;  // stages this thread's ring received before the CTA-wide barrier
   if (threadIdx.x == 0) {
     // The next kernel of the stream may start now: it takes SMs that this grid does not use.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -155,10 +159,53 @@ __global__ void __launch_bounds__(kDirectThreads, 1)
       mbar_init(bar_ifull + 8u * s, 1);
       mbar_init(bar_iempty + 8u * s, 1);
     }
+    fence_barrier_init();
+    if (p.wait_prev) asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (int(blockIdx.x) < p.total_tiles) {
+      int t = int(blockIdx.x) / p.tiles_k;
+      const int bt = t % p.tiles_b; t /= p.tiles_b;
+      const int wt = t % p.tiles_w; t /= p.tiles_w;
+      const int n_pre = p.i_stages < p.cchunks ? p.i_stages : p.cchunks;
+      for (int cc = 0; cc < n_pre; ++cc) {
+        const uint32_t full = bar_ifull + 8u * cc;
+        if (p.diag_mode == 2) {
+          mbar_arrive(full);  // diagnostics: no copies, the MMAs run on whatever the ring holds
+        } else {
+          mbar_arrive_expect_tx(full, p.img_stage_bytes);
+          tma_load_4d(img_ring + cc * p.img_stage_bytes, &tm_image, bt * p.bb, cc * p.bc,
+                      wt * p.bw * p.sw, t * p.bh * p.sh, full);
+        }
+        if (cc == 0) CCONV_TRACE(2);
+      }
+      pre_issued = uint32_t(n_pre);
+    }
+  } else if (threadIdx.x == kFilterWarp * 32) {
     for (int s = 0; s < p.f_stages; ++s) {
       mbar_init(bar_ffull + 8u * s, 1);
       mbar_init(bar_fempty + 8u * s, 1);
     }
+    fence_barrier_init();
+    if (p.wait_prev) asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (int(blockIdx.x) < p.total_tiles) {
+      const int k0 = (int(blockIdx.x) % p.tiles_k) * 128 * KT;
+      const int all = p.cchunks * p.fgroups;
+      const int n_pre = p.f_stages < all ? p.f_stages : all;
+      for (int q = 0, cc = 0, fg = 0; q < n_pre; ++q) {
+        const uint32_t full = bar_ffull + 8u * q;
+        if (p.diag_mode == 2) {
+          mbar_arrive(full);
+        } else if (q != p.skip_filter_stage) {
+          mbar_arrive_expect_tx(full, p.filt_stage_bytes);
+          tma_load_3d(filt_ring + q * p.filt_stage_bytes, &tm_filter, cc * p.bc, k0, fg * p.tg, full);
+        }
+        if (++fg == p.fgroups) {
+          fg = 0;
+          ++cc;
+        }
+      }
+      pre_issued = uint32_t(n_pre);
+    }
+  } else if (threadIdx.x == 64) {
     for (int a = 0; a < 2; ++a) {
       mbar_init(bar_tfull + 8u * a, 1);
       mbar_init(bar_tempty + 8u * a, kEpiWarps);  // one arrival per epilogue warp
@@ -166,8 +213,6 @@ __global__ void __launch_bounds__(kDirectThreads, 1)
     mbar_init(bar_drain, 1);
     *abort_flag = 0;
     fence_barrier_init();
-    prefetch_tensormap(&tm_image);
-    prefetch_tensormap(&tm_filter);
   }
   if (warp == 1) {
     tmem_alloc(slot_addr, uint32_t(p.tmem_cols));
@@ -189,7 +234,6 @@ __global__ void __launch_bounds__(kDirectThreads, 1)
       const uint32_t n_st = uint32_t(p.i_stages);
       uint32_t seq = 0, s = 0, ph = 0;
       bool ok = true;
-      if (p.wait_prev) asm volatile("griddepcontrol.wait;" ::: "memory");
       auto coords = [&](int tile, int& b0, int& x0, int& y0) {
         int t = tile / p.tiles_k;
         const int bt = t % p.tiles_b; t /= p.tiles_b;
@@ -202,18 +246,19 @@ __global__ void __launch_bounds__(kDirectThreads, 1)
         int b0, x0, y0;
         coords(tile, b0, x0, y0);
         for (int cc = 0, c0 = 0; cc < p.cchunks; ++cc, c0 += p.bc, ++seq) {
-          if (!mbar_wait(bar_iempty + 8u * s, ph ^ 1u, abort_flag, status, kStatProducerWait, limit)) {
-            ok = false;
-            break;
+          if (seq >= pre_issued) {  // (the first stages went out before the CTA-wide barrier)
+            if (!mbar_wait(bar_iempty + 8u * s, ph ^ 1u, abort_flag, status, kStatProducerWait, limit)) {
+              ok = false;
+              break;
+            }
+            const uint32_t full = bar_ifull + 8u * s;
+            if (p.diag_mode == 2) {
+              mbar_arrive(full);
+            } else {
+              mbar_arrive_expect_tx(full, p.img_stage_bytes);
+              tma_load_4d(img_ring + s * p.img_stage_bytes, &tm_image, b0, c0, x0, y0, full);
+            }
           }
-          const uint32_t full = bar_ifull + 8u * s;
-          if (p.diag_mode == 2) {
-            mbar_arrive(full);  // diagnostics: no copies, the MMAs run on whatever the ring holds
-          } else {
-            mbar_arrive_expect_tx(full, p.img_stage_bytes);
-            tma_load_4d(img_ring + s * p.img_stage_bytes, &tm_image, b0, c0, x0, y0, full);
-          }
-          if (seq == 0) CCONV_TRACE(2);
           if (++s == n_st) {
             s = 0;
             ph ^= 1u;
@@ -229,21 +274,22 @@ __global__ void __launch_bounds__(kDirectThreads, 1)
       const uint32_t n_st = uint32_t(p.f_stages);
       uint32_t seq = 0, s = 0, ph = 0;
       bool ok = true;
-      if (p.wait_prev) asm volatile("griddepcontrol.wait;" ::: "memory");
       for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
         const int k0 = (tile % p.tiles_k) * 128 * KT;
         for (int cc = 0, c0 = 0; ok && cc < p.cchunks; ++cc, c0 += p.bc) {
           for (int fg = 0, t0 = 0; fg < p.fgroups; ++fg, t0 += p.tg, ++seq) {
-            if (!mbar_wait(bar_fempty + 8u * s, ph ^ 1u, abort_flag, status, kStatFilterWait, limit)) {
-              ok = false;
-              break;
-            }
-            const uint32_t full = bar_ffull + 8u * s;
-            if (p.diag_mode == 2) {
-              mbar_arrive(full);
-            } else if (int(seq) != p.skip_filter_stage) {
-              mbar_arrive_expect_tx(full, p.filt_stage_bytes);
-              tma_load_3d(filt_ring + s * p.filt_stage_bytes, &tm_filter, c0, k0, t0, full);
+            if (seq >= pre_issued) {
+              if (!mbar_wait(bar_fempty + 8u * s, ph ^ 1u, abort_flag, status, kStatFilterWait, limit)) {
+                ok = false;
+                break;
+              }
+              const uint32_t full = bar_ffull + 8u * s;
+              if (p.diag_mode == 2) {
+                mbar_arrive(full);
+              } else if (int(seq) != p.skip_filter_stage) {
+                mbar_arrive_expect_tx(full, p.filt_stage_bytes);
+                tma_load_3d(filt_ring + s * p.filt_stage_bytes, &tm_filter, c0, k0, t0, full);
+              }
             }
             if (++s == n_st) {
               s = 0;

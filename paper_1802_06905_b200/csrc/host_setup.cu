@@ -291,11 +291,15 @@ CallSpans spans_of(const Dims& d, int out_dtype, const void* Image, const void* 
 }
 
 bool note_call(void* stream, const CallSpans& c, Overlap how, int sm_count) {
+  return note_call_hazards(stream, c, how, sm_count) != 0;
+}
+
+int note_call_hazards(void* stream, const CallSpans& c, Overlap how, int sm_count) {
   std::lock_guard<std::mutex> lk(g_inflight_mu);
   StreamCalls& sc = g_inflight[stream];
   if (how == Overlap::kNone) {
     sc.n = 0;  // starts after, and is complete before, its neighbours
-    return false;
+    return 0;
   }
   // forget the calls that must be complete by the time this one starts: walking back from the
   // latest call, everything behind more than sm_count SMs' worth of resident CTAs
@@ -314,16 +318,18 @@ bool note_call(void* stream, const CallSpans& c, Overlap how, int sm_count) {
       sc.n = keep;
     }
   }
-  bool conflict = sc.n >= kMaxTracked;  // bound the list: a waiting call completes everything before it
-  for (int i = 0; i < sc.n && !conflict; ++i) {
+  // (a full list counts as both kinds: a waiting call completes everything before it)
+  int hazards = sc.n >= kMaxTracked ? (kHazardInputs | kHazardOut) : 0;
+  for (int i = 0; i < sc.n && hazards != (kHazardInputs | kHazardOut); ++i) {
     const CallSpans& e = sc.calls[i];
-    conflict = e.out.meets(c.image) || e.out.meets(c.filter);
-    if (how == Overlap::kDeep)
-      conflict = conflict || e.out.meets(c.out) || e.image.meets(c.out) || e.filter.meets(c.out);
+    if (e.out.meets(c.image) || e.out.meets(c.filter)) hazards |= kHazardInputs;
+    if (how == Overlap::kDeep &&
+        (e.out.meets(c.out) || e.image.meets(c.out) || e.filter.meets(c.out)))
+      hazards |= kHazardOut;
   }
-  if (conflict || how == Overlap::kInputsEarly) sc.n = 0;
+  if (hazards || how == Overlap::kInputsEarly) sc.n = 0;
   sc.calls[sc.n++] = c;
-  return conflict;
+  return hazards;
 }
 
 void note_ordinary_launch(void* stream) {

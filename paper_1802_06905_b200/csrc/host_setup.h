@@ -67,6 +67,10 @@ enum class Overlap {
 // resident until the call in front of it is complete, so a call can still be running only while
 // the CTAs of all calls launched after it (but the newest) fit the `sm_count` SMs together.
 bool note_call(void* stream, const CallSpans& c, Overlap how, int sm_count);
+// The same, telling the two kinds of conflict apart: kHazardInputs = this call's Image or Filter
+// meets the Out of a call that may still be running; kHazardOut = its Out meets one of their arrays.
+constexpr int kHazardInputs = 1, kHazardOut = 2;
+int note_call_hazards(void* stream, const CallSpans& c, Overlap how, int sm_count);
 // An ordinary launch of this library (pooling, the accumulate pass, ...) went into the stream.
 void note_ordinary_launch(void* stream);
 

@@ -288,3 +288,46 @@ def test_cconv_forward_on_two_streams_with_one_shape():
         exp, ab = ocnn.cnn_bf16(ins[j][0], ins[j][1], oshape(c))
         for i in (0, 3, 7):
             assert_close(outs[j][i].cpu().numpy().astype(np.float64), exp, ab, what=f"stream {j} call {i}")
+
+
+def test_a_call_that_has_to_wait_runs_the_halo_tiling_and_stays_in_order():
+    """AUTO plans that take the direct kernel keep a halo-kernel plan for calls that conflict with a
+    call still in flight (they cannot run beside it, and one call alone finishes sooner on many small
+    tiles).  A chain B(A(x)) with a third call that rewrites A's Out while B reads it, repeated
+    without synchronisation, must match the oracle whichever kernel each call ran."""
+    a = cs("wait_a", 64, 96, 128, 24, 28, 3, 3)                   # Out (128, 28, 24, 64) bf16
+    b = cs("wait_b", 64, 24, 64, 126, 26, 3, 3)                   # Image (128, 28, 24, 64)
+    assert a.out_shape == b.image_shape
+    ia, fa = synth.make_inputs(a)
+    _, fb = synth.make_inputs(b)
+    fa2 = synth.make_inputs(cs("wait_a2", *a.dims(), seed=991))[1]
+    img_a, flt_a, flt_a2, flt_b = to_dev(ia), to_dev(fa), to_dev(fa2), to_dev(fb)
+    plan_a = binding.Plan(*a.dims(), device=0, out_dtype=binding.OUT_BF16)
+    plan_b = binding.Plan(*b.dims(), device=0, out_dtype=binding.OUT_F32)
+    infos = [plan_a.info(), plan_b.info()]
+    assert any(i["variant"] == binding.VARIANT_DIRECT for i in infos)
+    for i in infos:
+        assert i["wait_variant"] == (binding.VARIANT_HALO if i["variant"] == binding.VARIANT_DIRECT
+                                     else i["variant"])
+    mid = torch.zeros(a.out_shape, dtype=torch.bfloat16, device="cuda")
+    out_b = torch.empty(b.out_shape, dtype=torch.float32, device="cuda")
+    exp_mid, _ = ocnn.cnn_bf16(ia, fa, oshape(a))
+    for rep in range(6):
+        mid.zero_()
+        out_b.fill_(float("nan"))
+        plan_a.forward(img_a, flt_a, mid)                         # independent of what is in flight
+        plan_b.forward(mid, flt_b, out_b)                         # read after write: waits
+        keep = mid.clone() if rep == 0 else None
+        plan_a.forward(img_a, flt_a2, mid)                        # write after read: waits
+        plan_a.forward(img_a, flt_a, mid)                         # write after write: waits
+        plan_a.check()
+        plan_b.check()
+        exp, ab = ocnn.cnn_bf16(to_bits(mid), fb, oshape(b))
+        assert_close(out_b.cpu().numpy().astype(np.float64), exp, ab, what=f"chain, repeat {rep}")
+        got_mid = ocnn.bf16_bits_to_f64(to_bits(mid))
+        _, ab_mid = ocnn.cnn_bf16(ia, fa, oshape(a))
+        assert_close(got_mid, exp_mid, ab_mid, what=f"rewritten Out, repeat {rep}", bf16_out=True)
+        if keep is not None:                                      # (written by the call that did not wait)
+            assert_close(ocnn.bf16_bits_to_f64(to_bits(keep)), exp_mid, ab_mid, what="first Out", bf16_out=True)
+    plan_a.close()
+    plan_b.close()
