@@ -540,10 +540,10 @@ __global__ void __launch_bounds__(kDirectThreads, 1)
           const uint32_t col0 = uint32_t((kt * p.bh + hh) * p.n_mma);
           for (int c = part * kPiece; c + kPiece <= p.n_mma; c += kParts * kPiece) {
             uint32_t va[32], sec[4][8];
-            tmem_ld_32x32b_x32(t_base + col0 + uint32_t(c), va);
+            if (p.diag_mode != 4) tmem_ld_32x32b_x32(t_base + col0 + uint32_t(c), va);
             if constexpr (sizeof(OutT) == 2) {
               uint32_t vb[32];
-              tmem_ld_32x32b_x32(t_base + col0 + uint32_t(c + 32), vb);
+              if (p.diag_mode != 4) tmem_ld_32x32b_x32(t_base + col0 + uint32_t(c + 32), vb);
               tmem_ld_wait();
 #pragma unroll
               for (int i = 0; i < 8; ++i) {
@@ -588,7 +588,7 @@ __global__ void __launch_bounds__(kDirectThreads, 1)
               row0 = lane & ~3;
               row_step = 1;
             }
-            if (wt * p.bw + ww < p.W && left > 0) {
+            if (wt * p.bw + ww < p.W && left > 0 && p.diag_mode != 3) {
               OutT* const d0 = roww + (long long)row0 * plane + (long long)ww * p.B + b;
 #pragma unroll
               for (int j = 0; j < 4; ++j) {

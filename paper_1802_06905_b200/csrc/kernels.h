@@ -117,7 +117,8 @@ struct DirectKernelParams {
   uint64_t a_desc, b_desc;       // shared-memory descriptors with a zero start address
   uint64_t wait_limit_ns;
   int diag_mode;                 // diagnostics (results are meaningless): 1 = stage operands but
-                                 // issue no MMA, 2 = issue the MMAs but copy nothing
+                                 // issue no MMA, 2 = issue the MMAs but copy nothing, 3 = the
+                                 // epilogue stores nothing, 4 = the epilogue loads no accumulators
   int skip_filter_stage;         // diagnostics: the Filter producer leaves out the stage with this
                                  // sequence number (-1 = none), so that a bounded wait runs out
   unsigned long long* trace;     // optional [grid][16] time stamps, or null

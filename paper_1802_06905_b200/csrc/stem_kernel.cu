@@ -151,7 +151,10 @@ __global__ void __launch_bounds__(kStemThreads, 1)
   const int lane = threadIdx.x & 31;
   // diagnostics: per-CTA row of 16 counters (0 entry ns, 1 exit ns, 2.. cycles spent per role)
   unsigned long long* const tr = p.trace ? p.trace + 16ull * blockIdx.x : nullptr;
-  if (tr && threadIdx.x == 0) tr[0] = globaltimer_ns();
+  if (tr && threadIdx.x == 0) {
+    tr[0] = globaltimer_ns();
+    tr[11] = (unsigned long long)clock64();
+  }
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.i_stages; ++s) {
@@ -465,7 +468,10 @@ __global__ void __launch_bounds__(kStemThreads, 1)
   }
   // This kernel ran beside the kernels in front of it; it ends only after they have.
   if (threadIdx.x == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
-  if (tr && threadIdx.x == 0) tr[1] = globaltimer_ns();
+  if (tr && threadIdx.x == 0) {
+    tr[1] = globaltimer_ns();
+    tr[12] = (unsigned long long)clock64();
+  }
 }
 
 // (The attribute is a per-kernel ceiling and the value set last wins: it is raised to the device's
