@@ -252,6 +252,9 @@ struct cconv_plan {
   static constexpr int kMapSlots = 64;
   mutable MapSlot img_maps[kMapSlots];
   mutable MapSlot flt_maps[kMapSlots];
+  mutable MapSlot out_maps[kMapSlots];
+  bool direct_tma_store = false;  // single-tile CTAs store Out through the TMA engine
+  int direct_tma_mode = 1;        // DirectKernelParams::out_tma of such calls
   static int map_slot(const void* p) {
     return int((reinterpret_cast<uintptr_t>(p) >> 8) * 0x9E3779B97F4A7C15ull >> 58);
   }
@@ -563,6 +566,14 @@ static int plan_create_impl(cconv_plan** plan_out, int B, int C, int K, int W, i
   if (variant == CCONV_VARIANT_DIRECT) {
     build_direct_params(dk, pl->dtile, &pl->dkp);
     pl->diag_skip_once = env_int("CCONV_DIAG_SKIP_FILTER_STAGE", -1);
+    // (the staging buffers of the TMA-store epilogue live in the rings of a CTA with a single tile)
+    pl->direct_tma_store = pl->dtile.tiles <= pl->dtile.grid && env_int("CCONV_DIRECT_TMA_STORE", 1) != 0;
+    if (pl->direct_tma_store) {  // is a piece 128 contiguous bytes of Out?  (same rule as the encoder's)
+      const bool f32 = out_dtype == CCONV_OUT_F32;
+      const bool merged = !f32 && pl->dtile.bb == 32 && dk.B == 32;
+      pl->direct_tma_mode = merged ? 2 : 1;
+      if (!merged && pl->dtile.bb * (f32 ? 4 : 2) < 128) pl->direct_tma_store = false;
+    }
   }
 
   if (device >= 0) {
@@ -840,7 +851,7 @@ int cconv_forward_planned(const cconv_plan* pl, const void* Image, const void* F
       // after every earlier kernel is complete; its inputs wait when they are what conflicts.
       return launch_tensor_core(pl->wait_twin, Image, Filter, Out, (hazards & kHazardInputs) != 0, stream);
     }
-    CUtensorMap tmi, tmf;
+    CUtensorMap tmi, tmf, tmo{};
     {
       std::lock_guard<std::mutex> lk(pl->mu);
       cconv_plan::MapSlot& si = pl->img_maps[cconv_plan::map_slot(Image)];
@@ -857,6 +868,17 @@ int cconv_forward_planned(const cconv_plan* pl, const void* Image, const void* F
       }
       tmi = si.tm;
       tmf = sf.tm;
+      if (pl->direct_tma_store) {
+        cconv_plan::MapSlot& so = pl->out_maps[cconv_plan::map_slot(Out)];
+        if (so.ptr != Out) {
+          int merged = 0;
+          const int rc = encode_direct_out_map(pl->view.dk, pl->dtile, pl->out_dtype == CCONV_OUT_F32, Out,
+                                               &so.tm, &merged);
+          if (rc != CCONV_OK) return rc;
+          so.ptr = Out;
+        }
+        tmo = so.tm;
+      }
     }
     DirectKernelParams kp = pl->dkp;
     {
@@ -865,7 +887,8 @@ int cconv_forward_planned(const cconv_plan* pl, const void* Image, const void* F
       pl->diag_skip_once = -1;
     }
     kp.wait_prev = hazard ? 1 : 0;
-    cudaError_t e = launch_direct(tmi, tmf, Out, pl->out_dtype == CCONV_OUT_F32, kp, pl->dtile.grid,
+    kp.out_tma = pl->direct_tma_store ? pl->direct_tma_mode : 0;
+    cudaError_t e = launch_direct(tmi, tmf, tmo, Out, pl->out_dtype == CCONV_OUT_F32, kp, pl->dtile.grid,
                                   pl->dtile.smem_bytes, pl->d_status, stream);
     return e == cudaSuccess ? CCONV_OK : cuda_fail(e, "launch_direct");
   }

@@ -121,7 +121,8 @@ __device__ __forceinline__ void direct_store32(OutT* dst, const uint32_t (&v)[32
 template <typename OutT, int BH, int KT, int NC16>
 __global__ void __launch_bounds__(kDirectThreads, 1)
     cconv_direct_kernel(const __grid_constant__ CUtensorMap tm_image,
-                        const __grid_constant__ CUtensorMap tm_filter, OutT* __restrict__ out,
+                        const __grid_constant__ CUtensorMap tm_filter,
+                        const __grid_constant__ CUtensorMap tm_out, OutT* __restrict__ out,
                         const DirectKernelParams p, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;  // swizzle atoms need 1024 B
@@ -525,9 +526,17 @@ __global__ void __launch_bounds__(kDirectThreads, 1)
       const long long plane = (long long)p.H * p.W * p.B;   // elements of one out-channel plane
       const int bb_shift = p.bb == 64 ? 6 : 5;
       const int sj = lane & 3;
-      const uint32_t stage = smem0 + uint32_t(warp - 2) * 4608u;  // 32 rows of 144 bytes per warp
-      const bool via_smem = p.total_tiles <= int(gridDim.x) &&
-                            uint32_t(kEpiWarps) * 4608u <= bars - smem0;
+      // A CTA with a single tile: the rings are idle by now and serve as staging memory, 8 KB per
+      // epilogue warp.
+      const bool idle_rings = p.total_tiles <= int(gridDim.x) && uint32_t(kEpiWarps) * 8192u <= bars - smem0;
+      const uint32_t stage = smem0 + uint32_t(warp - 2) * 8192u;
+      // With a tensor map of Out, every piece is stored by the TMA engine from a swizzled 4 KB
+      // buffer (two per warp, so a warp converts its next piece while the last one drains); the
+      // engine clips what lies outside Out.  Else the quad's sectors are exchanged -- through the
+      // staging memory if there is some, by shuffles otherwise -- and stored by the lanes.
+      const bool via_tma = idle_rings && p.out_tma != 0 && p.diag_mode != 3;
+      const bool via_smem = idle_rings;
+      uint32_t n_stored = 0;  // pieces this warp handed to the TMA engine
 #pragma unroll
       for (int kt = 0; kt < KT; ++kt) {
         const int kw = (ktile * KT + kt) * 128 + q * 32;  // first out-channel of this warp's 32 rows
@@ -557,16 +566,43 @@ __global__ void __launch_bounds__(kDirectThreads, 1)
 #pragma unroll
               for (int i = 0; i < 32; ++i) sec[i >> 3][i & 7] = va[i];
             }
+            if (via_tma) {
+              const uint32_t buf = stage + (n_stored & 1u) * 4096u;
+              if (n_stored >= 2) {  // the store that read this buffer two pieces ago
+                if (lane == 0) bulk_wait_group_read<1>();
+                __syncwarp();
+              }
+              // lane = row of the box; its eight 16-byte chunks land XOR-swizzled by the row (the
+              // 128-byte swizzle of the tensor map), which also keeps the stores free of conflicts
+              const uint32_t rowa = buf + uint32_t(lane) * 128u;
+              const uint32_t x = uint32_t(lane & 7);
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                st_shared_v4(rowa + (((2u * i) ^ x) << 4), sec[i][0], sec[i][1], sec[i][2], sec[i][3]);
+                st_shared_v4(rowa + (((2u * i + 1u) ^ x) << 4), sec[i][4], sec[i][5], sec[i][6], sec[i][7]);
+              }
+              fence_proxy_async_smem();
+              __syncwarp();
+              if (lane == 0) {
+                const int ww0 = c >> bb_shift, bb0 = c - (ww0 << bb_shift);
+                const int w = wt * p.bw + ww0;
+                if (p.out_tma == 2) tma_store_4d(&tm_out, buf, w * p.B + b0 + bb0, 0, h, kw);
+                else tma_store_4d(&tm_out, buf, b0 + bb0, w, h, kw);
+                bulk_commit_group();
+              }
+              ++n_stored;
+              continue;
+            }
             // the sector this lane stores: columns cc .. cc + kSec of the run = images b .. of pixel ww
             const int cc = c + kSec * sj;
             const int ww = cc >> bb_shift, b = cc - (ww << bb_shift);
             const int left = p.B - (b0 + b);   // images of the sector inside the batch (a multiple of 8)
             int row0, row_step;                 // this lane stores rows row0 + j*row_step of the warp's 32
             if (via_smem) {
-              // A CTA with a single tile: the rings are idle by now, so the 4x4 exchange of sectors
-              // goes through shared memory (16 vector accesses instead of 64 shuffles and as many
-              // selects): every lane parks its 128-byte piece in a row of 144 bytes (the pitch keeps
-              // both phases free of bank conflicts), then reads sector sj of rows 8j + lane/4.
+              // The 4x4 exchange of sectors through shared memory (16 vector accesses instead of
+              // 64 shuffles and as many selects): every lane parks its 128-byte piece in a row of
+              // 144 bytes (the pitch keeps both phases free of bank conflicts), then reads sector sj
+              // of rows 8j + lane/4.
               const uint32_t wrow = stage + uint32_t(lane) * 144u;
 #pragma unroll
               for (int i = 0; i < 4; ++i) {
@@ -624,6 +660,10 @@ __global__ void __launch_bounds__(kDirectThreads, 1)
           }
         }
       }
+      if (via_tma) {  // Out is complete before this CTA reports completion
+        if (lane == 0) bulk_wait_group<0>();
+        __syncwarp();
+      }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_tempty + 8u * abuf);
@@ -655,7 +695,7 @@ __global__ void __launch_bounds__(kDirectThreads, 1)
 namespace {
 
 template <typename OutT>
-using DirectFn = void (*)(CUtensorMap, CUtensorMap, OutT*, DirectKernelParams, int*);
+using DirectFn = void (*)(CUtensorMap, CUtensorMap, CUtensorMap, OutT*, DirectKernelParams, int*);
 
 template <typename OutT, int KT, int NC16>
 DirectFn<OutT> direct_fn_bh(int bh) {
@@ -706,8 +746,8 @@ cudaError_t direct_kernel_prepare() {
   return direct_prepare_all<float>(cap);
 }
 
-cudaError_t launch_direct(const CUtensorMap& tm_image, const CUtensorMap& tm_filter, void* out,
-                          bool out_f32, const DirectKernelParams& p, int grid, int smem_bytes,
+cudaError_t launch_direct(const CUtensorMap& tm_image, const CUtensorMap& tm_filter,
+                          const CUtensorMap& tm_out, void* out, bool out_f32, const DirectKernelParams& p, int grid, int smem_bytes,
                           int* status, cudaStream_t stream) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(unsigned(grid));
@@ -722,9 +762,9 @@ cudaError_t launch_direct(const CUtensorMap& tm_image, const CUtensorMap& tm_fil
   const int nc16 = p.bc / 16;
   if (out_f32)
     return cudaLaunchKernelEx(&cfg, direct_fn<float>(p.kt, nc16, p.mma_rows), tm_image, tm_filter,
-                              static_cast<float*>(out), p, status);
+                              tm_out, static_cast<float*>(out), p, status);
   return cudaLaunchKernelEx(&cfg, direct_fn<__nv_bfloat16>(p.kt, nc16, p.mma_rows), tm_image, tm_filter,
-                            static_cast<__nv_bfloat16*>(out), p, status);
+                            tm_out, static_cast<__nv_bfloat16*>(out), p, status);
 }
 
 }  // namespace cconv

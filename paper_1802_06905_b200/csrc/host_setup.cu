@@ -179,6 +179,7 @@ void build_direct_params(const Dims& d, const DirectTile& t, DirectKernelParams*
   p.b_desc = make_smem_desc(uint32_t(d.sw) * p.slab_bytes, 8 * b_row, b_layout);
   p.wait_limit_ns = uint64_t(env_int("CCONV_WAIT_LIMIT_MS", 1000)) * 1000000ull;
   p.diag_mode = env_int("CCONV_DIAG_MODE", 0);
+  p.out_tma = 0;  // set per call when the Out tensor map could be built
   p.skip_filter_stage = -1;
   p.trace = nullptr;
 }
@@ -209,6 +210,37 @@ int encode_direct_filter_map(const Dims& d, const DirectTile& t, const void* fil
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
     set_last_cuda_error("cuTensorMapEncodeTiled(Filter) failed with CUresult " + std::to_string(int(r)));
+    return CCONV_ECUDA;
+  }
+  return CCONV_OK;
+}
+
+int encode_direct_out_map(const Dims& d, const DirectTile& t, bool out_f32, void* out, CUtensorMap* tm,
+                          int* merged_wb) {
+  EncodeTiledFn enc = encode_tiled_fn();
+  if (!enc) {
+    set_last_cuda_error("cuTensorMapEncodeTiled is not available from this driver");
+    return CCONV_ECUDA;
+  }
+  // A piece is 128 bytes of one accumulator row (64 bf16 / 32 fp32 columns, images fastest) and
+  // must be 128 contiguous bytes of Out, so that the box's inner extent is the swizzle span:
+  // one pixel's 64 images (bf16) or half of them (fp32), a 32-image block in fp32, or -- bf16 with
+  // b_b = B = 32 -- two neighbouring pixels, addressed through the merged subscript w*B + b.
+  const cuuint64_t es = out_f32 ? 4 : 2;
+  const bool merged = !out_f32 && t.bb == 32 && d.B == 32;
+  if (!merged && uint64_t(t.bb) * es < 128) return CCONV_EUNSUPPORTED;
+  *merged_wb = merged ? 1 : 0;
+  const cuuint64_t row = cuuint64_t(d.W) * d.B * es;
+  const cuuint64_t dims[4] = {merged ? cuuint64_t(d.W) * d.B : cuuint64_t(d.B),
+                              merged ? cuuint64_t(1) : cuuint64_t(d.W), cuuint64_t(d.H), cuuint64_t(d.K)};
+  const cuuint64_t strides[3] = {merged ? row : cuuint64_t(d.B) * es, row, cuuint64_t(d.H) * row};
+  const cuuint32_t box[4] = {cuuint32_t(128 / es), 1, 1, 32};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult r = enc(tm, out_f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4,
+                   out, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    set_last_cuda_error("cuTensorMapEncodeTiled(Out) failed with CUresult " + std::to_string(int(r)));
     return CCONV_ECUDA;
   }
   return CCONV_OK;

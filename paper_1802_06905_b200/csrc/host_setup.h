@@ -26,6 +26,12 @@ int encode_image_map(const ImageView& v, const HaloTile& t, const void* image, C
 void build_direct_params(const Dims& d, const DirectTile& t, DirectKernelParams* p);
 int encode_direct_image_map(const ImageView& v, const DirectTile& t, const void* image, CUtensorMap* tm);
 int encode_direct_filter_map(const Dims& d, const DirectTile& t, const void* filter, CUtensorMap* tm);
+// Out [K][H][W][B] as a 4-D tensor (b, w, h, k) whose box is one epilogue warp's piece: 32 out-channel
+// rows of 128 contiguous bytes, 128-byte swizzle; *merged_wb = 1 when the first coordinate is the
+// merged subscript w*B + b and the second is unused.  CCONV_EUNSUPPORTED where a piece is not
+// contiguous in Out (bf16, b_b = 32 < B).
+int encode_direct_out_map(const Dims& d, const DirectTile& t, bool out_f32, void* out, CUtensorMap* tm,
+                          int* merged_wb);
 
 // The same two pieces for the small-C ("stem") kernel: Image viewed as (b, m = y*C + c, x).
 void build_stem_params(const Dims& d, const StemTile& t, StemKernelParams* p);

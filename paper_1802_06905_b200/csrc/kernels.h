@@ -116,6 +116,9 @@ struct DirectKernelParams {
   uint32_t idesc;
   uint64_t a_desc, b_desc;       // shared-memory descriptors with a zero start address
   uint64_t wait_limit_ns;
+  int out_tma;                   // 1: the Out tensor map is valid and CTAs with a single tile store
+                                 // their 128-byte row pieces with TMA tensor stores from shared memory;
+                                 // 2: the same, and the map's first coordinate is w*B + b
   int diag_mode;                 // diagnostics (results are meaningless): 1 = stage operands but
                                  // issue no MMA, 2 = issue the MMAs but copy nothing, 3 = the
                                  // epilogue stores nothing, 4 = the epilogue loads no accumulators
@@ -125,7 +128,8 @@ struct DirectKernelParams {
 };
 
 cudaError_t direct_kernel_prepare();
-cudaError_t launch_direct(const CUtensorMap& tm_image, const CUtensorMap& tm_filter, void* out,
+cudaError_t launch_direct(const CUtensorMap& tm_image, const CUtensorMap& tm_filter,
+                          const CUtensorMap& tm_out, void* out,
                           bool out_f32, const DirectKernelParams& p, int grid, int smem_bytes,
                           int* status, cudaStream_t stream);
 
