@@ -474,6 +474,10 @@ def roofline_for(cfg, info, secs_per_launch, peaks, binding):
         peak = peaks["bf16_tflops"]
         return {"bound": "tensor", "achieved": ach, "peak": peak, "unit": "TFLOP/s",
                 "frac": ach / peak, "traffic": traffic, "peak_source": peaks["source"],
+                # the burst figure is the denominator; the timed loop of a large shape runs for
+                # hundreds of milliseconds under the power cap, so the sustained figure stands beside it
+                "peak_sustained": peaks["bf16_tflops_sustained"],
+                "frac_of_sustained_peak": ach / peaks["bf16_tflops_sustained"],
                 "kernel": KERNEL_NAMES[info["variant"]],
                 "duration": "CUDA-event time of `steps` back-to-back forward calls / steps, median of "
                             "`repeats` such regions (calls of small shapes overlap on the GPU)"}
