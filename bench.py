@@ -707,7 +707,13 @@ def main():
             roof["applicable"]["write_only_stream_gbs"] = wgbs
             per, rows = {}, []
             for c in CONFIGS:
-                n_i = 100 if c.flops < 1e11 else 20
+                # Regions of about 4 ms (20 to 1000 calls, sized from the roofline time): calls of the
+                # small shapes overlap on the GPU, and a short region would add the drain of its last
+                # call, (CTA life - period) / calls, to every call; much longer regions leave the burst
+                # regime in which the roofline's denominators were measured (after some 40 ms of
+                # continuous work cfg3 settles 17 % lower, as cfg5 does under the power cap).
+                t_guess = 1.5 * applicable_roofline_seconds(c, binding.Plan(*c.dims(), device=-1).info(), peaks)[0]
+                n_i = int(min(1000, max(20, round(4e-3 / max(t_guess, 4e-6)))))
                 res, info_i = time_repeats(c, torch, binding, dev, n_i)
                 cold = res["stream"]
                 tr, lbb = applicable_roofline_seconds(c, info_i, peaks)
@@ -731,9 +737,10 @@ def main():
                     "G_over_lp_G": round(info_i["tile_G_over_lp_G"], 3) if tensor else None}
                 rows.append({"workload": c.name, "plan": info_i, "timing_s": res, "oracle": oracle_sample(c)})
             roof["per_config"] = per
-            roof["per_config_note"] = ("us = L2-cold back-to-back calls on one stream (independent calls "
-                                       "of small shapes run side by side on the SMs); us_alone = one "
-                                       "call between synchronisations, launch included; frac = t_roof_us / us")
+            roof["per_config_note"] = ("us = L2-cold back-to-back calls on one stream, median of 5 regions of "
+                                       "about 4 ms (20 to 1000 calls); independent calls of small shapes "
+                                       "run side by side on the SMs; us_alone = one call between "
+                                       "synchronisations, launch included; frac = t_roof_us / us")
             pool = time_pooling(torch, binding, dev, peaks)
             roof["pooling"] = {f"{r['workload']}_{r['op']}": {"us": round(r["us_per_launch"], 2),
                                                                "frac_of_hbm_copy": round(r["roofline"]["frac"], 3)}

@@ -156,6 +156,11 @@ __global__ void __launch_bounds__(kDirectThreads, 1)
     // The next kernel of the stream may start now: it takes SMs that this grid does not use.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     CCONV_TRACE(0);
+    if (p.trace) {
+      uint32_t smid;
+      asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+      p.trace[blockIdx.x * 16 + 12] = smid;
+    }
     for (int s = 0; s < p.i_stages; ++s) {
       mbar_init(bar_ifull + 8u * s, 1);
       mbar_init(bar_iempty + 8u * s, 1);
