@@ -331,3 +331,38 @@ def test_a_call_that_has_to_wait_runs_the_halo_tiling_and_stays_in_order():
             assert_close(ocnn.bf16_bits_to_f64(to_bits(keep)), exp_mid, ab_mid, what="first Out", bf16_out=True)
     plan_a.close()
     plan_b.close()
+
+
+def test_direct_calls_inside_a_cuda_graph():
+    """An AUTO plan that took the direct kernel, captured: three calls on two Out buffers (the third
+    has to wait for the first: it runs the plan's halo-kernel tiling), replayed on new contents of the
+    same buffers."""
+    c = cs("graph_direct", 32, 128, 128, 14, 12, 3, 3)
+    ib, fb = synth.make_inputs(c)
+    img, flt = to_dev(ib), to_dev(fb)
+    outs = [torch.full(c.out_shape, float("nan"), device="cuda", dtype=torch.bfloat16) for _ in range(2)]
+    plan = binding.Plan(*c.dims(), device=0, out_dtype=binding.OUT_BF16)
+    assert plan.info()["variant"] == binding.VARIANT_DIRECT
+    plan.forward(img, flt, outs[0])           # warm-up outside the capture
+    plan.check()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.graph(graph, stream=side):
+        plan.forward(img, flt, outs[0])
+        plan.forward(img, flt, outs[1])
+        plan.forward(img, flt, outs[0])
+    for seed in (91, 92):
+        ib2, fb2 = synth.make_inputs(ConvShape("graph_direct", *c.dims(), seed=seed))
+        img.copy_(to_dev(ib2))
+        flt.copy_(to_dev(fb2))
+        for o in outs:
+            o.fill_(float("nan"))
+        graph.replay()
+        torch.cuda.synchronize()
+        exp, ab = ocnn.cnn_bf16(ib2, fb2, oshape(c))
+        for n, o in enumerate(outs):
+            assert_close(ocnn.bf16_bits_to_f64(to_bits(o)), exp, ab, what=f"graph replay, seed {seed}, Out {n}",
+                         bf16_out=True)
+    plan.check()
+    plan.close()
