@@ -366,3 +366,48 @@ def test_direct_calls_inside_a_cuda_graph():
                          bf16_out=True)
     plan.check()
     plan.close()
+
+
+@pytest.mark.parametrize("seed", [1, 2])
+def test_random_dependent_sequences_match_their_synchronised_run(seed):
+    """Stream order as a property (parity with the oracle is the business of the tests above): 150
+    random calls -- convolution A writing one of three buffers, convolution B reading one of them as
+    its Image, pooling reading one of them -- issued without synchronisation must leave every buffer
+    bit-identical to the same sequence with a synchronisation after every call.  (Which kernel a call
+    runs depends only on the sequence of calls, so the two runs take the same decisions.)"""
+    import random
+    a = cs("seq_a", 64, 96, 128, 24, 28, 3, 3)                    # Out (128, 28, 24, 64) bf16
+    b = cs("seq_b", 64, 24, 64, 126, 26, 3, 3)                    # Image (128, 28, 24, 64)
+    pool_dims = (64, 24, 4, 63, 13, 4, 4, 2, 2)                   # Image (128, 28, 24, 64), Out (4, 13, 63, 64)
+    assert a.out_shape == b.image_shape
+    ia = [to_dev(synth.make_inputs(cs("seq_a", *a.dims()[:7], seed=10 + i))[0]) for i in range(2)]
+    fa = [to_dev(synth.make_inputs(cs("seq_a", *a.dims()[:7], seed=20 + i))[1]) for i in range(2)]
+    fb = [to_dev(synth.make_inputs(cs("seq_b", *b.dims()[:7], seed=30 + i))[1]) for i in range(2)]
+
+    def run(sync):
+        rng = random.Random(seed)
+        mid = [torch.zeros(a.out_shape, dtype=torch.bfloat16, device="cuda") for _ in range(3)]
+        outb = [torch.zeros(b.out_shape, dtype=torch.float32, device="cuda") for _ in range(3)]
+        pout = [torch.zeros((4, 13, 63, 64), dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+        pa = binding.Plan(*a.dims(), device=0, out_dtype=binding.OUT_BF16)
+        pb = binding.Plan(*b.dims(), device=0, out_dtype=binding.OUT_F32)
+        for _ in range(150):
+            r = rng.random()
+            if r < 0.45:
+                pa.forward(ia[rng.randrange(2)], fa[rng.randrange(2)], mid[rng.randrange(3)])
+            elif r < 0.8:
+                pb.forward(mid[rng.randrange(3)], fb[rng.randrange(2)], outb[rng.randrange(3)])
+            else:
+                binding.pool_forward(mid[rng.randrange(3)], pout[rng.randrange(2)], *pool_dims,
+                                     op=binding.POOL_MAX)
+            if sync:
+                torch.cuda.synchronize()
+        pa.check()
+        pb.check()
+        res = [t.clone() for t in mid + outb + pout]
+        pa.close()
+        pb.close()
+        return res
+
+    for n, (x, y) in enumerate(zip(run(False), run(True))):
+        assert torch.equal(x, y), f"buffer {n} differs between the two runs"
