@@ -336,6 +336,21 @@ int cconv_plan_status(const cconv_plan* plan, void* cuda_stream, int* detail_out
  * max_u64 values); returns the number of values copied, 0 when tracing is off, or a negative code. */
 int cconv_plan_trace_read(const cconv_plan* plan, unsigned long long* host_out, int max_u64);
 
+/* Diagnostics of the stream-order bookkeeping (host logic only: nothing is launched, no pointer is
+ * dereferenced).  Registers a call on `stream_key` exactly as a forward call on that stream would
+ * -- the byte ranges [lo, hi) of its Image, Filter and Out (a null lo: the call has no such array),
+ * how it overlaps its neighbours (0 = an ordinary launch, 1 = inputs may be read early and Out is
+ * written only after every earlier call is complete, 2 = reads and writes may overlap any number of
+ * earlier calls), and the SMs' worth of CTAs it keeps resident, counted by shared/tensor memory and
+ * by thread slots -- and returns the hazards found against the calls that may still be running:
+ * bit 0 = its Image or Filter meets an earlier Out, bit 1 = its Out meets an earlier array (checked
+ * for `overlap` 2 only); a list that is full reports both.  CCONV_EINVAL for an unknown `overlap`
+ * or sm_count <= 0.  A key that no real stream uses keeps the test apart from real calls. */
+int cconv_stream_order_probe(void* stream_key, const void* image_lo, const void* image_hi,
+                             const void* filter_lo, const void* filter_hi, const void* out_lo,
+                             const void* out_hi, int overlap, double sms_by_memory,
+                             double sms_by_threads, int sm_count);
+
 const char* cconv_strerror(int code);
 const char* cconv_last_cuda_error(void); /* message of the last failed CUDA call on this thread */
 int cconv_version(void);

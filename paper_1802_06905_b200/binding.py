@@ -28,7 +28,8 @@ EXPORTS = (
     "cconv_forward_host_async", "cconv_host_wait",
     "cconv_forward_noalloc", "cconv_noalloc_status", "cconv_pool_lower_bound", "cconv_pool_forward",
     "cconv_parallel_lower_bound", "cconv_parallel_partition", "cconv_theorem2_case",
-    "cconv_plan_status", "cconv_plan_trace_read", "cconv_strerror", "cconv_last_cuda_error", "cconv_version",
+    "cconv_plan_status", "cconv_plan_trace_read", "cconv_stream_order_probe", "cconv_strerror",
+    "cconv_last_cuda_error", "cconv_version",
 )
 
 
@@ -110,6 +111,8 @@ def load_library():
     lib.cconv_forward.restype = i
     lib.cconv_forward.argtypes = [vp, vp, vp] + nine + [i, vp]
     i64p = ctypes.POINTER(ctypes.c_int64)
+    lib.cconv_stream_order_probe.restype = i
+    lib.cconv_stream_order_probe.argtypes = [vp] * 7 + [i, d, d, i]
     lib.cconv_forward_strided.restype = i
     lib.cconv_forward_strided.argtypes = [vp, i64p, vp, i64p, vp, i64p] + nine + [i, vp]
     lib.cconv_forward_noalloc.restype = i
@@ -215,6 +218,21 @@ def pool_forward(image, out, B, C, K, W, H, R, S, sw=1, sh=1, op=0, stream=None)
     with torch.cuda.device(image.device):
         pool_forward_ptrs(image.data_ptr(), out.data_ptr(), B, C, K, W, H, R, S, sw, sh, op,
                           OUT_F32 if out.dtype == torch.float32 else OUT_BF16, sp)
+
+
+def stream_order_probe(stream_key, image, filt, out, overlap, sms_by_memory=0.0, sms_by_threads=0.0,
+                       sm_count=148):
+    """cconv_stream_order_probe: registers a call given as three (lo, hi) byte ranges (None = no such
+    array) with the stream-order bookkeeping of ``stream_key`` and returns the hazard bits."""
+    def rng(r):
+        return (None, None) if r is None else (ctypes.c_void_p(r[0]), ctypes.c_void_p(r[1]))
+    (il, ih), (fl, fh), (ol, oh) = rng(image), rng(filt), rng(out)
+    rc = load_library().cconv_stream_order_probe(ctypes.c_void_p(stream_key), il, ih, fl, fh, ol, oh,
+                                                 int(overlap), float(sms_by_memory), float(sms_by_threads),
+                                                 int(sm_count))
+    if rc < 0:
+        _check(rc, "cconv_stream_order_probe")
+    return rc
 
 
 def tiling_lp(B, C, K, W, H, R, S, sw, sh, M_words, pooling=False):

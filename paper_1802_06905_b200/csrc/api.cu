@@ -1117,6 +1117,21 @@ int cconv_plan_trace_read(const cconv_plan* pl, unsigned long long* host_out, in
   return n;
 }
 
+int cconv_stream_order_probe(void* stream_key, const void* image_lo, const void* image_hi,
+                             const void* filter_lo, const void* filter_hi, const void* out_lo,
+                             const void* out_hi, int overlap, double sms_by_memory,
+                             double sms_by_threads, int sm_count) {
+  if (overlap < 0 || overlap > 2 || sm_count <= 0) return CCONV_EINVAL;
+  CallSpans c;
+  c.image = Span{static_cast<const char*>(image_lo), static_cast<const char*>(image_hi)};
+  c.filter = Span{static_cast<const char*>(filter_lo), static_cast<const char*>(filter_hi)};
+  c.out = Span{static_cast<const char*>(out_lo), static_cast<const char*>(out_hi)};
+  c.sms = sms_by_memory;
+  c.sms_by_threads = sms_by_threads;
+  const Overlap how = overlap == 0 ? Overlap::kNone : overlap == 1 ? Overlap::kInputsEarly : Overlap::kDeep;
+  return note_call_hazards(stream_key, c, how, sm_count);
+}
+
 int cconv_plan_status(const cconv_plan* pl, void* cuda_stream, int* detail_out) {
   if (!pl || pl->device < 0 || !pl->d_status) return CCONV_EINVAL;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
