@@ -332,7 +332,8 @@ int cconv_plan_status(const cconv_plan* plan, void* cuda_stream, int* detail_out
  * kernel stamps %globaltimer (ns) at fixed points of each CTA's roles into a [grid][16] table:
  * 0 entry, 1 set-up done, 2 first Image copy issued, 3 Image producer done, 4 Filter producer done,
  * 5 first MMA issued, 6 first tile's MMAs issued, 7 all MMAs issued, 8 first accumulator ready,
- * 9 first tile stored, 10 all tiles stored, 11 exit.  Synchronous copy to host_out (at most
+ * 9 first tile stored, 10 all tiles stored, 11 exit (the DIRECT kernel stamps the same points, and
+ * puts the SM's id in slot 12 and the cycles of its first tile's main loop in slot 15).  Synchronous copy to host_out (at most
  * max_u64 values); returns the number of values copied, 0 when tracing is off, or a negative code. */
 int cconv_plan_trace_read(const cconv_plan* plan, unsigned long long* host_out, int max_u64);
 
