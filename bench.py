@@ -238,6 +238,23 @@ def time_repeats(cfg, torch, binding, dev, launches, repeats=5):
         torch.cuda.synchronize()
         alone.append(e0.elapsed_time(e1) * 1e-3)
     res["alone"] = float(np.median(alone))
+    res["alone_latency_plan"] = None
+    if plan.info()["variant"] == binding.VARIANT_DIRECT:
+        # the same call on a plan made for one call at a time (what CCONV_OBJECTIVE=latency selects)
+        lat_plan = binding.Plan(*cfg.dims(), device=dev.index, variant=binding.VARIANT_HALO,
+                                out_dtype=binding.OUT_BF16)
+        alone = []
+        for i in range(8):
+            a, b, c = ptrs[i % nsets]
+            torch.cuda.synchronize()
+            e0.record(stream)
+            lat_plan.forward_ptrs(a, b, c, sp)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            alone.append(e0.elapsed_time(e1) * 1e-3)
+        res["alone_latency_plan"] = float(np.median(alone[1:]))
+        lat_plan.check()
+        lat_plan.close()
     try:
         side = torch.cuda.Stream()
         side.wait_stream(stream)
@@ -726,6 +743,8 @@ def main():
                     "us": round(cold * 1e6, 2),
                     "us_graph": None if res["graph"] is None else round(res["graph"] * 1e6, 2),
                     "us_alone": round(res["alone"] * 1e6, 1),
+                    "us_alone_latency_plan": (None if res["alone_latency_plan"] is None
+                                              else round(res["alone_latency_plan"] * 1e6, 1)),
                     "tflops": round(c.flops / cold / 1e12, 1), "t_roof_us": round(tr * 1e6, 2),
                     "frac": round(tr / cold, 3), "bound": bound, "kernel": KERNEL_NAMES[info_i["variant"]],
                     "dram_bytes_ncu": dram_traffic_from_profiles(c.name),
@@ -740,7 +759,8 @@ def main():
             roof["per_config_note"] = ("us = L2-cold back-to-back calls on one stream, median of 5 regions of "
                                        "about 4 ms (20 to 1000 calls); independent calls of small shapes "
                                        "run side by side on the SMs; us_alone = one call between "
-                                       "synchronisations, launch included; frac = t_roof_us / us")
+                                       "synchronisations, launch included (us_alone_latency_plan: on a plan "
+                                       "made with CCONV_OBJECTIVE=latency); frac = t_roof_us / us")
             pool = time_pooling(torch, binding, dev, peaks)
             roof["pooling"] = {f"{r['workload']}_{r['op']}": {"us": round(r["us_per_launch"], 2),
                                                                "frac_of_hbm_copy": round(r["roofline"]["frac"], 3)}
